@@ -231,7 +231,8 @@ def test_matches_grid_sample_softmax_autograd(window, sigma):
     assert float(doff.abs().max()) > 1e-3          # the comparison is not vacuous
 
 
-def test_grid_sample_on_exact_lattice_and_boundary_positions():
+@pytest.mark.parametrize("dtype", [F64, torch.float32])
+def test_grid_sample_on_exact_lattice_and_boundary_positions(dtype):
     """Sizes with size-1 a power of two make the normalisation exact, so positions exactly
     on integers, at -1 and at size agree with grid_sample including its one-sided
     derivative convention at the kinks."""
@@ -242,7 +243,9 @@ def test_grid_sample_on_exact_lattice_and_boundary_positions():
                        for s in (T, H, W)], -1)                     # multiples of 1/8 in [-1, size]
     coords = torch.tensor(tokens(T, H, W), dtype=F64).view(T, H, W, 1, 1, 3)
     off = pos - coords
+    q, k, v, off, dout = (z.to(dtype) for z in (q, k, v, off, dout))    # all exactly representable
     out, lse, dq, dk, dv, doff = run_oracle(q, k, v, off, window, dout)
+    q, k, v, off, dout = (z.to(F64) for z in (q, k, v, off, dout))
     tk, tv, toff = (z.clone().requires_grad_(True) for z in (k, v, off))
     ref_out, ref_lse = torch_grid_sample_dsa(q, tk, tv, toff, window)
     (ref_out * dout).sum().backward()
