@@ -1,0 +1,103 @@
+/*
+ * dsa3d.h - C ABI of the B200 (sm_100a) 3D Deformable Slide Attention library.
+ *
+ * The operator (paper, section "3D Deformable Slide Attention": Formulation, Eq. 1 second
+ * term, and the softmax definition below Eq. 1; sampling as in "Implementation
+ * considerations"):
+ *
+ *   Query token n = (t, y, x) on a (T, H, W) grid, head m, window (kt, kh, kw) with
+ *   P = kt*kh*kw cells; cell p = (u*kh + v)*kw + w has the integer displacement
+ *   b(p) = (u - kt/2, v - kh/2, w - kw/2) (integer division: a window of 2 covers {-1, 0},
+ *   of 3 covers {-1, 0, 1}).  The sample position is
+ *       pi = (t, y, x) + b(p) + offsets[n, m, p, :]            in grid-index units,
+ *   formed in fp32 as float(coord + b) + offset.  K and V are sampled there by trilinear
+ *   interpolation with zero padding: a corner outside the grid contributes nothing and
+ *   the other corner weights are not renormalised.  Then
+ *       s_p = q[n, m, :] . k_p / sqrt(d),  alpha = softmax over the P samples,
+ *       out[n, m, :] = sum_p alpha_p v_p,  lse[n, m] = ln sum_p exp(s_p).
+ *   A sample with no corner inside the grid (or a NaN/inf position) has k_p = v_p = 0 and
+ *   s_p = 0; it still takes part in the softmax.  With all offsets zero the operator is
+ *   fixed 3D sliding-window attention (paper, Ablations, "Effect of offsets").
+ *   The depthwise-convolution term of Eq. 1, the projections and the offset predictor are
+ *   not part of this library.  There is no causal mask.
+ *
+ * Layouts (row-major, channels last, one video per call; a batch is one call per item):
+ *   q, k, v, out, dout, dq, dk, dv : [T, H, W, heads, d]     element type = `dtype`
+ *   offsets, doffsets              : [T, H, W, heads, P, 3]  fp32, last axis (t, y, x)
+ *   lse                            : [T, H, W, heads]        fp32
+ *
+ * Pointers.  Unless a parameter says HOST, every pointer is a DEVICE pointer owned by the
+ * caller, contiguous and 16-byte aligned.  The library does not allocate, free or keep
+ * them.  Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is the
+ * default stream); the buffers must stay valid until the stream has run the work.
+ * Outputs are fully overwritten.  Inputs and outputs must not alias.
+ *
+ * Supported: dtype DSA3D_F32 or DSA3D_BF16; d in {32, 64, 128}; 1 <= P <= 256;
+ * T, H, W, heads >= 1; T*H*W < 2^31.  Arithmetic is fp32 whatever the storage type.
+ *
+ * Errors.  Every function returns a dsa3d_status (0 = success).  Arguments are checked
+ * before anything is launched; nothing aborts, throws or traps.
+ */
+#ifndef DSA3D_H
+#define DSA3D_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DSA3D_OK = 0,
+    DSA3D_ERR_NULL_POINTER = 1,   /* a required pointer is NULL */
+    DSA3D_ERR_BAD_SHAPE = 2,      /* a size is < 1 or the grid has 2^31 tokens or more */
+    DSA3D_ERR_UNSUPPORTED = 3,    /* dtype, head dimension or window outside the supported set */
+    DSA3D_ERR_MISALIGNED = 4,     /* a pointer is not 16-byte aligned */
+    DSA3D_ERR_WORKSPACE = 5,      /* workspace missing or smaller than required */
+    DSA3D_ERR_CUDA = 6            /* a CUDA runtime call failed; see dsa3d_last_cuda_error */
+} dsa3d_status;
+
+typedef enum { DSA3D_F32 = 0, DSA3D_BF16 = 1 } dsa3d_dtype;
+
+/*
+ * Forward (Eq. 1 second term + softmax definition).  Reads q, k, v, offsets; writes out
+ * and lse.  `window` is a HOST pointer to (kt, kh, kw).  No workspace.
+ */
+int dsa3d_forward(const void* q, const void* k, const void* v, const float* offsets,
+                  int T, int H, int W, int heads, int d, const int window[3],
+                  void* out, float* lse, int dtype, void* stream);
+
+/*
+ * Backward of the forward above (chain rule through sampling, softmax and weighted sum;
+ * the paper trains through this operator by automatic differentiation and prints no
+ * formulas).  Given dout = dLoss/dout and the lse saved by the forward, writes
+ *   dq, dk, dv   same shape and type as q, k, v
+ *   doffsets     same shape as offsets; the derivative of the trilinear weights, with the
+ *                one-sided convention of the floor at integer positions (cell [i, i+1))
+ * The sampling weights are recomputed, nothing of size N*P*d is stored.
+ * `workspace` is device scratch of at least dsa3d_backward_workspace_bytes(...) bytes,
+ * 16-byte aligned (fp32 accumulators for dk and dv; may be NULL when that size is 0).
+ * Its contents on entry do not matter.  dk and dv are summed with floating-point atomics,
+ * so their last bits can differ from run to run; dq, doffsets are deterministic.
+ */
+int dsa3d_backward(const void* q, const void* k, const void* v, const float* offsets,
+                   const float* lse, const void* dout,
+                   int T, int H, int W, int heads, int d, const int window[3],
+                   void* dq, void* dk, void* dv, float* doffsets,
+                   void* workspace, size_t workspace_bytes, int dtype, void* stream);
+
+/* Scratch bytes dsa3d_backward needs for this problem (0 for DSA3D_F32; 0 also for
+ * arguments the library would reject). */
+size_t dsa3d_backward_workspace_bytes(int T, int H, int W, int heads, int d,
+                                      const int window[3], int dtype);
+
+/* Static, NUL-terminated description of a status code. */
+const char* dsa3d_status_string(int status);
+
+/* cudaError_t of the most recent DSA3D_ERR_CUDA on the calling thread (0 if none). */
+int dsa3d_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DSA3D_H */

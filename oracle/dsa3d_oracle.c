@@ -253,7 +253,13 @@ int dsa3d_oracle_forward(const void *q_rows, const void *k, const void *v, const
 /* dq_rows [nq, heads, d], doff_rows [nq, heads, P, 3], fully overwritten.
  * dk_rows, dv_rows [nk, heads, d] are ACCUMULATED INTO (the caller zeroes them).
  * kslot: NULL means slot = token index (nk = T*H*W); otherwise kslot[token] is the output
- * row of that key token, or -1 if its gradient is not wanted. */
+ * row of that key token, or -1 if its gradient is not wanted.
+ *
+ * Two phases.  Phase A visits every (query row, head) independently and produces dQ,
+ * dOffsets and the two per-sample scatter coefficients  ck_p = dS_p / sqrt(d)  and
+ * cv_p = alpha_p.  Phase B adds  w_c ck_p q  into dK and  w_c cv_p dO  into dV; it is
+ * split over (head, channel range) so that every dK/dV element belongs to one thread and
+ * is summed in query-row order whatever the thread count. */
 int dsa3d_oracle_backward(const void *q_rows, const void *k, const void *v, const void *off_rows,
                           const void *dout_rows, const int64_t *qtok, int64_t nq, int T, int H,
                           int W, int heads, int d, const int *window, int dtype,
@@ -263,15 +269,16 @@ int dsa3d_oracle_backward(const void *q_rows, const void *k, const void *v, cons
     const int size[3] = {T, H, W};
     const int P = window[0] * window[1] * window[2];
     const double scale = 1.0 / sqrt((double)d);
+    const int off_is_f64 = (dtype == ORC_F64);
+    const size_t off_elt = off_is_f64 ? sizeof(double) : sizeof(float);
     int failed = 0;
-    int used = dsa3d_oracle_max_threads();
-    if (used > heads) used = heads;
-    g_last_threads = used;
-    /* One head per thread at a time: every output of a head (its dK/dV channels included)
-     * belongs to exactly one thread, and queries are visited in row order, so the
-     * summation order is fixed. */
-#pragma omp parallel for schedule(dynamic, 1)
-    for (int m = 0; m < heads; ++m) {
+    g_last_threads = dsa3d_oracle_max_threads();
+    double *coef = (double *)malloc(sizeof(double) * 2 * (size_t)nq * heads * P + 16);
+    if (!coef) return 2;
+
+    /* ---- phase A: dQ, dOffsets, scatter coefficients ---- */
+#pragma omp parallel
+    {
         sample_geom *geom = (sample_geom *)malloc(sizeof(sample_geom) * P);
         double *kp = (double *)malloc(sizeof(double) * P * d);
         double *vp = (double *)malloc(sizeof(double) * P * d);
@@ -283,56 +290,52 @@ int dsa3d_oracle_backward(const void *q_rows, const void *k, const void *v, cons
         } else {
             double *alpha = s + P, *g = s + 2 * P, *dS = s + 3 * P;
             double *dov = qv + d;
+#pragma omp for collapse(2) schedule(dynamic, 16)
             for (int64_t i = 0; i < nq; ++i) {
-                const int64_t n = qtok ? qtok[i] : i;
-                forward_one(q_rows, k, v, off_rows, i, n, m, size, heads, d, window, P, dtype, geom,
-                            kp, vp, s, alpha);
-                const int64_t qbase = (i * heads + m) * (int64_t)d;
-                for (int j = 0; j < d; ++j) {
-                    qv[j] = load_elt(q_rows, dtype, qbase + j);
-                    dov[j] = load_elt(dout_rows, dtype, qbase + j);
-                }
-                double delta = 0.0;
-                for (int p = 0; p < P; ++p) {
-                    double acc = 0.0;
-                    for (int j = 0; j < d; ++j) acc += dov[j] * vp[(size_t)p * d + j];
-                    g[p] = acc;
-                    delta += alpha[p] * acc;
-                }
-                for (int p = 0; p < P; ++p) dS[p] = alpha[p] * (g[p] - delta);
-                double *dq = dq_rows + qbase;
-                for (int j = 0; j < d; ++j) dq[j] = 0.0;
-                for (int p = 0; p < P; ++p)
-                    for (int j = 0; j < d; ++j) dq[j] += scale * dS[p] * kp[(size_t)p * d + j];
-                for (int p = 0; p < P; ++p) {
-                    double *doff = doff_rows + ((i * heads + m) * (int64_t)P + p) * 3;
-                    doff[0] = doff[1] = doff[2] = 0.0;
-                    for (int c = 0; c < 8; ++c) {
-                        if (!geom[p].valid[c]) continue;
-                        const int cc[3] = {(c >> 2) & 1, (c >> 1) & 1, c & 1};
-                        const int64_t kbase = (geom[p].tok[c] * heads + m) * (int64_t)d;
-                        double qk = 0.0, dov_v = 0.0;
-                        for (int j = 0; j < d; ++j) {
-                            qk += qv[j] * load_elt(k, dtype, kbase + j);
-                            dov_v += dov[j] * load_elt(v, dtype, kbase + j);
+                for (int m = 0; m < heads; ++m) {
+                    const int64_t n = qtok ? qtok[i] : i;
+                    forward_one(q_rows, k, v, off_rows, i, n, m, size, heads, d, window, P, dtype,
+                                geom, kp, vp, s, alpha);
+                    const int64_t qbase = (i * heads + m) * (int64_t)d;
+                    for (int j = 0; j < d; ++j) {
+                        qv[j] = load_elt(q_rows, dtype, qbase + j);
+                        dov[j] = load_elt(dout_rows, dtype, qbase + j);
+                    }
+                    double delta = 0.0;
+                    for (int p = 0; p < P; ++p) {
+                        double acc = 0.0;
+                        for (int j = 0; j < d; ++j) acc += dov[j] * vp[(size_t)p * d + j];
+                        g[p] = acc;
+                        delta += alpha[p] * acc;
+                    }
+                    for (int p = 0; p < P; ++p) dS[p] = alpha[p] * (g[p] - delta);
+                    double *dq = dq_rows + qbase;
+                    for (int j = 0; j < d; ++j) dq[j] = 0.0;
+                    for (int p = 0; p < P; ++p)
+                        for (int j = 0; j < d; ++j) dq[j] += scale * dS[p] * kp[(size_t)p * d + j];
+                    for (int p = 0; p < P; ++p) {
+                        double *doff = doff_rows + ((i * heads + m) * (int64_t)P + p) * 3;
+                        doff[0] = doff[1] = doff[2] = 0.0;
+                        for (int c = 0; c < 8; ++c) {
+                            if (!geom[p].valid[c]) continue;
+                            const int cc[3] = {(c >> 2) & 1, (c >> 1) & 1, c & 1};
+                            const int64_t kbase = (geom[p].tok[c] * heads + m) * (int64_t)d;
+                            double qk = 0.0, dov_v = 0.0;
+                            for (int j = 0; j < d; ++j) {
+                                qk += qv[j] * load_elt(k, dtype, kbase + j);
+                                dov_v += dov[j] * load_elt(v, dtype, kbase + j);
+                            }
+                            const double Cc = scale * dS[p] * qk + alpha[p] * dov_v;
+                            for (int a = 0; a < 3; ++a) {
+                                double prod = cc[a] ? 1.0 : -1.0;
+                                for (int a2 = 0; a2 < 3; ++a2)
+                                    if (a2 != a) prod *= geom[p].wt[a2][cc[a2]];
+                                doff[a] += prod * Cc;
+                            }
                         }
-                        const double Cc = scale * dS[p] * qk + alpha[p] * dov_v;
-                        for (int a = 0; a < 3; ++a) {
-                            double prod = cc[a] ? 1.0 : -1.0;
-                            for (int a2 = 0; a2 < 3; ++a2)
-                                if (a2 != a) prod *= geom[p].wt[a2][cc[a2]];
-                            doff[a] += prod * Cc;
-                        }
-                        const int64_t slot = kslot ? kslot[geom[p].tok[c]] : geom[p].tok[c];
-                        if (slot < 0) continue;
-                        double *dk = dk_rows + (slot * heads + m) * (int64_t)d;
-                        double *dv = dv_rows + (slot * heads + m) * (int64_t)d;
-                        const double ck = geom[p].w[c] * scale * dS[p];
-                        const double cv = geom[p].w[c] * alpha[p];
-                        for (int j = 0; j < d; ++j) {
-                            dk[j] += ck * qv[j];
-                            dv[j] += cv * dov[j];
-                        }
+                        double *cf = coef + 2 * ((i * heads + m) * (int64_t)P + p);
+                        cf[0] = scale * dS[p];
+                        cf[1] = alpha[p];
                     }
                 }
             }
@@ -343,5 +346,50 @@ int dsa3d_oracle_backward(const void *q_rows, const void *k, const void *v, cons
         free(s);
         free(qv);
     }
+
+    /* ---- phase B: dK, dV ---- */
+    if (!failed) {
+        int nchunk = (g_last_threads + heads - 1) / heads;
+        if (nchunk > d) nchunk = d;
+        if (nchunk < 1) nchunk = 1;
+        const int cw = (d + nchunk - 1) / nchunk;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+        for (int m = 0; m < heads; ++m) {
+            for (int ch = 0; ch < nchunk; ++ch) {
+                const int j0 = ch * cw, j1 = (j0 + cw < d) ? j0 + cw : d;
+                sample_geom geom;
+                for (int64_t i = 0; i < nq; ++i) {
+                    const int64_t n = qtok ? qtok[i] : i;
+                    int coord[3];
+                    coord[2] = (int)(n % W);
+                    coord[1] = (int)((n / W) % H);
+                    coord[0] = (int)(n / ((int64_t)W * H));
+                    const int64_t qbase = (i * heads + m) * (int64_t)d;
+                    for (int p = 0; p < P; ++p) {
+                        int b[3];
+                        window_displacement(p, window, b);
+                        const char *off = (const char *)off_rows +
+                                          (size_t)(((i * heads + m) * P + p) * 3) * off_elt;
+                        sample_geometry(coord, b, off, off_is_f64, size, &geom);
+                        const double *cf = coef + 2 * ((i * heads + m) * (int64_t)P + p);
+                        for (int c = 0; c < 8; ++c) {
+                            if (!geom.valid[c]) continue;
+                            const int64_t slot = kslot ? kslot[geom.tok[c]] : geom.tok[c];
+                            if (slot < 0) continue;
+                            double *dk = dk_rows + (slot * heads + m) * (int64_t)d;
+                            double *dv = dv_rows + (slot * heads + m) * (int64_t)d;
+                            const double ck = geom.w[c] * cf[0];
+                            const double cv = geom.w[c] * cf[1];
+                            for (int j = j0; j < j1; ++j) {
+                                dk[j] += ck * load_elt(q_rows, dtype, qbase + j);
+                                dv[j] += cv * load_elt(dout_rows, dtype, qbase + j);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+    free(coef);
     return failed ? 2 : 0;
 }

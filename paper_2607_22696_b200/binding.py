@@ -1,0 +1,140 @@
+"""Thin ctypes binding of libdsa3d.so: same names and argument order as include/dsa3d.h.
+
+Only argument marshalling happens here (tensor -> device pointer, window -> int[3],
+status -> exception).  Every step of the operator runs in the library's CUDA kernels; there
+is no fallback: if the shared library is missing or a tensor is not on a CUDA device the
+call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdsa3d.so")
+
+DSA3D_F32, DSA3D_BF16 = 0, 1
+_DTYPES = {torch.float32: DSA3D_F32, torch.bfloat16: DSA3D_BF16}
+
+_lib = None
+
+
+class Dsa3dError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"dsa3d status {status}: {message}")
+        self.status = status
+
+
+def load():
+    """Load libdsa3d.so (built by paper_2607_22696_b200.build) and declare its prototypes."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2607_22696_b200.build`; "
+            "there is no CPU or PyTorch fallback for this operator")
+    lib = ctypes.CDLL(LIB_PATH)
+    p, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    win = ctypes.POINTER(ctypes.c_int)
+    lib.dsa3d_forward.restype = i
+    lib.dsa3d_forward.argtypes = [p, p, p, p, i, i, i, i, i, win, p, p, i, p]
+    lib.dsa3d_backward.restype = i
+    lib.dsa3d_backward.argtypes = [p, p, p, p, p, p, i, i, i, i, i, win, p, p, p, p, p, sz, i, p]
+    lib.dsa3d_backward_workspace_bytes.restype = sz
+    lib.dsa3d_backward_workspace_bytes.argtypes = [i, i, i, i, i, win, i]
+    lib.dsa3d_status_string.restype = ctypes.c_char_p
+    lib.dsa3d_status_string.argtypes = [i]
+    lib.dsa3d_last_cuda_error.restype = i
+    lib.dsa3d_last_cuda_error.argtypes = []
+    _lib = lib
+    return lib
+
+
+def _window(window: Sequence[int]):
+    if len(window) != 3:
+        raise ValueError("window must be (kt, kh, kw)")
+    return (ctypes.c_int * 3)(int(window[0]), int(window[1]), int(window[2]))
+
+
+def _ptr(t: Optional[torch.Tensor], name: str, numel: Optional[int] = None, dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    if not isinstance(t, torch.Tensor):
+        return int(t)                        # a raw device address
+    if t.device.type != "cuda":
+        raise ValueError(f"{name} must be a CUDA tensor (the library takes device pointers)")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"{name} must be {dtype}, got {t.dtype}")
+    if numel is not None and t.numel() != numel:
+        raise ValueError(f"{name} has {t.numel()} elements, expected {numel}")
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream or None
+    if isinstance(stream, torch.cuda.Stream):
+        return stream.cuda_stream or None
+    return int(stream) or None
+
+
+def _check(status: int) -> None:
+    if status != 0:
+        lib = load()
+        msg = lib.dsa3d_status_string(status).decode()
+        if status == 6:
+            msg += f" (cudaError {lib.dsa3d_last_cuda_error()})"
+        raise Dsa3dError(status, msg)
+
+
+def dsa3d_status_string(status: int) -> str:
+    return load().dsa3d_status_string(int(status)).decode()
+
+
+def dsa3d_last_cuda_error() -> int:
+    return int(load().dsa3d_last_cuda_error())
+
+
+def dsa3d_backward_workspace_bytes(T, H, W, heads, d, window, dtype) -> int:
+    code = _DTYPES[dtype] if isinstance(dtype, torch.dtype) else int(dtype)
+    return int(load().dsa3d_backward_workspace_bytes(T, H, W, heads, d, _window(window), code))
+
+
+def dsa3d_forward(q, k, v, offsets, T, H, W, heads, d, window, out, lse, dtype=None, stream=None) -> None:
+    """out, lse <- 3D-DSA forward of (q, k, v, offsets); see include/dsa3d.h.  `dtype`
+    defaults to q's dtype; `stream` to torch's current stream."""
+    lib = load()
+    dt = q.dtype if dtype is None else dtype
+    code = _DTYPES[dt] if isinstance(dt, torch.dtype) else int(dt)
+    n = T * H * W * heads
+    P = int(window[0]) * int(window[1]) * int(window[2])
+    _check(lib.dsa3d_forward(
+        _ptr(q, "q", n * d), _ptr(k, "k", n * d), _ptr(v, "v", n * d),
+        _ptr(offsets, "offsets", n * P * 3, torch.float32), T, H, W, heads, d, _window(window),
+        _ptr(out, "out", n * d), _ptr(lse, "lse", n, torch.float32), code, _stream(stream)))
+
+
+def dsa3d_backward(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets,
+                   workspace=None, workspace_bytes=None, dtype=None, stream=None) -> None:
+    """dq, dk, dv, doffsets <- 3D-DSA backward; see include/dsa3d.h.  `workspace` is a CUDA
+    tensor (any dtype) of at least dsa3d_backward_workspace_bytes(...) bytes."""
+    lib = load()
+    dt = q.dtype if dtype is None else dtype
+    code = _DTYPES[dt] if isinstance(dt, torch.dtype) else int(dt)
+    n = T * H * W * heads
+    P = int(window[0]) * int(window[1]) * int(window[2])
+    if workspace_bytes is None:
+        workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.dsa3d_backward(
+        _ptr(q, "q", n * d), _ptr(k, "k", n * d), _ptr(v, "v", n * d),
+        _ptr(offsets, "offsets", n * P * 3, torch.float32), _ptr(lse, "lse", n, torch.float32),
+        _ptr(dout, "dout", n * d), T, H, W, heads, d, _window(window),
+        _ptr(dq, "dq", n * d), _ptr(dk, "dk", n * d), _ptr(dv, "dv", n * d),
+        _ptr(doffsets, "doffsets", n * P * 3, torch.float32),
+        _ptr(workspace, "workspace"), int(workspace_bytes), code, _stream(stream)))

@@ -1,0 +1,127 @@
+// Forward of 3D Deformable Slide Attention (Eq. 1 second term and the softmax under it).
+//
+// One group of LPR = d / VEC lanes owns one (token, head) item; each lane holds VEC
+// consecutive channels (16 bytes) of every row it touches.  Work items are ordered
+// head-major (item = head * N + token) so that the CTAs in flight at any time gather from
+// one head's K/V over a few neighbouring frames, which is what keeps the corner gathers in
+// L2.  Per sample: the 8 corner rows of K and of V are loaded with 16-byte loads, the
+// logit is the weighted sum of the corner dot products, and the output is accumulated with
+// an online softmax in fp32 registers; nothing of size N*P is written.
+#include "dsa3d_common.cuh"
+#include "dsa3d_kernels.h"
+
+namespace dsa3d {
+
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+               const float* __restrict__ offsets, T* __restrict__ out, float* __restrict__ lse,
+               const Problem pr) {
+    constexpr int VEC = Elt<T>::VEC;
+    constexpr int LPR = D / VEC;
+    const int lane = threadIdx.x & 31;
+    const int gl = lane & (LPR - 1);
+    const unsigned gmask = group_mask<LPR>(lane);
+    const long long item = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) / LPR;
+    if (item >= pr.items) return;
+
+    const int m = static_cast<int>(item / pr.N);
+    const long long n = item - static_cast<long long>(m) * pr.N;
+    const int x = static_cast<int>(n % pr.W);
+    const int y = static_cast<int>((n / pr.W) % pr.H);
+    const int t = static_cast<int>(n / (static_cast<long long>(pr.W) * pr.H));
+    const int HW = pr.H * pr.W;
+    const long long row = (n * pr.heads + m);               // row index into [N*heads, ...]
+    const int ch = gl * VEC;
+
+    float qf[VEC];
+    Elt<T>::load(q + row * D + ch, qf);
+    const float qscale = rsqrtf(static_cast<float>(D)) * kLog2e;   // logits in log2 units
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) qf[j] *= qscale;
+
+    const float* off_row = offsets + row * pr.P * 3;
+    const T* kh = k + static_cast<long long>(m) * D + ch;    // + tok * heads * D
+    const T* vh = v + static_cast<long long>(m) * D + ch;
+    const long long tok_stride = static_cast<long long>(pr.heads) * D;
+
+    float acc[VEC];
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) acc[j] = 0.0f;
+    float m_run = -INFINITY, l_run = 0.0f;
+
+    for (int pb = 0; pb < pr.P; pb += LPR) {
+        Sample mine;
+        mine.base = 0; mine.mask = 0u; mine.ft = mine.fy = mine.fx = 0.0f;
+        if (pb + gl < pr.P) mine = make_sample(pr, t, y, x, pb + gl, off_row + (pb + gl) * 3);
+        const int cnt = min(LPR, pr.P - pb);
+        for (int j = 0; j < cnt; ++j) {
+            const Sample s = group_bcast<LPR>(mine, j, gmask);
+            const float wt[2] = {1.0f - s.ft, s.ft}, wy[2] = {1.0f - s.fy, s.fy}, wx[2] = {1.0f - s.fx, s.fx};
+            float sdot = 0.0f;
+            float vp[VEC];
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) vp[e] = 0.0f;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const float w = wt[c >> 2] * wy[(c >> 1) & 1] * wx[c & 1];
+                if (((s.mask >> c) & 1u) && w != 0.0f) {
+                    const int tok = s.base + (c >> 2) * HW + ((c >> 1) & 1) * pr.W + (c & 1);
+                    float kk[VEC], vv[VEC];
+                    Elt<T>::load(kh + tok * tok_stride, kk);
+                    Elt<T>::load(vh + tok * tok_stride, vv);
+                    float dot = 0.0f;
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) {
+                        dot = fmaf(qf[e], kk[e], dot);
+                        vp[e] = fmaf(w, vv[e], vp[e]);
+                    }
+                    sdot = fmaf(w, dot, sdot);
+                }
+            }
+            const float sp = group_sum<LPR>(sdot, gmask);
+            const float m_new = fmaxf(m_run, sp);
+            const float corr = exp2f(m_run - m_new);
+            const float pe = exp2f(sp - m_new);
+            l_run = fmaf(l_run, corr, pe);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) acc[e] = fmaf(pe, vp[e], acc[e] * corr);
+            m_run = m_new;
+        }
+    }
+    const float inv = 1.0f / l_run;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) acc[e] *= inv;
+    Elt<T>::store(out + row * D + ch, acc);
+    if (gl == 0) lse[row] = (m_run + log2f(l_run)) * kLn2;
+}
+
+template <typename T, int D>
+static cudaError_t launch_forward_t(const void* q, const void* k, const void* v, const float* offsets,
+                                    void* out, float* lse, const Problem& pr, cudaStream_t stream) {
+    constexpr int LPR = D / Elt<T>::VEC;
+    constexpr int threads = 256;
+    const long long groups_per_block = threads / LPR;
+    const long long blocks = (pr.items + groups_per_block - 1) / groups_per_block;
+    forward_kernel<T, D><<<static_cast<unsigned>(blocks), threads, 0, stream>>>(
+        static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), offsets,
+        static_cast<T*>(out), lse, pr);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_forward(const void* q, const void* k, const void* v, const float* offsets, void* out,
+                           float* lse, const Problem& pr, bool bf16, cudaStream_t stream) {
+#define DSA3D_CASE(DD)                                                                              \
+    case DD:                                                                                        \
+        return bf16 ? launch_forward_t<__nv_bfloat16, DD>(q, k, v, offsets, out, lse, pr, stream)   \
+                    : launch_forward_t<float, DD>(q, k, v, offsets, out, lse, pr, stream);
+    switch (pr.d) {
+        DSA3D_CASE(32)
+        DSA3D_CASE(64)
+        DSA3D_CASE(128)
+    }
+#undef DSA3D_CASE
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace dsa3d

@@ -1,0 +1,105 @@
+"""Host-side checks of the C ABI: the library loads, exports every symbol the header
+declares, and rejects bad arguments with the documented status before launching."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2607_22696_b200 import build, binding
+    build.build()
+    return binding.load()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "dsa3d.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(dsa3d_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_declares_the_expected_entry_points():
+    syms = declared_symbols()
+    for name in ["dsa3d_forward", "dsa3d_backward", "dsa3d_backward_workspace_bytes",
+                 "dsa3d_status_string", "dsa3d_last_cuda_error"]:
+        assert name in syms
+
+
+def test_library_exports_every_declared_symbol(lib):
+    for name in declared_symbols():
+        assert hasattr(lib, name), name
+
+
+def test_status_strings(lib):
+    assert lib.dsa3d_status_string(0) == b"success"
+    for code in range(1, 7):
+        s = lib.dsa3d_status_string(code)
+        assert s and s != b"unknown status"
+    assert lib.dsa3d_status_string(99) == b"unknown status"
+
+
+def test_workspace_size(lib):
+    win = (ctypes.c_int * 3)(3, 3, 3)
+    assert lib.dsa3d_backward_workspace_bytes(4, 8, 8, 2, 32, win, 0) == 0
+    assert lib.dsa3d_backward_workspace_bytes(4, 8, 8, 2, 32, win, 1) == 256 * 2 * 32 * 4 * 2
+    assert lib.dsa3d_backward_workspace_bytes(256, 68, 120, 16, 128, win, 1) == 2088960 * 16 * 128 * 4 * 2
+    assert lib.dsa3d_backward_workspace_bytes(4, 8, 8, 2, 48, win, 1) == 0      # rejected shape
+
+
+def test_forward_rejects_bad_arguments_without_launching(lib):
+    win = (ctypes.c_int * 3)(3, 3, 3)
+    a = 4096                                     # fake, aligned, never dereferenced
+    ok = [a, a, a, a, 4, 8, 8, 2, 32, win, a, a, 0, None]
+
+    def call(**kw):
+        args = list(ok)
+        for idx, val in kw.items():
+            args[int(idx[1:])] = val
+        return lib.dsa3d_forward(*args)
+
+    assert call(_0=None) == 1
+    assert call(_10=None) == 1
+    assert call(_9=None) == 1
+    assert call(_4=0) == 2
+    assert call(_7=-1) == 2
+    assert call(_9=(ctypes.c_int * 3)(3, 0, 3)) == 2
+    assert call(_4=1 << 15, _5=1 << 15, _6=4) == 2           # 2^32 tokens
+    assert call(_8=48) == 3
+    assert call(_12=7) == 3
+    assert call(_9=(ctypes.c_int * 3)(7, 7, 7)) == 3         # P = 343 > 256
+    assert call(_1=a + 8) == 4
+    assert call(_11=a + 4) == 4
+
+
+def test_backward_rejects_bad_arguments_without_launching(lib):
+    win = (ctypes.c_int * 3)(3, 3, 3)
+    a = 4096
+    ok = [a, a, a, a, a, a, 4, 8, 8, 2, 32, win, a, a, a, a, a, 1 << 30, 1, None]
+
+    def call(**kw):
+        args = list(ok)
+        for idx, val in kw.items():
+            args[int(idx[1:])] = val
+        return lib.dsa3d_backward(*args)
+
+    assert call(_5=None) == 1
+    assert call(_15=None) == 1
+    assert call(_10=100) == 3
+    assert call(_16=None) == 5
+    assert call(_17=1024) == 5
+    assert call(_16=a + 4) == 4
+    assert call(_13=a + 2) == 4
+
+
+def test_binding_refuses_cpu_tensors():
+    import torch
+    from paper_2607_22696_b200 import binding
+    z = torch.zeros(4 * 8 * 8 * 2 * 32)
+    off = torch.zeros(4 * 8 * 8 * 2 * 27 * 3)
+    lse = torch.zeros(4 * 8 * 8 * 2)
+    with pytest.raises(ValueError, match="CUDA tensor"):
+        binding.dsa3d_forward(z, z, z, off, 4, 8, 8, 2, 32, (3, 3, 3), z, lse, stream=0)

@@ -1,0 +1,150 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the
+same seeded inputs.  Small problems are compared element by element over every output;
+the 720p-class, 1080p and sweep workloads are compared on sampled queries and key rows
+plus whole-tensor invariants (see parity_util).  Tolerances are stated in parity_util."""
+import math
+
+import pytest
+import torch
+
+import parity_util as pu
+from paper_2607_22696_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+BF16, F32 = torch.bfloat16, torch.float32
+
+
+def small_problem(T, H, W, heads, d, window, dtype, sigma, seed):
+    wl = inputs.Workload("case", T, H, W, heads, d, tuple(window), dtype, sigma, seed)
+    t = inputs.make_inputs(wl, "cpu", with_dout=True)
+    return t["q"], t["k"], t["v"], t["offsets"], t["dout"]
+
+
+def test_extension_is_loaded():
+    lib = binding.load()
+    assert lib.dsa3d_status_string(0) == b"success"
+
+
+# ----------------------------------------------------------------- BASELINE configs 1, 2
+
+def test_config_tiny_f32_forward_backward():
+    wl = inputs.WORKLOADS["tiny_f32"]
+    t = inputs.make_inputs(wl, "cpu")
+    pu.full_parity(t["q"], t["k"], t["v"], t["offsets"], t["dout"], wl.window)
+
+
+def test_config_480p_bf16_forward_full():
+    wl = inputs.WORKLOADS["480p_bf16_fwd"]
+    t = inputs.make_inputs(wl, "cuda")
+    q, k, v, off = (t[n].cpu() for n in ("q", "k", "v", "offsets"))
+    pu.full_parity(q, k, v, off, None, wl.window, check_backward=False)
+
+
+# ------------------------------------------------------------- small cases, every output
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+@pytest.mark.parametrize("d", [32, 64, 128])
+def test_head_dims_and_ragged_item_counts(dtype, d):
+    # 5*7*9*3 = 945 items: not a multiple of any block's group count
+    pu.full_parity(*small_problem(5, 7, 9, 3, d, (3, 3, 3), dtype, 1.0, 20 + d), (3, 3, 3))
+
+
+@pytest.mark.parametrize("window", [(1, 1, 1), (2, 2, 2), (3, 5, 5), (3, 7, 7), (4, 8, 8)])
+def test_windows(window):
+    sigma = 1.5
+    pu.full_parity(*small_problem(4, 9, 10, 2, 64, window, BF16, sigma, 31), window)
+    pu.full_parity(*small_problem(3, 6, 7, 2, 32, window, F32, sigma, 32), window)
+
+
+@pytest.mark.parametrize("dims", [(1, 9, 11), (6, 1, 11), (6, 9, 1), (1, 1, 1), (1, 1, 40)])
+def test_grid_dimensions_of_one(dims):
+    pu.full_parity(*small_problem(*dims, 2, 32, (3, 3, 3), F32, 0.7, 33), (3, 3, 3))
+    pu.full_parity(*small_problem(*dims, 2, 128, (3, 3, 3), BF16, 0.7, 34), (3, 3, 3))
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_zero_and_integer_offsets(dtype):
+    q, k, v, off, dout = small_problem(5, 6, 7, 2, 64, (3, 3, 3), dtype, 1.0, 35)
+    pu.full_parity(q, k, v, torch.zeros_like(off), dout, (3, 3, 3))
+    ioff = inputs.uniform_int(off.shape, 36, 3, -3, 3, torch.float32)      # reaches -1 and size exactly
+    pu.full_parity(q, k, v, ioff, dout, (3, 3, 3))
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_out_of_range_nan_and_huge_offsets(dtype):
+    q, k, v, off, dout = small_problem(4, 5, 6, 2, 32, (3, 3, 3), dtype, 1.0, 37)
+    far = torch.full_like(off, 100.0)
+    pu.full_parity(q, k, v, far, dout, (3, 3, 3))                        # every sample dead
+    mixed = off.clone()
+    flat = mixed.view(-1, 3)
+    flat[0::7, 0] = float("nan")
+    flat[1::7, 1] = float("inf")
+    flat[2::7, 2] = -float("inf")
+    flat[3::7, 0] = 3e38
+    flat[4::7, 1] = -1e30
+    pu.full_parity(q, k, v, mixed, dout, (3, 3, 3))
+
+
+def test_positions_near_cell_boundaries_take_the_fp32_decision():
+    """Offsets a hair away from integers: the cell is decided by the fp32 position, the
+    same way on both sides, so even dOffsets agrees."""
+    q, k, v, off, dout = small_problem(3, 40, 60, 1, 32, (3, 3, 3), F32, 1.0, 38)
+    near = torch.round(off) + (inputs.normal(off.shape, 39, 3, 1.0, torch.float32) * 1e-6)
+    pu.full_parity(q, k, v, near, dout, (3, 3, 3))
+
+
+def test_per_query_outputs_are_run_to_run_deterministic():
+    q, k, v, off, dout = (z.cuda() for z in small_problem(6, 10, 12, 4, 128, (3, 3, 3), BF16, 1.5, 40))
+    dims = tuple(q.shape)
+    o1, l1 = pu.gpu_forward(q, k, v, off, dims, (3, 3, 3))
+    g1 = pu.gpu_backward(q, k, v, off, l1, dout, dims, (3, 3, 3))
+    o2, l2 = pu.gpu_forward(q, k, v, off, dims, (3, 3, 3))
+    g2 = pu.gpu_backward(q, k, v, off, l2, dout, dims, (3, 3, 3))
+    assert torch.equal(o1, o2) and torch.equal(l1, l2)
+    assert torch.equal(g1[0], g2[0]) and torch.equal(g1[3], g2[3])
+    for a, b in ((g1[1], g2[1]), (g1[2], g2[2])):        # atomics: order may differ
+        assert float((a.float() - b.float()).abs().max()) <= 2e-2 * float(a.float().abs().max())
+
+
+def test_binding_reports_library_errors():
+    z = torch.zeros(4 * 8 * 8 * 2 * 48, device="cuda")
+    off = torch.zeros(4 * 8 * 8 * 2 * 27 * 3, device="cuda")
+    lse = torch.zeros(4 * 8 * 8 * 2, device="cuda")
+    with pytest.raises(binding.Dsa3dError) as e:
+        binding.dsa3d_forward(z, z, z, off, 4, 8, 8, 2, 48, (3, 3, 3), z, lse)
+    assert e.value.status == 3
+
+
+# ------------------------------------------------- BASELINE configs 3, 4, 5 at full size
+
+def run_large(name, heads_sel, key_boxes, n_random=1024, backward=True):
+    wl = inputs.WORKLOADS[name]
+    dims = (wl.T, wl.H, wl.W, wl.heads, wl.d)
+    t = inputs.make_inputs(wl, "cuda")
+    out, lse = pu.gpu_forward(t["q"], t["k"], t["v"], t["offsets"], dims, wl.window)
+    t["out"] = out
+    grads = None
+    if backward:
+        grads = pu.gpu_backward(t["q"], t["k"], t["v"], t["offsets"], lse, t["dout"], dims, wl.window)
+        pu.assert_bilinearity_invariants(t, out, grads)
+    pu.sampled_parity(t, dims, wl.window, lse, grads, heads_sel, n_random=n_random, key_boxes=key_boxes)
+    del t, out, lse, grads
+    torch.cuda.empty_cache()
+
+
+def test_config_720p_bf16_forward_backward():
+    run_large("720p_bf16", [0, 11, 23], [((0, 0, 0), (2, 2, 2)), ((31, 22, 40), (32, 24, 42)),
+                                          ((63, 44, 78), (64, 45, 80))])
+
+
+def test_config_1080p_256f_bf16_forward_backward():
+    run_large("1080p_256f_bf16", [0, 7, 15], [((0, 0, 0), (2, 2, 2)), ((128, 33, 60), (129, 35, 62)),
+                                               ((255, 67, 118), (256, 68, 120))])
+
+
+@pytest.mark.parametrize("kind", ["zero", "int", "normal"])
+@pytest.mark.parametrize("window", ["222", "333", "355"])
+def test_config_sweep_720p_grid(window, kind):
+    boxes = [((0, 0, 0), (1, 2, 2)), ((32, 22, 40), (33, 23, 42))]
+    run_large(f"sweep_w{window}_{kind}", [0, 15], boxes, n_random=512)
