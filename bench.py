@@ -1,0 +1,377 @@
+#!/usr/bin/env python
+"""Benchmark of the 3D-DSA library: forward + backward Mtokens/s on synthetic latent video.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A step is one forward plus one backward over one video of the workload (default: the
+1080p x 256-frame bf16 configuration).  With N > 1 (launched by torch.distributed.run,
+one rank per GPU) every rank processes its own video of a batch of N: videos are
+independent, there is no collective on the data path, and the result is weak scaling.
+
+The printed JSON line carries: `value` (Mtokens/s with the inputs resident in HBM, CUDA
+events on the launching stream, max over ranks), `e2e` (the same through dsa3d_step_host
+with pinned HOST buffers, copies inside the timed region), `roofline` (algorithmic bytes
+of the dominant kernel / its event-timed duration, against the measured HBM copy rate),
+`cpu_baseline` (the CPU oracle timed on a bounded sample, rank 0, N = 1 only), `clocks`
+(nvidia-smi samples taken during the timed region) and `gpu_launches`.
+
+`--impl reference` times the CPU oracle alone on the host cores on bounded samples of the
+same workload and prints the same kind of line with "impl": "reference".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch
+
+from paper_2607_22696_b200 import inputs
+
+METRIC = "3D-DSA fwd+bwd Mtokens/s (bf16), inputs resident in HBM"
+UNIT = "Mtokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ----------------------------------------------------------------------------- utilities
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (no MEASURED_PEAKS.json)"
+
+
+class ClockSampler:
+    """nvidia-smi samples every 200 ms while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "200", "-i", str(gpu_index)], stdout=self.file, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), power_w_max=max(power),
+                       reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------- CPU oracle sampling
+
+def oracle_sample(wl, rows: int, device_for_generation):
+    """A bounded, exact sample of the workload for the CPU oracle: the first `rows` grid rows
+    of the middle frame as queries, evaluated on the crop of frames that their samples can
+    reach (exact, because no sample leaves the crop: |offset_t| is bounded by the largest
+    offset actually drawn for these queries).  Returns the cropped problem as CPU tensors."""
+    tq = wl.T // 2
+    rows = max(1, min(rows, wl.H))
+    off_q = inputs.make_offsets(wl, device_for_generation, frames=(tq, tq + 1))[:, :rows].contiguous()
+    finite = off_q[torch.isfinite(off_q)]
+    reach = int(math.floor(2 + wl.window[0] // 2 + (float(finite.abs().max()) if finite.numel() else 0.0)))
+    t0, t1 = max(0, tq - reach), min(wl.T, tq + reach + 1)
+    k = inputs.make_rows(wl, "k", device_for_generation, frames=(t0, t1)).cpu()
+    v = inputs.make_rows(wl, "v", device_for_generation, frames=(t0, t1)).cpu()
+    q = inputs.make_rows(wl, "q", device_for_generation, frames=(tq, tq + 1))[:, :rows].contiguous().cpu()
+    dout = inputs.make_rows(wl, "dout", device_for_generation, frames=(tq, tq + 1))[:, :rows].contiguous().cpu()
+    Tc = t1 - t0
+    qtok = ((tq - t0) * wl.H * wl.W + torch.arange(rows * wl.W)).to(torch.int64)
+    return dict(q=q.view(-1, wl.heads, wl.d), k=k, v=v, offsets=off_q.cpu().view(-1, wl.heads, wl.P, 3),
+                dout=dout.view(-1, wl.heads, wl.d), qtok=qtok, dims=(Tc, wl.H, wl.W, wl.heads, wl.d),
+                tokens=rows * wl.W,
+                desc=f"{rows} grid rows ({rows * wl.W} query tokens, all {wl.heads} heads) of frame {tq}, "
+                     f"{'fwd+bwd incl. dK/dV' if wl.backward else 'forward only'}, on the exact {Tc}-frame "
+                     f"crop their samples reach")
+
+
+def time_oracle(sample, wl, backward=True):
+    import oracle
+    T, H, W, heads, d = sample["dims"]
+    t0 = time.perf_counter()
+    oracle.forward(sample["q"], sample["k"], sample["v"], sample["offsets"], T, H, W, heads, d, wl.window,
+                   qtok=sample["qtok"])
+    threads = oracle.last_threads()
+    if backward:
+        oracle.backward(sample["q"], sample["k"], sample["v"], sample["offsets"], sample["dout"], T, H, W,
+                        heads, d, wl.window, qtok=sample["qtok"])
+    return time.perf_counter() - t0, threads
+
+
+def run_reference(args, wl):
+    """The CPU oracle as it stands, on the host cores, on bounded samples of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    gen_dev = "cuda" if torch.cuda.is_available() else "cpu"
+    probe = oracle_sample(wl, 1, gen_dev)
+    dt, _ = time_oracle(probe, wl, wl.backward)                       # sizes the sample; not reported
+    per_row = max(dt, 1e-3)
+    target = min(4.0, 150.0 / max(1, args.steps + args.warmup))
+    rows = max(1, min(wl.H, int(target / per_row)))
+    sample = oracle_sample(wl, rows, gen_dev)
+    for _ in range(args.warmup):
+        time_oracle(sample, wl, wl.backward)
+    times, threads = [], 1
+    for _ in range(args.steps):
+        dt, threads = time_oracle(sample, wl, wl.backward)
+        times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    value = sample["tokens"] / (ms * 1e-3) / 1e6
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "grid": [wl.T, wl.H, wl.W], "heads": wl.heads, "d": wl.d,
+                   "window": list(wl.window), "storage": str(wl.dtype).replace("torch.", ""),
+                   "offsets": f"{wl.offsets} sigma={wl.sigma}", "step": "one bounded sample per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": sample["desc"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------ GPU arm
+
+def run_ours(args, wl):
+    from paper_2607_22696_b200 import binding
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the operator has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    binding.load()
+    dims = (wl.T, wl.H, wl.W, wl.heads, wl.d)
+    # every rank takes its own video of the batch: same shape, its own seed
+    wl_rank = wl if rank == 0 else inputs.dataclasses.replace(wl, seed=wl.seed + 1000 * rank)
+    t = inputs.make_inputs(wl_rank, dev, with_dout=True)
+    ws_bytes = binding.dsa3d_backward_workspace_bytes(*dims, wl.window, wl.dtype)
+    b = {"out": torch.empty_like(t["q"]),
+         "lse": torch.empty(wl.T, wl.H, wl.W, wl.heads, dtype=torch.float32, device=dev),
+         "dq": torch.empty_like(t["q"]), "dk": torch.empty_like(t["q"]), "dv": torch.empty_like(t["q"]),
+         "doff": torch.empty_like(t["offsets"]),
+         "ws": torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=dev)}
+
+    def step():
+        binding.dsa3d_forward(t["q"], t["k"], t["v"], t["offsets"], *dims, wl.window, b["out"], b["lse"])
+        if wl.backward:
+            binding.dsa3d_backward(t["q"], t["k"], t["v"], t["offsets"], b["lse"], t["dout"], *dims,
+                                   wl.window, b["dq"], b["dk"], b["dv"], b["doff"], b["ws"])
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(K)]
+    for row in ev:                      # give every event a handle before the hook sees it
+        for e in row:
+            e.record()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    barrier()
+    torch.cuda.synchronize()
+    for i in range(K):
+        binding.dsa3d_set_profile_events(ev[i][2], ev[i][3], ev[i][4], ev[i][5])
+        ev[i][0].record()
+        step()
+        ev[i][1].record()
+    torch.cuda.synchronize()
+    barrier()
+    binding.dsa3d_set_profile_events(None, None, None, None)
+    clocks = sampler.stop() if sampler else None
+
+    step_ms = ev[0][0].elapsed_time(ev[K - 1][1]) / K
+    fwd_ms = sum(ev[i][2].elapsed_time(ev[i][3]) for i in range(K)) / K
+    bwd_ms = sum(ev[i][4].elapsed_time(ev[i][5]) for i in range(K)) / K if wl.backward else 0.0
+    step_ms = max_over_ranks(step_ms)
+    fwd_ms, bwd_ms = max_over_ranks(fwd_ms), max_over_ranks(bwd_ms)
+    value = wl.N * world / (step_ms * 1e-3) / 1e6
+
+    # ---------------------------------------------------------------- end to end (host)
+    e2e = None
+    b.clear()                           # the end-to-end leg brings its own device arena
+    torch.cuda.empty_cache()
+    if not args.no_e2e:
+        e2e = run_e2e(args, wl, t, dims, dev, barrier, max_over_ranks, world)
+    # --------------------------------------------------------------------- CPU baseline
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        sample = oracle_sample(wl, args.cpu_rows, dev)
+        dt, threads = time_oracle(sample, wl, wl.backward)
+        cpu = {"value": sample["tokens"] / dt / 1e6, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": sample["desc"], "seconds": dt}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peak, peak_src = measured_hbm_peak()
+    fwd_gbs = wl.fwd_bytes() / (fwd_ms * 1e-3) / 1e9
+    bwd_gbs = wl.bwd_bytes() / (bwd_ms * 1e-3) / 1e9 if wl.backward else None
+    dominant_bwd = wl.backward and bwd_ms >= fwd_ms
+    dom = {"kernel": "backward_kernel" if dominant_bwd else "forward_kernel",
+           "achieved": bwd_gbs if dominant_bwd else fwd_gbs,
+           "ms": bwd_ms if dominant_bwd else fwd_ms,
+           "bytes": wl.bwd_bytes() if dominant_bwd else wl.fwd_bytes()}
+    step_bytes = wl.fwd_bytes() + (wl.bwd_bytes() if wl.backward else 0)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+        "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "grid": [wl.T, wl.H, wl.W], "tokens": wl.N, "heads": wl.heads,
+                   "d": wl.d, "window": list(wl.window), "storage": str(wl.dtype).replace("torch.", ""),
+                   "offsets": f"{wl.offsets} sigma={wl.sigma}", "batch_per_gpu": 1,
+                   "parallelism": f"independent videos x{world}",
+                   "l2": "inputs (tens of GB) exceed the 126 MB L2; no flush needed"},
+        "roofline": {"bound": "hbm", "kernel": dom["kernel"], "achieved": dom["achieved"], "peak": peak,
+                     "unit": "GB/s", "frac": dom["achieved"] / peak, "traffic": None,
+                     "peak_source": peak_src, "algorithmic_bytes_per_launch": dom["bytes"],
+                     "kernel_ms": dom["ms"],
+                     "forward_kernel": {"ms": fwd_ms, "achieved": fwd_gbs, "frac": fwd_gbs / peak},
+                     "backward_kernel": ({"ms": bwd_ms, "achieved": bwd_gbs, "frac": bwd_gbs / peak}
+                                         if wl.backward else None),
+                     "whole_step": {"bytes": step_bytes, "achieved": step_bytes / (step_ms * 1e-3) / 1e9,
+                                    "frac": step_bytes / (step_ms * 1e-3) / 1e9 / peak}},
+        "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+        "gpu_launches": K * (4 if (wl.backward and wl.dtype == torch.bfloat16) else 2 if wl.backward else 1),
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, wl, t, dims, dev, barrier, max_over_ranks, world):
+    """Forward + backward through dsa3d_step_host: inputs start in pinned host memory and
+    every output ends in pinned host memory, each step."""
+    from paper_2607_22696_b200 import binding
+    names_in = ["q", "k", "v", "offsets", "dout"]
+    host_in = {}
+    for n in names_in:
+        h = torch.empty(t[n].shape, dtype=t[n].dtype, pin_memory=True)
+        h.copy_(t[n])
+        host_in[n] = h
+    shapes = {n: (t[n].shape, t[n].dtype) for n in names_in}
+    for n in names_in:
+        t[n] = None
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()
+    row_shape, row_dtype = shapes["q"]
+    host_out = {n: torch.empty(row_shape, dtype=row_dtype, pin_memory=True) for n in ("out", "dq", "dk", "dv")}
+    host_out["lse"] = torch.empty(dims[:4], dtype=torch.float32, pin_memory=True)
+    host_out["doffsets"] = torch.empty(shapes["offsets"][0], dtype=torch.float32, pin_memory=True)
+    arena_bytes = binding.dsa3d_step_host_arena_bytes(*dims, wl.window, wl.dtype)
+    arena = torch.empty(arena_bytes, dtype=torch.uint8, device=dev)
+
+    def step():
+        binding.dsa3d_step_host(host_in["q"], host_in["k"], host_in["v"], host_in["offsets"], host_in["dout"],
+                                *dims, wl.window, host_out["out"], host_out["lse"], host_out["dq"],
+                                host_out["dk"], host_out["dv"], host_out["doffsets"], arena)
+
+    steps = max(1, min(args.steps, args.e2e_steps))
+    step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    wall0 = time.perf_counter()
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    wall = (time.perf_counter() - wall0) / steps
+    barrier()
+    ms = max_over_ranks(e0.elapsed_time(e1) / steps)
+    h2d = sum(h.numel() * h.element_size() for h in host_in.values())
+    d2h = sum(h.numel() * h.element_size() for h in host_out.values())
+    return {"value": wl.N * world / (ms * 1e-3) / 1e6, "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": ms, "wall_ms_per_step": wall * 1e3, "steps": steps,
+            "entry_point": "dsa3d_step_host"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="1080p_256f_bf16", choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--cpu-rows", type=int, default=8, help="grid rows of one frame the CPU baseline processes")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    wl = inputs.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

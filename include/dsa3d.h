@@ -91,6 +91,36 @@ int dsa3d_backward(const void* q, const void* k, const void* v, const float* off
 size_t dsa3d_backward_workspace_bytes(int T, int H, int W, int heads, int d,
                                       const int window[3], int dtype);
 
+/*
+ * One whole step from HOST buffers: copies q, k, v, offsets, dout to the device, runs the
+ * forward and the backward above, and copies out, lse, dq, dk, dv, doffsets back.  This is
+ * the operator of Eq. 1 (second term) and its gradient exactly as in dsa3d_forward /
+ * dsa3d_backward; only the location of the buffers differs.
+ * Every *_h pointer is a HOST pointer (page-locked memory makes the copies asynchronous
+ * and fast; pageable memory works but serialises).  `arena` is DEVICE scratch of at least
+ * dsa3d_step_host_arena_bytes(...) bytes, 256-byte aligned, which holds the device copies
+ * and the backward workspace; the library allocates nothing.  All work is enqueued on
+ * `stream`; the host buffers must not be touched until the stream has finished.
+ */
+int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const float* offsets_h,
+                    const void* dout_h, int T, int H, int W, int heads, int d, const int window[3],
+                    void* out_h, float* lse_h, void* dq_h, void* dk_h, void* dv_h, float* doffsets_h,
+                    void* arena, size_t arena_bytes, int dtype, void* stream);
+
+/* Device scratch bytes dsa3d_step_host needs (0 for arguments the library would reject). */
+size_t dsa3d_step_host_arena_bytes(int T, int H, int W, int heads, int d, const int window[3],
+                                   int dtype);
+
+/*
+ * Timing hook (a measurement aid; the paper has no counterpart).  The four arguments are
+ * cudaEvent_t handles created by the caller, or NULL.  While set (per calling thread),
+ * dsa3d_forward records fwd_start / fwd_stop on its stream immediately around the forward
+ * kernel, and dsa3d_backward records bwd_start / bwd_stop immediately around the main
+ * backward kernel (excluding the accumulator clear and the final conversion), so a caller
+ * can time those kernels alone inside a longer step.  Pass four NULLs to switch it off.
+ */
+int dsa3d_set_profile_events(void* fwd_start, void* fwd_stop, void* bwd_start, void* bwd_stop);
+
 /* Static, NUL-terminated description of a status code. */
 const char* dsa3d_status_string(int status);
 

@@ -46,6 +46,12 @@ def load():
     lib.dsa3d_backward.argtypes = [p, p, p, p, p, p, i, i, i, i, i, win, p, p, p, p, p, sz, i, p]
     lib.dsa3d_backward_workspace_bytes.restype = sz
     lib.dsa3d_backward_workspace_bytes.argtypes = [i, i, i, i, i, win, i]
+    lib.dsa3d_step_host.restype = i
+    lib.dsa3d_step_host.argtypes = [p, p, p, p, p, i, i, i, i, i, win, p, p, p, p, p, p, p, sz, i, p]
+    lib.dsa3d_step_host_arena_bytes.restype = sz
+    lib.dsa3d_step_host_arena_bytes.argtypes = [i, i, i, i, i, win, i]
+    lib.dsa3d_set_profile_events.restype = i
+    lib.dsa3d_set_profile_events.argtypes = [p, p, p, p]
     lib.dsa3d_status_string.restype = ctypes.c_char_p
     lib.dsa3d_status_string.argtypes = [i]
     lib.dsa3d_last_cuda_error.restype = i
@@ -138,3 +144,44 @@ def dsa3d_backward(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, d
         _ptr(dq, "dq", n * d), _ptr(dk, "dk", n * d), _ptr(dv, "dv", n * d),
         _ptr(doffsets, "doffsets", n * P * 3, torch.float32),
         _ptr(workspace, "workspace"), int(workspace_bytes), code, _stream(stream)))
+
+
+def _host_ptr(t: torch.Tensor, name: str, numel: int, dtype) -> int:
+    if t.device.type != "cpu" or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CPU tensor")
+    if t.dtype != dtype or t.numel() != numel:
+        raise ValueError(f"{name}: expected {numel} elements of {dtype}")
+    return t.data_ptr()
+
+
+def dsa3d_step_host_arena_bytes(T, H, W, heads, d, window, dtype) -> int:
+    code = _DTYPES[dtype] if isinstance(dtype, torch.dtype) else int(dtype)
+    return int(load().dsa3d_step_host_arena_bytes(T, H, W, heads, d, _window(window), code))
+
+
+def dsa3d_step_host(q_h, k_h, v_h, offsets_h, dout_h, T, H, W, heads, d, window,
+                    out_h, lse_h, dq_h, dk_h, dv_h, doffsets_h, arena, stream=None) -> None:
+    """Forward + backward from HOST tensors (pinned for speed) through a caller-owned
+    device arena (a CUDA uint8 tensor); see include/dsa3d.h.  Asynchronous on `stream`."""
+    lib = load()
+    dt = q_h.dtype
+    n = T * H * W * heads
+    P = int(window[0]) * int(window[1]) * int(window[2])
+    f32 = torch.float32
+    _check(lib.dsa3d_step_host(
+        _host_ptr(q_h, "q_h", n * d, dt), _host_ptr(k_h, "k_h", n * d, dt), _host_ptr(v_h, "v_h", n * d, dt),
+        _host_ptr(offsets_h, "offsets_h", n * P * 3, f32), _host_ptr(dout_h, "dout_h", n * d, dt),
+        T, H, W, heads, d, _window(window),
+        _host_ptr(out_h, "out_h", n * d, dt), _host_ptr(lse_h, "lse_h", n, f32),
+        _host_ptr(dq_h, "dq_h", n * d, dt), _host_ptr(dk_h, "dk_h", n * d, dt),
+        _host_ptr(dv_h, "dv_h", n * d, dt), _host_ptr(doffsets_h, "doffsets_h", n * P * 3, f32),
+        _ptr(arena, "arena"), arena.numel() * arena.element_size(), _DTYPES[dt], _stream(stream)))
+
+
+def dsa3d_set_profile_events(fwd_start=None, fwd_stop=None, bwd_start=None, bwd_stop=None) -> None:
+    """Timing hook: torch.cuda.Event objects (created with enable_timing=True and already
+    recorded once so that their handles exist) or None."""
+    def handle(ev):
+        return None if ev is None else ev.cuda_event
+    _check(load().dsa3d_set_profile_events(handle(fwd_start), handle(fwd_stop), handle(bwd_start),
+                                           handle(bwd_stop)))

@@ -61,13 +61,15 @@ def _hash_chunk(seed: int, tensor_id: int, start: int, count: int, device) -> to
 
 
 def normal(shape, seed: int, tensor_id: int, sigma: float, dtype: torch.dtype, device="cpu",
-           chunk: int = 1 << 24) -> torch.Tensor:
-    """iid N(0, sigma^2) tensor, rounded once (RNE) to ``dtype``."""
+           chunk: int = 1 << 24, first: int = 0) -> torch.Tensor:
+    """iid N(0, sigma^2) tensor, rounded once (RNE) to ``dtype``.  ``first`` is the flat index
+    of the tensor's first element inside a larger logical tensor, so a slice of a big
+    workload can be produced without the rest."""
     n = math.prod(shape)
     out = torch.empty(n, dtype=dtype, device=device)
     for start in range(0, n, chunk):
         cnt = min(chunk, n - start)
-        h = _hash_chunk(seed, tensor_id, start, cnt, device)
+        h = _hash_chunk(seed, tensor_id, first + start, cnt, device)
         u1 = (_lsr(h, 32).to(torch.float64) + 0.5) * (1.0 / 4294967296.0)
         u2 = ((h & 0xFFFFFFFF).to(torch.float64) + 0.5) * (1.0 / 4294967296.0)
         z = torch.sqrt(-2.0 * torch.log(u1)) * torch.cos((2.0 * math.pi) * u2)
@@ -76,14 +78,14 @@ def normal(shape, seed: int, tensor_id: int, sigma: float, dtype: torch.dtype, d
 
 
 def uniform_int(shape, seed: int, tensor_id: int, lo: int, hi: int, dtype: torch.dtype,
-                device="cpu", chunk: int = 1 << 24) -> torch.Tensor:
+                device="cpu", chunk: int = 1 << 24, first: int = 0) -> torch.Tensor:
     """iid integers uniform on {lo..hi}, stored as ``dtype``."""
     n = math.prod(shape)
     out = torch.empty(n, dtype=dtype, device=device)
     span = hi - lo + 1
     for start in range(0, n, chunk):
         cnt = min(chunk, n - start)
-        h = _lsr(_hash_chunk(seed, tensor_id, start, cnt, device), 16)
+        h = _lsr(_hash_chunk(seed, tensor_id, first + start, cnt, device), 16)
         out[start:start + cnt] = (h % span + lo).to(dtype)
     return out.view(*shape)
 
@@ -142,14 +144,26 @@ WORKLOADS: Dict[str, Workload] = {w.name: w for w in [
 ]}
 
 
-def make_offsets(wl: Workload, device="cpu") -> torch.Tensor:
-    shape = (wl.T, wl.H, wl.W, wl.heads, wl.P, 3)
+def make_offsets(wl: Workload, device="cpu", frames=None) -> torch.Tensor:
+    """Offsets of the whole grid, or of frames [frames[0], frames[1]) only."""
+    t0, t1 = (0, wl.T) if frames is None else frames
+    shape = (t1 - t0, wl.H, wl.W, wl.heads, wl.P, 3)
+    first = t0 * wl.H * wl.W * wl.heads * wl.P * 3
     if wl.offsets == "zero":
         return torch.zeros(shape, dtype=torch.float32, device=device)
     if wl.offsets == "int":
         return uniform_int(shape, wl.seed, TENSOR_IDS["offsets"], -wl.int_range, wl.int_range,
-                           torch.float32, device)
-    return normal(shape, wl.seed, TENSOR_IDS["offsets"], wl.sigma, torch.float32, device)
+                           torch.float32, device, first=first)
+    return normal(shape, wl.seed, TENSOR_IDS["offsets"], wl.sigma, torch.float32, device, first=first)
+
+
+def make_rows(wl: Workload, name: str, device="cpu", frames=None) -> torch.Tensor:
+    """Tensor ``name`` in (q, k, v, dout) for the whole grid or for frames [t0, t1) only; the
+    slice equals the same frames of the full tensor generated on the same kind of device."""
+    t0, t1 = (0, wl.T) if frames is None else frames
+    shape = (t1 - t0, wl.H, wl.W, wl.heads, wl.d)
+    first = t0 * wl.H * wl.W * wl.heads * wl.d
+    return normal(shape, wl.seed, TENSOR_IDS[name], 1.0, wl.dtype, device, first=first)
 
 
 def make_inputs(wl: Workload, device="cpu", with_dout: bool | None = None) -> Dict[str, torch.Tensor]:
