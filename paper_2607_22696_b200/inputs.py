@@ -137,6 +137,9 @@ WORKLOADS: Dict[str, Workload] = {w.name: w for w in [
     Workload("480p_bf16_fwd", 16, 30, 52, 16, 64, (3, 3, 3), _BF16, 1.0, 1, backward=False),
     Workload("720p_bf16", 64, 45, 80, 24, 128, (3, 3, 3), _BF16, 1.5, 2),
     Workload("1080p_256f_bf16", 256, 68, 120, 16, 128, (3, 3, 3), _BF16, 2.0, 3),
+    # a 3 GB cut of the 1080p workload (same heads' row size, window and offset spread, inputs
+    # still several times the L2) for profiler captures that must stay small
+    Workload("profile_small_bf16", 32, 45, 80, 8, 128, (3, 3, 3), _BF16, 2.0, 5),
 ] + [
     Workload(f"sweep_w{kt}{kh}{kw}_{kind}", 64, 45, 80, 16, 128, (kt, kh, kw), _BF16,
              3.0 if kind == "normal" else 0.0, 4, offsets=kind)
