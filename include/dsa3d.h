@@ -112,6 +112,38 @@ size_t dsa3d_step_host_arena_bytes(int T, int H, int W, int heads, int d, const 
                                    int dtype);
 
 /*
+ * Backward without any caller-provided or allocated scratch (the paper has no counterpart;
+ * this exists for deployment reasons only).  Meant for callers that cannot give the
+ * library a workspace: code running where all device memory was planned ahead of time,
+ * plug-ins whose host application owns the allocator, loops where cudaMalloc's implicit
+ * device synchronisation is not acceptable.  Same inputs, outputs and results as
+ * dsa3d_backward, but the fp32 dk/dv accumulators live in a fixed 64 MiB array inside the
+ * library image (each GPU that loads the library holds it until the process exits), so:
+ *   - T*H*W*heads*d must not exceed DSA3D_NOALLOC_MAX_ELEMENTS; larger problems are
+ *     rejected with DSA3D_ERR_WORKSPACE before anything is launched;
+ *   - the function calls no cudaMalloc / cudaFree and nothing else that allocates;
+ *   - the first call on each device looks up the array's device address (one
+ *     cudaGetSymbolAddress with that device current) and caches it; make that first call
+ *     outside any stream capture;
+ *   - all calls share the one array, which keeps the previous call's contents; every call
+ *     clears it on `stream` before use.  Two calls whose GPU work can overlap (different
+ *     streams, or different threads on one device) race on it and give wrong dk/dv:
+ *     serialise them.
+ */
+#define DSA3D_NOALLOC_MAX_ELEMENTS (8u * 1024u * 1024u)
+int dsa3d_backward_noalloc(const void* q, const void* k, const void* v, const float* offsets,
+                           const float* lse, const void* dout,
+                           int T, int H, int W, int heads, int d, const int window[3],
+                           void* dq, void* dk, void* dv, float* doffsets, int dtype, void* stream);
+
+/* DSA3D_NOALLOC_MAX_ELEMENTS as the loaded library was built. */
+size_t dsa3d_backward_noalloc_max_elements(void);
+
+/* cudaError_t of the most recent failed address lookup of dsa3d_backward_noalloc on the
+ * calling thread (0 if none). */
+int dsa3d_backward_noalloc_last_cuda_error(void);
+
+/*
  * Timing hook (a measurement aid; the paper has no counterpart).  The four arguments are
  * cudaEvent_t handles created by the caller, or NULL.  While set (per calling thread),
  * dsa3d_forward records fwd_start / fwd_stop on its stream immediately around the forward

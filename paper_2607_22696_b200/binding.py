@@ -52,6 +52,12 @@ def load():
     lib.dsa3d_step_host_arena_bytes.argtypes = [i, i, i, i, i, win, i]
     lib.dsa3d_set_profile_events.restype = i
     lib.dsa3d_set_profile_events.argtypes = [p, p, p, p]
+    lib.dsa3d_backward_noalloc.restype = i
+    lib.dsa3d_backward_noalloc.argtypes = [p, p, p, p, p, p, i, i, i, i, i, win, p, p, p, p, i, p]
+    lib.dsa3d_backward_noalloc_max_elements.restype = sz
+    lib.dsa3d_backward_noalloc_max_elements.argtypes = []
+    lib.dsa3d_backward_noalloc_last_cuda_error.restype = i
+    lib.dsa3d_backward_noalloc_last_cuda_error.argtypes = []
     lib.dsa3d_status_string.restype = ctypes.c_char_p
     lib.dsa3d_status_string.argtypes = [i]
     lib.dsa3d_last_cuda_error.restype = i
@@ -185,3 +191,26 @@ def dsa3d_set_profile_events(fwd_start=None, fwd_stop=None, bwd_start=None, bwd_
         return None if ev is None else ev.cuda_event
     _check(load().dsa3d_set_profile_events(handle(fwd_start), handle(fwd_stop), handle(bwd_start),
                                            handle(bwd_stop)))
+
+
+def dsa3d_backward_noalloc_max_elements() -> int:
+    return int(load().dsa3d_backward_noalloc_max_elements())
+
+
+def dsa3d_backward_noalloc(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets,
+                           dtype=None, stream=None) -> None:
+    """Backward for callers that cannot supply scratch memory: same results as
+    dsa3d_backward, accumulators in a fixed array inside the library (problems up to
+    dsa3d_backward_noalloc_max_elements() = T*H*W*heads*d elements).  Calls on one device
+    must not overlap; see include/dsa3d.h."""
+    lib = load()
+    dt = q.dtype if dtype is None else dtype
+    code = _DTYPES[dt] if isinstance(dt, torch.dtype) else int(dt)
+    n = T * H * W * heads
+    P = int(window[0]) * int(window[1]) * int(window[2])
+    _check(lib.dsa3d_backward_noalloc(
+        _ptr(q, "q", n * d), _ptr(k, "k", n * d), _ptr(v, "v", n * d),
+        _ptr(offsets, "offsets", n * P * 3, torch.float32), _ptr(lse, "lse", n, torch.float32),
+        _ptr(dout, "dout", n * d), T, H, W, heads, d, _window(window),
+        _ptr(dq, "dq", n * d), _ptr(dk, "dk", n * d), _ptr(dv, "dv", n * d),
+        _ptr(doffsets, "doffsets", n * P * 3, torch.float32), code, _stream(stream)))
