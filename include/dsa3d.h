@@ -76,7 +76,8 @@ int dsa3d_forward(const void* q, const void* k, const void* v, const float* offs
  *                one-sided convention of the floor at integer positions (cell [i, i+1))
  * The sampling weights are recomputed, nothing of size N*P*d is stored.
  * `workspace` is device scratch of at least dsa3d_backward_workspace_bytes(...) bytes,
- * 16-byte aligned (fp32 accumulators for dk and dv; may be NULL when that size is 0).
+ * 16-byte aligned (bf16 storage: fp32 accumulators for dk and dv, two fp32 coefficients per
+ * sample, and the bins of the tile pre-reduction; may be NULL when that size is 0).
  * Its contents on entry do not matter.  dk and dv are summed with floating-point atomics,
  * so their last bits can differ from run to run; dq, doffsets are deterministic.
  */
@@ -144,14 +145,15 @@ size_t dsa3d_backward_noalloc_max_elements(void);
 int dsa3d_backward_noalloc_last_cuda_error(void);
 
 /*
- * Timing hook (a measurement aid; the paper has no counterpart).  The four arguments are
+ * Timing hook (a measurement aid; the paper has no counterpart).  The six arguments are
  * cudaEvent_t handles created by the caller, or NULL.  While set (per calling thread),
  * dsa3d_forward records fwd_start / fwd_stop on its stream immediately around the forward
- * kernel, and dsa3d_backward records bwd_start / bwd_stop immediately around the main
- * backward kernel (excluding the accumulator clear and the final conversion), so a caller
- * can time those kernels alone inside a longer step.  Pass four NULLs to switch it off.
+ * kernel, and dsa3d_backward records bwd_start / bwd_stop around its gather kernel and
+ * scatter_start / scatter_stop around its tile scatter kernel (when that kernel runs), so a
+ * caller can time those kernels alone inside a longer step.  Pass NULLs to switch it off.
  */
-int dsa3d_set_profile_events(void* fwd_start, void* fwd_stop, void* bwd_start, void* bwd_stop);
+int dsa3d_set_profile_events(void* fwd_start, void* fwd_stop, void* bwd_start, void* bwd_stop,
+                             void* scatter_start, void* scatter_stop);
 
 /* Static, NUL-terminated description of a status code. */
 const char* dsa3d_status_string(int status);

@@ -51,7 +51,7 @@ def load():
     lib.dsa3d_step_host_arena_bytes.restype = sz
     lib.dsa3d_step_host_arena_bytes.argtypes = [i, i, i, i, i, win, i]
     lib.dsa3d_set_profile_events.restype = i
-    lib.dsa3d_set_profile_events.argtypes = [p, p, p, p]
+    lib.dsa3d_set_profile_events.argtypes = [p, p, p, p, p, p]
     lib.dsa3d_backward_noalloc.restype = i
     lib.dsa3d_backward_noalloc.argtypes = [p, p, p, p, p, p, i, i, i, i, i, win, p, p, p, p, i, p]
     lib.dsa3d_backward_noalloc_max_elements.restype = sz
@@ -184,13 +184,14 @@ def dsa3d_step_host(q_h, k_h, v_h, offsets_h, dout_h, T, H, W, heads, d, window,
         _ptr(arena, "arena"), arena.numel() * arena.element_size(), _DTYPES[dt], _stream(stream)))
 
 
-def dsa3d_set_profile_events(fwd_start=None, fwd_stop=None, bwd_start=None, bwd_stop=None) -> None:
+def dsa3d_set_profile_events(fwd_start=None, fwd_stop=None, bwd_start=None, bwd_stop=None,
+                             scatter_start=None, scatter_stop=None) -> None:
     """Timing hook: torch.cuda.Event objects (created with enable_timing=True and already
     recorded once so that their handles exist) or None."""
     def handle(ev):
         return None if ev is None else ev.cuda_event
     _check(load().dsa3d_set_profile_events(handle(fwd_start), handle(fwd_stop), handle(bwd_start),
-                                           handle(bwd_stop)))
+                                           handle(bwd_stop), handle(scatter_start), handle(scatter_stop)))
 
 
 def dsa3d_backward_noalloc_max_elements() -> int:

@@ -1,6 +1,8 @@
 // C ABI of the 3D-DSA library: argument validation, workspace layout, launches.
 // Declarations and the contract of every entry point are in include/dsa3d.h.
 #include <stdint.h>
+#include <stdio.h>
+#include <stdlib.h>
 
 #include "../../include/dsa3d.h"
 #include "dsa3d_kernels.h"
@@ -8,7 +10,7 @@
 namespace {
 
 thread_local int g_last_cuda_error = 0;
-thread_local cudaEvent_t g_events[4] = {nullptr, nullptr, nullptr, nullptr};   // fwd start/stop, bwd start/stop
+thread_local cudaEvent_t g_events[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};   // fwd, bwd gather, bwd tile scatter: start/stop each
 
 cudaError_t record(int which, cudaStream_t stream) {
     return g_events[which] ? cudaEventRecord(g_events[which], stream) : cudaSuccess;
@@ -36,10 +38,57 @@ int make_problem(int T, int H, int W, int heads, int d, const int* window, int d
     if (N * heads / 8 >= (1LL << 31) - 1) return DSA3D_ERR_BAD_SHAPE;
     pr.T = T; pr.H = H; pr.W = W; pr.heads = heads; pr.d = d;
     pr.kt = window[0]; pr.kh = window[1]; pr.kw = window[2];
+    // one frame of rows must be addressable with 32-bit element offsets
+    if (static_cast<long long>(H) * W * heads * d >= (1LL << 31)) return DSA3D_ERR_BAD_SHAPE;
     pr.P = static_cast<int>(P);
     pr.N = N;
     pr.items = N * heads;
+    pr.tile_t = pr.tile_y = pr.tile_x = 0;
+    pr.halo = 0;
+    pr.tiles_t = pr.tiles_y = pr.tiles_x = 0;
     return DSA3D_OK;
+}
+
+// Query tiling of the backward scatter: 4 x 8 x 8 queries per tile, halo of 6 cells.  The
+// environment variable DSA3D_TILE="tt,ty,tx,halo" overrides it for experiments ("0" turns
+// the tile kernel off); values that do not fit shared memory fall back to the default.
+constexpr int kTileSlots = 304;          // upper bound on resident tile CTAs (scratch regions)
+constexpr size_t kTileSmemLimit = 200 * 1024;
+
+void set_tiling(dsa3d::Problem& pr) {
+    int tt = 4, ty = 8, tx = 8, halo = 6;
+    if (const char* env = getenv("DSA3D_TILE")) {
+        int a = 0, b = 0, c = 0, h = 0;
+        const int got = sscanf(env, "%d,%d,%d,%d", &a, &b, &c, &h);
+        if (got == 1 && a == 0) return;                       // tiling off
+        if (got == 4 && a >= 1 && b >= 1 && c >= 1 && h >= 0 && a * b * c <= 1024) {
+            dsa3d::Problem probe = pr;
+            probe.tile_t = a; probe.tile_y = b; probe.tile_x = c; probe.halo = h;
+            if (dsa3d::tile_smem_bytes(probe) <= kTileSmemLimit) { tt = a; ty = b; tx = c; halo = h; }
+        }
+    }
+    pr.tile_t = tt; pr.tile_y = ty; pr.tile_x = tx; pr.halo = halo;
+    pr.tiles_t = (pr.T + tt - 1) / tt;
+    pr.tiles_y = (pr.H + ty - 1) / ty;
+    pr.tiles_x = (pr.W + tx - 1) / tx;
+}
+
+struct BackwardWorkspace {
+    size_t acc_bytes, coef_bytes, scratch_bytes, total;
+    long long entries_per_cta;
+};
+
+BackwardWorkspace backward_workspace(const dsa3d::Problem& pr, int dtype, bool tiled) {
+    BackwardWorkspace w{};
+    if (dtype != DSA3D_BF16) return w;
+    w.acc_bytes = static_cast<size_t>(pr.items) * pr.d * sizeof(float) * 2;
+    if (tiled && pr.tile_t >= 1) {
+        w.coef_bytes = static_cast<size_t>(pr.items) * pr.P * sizeof(float2);
+        w.entries_per_cta = static_cast<long long>(pr.tile_t) * pr.tile_y * pr.tile_x * pr.P * 8;
+        w.scratch_bytes = static_cast<size_t>(kTileSlots) * w.entries_per_cta * sizeof(uint2);
+    }
+    w.total = w.acc_bytes + w.coef_bytes + w.scratch_bytes;
+    return w;
 }
 
 }  // namespace
@@ -67,14 +116,24 @@ int dsa3d_forward(const void* q, const void* k, const void* v, const float* offs
 size_t dsa3d_backward_workspace_bytes(int T, int H, int W, int heads, int d, const int window[3], int dtype) {
     dsa3d::Problem pr;
     if (make_problem(T, H, W, heads, d, window, dtype, pr) != DSA3D_OK) return 0;
-    if (dtype == DSA3D_F32) return 0;
-    return static_cast<size_t>(pr.items) * pr.d * sizeof(float) * 2;   // fp32 dK and dV accumulators
+    if (dtype == DSA3D_BF16) set_tiling(pr);
+    return backward_workspace(pr, dtype, true).total;
 }
 
 int dsa3d_backward(const void* q, const void* k, const void* v, const float* offsets, const float* lse,
                    const void* dout, int T, int H, int W, int heads, int d, const int window[3], void* dq,
                    void* dk, void* dv, float* doffsets, void* workspace, size_t workspace_bytes, int dtype,
-                   void* stream_) {
+                   void* stream) {
+    return dsa3d::backward_impl(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets,
+                                workspace, workspace_bytes, dtype, stream, true);
+}
+
+}  // extern "C"
+
+int dsa3d::backward_impl(const void* q, const void* k, const void* v, const float* offsets, const float* lse,
+                         const void* dout, int T, int H, int W, int heads, int d, const int window[3],
+                         void* dq, void* dk, void* dv, float* doffsets, void* workspace,
+                         size_t workspace_bytes, int dtype, void* stream_, bool tiled) {
     if (!q || !k || !v || !offsets || !lse || !dout || !dq || !dk || !dv || !doffsets)
         return DSA3D_ERR_NULL_POINTER;
     dsa3d::Problem pr;
@@ -83,19 +142,23 @@ int dsa3d_backward(const void* q, const void* k, const void* v, const float* off
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(offsets) || !aligned16(lse) ||
         !aligned16(dout) || !aligned16(dq) || !aligned16(dk) || !aligned16(dv) || !aligned16(doffsets))
         return DSA3D_ERR_MISALIGNED;
-    const size_t need = dsa3d_backward_workspace_bytes(T, H, W, heads, d, window, dtype);
-    if (need > 0) {
-        if (!workspace || workspace_bytes < need) return DSA3D_ERR_WORKSPACE;
+    const bool bf16 = dtype == DSA3D_BF16;
+    if (bf16 && tiled) set_tiling(pr);
+    const BackwardWorkspace ws = backward_workspace(pr, dtype, tiled);
+    if (ws.total > 0) {
+        if (!workspace || workspace_bytes < ws.total) return DSA3D_ERR_WORKSPACE;
         if (!aligned16(workspace)) return DSA3D_ERR_MISALIGNED;
     }
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    const bool bf16 = dtype == DSA3D_BF16;
     const size_t count = static_cast<size_t>(pr.items) * pr.d;
-    float* acc_dk = bf16 ? static_cast<float*>(workspace) : static_cast<float*>(dk);
-    float* acc_dv = bf16 ? static_cast<float*>(workspace) + count : static_cast<float*>(dv);
+    char* wsp = static_cast<char*>(workspace);
+    float* acc_dk = bf16 ? reinterpret_cast<float*>(wsp) : static_cast<float*>(dk);
+    float* acc_dv = bf16 ? reinterpret_cast<float*>(wsp) + count : static_cast<float*>(dv);
+    float2* coef = ws.coef_bytes ? reinterpret_cast<float2*>(wsp + ws.acc_bytes) : nullptr;
+    void* scratch = ws.scratch_bytes ? wsp + ws.acc_bytes + ws.coef_bytes : nullptr;
     cudaError_t e;
     if (bf16) {
-        e = cudaMemsetAsync(workspace, 0, need, stream);
+        e = cudaMemsetAsync(workspace, 0, ws.acc_bytes, stream);
         if (e != cudaSuccess) return cuda_failed(e);
     } else {
         e = cudaMemsetAsync(dk, 0, count * sizeof(float), stream);
@@ -105,10 +168,26 @@ int dsa3d_backward(const void* q, const void* k, const void* v, const float* off
     }
     e = record(2, stream);
     if (e != cudaSuccess) return cuda_failed(e);
-    e = dsa3d::launch_backward(q, k, v, offsets, lse, dout, dq, acc_dk, acc_dv, doffsets, pr, bf16, stream);
+    e = dsa3d::launch_backward(q, k, v, offsets, lse, dout, dq, acc_dk, acc_dv, doffsets, coef, pr, bf16, stream);
     if (e != cudaSuccess) return cuda_failed(e);
     e = record(3, stream);
     if (e != cudaSuccess) return cuda_failed(e);
+    if (coef) {
+        int dev = 0, sms = 0;
+        e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return cuda_failed(e);
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return cuda_failed(e);
+        int ctas = sms * (dsa3d::tile_smem_bytes(pr) <= 110 * 1024 ? 2 : 1);
+        if (ctas > kTileSlots) ctas = kTileSlots;
+        e = record(4, stream);
+        if (e != cudaSuccess) return cuda_failed(e);
+        e = dsa3d::launch_scatter_tiles(q, dout, offsets, coef, acc_dk, acc_dv, scratch, ctas,
+                                        ws.entries_per_cta, pr, stream);
+        if (e != cudaSuccess) return cuda_failed(e);
+        e = record(5, stream);
+        if (e != cudaSuccess) return cuda_failed(e);
+    }
     if (bf16) {
         e = dsa3d::launch_convert_bf16(acc_dk, dk, static_cast<long long>(count), stream);
         if (e != cudaSuccess) return cuda_failed(e);
@@ -117,6 +196,8 @@ int dsa3d_backward(const void* q, const void* k, const void* v, const float* off
     }
     return DSA3D_OK;
 }
+
+extern "C" {
 
 namespace {
 
@@ -134,7 +215,11 @@ Arena arena_layout(const dsa3d::Problem& pr, int dtype) {
     a.row_bytes = static_cast<size_t>(pr.items) * pr.d * elt;
     a.off_bytes = static_cast<size_t>(pr.items) * pr.P * 3 * sizeof(float);
     a.lse_bytes = static_cast<size_t>(pr.items) * sizeof(float);
-    a.ws_bytes = dtype == DSA3D_BF16 ? static_cast<size_t>(pr.items) * pr.d * sizeof(float) * 2 : 0;
+    {
+        dsa3d::Problem tiled = pr;
+        if (dtype == DSA3D_BF16) set_tiling(tiled);
+        a.ws_bytes = backward_workspace(tiled, dtype, true).total;
+    }
     size_t at = 0;
     size_t* rows[8] = {&a.q, &a.k, &a.v, &a.dout, &a.out, &a.dq, &a.dk, &a.dv};
     for (size_t* r : rows) { *r = at; at += round256(a.row_bytes); }
@@ -195,11 +280,14 @@ int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const flo
     return DSA3D_OK;
 }
 
-int dsa3d_set_profile_events(void* fwd_start, void* fwd_stop, void* bwd_start, void* bwd_stop) {
+int dsa3d_set_profile_events(void* fwd_start, void* fwd_stop, void* bwd_start, void* bwd_stop,
+                             void* scatter_start, void* scatter_stop) {
     g_events[0] = static_cast<cudaEvent_t>(fwd_start);
     g_events[1] = static_cast<cudaEvent_t>(fwd_stop);
     g_events[2] = static_cast<cudaEvent_t>(bwd_start);
     g_events[3] = static_cast<cudaEvent_t>(bwd_stop);
+    g_events[4] = static_cast<cudaEvent_t>(scatter_start);
+    g_events[5] = static_cast<cudaEvent_t>(scatter_stop);
     return DSA3D_OK;
 }
 

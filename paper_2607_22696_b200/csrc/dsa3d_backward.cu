@@ -1,19 +1,32 @@
 // Backward of 3D Deformable Slide Attention: dQ, dK, dV and dOffsets.
 //
-// Same work decomposition as the forward: a group of LPR = d / VEC lanes owns one
-// (token, head) item, items are ordered head-major.  The sampling weights are recomputed
-// from the offsets, the softmax weights from the saved lse; nothing of size N*P*d exists.
+// Two kernels.
 //
-// Pass 1 (gather): for every sample the corner rows of K and V are loaded once; the lane
+// backward_kernel (one group of LPR = d / VEC lanes per (token, head) item, head-major
+// order, as in the forward).  The sampling weights are recomputed from the offsets, the
+// softmax weights from the saved lse; nothing of size N*P*d exists.
+//   Pass 1 (gather): for every sample the corner rows of K and V are loaded once; the lane
 //   partials of  s = sum_c w_c (q.K_c),  g = sum_c w_c (dO.V_c)  and of the six
 //   derivative sums  A_a = sum_c (dw_c/da)(q.K_c),  B_a = sum_c (dw_c/da)(dO.V_c)  are
 //   reduced over the group; alpha_p = exp(s_p - lse).  With delta = sum_p alpha_p g_p,
 //   dQ = scale * (sum_p alpha_p g_p k_p - delta * sum_p alpha_p k_p) needs no second look
 //   at K.  The eight per-sample numbers are parked in shared memory.
-// Pass 2 (scatter): dS_p = alpha_p (g_p - delta);
-//   dOffsets[p, a] = scale dS_p A_a + alpha_p B_a;  for each corner with a non-zero weight
-//   dK[corner] += w_c scale dS_p q  and  dV[corner] += w_c alpha_p dO  go to the fp32
-//   accumulators with 16-byte vector reductions (red.global.add.v4.f32).
+//   Pass 2: dS_p = alpha_p (g_p - delta);  dOffsets[p, a] = scale dS_p A_a + alpha_p B_a.
+//   The two scatter coefficients of the sample, ck_p = scale dS_p and cv_p = alpha_p, are
+//   written out for the tile kernel; corners that fall OUTSIDE the halo box of the query's
+//   tile are scattered right here, dK[corner] += w_c ck_p q and dV[corner] += w_c cv_p dO,
+//   with 16-byte vector reductions (red.global.add.v4.f32) into fp32 accumulators.
+//
+// scatter_tile_kernel (bf16 storage; one CTA per (head, tile of TQ queries), persistent).
+//   The dK/dV contributions of a tile of neighbouring queries land on a few thousand key
+//   rows around the tile, ~10 contributions per row.  Sending each one to L2 as a 512-byte
+//   fp32 reduction is what bounds the simple scheme (L2 reduction throughput), so the tile
+//   kernel sums them on chip first: it bins the (query, sample, corner) contributions of
+//   the tile by target row (counting sort, counters in shared memory, 8-byte entries in a
+//   per-CTA global scratch that stays in L2), then each half-warp owns a row, walks its
+//   entries, accumulates  coefficient x q-row  and  coefficient x dO-row  in fp32 registers
+//   from the tile's q/dO rows held in shared memory, and issues ONE reduction per row and
+//   tensor.  Coefficients are rounded to bf16 for the mixed-precision FMA.
 #include "dsa3d_common.cuh"
 #include "dsa3d_kernels.h"
 
@@ -31,8 +44,11 @@ __global__ void __launch_bounds__(256)
 backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                 const float* __restrict__ offsets, const float* __restrict__ lse,
                 const T* __restrict__ dout, T* __restrict__ dq, float* __restrict__ acc_dk,
-                float* __restrict__ acc_dv, float* __restrict__ doffsets, const Problem pr) {
-    constexpr int VEC = Elt<T>::VEC;
+                float* __restrict__ acc_dv, float* __restrict__ doffsets, float2* __restrict__ coef,
+                const Problem pr) {
+    using E = Elt<T>;
+    using Row = typename E::Row;
+    constexpr int VEC = E::VEC;
     constexpr int LPR = D / VEC;
     extern __shared__ float smem[];
     const int lane = threadIdx.x & 31;
@@ -47,17 +63,18 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
     const int x = static_cast<int>(n % pr.W);
     const int y = static_cast<int>((n / pr.W) % pr.H);
     const int t = static_cast<int>(n / (static_cast<long long>(pr.W) * pr.H));
-    const int HW = pr.H * pr.W;
     const long long row = n * pr.heads + m;
     const int ch = gl * VEC;
     const float scale = rsqrtf(static_cast<float>(D));
+    const long long tok_stride = static_cast<long long>(pr.heads) * D;
+    const int sx = static_cast<int>(tok_stride);
+    const int sy = pr.W * sx;
+    const int st = pr.H * sy;
 
-    float qf[VEC], dof[VEC];
-    Elt<T>::load(q + row * D + ch, qf);
-    Elt<T>::load(dout + row * D + ch, dof);
+    const Row qr = E::load(q + row * D + ch);
+    const Row dor = E::load(dout + row * D + ch);
     const float lse2 = __ldg(lse + row) * kLog2e;            // lse in log2 units
     const float* off_row = offsets + row * pr.P * 3;
-    const long long tok_stride = static_cast<long long>(pr.heads) * D;
     const long long head_off = static_cast<long long>(m) * D + ch;
     const T* kh = k + head_off;
     const T* vh = v + head_off;
@@ -71,37 +88,36 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
     for (int pb = 0; pb < pr.P; pb += LPR) {
         Sample mine;
         mine.base = 0; mine.mask = 0u; mine.ft = mine.fy = mine.fx = 0.0f;
-        if (pb + gl < pr.P) mine = make_sample(pr, t, y, x, pb + gl, off_row + (pb + gl) * 3);
+        if (pb + gl < pr.P) mine = to_sample(pr, make_cell(pr, t, y, x, pb + gl, off_row + (pb + gl) * 3));
         const int cnt = min(LPR, pr.P - pb);
         for (int j = 0; j < cnt; ++j) {
             const Sample s = group_bcast<LPR>(mine, j, gmask);
             const float wt[2] = {1.0f - s.ft, s.ft}, wy[2] = {1.0f - s.fy, s.fy}, wx[2] = {1.0f - s.fx, s.fx};
+            const T* kb = kh + s.base * tok_stride;
+            const T* vb = vh + s.base * tok_stride;
             float r[kStats];
 #pragma unroll
             for (int i = 0; i < kStats; ++i) r[i] = 0.0f;
             float kp[VEC];
 #pragma unroll
             for (int e = 0; e < VEC; ++e) kp[e] = 0.0f;
+            const bool full = s.mask == 0xffu && s.ft != 0.0f && s.fy != 0.0f && s.fx != 0.0f;
+            if (full) {                    // every corner inside the grid and needed: 16 loads back to back
+                Row kk[8], vv[8];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const int ct = c >> 2, cy = (c >> 1) & 1, cx = c & 1;
-                const float w = wt[ct] * wy[cy] * wx[cx];
-                const float dwt = (ct ? 1.0f : -1.0f) * wy[cy] * wx[cx];
-                const float dwy = (cy ? 1.0f : -1.0f) * wt[ct] * wx[cx];
-                const float dwx = (cx ? 1.0f : -1.0f) * wt[ct] * wy[cy];
-                const bool needed = (w != 0.0f) | (dwt != 0.0f) | (dwy != 0.0f) | (dwx != 0.0f);
-                if (((s.mask >> c) & 1u) && needed) {
-                    const int tok = s.base + ct * HW + cy * pr.W + cx;
-                    float kk[VEC], vv[VEC];
-                    Elt<T>::load(kh + tok * tok_stride, kk);
-                    Elt<T>::load(vh + tok * tok_stride, vv);
-                    float a = 0.0f, b = 0.0f;
+                for (int c = 0; c < 8; ++c) kk[c] = E::load(kb + ((c >> 2) * st + ((c >> 1) & 1) * sy + (c & 1) * sx));
 #pragma unroll
-                    for (int e = 0; e < VEC; ++e) {
-                        a = fmaf(qf[e], kk[e], a);
-                        b = fmaf(dof[e], vv[e], b);
-                        kp[e] = fmaf(w, kk[e], kp[e]);
-                    }
+                for (int c = 0; c < 8; ++c) vv[c] = E::load(vb + ((c >> 2) * st + ((c >> 1) & 1) * sy + (c & 1) * sx));
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const int ct = c >> 2, cy = (c >> 1) & 1, cx = c & 1;
+                    const float w = wt[ct] * wy[cy] * wx[cx];
+                    const float dwt = (ct ? 1.0f : -1.0f) * wy[cy] * wx[cx];
+                    const float dwy = (cy ? 1.0f : -1.0f) * wt[ct] * wx[cx];
+                    const float dwx = (cx ? 1.0f : -1.0f) * wt[ct] * wy[cy];
+                    const float a = E::dot(qr, kk[c], 0.0f);
+                    const float b = E::dot(dor, vv[c], 0.0f);
+                    E::axpy(w, kk[c], kp);
                     r[0] = fmaf(w, a, r[0]);
                     r[1] = fmaf(w, b, r[1]);
                     r[2] = fmaf(dwt, a, r[2]);
@@ -110,6 +126,32 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
                     r[5] = fmaf(dwt, b, r[5]);
                     r[6] = fmaf(dwy, b, r[6]);
                     r[7] = fmaf(dwx, b, r[7]);
+                }
+            } else {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const int ct = c >> 2, cy = (c >> 1) & 1, cx = c & 1;
+                    const float w = wt[ct] * wy[cy] * wx[cx];
+                    const float dwt = (ct ? 1.0f : -1.0f) * wy[cy] * wx[cx];
+                    const float dwy = (cy ? 1.0f : -1.0f) * wt[ct] * wx[cx];
+                    const float dwx = (cx ? 1.0f : -1.0f) * wt[ct] * wy[cy];
+                    const bool needed = (w != 0.0f) | (dwt != 0.0f) | (dwy != 0.0f) | (dwx != 0.0f);
+                    if (((s.mask >> c) & 1u) && needed) {
+                        const int o = ct * st + cy * sy + cx * sx;
+                        const Row kk = E::load(kb + o);
+                        const Row vv = E::load(vb + o);
+                        const float a = E::dot(qr, kk, 0.0f);
+                        const float b = E::dot(dor, vv, 0.0f);
+                        E::axpy(w, kk, kp);
+                        r[0] = fmaf(w, a, r[0]);
+                        r[1] = fmaf(w, b, r[1]);
+                        r[2] = fmaf(dwt, a, r[2]);
+                        r[3] = fmaf(dwy, a, r[3]);
+                        r[4] = fmaf(dwx, a, r[4]);
+                        r[5] = fmaf(dwt, b, r[5]);
+                        r[6] = fmaf(dwy, b, r[6]);
+                        r[7] = fmaf(dwx, b, r[7]);
+                    }
                 }
             }
 #pragma unroll
@@ -124,10 +166,10 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
                 kbar[e] = fmaf(alpha, kp[e], kbar[e]);
             }
             if (gl == 0) {
-                float* st = stats + (pb + j) * kStats;
-                st[0] = alpha; st[1] = g;
-                st[2] = r[2]; st[3] = r[3]; st[4] = r[4];
-                st[5] = r[5]; st[6] = r[6]; st[7] = r[7];
+                float* sts = stats + (pb + j) * kStats;
+                sts[0] = alpha; sts[1] = g;
+                sts[2] = r[2]; sts[3] = r[3]; sts[4] = r[4];
+                sts[5] = r[5]; sts[6] = r[6]; sts[7] = r[7];
             }
         }
     }
@@ -135,11 +177,14 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
         float dqv[VEC];
 #pragma unroll
         for (int e = 0; e < VEC; ++e) dqv[e] = scale * fmaf(-delta, kbar[e], u_acc[e]);
-        Elt<T>::store(dq + row * D + ch, dqv);
+        E::store(dq + row * D + ch, dqv);
     }
     __syncwarp(gmask);
 
-    // ---------------------------------------------------------------- pass 2: scatter
+    // ------------------------------------------- pass 2: dOffsets, coefficients, far scatter
+    float qf[VEC], dof[VEC];
+    E::to_float(qr, qf);
+    E::to_float(dor, dof);
     float* dk_h = acc_dk + head_off;
     float* dv_h = acc_dv + head_off;
     float* doff_row = doffsets + row * pr.P * 3;
@@ -149,31 +194,35 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
         float my_ck = 0.0f, my_cv = 0.0f;
         if (pb + gl < pr.P) {
             const int p = pb + gl;
-            mine = make_sample(pr, t, y, x, p, off_row + p * 3);
-            const float* st = stats + p * kStats;
-            const float alpha = st[0];
-            const float dS = alpha * (st[1] - delta);
+            const Cell cell = make_cell(pr, t, y, x, p, off_row + p * 3);
+            mine = to_sample(pr, cell);
+            mine.mask = cell.mask & ~halo_corner_mask(pr, cell, t, y, x);   // corners the tile kernel does not take
+            const float* sts = stats + p * kStats;
+            const float alpha = sts[0];
+            const float dS = alpha * (sts[1] - delta);
             my_ck = scale * dS;
             my_cv = alpha;
-            doff_row[p * 3 + 0] = fmaf(my_ck, st[2], alpha * st[5]);
-            doff_row[p * 3 + 1] = fmaf(my_ck, st[3], alpha * st[6]);
-            doff_row[p * 3 + 2] = fmaf(my_ck, st[4], alpha * st[7]);
+            doff_row[p * 3 + 0] = fmaf(my_ck, sts[2], alpha * sts[5]);
+            doff_row[p * 3 + 1] = fmaf(my_ck, sts[3], alpha * sts[6]);
+            doff_row[p * 3 + 2] = fmaf(my_ck, sts[4], alpha * sts[7]);
+            if (coef) coef[row * pr.P + p] = make_float2(my_ck, my_cv);
         }
         const int cnt = min(LPR, pr.P - pb);
         for (int j = 0; j < cnt; ++j) {
+            const unsigned mask = __shfl_sync(gmask, mine.mask, j, LPR);
+            if (mask == 0u) continue;
             const Sample s = group_bcast<LPR>(mine, j, gmask);
             const float ck = __shfl_sync(gmask, my_ck, j, LPR);
             const float cv = __shfl_sync(gmask, my_cv, j, LPR);
-            if (s.mask == 0u) continue;
             const float wt[2] = {1.0f - s.ft, s.ft}, wy[2] = {1.0f - s.fy, s.fy}, wx[2] = {1.0f - s.fx, s.fx};
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const float w = wt[c >> 2] * wy[(c >> 1) & 1] * wx[c & 1];
                 if (((s.mask >> c) & 1u) && w != 0.0f) {
-                    const int tok = s.base + (c >> 2) * HW + ((c >> 1) & 1) * pr.W + (c & 1);
+                    const long long o = s.base * tok_stride + ((c >> 2) * st + ((c >> 1) & 1) * sy + (c & 1) * sx);
                     const float wk = w * ck, wv = w * cv;
-                    float* pk = dk_h + tok * tok_stride;
-                    float* pv = dv_h + tok * tok_stride;
+                    float* pk = dk_h + o;
+                    float* pv = dv_h + o;
 #pragma unroll
                     for (int e = 0; e < VEC; e += 4) {
                         red_add_v4(pk + e, wk * qf[e], wk * qf[e + 1], wk * qf[e + 2], wk * qf[e + 3]);
@@ -185,10 +234,213 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Tile scatter (bf16 storage).
+// ---------------------------------------------------------------------------------------
+constexpr int kTileThreads = 512;
+
+template <int D>
+__global__ void __launch_bounds__(kTileThreads, 1)
+scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ dout,
+                    const float* __restrict__ offsets, const float2* __restrict__ coef,
+                    float* __restrict__ acc_dk, float* __restrict__ acc_dv, uint2* __restrict__ scratch,
+                    const long long scratch_entries_per_cta, const Problem pr) {
+    using E = Elt<__nv_bfloat16>;
+    using Row = E::Row;
+    constexpr int VPR = D / 8;                       // 16-byte vectors per row
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int TQ = pr.tile_t * pr.tile_y * pr.tile_x;
+    const int et = pr.tile_t + 2 * pr.halo, ey = pr.tile_y + 2 * pr.halo, ex = pr.tile_x + 2 * pr.halo;
+    const int NB = et * ey * ex;
+    uint4* qrows = reinterpret_cast<uint4*>(smem_raw);                 // [TQ][VPR]
+    uint4* dorows = qrows + static_cast<size_t>(TQ) * VPR;              // [TQ][VPR]
+    unsigned* cursor = reinterpret_cast<unsigned*>(dorows + static_cast<size_t>(TQ) * VPR);   // [NB]
+    __shared__ unsigned warp_sums[kTileThreads / 32];
+
+    const int tid = threadIdx.x;
+    const int tiles_per_head = pr.tiles_t * pr.tiles_y * pr.tiles_x;
+    const long long total_tiles = static_cast<long long>(tiles_per_head) * pr.heads;
+    uint2* my_scratch = scratch + static_cast<long long>(blockIdx.x) * scratch_entries_per_cta;
+    const long long tok_stride = static_cast<long long>(pr.heads) * D;
+
+    for (long long tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
+        const int m = static_cast<int>(tile_id / tiles_per_head);
+        int rem = static_cast<int>(tile_id - static_cast<long long>(m) * tiles_per_head);
+        const int tx = rem % pr.tiles_x; rem /= pr.tiles_x;
+        const int ty = rem % pr.tiles_y;
+        const int tt = rem / pr.tiles_y;
+        const int t0 = tt * pr.tile_t, y0 = ty * pr.tile_y, x0 = tx * pr.tile_x;
+        const int lo_t = t0 - pr.halo, lo_y = y0 - pr.halo, lo_x = x0 - pr.halo;
+
+        // ---- stage the tile's q and dO rows, clear the bin counters
+        for (int i = tid; i < NB; i += kTileThreads) cursor[i] = 0u;
+        for (int i = tid; i < TQ * VPR; i += kTileThreads) {
+            const int ql = i / VPR, vec = i - ql * VPR;
+            const int lx = ql % pr.tile_x, ly = (ql / pr.tile_x) % pr.tile_y, lt = ql / (pr.tile_x * pr.tile_y);
+            const int t = t0 + lt, y = y0 + ly, x = x0 + lx;
+            uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+            if (t < pr.T && y < pr.H && x < pr.W) {
+                const long long n = (static_cast<long long>(t) * pr.H + y) * pr.W + x;
+                const long long o = (n * pr.heads + m) * D + vec * 8;
+                a = __ldg(reinterpret_cast<const uint4*>(q + o));
+                b = __ldg(reinterpret_cast<const uint4*>(dout + o));
+            }
+            qrows[i] = a;
+            dorows[i] = b;
+        }
+        __syncthreads();
+
+        // ---- count and fill: two sweeps over the (query, sample) pairs of the tile
+        for (int sweep = 0; sweep < 2; ++sweep) {
+            for (int pair = tid; pair < TQ * pr.P; pair += kTileThreads) {
+                const int ql = pair / pr.P, p = pair - ql * pr.P;
+                const int lx = ql % pr.tile_x, ly = (ql / pr.tile_x) % pr.tile_y, lt = ql / (pr.tile_x * pr.tile_y);
+                const int t = t0 + lt, y = y0 + ly, x = x0 + lx;
+                if (t >= pr.T || y >= pr.H || x >= pr.W) continue;
+                const long long n = (static_cast<long long>(t) * pr.H + y) * pr.W + x;
+                const long long row = n * pr.heads + m;
+                const Cell cell = make_cell(pr, t, y, x, p, offsets + (row * pr.P + p) * 3);
+                const unsigned mask = cell.mask & corner_mask(cell.it - lo_t, cell.iy - lo_y, cell.ix - lo_x, et, ey, ex);
+                if (mask == 0u) continue;
+                const float wt[2] = {1.0f - cell.ft, cell.ft}, wy[2] = {1.0f - cell.fy, cell.fy},
+                            wx[2] = {1.0f - cell.fx, cell.fx};
+                const int bin0 = ((cell.it - lo_t) * ey + (cell.iy - lo_y)) * ex + (cell.ix - lo_x);
+                float2 cf = make_float2(0.f, 0.f);
+                if (sweep == 1) cf = __ldg(coef + row * pr.P + p);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const float w = wt[c >> 2] * wy[(c >> 1) & 1] * wx[c & 1];
+                    if (((mask >> c) & 1u) && w != 0.0f) {
+                        const int bin = bin0 + ((c >> 2) * ey + ((c >> 1) & 1)) * ex + (c & 1);
+                        if (sweep == 0) {
+                            atomicAdd(&cursor[bin], 1u);
+                        } else {
+                            const unsigned slot = atomicAdd(&cursor[bin], 1u);
+                            const __nv_bfloat162 pk = __floats2bfloat162_rn(w * cf.x, w * cf.y);   // (wk, wv)
+                            my_scratch[slot] = make_uint2(static_cast<unsigned>(ql),
+                                                          *reinterpret_cast<const unsigned*>(&pk));
+                        }
+                    }
+                }
+            }
+            __syncthreads();
+            if (sweep == 0) {
+                // exclusive prefix sum of the NB counters, in place
+                const int per = (NB + kTileThreads - 1) / kTileThreads;
+                const int b0 = tid * per, b1 = min(NB, b0 + per);
+                unsigned local = 0;
+                for (int i = b0; i < b1; ++i) local += cursor[i];
+                unsigned incl = local;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const unsigned nb = __shfl_up_sync(0xffffffffu, incl, o);
+                    if ((tid & 31) >= o) incl += nb;
+                }
+                if ((tid & 31) == 31) warp_sums[tid >> 5] = incl;
+                __syncthreads();
+                if (tid < 32) {
+                    unsigned ws = tid < kTileThreads / 32 ? warp_sums[tid] : 0u;
+                    unsigned wi = ws;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const unsigned nb = __shfl_up_sync(0xffffffffu, wi, o);
+                        if (tid >= o) wi += nb;
+                    }
+                    if (tid < kTileThreads / 32) warp_sums[tid] = wi - ws;     // exclusive
+                }
+                __syncthreads();
+                unsigned run = warp_sums[tid >> 5] + incl - local;
+                for (int i = b0; i < b1; ++i) {
+                    const unsigned c = cursor[i];
+                    cursor[i] = run;
+                    run += c;
+                }
+                __syncthreads();
+            }
+        }
+        // after the fill sweep cursor[b] is the END of bin b; its start is the end of bin b-1
+
+        // ---- reduce: one half-warp per key row
+        {
+            const int lane = tid & 31, hl = lane & 15;
+            const unsigned hmask = 0xffffu << (lane & 16);
+            const int hw = tid >> 4, nhw = kTileThreads / 16;
+            for (int bin = hw; bin < NB; bin += nhw) {
+                const unsigned end = cursor[bin];
+                const unsigned start = bin == 0 ? 0u : cursor[bin - 1];
+                if (start == end) continue;
+                float ak[8], av[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) ak[e] = av[e] = 0.0f;
+                for (unsigned base = start; base < end; base += 16) {
+                    uint2 ent = make_uint2(0u, 0u);
+                    if (base + hl < end) ent = __ldcg(my_scratch + base + hl);
+                    const int cnt = min(16u, end - base);
+                    for (int j = 0; j < cnt; ++j) {
+                        const unsigned ql = __shfl_sync(hmask, ent.x, j, 16);
+                        const unsigned cw = __shfl_sync(hmask, ent.y, j, 16);
+                        unsigned short ck, cv;
+                        split_b32(cw, ck, cv);
+                        if constexpr (VPR == 16) {
+                            const uint4 a = qrows[ql * VPR + hl];
+                            const uint4 b = dorows[ql * VPR + hl];
+                            const unsigned aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                unsigned short lo, hi;
+                                split_b32(aw[i], lo, hi);
+                                ak[2 * i] = fma_bf16(ck, lo, ak[2 * i]);
+                                ak[2 * i + 1] = fma_bf16(ck, hi, ak[2 * i + 1]);
+                                split_b32(bw[i], lo, hi);
+                                av[2 * i] = fma_bf16(cv, lo, av[2 * i]);
+                                av[2 * i + 1] = fma_bf16(cv, hi, av[2 * i + 1]);
+                            }
+                        } else {
+                            // narrower rows: lanes beyond the row idle (hl >= VPR)
+                            if (hl < VPR) {
+                                const uint4 a = qrows[ql * VPR + hl];
+                                const uint4 b = dorows[ql * VPR + hl];
+                                const unsigned aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    unsigned short lo, hi;
+                                    split_b32(aw[i], lo, hi);
+                                    ak[2 * i] = fma_bf16(ck, lo, ak[2 * i]);
+                                    ak[2 * i + 1] = fma_bf16(ck, hi, ak[2 * i + 1]);
+                                    split_b32(bw[i], lo, hi);
+                                    av[2 * i] = fma_bf16(cv, lo, av[2 * i]);
+                                    av[2 * i + 1] = fma_bf16(cv, hi, av[2 * i + 1]);
+                                }
+                            }
+                        }
+                    }
+                }
+                if (hl < VPR) {
+                    const int bx = bin % ex, by = (bin / ex) % ey, bt = bin / (ex * ey);
+                    const long long tok = (static_cast<long long>(lo_t + bt) * pr.H + (lo_y + by)) * pr.W + (lo_x + bx);
+                    const long long o = tok * tok_stride + static_cast<long long>(m) * D + hl * 8;
+                    red_add_v4(acc_dk + o, ak[0], ak[1], ak[2], ak[3]);
+                    red_add_v4(acc_dk + o + 4, ak[4], ak[5], ak[6], ak[7]);
+                    red_add_v4(acc_dv + o, av[0], av[1], av[2], av[3]);
+                    red_add_v4(acc_dv + o + 4, av[4], av[5], av[6], av[7]);
+                }
+            }
+        }
+        __syncthreads();     // the next tile reuses the rows, the counters and the scratch
+    }
+}
+
+size_t tile_smem_bytes(const Problem& pr) {
+    const size_t TQ = static_cast<size_t>(pr.tile_t) * pr.tile_y * pr.tile_x;
+    const size_t NB = static_cast<size_t>(pr.tile_t + 2 * pr.halo) * (pr.tile_y + 2 * pr.halo) *
+                      (pr.tile_x + 2 * pr.halo);
+    return TQ * pr.d * 2 * 2 + NB * sizeof(unsigned);
+}
+
 template <typename T, int D>
 static cudaError_t launch_backward_t(const void* q, const void* k, const void* v, const float* offsets,
                                      const float* lse, const void* dout, void* dq, float* acc_dk,
-                                     float* acc_dv, float* doffsets, const Problem& pr,
+                                     float* acc_dv, float* doffsets, float2* coef, const Problem& pr,
                                      cudaStream_t stream) {
     constexpr int LPR = D / Elt<T>::VEC;
     // Shared memory holds 8 floats per (group, sample); shrink the block for large windows.
@@ -206,25 +458,54 @@ static cudaError_t launch_backward_t(const void* q, const void* k, const void* v
     const long long blocks = (pr.items + groups_per_block - 1) / groups_per_block;
     kern<<<static_cast<unsigned>(blocks), threads, smem, stream>>>(
         static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), offsets, lse,
-        static_cast<const T*>(dout), static_cast<T*>(dq), acc_dk, acc_dv, doffsets, pr);
+        static_cast<const T*>(dout), static_cast<T*>(dq), acc_dk, acc_dv, doffsets, coef, pr);
     return cudaGetLastError();
 }
 
 cudaError_t launch_backward(const void* q, const void* k, const void* v, const float* offsets,
                             const float* lse, const void* dout, void* dq, float* acc_dk, float* acc_dv,
-                            float* doffsets, const Problem& pr, bool bf16, cudaStream_t stream) {
+                            float* doffsets, float2* coef, const Problem& pr, bool bf16,
+                            cudaStream_t stream) {
 #define DSA3D_CASE(DD)                                                                                   \
     case DD:                                                                                             \
         return bf16 ? launch_backward_t<__nv_bfloat16, DD>(q, k, v, offsets, lse, dout, dq, acc_dk,     \
-                                                           acc_dv, doffsets, pr, stream)                 \
+                                                           acc_dv, doffsets, coef, pr, stream)           \
                     : launch_backward_t<float, DD>(q, k, v, offsets, lse, dout, dq, acc_dk, acc_dv,      \
-                                                   doffsets, pr, stream);
+                                                   doffsets, coef, pr, stream);
     switch (pr.d) {
         DSA3D_CASE(32)
         DSA3D_CASE(64)
         DSA3D_CASE(128)
     }
 #undef DSA3D_CASE
+    return cudaErrorInvalidValue;
+}
+
+template <int D>
+static cudaError_t launch_scatter_tiles_t(const void* q, const void* dout, const float* offsets,
+                                          const float2* coef, float* acc_dk, float* acc_dv, void* scratch,
+                                          int ctas, long long entries_per_cta, const Problem& pr,
+                                          cudaStream_t stream) {
+    auto kern = scatter_tile_kernel<D>;
+    const size_t smem = tile_smem_bytes(pr);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    const long long total_tiles = static_cast<long long>(pr.tiles_t) * pr.tiles_y * pr.tiles_x * pr.heads;
+    const int grid = static_cast<int>(total_tiles < ctas ? total_tiles : ctas);
+    kern<<<grid, kTileThreads, smem, stream>>>(
+        static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(dout), offsets, coef, acc_dk,
+        acc_dv, static_cast<uint2*>(scratch), entries_per_cta, pr);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_scatter_tiles(const void* q, const void* dout, const float* offsets, const float2* coef,
+                                 float* acc_dk, float* acc_dv, void* scratch, int ctas,
+                                 long long entries_per_cta, const Problem& pr, cudaStream_t stream) {
+    switch (pr.d) {
+        case 32: return launch_scatter_tiles_t<32>(q, dout, offsets, coef, acc_dk, acc_dv, scratch, ctas, entries_per_cta, pr, stream);
+        case 64: return launch_scatter_tiles_t<64>(q, dout, offsets, coef, acc_dk, acc_dv, scratch, ctas, entries_per_cta, pr, stream);
+        case 128: return launch_scatter_tiles_t<128>(q, dout, offsets, coef, acc_dk, acc_dv, scratch, ctas, entries_per_cta, pr, stream);
+    }
     return cudaErrorInvalidValue;
 }
 

@@ -14,33 +14,91 @@ struct Problem {
     int kt, kh, kw, P;
     long long N;       // T*H*W
     long long items;   // N*heads: one work item per (token, head)
+    // Query tiling of the backward scatter (tile_t < 1: no tiling, every dK/dV contribution
+    // goes straight to the global accumulators).  A corner is "in the halo" of a query when
+    // it lies within `halo` grid cells of the query's tile on every axis.
+    int tile_t, tile_y, tile_x, halo;
+    int tiles_t, tiles_y, tiles_x;
 };
 
 // ---------------------------------------------------------------------------------------
-// Element access.  A "vector" is 16 bytes: 8 bf16 or 4 fp32 channels.
+// Element access.  A lane handles one 16-byte vector of a row: 8 bf16 or 4 fp32 channels.
+// `Row` keeps that vector in its storage form.  For bf16 the products use the sm_100
+// mixed-precision instruction fma.rn.f32.bf16 (bf16 x bf16 -> exact fp32 product, fp32
+// accumulate), which needs no unpacking; `axpy` rounds its fp32 coefficient to bf16 first.
 // ---------------------------------------------------------------------------------------
 template <typename T> struct Elt;
 
 template <> struct Elt<float> {
     static constexpr int VEC = 4;
-    static __device__ __forceinline__ void load(const float* p, float (&x)[4]) {
+    struct Row { float v[4]; };
+    static __device__ __forceinline__ Row load(const float* p) {
         const float4 r = __ldg(reinterpret_cast<const float4*>(p));
-        x[0] = r.x; x[1] = r.y; x[2] = r.z; x[3] = r.w;
+        return Row{{r.x, r.y, r.z, r.w}};
+    }
+    static __device__ __forceinline__ Row zero() { return Row{{0.f, 0.f, 0.f, 0.f}}; }
+    static __device__ __forceinline__ float dot(const Row& a, const Row& b, float acc) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc = fmaf(a.v[e], b.v[e], acc);
+        return acc;
+    }
+    static __device__ __forceinline__ void axpy(float c, const Row& x, float (&acc)[4]) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[e] = fmaf(c, x.v[e], acc[e]);
+    }
+    static __device__ __forceinline__ void to_float(const Row& x, float (&f)[4]) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) f[e] = x.v[e];
     }
     static __device__ __forceinline__ void store(float* p, const float (&x)[4]) {
         *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
     }
 };
 
+__device__ __forceinline__ float fma_bf16(unsigned short a, unsigned short b, float c) {
+    float d;
+    asm("fma.rn.f32.bf16 %0, %1, %2, %3;" : "=f"(d) : "h"(a), "h"(b), "f"(c));
+    return d;
+}
+
+__device__ __forceinline__ void split_b32(uint32_t r, unsigned short& lo, unsigned short& hi) {
+    asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(r));
+}
+
 template <> struct Elt<__nv_bfloat16> {
     static constexpr int VEC = 8;
-    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&x)[8]) {
+    struct Row { uint32_t w[4]; };
+    static __device__ __forceinline__ Row load(const __nv_bfloat16* p) {
         const uint4 r = __ldg(reinterpret_cast<const uint4*>(p));
-        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+        return Row{{r.x, r.y, r.z, r.w}};
+    }
+    static __device__ __forceinline__ Row zero() { return Row{{0u, 0u, 0u, 0u}}; }
+    static __device__ __forceinline__ float dot(const Row& a, const Row& b, float acc) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            unsigned short al, ah, bl, bh;
+            split_b32(a.w[i], al, ah);
+            split_b32(b.w[i], bl, bh);
+            acc = fma_bf16(al, bl, acc);
+            acc = fma_bf16(ah, bh, acc);
+        }
+        return acc;
+    }
+    static __device__ __forceinline__ void axpy(float c, const Row& x, float (&acc)[8]) {
+        const unsigned short cb = __bfloat16_as_ushort(__float2bfloat16_rn(c));
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            unsigned short xl, xh;
+            split_b32(x.w[i], xl, xh);
+            acc[2 * i] = fma_bf16(cb, xl, acc[2 * i]);
+            acc[2 * i + 1] = fma_bf16(cb, xh, acc[2 * i + 1]);
+        }
+    }
+    static __device__ __forceinline__ void to_float(const Row& x, float (&f)[8]) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {           // bf16 is the upper half of an fp32
-            x[2 * i] = __uint_as_float(w[i] << 16);
-            x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+            f[2 * i] = __uint_as_float(x.w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(x.w[i] & 0xffff0000u);
         }
     }
     static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&x)[8]) {
@@ -55,56 +113,87 @@ template <> struct Elt<__nv_bfloat16> {
 };
 
 // ---------------------------------------------------------------------------------------
-// Sample geometry.  `base` is the token index of corner (0,0,0) (it may be "virtual",
-// i.e. have a component of -1; only corners flagged in `mask` are ever dereferenced),
-// bit c = ct*4 + cy*2 + cx of `mask` says corner c lies inside the grid, f* are the
-// fractional parts.  A sample with a NaN position or one at < -1 or >= size on any axis
-// has mask 0.  The position is float(coord + b) + offset with one fp32 rounding, then
-// floorf, then the fp32 difference: the same sequence on every path so that the integer
-// cell decision never depends on who computes it.
+// Sample geometry.  (it, iy, ix) is corner (0,0,0) of the cell (a component may be -1;
+// only corners flagged in `mask` are ever dereferenced), bit c = ct*4 + cy*2 + cx of
+// `mask` says corner c lies inside the grid, f* are the fractional parts.  A sample with a
+// NaN position or one at < -1 or >= size on any axis has mask 0.  The position is
+// float(coord + b) + offset with one fp32 rounding, then floorf, then the fp32 difference:
+// the same sequence on every path so that the integer cell decision never depends on who
+// computes it.
 // ---------------------------------------------------------------------------------------
+struct Cell {
+    int it, iy, ix;
+    unsigned mask;
+    float ft, fy, fx;
+};
+
+// What a lane needs to process a sample somebody else located: linear index of corner
+// (0,0,0), corner mask, fractional parts.
 struct Sample {
     int base;
     unsigned mask;
     float ft, fy, fx;
 };
 
-__device__ __forceinline__ bool axis_cell(int coord_plus_b, float off, int size, int& i0, float& f,
-                                          unsigned& lo_ok, unsigned& hi_ok) {
+__device__ __forceinline__ bool axis_cell(int coord_plus_b, float off, int size, int& i0, float& f) {
     const float pi = __fadd_rn(static_cast<float>(coord_plus_b), off);
     if (!(pi >= -1.0f) || !(pi < static_cast<float>(size))) return false;
     const float fl = floorf(pi);
     i0 = static_cast<int>(fl);
     f = __fsub_rn(pi, fl);
-    lo_ok = i0 >= 0;
-    hi_ok = i0 + 1 <= size - 1;
     return true;
 }
 
-__device__ __forceinline__ Sample make_sample(const Problem& pr, int t, int y, int x, int p,
-                                              const float* __restrict__ off3) {
+// Bit c of the result is set when corner c = (ct, cy, cx) has lo <= i0 + c < hi on every axis,
+// where the test per axis is written as an unsigned range check on (i0 - lo).
+__device__ __forceinline__ unsigned corner_mask(int rt, int ry, int rx, int et, int ey, int ex) {
+    const unsigned t0 = static_cast<unsigned>(rt) < static_cast<unsigned>(et);
+    const unsigned t1 = static_cast<unsigned>(rt + 1) < static_cast<unsigned>(et);
+    const unsigned y0 = static_cast<unsigned>(ry) < static_cast<unsigned>(ey);
+    const unsigned y1 = static_cast<unsigned>(ry + 1) < static_cast<unsigned>(ey);
+    const unsigned x0 = static_cast<unsigned>(rx) < static_cast<unsigned>(ex);
+    const unsigned x1 = static_cast<unsigned>(rx + 1) < static_cast<unsigned>(ex);
+    const unsigned yx = (y0 & x0) | ((y0 & x1) << 1) | ((y1 & x0) << 2) | ((y1 & x1) << 3);
+    return (t0 ? yx : 0u) | (t1 ? (yx << 4) : 0u);
+}
+
+__device__ __forceinline__ Cell make_cell(const Problem& pr, int t, int y, int x, int p,
+                                          const float* __restrict__ off3) {
     const int w = p % pr.kw;
     const int v = (p / pr.kw) % pr.kh;
     const int u = p / (pr.kw * pr.kh);
-    Sample s;
-    s.base = 0; s.mask = 0u; s.ft = s.fy = s.fx = 0.0f;
+    Cell c;
+    c.it = c.iy = c.ix = 0;
+    c.mask = 0u;
+    c.ft = c.fy = c.fx = 0.0f;
     int it, iy, ix;
-    unsigned t0, t1, y0, y1, x0, x1;
     float ft, fy, fx;
     const float ot = __ldg(off3), oy = __ldg(off3 + 1), ox = __ldg(off3 + 2);
-    if (!axis_cell(t + u - pr.kt / 2, ot, pr.T, it, ft, t0, t1)) return s;
-    if (!axis_cell(y + v - pr.kh / 2, oy, pr.H, iy, fy, y0, y1)) return s;
-    if (!axis_cell(x + w - pr.kw / 2, ox, pr.W, ix, fx, x0, x1)) return s;
-    s.base = (it * pr.H + iy) * pr.W + ix;
-    s.ft = ft; s.fy = fy; s.fx = fx;
-    unsigned m = 0;
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        const unsigned ok = ((c & 4) ? t1 : t0) & ((c & 2) ? y1 : y0) & ((c & 1) ? x1 : x0);
-        m |= ok << c;
-    }
-    s.mask = m;
+    if (!axis_cell(t + u - pr.kt / 2, ot, pr.T, it, ft)) return c;
+    if (!axis_cell(y + v - pr.kh / 2, oy, pr.H, iy, fy)) return c;
+    if (!axis_cell(x + w - pr.kw / 2, ox, pr.W, ix, fx)) return c;
+    c.it = it; c.iy = iy; c.ix = ix;
+    c.ft = ft; c.fy = fy; c.fx = fx;
+    c.mask = corner_mask(it, iy, ix, pr.T, pr.H, pr.W);
+    return c;
+}
+
+__device__ __forceinline__ Sample to_sample(const Problem& pr, const Cell& c) {
+    Sample s;
+    s.base = (c.it * pr.H + c.iy) * pr.W + c.ix;
+    s.mask = c.mask;
+    s.ft = c.ft; s.fy = c.fy; s.fx = c.fx;
     return s;
+}
+
+// Corners of `c` that lie in the halo box of the tile containing query (t, y, x).
+__device__ __forceinline__ unsigned halo_corner_mask(const Problem& pr, const Cell& c, int t, int y, int x) {
+    if (pr.tile_t < 1) return 0u;
+    const int lo_t = (t / pr.tile_t) * pr.tile_t - pr.halo;
+    const int lo_y = (y / pr.tile_y) * pr.tile_y - pr.halo;
+    const int lo_x = (x / pr.tile_x) * pr.tile_x - pr.halo;
+    return corner_mask(c.it - lo_t, c.iy - lo_y, c.ix - lo_x, pr.tile_t + 2 * pr.halo,
+                       pr.tile_y + 2 * pr.halo, pr.tile_x + 2 * pr.halo);
 }
 
 // Shuffles inside a group of LPR consecutive lanes (LPR a power of two <= 32).

@@ -7,6 +7,11 @@
 // L2.  Per sample: the 8 corner rows of K and of V are loaded with 16-byte loads, the
 // logit is the weighted sum of the corner dot products, and the output is accumulated with
 // an online softmax in fp32 registers; nothing of size N*P is written.
+//
+// A sample whose 8 corners are all inside the grid with non-zero weights (the usual case
+// for real-valued offsets) takes a branch-free path that issues its 16 row loads back to
+// back; border samples and samples on integer positions take a per-corner path that skips
+// corners outside the grid and corners of weight zero.
 #include "dsa3d_common.cuh"
 #include "dsa3d_kernels.h"
 
@@ -17,7 +22,9 @@ __global__ void __launch_bounds__(256)
 forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                const float* __restrict__ offsets, T* __restrict__ out, float* __restrict__ lse,
                const Problem pr) {
-    constexpr int VEC = Elt<T>::VEC;
+    using E = Elt<T>;
+    using Row = typename E::Row;
+    constexpr int VEC = E::VEC;
     constexpr int LPR = D / VEC;
     const int lane = threadIdx.x & 31;
     const int gl = lane & (LPR - 1);
@@ -30,20 +37,18 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
     const int x = static_cast<int>(n % pr.W);
     const int y = static_cast<int>((n / pr.W) % pr.H);
     const int t = static_cast<int>(n / (static_cast<long long>(pr.W) * pr.H));
-    const int HW = pr.H * pr.W;
     const long long row = (n * pr.heads + m);               // row index into [N*heads, ...]
     const int ch = gl * VEC;
+    const long long tok_stride = static_cast<long long>(pr.heads) * D;
+    const int sx = static_cast<int>(tok_stride);            // element stride between x neighbours
+    const int sy = pr.W * sx;
+    const int st = pr.H * sy;                                // < 2^31: checked by the host
 
-    float qf[VEC];
-    Elt<T>::load(q + row * D + ch, qf);
-    const float qscale = rsqrtf(static_cast<float>(D)) * kLog2e;   // logits in log2 units
-#pragma unroll
-    for (int j = 0; j < VEC; ++j) qf[j] *= qscale;
-
+    const Row qr = E::load(q + row * D + ch);
+    const float lscale = rsqrtf(static_cast<float>(D)) * kLog2e;    // logits in log2 units
     const float* off_row = offsets + row * pr.P * 3;
     const T* kh = k + static_cast<long long>(m) * D + ch;    // + tok * heads * D
     const T* vh = v + static_cast<long long>(m) * D + ch;
-    const long long tok_stride = static_cast<long long>(pr.heads) * D;
 
     float acc[VEC];
 #pragma unroll
@@ -53,46 +58,57 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
     for (int pb = 0; pb < pr.P; pb += LPR) {
         Sample mine;
         mine.base = 0; mine.mask = 0u; mine.ft = mine.fy = mine.fx = 0.0f;
-        if (pb + gl < pr.P) mine = make_sample(pr, t, y, x, pb + gl, off_row + (pb + gl) * 3);
+        if (pb + gl < pr.P) mine = to_sample(pr, make_cell(pr, t, y, x, pb + gl, off_row + (pb + gl) * 3));
         const int cnt = min(LPR, pr.P - pb);
         for (int j = 0; j < cnt; ++j) {
             const Sample s = group_bcast<LPR>(mine, j, gmask);
             const float wt[2] = {1.0f - s.ft, s.ft}, wy[2] = {1.0f - s.fy, s.fy}, wx[2] = {1.0f - s.fx, s.fx};
+            float w[8];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) w[c] = wt[c >> 2] * wy[(c >> 1) & 1] * wx[c & 1];
+            const T* kb = kh + s.base * tok_stride;
+            const T* vb = vh + s.base * tok_stride;
+            const bool full = s.mask == 0xffu && s.ft != 0.0f && s.fy != 0.0f && s.fx != 0.0f;
             float sdot = 0.0f;
-            float vp[VEC];
+            Row vv[8];
+            if (full) {
+                Row kk[8];
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) vp[e] = 0.0f;
+                for (int c = 0; c < 8; ++c) kk[c] = E::load(kb + ((c >> 2) * st + ((c >> 1) & 1) * sy + (c & 1) * sx));
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const float w = wt[c >> 2] * wy[(c >> 1) & 1] * wx[c & 1];
-                if (((s.mask >> c) & 1u) && w != 0.0f) {
-                    const int tok = s.base + (c >> 2) * HW + ((c >> 1) & 1) * pr.W + (c & 1);
-                    float kk[VEC], vv[VEC];
-                    Elt<T>::load(kh + tok * tok_stride, kk);
-                    Elt<T>::load(vh + tok * tok_stride, vv);
-                    float dot = 0.0f;
+                for (int c = 0; c < 8; ++c) vv[c] = E::load(vb + ((c >> 2) * st + ((c >> 1) & 1) * sy + (c & 1) * sx));
 #pragma unroll
-                    for (int e = 0; e < VEC; ++e) {
-                        dot = fmaf(qf[e], kk[e], dot);
-                        vp[e] = fmaf(w, vv[e], vp[e]);
+                for (int c = 0; c < 8; ++c) sdot = fmaf(w[c], E::dot(qr, kk[c], 0.0f), sdot);
+            } else {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    vv[c] = E::zero();
+                    if (((s.mask >> c) & 1u) && w[c] != 0.0f) {
+                        const int o = (c >> 2) * st + ((c >> 1) & 1) * sy + (c & 1) * sx;
+                        const Row kk = E::load(kb + o);
+                        vv[c] = E::load(vb + o);
+                        sdot = fmaf(w[c], E::dot(qr, kk, 0.0f), sdot);
+                    } else {
+                        w[c] = 0.0f;
                     }
-                    sdot = fmaf(w, dot, sdot);
                 }
             }
-            const float sp = group_sum<LPR>(sdot, gmask);
+            const float sp = group_sum<LPR>(sdot, gmask) * lscale;
             const float m_new = fmaxf(m_run, sp);
             const float corr = exp2f(m_run - m_new);
             const float pe = exp2f(sp - m_new);
             l_run = fmaf(l_run, corr, pe);
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) acc[e] = fmaf(pe, vp[e], acc[e] * corr);
             m_run = m_new;
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) acc[e] *= corr;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) E::axpy(pe * w[c], vv[c], acc);
         }
     }
     const float inv = 1.0f / l_run;
 #pragma unroll
     for (int e = 0; e < VEC; ++e) acc[e] *= inv;
-    Elt<T>::store(out + row * D + ch, acc);
+    E::store(out + row * D + ch, acc);
     if (gl == 0) lse[row] = (m_run + log2f(l_run)) * kLn2;
 }
 

@@ -1,6 +1,7 @@
 // Internal launch interface between the C-ABI layer and the kernels.
 #pragma once
 #include <cuda_runtime.h>
+#include <stddef.h>
 
 #include "dsa3d_common.cuh"
 
@@ -10,12 +11,31 @@ cudaError_t launch_forward(const void* q, const void* k, const void* v, const fl
                            float* lse, const Problem& pr, bool bf16, cudaStream_t stream);
 
 // acc_dk / acc_dv: fp32 accumulators [N, heads, d], zeroed by the caller.  For fp32 storage
-// they are the dk / dv outputs themselves.
+// they are the dk / dv outputs themselves.  coef [N*heads, P] receives the two scatter
+// coefficients of every sample when the problem is tiled (pr.tile_t >= 1), else it may be
+// NULL.  Corners inside the halo of their query's tile are left to launch_scatter_tiles.
 cudaError_t launch_backward(const void* q, const void* k, const void* v, const float* offsets,
                             const float* lse, const void* dout, void* dq, float* acc_dk, float* acc_dv,
-                            float* doffsets, const Problem& pr, bool bf16, cudaStream_t stream);
+                            float* doffsets, float2* coef, const Problem& pr, bool bf16, cudaStream_t stream);
+
+// bf16 storage only: the in-halo part of the dK/dV scatter, pre-reduced per query tile.
+// `scratch` holds `ctas` regions of `entries_per_cta` 8-byte entries.
+cudaError_t launch_scatter_tiles(const void* q, const void* dout, const float* offsets, const float2* coef,
+                                 float* acc_dk, float* acc_dv, void* scratch, int ctas,
+                                 long long entries_per_cta, const Problem& pr, cudaStream_t stream);
+
+// Dynamic shared memory of the tile kernel for this problem's tiling.
+size_t tile_smem_bytes(const Problem& pr);
 
 // fp32 accumulators -> bf16 outputs (round to nearest even).
 cudaError_t launch_convert_bf16(const float* acc, void* dst, long long count, cudaStream_t stream);
+
+// Shared implementation of dsa3d_backward.  `tiled` selects the tile pre-reduction of the
+// dK/dV scatter (bf16 only; needs the large workspace); without it the workspace is just the
+// two fp32 accumulators.  Returns a dsa3d_status.
+int backward_impl(const void* q, const void* k, const void* v, const float* offsets, const float* lse,
+                  const void* dout, int T, int H, int W, int heads, int d, const int window[3], void* dq,
+                  void* dk, void* dv, float* doffsets, void* workspace, size_t workspace_bytes, int dtype,
+                  void* stream, bool tiled);
 
 }  // namespace dsa3d

@@ -72,15 +72,16 @@ int dsa3d_backward_noalloc(const void* q, const void* k, const void* v, const fl
         if (elements > kMaxElements) return DSA3D_ERR_WORKSPACE;
     }
     if (dtype == DSA3D_F32)   // fp32 storage accumulates straight into dk / dv: no scratch at all
-        return dsa3d_backward(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets,
-                              nullptr, 0, dtype, stream);
+        return dsa3d::backward_impl(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv,
+                                    doffsets, nullptr, 0, dtype, stream, false);
     float* scratch = nullptr;
     const int rc = scratch_for_current_device(&scratch);
     if (rc != DSA3D_OK) return rc;
-    // dsa3d_backward validates the rest, clears the accumulators (the array keeps whatever
-    // the previous call left) and runs the same kernels as the workspace variant.
-    return dsa3d_backward(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets,
-                          scratch, 2 * kMaxElements * sizeof(float), dtype, stream);
+    // The shared implementation validates the rest, clears the accumulators (the array keeps
+    // whatever the previous call left) and scatters every dK/dV contribution straight into
+    // them: the tile pre-reduction of dsa3d_backward needs far more scratch than this array.
+    return dsa3d::backward_impl(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets,
+                                scratch, 2 * kMaxElements * sizeof(float), dtype, stream, false);
 }
 
 }  // extern "C"
