@@ -31,7 +31,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     """Build libdsa3d.so if it is missing or older than its sources; return its path."""
     if not force and not _stale():
         return LIB
-    flags = list(NVCC_FLAGS)
+    flags = list(NVCC_FLAGS) + os.environ.get("DSA3D_NVCC_EXTRA", "").split()
     if verbose:
         flags += ["-Xptxas", "-v"]
     cmd = [_nvcc(), "-shared", "-o", LIB] + flags + [os.path.join(CSRC, s) for s in SOURCES]

@@ -39,8 +39,12 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
 
 constexpr int kStats = 8;   // per sample: alpha, g, A_t, A_y, A_x, B_t, B_y, B_x
 
+#ifndef DSA3D_BWD_MINBLOCKS
+#define DSA3D_BWD_MINBLOCKS 3
+#endif
+
 template <typename T, int D>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, DSA3D_BWD_MINBLOCKS)
 backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                 const float* __restrict__ offsets, const float* __restrict__ lse,
                 const T* __restrict__ dout, T* __restrict__ dq, float* __restrict__ acc_dk,
@@ -95,9 +99,13 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
             const float wt[2] = {1.0f - s.ft, s.ft}, wy[2] = {1.0f - s.fy, s.fy}, wx[2] = {1.0f - s.fx, s.fx};
             const T* kb = kh + s.base * tok_stride;
             const T* vb = vh + s.base * tok_stride;
-            float r[kStats];
+            float w[8];
+            {
+                const float wty[4] = {wt[0] * wy[0], wt[0] * wy[1], wt[1] * wy[0], wt[1] * wy[1]};
 #pragma unroll
-            for (int i = 0; i < kStats; ++i) r[i] = 0.0f;
+                for (int c = 0; c < 8; ++c) w[c] = wty[c >> 1] * wx[c & 1];
+            }
+            float a[8], b[8];            // lane partials of q.K_c and dO.V_c (0 for corners not loaded)
             float kp[VEC];
 #pragma unroll
             for (int e = 0; e < VEC; ++e) kp[e] = 0.0f;
@@ -110,54 +118,44 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
                 for (int c = 0; c < 8; ++c) vv[c] = E::load(vb + ((c >> 2) * st + ((c >> 1) & 1) * sy + (c & 1) * sx));
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
-                    const int ct = c >> 2, cy = (c >> 1) & 1, cx = c & 1;
-                    const float w = wt[ct] * wy[cy] * wx[cx];
-                    const float dwt = (ct ? 1.0f : -1.0f) * wy[cy] * wx[cx];
-                    const float dwy = (cy ? 1.0f : -1.0f) * wt[ct] * wx[cx];
-                    const float dwx = (cx ? 1.0f : -1.0f) * wt[ct] * wy[cy];
-                    const float a = E::dot(qr, kk[c], 0.0f);
-                    const float b = E::dot(dor, vv[c], 0.0f);
-                    E::axpy(w, kk[c], kp);
-                    r[0] = fmaf(w, a, r[0]);
-                    r[1] = fmaf(w, b, r[1]);
-                    r[2] = fmaf(dwt, a, r[2]);
-                    r[3] = fmaf(dwy, a, r[3]);
-                    r[4] = fmaf(dwx, a, r[4]);
-                    r[5] = fmaf(dwt, b, r[5]);
-                    r[6] = fmaf(dwy, b, r[6]);
-                    r[7] = fmaf(dwx, b, r[7]);
+                    a[c] = E::dot(qr, kk[c], 0.0f);
+                    b[c] = E::dot(dor, vv[c], 0.0f);
+                    E::axpy(w[c], kk[c], kp);
                 }
             } else {
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
                     const int ct = c >> 2, cy = (c >> 1) & 1, cx = c & 1;
-                    const float w = wt[ct] * wy[cy] * wx[cx];
-                    const float dwt = (ct ? 1.0f : -1.0f) * wy[cy] * wx[cx];
-                    const float dwy = (cy ? 1.0f : -1.0f) * wt[ct] * wx[cx];
-                    const float dwx = (cx ? 1.0f : -1.0f) * wt[ct] * wy[cy];
-                    const bool needed = (w != 0.0f) | (dwt != 0.0f) | (dwy != 0.0f) | (dwx != 0.0f);
+                    // a corner matters if its weight or one of its weight derivatives is non-zero
+                    const bool needed = (w[c] != 0.0f) | (wy[cy] * wx[cx] != 0.0f) | (wt[ct] * wx[cx] != 0.0f) |
+                                        (wt[ct] * wy[cy] != 0.0f);
+                    a[c] = b[c] = 0.0f;
                     if (((s.mask >> c) & 1u) && needed) {
                         const int o = ct * st + cy * sy + cx * sx;
                         const Row kk = E::load(kb + o);
                         const Row vv = E::load(vb + o);
-                        const float a = E::dot(qr, kk, 0.0f);
-                        const float b = E::dot(dor, vv, 0.0f);
-                        E::axpy(w, kk, kp);
-                        r[0] = fmaf(w, a, r[0]);
-                        r[1] = fmaf(w, b, r[1]);
-                        r[2] = fmaf(dwt, a, r[2]);
-                        r[3] = fmaf(dwy, a, r[3]);
-                        r[4] = fmaf(dwx, a, r[4]);
-                        r[5] = fmaf(dwt, b, r[5]);
-                        r[6] = fmaf(dwy, b, r[6]);
-                        r[7] = fmaf(dwx, b, r[7]);
+                        a[c] = E::dot(qr, kk, 0.0f);
+                        b[c] = E::dot(dor, vv, 0.0f);
+                        E::axpy(w[c], kk, kp);
                     }
                 }
             }
+            // r = (s, g, A_t, A_y, A_x, B_t, B_y, B_x) as lane partials, then summed over the group
+            float r[kStats];
+            trilerp_grad(a, s.ft, s.fy, s.fx, r[0], r[2], r[3], r[4]);
+            trilerp_grad(b, s.ft, s.fy, s.fx, r[1], r[5], r[6], r[7]);
+            float sdot, g;
+            if constexpr (LPR >= 8) {
+                group_reduce8<LPR>(r, gl, gmask);
+                sdot = __shfl_sync(gmask, r[0], reduce8_lane<LPR>(0), LPR);
+                g = __shfl_sync(gmask, r[0], reduce8_lane<LPR>(1), LPR);
+            } else {
 #pragma unroll
-            for (int i = 0; i < kStats; ++i) r[i] = group_sum<LPR>(r[i], gmask);
-            const float alpha = exp2f(fmaf(r[0], scale * kLog2e, -lse2));
-            const float g = r[1];
+                for (int i = 0; i < kStats; ++i) r[i] = group_sum<LPR>(r[i], gmask);
+                sdot = r[0];
+                g = r[1];
+            }
+            const float alpha = exp2f(fmaf(sdot, scale * kLog2e, -lse2));
             const float ag = alpha * g;
             delta += ag;
 #pragma unroll
@@ -165,11 +163,14 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
                 u_acc[e] = fmaf(ag, kp[e], u_acc[e]);
                 kbar[e] = fmaf(alpha, kp[e], kbar[e]);
             }
-            if (gl == 0) {
-                float* sts = stats + (pb + j) * kStats;
+            float* sts = stats + (pb + j) * kStats;
+            if constexpr (LPR >= 8) {
+                const int idx = reduce8_index<LPR>(gl);
+                if (gl == reduce8_lane<LPR>(idx)) sts[idx] = idx == 0 ? alpha : r[0];   // slot 1 keeps g
+            } else if (gl == 0) {
                 sts[0] = alpha; sts[1] = g;
-                sts[2] = r[2]; sts[3] = r[3]; sts[4] = r[4];
-                sts[5] = r[5]; sts[6] = r[6]; sts[7] = r[7];
+#pragma unroll
+                for (int i = 2; i < kStats; ++i) sts[i] = r[i];
             }
         }
     }
@@ -237,7 +238,10 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
 // ---------------------------------------------------------------------------------------
 // Tile scatter (bf16 storage).
 // ---------------------------------------------------------------------------------------
-constexpr int kTileThreads = 512;
+#ifndef DSA3D_TILE_THREADS
+#define DSA3D_TILE_THREADS 1024
+#endif
+constexpr int kTileThreads = DSA3D_TILE_THREADS;
 
 template <int D>
 __global__ void __launch_bounds__(kTileThreads, 1)

@@ -211,6 +211,61 @@ template <int LPR> __device__ __forceinline__ float group_sum(float v, unsigned 
     return v;
 }
 
+// Sum 8 per-lane numbers over the group so that every sum ends up on some lane, with a
+// quarter of the shuffles a butterfly per value would take: at each of the first three
+// xor distances a lane hands half of its values to its partner and keeps the other half.
+// On return v[0] of lane gl holds the complete sum number reduce8_index<LPR>(gl).
+// (LPR >= 8; narrower groups use group_sum.)
+template <int LPR> __device__ __forceinline__ int reduce8_index(int gl) {
+    return (((gl / (LPR / 2)) & 1) << 2) | (((gl / (LPR / 4)) & 1) << 1) | ((gl / (LPR / 8)) & 1);
+}
+template <int LPR> __device__ __forceinline__ int reduce8_lane(int index) {     // a lane holding sum `index`
+    return ((index >> 2) & 1) * (LPR / 2) + ((index >> 1) & 1) * (LPR / 4) + (index & 1) * (LPR / 8);
+}
+template <int LPR> __device__ __forceinline__ void group_reduce8(float (&v)[8], int gl, unsigned gmask) {
+    static_assert(LPR >= 8, "needs three halving steps");
+    int n = 8;
+#pragma unroll
+    for (int d = LPR / 2; d >= LPR / 8; d >>= 1) {
+        const bool upper = (gl & d) != 0;
+        n >>= 1;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (i < n) {
+                const float send = upper ? v[i] : v[i + n];
+                const float keep = upper ? v[i + n] : v[i];
+                v[i] = keep + __shfl_xor_sync(gmask, send, d, LPR);
+            }
+        }
+    }
+#pragma unroll
+    for (int d = LPR / 16; d > 0; d >>= 1) v[0] += __shfl_xor_sync(gmask, v[0], d, LPR);
+}
+
+// Value and the three partial derivatives (along t, y, x) of the trilinear interpolant of
+// eight corner numbers a[c], c = ct*4 + cy*2 + cx, at fractional position (ft, fy, fx):
+// value = sum_c w_c a_c, d/da = sum_c (dw_c/da) a_c.  Corners outside the grid enter as 0.
+__device__ __forceinline__ void trilerp_grad(const float (&a)[8], float ft, float fy, float fx, float& val,
+                                             float& dt, float& dy, float& dx) {
+    float L[4], X[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        X[i] = a[2 * i + 1] - a[2 * i];
+        L[i] = fmaf(fx, X[i], a[2 * i]);
+    }
+    float M[2], Y[2], Xy[2];
+#pragma unroll
+    for (int ct = 0; ct < 2; ++ct) {
+        Y[ct] = L[2 * ct + 1] - L[2 * ct];
+        M[ct] = fmaf(fy, Y[ct], L[2 * ct]);
+        Xy[ct] = fmaf(fy, X[2 * ct + 1] - X[2 * ct], X[2 * ct]);
+    }
+    dt = M[1] - M[0];
+    val = fmaf(ft, dt, M[0]);
+    dy = fmaf(ft, Y[1] - Y[0], Y[0]);
+    dx = fmaf(ft, Xy[1] - Xy[0], Xy[0]);
+}
+
 template <int LPR> __device__ __forceinline__ Sample group_bcast(const Sample& s, int src, unsigned gmask) {
     Sample r;
     r.base = __shfl_sync(gmask, s.base, src, LPR);

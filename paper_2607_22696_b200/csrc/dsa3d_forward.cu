@@ -17,8 +17,12 @@
 
 namespace dsa3d {
 
+#ifndef DSA3D_FWD_MINBLOCKS
+#define DSA3D_FWD_MINBLOCKS 3
+#endif
+
 template <typename T, int D>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, DSA3D_FWD_MINBLOCKS)
 forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                const float* __restrict__ offsets, T* __restrict__ out, float* __restrict__ lse,
                const Problem pr) {
