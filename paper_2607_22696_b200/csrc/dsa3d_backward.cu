@@ -57,9 +57,12 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
     extern __shared__ float smem[];
     const int lane = threadIdx.x & 31;
     const int gl = lane & (LPR - 1);
-    const unsigned gmask = group_mask<LPR>(lane);
-    const long long item = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) / LPR;
-    if (item >= pr.items) return;
+    constexpr unsigned gmask = kFullMask;
+    long long item = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) / LPR;
+    const long long warp_first = (static_cast<long long>(blockIdx.x) * blockDim.x + (threadIdx.x & ~31)) / LPR;
+    if (warp_first >= pr.items) return;                  // whole warp past the end
+    const bool active = item < pr.items;                 // a trailing group repeats the last item, stores off
+    if (!active) item = pr.items - 1;
     float* stats = smem + static_cast<size_t>(threadIdx.x / LPR) * pr.P * kStats;   // [P][8] of this group
 
     const int m = static_cast<int>(item / pr.N);
@@ -81,7 +84,7 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
     const float* off_row = offsets + row * pr.P * 3;
     const long long head_off = static_cast<long long>(m) * D + ch;
     const T* kh = k + head_off;
-    const T* vh = v + head_off;
+    const long long v_minus_k = v - k;                       // same layout: V row = K row + this
 
     float u_acc[VEC], kbar[VEC];
 #pragma unroll
@@ -97,8 +100,11 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
         for (int j = 0; j < cnt; ++j) {
             const Sample s = group_bcast<LPR>(mine, j, gmask);
             const float wt[2] = {1.0f - s.ft, s.ft}, wy[2] = {1.0f - s.fy, s.fy}, wx[2] = {1.0f - s.fx, s.fx};
-            const T* kb = kh + s.base * tok_stride;
-            const T* vb = vh + s.base * tok_stride;
+            const T* kp4[4];             // corner row pointers per (ct, cy); cx = 1 is one token further
+            kp4[0] = kh + s.base * tok_stride;
+            kp4[1] = kp4[0] + sy;
+            kp4[2] = kp4[0] + st;
+            kp4[3] = kp4[2] + sy;
             float w[8];
             {
                 const float wty[4] = {wt[0] * wy[0], wt[0] * wy[1], wt[1] * wy[0], wt[1] * wy[1]};
@@ -113,9 +119,9 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
             if (full) {                    // every corner inside the grid and needed: 16 loads back to back
                 Row kk[8], vv[8];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) kk[c] = E::load(kb + ((c >> 2) * st + ((c >> 1) & 1) * sy + (c & 1) * sx));
+                for (int c = 0; c < 8; ++c) kk[c] = E::load(kp4[c >> 1] + (c & 1) * sx);
 #pragma unroll
-                for (int c = 0; c < 8; ++c) vv[c] = E::load(vb + ((c >> 2) * st + ((c >> 1) & 1) * sy + (c & 1) * sx));
+                for (int c = 0; c < 8; ++c) vv[c] = E::load(kp4[c >> 1] + (c & 1) * sx + v_minus_k);
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
                     a[c] = E::dot(qr, kk[c], 0.0f);
@@ -131,9 +137,9 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
                                         (wt[ct] * wy[cy] != 0.0f);
                     a[c] = b[c] = 0.0f;
                     if (((s.mask >> c) & 1u) && needed) {
-                        const int o = ct * st + cy * sy + cx * sx;
-                        const Row kk = E::load(kb + o);
-                        const Row vv = E::load(vb + o);
+                        const T* pk = kp4[c >> 1] + cx * sx;
+                        const Row kk = E::load(pk);
+                        const Row vv = E::load(pk + v_minus_k);
                         a[c] = E::dot(qr, kk, 0.0f);
                         b[c] = E::dot(dor, vv, 0.0f);
                         E::axpy(w[c], kk, kp);
@@ -178,9 +184,9 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
         float dqv[VEC];
 #pragma unroll
         for (int e = 0; e < VEC; ++e) dqv[e] = scale * fmaf(-delta, kbar[e], u_acc[e]);
-        E::store(dq + row * D + ch, dqv);
+        if (active) E::store(dq + row * D + ch, dqv);
     }
-    __syncwarp(gmask);
+    __syncwarp();
 
     // ------------------------------------------- pass 2: dOffsets, coefficients, far scatter
     float qf[VEC], dof[VEC];
@@ -198,20 +204,23 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
             const Cell cell = make_cell(pr, t, y, x, p, off_row + p * 3);
             mine = to_sample(pr, cell);
             mine.mask = cell.mask & ~halo_corner_mask(pr, cell, t, y, x);   // corners the tile kernel does not take
+            if (!active) mine.mask = 0u;
             const float* sts = stats + p * kStats;
             const float alpha = sts[0];
             const float dS = alpha * (sts[1] - delta);
             my_ck = scale * dS;
             my_cv = alpha;
-            doff_row[p * 3 + 0] = fmaf(my_ck, sts[2], alpha * sts[5]);
-            doff_row[p * 3 + 1] = fmaf(my_ck, sts[3], alpha * sts[6]);
-            doff_row[p * 3 + 2] = fmaf(my_ck, sts[4], alpha * sts[7]);
-            if (coef) coef[row * pr.P + p] = make_float2(my_ck, my_cv);
+            if (active) {
+                doff_row[p * 3 + 0] = fmaf(my_ck, sts[2], alpha * sts[5]);
+                doff_row[p * 3 + 1] = fmaf(my_ck, sts[3], alpha * sts[6]);
+                doff_row[p * 3 + 2] = fmaf(my_ck, sts[4], alpha * sts[7]);
+                if (coef) coef[row * pr.P + p] = make_float2(my_ck, my_cv);
+            }
         }
         const int cnt = min(LPR, pr.P - pb);
         for (int j = 0; j < cnt; ++j) {
             const unsigned mask = __shfl_sync(gmask, mine.mask, j, LPR);
-            if (mask == 0u) continue;
+            if (!__any_sync(kFullMask, mask != 0u)) continue;      // warp-uniform: shuffles follow
             const Sample s = group_bcast<LPR>(mine, j, gmask);
             const float ck = __shfl_sync(gmask, my_ck, j, LPR);
             const float cv = __shfl_sync(gmask, my_cv, j, LPR);
@@ -249,19 +258,19 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                     const float* __restrict__ offsets, const float2* __restrict__ coef,
                     float* __restrict__ acc_dk, float* __restrict__ acc_dv, uint2* __restrict__ scratch,
                     const long long scratch_entries_per_cta, const Problem pr) {
-    using E = Elt<__nv_bfloat16>;
-    using Row = E::Row;
     constexpr int VPR = D / 8;                       // 16-byte vectors per row
+    constexpr int kPairBytes = 2 * VPR * 16;         // one query's q row followed by its dO row
+    constexpr unsigned kFull = 0xffffffffu;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int TQ = pr.tile_t * pr.tile_y * pr.tile_x;
     const int et = pr.tile_t + 2 * pr.halo, ey = pr.tile_y + 2 * pr.halo, ex = pr.tile_x + 2 * pr.halo;
     const int NB = et * ey * ex;
-    uint4* qrows = reinterpret_cast<uint4*>(smem_raw);                 // [TQ][VPR]
-    uint4* dorows = qrows + static_cast<size_t>(TQ) * VPR;              // [TQ][VPR]
-    unsigned* cursor = reinterpret_cast<unsigned*>(dorows + static_cast<size_t>(TQ) * VPR);   // [NB]
+    uint4* rows = reinterpret_cast<uint4*>(smem_raw);                                   // [TQ][2][VPR]
+    unsigned* cursor = reinterpret_cast<unsigned*>(smem_raw + static_cast<size_t>(TQ) * kPairBytes);   // [NB]
     __shared__ unsigned warp_sums[kTileThreads / 32];
 
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int kWarps = kTileThreads / 32;
     const int tiles_per_head = pr.tiles_t * pr.tiles_y * pr.tiles_x;
     const long long total_tiles = static_cast<long long>(tiles_per_head) * pr.heads;
     uint2* my_scratch = scratch + static_cast<long long>(blockIdx.x) * scratch_entries_per_cta;
@@ -289,40 +298,41 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                 a = __ldg(reinterpret_cast<const uint4*>(q + o));
                 b = __ldg(reinterpret_cast<const uint4*>(dout + o));
             }
-            qrows[i] = a;
-            dorows[i] = b;
+            rows[ql * 2 * VPR + vec] = a;
+            rows[ql * 2 * VPR + VPR + vec] = b;
         }
         __syncthreads();
 
-        // ---- count and fill: two sweeps over the (query, sample) pairs of the tile
+        // ---- count and fill: two sweeps over the (query, sample) pairs of the tile; a warp
+        //      takes one query at a time, its lanes the samples
         for (int sweep = 0; sweep < 2; ++sweep) {
-            for (int pair = tid; pair < TQ * pr.P; pair += kTileThreads) {
-                const int ql = pair / pr.P, p = pair - ql * pr.P;
+            for (int ql = warp; ql < TQ; ql += kWarps) {
                 const int lx = ql % pr.tile_x, ly = (ql / pr.tile_x) % pr.tile_y, lt = ql / (pr.tile_x * pr.tile_y);
                 const int t = t0 + lt, y = y0 + ly, x = x0 + lx;
                 if (t >= pr.T || y >= pr.H || x >= pr.W) continue;
                 const long long n = (static_cast<long long>(t) * pr.H + y) * pr.W + x;
                 const long long row = n * pr.heads + m;
-                const Cell cell = make_cell(pr, t, y, x, p, offsets + (row * pr.P + p) * 3);
-                const unsigned mask = cell.mask & corner_mask(cell.it - lo_t, cell.iy - lo_y, cell.ix - lo_x, et, ey, ex);
-                if (mask == 0u) continue;
-                const float wt[2] = {1.0f - cell.ft, cell.ft}, wy[2] = {1.0f - cell.fy, cell.fy},
-                            wx[2] = {1.0f - cell.fx, cell.fx};
-                const int bin0 = ((cell.it - lo_t) * ey + (cell.iy - lo_y)) * ex + (cell.ix - lo_x);
-                float2 cf = make_float2(0.f, 0.f);
-                if (sweep == 1) cf = __ldg(coef + row * pr.P + p);
+                for (int p = lane; p < pr.P; p += 32) {
+                    const Cell cell = make_cell(pr, t, y, x, p, offsets + (row * pr.P + p) * 3);
+                    const unsigned mask =
+                        cell.mask & corner_mask(cell.it - lo_t, cell.iy - lo_y, cell.ix - lo_x, et, ey, ex);
+                    if (mask == 0u) continue;
+                    const float wt[2] = {1.0f - cell.ft, cell.ft}, wy[2] = {1.0f - cell.fy, cell.fy},
+                                wx[2] = {1.0f - cell.fx, cell.fx};
+                    const int bin0 = ((cell.it - lo_t) * ey + (cell.iy - lo_y)) * ex + (cell.ix - lo_x);
+                    float2 cf = make_float2(0.f, 0.f);
+                    if (sweep == 1) cf = __ldg(coef + row * pr.P + p);
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const float w = wt[c >> 2] * wy[(c >> 1) & 1] * wx[c & 1];
-                    if (((mask >> c) & 1u) && w != 0.0f) {
-                        const int bin = bin0 + ((c >> 2) * ey + ((c >> 1) & 1)) * ex + (c & 1);
-                        if (sweep == 0) {
-                            atomicAdd(&cursor[bin], 1u);
-                        } else {
+                    for (int c = 0; c < 8; ++c) {
+                        const float w = wt[c >> 2] * wy[(c >> 1) & 1] * wx[c & 1];
+                        if (((mask >> c) & 1u) && w != 0.0f) {
+                            const int bin = bin0 + ((c >> 2) * ey + ((c >> 1) & 1)) * ex + (c & 1);
                             const unsigned slot = atomicAdd(&cursor[bin], 1u);
-                            const __nv_bfloat162 pk = __floats2bfloat162_rn(w * cf.x, w * cf.y);   // (wk, wv)
-                            my_scratch[slot] = make_uint2(static_cast<unsigned>(ql),
-                                                          *reinterpret_cast<const unsigned*>(&pk));
+                            if (sweep == 1) {
+                                const __nv_bfloat162 pk = __floats2bfloat162_rn(w * cf.x, w * cf.y);   // (wk, wv)
+                                my_scratch[slot] = make_uint2(static_cast<unsigned>(ql * kPairBytes),
+                                                              *reinterpret_cast<const unsigned*>(&pk));
+                            }
                         }
                     }
                 }
@@ -337,23 +347,23 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                 unsigned incl = local;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
-                    const unsigned nb = __shfl_up_sync(0xffffffffu, incl, o);
-                    if ((tid & 31) >= o) incl += nb;
+                    const unsigned nb = __shfl_up_sync(kFull, incl, o);
+                    if (lane >= o) incl += nb;
                 }
-                if ((tid & 31) == 31) warp_sums[tid >> 5] = incl;
+                if (lane == 31) warp_sums[warp] = incl;
                 __syncthreads();
                 if (tid < 32) {
-                    unsigned ws = tid < kTileThreads / 32 ? warp_sums[tid] : 0u;
+                    const unsigned ws = tid < kWarps ? warp_sums[tid] : 0u;
                     unsigned wi = ws;
 #pragma unroll
                     for (int o = 1; o < 32; o <<= 1) {
-                        const unsigned nb = __shfl_up_sync(0xffffffffu, wi, o);
+                        const unsigned nb = __shfl_up_sync(kFull, wi, o);
                         if (tid >= o) wi += nb;
                     }
-                    if (tid < kTileThreads / 32) warp_sums[tid] = wi - ws;     // exclusive
+                    if (tid < kWarps) warp_sums[tid] = wi - ws;     // exclusive
                 }
                 __syncthreads();
-                unsigned run = warp_sums[tid >> 5] + incl - local;
+                unsigned run = warp_sums[warp] + incl - local;
                 for (int i = b0; i < b1; ++i) {
                     const unsigned c = cursor[i];
                     cursor[i] = run;
@@ -364,62 +374,52 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         }
         // after the fill sweep cursor[b] is the END of bin b; its start is the end of bin b-1
 
-        // ---- reduce: one half-warp per key row
+        // ---- reduce: a warp takes two neighbouring key rows, one per half-warp; both halves
+        //      run the same number of steps (the shorter list is padded with zero entries)
         {
-            const int lane = tid & 31, hl = lane & 15;
-            const unsigned hmask = 0xffffu << (lane & 16);
-            const int hw = tid >> 4, nhw = kTileThreads / 16;
-            for (int bin = hw; bin < NB; bin += nhw) {
-                const unsigned end = cursor[bin];
-                const unsigned start = bin == 0 ? 0u : cursor[bin - 1];
-                if (start == end) continue;
+            const int half = lane >> 4, hl = lane & 15;
+            const int hv = hl < VPR ? hl : VPR - 1;         // lanes beyond a narrow row mirror its last vector
+            const unsigned char* my_rows = smem_raw + hv * 16;
+            for (int pairbin = warp * 2; pairbin < NB; pairbin += kWarps * 2) {
+                const int bin = pairbin + half;
+                unsigned start = 0u, end = 0u;
+                if (bin < NB) {
+                    end = cursor[bin];
+                    start = bin == 0 ? 0u : cursor[bin - 1];
+                }
+                const unsigned cnt_mine = end - start;
+                const unsigned cnt_max = max(cnt_mine, __shfl_xor_sync(kFull, cnt_mine, 16));
+                if (cnt_max == 0u) continue;
                 float ak[8], av[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) ak[e] = av[e] = 0.0f;
-                for (unsigned base = start; base < end; base += 16) {
-                    uint2 ent = make_uint2(0u, 0u);
-                    if (base + hl < end) ent = __ldcg(my_scratch + base + hl);
-                    const int cnt = min(16u, end - base);
-                    for (int j = 0; j < cnt; ++j) {
-                        const unsigned ql = __shfl_sync(hmask, ent.x, j, 16);
-                        const unsigned cw = __shfl_sync(hmask, ent.y, j, 16);
+                for (unsigned base = 0; base < cnt_max; base += 16) {
+                    uint2 ent = make_uint2(0u, 0u);                       // offset 0, coefficients 0
+                    if (base + hl < cnt_mine) ent = __ldcg(my_scratch + start + base + hl);
+                    const int steps = static_cast<int>(min(16u, cnt_max - base));
+#pragma unroll 4
+                    for (int j = 0; j < steps; ++j) {
+                        const int src = (lane & 16) | j;
+                        const unsigned off = __shfl_sync(kFull, ent.x, src);
+                        const unsigned cw = __shfl_sync(kFull, ent.y, src);
                         unsigned short ck, cv;
                         split_b32(cw, ck, cv);
-                        if constexpr (VPR == 16) {
-                            const uint4 a = qrows[ql * VPR + hl];
-                            const uint4 b = dorows[ql * VPR + hl];
-                            const unsigned aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+                        const uint4 a = *reinterpret_cast<const uint4*>(my_rows + off);
+                        const uint4 b = *reinterpret_cast<const uint4*>(my_rows + off + VPR * 16);
+                        const unsigned aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                unsigned short lo, hi;
-                                split_b32(aw[i], lo, hi);
-                                ak[2 * i] = fma_bf16(ck, lo, ak[2 * i]);
-                                ak[2 * i + 1] = fma_bf16(ck, hi, ak[2 * i + 1]);
-                                split_b32(bw[i], lo, hi);
-                                av[2 * i] = fma_bf16(cv, lo, av[2 * i]);
-                                av[2 * i + 1] = fma_bf16(cv, hi, av[2 * i + 1]);
-                            }
-                        } else {
-                            // narrower rows: lanes beyond the row idle (hl >= VPR)
-                            if (hl < VPR) {
-                                const uint4 a = qrows[ql * VPR + hl];
-                                const uint4 b = dorows[ql * VPR + hl];
-                                const unsigned aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-                                for (int i = 0; i < 4; ++i) {
-                                    unsigned short lo, hi;
-                                    split_b32(aw[i], lo, hi);
-                                    ak[2 * i] = fma_bf16(ck, lo, ak[2 * i]);
-                                    ak[2 * i + 1] = fma_bf16(ck, hi, ak[2 * i + 1]);
-                                    split_b32(bw[i], lo, hi);
-                                    av[2 * i] = fma_bf16(cv, lo, av[2 * i]);
-                                    av[2 * i + 1] = fma_bf16(cv, hi, av[2 * i + 1]);
-                                }
-                            }
+                        for (int i = 0; i < 4; ++i) {
+                            unsigned short lo, hi;
+                            split_b32(aw[i], lo, hi);
+                            ak[2 * i] = fma_bf16(ck, lo, ak[2 * i]);
+                            ak[2 * i + 1] = fma_bf16(ck, hi, ak[2 * i + 1]);
+                            split_b32(bw[i], lo, hi);
+                            av[2 * i] = fma_bf16(cv, lo, av[2 * i]);
+                            av[2 * i + 1] = fma_bf16(cv, hi, av[2 * i + 1]);
                         }
                     }
                 }
-                if (hl < VPR) {
+                if (cnt_mine > 0u && hl < VPR) {
                     const int bx = bin % ex, by = (bin / ex) % ey, bt = bin / (ex * ey);
                     const long long tok = (static_cast<long long>(lo_t + bt) * pr.H + (lo_y + by)) * pr.W + (lo_x + bx);
                     const long long o = tok * tok_stride + static_cast<long long>(m) * D + hl * 8;

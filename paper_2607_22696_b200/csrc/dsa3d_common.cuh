@@ -205,6 +205,11 @@ template <int LPR> __device__ __forceinline__ unsigned group_mask(int lane) {
     }
 }
 
+// All shuffles below name the full warp: the kernels keep every lane of a warp alive and
+// on the same control path at each shuffle (a group past the end of the problem repeats
+// the last item with its stores switched off), so no per-group mask is needed.
+constexpr unsigned kFullMask = 0xffffffffu;
+
 template <int LPR> __device__ __forceinline__ float group_sum(float v, unsigned gmask) {
 #pragma unroll
     for (int o = LPR / 2; o > 0; o >>= 1) v += __shfl_xor_sync(gmask, v, o, LPR);

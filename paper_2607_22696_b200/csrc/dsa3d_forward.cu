@@ -32,9 +32,12 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
     constexpr int LPR = D / VEC;
     const int lane = threadIdx.x & 31;
     const int gl = lane & (LPR - 1);
-    const unsigned gmask = group_mask<LPR>(lane);
-    const long long item = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) / LPR;
-    if (item >= pr.items) return;
+    constexpr unsigned gmask = kFullMask;
+    long long item = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) / LPR;
+    const long long warp_first = (static_cast<long long>(blockIdx.x) * blockDim.x + (threadIdx.x & ~31)) / LPR;
+    if (warp_first >= pr.items) return;                  // whole warp past the end
+    const bool active = item < pr.items;                 // a trailing group repeats the last item, stores off
+    if (!active) item = pr.items - 1;
 
     const int m = static_cast<int>(item / pr.N);
     const long long n = item - static_cast<long long>(m) * pr.N;
@@ -52,7 +55,7 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
     const float lscale = rsqrtf(static_cast<float>(D)) * kLog2e;    // logits in log2 units
     const float* off_row = offsets + row * pr.P * 3;
     const T* kh = k + static_cast<long long>(m) * D + ch;    // + tok * heads * D
-    const T* vh = v + static_cast<long long>(m) * D + ch;
+    const long long v_minus_k = v - k;                       // same layout: V row = K row + this
 
     float acc[VEC];
 #pragma unroll
@@ -70,17 +73,21 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
             float w[8];
 #pragma unroll
             for (int c = 0; c < 8; ++c) w[c] = wt[c >> 2] * wy[(c >> 1) & 1] * wx[c & 1];
-            const T* kb = kh + s.base * tok_stride;
-            const T* vb = vh + s.base * tok_stride;
+            // corner row pointers: (ct, cy) pairs, the cx = 1 row is one token further
+            const T* kp4[4];
+            kp4[0] = kh + s.base * tok_stride;
+            kp4[1] = kp4[0] + sy;
+            kp4[2] = kp4[0] + st;
+            kp4[3] = kp4[2] + sy;
             const bool full = s.mask == 0xffu && s.ft != 0.0f && s.fy != 0.0f && s.fx != 0.0f;
             float sdot = 0.0f;
             Row vv[8];
             if (full) {
                 Row kk[8];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) kk[c] = E::load(kb + ((c >> 2) * st + ((c >> 1) & 1) * sy + (c & 1) * sx));
+                for (int c = 0; c < 8; ++c) kk[c] = E::load(kp4[c >> 1] + (c & 1) * sx);
 #pragma unroll
-                for (int c = 0; c < 8; ++c) vv[c] = E::load(vb + ((c >> 2) * st + ((c >> 1) & 1) * sy + (c & 1) * sx));
+                for (int c = 0; c < 8; ++c) vv[c] = E::load(kp4[c >> 1] + (c & 1) * sx + v_minus_k);
 #pragma unroll
                 for (int c = 0; c < 8; ++c) sdot = fmaf(w[c], E::dot(qr, kk[c], 0.0f), sdot);
             } else {
@@ -88,9 +95,9 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
                 for (int c = 0; c < 8; ++c) {
                     vv[c] = E::zero();
                     if (((s.mask >> c) & 1u) && w[c] != 0.0f) {
-                        const int o = (c >> 2) * st + ((c >> 1) & 1) * sy + (c & 1) * sx;
-                        const Row kk = E::load(kb + o);
-                        vv[c] = E::load(vb + o);
+                        const T* pk = kp4[c >> 1] + (c & 1) * sx;
+                        const Row kk = E::load(pk);
+                        vv[c] = E::load(pk + v_minus_k);
                         sdot = fmaf(w[c], E::dot(qr, kk, 0.0f), sdot);
                     } else {
                         w[c] = 0.0f;
@@ -98,13 +105,18 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
                 }
             }
             const float sp = group_sum<LPR>(sdot, gmask) * lscale;
-            const float m_new = fmaxf(m_run, sp);
-            const float corr = exp2f(m_run - m_new);
-            const float pe = exp2f(sp - m_new);
-            l_run = fmaf(l_run, corr, pe);
-            m_run = m_new;
+            // Online softmax with a lazily updated reference: the running maximum m_run only
+            // moves when a logit exceeds it by more than 8 (log2 units), so exp2(sp - m_run)
+            // stays below 256 and the accumulators are rescaled only a few times per query.
+            if (sp > m_run + 8.0f) {
+                const float corr = exp2f(m_run - sp);
+                l_run *= corr;
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) acc[e] *= corr;
+                for (int e = 0; e < VEC; ++e) acc[e] *= corr;
+                m_run = sp;
+            }
+            const float pe = exp2f(sp - m_run);
+            l_run += pe;
 #pragma unroll
             for (int c = 0; c < 8; ++c) E::axpy(pe * w[c], vv[c], acc);
         }
@@ -112,8 +124,10 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
     const float inv = 1.0f / l_run;
 #pragma unroll
     for (int e = 0; e < VEC; ++e) acc[e] *= inv;
-    E::store(out + row * D + ch, acc);
-    if (gl == 0) lse[row] = (m_run + log2f(l_run)) * kLn2;
+    if (active) {
+        E::store(out + row * D + ch, acc);
+        if (gl == 0) lse[row] = (m_run + log2f(l_run)) * kLn2;
+    }
 }
 
 template <typename T, int D>
