@@ -43,14 +43,14 @@ constexpr int kStats = 8;   // per sample: alpha, g, A_t, A_y, A_x, B_t, B_y, B_
 #define DSA3D_BWD_MINBLOCKS 3
 #endif
 
-template <typename T, int D>
-__global__ void __launch_bounds__(256, DSA3D_BWD_MINBLOCKS)
+template <typename T, int D, int NV>
+__global__ void __launch_bounds__(256, NV == 2 ? 2 : DSA3D_BWD_MINBLOCKS)
 backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                 const float* __restrict__ offsets, const float* __restrict__ lse,
                 const T* __restrict__ dout, T* __restrict__ dq, float* __restrict__ acc_dk,
                 float* __restrict__ acc_dv, float* __restrict__ doffsets, float2* __restrict__ coef,
                 const Problem pr) {
-    using E = Elt<T>;
+    using E = Elt<T, NV>;
     using Row = typename E::Row;
     constexpr int VEC = E::VEC;
     constexpr int LPR = D / VEC;
@@ -441,18 +441,27 @@ size_t tile_smem_bytes(const Problem& pr) {
     return TQ * pr.d * 2 * 2 + NB * sizeof(unsigned);
 }
 
+// 16-byte vectors per lane: two for 128-channel bf16 rows (8 lanes per item, 4 items per warp,
+// 2 blocks per SM), which halves the per-item bookkeeping of the backward; one otherwise.
+#ifndef DSA3D_BWD_BF16_NV
+#define DSA3D_BWD_BF16_NV 2
+#endif
+template <typename T, int D> struct LaneWidth { static constexpr int NV = 1; };
+template <> struct LaneWidth<__nv_bfloat16, 128> { static constexpr int NV = DSA3D_BWD_BF16_NV; };
+
 template <typename T, int D>
 static cudaError_t launch_backward_t(const void* q, const void* k, const void* v, const float* offsets,
                                      const float* lse, const void* dout, void* dq, float* acc_dk,
                                      float* acc_dv, float* doffsets, float2* coef, const Problem& pr,
                                      cudaStream_t stream) {
-    constexpr int LPR = D / Elt<T>::VEC;
+    constexpr int NV = LaneWidth<T, D>::NV;
+    constexpr int LPR = D / Elt<T, NV>::VEC;
     // Shared memory holds 8 floats per (group, sample); shrink the block for large windows.
     int threads = 256;
     while (threads > 32 && static_cast<size_t>(threads / LPR) * pr.P * kStats * sizeof(float) > 64 * 1024)
         threads /= 2;
     const size_t smem = static_cast<size_t>(threads / LPR) * pr.P * kStats * sizeof(float);
-    auto kern = backward_kernel<T, D>;
+    auto kern = backward_kernel<T, D, NV>;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              static_cast<int>(smem));

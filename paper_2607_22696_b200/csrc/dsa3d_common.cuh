@@ -22,36 +22,49 @@ struct Problem {
 };
 
 // ---------------------------------------------------------------------------------------
-// Element access.  A lane handles one 16-byte vector of a row: 8 bf16 or 4 fp32 channels.
+// Element access.  A lane handles NV consecutive 16-byte vectors of a row (8 bf16 or 4 fp32
+// channels each).
 // `Row` keeps that vector in its storage form.  For bf16 the products use the sm_100
 // mixed-precision instruction fma.rn.f32.bf16 (bf16 x bf16 -> exact fp32 product, fp32
 // accumulate), which needs no unpacking; `axpy` rounds its fp32 coefficient to bf16 first.
 // ---------------------------------------------------------------------------------------
-template <typename T> struct Elt;
+template <typename T, int NV> struct Elt;       // NV = 16-byte vectors per lane (1 or 2)
 
-template <> struct Elt<float> {
-    static constexpr int VEC = 4;
-    struct Row { float v[4]; };
+template <int NV> struct Elt<float, NV> {
+    static constexpr int VEC = 4 * NV;
+    struct Row { float v[VEC]; };
     static __device__ __forceinline__ Row load(const float* p) {
-        const float4 r = __ldg(reinterpret_cast<const float4*>(p));
-        return Row{{r.x, r.y, r.z, r.w}};
+        Row r;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const float4 x = __ldg(reinterpret_cast<const float4*>(p) + i);
+            r.v[4 * i] = x.x; r.v[4 * i + 1] = x.y; r.v[4 * i + 2] = x.z; r.v[4 * i + 3] = x.w;
+        }
+        return r;
     }
-    static __device__ __forceinline__ Row zero() { return Row{{0.f, 0.f, 0.f, 0.f}}; }
+    static __device__ __forceinline__ Row zero() {
+        Row r;
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) r.v[e] = 0.0f;
+        return r;
+    }
     static __device__ __forceinline__ float dot(const Row& a, const Row& b, float acc) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) acc = fmaf(a.v[e], b.v[e], acc);
+        for (int e = 0; e < VEC; ++e) acc = fmaf(a.v[e], b.v[e], acc);
         return acc;
     }
-    static __device__ __forceinline__ void axpy(float c, const Row& x, float (&acc)[4]) {
+    static __device__ __forceinline__ void axpy(float c, const Row& x, float (&acc)[VEC]) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) acc[e] = fmaf(c, x.v[e], acc[e]);
+        for (int e = 0; e < VEC; ++e) acc[e] = fmaf(c, x.v[e], acc[e]);
     }
-    static __device__ __forceinline__ void to_float(const Row& x, float (&f)[4]) {
+    static __device__ __forceinline__ void to_float(const Row& x, float (&f)[VEC]) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) f[e] = x.v[e];
+        for (int e = 0; e < VEC; ++e) f[e] = x.v[e];
     }
-    static __device__ __forceinline__ void store(float* p, const float (&x)[4]) {
-        *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
+    static __device__ __forceinline__ void store(float* p, const float (&x)[VEC]) {
+#pragma unroll
+        for (int i = 0; i < NV; ++i)
+            reinterpret_cast<float4*>(p)[i] = make_float4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]);
     }
 };
 
@@ -65,17 +78,28 @@ __device__ __forceinline__ void split_b32(uint32_t r, unsigned short& lo, unsign
     asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(r));
 }
 
-template <> struct Elt<__nv_bfloat16> {
-    static constexpr int VEC = 8;
-    struct Row { uint32_t w[4]; };
+template <int NV> struct Elt<__nv_bfloat16, NV> {
+    static constexpr int VEC = 8 * NV;
+    static constexpr int NW = 4 * NV;            // 32-bit words per lane
+    struct Row { uint32_t w[NW]; };
     static __device__ __forceinline__ Row load(const __nv_bfloat16* p) {
-        const uint4 r = __ldg(reinterpret_cast<const uint4*>(p));
-        return Row{{r.x, r.y, r.z, r.w}};
+        Row r;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const uint4 x = __ldg(reinterpret_cast<const uint4*>(p) + i);
+            r.w[4 * i] = x.x; r.w[4 * i + 1] = x.y; r.w[4 * i + 2] = x.z; r.w[4 * i + 3] = x.w;
+        }
+        return r;
     }
-    static __device__ __forceinline__ Row zero() { return Row{{0u, 0u, 0u, 0u}}; }
+    static __device__ __forceinline__ Row zero() {
+        Row r;
+#pragma unroll
+        for (int i = 0; i < NW; ++i) r.w[i] = 0u;
+        return r;
+    }
     static __device__ __forceinline__ float dot(const Row& a, const Row& b, float acc) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < NW; ++i) {
             unsigned short al, ah, bl, bh;
             split_b32(a.w[i], al, ah);
             split_b32(b.w[i], bl, bh);
@@ -84,31 +108,34 @@ template <> struct Elt<__nv_bfloat16> {
         }
         return acc;
     }
-    static __device__ __forceinline__ void axpy(float c, const Row& x, float (&acc)[8]) {
+    static __device__ __forceinline__ void axpy(float c, const Row& x, float (&acc)[VEC]) {
         const unsigned short cb = __bfloat16_as_ushort(__float2bfloat16_rn(c));
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < NW; ++i) {
             unsigned short xl, xh;
             split_b32(x.w[i], xl, xh);
             acc[2 * i] = fma_bf16(cb, xl, acc[2 * i]);
             acc[2 * i + 1] = fma_bf16(cb, xh, acc[2 * i + 1]);
         }
     }
-    static __device__ __forceinline__ void to_float(const Row& x, float (&f)[8]) {
+    static __device__ __forceinline__ void to_float(const Row& x, float (&f)[VEC]) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {           // bf16 is the upper half of an fp32
+        for (int i = 0; i < NW; ++i) {          // bf16 is the upper half of an fp32
             f[2 * i] = __uint_as_float(x.w[i] << 16);
             f[2 * i + 1] = __uint_as_float(x.w[i] & 0xffff0000u);
         }
     }
-    static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&x)[8]) {
-        uint32_t w[4];
+    static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&x)[VEC]) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const __nv_bfloat162 h = __floats2bfloat162_rn(x[2 * i], x[2 * i + 1]);   // RNE
-            w[i] = *reinterpret_cast<const uint32_t*>(&h);
+        for (int i = 0; i < NV; ++i) {
+            uint32_t w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const __nv_bfloat162 h = __floats2bfloat162_rn(x[8 * i + 2 * j], x[8 * i + 2 * j + 1]);   // RNE
+                w[j] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+            reinterpret_cast<uint4*>(p)[i] = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
     }
 };
 

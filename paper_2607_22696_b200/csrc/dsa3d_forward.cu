@@ -21,12 +21,12 @@ namespace dsa3d {
 #define DSA3D_FWD_MINBLOCKS 3
 #endif
 
-template <typename T, int D>
-__global__ void __launch_bounds__(256, DSA3D_FWD_MINBLOCKS)
+template <typename T, int D, int NV>
+__global__ void __launch_bounds__(256, NV == 2 ? 2 : DSA3D_FWD_MINBLOCKS)
 forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                const float* __restrict__ offsets, T* __restrict__ out, float* __restrict__ lse,
                const Problem pr) {
-    using E = Elt<T>;
+    using E = Elt<T, NV>;
     using Row = typename E::Row;
     constexpr int VEC = E::VEC;
     constexpr int LPR = D / VEC;
@@ -130,14 +130,23 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
     }
 }
 
+// 16-byte vectors per lane.  One everywhere: two (8 lanes per 128-channel bf16 item) halves
+// the per-item bookkeeping but costs a block of occupancy, which the forward loses more by.
+#ifndef DSA3D_FWD_BF16_NV
+#define DSA3D_FWD_BF16_NV 1
+#endif
+template <typename T, int D> struct LaneWidth { static constexpr int NV = 1; };
+template <> struct LaneWidth<__nv_bfloat16, 128> { static constexpr int NV = DSA3D_FWD_BF16_NV; };
+
 template <typename T, int D>
 static cudaError_t launch_forward_t(const void* q, const void* k, const void* v, const float* offsets,
                                     void* out, float* lse, const Problem& pr, cudaStream_t stream) {
-    constexpr int LPR = D / Elt<T>::VEC;
+    constexpr int NV = LaneWidth<T, D>::NV;
+    constexpr int LPR = D / Elt<T, NV>::VEC;
     constexpr int threads = 256;
     const long long groups_per_block = threads / LPR;
     const long long blocks = (pr.items + groups_per_block - 1) / groups_per_block;
-    forward_kernel<T, D><<<static_cast<unsigned>(blocks), threads, 0, stream>>>(
+    forward_kernel<T, D, NV><<<static_cast<unsigned>(blocks), threads, 0, stream>>>(
         static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), offsets,
         static_cast<T*>(out), lse, pr);
     return cudaGetLastError();
