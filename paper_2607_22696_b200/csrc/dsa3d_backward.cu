@@ -376,6 +376,7 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
 
         // ---- reduce: a warp takes two neighbouring key rows, one per half-warp; both halves
         //      run the same number of steps (the shorter list is padded with zero entries)
+#ifndef DSA3D_DEBUG_SKIP_REDUCE
         {
             const int half = lane >> 4, hl = lane & 15;
             const int hv = hl < VPR ? hl : VPR - 1;         // lanes beyond a narrow row mirror its last vector
@@ -419,7 +420,11 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                         }
                     }
                 }
+#ifndef DSA3D_DEBUG_SKIP_FLUSH
                 if (cnt_mine > 0u && hl < VPR) {
+#else
+                if (cnt_mine > 0u && hl < VPR && ak[0] == 12345.678f) {
+#endif
                     const int bx = bin % ex, by = (bin / ex) % ey, bt = bin / (ex * ey);
                     const long long tok = (static_cast<long long>(lo_t + bt) * pr.H + (lo_y + by)) * pr.W + (lo_x + bx);
                     const long long o = tok * tok_stride + static_cast<long long>(m) * D + hl * 8;
@@ -430,6 +435,7 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                 }
             }
         }
+#endif
         __syncthreads();     // the next tile reuses the rows, the counters and the scratch
     }
 }
