@@ -42,6 +42,12 @@ METRIC = "3D-DSA fwd+bwd Mtokens/s (bf16), inputs resident in HBM"
 UNIT = "Mtokens/s"
 FALLBACK_HBM_GBS = 6650.0
 
+# DRAM bytes per (token, head) item, dram__bytes_read.sum + dram__bytes_write.sum of one ncu
+# capture per kernel on the profile_small_bf16 workload (profiles/*_profile_small_bf16.md).
+# Every kernel's traffic is proportional to the number of items, so a launch on another
+# workload with the same d and window is reported as items x these figures.
+NCU_DRAM_BYTES_PER_ITEM = {"forward_kernel": 1525.0, "backward_kernel": 2986.0, "scatter_tile_kernel": 8280.0}
+
 
 # ----------------------------------------------------------------------------- utilities
 
@@ -285,6 +291,12 @@ def run_ours(args, wl):
            "ms": bwd_pair_ms if dominant_bwd else fwd_ms,
            "bytes": wl.bwd_bytes() if dominant_bwd else wl.fwd_bytes()}
     step_bytes = wl.fwd_bytes() + (wl.bwd_bytes() if wl.backward else 0)
+    traffic = None
+    if wl.dtype == torch.bfloat16 and wl.d == 128 and wl.P == 27:
+        items = wl.N * wl.heads
+        per_item = (NCU_DRAM_BYTES_PER_ITEM["backward_kernel"] + (NCU_DRAM_BYTES_PER_ITEM["scatter_tile_kernel"]
+                    if tiled else 0.0)) if dominant_bwd else NCU_DRAM_BYTES_PER_ITEM["forward_kernel"]
+        traffic = items * per_item
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
         "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -295,7 +307,8 @@ def run_ours(args, wl):
                    "parallelism": f"independent videos x{world}",
                    "l2": "inputs (tens of GB) exceed the 126 MB L2; no flush needed"},
         "roofline": {"bound": "hbm", "kernel": dom["kernel"], "achieved": dom["achieved"], "peak": peak,
-                     "unit": "GB/s", "frac": dom["achieved"] / peak, "traffic": None,
+                     "unit": "GB/s", "frac": dom["achieved"] / peak, "traffic": traffic,
+                     "traffic_source": "ncu dram bytes per item on profile_small_bf16 x items of this launch",
                      "peak_source": peak_src, "algorithmic_bytes_per_launch": dom["bytes"],
                      "kernel_ms": dom["ms"],
                      "forward_kernel": {"ms": fwd_ms, "achieved": fwd_gbs, "frac": fwd_gbs / peak},

@@ -50,8 +50,8 @@ int make_problem(int T, int H, int W, int heads, int d, const int* window, int d
 }
 
 // Query tiling of the backward scatter: 4 x 8 x 8 queries per tile, halo of 6 cells.  The
-// environment variable DSA3D_TILE="tt,ty,tx,halo" overrides it for experiments ("0" turns
-// the tile kernel off); values that do not fit shared memory fall back to the default.
+// environment variable DSA3D_TILE="tt,ty,tx,halo" overrides it for experiments ("0"
+// turns the tile kernel off); values that do not fit shared memory fall back to the default.
 constexpr int kTileSlots = 304;          // upper bound on resident tile CTAs (scratch regions)
 constexpr size_t kTileSmemLimit = 200 * 1024;
 

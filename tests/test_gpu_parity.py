@@ -148,3 +148,21 @@ def test_config_1080p_256f_bf16_forward_backward():
 def test_config_sweep_720p_grid(window, kind):
     boxes = [((0, 0, 0), (1, 2, 2)), ((32, 22, 40), (33, 23, 42))]
     run_large(f"sweep_w{window}_{kind}", [0, 15], boxes, n_random=512)
+
+
+# ------------------------------------------------- tilings of the backward dK/dV scatter
+
+@pytest.mark.parametrize("tiling", ["0", "2,2,2,1", "4,8,8,0", "1,1,1,3", "3,5,7,2", "4,8,8,6"])
+def test_backward_is_the_same_for_every_tiling(tiling, monkeypatch):
+    """dK/dV are pre-reduced per query tile for corners inside the tile's halo and sent
+    straight to the accumulators otherwise; any split of the work (none tiled, tiles that
+    do not divide the grid, no halo, one-query tiles) must give the oracle's result."""
+    monkeypatch.setenv("DSA3D_TILE", tiling)
+    q, k, v, off, dout = small_problem(5, 11, 13, 3, 128, (3, 3, 3), BF16, 1.7, 50)
+    pu.full_parity(q, k, v, off, dout, (3, 3, 3))
+    q, k, v, off, dout = small_problem(3, 9, 10, 2, 64, (2, 2, 2), BF16, 0.8, 51)
+    pu.full_parity(q, k, v, off, dout, (2, 2, 2))
+
+
+def test_large_window_through_the_tile_kernel():
+    pu.full_parity(*small_problem(4, 10, 12, 2, 128, (3, 7, 7), BF16, 2.0, 52), (3, 7, 7))
