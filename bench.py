@@ -183,6 +183,31 @@ def run_reference(args, wl):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------- multi-rank plumbing
+
+def rank_workload(wl, rank: int):
+    """The video rank `rank` processes: the same shape for every rank (weak scaling), its own
+    seed, so that no two ranks hold the same data.  Videos are independent, so there is no
+    collective on the data path; ranks only meet in the timing barrier and the max below."""
+    return wl if rank == 0 else inputs.dataclasses.replace(wl, seed=wl.seed + 1000 * rank)
+
+
+def max_over_ranks(x: float, world: int, device=None) -> float:
+    """Largest value of `x` over the ranks of the default process group (x itself when
+    there is one rank)."""
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_mtokens_per_s(wl, world: int, step_ms: float) -> float:
+    """Whole-job throughput: every rank processed one video of wl.N tokens in step_ms."""
+    return wl.N * world / (step_ms * 1e-3) / 1e6
+
+
 # ------------------------------------------------------------------------------ GPU arm
 
 def run_ours(args, wl):
@@ -203,17 +228,13 @@ def run_ours(args, wl):
         if world > 1:
             dist.barrier()
 
-    def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    def max_ranks(x: float) -> float:
+        return max_over_ranks(x, world, dev)
 
     binding.load()
     dims = (wl.T, wl.H, wl.W, wl.heads, wl.d)
     # every rank takes its own video of the batch: same shape, its own seed
-    wl_rank = wl if rank == 0 else inputs.dataclasses.replace(wl, seed=wl.seed + 1000 * rank)
+    wl_rank = rank_workload(wl, rank)
     t = inputs.make_inputs(wl_rank, dev, with_dout=True)
     ws_bytes = binding.dsa3d_backward_workspace_bytes(*dims, wl.window, wl.dtype)
     b = {"out": torch.empty_like(t["q"]),
@@ -256,16 +277,16 @@ def run_ours(args, wl):
     bwd_ms = sum(ev[i][4].elapsed_time(ev[i][5]) for i in range(K)) / K if wl.backward else 0.0
     tiled = wl.backward and wl.dtype == torch.bfloat16 and os.environ.get("DSA3D_TILE", "") != "0"
     sct_ms = sum(ev[i][6].elapsed_time(ev[i][7]) for i in range(K)) / K if tiled else 0.0
-    step_ms = max_over_ranks(step_ms)
-    fwd_ms, bwd_ms, sct_ms = max_over_ranks(fwd_ms), max_over_ranks(bwd_ms), max_over_ranks(sct_ms)
-    value = wl.N * world / (step_ms * 1e-3) / 1e6
+    step_ms = max_ranks(step_ms)
+    fwd_ms, bwd_ms, sct_ms = max_ranks(fwd_ms), max_ranks(bwd_ms), max_ranks(sct_ms)
+    value = aggregate_mtokens_per_s(wl, world, step_ms)
 
     # ---------------------------------------------------------------- end to end (host)
     e2e = None
     b.clear()                           # the end-to-end leg brings its own device arena
     torch.cuda.empty_cache()
     if not args.no_e2e:
-        e2e = run_e2e(args, wl, t, dims, dev, barrier, max_over_ranks, world)
+        e2e = run_e2e(args, wl, t, dims, dev, barrier, max_ranks, world)
     # --------------------------------------------------------------------- CPU baseline
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -325,7 +346,7 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
-def run_e2e(args, wl, t, dims, dev, barrier, max_over_ranks, world):
+def run_e2e(args, wl, t, dims, dev, barrier, max_ranks, world):
     """Forward + backward through dsa3d_step_host: inputs start in pinned host memory and
     every output ends in pinned host memory, each step."""
     from paper_2607_22696_b200 import binding
@@ -366,10 +387,10 @@ def run_e2e(args, wl, t, dims, dev, barrier, max_over_ranks, world):
     torch.cuda.synchronize()
     wall = (time.perf_counter() - wall0) / steps
     barrier()
-    ms = max_over_ranks(e0.elapsed_time(e1) / steps)
+    ms = max_ranks(e0.elapsed_time(e1) / steps)
     h2d = sum(h.numel() * h.element_size() for h in host_in.values())
     d2h = sum(h.numel() * h.element_size() for h in host_out.values())
-    return {"value": wl.N * world / (ms * 1e-3) / 1e6, "unit": UNIT, "h2d_bytes_per_step": h2d,
+    return {"value": aggregate_mtokens_per_s(wl, world, ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": ms, "wall_ms_per_step": wall * 1e3, "steps": steps,
             "entry_point": "dsa3d_step_host"}
 

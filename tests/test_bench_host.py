@@ -1,0 +1,64 @@
+"""Host-side logic of bench.py: the reference arm's JSON contract (it runs the CPU oracle,
+so it needs no GPU) and the multi-rank plumbing, exercised with two gloo ranks on CPU."""
+import json
+import os
+import subprocess
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+
+def test_reference_arm_prints_one_contract_line():
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference",
+                          "--workload", "tiny_f32", "--steps", "2", "--warmup", "1"],
+                         capture_output=True, text=True, timeout=600, cwd=ROOT)
+    assert out.returncode == 0, out.stderr
+    lines = [l for l in out.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["unit"] == "Mtokens/s" and d["higher_is_better"] is True
+    assert d["value"] > 0 and d["steps"] == 2 and d["warmup"] == 1
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1
+    assert d["cpu_baseline"]["value"] == d["value"] == d["e2e"]["value"]
+    assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["d2h_bytes_per_step"] == 0
+    assert d["config"]["workload"] == "tiny_f32" and "model" not in d["config"]
+
+
+def test_reference_arm_other_ranks_print_nothing():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference",
+                          "--workload", "tiny_f32", "--steps", "1", "--warmup", "0", "--gpus", "2"],
+                         capture_output=True, text=True, timeout=600, cwd=ROOT, env=env)
+    assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def _rank_main(rank, world, port, results):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    from paper_2607_22696_b200 import inputs
+    wl = inputs.WORKLOADS["tiny_f32"]
+    mine = bench.rank_workload(wl, rank)
+    q = inputs.make_rows(mine, "q")
+    slowest = bench.max_over_ranks(10.0 + 5.0 * rank, world)          # rank 1 is the slow one
+    dist.barrier()
+    results[rank] = (mine.seed, mine.N, float(q.double().sum()), slowest,
+                     bench.aggregate_mtokens_per_s(wl, world, slowest))
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_take_different_videos_and_report_the_slowest_time():
+    world, port = 2, 29517
+    with mp.Manager() as manager:
+        results = manager.dict()
+        mp.spawn(_rank_main, args=(world, port, results), nprocs=world, join=True)
+        r0, r1 = results[0], results[1]
+    assert r0[0] != r1[0] and r0[1] == r1[1]            # different seeds, same shape (weak scaling)
+    assert r0[2] != r1[2]                               # different data
+    assert r0[3] == r1[3] == 15.0                       # max over ranks, seen by both
+    assert abs(r0[4] - 2 * 256 / 15e-3 / 1e6) < 1e-12   # whole-job tokens / slowest time
