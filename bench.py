@@ -47,6 +47,23 @@ FALLBACK_HBM_GBS = 6650.0
 # Every kernel's traffic is proportional to the number of items, so a launch on another
 # workload with the same d and window is reported as items x these figures.
 NCU_DRAM_BYTES_PER_ITEM = {"forward_kernel": 1525.0, "backward_kernel": 2986.0, "scatter_tile_kernel": 8280.0}
+# L2 -> SM bytes per item of the forward's corner gathers (l1tex__m_xbar2l1tex_read_bytes.sum
+# of the same capture / items): what is left of the 110,592 gathered bytes after L1 hits.
+NCU_L2_TO_SM_BYTES_PER_ITEM = {"forward_kernel": 83021.0, "backward_kernel": 94521.0}
+NCU_RED_BYTES_PER_ITEM = {"scatter_tile_kernel": 23470.0}      # lts red sectors x 32 B / items
+
+
+def measure_ceilings(dev):
+    """On-chip ceilings of this GPU, measured now with the library's probe kernels."""
+    from paper_2607_22696_b200 import binding
+    buf = torch.zeros(48 << 20, dtype=torch.uint8, device=dev)        # well inside the 126 MB L2
+    out = {"l2_row_gather_gbs": binding.dsa3d_probe_gather(buf, buf.numel()),
+           "l2_red_v4_f32_gbs": binding.dsa3d_probe_red(buf, buf.numel()),
+           "fma_f32_tfma": binding.dsa3d_probe_fma(buf, 0),
+           "fma_bf16_mixed_tfma": binding.dsa3d_probe_fma(buf, 1),
+           "working_set_mb": 48}
+    del buf
+    return out
 
 
 # ----------------------------------------------------------------------------- utilities
@@ -312,6 +329,23 @@ def run_ours(args, wl):
            "ms": bwd_pair_ms if dominant_bwd else fwd_ms,
            "bytes": wl.bwd_bytes() if dominant_bwd else wl.fwd_bytes()}
     step_bytes = wl.fwd_bytes() + (wl.bwd_bytes() if wl.backward else 0)
+    # Fractions of the ceilings that actually bind (the path is on-chip bound, not HBM bound)
+    ceil = measure_ceilings(dev)
+    items_all = wl.N * wl.heads
+    fma_fwd = items_all * wl.P * 8 * 2 * wl.d
+    onchip = {"ceilings": ceil,
+              "forward_kernel": {"fma_frac": fma_fwd / (fwd_ms * 1e-3) / 1e12 / ceil["fma_bf16_mixed_tfma"]}}
+    if wl.dtype == torch.bfloat16 and wl.d == 128 and wl.P == 27:
+        gather_gbs = items_all * NCU_L2_TO_SM_BYTES_PER_ITEM["forward_kernel"] / (fwd_ms * 1e-3) / 1e9
+        onchip["forward_kernel"].update(l2_gather_gbs=gather_gbs, l2_gather_frac=gather_gbs / ceil["l2_row_gather_gbs"])
+    if wl.backward:
+        onchip["backward_kernel"] = {"fma_frac": items_all * wl.P * 8 * 3 * wl.d / (bwd_ms * 1e-3) / 1e12
+                                     / ceil["fma_bf16_mixed_tfma"]}
+        if tiled:
+            onchip["scatter_tile_kernel"] = {"fma_frac": fma_fwd / (sct_ms * 1e-3) / 1e12 / ceil["fma_bf16_mixed_tfma"]}
+            if wl.d == 128 and wl.P == 27:
+                red_gbs = items_all * NCU_RED_BYTES_PER_ITEM["scatter_tile_kernel"] / (sct_ms * 1e-3) / 1e9
+                onchip["scatter_tile_kernel"].update(red_gbs=red_gbs, red_frac=red_gbs / ceil["l2_red_v4_f32_gbs"])
     traffic = None
     if wl.dtype == torch.bfloat16 and wl.d == 128 and wl.P == 27:
         items = wl.N * wl.heads
@@ -335,6 +369,7 @@ def run_ours(args, wl):
                      "forward_kernel": {"ms": fwd_ms, "achieved": fwd_gbs, "frac": fwd_gbs / peak},
                      "backward_kernels": ({"gather_ms": bwd_ms, "tile_scatter_ms": sct_ms, "achieved": bwd_gbs,
                                           "frac": bwd_gbs / peak} if wl.backward else None),
+                     "onchip": onchip,
                      "whole_step": {"bytes": step_bytes, "achieved": step_bytes / (step_ms * 1e-3) / 1e9,
                                     "frac": step_bytes / (step_ms * 1e-3) / 1e9 / peak}},
         "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,

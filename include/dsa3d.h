@@ -155,6 +155,27 @@ int dsa3d_backward_noalloc_last_cuda_error(void);
 int dsa3d_set_profile_events(void* fwd_start, void* fwd_stop, void* bwd_start, void* bwd_stop,
                              void* scatter_start, void* scatter_stop);
 
+/*
+ * Ceiling probes (measurement aids; the paper has no counterpart).  The operator gathers and
+ * scatters rows of a few hundred bytes, so what bounds it on a GPU is the rate of such
+ * accesses out of L2 and the FMA issue rate rather than streaming bandwidth.  Each probe
+ * launches one kernel on `stream` over a caller-owned DEVICE buffer and stores in its
+ * HOST out-parameter the work of that launch; the caller times the launch.
+ *   dsa3d_probe_gather : random 256-byte-row reads (16-byte loads, two rows per warp
+ *                        step) spread over `working_set_bytes` of `buffer`; `iters` a
+ *                        multiple of 8; *bytes_per_launch = bytes read.
+ *   dsa3d_probe_red    : red.global.add.v4.f32 of zeros onto random 512-byte rows of
+ *                        `buffer` (contents unchanged); *bytes_per_launch = operand bytes.
+ *   dsa3d_probe_fma    : 64 FMAs per thread and iteration on registers; kind 0 = fp32 FMA,
+ *                        kind 1 = bf16 x bf16 -> fp32 FMA; `seed_1kb` is any 1 KiB of
+ *                        device memory; *fma_per_launch = FMAs executed.
+ */
+int dsa3d_probe_gather(const void* buffer, size_t working_set_bytes, int iters, double* bytes_per_launch,
+                       void* stream);
+int dsa3d_probe_red(void* buffer, size_t working_set_bytes, int iters, double* bytes_per_launch,
+                    void* stream);
+int dsa3d_probe_fma(const void* seed_1kb, int iters, int kind, double* fma_per_launch, void* stream);
+
 /* Static, NUL-terminated description of a status code. */
 const char* dsa3d_status_string(int status);
 

@@ -58,6 +58,13 @@ def load():
     lib.dsa3d_backward_noalloc_max_elements.argtypes = []
     lib.dsa3d_backward_noalloc_last_cuda_error.restype = i
     lib.dsa3d_backward_noalloc_last_cuda_error.argtypes = []
+    dptr = ctypes.POINTER(ctypes.c_double)
+    lib.dsa3d_probe_gather.restype = i
+    lib.dsa3d_probe_gather.argtypes = [p, sz, i, dptr, p]
+    lib.dsa3d_probe_red.restype = i
+    lib.dsa3d_probe_red.argtypes = [p, sz, i, dptr, p]
+    lib.dsa3d_probe_fma.restype = i
+    lib.dsa3d_probe_fma.argtypes = [p, i, i, dptr, p]
     lib.dsa3d_status_string.restype = ctypes.c_char_p
     lib.dsa3d_status_string.argtypes = [i]
     lib.dsa3d_last_cuda_error.restype = i
@@ -215,3 +222,45 @@ def dsa3d_backward_noalloc(q, k, v, offsets, lse, dout, T, H, W, heads, d, windo
         _ptr(dout, "dout", n * d), T, H, W, heads, d, _window(window),
         _ptr(dq, "dq", n * d), _ptr(dk, "dk", n * d), _ptr(dv, "dv", n * d),
         _ptr(doffsets, "doffsets", n * P * 3, torch.float32), code, _stream(stream)))
+
+
+def _timed(launch, reps: int = 3) -> float:
+    """Best CUDA-event time (ms) of `launch()` over `reps` runs after one warm-up."""
+    launch()
+    torch.cuda.synchronize()
+    best = float("inf")
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        launch()
+        b.record()
+        b.synchronize()
+        best = min(best, a.elapsed_time(b))
+    return best
+
+
+def dsa3d_probe_gather(buffer: torch.Tensor, working_set_bytes: int, iters: int = 2048) -> float:
+    """GB/s of random 256-byte-row reads spread over the first `working_set_bytes` of `buffer`."""
+    lib, work = load(), ctypes.c_double()
+    def launch():
+        _check(lib.dsa3d_probe_gather(_ptr(buffer, "buffer"), working_set_bytes, iters, ctypes.byref(work), _stream(None)))
+    ms = _timed(launch)
+    return work.value / ms / 1e6
+
+
+def dsa3d_probe_red(buffer: torch.Tensor, working_set_bytes: int, iters: int = 512) -> float:
+    """GB/s of fp32 vector-reduction operands onto random 512-byte rows of `buffer`."""
+    lib, work = load(), ctypes.c_double()
+    def launch():
+        _check(lib.dsa3d_probe_red(_ptr(buffer, "buffer"), working_set_bytes, iters, ctypes.byref(work), _stream(None)))
+    ms = _timed(launch)
+    return work.value / ms / 1e6
+
+
+def dsa3d_probe_fma(seed: torch.Tensor, kind: int, iters: int = 4096) -> float:
+    """TFMA/s of register-resident FMAs: kind 0 fp32, kind 1 bf16 x bf16 -> fp32."""
+    lib, work = load(), ctypes.c_double()
+    def launch():
+        _check(lib.dsa3d_probe_fma(_ptr(seed, "seed"), iters, kind, ctypes.byref(work), _stream(None)))
+    ms = _timed(launch)
+    return work.value / ms / 1e9
