@@ -100,8 +100,12 @@ size_t dsa3d_backward_workspace_bytes(int T, int H, int W, int heads, int d,
  * Every *_h pointer is a HOST pointer (page-locked memory makes the copies asynchronous
  * and fast; pageable memory works but serialises).  `arena` is DEVICE scratch of at least
  * dsa3d_step_host_arena_bytes(...) bytes, 256-byte aligned, which holds the device copies
- * and the backward workspace; the library allocates nothing.  All work is enqueued on
- * `stream`; the host buffers must not be touched until the stream has finished.
+ * and the backward workspace; the library allocates no memory.  The upload of dout runs
+ * beside the forward and the downloads of out, lse, dq and doffsets beside the backward, on
+ * two side streams the library creates on the calling thread's first call (with a few
+ * events; they are kept for the life of the thread); everything is ordered after the work
+ * already in `stream`, and the step is complete when `stream` is.  The host buffers must
+ * not be touched until then.  Not for use inside a stream capture.
  */
 int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const float* offsets_h,
                     const void* dout_h, int T, int H, int W, int heads, int d, const int window[3],

@@ -133,7 +133,8 @@ int dsa3d_backward(const void* q, const void* k, const void* v, const float* off
 int dsa3d::backward_impl(const void* q, const void* k, const void* v, const float* offsets, const float* lse,
                          const void* dout, int T, int H, int W, int heads, int d, const int window[3],
                          void* dq, void* dk, void* dv, float* doffsets, void* workspace,
-                         size_t workspace_bytes, int dtype, void* stream_, bool tiled) {
+                         size_t workspace_bytes, int dtype, void* stream_, bool tiled,
+                         cudaEvent_t after_gather) {
     if (!q || !k || !v || !offsets || !lse || !dout || !dq || !dk || !dv || !doffsets)
         return DSA3D_ERR_NULL_POINTER;
     dsa3d::Problem pr;
@@ -172,6 +173,10 @@ int dsa3d::backward_impl(const void* q, const void* k, const void* v, const floa
     if (e != cudaSuccess) return cuda_failed(e);
     e = record(3, stream);
     if (e != cudaSuccess) return cuda_failed(e);
+    if (after_gather) {
+        e = cudaEventRecord(after_gather, stream);
+        if (e != cudaSuccess) return cuda_failed(e);
+    }
     if (coef) {
         int dev = 0, sms = 0;
         e = cudaGetDevice(&dev);
@@ -231,6 +236,35 @@ Arena arena_layout(const dsa3d::Problem& pr, int dtype) {
     return a;
 }
 
+// Two side streams and four events per (thread, device) for the copy/compute overlap of
+// dsa3d_step_host; created on first use and kept for the life of the thread.
+struct HostStep {
+    int device = -1;
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, dout_ready = nullptr, fwd_done = nullptr, gather_done = nullptr,
+                out_done = nullptr;
+};
+thread_local HostStep g_host_step[8];
+
+HostStep* host_step_resources() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    HostStep* slot = nullptr;
+    for (HostStep& h : g_host_step) {
+        if (h.device == dev) return &h;
+        if (!slot && h.device < 0) slot = &h;
+    }
+    if (!slot) return nullptr;                          // more than 8 devices used from one thread
+    cudaEvent_t* events[5] = {&slot->start, &slot->dout_ready, &slot->fwd_done, &slot->gather_done,
+                              &slot->out_done};
+    if (cudaStreamCreateWithFlags(&slot->in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithFlags(&slot->out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    for (cudaEvent_t* ev : events)
+        if (cudaEventCreateWithFlags(ev, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    slot->device = dev;
+    return slot;
+}
+
 }  // namespace
 
 size_t dsa3d_step_host_arena_bytes(int T, int H, int W, int heads, int d, const int window[3], int dtype) {
@@ -254,29 +288,51 @@ int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const flo
     if (arena_bytes < a.total) return DSA3D_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     char* base = static_cast<char*>(arena);
-    const struct { size_t at; const void* src; size_t bytes; } in[5] = {
-        {a.q, q_h, a.row_bytes}, {a.k, k_h, a.row_bytes}, {a.v, v_h, a.row_bytes},
-        {a.offsets, offsets_h, a.off_bytes}, {a.dout, dout_h, a.row_bytes}};
-    for (const auto& c : in) {
-        const cudaError_t e = cudaMemcpyAsync(base + c.at, c.src, c.bytes, cudaMemcpyHostToDevice, stream);
-        if (e != cudaSuccess) return cuda_failed(e);
-    }
+    HostStep* hs = host_step_resources();
+    if (!hs) return DSA3D_ERR_CUDA;
+    cudaError_t e;
+#define DSA3D_TRY(call)                         \
+    do {                                        \
+        e = (call);                             \
+        if (e != cudaSuccess) return cuda_failed(e); \
+    } while (0)
+    // Side stream `in`: dout is only needed by the backward, so its upload runs beside the
+    // forward.  Side stream `out`: results leave as soon as they are final - out and lse
+    // during the backward, dq and doffsets during the dk/dv kernels.
+    DSA3D_TRY(cudaEventRecord(hs->start, stream));
+    DSA3D_TRY(cudaStreamWaitEvent(hs->in, hs->start, 0));
+    DSA3D_TRY(cudaMemcpyAsync(base + a.dout, dout_h, a.row_bytes, cudaMemcpyHostToDevice, hs->in));
+    DSA3D_TRY(cudaEventRecord(hs->dout_ready, hs->in));
+
+    DSA3D_TRY(cudaMemcpyAsync(base + a.k, k_h, a.row_bytes, cudaMemcpyHostToDevice, stream));
+    DSA3D_TRY(cudaMemcpyAsync(base + a.v, v_h, a.row_bytes, cudaMemcpyHostToDevice, stream));
+    DSA3D_TRY(cudaMemcpyAsync(base + a.q, q_h, a.row_bytes, cudaMemcpyHostToDevice, stream));
+    DSA3D_TRY(cudaMemcpyAsync(base + a.offsets, offsets_h, a.off_bytes, cudaMemcpyHostToDevice, stream));
     int st = dsa3d_forward(base + a.q, base + a.k, base + a.v, reinterpret_cast<const float*>(base + a.offsets),
                            T, H, W, heads, d, window, base + a.out, reinterpret_cast<float*>(base + a.lse),
                            dtype, stream_);
     if (st != DSA3D_OK) return st;
-    st = dsa3d_backward(base + a.q, base + a.k, base + a.v, reinterpret_cast<const float*>(base + a.offsets),
-                        reinterpret_cast<const float*>(base + a.lse), base + a.dout, T, H, W, heads, d, window,
-                        base + a.dq, base + a.dk, base + a.dv, reinterpret_cast<float*>(base + a.doffsets),
-                        a.ws_bytes ? base + a.workspace : nullptr, a.ws_bytes, dtype, stream_);
+    DSA3D_TRY(cudaEventRecord(hs->fwd_done, stream));
+    DSA3D_TRY(cudaStreamWaitEvent(hs->out, hs->fwd_done, 0));
+    DSA3D_TRY(cudaMemcpyAsync(out_h, base + a.out, a.row_bytes, cudaMemcpyDeviceToHost, hs->out));
+    DSA3D_TRY(cudaMemcpyAsync(lse_h, base + a.lse, a.lse_bytes, cudaMemcpyDeviceToHost, hs->out));
+
+    DSA3D_TRY(cudaStreamWaitEvent(stream, hs->dout_ready, 0));
+    st = dsa3d::backward_impl(base + a.q, base + a.k, base + a.v, reinterpret_cast<const float*>(base + a.offsets),
+                              reinterpret_cast<const float*>(base + a.lse), base + a.dout, T, H, W, heads, d,
+                              window, base + a.dq, base + a.dk, base + a.dv,
+                              reinterpret_cast<float*>(base + a.doffsets),
+                              a.ws_bytes ? base + a.workspace : nullptr, a.ws_bytes, dtype, stream_, true,
+                              hs->gather_done);
     if (st != DSA3D_OK) return st;
-    const struct { size_t at; void* dst; size_t bytes; } outc[6] = {
-        {a.out, out_h, a.row_bytes}, {a.lse, lse_h, a.lse_bytes}, {a.dq, dq_h, a.row_bytes},
-        {a.dk, dk_h, a.row_bytes}, {a.dv, dv_h, a.row_bytes}, {a.doffsets, doffsets_h, a.off_bytes}};
-    for (const auto& c : outc) {
-        const cudaError_t e = cudaMemcpyAsync(c.dst, base + c.at, c.bytes, cudaMemcpyDeviceToHost, stream);
-        if (e != cudaSuccess) return cuda_failed(e);
-    }
+    DSA3D_TRY(cudaStreamWaitEvent(hs->out, hs->gather_done, 0));
+    DSA3D_TRY(cudaMemcpyAsync(dq_h, base + a.dq, a.row_bytes, cudaMemcpyDeviceToHost, hs->out));
+    DSA3D_TRY(cudaMemcpyAsync(doffsets_h, base + a.doffsets, a.off_bytes, cudaMemcpyDeviceToHost, hs->out));
+    DSA3D_TRY(cudaEventRecord(hs->out_done, hs->out));
+    DSA3D_TRY(cudaMemcpyAsync(dk_h, base + a.dk, a.row_bytes, cudaMemcpyDeviceToHost, stream));
+    DSA3D_TRY(cudaMemcpyAsync(dv_h, base + a.dv, a.row_bytes, cudaMemcpyDeviceToHost, stream));
+    DSA3D_TRY(cudaStreamWaitEvent(stream, hs->out_done, 0));     // the step is over when `stream` is
+#undef DSA3D_TRY
     return DSA3D_OK;
 }
 

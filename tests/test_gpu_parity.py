@@ -166,3 +166,34 @@ def test_backward_is_the_same_for_every_tiling(tiling, monkeypatch):
 
 def test_large_window_through_the_tile_kernel():
     pu.full_parity(*small_problem(4, 10, 12, 2, 128, (3, 7, 7), BF16, 2.0, 52), (3, 7, 7))
+
+
+# ------------------------------------------------------------- host-buffer entry point
+
+@pytest.mark.parametrize("dtype", [BF16, F32])
+def test_step_host_matches_the_device_entry_points(dtype):
+    """dsa3d_step_host (pinned host buffers in, pinned host buffers out, copies overlapped
+    with the kernels on side streams) must return what dsa3d_forward + dsa3d_backward
+    return on device buffers; run twice to catch a stale event or buffer."""
+    q, k, v, off, dout = small_problem(6, 10, 12, 3, 64, (3, 3, 3), dtype, 1.3, 60)
+    dims = tuple(q.shape)
+    dev = [z.cuda() for z in (q, k, v, off, dout)]
+    out_d, lse_d = pu.gpu_forward(*dev[:4], dims, (3, 3, 3))
+    g_d = pu.gpu_backward(*dev[:4], lse_d, dev[4], dims, (3, 3, 3))
+    pin = lambda z: z.clone().pin_memory()
+    hin = [pin(z) for z in (q, k, v, off, dout)]
+    hout = {n: torch.full_like(q, float("nan")).pin_memory() for n in ("out", "dq", "dk", "dv")}
+    hout["lse"] = torch.full(dims[:4], float("nan")).pin_memory()
+    hout["doff"] = torch.full_like(off, float("nan")).pin_memory()
+    arena = torch.empty(binding.dsa3d_step_host_arena_bytes(*dims, (3, 3, 3), dtype), dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        binding.dsa3d_step_host(*hin, *dims, (3, 3, 3), hout["out"], hout["lse"], hout["dq"], hout["dk"],
+                                hout["dv"], hout["doff"], arena)
+        torch.cuda.synchronize()
+        assert torch.equal(hout["out"], out_d.cpu()) and torch.equal(hout["lse"], lse_d.cpu())
+        assert torch.equal(hout["dq"], g_d[0].cpu()) and torch.equal(hout["doff"], g_d[3].cpu())
+        for got, ref in ((hout["dk"], g_d[1]), (hout["dv"], g_d[2])):
+            ref = ref.cpu().float()
+            assert float((got.float() - ref).abs().max()) <= 2e-2 * float(ref.abs().max())
+        for z in hout.values():
+            z.fill_(float("nan"))
