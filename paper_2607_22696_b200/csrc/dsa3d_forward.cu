@@ -67,6 +67,55 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
         mine.base = 0; mine.mask = 0u; mine.ft = mine.fy = mine.fx = 0.0f;
         if (pb + gl < pr.P) mine = to_sample(pr, make_cell(pr, t, y, x, pb + gl, off_row + (pb + gl) * 3));
         const int cnt = min(LPR, pr.P - pb);
+        if constexpr (LPR >= 8) {
+            // Fixed-window regime: every sample of this chunk (in every group of the warp) sits
+            // exactly on a grid position, so it needs one K row and one V row.  Eight samples
+            // are then taken together - 16 loads in flight instead of 2 - and their eight
+            // logits leave one transposed reduction.
+            const bool lattice = pb + gl >= pr.P || (mine.ft == 0.0f && mine.fy == 0.0f && mine.fx == 0.0f);
+            if (__all_sync(kFullMask, lattice)) {
+                for (int jb = 0; jb < cnt; jb += 8) {
+                    Row kk[8], vv[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int base = __shfl_sync(gmask, mine.base, jb + i, LPR);
+                        const unsigned mk = __shfl_sync(gmask, mine.mask, jb + i, LPR);
+                        kk[i] = E::zero();
+                        vv[i] = E::zero();
+                        if ((mk & 1u) && jb + i < cnt) {            // corner (0,0,0) inside the grid
+                            const T* pk = kh + base * tok_stride;
+                            kk[i] = E::load(pk);
+                            vv[i] = E::load(pk + v_minus_k);
+                        }
+                    }
+                    float dd[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) dd[i] = E::dot(qr, kk[i], 0.0f);
+                    group_reduce8<LPR>(dd, gl, gmask);
+                    float sp[8], mx = -INFINITY;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        sp[i] = __shfl_sync(gmask, dd[0], reduce8_lane<LPR>(i), LPR) * lscale;
+                        if (jb + i >= cnt) sp[i] = -INFINITY;       // no such sample
+                        mx = fmaxf(mx, sp[i]);
+                    }
+                    if (mx > m_run + 8.0f) {
+                        const float corr = exp2f(m_run - mx);
+                        l_run *= corr;
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) acc[e] *= corr;
+                        m_run = mx;
+                    }
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float pe = exp2f(sp[i] - m_run);
+                        l_run += pe;
+                        E::axpy(pe, vv[i], acc);
+                    }
+                }
+                continue;
+            }
+        }
         for (int j = 0; j < cnt; ++j) {
             const Sample s = group_bcast<LPR>(mine, j, gmask);
             const float wt[2] = {1.0f - s.ft, s.ft}, wy[2] = {1.0f - s.fy, s.fy}, wx[2] = {1.0f - s.fx, s.fx};

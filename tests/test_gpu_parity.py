@@ -197,3 +197,18 @@ def test_step_host_matches_the_device_entry_points(dtype):
             assert float((got.float() - ref).abs().max()) <= 2e-2 * float(ref.abs().max())
         for z in hout.values():
             z.fill_(float("nan"))
+
+
+@pytest.mark.parametrize("dtype,d", [(BF16, 128), (BF16, 64), (F32, 32)])
+def test_integer_positions_mixed_with_real_ones(dtype, d):
+    """The forward takes chunks of samples that all sit on grid positions through a batched
+    one-row-per-sample path; the choice is per chunk and per warp, so mix the cases: integer
+    offsets for the first 16 window cells only, and integer offsets for every other query."""
+    q, k, v, off, dout = small_problem(4, 9, 11, 2, d, (3, 3, 3), dtype, 1.4, 70)
+    ints = inputs.uniform_int(off.shape, 71, 3, -2, 2, torch.float32)
+    a = off.clone()
+    a[..., :16, :] = ints[..., :16, :]
+    pu.full_parity(q, k, v, a, dout, (3, 3, 3))
+    b = off.clone().view(-1, 2, 27, 3)
+    b[0::2] = ints.view(-1, 2, 27, 3)[0::2]
+    pu.full_parity(q, k, v, b.view_as(off), dout, (3, 3, 3))
