@@ -140,6 +140,9 @@ WORKLOADS: Dict[str, Workload] = {w.name: w for w in [
     # a 3 GB cut of the 1080p workload (same heads' row size, window and offset spread, inputs
     # still several times the L2) for profiler captures that must stay small
     Workload("profile_small_bf16", 32, 45, 80, 8, 128, (3, 3, 3), _BF16, 2.0, 5),
+    # the window the paper itself runs, (3,7,7) = 147 samples, on 64 frames of the 1080p grid
+    # (at 256 frames the offsets alone would be 59 GB)
+    Workload("1080p_64f_w377_bf16", 64, 68, 120, 16, 128, (3, 7, 7), _BF16, 2.0, 6),
 ] + [
     Workload(f"sweep_w{kt}{kh}{kw}_{kind}", 64, 45, 80, 16, 128, (kt, kh, kw), _BF16,
              3.0 if kind == "normal" else 0.0, 4, offsets=kind)

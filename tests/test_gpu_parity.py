@@ -143,6 +143,10 @@ def test_config_1080p_256f_bf16_forward_backward():
                                                ((255, 67, 118), (256, 68, 120))])
 
 
+def test_paper_window_3x7x7_on_the_1080p_grid():
+    run_large("1080p_64f_w377_bf16", [0, 15], [((0, 0, 0), (1, 1, 2)), ((32, 33, 60), (33, 34, 61))], n_random=256)
+
+
 @pytest.mark.parametrize("kind", ["zero", "int", "normal"])
 @pytest.mark.parametrize("window", ["222", "333", "355"])
 def test_config_sweep_720p_grid(window, kind):
