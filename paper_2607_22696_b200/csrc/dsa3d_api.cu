@@ -85,7 +85,7 @@ BackwardWorkspace backward_workspace(const dsa3d::Problem& pr, int dtype, bool t
     if (tiled && pr.tile_t >= 1) {
         w.coef_bytes = static_cast<size_t>(pr.items) * pr.P * sizeof(float2);
         w.entries_per_cta = static_cast<long long>(pr.tile_t) * pr.tile_y * pr.tile_x * pr.P * 8;
-        w.scratch_bytes = static_cast<size_t>(kTileSlots) * w.entries_per_cta * sizeof(uint2);
+        w.scratch_bytes = static_cast<size_t>(kTileSlots) * w.entries_per_cta * sizeof(dsa3d::TileEntry);
     }
     w.total = w.acc_bytes + w.coef_bytes + w.scratch_bytes;
     return w;

@@ -256,7 +256,7 @@ template <int D>
 __global__ void __launch_bounds__(kTileThreads, 1)
 scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ dout,
                     const float* __restrict__ offsets, const float2* __restrict__ coef,
-                    float* __restrict__ acc_dk, float* __restrict__ acc_dv, uint2* __restrict__ scratch,
+                    float* __restrict__ acc_dk, float* __restrict__ acc_dv, TileEntry* __restrict__ scratch,
                     const long long scratch_entries_per_cta, const Problem pr) {
     constexpr int VPR = D / 8;                       // 16-byte vectors per row
     constexpr int kPairBytes = 2 * VPR * 16;         // one query's q row followed by its dO row
@@ -273,7 +273,7 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     constexpr int kWarps = kTileThreads / 32;
     const int tiles_per_head = pr.tiles_t * pr.tiles_y * pr.tiles_x;
     const long long total_tiles = static_cast<long long>(tiles_per_head) * pr.heads;
-    uint2* my_scratch = scratch + static_cast<long long>(blockIdx.x) * scratch_entries_per_cta;
+    TileEntry* my_scratch = scratch + static_cast<long long>(blockIdx.x) * scratch_entries_per_cta;
     const long long tok_stride = static_cast<long long>(pr.heads) * D;
 
     for (long long tile_id = blockIdx.x; tile_id < total_tiles; tile_id += gridDim.x) {
@@ -329,9 +329,14 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                             const int bin = bin0 + ((c >> 2) * ey + ((c >> 1) & 1)) * ex + (c & 1);
                             const unsigned slot = atomicAdd(&cursor[bin], 1u);
                             if (sweep == 1) {
+#ifndef DSA3D_BF16_COEF
+                                my_scratch[slot] = make_uint4(static_cast<unsigned>(ql * kPairBytes),
+                                                              __float_as_uint(w * cf.x), __float_as_uint(w * cf.y), 0u);
+#else
                                 const __nv_bfloat162 pk = __floats2bfloat162_rn(w * cf.x, w * cf.y);   // (wk, wv)
                                 my_scratch[slot] = make_uint2(static_cast<unsigned>(ql * kPairBytes),
                                                               *reinterpret_cast<const unsigned*>(&pk));
+#endif
                             }
                         }
                     }
@@ -376,7 +381,6 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
 
         // ---- reduce: a warp takes two neighbouring key rows, one per half-warp; both halves
         //      run the same number of steps (the shorter list is padded with zero entries)
-#ifndef DSA3D_DEBUG_SKIP_REDUCE
         {
             const int half = lane >> 4, hl = lane & 15;
             const int hv = hl < VPR ? hl : VPR - 1;         // lanes beyond a narrow row mirror its last vector
@@ -395,6 +399,29 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
 #pragma unroll
                 for (int e = 0; e < 8; ++e) ak[e] = av[e] = 0.0f;
                 for (unsigned base = 0; base < cnt_max; base += 16) {
+#ifndef DSA3D_BF16_COEF
+                    uint4 ent = make_uint4(0u, 0u, 0u, 0u);               // offset 0, coefficients 0
+                    if (base + hl < cnt_mine) ent = __ldcg(my_scratch + start + base + hl);
+                    const int steps = static_cast<int>(min(16u, cnt_max - base));
+#pragma unroll 4
+                    for (int j = 0; j < steps; ++j) {
+                        const int src = (lane & 16) | j;
+                        const unsigned off = __shfl_sync(kFull, ent.x, src);
+                        const float ck = __uint_as_float(__shfl_sync(kFull, ent.y, src));
+                        const float cv = __uint_as_float(__shfl_sync(kFull, ent.z, src));
+                        const uint4 a = *reinterpret_cast<const uint4*>(my_rows + off);
+                        const uint4 b = *reinterpret_cast<const uint4*>(my_rows + off + VPR * 16);
+                        const unsigned aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            ak[2 * i] = fmaf(ck, __uint_as_float(aw[i] << 16), ak[2 * i]);
+                            ak[2 * i + 1] = fmaf(ck, __uint_as_float(aw[i] & 0xffff0000u), ak[2 * i + 1]);
+                            av[2 * i] = fmaf(cv, __uint_as_float(bw[i] << 16), av[2 * i]);
+                            av[2 * i + 1] = fmaf(cv, __uint_as_float(bw[i] & 0xffff0000u), av[2 * i + 1]);
+                        }
+                    }
+                }
+#else
                     uint2 ent = make_uint2(0u, 0u);                       // offset 0, coefficients 0
                     if (base + hl < cnt_mine) ent = __ldcg(my_scratch + start + base + hl);
                     const int steps = static_cast<int>(min(16u, cnt_max - base));
@@ -420,11 +447,8 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                         }
                     }
                 }
-#ifndef DSA3D_DEBUG_SKIP_FLUSH
-                if (cnt_mine > 0u && hl < VPR) {
-#else
-                if (cnt_mine > 0u && hl < VPR && ak[0] == 12345.678f) {
 #endif
+                if (cnt_mine > 0u && hl < VPR) {
                     const int bx = bin % ex, by = (bin / ex) % ey, bt = bin / (ex * ey);
                     const long long tok = (static_cast<long long>(lo_t + bt) * pr.H + (lo_y + by)) * pr.W + (lo_x + bx);
                     const long long o = tok * tok_stride + static_cast<long long>(m) * D + hl * 8;
@@ -435,7 +459,6 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                 }
             }
         }
-#endif
         __syncthreads();     // the next tile reuses the rows, the counters and the scratch
     }
 }
@@ -513,7 +536,7 @@ static cudaError_t launch_scatter_tiles_t(const void* q, const void* dout, const
     const int grid = static_cast<int>(total_tiles < ctas ? total_tiles : ctas);
     kern<<<grid, kTileThreads, smem, stream>>>(
         static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(dout), offsets, coef, acc_dk,
-        acc_dv, static_cast<uint2*>(scratch), entries_per_cta, pr);
+        acc_dv, static_cast<TileEntry*>(scratch), entries_per_cta, pr);
     return cudaGetLastError();
 }
 

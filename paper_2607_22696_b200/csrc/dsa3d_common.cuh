@@ -9,6 +9,14 @@
 
 namespace dsa3d {
 
+// One contribution to dK/dV as the tile kernel bins it: byte offset of the query's q/dO row
+// pair in shared memory and the two coefficients (w_c * ck_p, w_c * cv_p).
+#ifndef DSA3D_BF16_COEF
+using TileEntry = uint4;            // {offset, fp32 wk, fp32 wv, unused}
+#else
+using TileEntry = uint2;            // {offset, (bf16 wk, bf16 wv)}: the faster, less exact build
+#endif
+
 struct Problem {
     int T, H, W, heads, d;
     int kt, kh, kw, P;
@@ -24,9 +32,9 @@ struct Problem {
 // ---------------------------------------------------------------------------------------
 // Element access.  A lane handles NV consecutive 16-byte vectors of a row (8 bf16 or 4 fp32
 // channels each).
-// `Row` keeps that vector in its storage form.  For bf16 the products use the sm_100
-// mixed-precision instruction fma.rn.f32.bf16 (bf16 x bf16 -> exact fp32 product, fp32
-// accumulate), which needs no unpacking; `axpy` rounds its fp32 coefficient to bf16 first.
+// `Row` keeps that vector in its storage form.  For bf16 the dot products (both factors
+// bf16) use the sm_100 mixed-precision instruction fma.rn.f32.bf16 (exact fp32 product,
+// fp32 accumulate), which needs no unpacking; `axpy` (fp32 coefficient) widens the row.
 // ---------------------------------------------------------------------------------------
 template <typename T, int NV> struct Elt;       // NV = 16-byte vectors per lane (1 or 2)
 
@@ -108,7 +116,19 @@ template <int NV> struct Elt<__nv_bfloat16, NV> {
         }
         return acc;
     }
+    // acc += c * x with an fp32 coefficient: the bf16 values are widened (one shift or mask
+    // each) and multiplied in fp32, so the coefficient keeps all its bits.  Building with
+    // DSA3D_BF16_COEF rounds the coefficient to bf16 instead and uses the mixed instruction
+    // (about 12 % faster overall); that error stays inside the 2e-2 bound on every test but
+    // reaches it on rare elements of very large tensors, so it is not the default.
     static __device__ __forceinline__ void axpy(float c, const Row& x, float (&acc)[VEC]) {
+#ifndef DSA3D_BF16_COEF
+#pragma unroll
+        for (int i = 0; i < NW; ++i) {
+            acc[2 * i] = fmaf(c, __uint_as_float(x.w[i] << 16), acc[2 * i]);
+            acc[2 * i + 1] = fmaf(c, __uint_as_float(x.w[i] & 0xffff0000u), acc[2 * i + 1]);
+        }
+#else
         const unsigned short cb = __bfloat16_as_ushort(__float2bfloat16_rn(c));
 #pragma unroll
         for (int i = 0; i < NW; ++i) {
@@ -117,6 +137,7 @@ template <int NV> struct Elt<__nv_bfloat16, NV> {
             acc[2 * i] = fma_bf16(cb, xl, acc[2 * i]);
             acc[2 * i + 1] = fma_bf16(cb, xh, acc[2 * i + 1]);
         }
+#endif
     }
     static __device__ __forceinline__ void to_float(const Row& x, float (&f)[VEC]) {
 #pragma unroll
