@@ -46,10 +46,10 @@ FALLBACK_HBM_GBS = 6650.0
 # capture per kernel on the profile_small_bf16 workload (profiles/*_profile_small_bf16.md).
 # Every kernel's traffic is proportional to the number of items, so a launch on another
 # workload with the same d and window is reported as items x these figures.
-NCU_DRAM_BYTES_PER_ITEM = {"forward_kernel": 1525.0, "backward_kernel": 2986.0, "scatter_tile_kernel": 8280.0}
+NCU_DRAM_BYTES_PER_ITEM = {"forward_kernel": 1525.0, "backward_kernel": 2991.0, "scatter_tile_kernel": 12902.0}
 # L2 -> SM bytes per item of the forward's corner gathers (l1tex__m_xbar2l1tex_read_bytes.sum
 # of the same capture / items): what is left of the 110,592 gathered bytes after L1 hits.
-NCU_L2_TO_SM_BYTES_PER_ITEM = {"forward_kernel": 83021.0, "backward_kernel": 94521.0}
+NCU_L2_TO_SM_BYTES_PER_ITEM = {"forward_kernel": 82380.0, "backward_kernel": 95482.0}
 NCU_RED_BYTES_PER_ITEM = {"scatter_tile_kernel": 23470.0}      # lts red sectors x 32 B / items
 
 
