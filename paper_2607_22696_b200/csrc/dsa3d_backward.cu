@@ -22,11 +22,12 @@
 //   rows around the tile, ~10 contributions per row.  Sending each one to L2 as a 512-byte
 //   fp32 reduction is what bounds the simple scheme (L2 reduction throughput), so the tile
 //   kernel sums them on chip first: it bins the (query, sample, corner) contributions of
-//   the tile by target row (counting sort, counters in shared memory, 8-byte entries in a
-//   per-CTA global scratch that stays in L2), then each half-warp owns a row, walks its
-//   entries, accumulates  coefficient x q-row  and  coefficient x dO-row  in fp32 registers
-//   from the tile's q/dO rows held in shared memory, and issues ONE reduction per row and
-//   tensor.  Coefficients are rounded to bf16 for the mixed-precision FMA.
+//   the tile by target row (counting sort, counters in shared memory, 16-byte entries
+//   {row offset, fp32 coefficient pair} in a per-CTA global scratch), then each half-warp
+//   owns a row, walks its entries, accumulates  coefficient x q-row  and  coefficient x
+//   dO-row  in fp32 registers from the tile's q/dO rows held in shared memory, and issues
+//   ONE reduction per row and tensor.  (Built with DSA3D_BF16_COEF the entries are 8 bytes
+//   with bf16 coefficients and the products use the mixed-precision FMA.)
 #include "dsa3d_common.cuh"
 #include "dsa3d_kernels.h"
 
