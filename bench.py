@@ -381,11 +381,42 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
+def host_memory_available() -> int:
+    """Bytes of host memory this process can still take: the smaller of what the kernel
+    reports as available and what the container's memory cgroup leaves."""
+    avail = None
+    try:
+        with open("/proc/meminfo") as f:
+            for line in f:
+                if line.startswith("MemAvailable:"):
+                    avail = int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    try:
+        limit = open("/sys/fs/cgroup/memory.max").read().strip()
+        used = int(open("/sys/fs/cgroup/memory.current").read().strip())
+        if limit != "max":
+            room = int(limit) - used
+            avail = room if avail is None else min(avail, room)
+    except (OSError, ValueError):
+        pass
+    return avail if avail is not None else 0
+
+
 def run_e2e(args, wl, t, dims, dev, barrier, max_ranks, world):
     """Forward + backward through dsa3d_step_host: inputs start in pinned host memory and
     every output ends in pinned host memory, each step."""
     from paper_2607_22696_b200 import binding
     names_in = ["q", "k", "v", "offsets", "dout"]
+    # The step keeps every input and every output in page-locked host memory (about twice the
+    # input bytes per rank).  Page-locking more than the host can spare takes the machine
+    # down, so the leg is skipped, on all ranks together, unless every rank's share fits
+    # with a third to spare.
+    need = 2 * sum(t[n].numel() * t[n].element_size() for n in names_in)
+    fits = 1.0 if host_memory_available() >= 1.5 * need * world else 0.0
+    if -max_ranks(-fits) < 1.0:                           # min over ranks
+        return {"value": None, "unit": UNIT, "skipped": f"needs {need * world / 1e9:.0f} GB of pinned host "
+                "memory over all ranks; not available", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     host_in = {}
     for n in names_in:
         h = torch.empty(t[n].shape, dtype=t[n].dtype, pin_memory=True)
