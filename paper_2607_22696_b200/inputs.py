@@ -92,8 +92,9 @@ def uniform_int(shape, seed: int, tensor_id: int, lo: int, hi: int, dtype: torch
 
 @dataclasses.dataclass(frozen=True)
 class Workload:
-    """One synthetic 3D-DSA problem.  ``offsets`` is 'normal', 'zero' or 'int' (uniform
-    integers in [-int_range, int_range])."""
+    """One synthetic 3D-DSA problem.  ``offsets`` is 'normal', 'zero', 'int' (uniform
+    integers in [-int_range, int_range]) or 'drift' (one velocity per (token, head) plus a
+    small per-sample jitter)."""
     name: str
     T: int
     H: int
@@ -143,6 +144,9 @@ WORKLOADS: Dict[str, Workload] = {w.name: w for w in [
     # the window the paper itself runs, (3,7,7) = 147 samples, on 64 frames of the 1080p grid
     # (at 256 frames the offsets alone would be 59 GB)
     Workload("1080p_64f_w377_bf16", 64, 68, 120, 16, 128, (3, 7, 7), _BF16, 2.0, 6),
+    # not a BASELINE config: offsets with the coherence of a motion field (structured-motion
+    # data of the paper's quality ablation), same grid and spread as the 1080p workload
+    Workload("1080p_256f_drift_bf16", 256, 68, 120, 16, 128, (3, 3, 3), _BF16, 2.0, 7, offsets="drift"),
 ] + [
     Workload(f"sweep_w{kt}{kh}{kw}_{kind}", 64, 45, 80, 16, 128, (kt, kh, kw), _BF16,
              3.0 if kind == "normal" else 0.0, 4, offsets=kind)
@@ -160,6 +164,13 @@ def make_offsets(wl: Workload, device="cpu", frames=None) -> torch.Tensor:
     if wl.offsets == "int":
         return uniform_int(shape, wl.seed, TENSOR_IDS["offsets"], -wl.int_range, wl.int_range,
                            torch.float32, device, first=first)
+    if wl.offsets == "drift":
+        # every sample of a (token, head) shares one velocity ~N(0, sigma^2) per axis and adds
+        # its own small jitter ~N(0, 0.3^2): what offsets that follow motion would look like
+        vel = normal((t1 - t0, wl.H, wl.W, wl.heads, 1, 3), wl.seed, TENSOR_IDS["offsets"] + 16, wl.sigma,
+                     torch.float32, device, first=t0 * wl.H * wl.W * wl.heads * 3)
+        jit = normal(shape, wl.seed, TENSOR_IDS["offsets"], 0.3, torch.float32, device, first=first)
+        return jit.add_(vel)
     return normal(shape, wl.seed, TENSOR_IDS["offsets"], wl.sigma, torch.float32, device, first=first)
 
 
