@@ -75,9 +75,9 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
     const int ch = gl * VEC;
     const float scale = rsqrtf(static_cast<float>(D));
     const long long tok_stride = static_cast<long long>(pr.heads) * D;
-    const int sx = static_cast<int>(tok_stride);
-    const int sy = pr.W * sx;
-    const int st = pr.H * sy;
+    const long long sx = tok_stride;
+    const long long sy = static_cast<long long>(pr.W) * sx;      // 64-bit once, so that the pointer
+    const long long st = static_cast<long long>(pr.H) * sy;      // arithmetic below needs no widening
 
     const Row qr = E::load(q + row * D + ch);
     const Row dor = E::load(dout + row * D + ch);

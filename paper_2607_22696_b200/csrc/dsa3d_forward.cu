@@ -47,9 +47,9 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
     const long long row = (n * pr.heads + m);               // row index into [N*heads, ...]
     const int ch = gl * VEC;
     const long long tok_stride = static_cast<long long>(pr.heads) * D;
-    const int sx = static_cast<int>(tok_stride);            // element stride between x neighbours
-    const int sy = pr.W * sx;
-    const int st = pr.H * sy;                                // < 2^31: checked by the host
+    const long long sx = tok_stride;                         // element stride between x neighbours
+    const long long sy = static_cast<long long>(pr.W) * sx;      // 64-bit once, so that the pointer
+    const long long st = static_cast<long long>(pr.H) * sy;      // arithmetic below needs no widening                                // < 2^31: checked by the host
 
     const Row qr = E::load(q + row * D + ch);
     const float lscale = rsqrtf(static_cast<float>(D)) * kLog2e;    // logits in log2 units
