@@ -83,7 +83,8 @@ BackwardWorkspace backward_workspace(const dsa3d::Problem& pr, int dtype, bool t
     if (dtype != DSA3D_BF16) return w;
     w.acc_bytes = static_cast<size_t>(pr.items) * pr.d * sizeof(float) * 2;
     if (tiled && pr.tile_t >= 1) {
-        w.coef_bytes = static_cast<size_t>(pr.items) * pr.P * sizeof(float2);
+        // rounded up so that the 16-byte bin entries behind it stay 16-byte aligned
+        w.coef_bytes = (static_cast<size_t>(pr.items) * pr.P * sizeof(float2) + 255) & ~static_cast<size_t>(255);
         w.entries_per_cta = static_cast<long long>(pr.tile_t) * pr.tile_y * pr.tile_x * pr.P * 8;
         w.scratch_bytes = static_cast<size_t>(kTileSlots) * w.entries_per_cta * sizeof(dsa3d::TileEntry);
     }

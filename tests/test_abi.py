@@ -45,14 +45,18 @@ def test_status_strings(lib):
 def test_workspace_size(lib):
     win = (ctypes.c_int * 3)(3, 3, 3)
     assert lib.dsa3d_backward_workspace_bytes(4, 8, 8, 2, 32, win, 0) == 0
-    # bf16: fp32 dK/dV accumulators + two fp32 coefficients per sample + the tile bins
+    # bf16: fp32 dK/dV accumulators + two fp32 coefficients per sample (section rounded up to
+    # 256 bytes) + the tile bins, whose size depends on the tiling only
+    up = lambda x: (x + 255) // 256 * 256
     small = lib.dsa3d_backward_workspace_bytes(4, 8, 8, 2, 32, win, 1)
-    assert small >= 256 * 2 * 32 * 4 * 2 + 256 * 2 * 27 * 8
+    small_fixed = 256 * 2 * 32 * 4 * 2 + up(256 * 2 * 27 * 8)
+    assert small > small_fixed
     big = lib.dsa3d_backward_workspace_bytes(256, 68, 120, 16, 128, win, 1)
     items = 2088960 * 16
-    assert big >= items * 128 * 4 * 2 + items * 27 * 8
-    assert big - (items * 128 * 4 * 2 + items * 27 * 8) == small - (256 * 2 * 32 * 4 * 2 + 256 * 2 * 27 * 8)
+    assert big - (items * 128 * 4 * 2 + up(items * 27 * 8)) == small - small_fixed
     assert big < 45 * 10**9
+    odd = lib.dsa3d_backward_workspace_bytes(5, 7, 9, 3, 32, win, 1)       # 945 items: unaligned sizes
+    assert (odd - (small - small_fixed)) % 256 == 0
     assert lib.dsa3d_backward_workspace_bytes(4, 8, 8, 2, 48, win, 1) == 0      # rejected shape
 
 
