@@ -290,7 +290,7 @@ int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const flo
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     char* base = static_cast<char*>(arena);
     HostStep* hs = host_step_resources();
-    if (!hs) return DSA3D_ERR_CUDA;
+    if (!hs) return cuda_failed(cudaGetLastError());     // side streams / events could not be created
     cudaError_t e;
 #define DSA3D_TRY(call)                         \
     do {                                        \
