@@ -93,6 +93,23 @@ size_t dsa3d_backward_workspace_bytes(int T, int H, int W, int heads, int d,
                                       const int window[3], int dtype);
 
 /*
+ * Batched forms (the paper trains with batch 1; a batch here is `batch` independent videos
+ * stored back to back, [batch, T, H, W, heads, ...] for every tensor).  Videos never see
+ * each other's keys: each is the operator of Eq. 1 on its own grid.  The calls run the
+ * single-video kernels once per video on `stream`; the backward reuses one workspace of
+ * dsa3d_backward_workspace_bytes(...) bytes for all of them.  Every per-video slice must
+ * itself be 16-byte aligned (it is whenever T*H*W*heads is a multiple of 4).
+ */
+int dsa3d_forward_batch(const void* q, const void* k, const void* v, const float* offsets,
+                        int batch, int T, int H, int W, int heads, int d, const int window[3],
+                        void* out, float* lse, int dtype, void* stream);
+int dsa3d_backward_batch(const void* q, const void* k, const void* v, const float* offsets,
+                         const float* lse, const void* dout,
+                         int batch, int T, int H, int W, int heads, int d, const int window[3],
+                         void* dq, void* dk, void* dv, float* doffsets,
+                         void* workspace, size_t workspace_bytes, int dtype, void* stream);
+
+/*
  * One whole step from HOST buffers: copies q, k, v, offsets, dout to the device, runs the
  * forward and the backward above, and copies out, lse, dq, dk, dv, doffsets back.  This is
  * the operator of Eq. 1 (second term) and its gradient exactly as in dsa3d_forward /

@@ -65,6 +65,10 @@ def load():
     lib.dsa3d_probe_red.argtypes = [p, sz, i, dptr, p]
     lib.dsa3d_probe_fma.restype = i
     lib.dsa3d_probe_fma.argtypes = [p, i, i, dptr, p]
+    lib.dsa3d_forward_batch.restype = i
+    lib.dsa3d_forward_batch.argtypes = [p, p, p, p, i, i, i, i, i, i, win, p, p, i, p]
+    lib.dsa3d_backward_batch.restype = i
+    lib.dsa3d_backward_batch.argtypes = [p, p, p, p, p, p, i, i, i, i, i, i, win, p, p, p, p, p, sz, i, p]
     lib.dsa3d_status_string.restype = ctypes.c_char_p
     lib.dsa3d_status_string.argtypes = [i]
     lib.dsa3d_last_cuda_error.restype = i
@@ -264,3 +268,35 @@ def dsa3d_probe_fma(seed: torch.Tensor, kind: int, iters: int = 4096) -> float:
         _check(lib.dsa3d_probe_fma(_ptr(seed, "seed"), iters, kind, ctypes.byref(work), _stream(None)))
     ms = _timed(launch)
     return work.value / ms / 1e9
+
+
+def dsa3d_forward_batch(q, k, v, offsets, batch, T, H, W, heads, d, window, out, lse, dtype=None,
+                        stream=None) -> None:
+    """Forward of `batch` independent videos stored back to back; see include/dsa3d.h."""
+    lib = load()
+    dt = q.dtype if dtype is None else dtype
+    code = _DTYPES[dt] if isinstance(dt, torch.dtype) else int(dt)
+    n = batch * T * H * W * heads
+    P = int(window[0]) * int(window[1]) * int(window[2])
+    _check(lib.dsa3d_forward_batch(
+        _ptr(q, "q", n * d), _ptr(k, "k", n * d), _ptr(v, "v", n * d),
+        _ptr(offsets, "offsets", n * P * 3, torch.float32), batch, T, H, W, heads, d, _window(window),
+        _ptr(out, "out", n * d), _ptr(lse, "lse", n, torch.float32), code, _stream(stream)))
+
+
+def dsa3d_backward_batch(q, k, v, offsets, lse, dout, batch, T, H, W, heads, d, window, dq, dk, dv, doffsets,
+                         workspace=None, dtype=None, stream=None) -> None:
+    """Backward of `batch` independent videos stored back to back; see include/dsa3d.h."""
+    lib = load()
+    dt = q.dtype if dtype is None else dtype
+    code = _DTYPES[dt] if isinstance(dt, torch.dtype) else int(dt)
+    n = batch * T * H * W * heads
+    P = int(window[0]) * int(window[1]) * int(window[2])
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.dsa3d_backward_batch(
+        _ptr(q, "q", n * d), _ptr(k, "k", n * d), _ptr(v, "v", n * d),
+        _ptr(offsets, "offsets", n * P * 3, torch.float32), _ptr(lse, "lse", n, torch.float32),
+        _ptr(dout, "dout", n * d), batch, T, H, W, heads, d, _window(window),
+        _ptr(dq, "dq", n * d), _ptr(dk, "dk", n * d), _ptr(dv, "dv", n * d),
+        _ptr(doffsets, "doffsets", n * P * 3, torch.float32), _ptr(workspace, "workspace"), nbytes, code,
+        _stream(stream)))

@@ -348,6 +348,53 @@ int dsa3d_set_profile_events(void* fwd_start, void* fwd_stop, void* bwd_start, v
     return DSA3D_OK;
 }
 
+// A batch is `batch` independent videos stored back to back; each one is a problem of its
+// own (no sample of one video ever reads another), so the batched entry points run the
+// single-video kernels once per video on the same stream, reusing one workspace.
+int dsa3d_forward_batch(const void* q, const void* k, const void* v, const float* offsets, int batch, int T,
+                        int H, int W, int heads, int d, const int window[3], void* out, float* lse, int dtype,
+                        void* stream) {
+    if (batch < 1) return DSA3D_ERR_BAD_SHAPE;
+    if (!q || !k || !v || !offsets || !out || !lse) return DSA3D_ERR_NULL_POINTER;
+    dsa3d::Problem pr;
+    const int rc = make_problem(T, H, W, heads, d, window, dtype, pr);
+    if (rc != DSA3D_OK) return rc;
+    const size_t rows = static_cast<size_t>(pr.items) * pr.d * (dtype == DSA3D_BF16 ? 2 : 4);
+    const size_t offs = static_cast<size_t>(pr.items) * pr.P * 3;
+    for (int b = 0; b < batch; ++b) {
+        const int st = dsa3d_forward(static_cast<const char*>(q) + b * rows, static_cast<const char*>(k) + b * rows,
+                                     static_cast<const char*>(v) + b * rows, offsets + b * offs, T, H, W, heads, d,
+                                     window, static_cast<char*>(out) + b * rows, lse + b * static_cast<size_t>(pr.items),
+                                     dtype, stream);
+        if (st != DSA3D_OK) return st;
+    }
+    return DSA3D_OK;
+}
+
+int dsa3d_backward_batch(const void* q, const void* k, const void* v, const float* offsets, const float* lse,
+                         const void* dout, int batch, int T, int H, int W, int heads, int d, const int window[3],
+                         void* dq, void* dk, void* dv, float* doffsets, void* workspace, size_t workspace_bytes,
+                         int dtype, void* stream) {
+    if (batch < 1) return DSA3D_ERR_BAD_SHAPE;
+    if (!q || !k || !v || !offsets || !lse || !dout || !dq || !dk || !dv || !doffsets)
+        return DSA3D_ERR_NULL_POINTER;
+    dsa3d::Problem pr;
+    const int rc = make_problem(T, H, W, heads, d, window, dtype, pr);
+    if (rc != DSA3D_OK) return rc;
+    const size_t rows = static_cast<size_t>(pr.items) * pr.d * (dtype == DSA3D_BF16 ? 2 : 4);
+    const size_t offs = static_cast<size_t>(pr.items) * pr.P * 3;
+    for (int b = 0; b < batch; ++b) {
+        const int st = dsa3d_backward(
+            static_cast<const char*>(q) + b * rows, static_cast<const char*>(k) + b * rows,
+            static_cast<const char*>(v) + b * rows, offsets + b * offs, lse + b * static_cast<size_t>(pr.items),
+            static_cast<const char*>(dout) + b * rows, T, H, W, heads, d, window, static_cast<char*>(dq) + b * rows,
+            static_cast<char*>(dk) + b * rows, static_cast<char*>(dv) + b * rows, doffsets + b * offs, workspace,
+            workspace_bytes, dtype, stream);
+        if (st != DSA3D_OK) return st;
+    }
+    return DSA3D_OK;
+}
+
 const char* dsa3d_status_string(int status) {
     switch (status) {
         case DSA3D_OK: return "success";

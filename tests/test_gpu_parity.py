@@ -216,3 +216,29 @@ def test_integer_positions_mixed_with_real_ones(dtype, d):
     b = off.clone().view(-1, 2, 27, 3)
     b[0::2] = ints.view(-1, 2, 27, 3)[0::2]
     pu.full_parity(q, k, v, b.view_as(off), dout, (3, 3, 3))
+
+
+# ------------------------------------------------------------------------ batched forms
+
+def test_batched_entry_points_equal_one_call_per_video():
+    """Two different videos stored back to back must come out exactly as from two single
+    calls (per-query results bitwise; dk/dv up to the order of their atomic sums)."""
+    vids = [small_problem(4, 8, 10, 2, 64, (3, 3, 3), BF16, 1.2, seed) for seed in (80, 81)]
+    dims, win = (4, 8, 10, 2, 64), (3, 3, 3)
+    cat = [torch.stack([vids[0][i], vids[1][i]]).cuda() for i in range(5)]       # q, k, v, off, dout
+    out = torch.empty_like(cat[0])
+    lse = torch.empty(2, *dims[:4], dtype=torch.float32, device="cuda")
+    binding.dsa3d_forward_batch(*cat[:4], 2, *dims, win, out, lse)
+    dq, dk, dv = (torch.full_like(cat[0], float("nan")) for _ in range(3))
+    doff = torch.full_like(cat[3], float("nan"))
+    ws = torch.empty(binding.dsa3d_backward_workspace_bytes(*dims, win, BF16), dtype=torch.uint8, device="cuda")
+    binding.dsa3d_backward_batch(*cat[:4], lse, cat[4], 2, *dims, win, dq, dk, dv, doff, ws)
+    torch.cuda.synchronize()
+    for b in range(2):
+        single = [z.cuda() for z in vids[b]]
+        o1, l1 = pu.gpu_forward(*single[:4], dims, win)
+        g1 = pu.gpu_backward(*single[:4], l1, single[4], dims, win)
+        assert torch.equal(out[b], o1) and torch.equal(lse[b], l1)
+        assert torch.equal(dq[b], g1[0]) and torch.equal(doff[b], g1[3])
+        for got, ref in ((dk[b], g1[1]), (dv[b], g1[2])):
+            assert float((got.float() - ref.float()).abs().max()) <= 2e-2 * float(ref.float().abs().max())
