@@ -242,3 +242,46 @@ def test_batched_entry_points_equal_one_call_per_video():
         assert torch.equal(dq[b], g1[0]) and torch.equal(doff[b], g1[3])
         for got, ref in ((dk[b], g1[1]), (dv[b], g1[2])):
             assert float((got.float() - ref.float()).abs().max()) <= 2e-2 * float(ref.float().abs().max())
+
+
+# ----------------------------------------------------------------- stays inside its buffers
+
+@pytest.mark.parametrize("dtype", [BF16, F32])
+def test_nothing_is_written_outside_the_output_buffers(dtype):
+    """Every output and the workspace are carved out of one arena with 4 KiB guard bands
+    between them; after a forward and a backward on a ragged problem with many samples
+    outside the grid the guard bands must still hold their pattern."""
+    q, k, v, off, dout = small_problem(5, 7, 9, 3, 64, (3, 3, 3), dtype, 2.5, 90)
+    dims, win = tuple(q.shape), (3, 3, 3)
+    dev = [z.cuda() for z in (q, k, v, off, dout)]
+    elt = q.element_size()
+    n_rows, n_off, n_lse = q.numel() * elt, off.numel() * 4, q.numel() // dims[4] * 4
+    ws_bytes = max(binding.dsa3d_backward_workspace_bytes(*dims, win, dtype), 16)
+    sizes = {"out": n_rows, "lse": n_lse, "dq": n_rows, "dk": n_rows, "dv": n_rows, "doff": n_off, "ws": ws_bytes}
+    guard, at, spans = 4096, 4096, {}
+    for name, nbytes in sizes.items():
+        spans[name] = (at, nbytes)
+        at += (nbytes + 255) // 256 * 256 + guard
+    arena = torch.full((at,), 0xA5, dtype=torch.uint8, device="cuda")
+
+    def view(name, like_dtype, shape):
+        start, nbytes = spans[name]
+        return arena[start:start + nbytes].view(like_dtype).view(shape)
+
+    out, lse = view("out", dtype, dims), view("lse", torch.float32, dims[:4])
+    dq, dk, dv = (view(n, dtype, dims) for n in ("dq", "dk", "dv"))
+    doff, ws = view("doff", torch.float32, off.shape), view("ws", torch.uint8, (ws_bytes,))
+    binding.dsa3d_forward(*dev[:4], *dims, win, out, lse)
+    binding.dsa3d_backward(*dev[:4], lse, dev[4], *dims, win, dq, dk, dv, doff, ws)
+    torch.cuda.synchronize()
+    inside = torch.zeros(at, dtype=torch.bool, device="cuda")
+    for start, nbytes in spans.values():
+        inside[start:start + nbytes] = True
+    assert bool((arena[~inside] == 0xA5).all())
+    o_ref, _ = oracle_forward(q, k, v, off, dims, win)
+    pu.assert_close("out", out, o_ref, dtype)
+
+
+def oracle_forward(q, k, v, off, dims, win):
+    import oracle
+    return oracle.forward(q, k, v, off, *dims, win)
