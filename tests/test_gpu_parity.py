@@ -138,6 +138,27 @@ def test_config_720p_bf16_forward_backward():
                                           ((63, 44, 78), (64, 45, 80))])
 
 
+def test_config_720p_bf16_every_element():
+    """The whole 720p-class workload (708 M elements per tensor) against a full oracle run
+    (about a minute on 16 host cores): every element of every output inside the bound."""
+    wl = inputs.WORKLOADS["720p_bf16"]
+    dims = (wl.T, wl.H, wl.W, wl.heads, wl.d)
+    t = inputs.make_inputs(wl, "cuda")
+    out, lse = pu.gpu_forward(t["q"], t["k"], t["v"], t["offsets"], dims, wl.window)
+    grads = pu.gpu_backward(t["q"], t["k"], t["v"], t["offsets"], lse, t["dout"], dims, wl.window)
+    host = {n: z.cpu() for n, z in t.items()}
+    del t
+    torch.cuda.empty_cache()
+    import oracle
+    o_ref, l_ref = oracle.forward(host["q"], host["k"], host["v"], host["offsets"], *dims, wl.window)
+    pu.assert_close("out", out, o_ref, wl.dtype)
+    pu.assert_close("lse", lse, l_ref, wl.dtype)
+    del o_ref, l_ref, out, lse
+    refs = oracle.backward(host["q"], host["k"], host["v"], host["offsets"], host["dout"], *dims, wl.window)
+    for name, got, ref in zip(("dq", "dk", "dv", "doffsets"), grads, refs):
+        pu.assert_close(name, got, ref, wl.dtype, backward=True)
+
+
 def test_config_1080p_256f_bf16_forward_backward():
     run_large("1080p_256f_bf16", [0, 7, 15], [((0, 0, 0), (2, 2, 2)), ((128, 33, 60), (129, 35, 62)),
                                                ((255, 67, 118), (256, 68, 120))])
