@@ -117,10 +117,12 @@ int dsa3d_backward_batch(const void* q, const void* k, const void* v, const floa
  * Every *_h pointer is a HOST pointer (page-locked memory makes the copies asynchronous
  * and fast; pageable memory works but serialises).  `arena` is DEVICE scratch of at least
  * dsa3d_step_host_arena_bytes(...) bytes, 256-byte aligned, which holds the device copies
- * and the backward workspace; the library allocates no memory.  The upload of dout runs
- * beside the forward and the downloads of out, lse, dq and doffsets beside the backward, on
- * two side streams the library creates on the calling thread's first call (with a few
- * events; they are kept for the life of the thread); everything is ordered after the work
+ * and the backward workspace; the library allocates no memory.  The step is pipelined over
+ * slabs of whole frames: K and V go up first, then each slab's q, offsets and dout while
+ * earlier slabs compute, and each slab's out, lse, dq and doffsets come back while later
+ * slabs compute; dk and dv follow the last slab.  This uses two side streams the library
+ * creates on the calling thread's first call (with a few dozen events; they are kept for
+ * the life of the thread); everything is ordered after the work
  * already in `stream`, and the step is complete when `stream` is.  The host buffers must
  * not be touched until then.  Not for use inside a stream capture.
  */

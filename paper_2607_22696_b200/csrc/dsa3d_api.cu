@@ -43,9 +43,12 @@ int make_problem(int T, int H, int W, int heads, int d, const int* window, int d
     pr.P = static_cast<int>(P);
     pr.N = N;
     pr.items = N * heads;
+    pr.q_begin = 0;
+    pr.q_count = N;
     pr.tile_t = pr.tile_y = pr.tile_x = 0;
     pr.halo = 0;
     pr.tiles_t = pr.tiles_y = pr.tiles_x = 0;
+    pr.tt_begin = pr.tt_count = 0;
     return DSA3D_OK;
 }
 
@@ -71,6 +74,8 @@ void set_tiling(dsa3d::Problem& pr) {
     pr.tiles_t = (pr.T + tt - 1) / tt;
     pr.tiles_y = (pr.H + ty - 1) / ty;
     pr.tiles_x = (pr.W + tx - 1) / tx;
+    pr.tt_begin = 0;
+    pr.tt_count = pr.tiles_t;
 }
 
 struct BackwardWorkspace {
@@ -131,46 +136,91 @@ int dsa3d_backward(const void* q, const void* k, const void* v, const float* off
 
 }  // extern "C"
 
-int dsa3d::backward_impl(const void* q, const void* k, const void* v, const float* offsets, const float* lse,
-                         const void* dout, int T, int H, int W, int heads, int d, const int window[3],
-                         void* dq, void* dk, void* dv, float* doffsets, void* workspace,
-                         size_t workspace_bytes, int dtype, void* stream_, bool tiled,
-                         cudaEvent_t after_gather) {
-    if (!q || !k || !v || !offsets || !lse || !dout || !dq || !dk || !dv || !doffsets)
-        return DSA3D_ERR_NULL_POINTER;
+namespace {
+
+// Everything dsa3d_backward derives from its arguments before it launches anything.
+struct BackwardPlan {
     dsa3d::Problem pr;
-    const int rc = make_problem(T, H, W, heads, d, window, dtype, pr);
+    bool bf16 = false;
+    BackwardWorkspace ws{};
+    size_t count = 0;                 // elements of dk (= of dv)
+    float* acc_dk = nullptr;          // fp32 accumulators (the outputs themselves for fp32 storage)
+    float* acc_dv = nullptr;
+    float2* coef = nullptr;
+    void* scratch = nullptr;
+    void* workspace = nullptr;
+    int ctas = 0;                     // resident CTAs of the tile kernel
+};
+
+int backward_plan(int T, int H, int W, int heads, int d, const int* window, int dtype, bool tiled, void* dk,
+                  void* dv, void* workspace, size_t workspace_bytes, BackwardPlan& plan) {
+    const int rc = make_problem(T, H, W, heads, d, window, dtype, plan.pr);
     if (rc != DSA3D_OK) return rc;
-    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(offsets) || !aligned16(lse) ||
-        !aligned16(dout) || !aligned16(dq) || !aligned16(dk) || !aligned16(dv) || !aligned16(doffsets))
-        return DSA3D_ERR_MISALIGNED;
-    const bool bf16 = dtype == DSA3D_BF16;
-    if (bf16 && tiled) set_tiling(pr);
-    const BackwardWorkspace ws = backward_workspace(pr, dtype, tiled);
-    if (ws.total > 0) {
-        if (!workspace || workspace_bytes < ws.total) return DSA3D_ERR_WORKSPACE;
+    plan.bf16 = dtype == DSA3D_BF16;
+    if (plan.bf16 && tiled) set_tiling(plan.pr);
+    plan.ws = backward_workspace(plan.pr, dtype, tiled);
+    if (plan.ws.total > 0) {
+        if (!workspace || workspace_bytes < plan.ws.total) return DSA3D_ERR_WORKSPACE;
         if (!aligned16(workspace)) return DSA3D_ERR_MISALIGNED;
     }
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    const size_t count = static_cast<size_t>(pr.items) * pr.d;
+    plan.count = static_cast<size_t>(plan.pr.items) * plan.pr.d;
     char* wsp = static_cast<char*>(workspace);
-    float* acc_dk = bf16 ? reinterpret_cast<float*>(wsp) : static_cast<float*>(dk);
-    float* acc_dv = bf16 ? reinterpret_cast<float*>(wsp) + count : static_cast<float*>(dv);
-    float2* coef = ws.coef_bytes ? reinterpret_cast<float2*>(wsp + ws.acc_bytes) : nullptr;
-    void* scratch = ws.scratch_bytes ? wsp + ws.acc_bytes + ws.coef_bytes : nullptr;
+    plan.workspace = workspace;
+    plan.acc_dk = plan.bf16 ? reinterpret_cast<float*>(wsp) : static_cast<float*>(dk);
+    plan.acc_dv = plan.bf16 ? reinterpret_cast<float*>(wsp) + plan.count : static_cast<float*>(dv);
+    plan.coef = plan.ws.coef_bytes ? reinterpret_cast<float2*>(wsp + plan.ws.acc_bytes) : nullptr;
+    plan.scratch = plan.ws.scratch_bytes ? wsp + plan.ws.acc_bytes + plan.ws.coef_bytes : nullptr;
+    if (plan.coef) {
+        int dev = 0, sms = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return cuda_failed(e);
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return cuda_failed(e);
+        plan.ctas = sms * (dsa3d::tile_smem_bytes(plan.pr) <= 110 * 1024 ? 2 : 1);
+        if (plan.ctas > kTileSlots) plan.ctas = kTileSlots;
+    }
+    return DSA3D_OK;
+}
+
+// Zero the dK/dV accumulators.
+int backward_clear(const BackwardPlan& plan, cudaStream_t stream) {
     cudaError_t e;
-    if (bf16) {
-        e = cudaMemsetAsync(workspace, 0, ws.acc_bytes, stream);
+    if (plan.bf16) {
+        e = cudaMemsetAsync(plan.workspace, 0, plan.ws.acc_bytes, stream);
         if (e != cudaSuccess) return cuda_failed(e);
     } else {
-        e = cudaMemsetAsync(dk, 0, count * sizeof(float), stream);
+        e = cudaMemsetAsync(plan.acc_dk, 0, plan.count * sizeof(float), stream);
         if (e != cudaSuccess) return cuda_failed(e);
-        e = cudaMemsetAsync(dv, 0, count * sizeof(float), stream);
+        e = cudaMemsetAsync(plan.acc_dv, 0, plan.count * sizeof(float), stream);
         if (e != cudaSuccess) return cuda_failed(e);
     }
-    e = record(2, stream);
+    return DSA3D_OK;
+}
+
+// The query tokens of frames [f0, f1) as a launch of their own.  With tiling on, f0 must be a
+// multiple of the tile's frame count (f1 too unless it is T).
+dsa3d::Problem frames_of(const dsa3d::Problem& pr, int f0, int f1) {
+    dsa3d::Problem s = pr;
+    const long long per_frame = static_cast<long long>(pr.H) * pr.W;
+    s.q_begin = f0 * per_frame;
+    s.q_count = (f1 - f0) * per_frame;
+    s.items = s.q_count * pr.heads;
+    if (pr.tile_t >= 1) {
+        s.tt_begin = f0 / pr.tile_t;
+        s.tt_count = (f1 + pr.tile_t - 1) / pr.tile_t - s.tt_begin;
+    }
+    return s;
+}
+
+// dQ, dOffsets of the queries of frames [f0, f1) and their contributions to dK/dV.
+int backward_frames(const BackwardPlan& plan, const void* q, const void* k, const void* v, const float* offsets,
+                    const float* lse, const void* dout, void* dq, float* doffsets, int f0, int f1,
+                    cudaStream_t stream, cudaEvent_t after_gather) {
+    const dsa3d::Problem pr = frames_of(plan.pr, f0, f1);
+    cudaError_t e = record(2, stream);
     if (e != cudaSuccess) return cuda_failed(e);
-    e = dsa3d::launch_backward(q, k, v, offsets, lse, dout, dq, acc_dk, acc_dv, doffsets, coef, pr, bf16, stream);
+    e = dsa3d::launch_backward(q, k, v, offsets, lse, dout, dq, plan.acc_dk, plan.acc_dv, doffsets, plan.coef, pr,
+                               plan.bf16, stream);
     if (e != cudaSuccess) return cuda_failed(e);
     e = record(3, stream);
     if (e != cudaSuccess) return cuda_failed(e);
@@ -178,29 +228,59 @@ int dsa3d::backward_impl(const void* q, const void* k, const void* v, const floa
         e = cudaEventRecord(after_gather, stream);
         if (e != cudaSuccess) return cuda_failed(e);
     }
-    if (coef) {
-        int dev = 0, sms = 0;
-        e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return cuda_failed(e);
-        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return cuda_failed(e);
-        int ctas = sms * (dsa3d::tile_smem_bytes(pr) <= 110 * 1024 ? 2 : 1);
-        if (ctas > kTileSlots) ctas = kTileSlots;
+    if (plan.coef) {
         e = record(4, stream);
         if (e != cudaSuccess) return cuda_failed(e);
-        e = dsa3d::launch_scatter_tiles(q, dout, offsets, coef, acc_dk, acc_dv, scratch, ctas,
-                                        ws.entries_per_cta, pr, stream);
+        e = dsa3d::launch_scatter_tiles(q, dout, offsets, plan.coef, plan.acc_dk, plan.acc_dv, plan.scratch,
+                                        plan.ctas, plan.ws.entries_per_cta, pr, stream);
         if (e != cudaSuccess) return cuda_failed(e);
         e = record(5, stream);
         if (e != cudaSuccess) return cuda_failed(e);
     }
-    if (bf16) {
-        e = dsa3d::launch_convert_bf16(acc_dk, dk, static_cast<long long>(count), stream);
-        if (e != cudaSuccess) return cuda_failed(e);
-        e = dsa3d::launch_convert_bf16(acc_dv, dv, static_cast<long long>(count), stream);
-        if (e != cudaSuccess) return cuda_failed(e);
-    }
     return DSA3D_OK;
+}
+
+// Accumulators -> dk, dv (bf16 storage only; fp32 storage accumulated in place).
+int backward_finish(const BackwardPlan& plan, void* dk, void* dv, cudaStream_t stream) {
+    if (!plan.bf16) return DSA3D_OK;
+    cudaError_t e = dsa3d::launch_convert_bf16(plan.acc_dk, dk, static_cast<long long>(plan.count), stream);
+    if (e != cudaSuccess) return cuda_failed(e);
+    e = dsa3d::launch_convert_bf16(plan.acc_dv, dv, static_cast<long long>(plan.count), stream);
+    if (e != cudaSuccess) return cuda_failed(e);
+    return DSA3D_OK;
+}
+
+int forward_frames(const dsa3d::Problem& full, const void* q, const void* k, const void* v, const float* offsets,
+                   void* out, float* lse, bool bf16, int f0, int f1, cudaStream_t stream) {
+    const dsa3d::Problem pr = frames_of(full, f0, f1);
+    cudaError_t e = record(0, stream);
+    if (e != cudaSuccess) return cuda_failed(e);
+    e = dsa3d::launch_forward(q, k, v, offsets, out, lse, pr, bf16, stream);
+    if (e != cudaSuccess) return cuda_failed(e);
+    e = record(1, stream);
+    return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
+}
+
+}  // namespace
+
+int dsa3d::backward_impl(const void* q, const void* k, const void* v, const float* offsets, const float* lse,
+                         const void* dout, int T, int H, int W, int heads, int d, const int window[3],
+                         void* dq, void* dk, void* dv, float* doffsets, void* workspace,
+                         size_t workspace_bytes, int dtype, void* stream_, bool tiled) {
+    if (!q || !k || !v || !offsets || !lse || !dout || !dq || !dk || !dv || !doffsets)
+        return DSA3D_ERR_NULL_POINTER;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(offsets) || !aligned16(lse) ||
+        !aligned16(dout) || !aligned16(dq) || !aligned16(dk) || !aligned16(dv) || !aligned16(doffsets))
+        return DSA3D_ERR_MISALIGNED;
+    BackwardPlan plan;
+    int rc = backward_plan(T, H, W, heads, d, window, dtype, tiled, dk, dv, workspace, workspace_bytes, plan);
+    if (rc != DSA3D_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    rc = backward_clear(plan, stream);
+    if (rc != DSA3D_OK) return rc;
+    rc = backward_frames(plan, q, k, v, offsets, lse, dout, dq, doffsets, 0, T, stream, nullptr);
+    if (rc != DSA3D_OK) return rc;
+    return backward_finish(plan, dk, dv, stream);
 }
 
 extern "C" {
@@ -237,13 +317,15 @@ Arena arena_layout(const dsa3d::Problem& pr, int dtype) {
     return a;
 }
 
-// Two side streams and four events per (thread, device) for the copy/compute overlap of
-// dsa3d_step_host; created on first use and kept for the life of the thread.
+// Two side streams and the events of the copy/compute pipeline of dsa3d_step_host, per
+// (thread, device); created on first use and kept for the life of the thread.
+constexpr int kMaxSlabs = 8;
 struct HostStep {
     int device = -1;
     cudaStream_t in = nullptr, out = nullptr;
-    cudaEvent_t start = nullptr, dout_ready = nullptr, fwd_done = nullptr, gather_done = nullptr,
-                out_done = nullptr;
+    cudaEvent_t start = nullptr, kv_ready = nullptr, out_done = nullptr;
+    cudaEvent_t q_ready[kMaxSlabs] = {}, dout_ready[kMaxSlabs] = {}, fwd_done[kMaxSlabs] = {},
+                gather_done[kMaxSlabs] = {};
 };
 thread_local HostStep g_host_step[8];
 
@@ -256,12 +338,15 @@ HostStep* host_step_resources() {
         if (!slot && h.device < 0) slot = &h;
     }
     if (!slot) return nullptr;                          // more than 8 devices used from one thread
-    cudaEvent_t* events[5] = {&slot->start, &slot->dout_ready, &slot->fwd_done, &slot->gather_done,
-                              &slot->out_done};
     if (cudaStreamCreateWithFlags(&slot->in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
     if (cudaStreamCreateWithFlags(&slot->out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-    for (cudaEvent_t* ev : events)
+    cudaEvent_t* single[3] = {&slot->start, &slot->kv_ready, &slot->out_done};
+    for (cudaEvent_t* ev : single)
         if (cudaEventCreateWithFlags(ev, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    cudaEvent_t* per_slab[4] = {slot->q_ready, slot->dout_ready, slot->fwd_done, slot->gather_done};
+    for (cudaEvent_t* arr : per_slab)
+        for (int i = 0; i < kMaxSlabs; ++i)
+            if (cudaEventCreateWithFlags(&arr[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
     slot->device = dev;
     return slot;
 }
@@ -297,39 +382,86 @@ int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const flo
         e = (call);                             \
         if (e != cudaSuccess) return cuda_failed(e); \
     } while (0)
-    // Side stream `in`: dout is only needed by the backward, so its upload runs beside the
-    // forward.  Side stream `out`: results leave as soon as they are final - out and lse
-    // during the backward, dq and doffsets during the dk/dv kernels.
+    // The query side of the step (q, offsets, dout in; out, lse, dq, doffsets back) is cut
+    // into slabs of whole frames.  Side stream `in` uploads K and V, then slab after slab;
+    // the main stream runs the forward and the backward of a slab as soon as its inputs are
+    // there; side stream `out` carries each slab's results back while the next slab computes.
+    // Only K/V (needed by every query) at the start and dK/dV (final after the last slab) at
+    // the end are not hidden behind kernels.
+    const bool bf16 = dtype == DSA3D_BF16;
+    BackwardPlan plan;
+    int st = backward_plan(T, H, W, heads, d, window, dtype, true, base + a.dk, base + a.dv,
+                           a.ws_bytes ? base + a.workspace : nullptr, a.ws_bytes, plan);
+    if (st != DSA3D_OK) return st;
+    const int unit = plan.pr.tile_t >= 1 ? plan.pr.tile_t : 1;          // slabs start on tile boundaries
+    int slab_frames = (T + kMaxSlabs - 1) / kMaxSlabs;
+    slab_frames = (slab_frames + unit - 1) / unit * unit;
+    const int slabs = (T + slab_frames - 1) / slab_frames;
+    const size_t elt = bf16 ? 2 : 4;
+    const size_t frame_rows = static_cast<size_t>(H) * W * heads;
+    const size_t frame_row_bytes = frame_rows * d * elt;
+    const size_t frame_off_bytes = frame_rows * pr.P * 3 * sizeof(float);
+    const size_t frame_lse_bytes = frame_rows * sizeof(float);
+    const char* q_hb = static_cast<const char*>(q_h);
+    const char* off_hb = reinterpret_cast<const char*>(offsets_h);
+    const char* dout_hb = static_cast<const char*>(dout_h);
+
     DSA3D_TRY(cudaEventRecord(hs->start, stream));
     DSA3D_TRY(cudaStreamWaitEvent(hs->in, hs->start, 0));
-    DSA3D_TRY(cudaMemcpyAsync(base + a.dout, dout_h, a.row_bytes, cudaMemcpyHostToDevice, hs->in));
-    DSA3D_TRY(cudaEventRecord(hs->dout_ready, hs->in));
+    DSA3D_TRY(cudaStreamWaitEvent(hs->out, hs->start, 0));
+    DSA3D_TRY(cudaMemcpyAsync(base + a.k, k_h, a.row_bytes, cudaMemcpyHostToDevice, hs->in));
+    DSA3D_TRY(cudaMemcpyAsync(base + a.v, v_h, a.row_bytes, cudaMemcpyHostToDevice, hs->in));
+    DSA3D_TRY(cudaEventRecord(hs->kv_ready, hs->in));
+    for (int s = 0; s < slabs; ++s) {
+        const int f0 = s * slab_frames, f1 = f0 + slab_frames < T ? f0 + slab_frames : T;
+        const size_t nf = static_cast<size_t>(f1 - f0);
+        DSA3D_TRY(cudaMemcpyAsync(base + a.q + f0 * frame_row_bytes, q_hb + f0 * frame_row_bytes,
+                                  nf * frame_row_bytes, cudaMemcpyHostToDevice, hs->in));
+        DSA3D_TRY(cudaMemcpyAsync(base + a.offsets + f0 * frame_off_bytes, off_hb + f0 * frame_off_bytes,
+                                  nf * frame_off_bytes, cudaMemcpyHostToDevice, hs->in));
+        DSA3D_TRY(cudaEventRecord(hs->q_ready[s], hs->in));
+        DSA3D_TRY(cudaMemcpyAsync(base + a.dout + f0 * frame_row_bytes, dout_hb + f0 * frame_row_bytes,
+                                  nf * frame_row_bytes, cudaMemcpyHostToDevice, hs->in));
+        DSA3D_TRY(cudaEventRecord(hs->dout_ready[s], hs->in));
+    }
 
-    DSA3D_TRY(cudaMemcpyAsync(base + a.k, k_h, a.row_bytes, cudaMemcpyHostToDevice, stream));
-    DSA3D_TRY(cudaMemcpyAsync(base + a.v, v_h, a.row_bytes, cudaMemcpyHostToDevice, stream));
-    DSA3D_TRY(cudaMemcpyAsync(base + a.q, q_h, a.row_bytes, cudaMemcpyHostToDevice, stream));
-    DSA3D_TRY(cudaMemcpyAsync(base + a.offsets, offsets_h, a.off_bytes, cudaMemcpyHostToDevice, stream));
-    int st = dsa3d_forward(base + a.q, base + a.k, base + a.v, reinterpret_cast<const float*>(base + a.offsets),
-                           T, H, W, heads, d, window, base + a.out, reinterpret_cast<float*>(base + a.lse),
-                           dtype, stream_);
+    st = backward_clear(plan, stream);
     if (st != DSA3D_OK) return st;
-    DSA3D_TRY(cudaEventRecord(hs->fwd_done, stream));
-    DSA3D_TRY(cudaStreamWaitEvent(hs->out, hs->fwd_done, 0));
-    DSA3D_TRY(cudaMemcpyAsync(out_h, base + a.out, a.row_bytes, cudaMemcpyDeviceToHost, hs->out));
-    DSA3D_TRY(cudaMemcpyAsync(lse_h, base + a.lse, a.lse_bytes, cudaMemcpyDeviceToHost, hs->out));
+    DSA3D_TRY(cudaStreamWaitEvent(stream, hs->kv_ready, 0));
+    const float* off_d = reinterpret_cast<const float*>(base + a.offsets);
+    float* lse_d = reinterpret_cast<float*>(base + a.lse);
+    float* doff_d = reinterpret_cast<float*>(base + a.doffsets);
+    for (int s = 0; s < slabs; ++s) {
+        const int f0 = s * slab_frames, f1 = f0 + slab_frames < T ? f0 + slab_frames : T;
+        const size_t nf = static_cast<size_t>(f1 - f0);
+        DSA3D_TRY(cudaStreamWaitEvent(stream, hs->q_ready[s], 0));
+        st = forward_frames(pr, base + a.q, base + a.k, base + a.v, off_d, base + a.out, lse_d, bf16, f0, f1,
+                            stream);
+        if (st != DSA3D_OK) return st;
+        DSA3D_TRY(cudaEventRecord(hs->fwd_done[s], stream));
+        DSA3D_TRY(cudaStreamWaitEvent(hs->out, hs->fwd_done[s], 0));
+        DSA3D_TRY(cudaMemcpyAsync(static_cast<char*>(out_h) + f0 * frame_row_bytes,
+                                  base + a.out + f0 * frame_row_bytes, nf * frame_row_bytes,
+                                  cudaMemcpyDeviceToHost, hs->out));
+        DSA3D_TRY(cudaMemcpyAsync(reinterpret_cast<char*>(lse_h) + f0 * frame_lse_bytes,
+                                  base + a.lse + f0 * frame_lse_bytes, nf * frame_lse_bytes,
+                                  cudaMemcpyDeviceToHost, hs->out));
 
-    DSA3D_TRY(cudaStreamWaitEvent(stream, hs->dout_ready, 0));
-    st = dsa3d::backward_impl(base + a.q, base + a.k, base + a.v, reinterpret_cast<const float*>(base + a.offsets),
-                              reinterpret_cast<const float*>(base + a.lse), base + a.dout, T, H, W, heads, d,
-                              window, base + a.dq, base + a.dk, base + a.dv,
-                              reinterpret_cast<float*>(base + a.doffsets),
-                              a.ws_bytes ? base + a.workspace : nullptr, a.ws_bytes, dtype, stream_, true,
-                              hs->gather_done);
-    if (st != DSA3D_OK) return st;
-    DSA3D_TRY(cudaStreamWaitEvent(hs->out, hs->gather_done, 0));
-    DSA3D_TRY(cudaMemcpyAsync(dq_h, base + a.dq, a.row_bytes, cudaMemcpyDeviceToHost, hs->out));
-    DSA3D_TRY(cudaMemcpyAsync(doffsets_h, base + a.doffsets, a.off_bytes, cudaMemcpyDeviceToHost, hs->out));
+        DSA3D_TRY(cudaStreamWaitEvent(stream, hs->dout_ready[s], 0));
+        st = backward_frames(plan, base + a.q, base + a.k, base + a.v, off_d, lse_d, base + a.dout, base + a.dq,
+                             doff_d, f0, f1, stream, hs->gather_done[s]);
+        if (st != DSA3D_OK) return st;
+        DSA3D_TRY(cudaStreamWaitEvent(hs->out, hs->gather_done[s], 0));
+        DSA3D_TRY(cudaMemcpyAsync(static_cast<char*>(dq_h) + f0 * frame_row_bytes,
+                                  base + a.dq + f0 * frame_row_bytes, nf * frame_row_bytes,
+                                  cudaMemcpyDeviceToHost, hs->out));
+        DSA3D_TRY(cudaMemcpyAsync(reinterpret_cast<char*>(doffsets_h) + f0 * frame_off_bytes,
+                                  base + a.doffsets + f0 * frame_off_bytes, nf * frame_off_bytes,
+                                  cudaMemcpyDeviceToHost, hs->out));
+    }
     DSA3D_TRY(cudaEventRecord(hs->out_done, hs->out));
+    st = backward_finish(plan, base + a.dk, base + a.dv, stream);
+    if (st != DSA3D_OK) return st;
     DSA3D_TRY(cudaMemcpyAsync(dk_h, base + a.dk, a.row_bytes, cudaMemcpyDeviceToHost, stream));
     DSA3D_TRY(cudaMemcpyAsync(dv_h, base + a.dv, a.row_bytes, cudaMemcpyDeviceToHost, stream));
     DSA3D_TRY(cudaStreamWaitEvent(stream, hs->out_done, 0));     // the step is over when `stream` is

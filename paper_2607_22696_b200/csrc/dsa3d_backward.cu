@@ -66,8 +66,8 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
     if (!active) item = pr.items - 1;
     float* stats = smem + static_cast<size_t>(threadIdx.x / LPR) * pr.P * kStats;   // [P][8] of this group
 
-    const int m = static_cast<int>(item / pr.N);
-    const long long n = item - static_cast<long long>(m) * pr.N;
+    const int m = static_cast<int>(item / pr.q_count);
+    const long long n = pr.q_begin + (item - static_cast<long long>(m) * pr.q_count);
     const int x = static_cast<int>(n % pr.W);
     const int y = static_cast<int>((n / pr.W) % pr.H);
     const int t = static_cast<int>(n / (static_cast<long long>(pr.W) * pr.H));
@@ -272,7 +272,7 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kWarps = kTileThreads / 32;
-    const int tiles_per_head = pr.tiles_t * pr.tiles_y * pr.tiles_x;
+    const int tiles_per_head = pr.tt_count * pr.tiles_y * pr.tiles_x;
     const long long total_tiles = static_cast<long long>(tiles_per_head) * pr.heads;
     TileEntry* my_scratch = scratch + static_cast<long long>(blockIdx.x) * scratch_entries_per_cta;
     const long long tok_stride = static_cast<long long>(pr.heads) * D;
@@ -282,7 +282,7 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         int rem = static_cast<int>(tile_id - static_cast<long long>(m) * tiles_per_head);
         const int tx = rem % pr.tiles_x; rem /= pr.tiles_x;
         const int ty = rem % pr.tiles_y;
-        const int tt = rem / pr.tiles_y;
+        const int tt = pr.tt_begin + rem / pr.tiles_y;
         const int t0 = tt * pr.tile_t, y0 = ty * pr.tile_y, x0 = tx * pr.tile_x;
         const int lo_t = t0 - pr.halo, lo_y = y0 - pr.halo, lo_x = x0 - pr.halo;
 
@@ -533,7 +533,7 @@ static cudaError_t launch_scatter_tiles_t(const void* q, const void* dout, const
     const size_t smem = tile_smem_bytes(pr);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
-    const long long total_tiles = static_cast<long long>(pr.tiles_t) * pr.tiles_y * pr.tiles_x * pr.heads;
+    const long long total_tiles = static_cast<long long>(pr.tt_count) * pr.tiles_y * pr.tiles_x * pr.heads;
     const int grid = static_cast<int>(total_tiles < ctas ? total_tiles : ctas);
     kern<<<grid, kTileThreads, smem, stream>>>(
         static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(dout), offsets, coef, acc_dk,

@@ -21,12 +21,16 @@ struct Problem {
     int T, H, W, heads, d;
     int kt, kh, kw, P;
     long long N;       // T*H*W
-    long long items;   // N*heads: one work item per (token, head)
+    long long items;   // work items of this launch: one per (query token, head) = q_count*heads
+    // Query tokens [q_begin, q_begin + q_count) are processed (the whole grid unless a caller
+    // works through the video in slabs of frames); K and V always cover the whole grid.
+    long long q_begin, q_count;
     // Query tiling of the backward scatter (tile_t < 1: no tiling, every dK/dV contribution
     // goes straight to the global accumulators).  A corner is "in the halo" of a query when
     // it lies within `halo` grid cells of the query's tile on every axis.
     int tile_t, tile_y, tile_x, halo;
     int tiles_t, tiles_y, tiles_x;
+    int tt_begin, tt_count;   // tile rows along t that the tile kernel visits (all: 0, tiles_t)
 };
 
 // ---------------------------------------------------------------------------------------

@@ -39,8 +39,8 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
     const bool active = item < pr.items;                 // a trailing group repeats the last item, stores off
     if (!active) item = pr.items - 1;
 
-    const int m = static_cast<int>(item / pr.N);
-    const long long n = item - static_cast<long long>(m) * pr.N;
+    const int m = static_cast<int>(item / pr.q_count);
+    const long long n = pr.q_begin + (item - static_cast<long long>(m) * pr.q_count);
     const int x = static_cast<int>(n % pr.W);
     const int y = static_cast<int>((n / pr.W) % pr.H);
     const int t = static_cast<int>(n / (static_cast<long long>(pr.W) * pr.H));

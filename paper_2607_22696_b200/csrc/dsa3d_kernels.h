@@ -32,11 +32,10 @@ cudaError_t launch_convert_bf16(const float* acc, void* dst, long long count, cu
 
 // Shared implementation of dsa3d_backward.  `tiled` selects the tile pre-reduction of the
 // dK/dV scatter (bf16 only; needs the large workspace); without it the workspace is just the
-// two fp32 accumulators.  `after_gather`, if given, is recorded on the stream once dq and
-// doffsets are final (before the dk/dv kernels).  Returns a dsa3d_status.
+// two fp32 accumulators.  Returns a dsa3d_status.
 int backward_impl(const void* q, const void* k, const void* v, const float* offsets, const float* lse,
                   const void* dout, int T, int H, int W, int heads, int d, const int window[3], void* dq,
                   void* dk, void* dv, float* doffsets, void* workspace, size_t workspace_bytes, int dtype,
-                  void* stream, bool tiled, cudaEvent_t after_gather = nullptr);
+                  void* stream, bool tiled);
 
 }  // namespace dsa3d
