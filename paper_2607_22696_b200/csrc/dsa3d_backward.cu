@@ -23,8 +23,8 @@
 //   fp32 reduction is what bounds the simple scheme (L2 reduction throughput), so the tile
 //   kernel sums them on chip first: it bins the (query, sample, corner) contributions of
 //   the tile by target row (counting sort, counters in shared memory, 16-byte entries
-//   {row offset, fp32 coefficient pair} in a per-CTA global scratch), then each half-warp
-//   owns a row, walks its entries, accumulates  coefficient x q-row  and  coefficient x
+//   {row offset, fp32 coefficient pair} in a per-CTA global scratch), then each group of
+//   d/8 lanes (a half-warp at 128 channels, a quarter-warp at 64) owns a row, walks its entries, accumulates  coefficient x q-row  and  coefficient x
 //   dO-row  in fp32 registers from the tile's q/dO rows held in shared memory, and issues
 //   ONE reduction per row and tensor.  (Built with DSA3D_BF16_COEF the entries are 8 bytes
 //   with bf16 coefficients and the products use the mixed-precision FMA.)
@@ -380,33 +380,38 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         }
         // after the fill sweep cursor[b] is the END of bin b; its start is the end of bin b-1
 
-        // ---- reduce: a warp takes two neighbouring key rows, one per half-warp; both halves
-        //      run the same number of steps (the shorter list is padded with zero entries)
+        // ---- reduce: a row is VPR 16-byte vectors, one per lane, so a warp takes 32 / VPR
+        //      neighbouring key rows at once (two at 128 channels); every group runs the same
+        //      number of steps (the shorter lists are padded with zero entries)
         {
-            const int half = lane >> 4, hl = lane & 15;
-            const int hv = hl < VPR ? hl : VPR - 1;         // lanes beyond a narrow row mirror its last vector
-            const unsigned char* my_rows = smem_raw + hv * 16;
-            for (int pairbin = warp * 2; pairbin < NB; pairbin += kWarps * 2) {
-                const int bin = pairbin + half;
+            constexpr int GW = VPR;                          // lanes per key row
+            constexpr int kGroups = 32 / GW;
+            const int grp = lane / GW, hl = lane & (GW - 1);
+            const int lane0 = lane & ~(GW - 1);              // first lane of this group
+            const unsigned char* my_rows = smem_raw + hl * 16;
+            for (int firstbin = warp * kGroups; firstbin < NB; firstbin += kWarps * kGroups) {
+                const int bin = firstbin + grp;
                 unsigned start = 0u, end = 0u;
                 if (bin < NB) {
                     end = cursor[bin];
                     start = bin == 0 ? 0u : cursor[bin - 1];
                 }
                 const unsigned cnt_mine = end - start;
-                const unsigned cnt_max = max(cnt_mine, __shfl_xor_sync(kFull, cnt_mine, 16));
+                unsigned cnt_max = cnt_mine;
+#pragma unroll
+                for (int o = GW; o < 32; o <<= 1) cnt_max = max(cnt_max, __shfl_xor_sync(kFull, cnt_max, o));
                 if (cnt_max == 0u) continue;
                 float ak[8], av[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) ak[e] = av[e] = 0.0f;
-                for (unsigned base = 0; base < cnt_max; base += 16) {
+                for (unsigned base = 0; base < cnt_max; base += GW) {
 #ifndef DSA3D_BF16_COEF
                     uint4 ent = make_uint4(0u, 0u, 0u, 0u);               // offset 0, coefficients 0
                     if (base + hl < cnt_mine) ent = __ldcg(my_scratch + start + base + hl);
-                    const int steps = static_cast<int>(min(16u, cnt_max - base));
+                    const int steps = static_cast<int>(min(static_cast<unsigned>(GW), cnt_max - base));
 #pragma unroll 4
                     for (int j = 0; j < steps; ++j) {
-                        const int src = (lane & 16) | j;
+                        const int src = lane0 | j;
                         const unsigned off = __shfl_sync(kFull, ent.x, src);
                         const float ck = __uint_as_float(__shfl_sync(kFull, ent.y, src));
                         const float cv = __uint_as_float(__shfl_sync(kFull, ent.z, src));
@@ -425,10 +430,10 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
 #else
                     uint2 ent = make_uint2(0u, 0u);                       // offset 0, coefficients 0
                     if (base + hl < cnt_mine) ent = __ldcg(my_scratch + start + base + hl);
-                    const int steps = static_cast<int>(min(16u, cnt_max - base));
+                    const int steps = static_cast<int>(min(static_cast<unsigned>(GW), cnt_max - base));
 #pragma unroll 4
                     for (int j = 0; j < steps; ++j) {
-                        const int src = (lane & 16) | j;
+                        const int src = lane0 | j;
                         const unsigned off = __shfl_sync(kFull, ent.x, src);
                         const unsigned cw = __shfl_sync(kFull, ent.y, src);
                         unsigned short ck, cv;
@@ -449,7 +454,7 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                     }
                 }
 #endif
-                if (cnt_mine > 0u && hl < VPR) {
+                if (cnt_mine > 0u) {
                     const int bx = bin % ex, by = (bin / ex) % ey, bt = bin / (ex * ey);
                     const long long tok = (static_cast<long long>(lo_t + bt) * pr.H + (lo_y + by)) * pr.W + (lo_x + bx);
                     const long long o = tok * tok_stride + static_cast<long long>(m) * D + hl * 8;

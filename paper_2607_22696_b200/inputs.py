@@ -144,6 +144,9 @@ WORKLOADS: Dict[str, Workload] = {w.name: w for w in [
     # the window the paper itself runs, (3,7,7) = 147 samples, on 64 frames of the 1080p grid
     # (at 256 frames the offsets alone would be 59 GB)
     Workload("1080p_64f_w377_bf16", 64, 68, 120, 16, 128, (3, 7, 7), _BF16, 2.0, 6),
+    # not a BASELINE config: the head shape of the paper's 1B model (2048 hidden, 32 heads of 64
+    # channels) on 128 frames of the 1080p grid, same bytes per token as 16 heads of 128
+    Workload("1080p_128f_h32d64_bf16", 128, 68, 120, 32, 64, (3, 3, 3), _BF16, 2.0, 8),
     # not a BASELINE config: offsets with the coherence of a motion field (structured-motion
     # data of the paper's quality ablation), same grid and spread as the 1080p workload
     Workload("1080p_256f_drift_bf16", 256, 68, 120, 16, 128, (3, 3, 3), _BF16, 2.0, 7, offsets="drift"),
