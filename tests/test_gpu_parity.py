@@ -195,12 +195,16 @@ def test_large_window_through_the_tile_kernel():
 
 # ------------------------------------------------------------- host-buffer entry point
 
-@pytest.mark.parametrize("dtype", [BF16, F32])
-def test_step_host_matches_the_device_entry_points(dtype):
-    """dsa3d_step_host (pinned host buffers in, pinned host buffers out, copies overlapped
-    with the kernels on side streams) must return what dsa3d_forward + dsa3d_backward
-    return on device buffers; run twice to catch a stale event or buffer."""
-    q, k, v, off, dout = small_problem(6, 10, 12, 3, 64, (3, 3, 3), dtype, 1.3, 60)
+@pytest.mark.parametrize("dtype,shape", [(BF16, (6, 10, 12, 3, 64)), (F32, (6, 10, 12, 3, 64)),
+                                         (BF16, (19, 9, 10, 2, 128)), (F32, (11, 5, 6, 2, 32)),
+                                         (BF16, (1, 7, 9, 2, 64))])
+def test_step_host_matches_the_device_entry_points(dtype, shape):
+    """dsa3d_step_host (pinned host buffers in, pinned host buffers out, the step pipelined
+    over slabs of frames with the copies on side streams) must return what dsa3d_forward +
+    dsa3d_backward return on device buffers; run twice to catch a stale event or buffer.
+    The shapes give two slabs, several slabs with a ragged last one (on tile boundaries for
+    bf16, two frames each for fp32), and a single frame."""
+    q, k, v, off, dout = small_problem(*shape, (3, 3, 3), dtype, 1.3, 60)
     dims = tuple(q.shape)
     dev = [z.cuda() for z in (q, k, v, off, dout)]
     out_d, lse_d = pu.gpu_forward(*dev[:4], dims, (3, 3, 3))
