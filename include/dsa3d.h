@@ -199,6 +199,54 @@ int dsa3d_probe_red(void* buffer, size_t working_set_bytes, int iters, double* b
                     void* stream);
 int dsa3d_probe_fma(const void* seed_1kb, int iters, int kind, double* fma_per_launch, void* stream);
 
+/*
+ * The layers around the operator in Eq. 1 (device pointers, asynchronous on `stream`, same
+ * ownership rules as above).  The paper specifies them only as "a lightweight depthwise 3D
+ * convolution followed by a linear layer" for the offsets (Formulation section) and as the
+ * DWConv3D(X) term of Eq. 1, built from grouped nn.Conv3d and pointwise layers
+ * (Implementation considerations); kernel size, padding and parameter layout below are this
+ * library's choices.
+ *
+ * dsa3d_dwconv3d_forward: y[t,y,x,c] = bias[c] + sum over taps (i,j,l) of
+ *   weight[(i*kh + j)*kw + l][c] * x[t + i - kt/2, y + j - kh/2, x + l - kw/2][c]
+ * (cross-correlation, unit stride, zero outside the grid, integer division in the centring:
+ * the same centring as the attention window).  x, y: [T,H,W,C] channels-last in `dtype`,
+ * C a multiple of 8; weight fp32 [kt*kh*kw, C]; bias fp32 [C] or NULL; kernel = (kt,kh,kw),
+ * HOST pointer, kt,kh <= 15, kw <= 7.  fp32 accumulation in tap order, one rounding to `dtype`.
+ * y must not alias x.
+ */
+int dsa3d_dwconv3d_forward(const void* x, const float* weight, const float* bias, int T, int H, int W, int C,
+                           const int kernel[3], void* y, int dtype, void* stream);
+
+/*
+ * dsa3d_offsets_linear_forward: offsets[n][o] = bias[o] + sum_c u[n][c] * w[o][c], the linear
+ * layer of the offset predictor; with O = heads*P*3 the result is the offsets tensor of
+ * dsa3d_forward.  u [tokens, C] and w [O, C] in `dtype` (row-major, C a multiple of 8),
+ * bias fp32 [O], offsets fp32 [tokens, O]; tokens < 2^31.  bf16 runs on the tensor cores
+ * (exact bf16 products, fp32 accumulation in the hardware's order); fp32 uses fp32 FMAs in
+ * channel order.  Its waits on hardware barriers are bounded: if one ever runs out the
+ * kernel stops early, the output is incomplete and dsa3d_device_timeout_flag() returns
+ * non-zero afterwards.
+ */
+int dsa3d_offsets_linear_forward(const void* u, const void* w, const float* bias, long long tokens, int C, int O,
+                                 float* offsets, int dtype, void* stream);
+
+/* Synchronises with the device and returns the flag described above (0: no wait ever ran
+ * out; -1: the flag could not be read). */
+int dsa3d_device_timeout_flag(void);
+
+/*
+ * dsa3d_forward_residual: Eq. 1 with its first term: out = residual + attention output,
+ * where `residual` ([T,H,W,heads,d] in `dtype`, e.g. the result of dsa3d_dwconv3d_forward
+ * on the layer input with C = heads*d) is added in fp32 before the one rounding to `dtype`.
+ * `residual` may be the same buffer as `out`.  Everything else as dsa3d_forward; the
+ * gradient of the loss with respect to `residual` is dout itself, so dsa3d_backward is
+ * unchanged.
+ */
+int dsa3d_forward_residual(const void* q, const void* k, const void* v, const float* offsets, const void* residual,
+                           int T, int H, int W, int heads, int d, const int window[3], void* out, float* lse,
+                           int dtype, void* stream);
+
 /* Static, NUL-terminated description of a status code. */
 const char* dsa3d_status_string(int status);
 

@@ -69,6 +69,14 @@ def load():
     lib.dsa3d_forward_batch.argtypes = [p, p, p, p, i, i, i, i, i, i, win, p, p, i, p]
     lib.dsa3d_backward_batch.restype = i
     lib.dsa3d_backward_batch.argtypes = [p, p, p, p, p, p, i, i, i, i, i, i, win, p, p, p, p, p, sz, i, p]
+    lib.dsa3d_dwconv3d_forward.restype = i
+    lib.dsa3d_dwconv3d_forward.argtypes = [p, p, p, i, i, i, i, win, p, i, p]
+    lib.dsa3d_offsets_linear_forward.restype = i
+    lib.dsa3d_offsets_linear_forward.argtypes = [p, p, p, ctypes.c_longlong, i, i, p, i, p]
+    lib.dsa3d_device_timeout_flag.restype = i
+    lib.dsa3d_device_timeout_flag.argtypes = []
+    lib.dsa3d_forward_residual.restype = i
+    lib.dsa3d_forward_residual.argtypes = [p, p, p, p, p, i, i, i, i, i, win, p, p, i, p]
     lib.dsa3d_status_string.restype = ctypes.c_char_p
     lib.dsa3d_status_string.argtypes = [i]
     lib.dsa3d_last_cuda_error.restype = i
@@ -141,6 +149,46 @@ def dsa3d_forward(q, k, v, offsets, T, H, W, heads, d, window, out, lse, dtype=N
         _ptr(q, "q", n * d), _ptr(k, "k", n * d), _ptr(v, "v", n * d),
         _ptr(offsets, "offsets", n * P * 3, torch.float32), T, H, W, heads, d, _window(window),
         _ptr(out, "out", n * d), _ptr(lse, "lse", n, torch.float32), code, _stream(stream)))
+
+
+def dsa3d_forward_residual(q, k, v, offsets, residual, T, H, W, heads, d, window, out, lse, dtype=None,
+                           stream=None) -> None:
+    """out, lse <- residual + 3D-DSA forward (Eq. 1 with its first term); see include/dsa3d.h."""
+    lib = load()
+    dt = q.dtype if dtype is None else dtype
+    code = _DTYPES[dt] if isinstance(dt, torch.dtype) else int(dt)
+    n = T * H * W * heads
+    P = int(window[0]) * int(window[1]) * int(window[2])
+    _check(lib.dsa3d_forward_residual(
+        _ptr(q, "q", n * d), _ptr(k, "k", n * d), _ptr(v, "v", n * d),
+        _ptr(offsets, "offsets", n * P * 3, torch.float32), _ptr(residual, "residual", n * d), T, H, W, heads, d,
+        _window(window), _ptr(out, "out", n * d), _ptr(lse, "lse", n, torch.float32), code, _stream(stream)))
+
+
+def dsa3d_dwconv3d_forward(x, weight, bias, T, H, W, C, kernel, y, dtype=None, stream=None) -> None:
+    """y <- depthwise 3-D convolution of x (channels-last); see include/dsa3d.h."""
+    lib = load()
+    dt = x.dtype if dtype is None else dtype
+    code = _DTYPES[dt] if isinstance(dt, torch.dtype) else int(dt)
+    taps = int(kernel[0]) * int(kernel[1]) * int(kernel[2])
+    _check(lib.dsa3d_dwconv3d_forward(
+        _ptr(x, "x", T * H * W * C), _ptr(weight, "weight", taps * C, torch.float32),
+        _ptr(bias, "bias", C, torch.float32), T, H, W, C, _window(kernel), _ptr(y, "y", T * H * W * C), code,
+        _stream(stream)))
+
+
+def dsa3d_offsets_linear_forward(u, w, bias, tokens, C, O, offsets, dtype=None, stream=None) -> None:
+    """offsets <- u . w^T + bias (the linear layer of the offset predictor); see include/dsa3d.h."""
+    lib = load()
+    dt = u.dtype if dtype is None else dtype
+    code = _DTYPES[dt] if isinstance(dt, torch.dtype) else int(dt)
+    _check(lib.dsa3d_offsets_linear_forward(
+        _ptr(u, "u", tokens * C), _ptr(w, "w", O * C), _ptr(bias, "bias", O, torch.float32), tokens, C, O,
+        _ptr(offsets, "offsets", tokens * O, torch.float32), code, _stream(stream)))
+
+
+def dsa3d_device_timeout_flag() -> int:
+    return int(load().dsa3d_device_timeout_flag())
 
 
 def dsa3d_backward(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets,

@@ -16,10 +16,7 @@ cudaError_t record(int which, cudaStream_t stream) {
     return g_events[which] ? cudaEventRecord(g_events[which], stream) : cudaSuccess;
 }
 
-int cuda_failed(cudaError_t e) {
-    g_last_cuda_error = static_cast<int>(e);
-    return DSA3D_ERR_CUDA;
-}
+int cuda_failed(cudaError_t e) { return dsa3d::note_cuda_error(e); }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -99,24 +96,43 @@ BackwardWorkspace backward_workspace(const dsa3d::Problem& pr, int dtype, bool t
 
 }  // namespace
 
+int dsa3d::note_cuda_error(cudaError_t e) {
+    g_last_cuda_error = static_cast<int>(e);
+    return DSA3D_ERR_CUDA;
+}
+
 extern "C" {
 
-int dsa3d_forward(const void* q, const void* k, const void* v, const float* offsets, int T, int H, int W,
-                  int heads, int d, const int window[3], void* out, float* lse, int dtype, void* stream) {
+namespace {
+int forward_entry(const void* q, const void* k, const void* v, const float* offsets, const void* addend, int T, int H,
+                  int W, int heads, int d, const int window[3], void* out, float* lse, int dtype, void* stream) {
     if (!q || !k || !v || !offsets || !out || !lse) return DSA3D_ERR_NULL_POINTER;
     dsa3d::Problem pr;
     const int rc = make_problem(T, H, W, heads, d, window, dtype, pr);
     if (rc != DSA3D_OK) return rc;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(offsets) || !aligned16(out) ||
-        !aligned16(lse))
+        !aligned16(lse) || (addend && !aligned16(addend)))
         return DSA3D_ERR_MISALIGNED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = record(0, st);
     if (e != cudaSuccess) return cuda_failed(e);
-    e = dsa3d::launch_forward(q, k, v, offsets, out, lse, pr, dtype == DSA3D_BF16, st);
+    e = dsa3d::launch_forward(q, k, v, offsets, addend, out, lse, pr, dtype == DSA3D_BF16, st);
     if (e != cudaSuccess) return cuda_failed(e);
     e = record(1, st);
     return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
+}
+}  // namespace
+
+int dsa3d_forward(const void* q, const void* k, const void* v, const float* offsets, int T, int H, int W,
+                  int heads, int d, const int window[3], void* out, float* lse, int dtype, void* stream) {
+    return forward_entry(q, k, v, offsets, nullptr, T, H, W, heads, d, window, out, lse, dtype, stream);
+}
+
+int dsa3d_forward_residual(const void* q, const void* k, const void* v, const float* offsets, const void* residual,
+                           int T, int H, int W, int heads, int d, const int window[3], void* out, float* lse,
+                           int dtype, void* stream) {
+    if (!residual) return DSA3D_ERR_NULL_POINTER;
+    return forward_entry(q, k, v, offsets, residual, T, H, W, heads, d, window, out, lse, dtype, stream);
 }
 
 size_t dsa3d_backward_workspace_bytes(int T, int H, int W, int heads, int d, const int window[3], int dtype) {
@@ -255,7 +271,7 @@ int forward_frames(const dsa3d::Problem& full, const void* q, const void* k, con
     const dsa3d::Problem pr = frames_of(full, f0, f1);
     cudaError_t e = record(0, stream);
     if (e != cudaSuccess) return cuda_failed(e);
-    e = dsa3d::launch_forward(q, k, v, offsets, out, lse, pr, bf16, stream);
+    e = dsa3d::launch_forward(q, k, v, offsets, nullptr, out, lse, pr, bf16, stream);
     if (e != cudaSuccess) return cuda_failed(e);
     e = record(1, stream);
     return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);

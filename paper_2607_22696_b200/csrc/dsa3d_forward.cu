@@ -21,10 +21,10 @@ namespace dsa3d {
 #define DSA3D_FWD_MINBLOCKS 3
 #endif
 
-template <typename T, int D, int NV>
+template <typename T, int D, int NV, bool kAdd>
 __global__ void __launch_bounds__(256, NV == 2 ? 2 : DSA3D_FWD_MINBLOCKS)
 forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
-               const float* __restrict__ offsets, T* __restrict__ out, float* __restrict__ lse,
+               const float* __restrict__ offsets, const T* addend, T* out, float* __restrict__ lse,
                const Problem pr) {
     using E = Elt<T, NV>;
     using Row = typename E::Row;
@@ -174,6 +174,12 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
 #pragma unroll
     for (int e = 0; e < VEC; ++e) acc[e] *= inv;
     if (active) {
+        if constexpr (kAdd) {                            // first term of Eq. 1, added before the rounding
+            float add[VEC];
+            E::to_float(E::load(addend + row * D + ch), add);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) acc[e] += add[e];
+        }
         E::store(out + row * D + ch, acc);
         if (gl == 0) lse[row] = (m_run + log2f(l_run)) * kLn2;
     }
@@ -189,24 +195,30 @@ template <> struct LaneWidth<__nv_bfloat16, 128> { static constexpr int NV = DSA
 
 template <typename T, int D>
 static cudaError_t launch_forward_t(const void* q, const void* k, const void* v, const float* offsets,
-                                    void* out, float* lse, const Problem& pr, cudaStream_t stream) {
+                                    const void* addend, void* out, float* lse, const Problem& pr,
+                                    cudaStream_t stream) {
     constexpr int NV = LaneWidth<T, D>::NV;
     constexpr int LPR = D / Elt<T, NV>::VEC;
     constexpr int threads = 256;
     const long long groups_per_block = threads / LPR;
     const long long blocks = (pr.items + groups_per_block - 1) / groups_per_block;
-    forward_kernel<T, D, NV><<<static_cast<unsigned>(blocks), threads, 0, stream>>>(
-        static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), offsets,
-        static_cast<T*>(out), lse, pr);
+    if (addend)
+        forward_kernel<T, D, NV, true><<<static_cast<unsigned>(blocks), threads, 0, stream>>>(
+            static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), offsets,
+            static_cast<const T*>(addend), static_cast<T*>(out), lse, pr);
+    else
+        forward_kernel<T, D, NV, false><<<static_cast<unsigned>(blocks), threads, 0, stream>>>(
+            static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), offsets, nullptr,
+            static_cast<T*>(out), lse, pr);
     return cudaGetLastError();
 }
 
-cudaError_t launch_forward(const void* q, const void* k, const void* v, const float* offsets, void* out,
-                           float* lse, const Problem& pr, bool bf16, cudaStream_t stream) {
+cudaError_t launch_forward(const void* q, const void* k, const void* v, const float* offsets, const void* addend,
+                           void* out, float* lse, const Problem& pr, bool bf16, cudaStream_t stream) {
 #define DSA3D_CASE(DD)                                                                              \
     case DD:                                                                                        \
-        return bf16 ? launch_forward_t<__nv_bfloat16, DD>(q, k, v, offsets, out, lse, pr, stream)   \
-                    : launch_forward_t<float, DD>(q, k, v, offsets, out, lse, pr, stream);
+        return bf16 ? launch_forward_t<__nv_bfloat16, DD>(q, k, v, offsets, addend, out, lse, pr, stream)   \
+                    : launch_forward_t<float, DD>(q, k, v, offsets, addend, out, lse, pr, stream);
     switch (pr.d) {
         DSA3D_CASE(32)
         DSA3D_CASE(64)

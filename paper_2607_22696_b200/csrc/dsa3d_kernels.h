@@ -7,8 +7,14 @@
 
 namespace dsa3d {
 
-cudaError_t launch_forward(const void* q, const void* k, const void* v, const float* offsets, void* out,
-                           float* lse, const Problem& pr, bool bf16, cudaStream_t stream);
+// `addend` (same layout and type as out, or NULL) is added to the attention output before the
+// single rounding to the storage type: the first term of Eq. 1.
+cudaError_t launch_forward(const void* q, const void* k, const void* v, const float* offsets, const void* addend,
+                           void* out, float* lse, const Problem& pr, bool bf16, cudaStream_t stream);
+
+// Remember `e` as the calling thread's last CUDA error (dsa3d_last_cuda_error) and return
+// DSA3D_ERR_CUDA.
+int note_cuda_error(cudaError_t e);
 
 // acc_dk / acc_dv: fp32 accumulators [N, heads, d], zeroed by the caller.  For fp32 storage
 // they are the dk / dv outputs themselves.  coef [N*heads, P] receives the two scatter

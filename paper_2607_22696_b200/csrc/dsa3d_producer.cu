@@ -1,0 +1,494 @@
+// The two layers that surround the attention operator in Eq. 1 and feed it its offsets:
+//   dwconv3d_kernel        depthwise 3-D convolution on channels-last activations (first term of
+//                          Eq. 1; first stage of the offset predictor of the Formulation section)
+//   offsets_gemm_kernel    offsets = u . w^T + bias, the linear layer of the offset predictor, as
+//                          a dense bf16 contraction on the 5th-generation tensor cores:
+//                          TMA tiles (128-byte swizzle) -> tcgen05.mma -> fp32 accumulators in
+//                          TMEM -> bias + fp32 stores.  Persistent, one CTA per SM, warp-
+//                          specialised (TMA producer, MMA issuer, four epilogue warps), four
+//                          shared-memory stages, two TMEM accumulator buffers so the epilogue of
+//                          one tile overlaps the contraction of the next.
+//   offsets_linear_f32_kernel  the same layer in plain fp32 FMAs for fp32 storage.
+// Every wait on an mbarrier is bounded; a wait that runs out raises a device flag (readable
+// with dsa3d_device_timeout_flag) and the roles drain and free TMEM instead of spinning.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <mutex>
+
+#include "../../include/dsa3d.h"
+#include "dsa3d_kernels.h"
+
+namespace {
+
+__device__ int g_timeout_flag = 0;
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ------------------------------------------------------------------------------------------
+// Depthwise convolution.  A thread owns 8 consecutive channels (one 16-byte vector of bf16,
+// two of fp32) of RX = 8 consecutive outputs along x; per (dt, dy) row of the kernel it loads
+// the kw weight vectors and the RX + kw - 1 input vectors once and slides the taps over them
+// in registers.  Consecutive threads take consecutive channel vectors (coalesced rows).
+// ------------------------------------------------------------------------------------------
+constexpr int kConvRX = 8;
+constexpr int kConvMaxKw = 7;
+
+template <typename T> struct Vec8;
+template <> struct Vec8<__nv_bfloat16> {
+    using Raw = uint4;
+    static __device__ __forceinline__ Raw load_raw(const __nv_bfloat16* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+    static __device__ __forceinline__ Raw zero_raw() { return make_uint4(0u, 0u, 0u, 0u); }
+    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&f)[8]) { widen(load_raw(p), f); }
+    static __device__ __forceinline__ void widen(const Raw& r, float (&f)[8]) {
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __uint_as_float(w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    }
+    static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&f)[8]) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+            w[i] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+template <> struct Vec8<float> {
+    struct Raw { float4 a, b; };
+    static __device__ __forceinline__ Raw load_raw(const float* p) {
+        Raw r;
+        r.a = __ldg(reinterpret_cast<const float4*>(p));
+        r.b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+        return r;
+    }
+    static __device__ __forceinline__ Raw zero_raw() {
+        Raw r;
+        r.a = r.b = make_float4(0.f, 0.f, 0.f, 0.f);
+        return r;
+    }
+    static __device__ __forceinline__ void load(const float* p, float (&f)[8]) { widen(load_raw(p), f); }
+    static __device__ __forceinline__ void widen(const Raw& r, float (&f)[8]) {
+        f[0] = r.a.x; f[1] = r.a.y; f[2] = r.a.z; f[3] = r.a.w; f[4] = r.b.x; f[5] = r.b.y; f[6] = r.b.z; f[7] = r.b.w;
+    }
+    static __device__ __forceinline__ void store(float* p, const float (&f)[8]) {
+        reinterpret_cast<float4*>(p)[0] = make_float4(f[0], f[1], f[2], f[3]);
+        reinterpret_cast<float4*>(p)[1] = make_float4(f[4], f[5], f[6], f[7]);
+    }
+};
+
+// KW > 0: kernel width known at compile time (weights of a kernel row held in registers, the
+// slide fully unrolled); KW == 0: any width up to kConvMaxKw, weights re-read per use.
+template <typename T, int KW>
+__global__ void __launch_bounds__(256)
+dwconv3d_kernel(const T* __restrict__ x, const float* __restrict__ weight, const float* __restrict__ bias,
+                T* __restrict__ y, int Tn, int H, int W, int C, int kt, int kh, int kw_rt) {
+    const int kw = KW > 0 ? KW : kw_rt;
+    const int cvecs = C / 8;
+    const int xruns = (W + kConvRX - 1) / kConvRX;
+    const long long total = static_cast<long long>(Tn) * H * xruns * cvecs;
+    const long long id = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (id >= total) return;
+    const int cv = static_cast<int>(id % cvecs);
+    long long rest = id / cvecs;
+    const int xr = static_cast<int>(rest % xruns); rest /= xruns;
+    const int yy = static_cast<int>(rest % H);
+    const int tt = static_cast<int>(rest / H);
+    const int c0 = cv * 8, x0 = xr * kConvRX;
+
+    float acc[kConvRX][8];
+#pragma unroll
+    for (int r = 0; r < kConvRX; ++r)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[r][e] = bias ? __ldg(bias + c0 + e) : 0.0f;
+
+    for (int i = 0; i < kt; ++i) {
+        const int st = tt + i - kt / 2;
+        if (st < 0 || st >= Tn) continue;
+        for (int j = 0; j < kh; ++j) {
+            const int sy = yy + j - kh / 2;
+            if (sy < 0 || sy >= H) continue;
+            const T* row = x + (static_cast<long long>(st) * H + sy) * W * C + c0;
+            const float* wrow = weight + static_cast<long long>((i * kh + j) * kw) * C + c0;
+            if constexpr (KW > 0) {
+                float wv[KW][8];
+#pragma unroll
+                for (int l = 0; l < KW; ++l) {
+                    const float4 wa = __ldg(reinterpret_cast<const float4*>(wrow + static_cast<long long>(l) * C));
+                    const float4 wb = __ldg(reinterpret_cast<const float4*>(wrow + static_cast<long long>(l) * C) + 1);
+                    wv[l][0] = wa.x; wv[l][1] = wa.y; wv[l][2] = wa.z; wv[l][3] = wa.w;
+                    wv[l][4] = wb.x; wv[l][5] = wb.y; wv[l][6] = wb.z; wv[l][7] = wb.w;
+                }
+                // all input vectors of this kernel row first (RX + KW - 1 independent loads in
+                // flight), then the slide
+                typename Vec8<T>::Raw raw[KW + kConvRX - 1];
+#pragma unroll
+                for (int s = 0; s < KW + kConvRX - 1; ++s) {
+                    const int sx = x0 + s - KW / 2;
+                    raw[s] = (sx >= 0 && sx < W) ? Vec8<T>::load_raw(row + static_cast<long long>(sx) * C)
+                                                 : Vec8<T>::zero_raw();
+                }
+#pragma unroll
+                for (int s = 0; s < KW + kConvRX - 1; ++s) {
+                    float in[8];
+                    Vec8<T>::widen(raw[s], in);
+#pragma unroll
+                    for (int r = 0; r < kConvRX; ++r) {
+                        const int l = s - r;                      // tap that maps input s to output r
+                        if (l < 0 || l >= KW) continue;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[r][e] = fmaf(wv[l][e], in[e], acc[r][e]);
+                    }
+                }
+            } else {
+                for (int s = 0; s < kw + kConvRX - 1; ++s) {
+                    const int sx = x0 + s - kw / 2;
+                    if (sx < 0 || sx >= W) continue;
+                    float in[8];
+                    Vec8<T>::load(row + static_cast<long long>(sx) * C, in);
+#pragma unroll
+                    for (int r = 0; r < kConvRX; ++r) {
+                        const int l = s - r;
+                        if (l < 0 || l >= kw) continue;
+                        const float4 wa = __ldg(reinterpret_cast<const float4*>(wrow + static_cast<long long>(l) * C));
+                        const float4 wb = __ldg(reinterpret_cast<const float4*>(wrow + static_cast<long long>(l) * C) + 1);
+                        const float wv[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[r][e] = fmaf(wv[e], in[e], acc[r][e]);
+                    }
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < kConvRX; ++r) {
+        const int ox = x0 + r;
+        if (ox < W) Vec8<T>::store(y + ((static_cast<long long>(tt) * H + yy) * W + ox) * C + c0, acc[r]);
+    }
+}
+
+template <typename T>
+void launch_dwconv(const void* x, const float* weight, const float* bias, void* y, int T_, int H, int W, int C,
+                   const int kernel[3], unsigned blocks, cudaStream_t st) {
+    const T* xp = static_cast<const T*>(x);
+    T* yp = static_cast<T*>(y);
+#define DSA3D_CONV_CASE(KW) \
+    case KW: dwconv3d_kernel<T, KW><<<blocks, 256, 0, st>>>(xp, weight, bias, yp, T_, H, W, C, kernel[0], kernel[1], KW); break;
+    switch (kernel[2]) {
+        DSA3D_CONV_CASE(1)
+        DSA3D_CONV_CASE(3)
+        DSA3D_CONV_CASE(5)
+        DSA3D_CONV_CASE(7)
+        default: dwconv3d_kernel<T, 0><<<blocks, 256, 0, st>>>(xp, weight, bias, yp, T_, H, W, C, kernel[0], kernel[1], kernel[2]);
+    }
+#undef DSA3D_CONV_CASE
+}
+
+// ------------------------------------------------------------------------------------------
+// Linear layer on tensor cores.
+// ------------------------------------------------------------------------------------------
+constexpr int BM = 128, BK = 64, kStages = 4, kMaxBN = 256;
+constexpr int kGemmThreads = 192;                 // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Bounded wait for the phase of parity `parity` to complete; false when it gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+// Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes with the
+// 128-byte swizzle (what the TMA load above writes): 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
+    uint64_t d = static_cast<uint64_t>((saddr >> 4) & 0x3fff);
+    d |= static_cast<uint64_t>(1) << 16;            // leading byte offset: unused with this layout
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;    // stride byte offset between 8-row groups
+    d |= static_cast<uint64_t>(1) << 46;            // descriptor version of this architecture
+    d |= static_cast<uint64_t>(2) << 61;            // 128-byte swizzle
+    return d;
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_load_32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+struct __align__(1024) GemmSmem {
+    __nv_bfloat16 a[kStages][BM * BK];
+    __nv_bfloat16 b[kStages][kMaxBN * BK];
+    uint64_t full[kStages], empty[kStages], acc_full[2], acc_empty[2];
+    uint32_t tmem_base;
+};
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+offsets_gemm_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_constant__ CUtensorMap map_w,
+                    const float* __restrict__ bias, float* __restrict__ out, long long M, int N, int K, int BN,
+                    long long m_tiles, int n_tiles) {
+    extern __shared__ unsigned char raw[];
+    GemmSmem& s = *reinterpret_cast<GemmSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int kblocks = (K + BK - 1) / BK;
+    const long long tiles = m_tiles * n_tiles;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&s.full[i]), 1); mbar_init(smem_u32(&s.empty[i]), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&s.acc_full[i]), 1); mbar_init(smem_u32(&s.acc_empty[i]), 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) {                               // both accumulator buffers: all 512 columns
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&s.tmem_base)), "r"(2 * kMaxBN));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = s.tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0;                       // k-block counter across tiles: stage and phase
+            for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+                const int n0 = static_cast<int>(tile % n_tiles) * BN;
+                const long long m0 = (tile / n_tiles) * BM;
+                bool ok = true;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int st = it % kStages;
+                    if (!mbar_wait(smem_u32(&s.empty[st]), ((it / kStages) & 1) ^ 1)) { ok = false; break; }
+                    mbar_expect_tx(smem_u32(&s.full[st]), static_cast<uint32_t>((BM + BN) * BK * 2));
+                    tma_load_2d(smem_u32(s.a[st]), &map_u, smem_u32(&s.full[st]), kb * BK, static_cast<int>(m0));
+                    tma_load_2d(smem_u32(s.b[st]), &map_w, smem_u32(&s.full[st]), kb * BK, n0);
+                }
+                if (!ok) { atomicExch(&g_timeout_flag, 1); break; }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
+                                   (static_cast<uint32_t>(BM >> 4) << 24);   // fp32 accumulate, bf16 x bf16, K-major
+            uint32_t it = 0, local = 0;
+            bool ok = true;
+            for (long long tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++local) {
+                const uint32_t buf = local & 1;
+                if (!mbar_wait(smem_u32(&s.acc_empty[buf]), ((local >> 1) & 1) ^ 1)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t d_tmem = tmem + buf * kMaxBN;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int st = it % kStages;
+                    if (!mbar_wait(smem_u32(&s.full[st]), (it / kStages) & 1)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint64_t da = smem_desc(smem_u32(s.a[st])), db = smem_desc(smem_u32(s.b[st]));
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)                         // 16 channels = 32 bytes per step
+                        umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) ? 1u : 0u);
+                    umma_commit(smem_u32(&s.empty[st]));                      // stage free once these MMAs have read it
+                }
+                umma_commit(smem_u32(&s.acc_full[buf]));
+            }
+            if (!ok) atomicExch(&g_timeout_flag, 2);
+        }
+    } else {
+        const int quarter = warp & 3;                 // the 32 TMEM lanes this warp can read
+        uint32_t local = 0;
+        for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++local) {
+            const uint32_t buf = local & 1;
+            const int n0 = static_cast<int>(tile % n_tiles) * BN;
+            const long long row = (tile / n_tiles) * BM + quarter * 32 + lane;
+            if (!mbar_wait(smem_u32(&s.acc_full[buf]), (local >> 1) & 1)) {
+                if (lane == 0) atomicExch(&g_timeout_flag, 3);
+                break;
+            }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                tmem_load_32(tmem + (static_cast<uint32_t>(quarter * 32) << 16) + buf * kMaxBN + c0, r);
+                if (row < M) {
+                    float* dst = out + row * N + n0 + c0;
+                    if (n0 + c0 + 32 <= N && (N & 3) == 0) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const float4 b4 = __ldg(reinterpret_cast<const float4*>(bias + n0 + c0 + j));
+                            *reinterpret_cast<float4*>(dst + j) =
+                                make_float4(__uint_as_float(r[j]) + b4.x, __uint_as_float(r[j + 1]) + b4.y,
+                                            __uint_as_float(r[j + 2]) + b4.z, __uint_as_float(r[j + 3]) + b4.w);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (n0 + c0 + j < N) dst[j] = __uint_as_float(r[j]) + __ldg(bias + n0 + c0 + j);
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s.acc_empty[buf]));
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 2) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(2 * kMaxBN));
+}
+
+// fp32 storage: one thread per output, plain fp32 FMAs in channel order.
+__global__ void __launch_bounds__(256)
+offsets_linear_f32_kernel(const float* __restrict__ u, const float* __restrict__ w, const float* __restrict__ bias,
+                          float* __restrict__ out, long long M, int N, int K) {
+    const long long id = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (id >= M * N) return;
+    const long long m = id / N;
+    const int n = static_cast<int>(id - m * N);
+    const float* ur = u + m * K;
+    const float* wr = w + static_cast<long long>(n) * K;
+    float acc = 0.0f;
+    for (int c = 0; c < K; ++c) acc = fmaf(__ldg(ur + c), __ldg(wr + c), acc);
+    out[id] = acc + (bias ? __ldg(bias + n) : 0.0f);
+}
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult res;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &res) == cudaSuccess &&
+            res == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+// Row-major [rows, cols] bf16 matrix, tiles of box_rows x 64 columns, 128-byte swizzle, zero fill
+// outside the matrix.
+bool make_map(CUtensorMap* map, const void* ptr, unsigned long long rows, unsigned long long cols, unsigned box_rows) {
+    EncodeTiledFn enc = encode_tiled();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {BK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int cuda_failed(cudaError_t e) { return dsa3d::note_cuda_error(e); }
+
+}  // namespace
+
+extern "C" {
+
+int dsa3d_dwconv3d_forward(const void* x, const float* weight, const float* bias, int T, int H, int W, int C,
+                           const int kernel[3], void* y, int dtype, void* stream) {
+    if (!x || !weight || !y || !kernel) return DSA3D_ERR_NULL_POINTER;
+    if (T < 1 || H < 1 || W < 1 || C < 8 || C % 8) return DSA3D_ERR_BAD_SHAPE;
+    if (kernel[0] < 1 || kernel[1] < 1 || kernel[2] < 1 || kernel[2] > kConvMaxKw || kernel[0] > 15 || kernel[1] > 15)
+        return DSA3D_ERR_BAD_SHAPE;
+    if (dtype != DSA3D_F32 && dtype != DSA3D_BF16) return DSA3D_ERR_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(y) || !aligned16(weight) || (bias && !aligned16(bias))) return DSA3D_ERR_MISALIGNED;
+    const long long total = static_cast<long long>(T) * H * ((W + kConvRX - 1) / kConvRX) * (C / 8);
+    const long long blocks = (total + 255) / 256;
+    if (blocks > 0x7fffffffLL) return DSA3D_ERR_BAD_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (dtype == DSA3D_BF16)
+        launch_dwconv<__nv_bfloat16>(x, weight, bias, y, T, H, W, C, kernel, static_cast<unsigned>(blocks), st);
+    else
+        launch_dwconv<float>(x, weight, bias, y, T, H, W, C, kernel, static_cast<unsigned>(blocks), st);
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
+}
+
+int dsa3d_offsets_linear_forward(const void* u, const void* w, const float* bias, long long tokens, int C, int O,
+                                 float* offsets, int dtype, void* stream) {
+    if (!u || !w || !bias || !offsets) return DSA3D_ERR_NULL_POINTER;
+    if (tokens < 1 || C < 8 || C % 8 || O < 1 || tokens > 0x7fffffffLL) return DSA3D_ERR_BAD_SHAPE;
+    if (dtype != DSA3D_F32 && dtype != DSA3D_BF16) return DSA3D_ERR_UNSUPPORTED;
+    if (!aligned16(u) || !aligned16(w) || !aligned16(bias) || !aligned16(offsets)) return DSA3D_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (dtype == DSA3D_F32) {
+        const long long blocks = (tokens * O + 255) / 256;
+        if (blocks > 0x7fffffffLL) return DSA3D_ERR_BAD_SHAPE;
+        offsets_linear_f32_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(
+            static_cast<const float*>(u), static_cast<const float*>(w), bias, offsets, tokens, O, C);
+        const cudaError_t e = cudaGetLastError();
+        return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
+    }
+    // column tiles of equal width, a multiple of 32 columns, at most 256
+    const int n_tiles = (O + kMaxBN - 1) / kMaxBN;
+    const int BN = ((O + n_tiles - 1) / n_tiles + 31) / 32 * 32;
+    const long long m_tiles = (tokens + BM - 1) / BM;
+    CUtensorMap map_u, map_w;
+    if (!make_map(&map_u, u, static_cast<unsigned long long>(tokens), static_cast<unsigned long long>(C), BM) ||
+        !make_map(&map_w, w, static_cast<unsigned long long>(O), static_cast<unsigned long long>(C),
+                  static_cast<unsigned>(BN)))
+        return DSA3D_ERR_UNSUPPORTED;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_failed(e);
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_failed(e);
+    const size_t smem = sizeof(GemmSmem) + 1024;
+    e = cudaFuncSetAttribute(offsets_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return cuda_failed(e);
+    const long long tiles = m_tiles * n_tiles;
+    const int grid = static_cast<int>(tiles < sms ? tiles : sms);
+    offsets_gemm_kernel<<<grid, kGemmThreads, smem, st>>>(map_u, map_w, bias, offsets, tokens, O, C, BN, m_tiles,
+                                                           n_tiles);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
+}
+
+int dsa3d_device_timeout_flag(void) {
+    int flag = 0;
+    if (cudaMemcpyFromSymbol(&flag, g_timeout_flag, sizeof(int)) != cudaSuccess) return -1;
+    return flag;
+}
+
+}  // extern "C"
