@@ -373,6 +373,128 @@ offsets_gemm_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_cons
     if (warp == 2) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(2 * kMaxBN));
 }
 
+// ------------------------------------------------------------------------------------------
+// Depthwise convolution, bf16, staged through shared memory by TMA.  A CTA owns a column of
+// the grid - TY x TX positions, 64 channels (one 128-byte row per position) - and marches
+// along t.  Each input plane of the column (with its kh-1 / kw-1 halo, zero-filled by the
+// TMA unit outside the grid) is fetched once into a ring of kt+1 shared-memory slots, one
+// plane ahead of the arithmetic; a thread produces 4 outputs along x for 8 channels and
+// slides the kernel row over kw+3 shared-memory vectors held in registers.
+// ------------------------------------------------------------------------------------------
+constexpr int kCvTY = 4, kCvTX = 16, kCvRX = 4, kCvCh = 64, kCvThreads = 128, kCvMaxKt = 7;
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+
+template <int KW>
+__global__ void __launch_bounds__(kCvThreads)
+dwconv3d_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* __restrict__ weight,
+                    const float* __restrict__ bias, __nv_bfloat16* __restrict__ y, int Tn, int H, int W, int C,
+                    int kt, int kh, int t_chunk) {
+    extern __shared__ unsigned char raw_smem[];
+    unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(raw_smem) + 127) & ~uintptr_t(127));
+    const int ring = kt + 1;
+    const int ph = kCvTY + kh - 1, pw = kCvTX + KW - 1;                 // plane extent with halo
+    const uint32_t plane_bytes = static_cast<uint32_t>(ph * pw * kCvCh * 2);
+    float* wsm = reinterpret_cast<float*>(base + static_cast<size_t>(ring) * plane_bytes);   // [taps][64]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(wsm + kt * kh * KW * kCvCh);                 // [ring]
+
+    const int tid = threadIdx.x;
+    const int cv = tid & 7, xg = (tid >> 3) & 3, yl = tid >> 5;         // 8 channel vectors x 4 x-groups x 4 rows
+    const int c0 = blockIdx.x * kCvCh;
+    const int tiles_x = (W + kCvTX - 1) / kCvTX;
+    const int x0 = (blockIdx.y % tiles_x) * kCvTX, y0 = (blockIdx.y / tiles_x) * kCvTY;
+    const int t_begin = blockIdx.z * t_chunk, t_end = min(Tn, t_begin + t_chunk);
+    const int lo = kt / 2;                                              // planes t-lo .. t-lo+kt-1 feed output t
+
+    for (int i = tid; i < kt * kh * KW * kCvCh; i += kCvThreads)
+        wsm[i] = __ldg(weight + static_cast<long long>(i / kCvCh) * C + c0 + (i % kCvCh));
+    if (tid == 0) {
+        for (int i = 0; i < ring; ++i) mbar_init(smem_u32(&bars[i]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    // plane index n = p - (t_begin - lo) counts the planes of this CTA from 0; slot n % ring
+    auto issue = [&](int n) {
+        const int p = t_begin - lo + n, slot = n % ring;
+        mbar_expect_tx(smem_u32(&bars[slot]), plane_bytes);
+        tma_load_4d(smem_u32(base + static_cast<size_t>(slot) * plane_bytes), &map_x, smem_u32(&bars[slot]), c0,
+                    x0 - KW / 2, y0 - kh / 2, p);
+    };
+    if (tid == 0)
+        for (int n = 0; n < kt; ++n) issue(n);
+
+    float bias_v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) bias_v[e] = bias ? __ldg(bias + c0 + cv * 8 + e) : 0.0f;
+    const int oy = y0 + yl, ox0 = x0 + xg * kCvRX;
+    bool ok = true;
+
+    for (int t = t_begin; t < t_end && ok; ++t) {
+        const int n_last = t - t_begin + kt - 1;                        // newest plane output t needs
+        if (tid == 0 && t + 1 < t_end) issue(n_last + 1);              // its slot was last read by output t-1
+        // the first output waits for all of its kt planes, later ones only for the newest
+        for (int n = (t == t_begin ? n_last - (kt - 1) : n_last); n <= n_last; ++n)
+            if (!mbar_wait(smem_u32(&bars[n % ring]), (n / ring) & 1)) {
+                atomicExch(&g_timeout_flag, 4);
+                ok = false;
+                break;
+            }
+        float acc[kCvRX][8];
+#pragma unroll
+        for (int r = 0; r < kCvRX; ++r)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[r][e] = bias_v[e];
+        if (ok) {
+            for (int i = 0; i < kt; ++i) {
+                const int n = t - t_begin + i;                          // plane t - lo + i
+                const unsigned char* plane = base + static_cast<size_t>(n % ring) * plane_bytes;
+                for (int j = 0; j < kh; ++j) {
+                    const unsigned char* row = plane + (static_cast<size_t>(yl + j) * pw + xg * kCvRX) * (kCvCh * 2) + cv * 16;
+                    const float* wrow = wsm + (i * kh + j) * KW * kCvCh + cv * 8;
+                    float wv[KW][8];
+#pragma unroll
+                    for (int l = 0; l < KW; ++l) {
+                        const float4 wa = *reinterpret_cast<const float4*>(wrow + l * kCvCh);
+                        const float4 wb = *reinterpret_cast<const float4*>(wrow + l * kCvCh + 4);
+                        wv[l][0] = wa.x; wv[l][1] = wa.y; wv[l][2] = wa.z; wv[l][3] = wa.w;
+                        wv[l][4] = wb.x; wv[l][5] = wb.y; wv[l][6] = wb.z; wv[l][7] = wb.w;
+                    }
+                    uint4 in_raw[KW + kCvRX - 1];
+#pragma unroll
+                    for (int s = 0; s < KW + kCvRX - 1; ++s)
+                        in_raw[s] = *reinterpret_cast<const uint4*>(row + s * (kCvCh * 2));
+#pragma unroll
+                    for (int s = 0; s < KW + kCvRX - 1; ++s) {
+                        float in[8];
+                        Vec8<__nv_bfloat16>::widen(in_raw[s], in);
+#pragma unroll
+                        for (int r = 0; r < kCvRX; ++r) {
+                            const int l = s - r;
+                            if (l < 0 || l >= KW) continue;
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) acc[r][e] = fmaf(wv[l][e], in[e], acc[r][e]);
+                        }
+                    }
+                }
+            }
+            if (oy < H) {
+#pragma unroll
+                for (int r = 0; r < kCvRX; ++r)
+                    if (ox0 + r < W)
+                        Vec8<__nv_bfloat16>::store(
+                            y + ((static_cast<long long>(t) * H + oy) * W + ox0 + r) * C + c0 + cv * 8, acc[r]);
+            }
+        }
+        __syncthreads();                                                // plane t - lo may now be overwritten
+    }
+}
+
 // fp32 storage: one thread per output, plain fp32 FMAs in channel order.
 __global__ void __launch_bounds__(256)
 offsets_linear_f32_kernel(const float* __restrict__ u, const float* __restrict__ w, const float* __restrict__ bias,
@@ -419,6 +541,64 @@ bool make_map(CUtensorMap* map, const void* ptr, unsigned long long rows, unsign
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Channels-last activations [T, H, W, C] bf16 as a 4-D map with boxes of 64 channels x pw x ph x 1.
+bool make_map_activations(CUtensorMap* map, const void* ptr, int T, int H, int W, int C, int pw, int ph) {
+    EncodeTiledFn enc = encode_tiled();
+    if (!enc) return false;
+    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W), static_cast<cuuint64_t>(H),
+                                static_cast<cuuint64_t>(T)};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(C) * 2, static_cast<cuuint64_t>(W) * C * 2,
+                                   static_cast<cuuint64_t>(H) * W * C * 2};
+    const cuuint32_t box[4] = {kCvCh, static_cast<cuuint32_t>(pw), static_cast<cuuint32_t>(ph), 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Launch the staged kernel if the shape suits it; returns false when the caller should use the
+// plain kernel instead (fp32, odd channel counts, wide kernels).  *err receives a launch error.
+bool try_dwconv_tma(const void* x, const float* weight, const float* bias, void* y, int T, int H, int W, int C,
+                    const int kernel[3], cudaStream_t st, cudaError_t* err) {
+    *err = cudaSuccess;
+    const int kt = kernel[0], kh = kernel[1], kw = kernel[2];
+    if (C % kCvCh || kt > kCvMaxKt || (kw != 1 && kw != 3 && kw != 5 && kw != 7)) return false;
+    const int ph = kCvTY + kh - 1, pw = kCvTX + kw - 1;
+    if (ph > 256 || pw > 256) return false;
+    const size_t plane = static_cast<size_t>(ph) * pw * kCvCh * 2;
+    const size_t smem = 128 + (kt + 1) * plane + static_cast<size_t>(kt) * kh * kw * kCvCh * 4 + (kt + 1) * 8;
+    if (smem > 200 * 1024) return false;
+    CUtensorMap map;
+    if (!make_map_activations(&map, x, T, H, W, C, pw, ph)) return false;
+    const int tiles = ((W + kCvTX - 1) / kCvTX) * ((H + kCvTY - 1) / kCvTY);
+    if (tiles > 65535) return false;
+    // split t so that the grid fills the GPU a few times over, but keep chunks long enough to
+    // amortise the kt-1 planes of run-in
+    int splits = 1;
+    const long long columns = static_cast<long long>(C / kCvCh) * tiles;
+    while (columns * splits < 148 * 8 && T / (splits * 2) >= 4 * kt) splits *= 2;
+    const int t_chunk = (T + splits - 1) / splits;
+    const dim3 grid(C / kCvCh, tiles, (T + t_chunk - 1) / t_chunk);
+#define DSA3D_CONV_TMA_CASE(KW)                                                                                    \
+    case KW:                                                                                                       \
+        *err = cudaFuncSetAttribute(dwconv3d_tma_kernel<KW>, cudaFuncAttributeMaxDynamicSharedMemorySize,          \
+                                    static_cast<int>(smem));                                                       \
+        if (*err == cudaSuccess) {                                                                                 \
+            dwconv3d_tma_kernel<KW><<<grid, kCvThreads, smem, st>>>(map, weight, bias, static_cast<__nv_bfloat16*>(y), \
+                                                                    T, H, W, C, kt, kh, t_chunk);                  \
+            *err = cudaGetLastError();                                                                             \
+        }                                                                                                          \
+        break;
+    switch (kw) {
+        DSA3D_CONV_TMA_CASE(1)
+        DSA3D_CONV_TMA_CASE(3)
+        DSA3D_CONV_TMA_CASE(5)
+        DSA3D_CONV_TMA_CASE(7)
+    }
+#undef DSA3D_CONV_TMA_CASE
+    return true;
+}
+
 int cuda_failed(cudaError_t e) { return dsa3d::note_cuda_error(e); }
 
 }  // namespace
@@ -437,6 +617,11 @@ int dsa3d_dwconv3d_forward(const void* x, const float* weight, const float* bias
     const long long blocks = (total + 255) / 256;
     if (blocks > 0x7fffffffLL) return DSA3D_ERR_BAD_SHAPE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (dtype == DSA3D_BF16) {
+        cudaError_t te;
+        if (try_dwconv_tma(x, weight, bias, y, T, H, W, C, kernel, st, &te))
+            return te == cudaSuccess ? DSA3D_OK : cuda_failed(te);
+    }
     if (dtype == DSA3D_BF16)
         launch_dwconv<__nv_bfloat16>(x, weight, bias, y, T, H, W, C, kernel, static_cast<unsigned>(blocks), st);
     else

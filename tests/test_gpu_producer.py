@@ -38,6 +38,32 @@ def test_dwconv3d_matches_the_oracle(dtype, shape, kernel):
         pu.assert_close("dwconv3d", y, ref, dtype)
 
 
+@pytest.mark.parametrize("shape,kernel", [((6, 7, 19, 64), (3, 3, 3)), ((48, 4, 16, 64), (3, 3, 3)),
+                                          ((5, 9, 33, 128), (3, 7, 7)), ((4, 5, 6, 64), (1, 1, 1)),
+                                          ((9, 3, 40, 192), (5, 3, 5)), ((2, 1, 1, 64), (7, 5, 7)),
+                                          ((40, 6, 17, 64), (2, 4, 3))])
+def test_dwconv3d_staged_kernel_matches_the_oracle(shape, kernel):
+    """bf16 with a multiple of 64 channels takes the kernel that stages planes in shared
+    memory with TMA and marches along t: grids that are not multiples of the 4 x 16 tile,
+    fewer frames than kernel taps, even kernel sizes, and grids small enough that the march
+    is cut into several chunks of frames (whose first planes are real data, not padding)."""
+    T, H, W, C = shape
+    taps = kernel[0] * kernel[1] * kernel[2]
+    x = _normal(shape, 101, 0, 1.0, BF16)
+    w = _normal((taps, C), 101, 1, 0.3, F32)
+    bias = _normal((C,), 101, 2, 0.5, F32)
+    ref = producer.dwconv3d(x, w, bias, kernel)
+    y = torch.full(shape, float("nan"), dtype=BF16, device="cuda")
+    guard = torch.full((64,), 3.0, dtype=F32, device="cuda")
+    xd, wd, bd = x.cuda(), w.cuda(), bias.cuda()
+    for _ in range(2):
+        binding.dsa3d_dwconv3d_forward(xd, wd, bd, T, H, W, C, kernel, y)
+    torch.cuda.synchronize()
+    assert binding.dsa3d_device_timeout_flag() == 0
+    pu.assert_close("dwconv3d", y, ref, BF16)
+    assert torch.equal(guard.cpu(), torch.full((64,), 3.0))
+
+
 @pytest.mark.parametrize("tokens,C,O", [(300, 192, 162), (128, 64, 32), (1000, 256, 1296), (77, 200, 40),
                                         (513, 128, 520), (1, 8, 1), (260, 2048, 81)])
 def test_offsets_linear_bf16_on_tensor_cores(tokens, C, O):
