@@ -235,6 +235,59 @@ def aggregate_mtokens_per_s(wl, world: int, step_ms: float) -> float:
 
 # ------------------------------------------------------------------------------ GPU arm
 
+def measure_producer(wl, dev, reps: int = 5):
+    """Times the layers around the operator (Eq. 1 first term and the offset predictor) on the
+    workload's grid with hidden size heads*d: two 3x3x3 depthwise convolutions, the
+    offset-producing linear layer on the tensor cores, and the forward with the convolution
+    term added.  Buffers are freed before the main measurement allocates its own."""
+    from paper_2607_22696_b200 import binding
+    T, H, W, heads, d = wl.T, wl.H, wl.W, wl.heads, wl.d
+    C, O, N = heads * d, heads * wl.P * 3, wl.N
+    x = inputs.normal((T, H, W, C), wl.seed, 20, 1.0, wl.dtype, dev)
+    wc = inputs.normal((27, C), wl.seed, 21, 0.2, torch.float32, dev)
+    wlin = inputs.normal((O, C), wl.seed, 22, wl.sigma / math.sqrt(C), wl.dtype, dev)
+    blin = inputs.normal((O,), wl.seed, 23, 0.1, torch.float32, dev)
+    u = torch.empty_like(x)
+    off = torch.empty((N, O), dtype=torch.float32, device=dev)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize(dev)
+        return e0.elapsed_time(e1) / reps
+
+    conv_ms = timed(lambda: binding.dsa3d_dwconv3d_forward(x, wc, None, T, H, W, C, (3, 3, 3), u))
+    gemm_ms = timed(lambda: binding.dsa3d_offsets_linear_forward(u, wlin, blin, N, C, O, off))
+    flag = binding.dsa3d_device_timeout_flag()
+    elt = wl.elt
+    peaks = {}
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peaks = json.load(f)
+    except (OSError, ValueError):
+        pass
+    tf_peak = float(peaks.get("bf16_tflops", 1590.0))
+    hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
+    gemm_tf = 2.0 * N * C * O / (gemm_ms * 1e-3) / 1e12
+    conv_gbs = 2.0 * N * C * elt / (conv_ms * 1e-3) / 1e9
+    res = {"hidden": C, "offset_outputs": O, "timeout_flag": flag,
+           "dwconv3d_3x3x3": {"ms": conv_ms, "bound": "hbm", "achieved": conv_gbs, "peak": hbm_peak, "unit": "GB/s",
+                              "frac": conv_gbs / hbm_peak, "algorithmic_bytes": 2.0 * N * C * elt},
+           "offsets_linear": {"ms": gemm_ms, "bound": "tensor", "achieved": gemm_tf, "peak": tf_peak,
+                              "unit": "TFLOP/s", "frac": gemm_tf / tf_peak, "dtype": "bf16 x bf16 -> f32",
+                              "peak_source": "measured burst (MEASURED_PEAKS.json bf16_tflops)" if peaks else "fallback"},
+           "per_layer_ms": 2 * conv_ms + gemm_ms}
+    del x, wc, wlin, blin, u, off
+    torch.cuda.empty_cache()
+    return res
+
+
 def run_ours(args, wl):
     from paper_2607_22696_b200 import binding
     import torch.distributed as dist
@@ -258,6 +311,10 @@ def run_ours(args, wl):
 
     binding.load()
     dims = (wl.T, wl.H, wl.W, wl.heads, wl.d)
+    producer = None
+    if args.producer and rank == 0 and wl.dtype == torch.bfloat16:
+        producer = measure_producer(wl, dev)
+    barrier()
     # every rank takes its own video of the batch: same shape, its own seed
     wl_rank = rank_workload(wl, rank)
     t = inputs.make_inputs(wl_rank, dev, with_dout=True)
@@ -380,7 +437,7 @@ def run_ours(args, wl):
                      "onchip": onchip,
                      "whole_step": {"bytes": step_bytes, "achieved": step_bytes / (step_ms * 1e-3) / 1e9,
                                     "frac": step_bytes / (step_ms * 1e-3) / 1e9 / peak}},
-        "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+        "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks, "producer": producer,
         "gpu_launches": K * ((5 if tiled else 4) if (wl.backward and wl.dtype == torch.bfloat16)
                              else 2 if wl.backward else 1),
     }
@@ -480,6 +537,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--producer", action="store_true",
+                    help="also time the depthwise convolution and the offset-producing linear layer (bf16 workloads)")
     args = ap.parse_args()
     wl = inputs.WORKLOADS[args.workload]
     if args.impl == "reference":
