@@ -411,8 +411,13 @@ dwconv3d_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* __re
     const int t_begin = blockIdx.z * t_chunk, t_end = min(Tn, t_begin + t_chunk);
     const int lo = kt / 2;                                              // planes t-lo .. t-lo+kt-1 feed output t
 
-    for (int i = tid; i < kt * kh * KW * kCvCh; i += kCvThreads)
-        wsm[i] = __ldg(weight + static_cast<long long>(i / kCvCh) * C + c0 + (i % kCvCh));
+    // per tap: the first four channels of every 8-channel vector, then the last four, so that
+    // the 8 lanes of a quarter-warp read 128 contiguous bytes (no bank conflicts)
+    for (int i = tid; i < kt * kh * KW * kCvCh; i += kCvThreads) {
+        const int tap = i / kCvCh, ch = i % kCvCh;
+        wsm[tap * kCvCh + ((ch >> 2) & 1) * 32 + (ch >> 3) * 4 + (ch & 3)] =
+            __ldg(weight + static_cast<long long>(tap) * C + c0 + ch);
+    }
     if (tid == 0) {
         for (int i = 0; i < ring; ++i) mbar_init(smem_u32(&bars[i]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -456,12 +461,12 @@ dwconv3d_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* __re
                 const unsigned char* plane = base + static_cast<size_t>(n % ring) * plane_bytes;
                 for (int j = 0; j < kh; ++j) {
                     const unsigned char* row = plane + (static_cast<size_t>(yl + j) * pw + xg * kCvRX) * (kCvCh * 2) + cv * 16;
-                    const float* wrow = wsm + (i * kh + j) * KW * kCvCh + cv * 8;
+                    const float* wrow = wsm + (i * kh + j) * KW * kCvCh + cv * 4;
                     float wv[KW][8];
 #pragma unroll
                     for (int l = 0; l < KW; ++l) {
                         const float4 wa = *reinterpret_cast<const float4*>(wrow + l * kCvCh);
-                        const float4 wb = *reinterpret_cast<const float4*>(wrow + l * kCvCh + 4);
+                        const float4 wb = *reinterpret_cast<const float4*>(wrow + l * kCvCh + 32);
                         wv[l][0] = wa.x; wv[l][1] = wa.y; wv[l][2] = wa.z; wv[l][3] = wa.w;
                         wv[l][4] = wb.x; wv[l][5] = wb.y; wv[l][6] = wb.z; wv[l][7] = wb.w;
                     }
