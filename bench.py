@@ -533,7 +533,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="1080p_256f_bf16", choices=sorted(inputs.WORKLOADS))
-    ap.add_argument("--cpu-rows", type=int, default=8, help="grid rows of one frame the CPU baseline processes")
+    ap.add_argument("--cpu-rows", type=int, default=32, help="grid rows of one frame the CPU baseline processes")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

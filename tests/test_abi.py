@@ -113,3 +113,39 @@ def test_binding_refuses_cpu_tensors():
     lse = torch.zeros(4 * 8 * 8 * 2)
     with pytest.raises(ValueError, match="CUDA tensor"):
         binding.dsa3d_forward(z, z, z, off, 4, 8, 8, 2, 32, (3, 3, 3), z, lse, stream=0)
+
+
+def test_producer_entry_points_reject_bad_arguments_without_launching(lib):
+    """The convolution, the linear layer and the forward with the convolution term validate
+    their arguments before touching the device (fake aligned addresses, never dereferenced)."""
+    a = 4096
+    win = (ctypes.c_int * 3)(3, 3, 3)
+    lib.dsa3d_dwconv3d_forward.restype = ctypes.c_int
+    lib.dsa3d_dwconv3d_forward.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int] * 4 + \
+        [ctypes.POINTER(ctypes.c_int), ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
+    conv = lambda *args: lib.dsa3d_dwconv3d_forward(*args)
+    assert conv(None, a, None, 2, 2, 2, 8, win, a, 1, None) == 1          # null x
+    assert conv(a, a, None, 2, 2, 2, 12, win, a, 1, None) == 2            # channels not a multiple of 8
+    assert conv(a, a, None, 0, 2, 2, 8, win, a, 1, None) == 2             # empty grid
+    assert conv(a, a, None, 2, 2, 2, 8, (ctypes.c_int * 3)(3, 3, 9), a, 1, None) == 2   # kernel too wide
+    assert conv(a, a, None, 2, 2, 2, 8, win, a, 5, None) == 3             # unknown dtype
+    assert conv(a + 4, a, None, 2, 2, 2, 8, win, a, 1, None) == 4         # misaligned x
+
+    lib.dsa3d_offsets_linear_forward.restype = ctypes.c_int
+    lib.dsa3d_offsets_linear_forward.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_longlong, ctypes.c_int, ctypes.c_int,
+                                                                        ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
+    lin = lambda *args: lib.dsa3d_offsets_linear_forward(*args)
+    assert lin(a, a, None, 16, 64, 81, a, 1, None) == 1                   # bias is required
+    assert lin(a, a, a, 0, 64, 81, a, 1, None) == 2                       # no tokens
+    assert lin(a, a, a, 16, 60, 81, a, 1, None) == 2                      # channels not a multiple of 8
+    assert lin(a, a, a, 1 << 31, 64, 81, a, 1, None) == 2                 # too many tokens for the tile maps
+    assert lin(a, a, a, 16, 64, 81, a, 7, None) == 3
+    assert lin(a, a + 8, a, 16, 64, 81, a, 1, None) == 4
+
+    lib.dsa3d_forward_residual.restype = ctypes.c_int
+    lib.dsa3d_forward_residual.argtypes = [ctypes.c_void_p] * 5 + [ctypes.c_int] * 5 + \
+        [ctypes.POINTER(ctypes.c_int), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
+    res = lambda *args: lib.dsa3d_forward_residual(*args)
+    assert res(a, a, a, a, None, 4, 8, 8, 2, 32, win, a, a, 0, None) == 1  # the term itself is required
+    assert res(a, a, a, a, a + 2, 4, 8, 8, 2, 32, win, a, a, 0, None) == 4
+    assert res(a, a, a, a, a, 4, 8, 8, 2, 48, win, a, a, 0, None) == 3     # head size not supported
