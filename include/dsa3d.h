@@ -61,7 +61,10 @@ typedef enum { DSA3D_F32 = 0, DSA3D_BF16 = 1 } dsa3d_dtype;
 
 /*
  * Forward (Eq. 1 second term + softmax definition).  Reads q, k, v, offsets; writes out
- * and lse.  `window` is a HOST pointer to (kt, kh, kw).  No workspace.
+ * and lse.  `window` is a HOST pointer to (kt, kh, kw).  No workspace.  dsa3d_forward and
+ * dsa3d_backward only enqueue work on `stream` (kernels and a clear of the accumulators; no
+ * allocation, no synchronisation), so they may be recorded into a CUDA graph by stream
+ * capture and replayed.
  */
 int dsa3d_forward(const void* q, const void* k, const void* v, const float* offsets,
                   int T, int H, int W, int heads, int d, const int window[3],

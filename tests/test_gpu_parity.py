@@ -310,3 +310,40 @@ def test_nothing_is_written_outside_the_output_buffers(dtype):
 def oracle_forward(q, k, v, off, dims, win):
     import oracle
     return oracle.forward(q, k, v, off, *dims, win)
+
+
+# ------------------------------------------------------------- CUDA graph capture
+
+@pytest.mark.parametrize("dtype", [BF16, F32])
+def test_forward_and_backward_can_be_captured_in_a_cuda_graph(dtype):
+    """Small problems are launch-bound, so a caller will want the step in a CUDA graph: the
+    device entry points only enqueue work on the given stream (no allocation, no
+    synchronisation), so forward + backward capture into one graph whose replays reproduce
+    the eager results (dk/dv up to the order of their atomic sums)."""
+    q, k, v, off, dout = small_problem(4, 9, 10, 2, 64, (3, 3, 3), dtype, 1.1, 95)
+    dims = tuple(q.shape)
+    T, H, W, heads, d = dims
+    dev = [z.cuda() for z in (q, k, v, off, dout)]
+    out_e, lse_e = pu.gpu_forward(*dev[:4], dims, (3, 3, 3))
+    g_e = pu.gpu_backward(*dev[:4], lse_e, dev[4], dims, (3, 3, 3))
+    out, lse = torch.empty_like(out_e), torch.empty_like(lse_e)
+    dq, dk, dv, doff = (torch.empty_like(z) for z in g_e)
+    ws = torch.empty(max(binding.dsa3d_backward_workspace_bytes(*dims, (3, 3, 3), dtype), 16), dtype=torch.uint8,
+                     device="cuda")
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            binding.dsa3d_forward(*dev[:4], T, H, W, heads, d, (3, 3, 3), out, lse)
+            binding.dsa3d_backward(*dev[:4], lse, dev[4], T, H, W, heads, d, (3, 3, 3), dq, dk, dv, doff, ws)
+    for _ in range(2):
+        for z in (out, lse, dq, dk, dv, doff):
+            z.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, out_e) and torch.equal(lse, lse_e)
+        assert torch.equal(dq, g_e[0]) and torch.equal(doff, g_e[3])
+        for got, ref in ((dk, g_e[1]), (dv, g_e[2])):
+            ref = ref.float()
+            assert float((got.float() - ref).abs().max()) <= 2e-2 * float(ref.abs().max())
