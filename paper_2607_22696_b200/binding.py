@@ -77,6 +77,8 @@ def load():
     lib.dsa3d_device_timeout_flag.argtypes = []
     lib.dsa3d_forward_residual.restype = i
     lib.dsa3d_forward_residual.argtypes = [p, p, p, p, p, i, i, i, i, i, win, p, p, i, p]
+    lib.dsa3d_forward_fixed_window.restype = i
+    lib.dsa3d_forward_fixed_window.argtypes = [p, p, p, i, i, i, i, i, win, p, p, i, p]
     lib.dsa3d_status_string.restype = ctypes.c_char_p
     lib.dsa3d_status_string.argtypes = [i]
     lib.dsa3d_last_cuda_error.restype = i
@@ -163,6 +165,17 @@ def dsa3d_forward_residual(q, k, v, offsets, residual, T, H, W, heads, d, window
         _ptr(q, "q", n * d), _ptr(k, "k", n * d), _ptr(v, "v", n * d),
         _ptr(offsets, "offsets", n * P * 3, torch.float32), _ptr(residual, "residual", n * d), T, H, W, heads, d,
         _window(window), _ptr(out, "out", n * d), _ptr(lse, "lse", n, torch.float32), code, _stream(stream)))
+
+
+def dsa3d_forward_fixed_window(q, k, v, T, H, W, heads, d, window, out, lse, dtype=None, stream=None) -> None:
+    """out, lse <- 3D-DSA forward with all offsets zero (no offsets tensor); see include/dsa3d.h."""
+    lib = load()
+    dt = q.dtype if dtype is None else dtype
+    code = _DTYPES[dt] if isinstance(dt, torch.dtype) else int(dt)
+    n = T * H * W * heads
+    _check(lib.dsa3d_forward_fixed_window(
+        _ptr(q, "q", n * d), _ptr(k, "k", n * d), _ptr(v, "v", n * d), T, H, W, heads, d, _window(window),
+        _ptr(out, "out", n * d), _ptr(lse, "lse", n, torch.float32), code, _stream(stream)))
 
 
 def dsa3d_dwconv3d_forward(x, weight, bias, T, H, W, C, kernel, y, dtype=None, stream=None) -> None:

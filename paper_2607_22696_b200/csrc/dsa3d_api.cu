@@ -1,5 +1,6 @@
 // C ABI of the 3D-DSA library: argument validation, workspace layout, launches.
 // Declarations and the contract of every entry point are in include/dsa3d.h.
+#include <cstdlib>
 #include <stdint.h>
 #include <stdio.h>
 #include <stdlib.h>
@@ -126,6 +127,29 @@ int forward_entry(const void* q, const void* k, const void* v, const float* offs
 int dsa3d_forward(const void* q, const void* k, const void* v, const float* offsets, int T, int H, int W,
                   int heads, int d, const int window[3], void* out, float* lse, int dtype, void* stream) {
     return forward_entry(q, k, v, offsets, nullptr, T, H, W, heads, d, window, out, lse, dtype, stream);
+}
+
+int dsa3d_forward_fixed_window(const void* q, const void* k, const void* v, int T, int H, int W, int heads, int d,
+                               const int window[3], void* out, float* lse, int dtype, void* stream) {
+    if (!q || !k || !v || !out || !lse) return DSA3D_ERR_NULL_POINTER;
+    dsa3d::Problem pr;
+    const int rc = make_problem(T, H, W, heads, d, window, dtype, pr);
+    if (rc != DSA3D_OK) return rc;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(lse)) return DSA3D_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = record(0, st);
+    if (e != cudaSuccess) return cuda_failed(e);
+    bool done = false;
+    if (dtype == DSA3D_BF16 && !std::getenv("DSA3D_NO_TENSOR_FIXED_WINDOW")) {
+        done = dsa3d::try_fixed_window_forward(q, k, v, out, lse, pr, st, &e);
+        if (done && e != cudaSuccess) return cuda_failed(e);
+    }
+    if (!done) {                      // general kernel, a NULL offsets tensor reads as all zeros
+        e = dsa3d::launch_forward(q, k, v, nullptr, nullptr, out, lse, pr, dtype == DSA3D_BF16, st);
+        if (e != cudaSuccess) return cuda_failed(e);
+    }
+    e = record(1, st);
+    return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
 }
 
 int dsa3d_forward_residual(const void* q, const void* k, const void* v, const float* offsets, const void* residual,

@@ -1,0 +1,269 @@
+// Fixed-window forward (all offsets zero: the local-attention variant of the ablation on the
+// effect of offsets) as dense tile attention.  With zero offsets sample p of a query sits
+// exactly on the grid position query + b(p), so the logits of a tile of queries are entries
+// of the dense product  Q_tile . K_region^T  over the tile's halo region, and the window is a
+// mask on that score tile.
+//
+// One CTA per (tile of 4 x 4 x 8 queries, head), bf16, 128 channels:
+//   1. TMA 5-D boxes bring the tile's Q rows (128 x 128), the K rows of the region
+//      (tile + kt-1, kh-1, kw-1 halo; zero rows outside the grid, which is exactly the
+//      zero-padded key of a sample outside the grid) in the 128-byte-swizzled K-major layout,
+//      and the V rows of the region unswizzled.
+//   2. One thread issues tcgen05.mma (M = 128, N <= 192 per instruction, K = 16 x 8) into
+//      fp32 accumulators in TMEM: S[query, region position].
+//   3. Warp w owns the queries of tile plane w.  It copies the score columns of the kt region
+//      planes its queries can see from TMEM to shared memory (tcgen05.ld, one column per
+//      bank), each thread picks the P entries of its window, does the softmax in registers
+//      (dead samples keep logit 0, as in the general kernel) and leaves normalised weights
+//      in shared memory.
+//   4. All 8 warps form the output: a half-warp per query, 8 channels per lane, P rows of V
+//      read from shared memory, fp32 coefficients (no rounding of the weights).
+// Waits on mbarriers are bounded and raise the library's timeout flag.
+#include <cuda_bf16.h>
+
+#include "dsa3d_common.cuh"
+#include "dsa3d_kernels.h"
+#include "dsa3d_tcgen05.cuh"
+
+namespace dsa3d {
+namespace {
+
+constexpr int kFwTT = 4, kFwTY = 4, kFwTX = 8, kFwQ = kFwTT * kFwTY * kFwTX;   // 128 queries per tile
+constexpr int kFwD = 128;
+constexpr int kFwThreads = 256;
+constexpr int kFwMaxRows = 368;                   // region rows held per K half / V (multiple of 16)
+constexpr int kFwStageCols = 64;                  // score columns of one region plane staged per warp
+
+struct __align__(1024) FwSmem {
+    unsigned char q[2][kFwQ * 128];               // two 64-channel halves, 128-byte rows; later the score staging
+    unsigned char k[2][kFwMaxRows * 128];         // two halves; later the softmax weights
+    unsigned char v[kFwMaxRows * 256];            // full 256-byte rows
+    uint64_t bar_qk, bar_v, bar_mma;
+    uint32_t tmem_base;
+};
+
+template <int KT, int KH, int KW>
+__global__ void __launch_bounds__(kFwThreads, 1)
+fixed_window_forward_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                            const __grid_constant__ CUtensorMap map_v, __nv_bfloat16* __restrict__ out,
+                            float* __restrict__ lse, int T, int H, int W, int heads, int tiles_x, int tiles_y,
+                            int* timeout_flag) {
+    constexpr int P = KT * KH * KW;
+    constexpr int RT = kFwTT + KT - 1, RY = kFwTY + KH - 1, RX = kFwTX + KW - 1;
+    constexpr int PS = RY * RX;                                   // rows of one region plane
+    constexpr int R = RT * PS;                                    // region rows
+    constexpr int RP = (R + 15) / 16 * 16;                        // padded to the MMA's N granularity
+    constexpr int N1 = RP <= 192 ? RP : 192, N2 = RP - N1;
+    static_assert(RP <= kFwMaxRows && PS <= kFwStageCols && N2 <= 256 && P <= 32, "shape not covered");
+    static_assert((RT - 1) * PS + kFwStageCols <= 512, "staged columns must stay inside the TMEM allocation");
+
+    extern __shared__ unsigned char raw[];
+    FwSmem& s = *reinterpret_cast<FwSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int m = blockIdx.y;
+    int tile = blockIdx.x;
+    const int tx = tile % tiles_x; tile /= tiles_x;
+    const int ty = tile % tiles_y;
+    const int tt = tile / tiles_y;
+    const int t0 = tt * kFwTT, y0 = ty * kFwTY, x0 = tx * kFwTX;
+
+    if (tid == 0) {
+        mbar_init(smem_u32(&s.bar_qk), 1);
+        mbar_init(smem_u32(&s.bar_v), 1);
+        mbar_init(smem_u32(&s.bar_mma), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&s.tmem_base)), "r"(512));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = s.tmem_base;
+    bool ok = true;
+
+    // ---- 1. loads, 2. score tile
+    if (tid == 0) {
+        const int kx = x0 - KW / 2, ky = y0 - KH / 2, kt0 = t0 - KT / 2;
+        mbar_expect_tx(smem_u32(&s.bar_qk), 2u * kFwQ * 128u + 2u * R * 128u);
+        for (int h = 0; h < 2; ++h) {
+            tma_load_5d(smem_u32(s.q[h]), &map_q, smem_u32(&s.bar_qk), h * 64, m, x0, y0, t0);
+            tma_load_5d(smem_u32(s.k[h]), &map_k, smem_u32(&s.bar_qk), h * 64, m, kx, ky, kt0);
+        }
+        mbar_expect_tx(smem_u32(&s.bar_v), static_cast<uint32_t>(R) * 256u);
+        tma_load_5d(smem_u32(s.v), &map_v, smem_u32(&s.bar_v), 0, m, kx, ky, kt0);
+
+        if (mbar_wait(smem_u32(&s.bar_qk), 0)) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            constexpr uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kFwQ >> 4) << 24);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const uint64_t da = smem_desc(smem_u32(s.q[h]));
+                const uint64_t db1 = smem_desc(smem_u32(s.k[h]));
+                const uint64_t db2 = smem_desc(smem_u32(s.k[h]) + N1 * 128);       // N1 rows = a multiple of 8
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {                                   // 16 channels = 32 bytes per step
+                    umma_bf16(tmem, da + 2 * kk, db1 + 2 * kk, idesc_base | (static_cast<uint32_t>(N1 >> 3) << 17),
+                              (h | kk) ? 1u : 0u);
+                    if (N2 > 0)
+                        umma_bf16(tmem + N1, da + 2 * kk, db2 + 2 * kk,
+                                  idesc_base | (static_cast<uint32_t>(N2 >> 3) << 17), (h | kk) ? 1u : 0u);
+                }
+            }
+        } else {
+            atomicExch(timeout_flag, 5);
+        }
+        umma_commit(smem_u32(&s.bar_mma));
+    }
+
+    // ---- 3. window extraction and softmax: warps 0-3, one query per thread
+    float* stage = reinterpret_cast<float*>(s.q);                 // [64 columns][128 threads], free once the MMAs are done
+    float* wts = reinterpret_cast<float*>(s.k);                   // [128 queries][P], free once the MMAs are done
+    if (warp < 4) {
+        if (!mbar_wait(smem_u32(&s.bar_mma), 0)) {
+            if (lane == 0) atomicExch(timeout_flag, 6);
+            ok = false;
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        __syncwarp();
+        const int r = tid;                                        // query row = TMEM lane
+        const int lt = warp, ly = lane >> 3, lx = lane & 7;       // box order of the Q load: x fastest, then y, then t
+        float sc[P];
+        if (ok) {
+#pragma unroll
+            for (int u = 0; u < KT; ++u) {
+                // columns of region plane lt + u, 32 at a time, to shared memory: stage[column][thread]
+#pragma unroll
+                for (int c0 = 0; c0 < kFwStageCols; c0 += 32) {
+                    uint32_t regs[32];
+                    tmem_load_32(tmem + (static_cast<uint32_t>(warp * 32) << 16) + (lt + u) * PS + c0, regs);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) stage[(c0 + i) * kFwQ + r] = __uint_as_float(regs[i]);
+                }
+                __syncwarp();
+#pragma unroll
+                for (int vv = 0; vv < KH; ++vv)
+#pragma unroll
+                    for (int ww = 0; ww < KW; ++ww)
+                        sc[(u * KH + vv) * KW + ww] = stage[((ly + vv) * RX + lx + ww) * kFwQ + r];
+                __syncwarp();
+            }
+            const float lscale = rsqrtf(static_cast<float>(kFwD)) * kLog2e;
+            float mx = -INFINITY;
+#pragma unroll
+            for (int p = 0; p < P; ++p) { sc[p] *= lscale; mx = fmaxf(mx, sc[p]); }
+            float sum = 0.0f;
+#pragma unroll
+            for (int p = 0; p < P; ++p) { sc[p] = exp2f(sc[p] - mx); sum += sc[p]; }
+            const float inv = 1.0f / sum;
+#pragma unroll
+            for (int p = 0; p < P; ++p) wts[r * P + p] = sc[p] * inv;
+            const int t = t0 + lt, y = y0 + ly, x = x0 + lx;
+            if (t < T && y < H && x < W) {
+                const long long n = (static_cast<long long>(t) * H + y) * W + x;
+                lse[n * heads + m] = (mx + log2f(sum)) * kLn2;
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+    if (!mbar_wait(smem_u32(&s.bar_v), 0)) {
+        if (tid == 0) atomicExch(timeout_flag, 7);
+        ok = false;
+    }
+    __syncthreads();
+
+    // ---- 4. output: half-warp per query, 8 channels per lane
+    {
+        const int hw = tid >> 4, hl = tid & 15;
+        for (int qi = hw; qi < kFwQ; qi += kFwThreads / 16) {
+            const int lt = qi >> 5, ly = (qi >> 3) & 3, lx = qi & 7;
+            const int t = t0 + lt, y = y0 + ly, x = x0 + lx;
+            float acc[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
+#pragma unroll
+            for (int u = 0; u < KT; ++u)
+#pragma unroll
+                for (int vv = 0; vv < KH; ++vv)
+#pragma unroll
+                    for (int ww = 0; ww < KW; ++ww) {
+                        const int j = ((lt + u) * RY + ly + vv) * RX + lx + ww;
+                        const float c = wts[qi * P + (u * KH + vv) * KW + ww];
+                        const uint4 row = *reinterpret_cast<const uint4*>(s.v + j * 256 + hl * 16);
+                        const uint32_t w4[4] = {row.x, row.y, row.z, row.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            acc[2 * i] = fmaf(c, __uint_as_float(w4[i] << 16), acc[2 * i]);
+                            acc[2 * i + 1] = fmaf(c, __uint_as_float(w4[i] & 0xffff0000u), acc[2 * i + 1]);
+                        }
+                    }
+            if (ok && t < T && y < H && x < W) {
+                const long long n = (static_cast<long long>(t) * H + y) * W + x;
+                uint32_t o[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
+                    o[i] = *reinterpret_cast<const uint32_t*>(&h2);
+                }
+                *reinterpret_cast<uint4*>(out + (n * heads + m) * kFwD + hl * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512));
+}
+
+bool make_maps(const void* q, const void* k, const void* v, const Problem& pr, int kt, int kh, int kw, CUtensorMap* mq,
+               CUtensorMap* mk, CUtensorMap* mv) {
+    const unsigned long long d = static_cast<unsigned long long>(pr.d), hd = static_cast<unsigned long long>(pr.heads);
+    const unsigned long long dims[5] = {d, hd, static_cast<unsigned long long>(pr.W), static_cast<unsigned long long>(pr.H),
+                                        static_cast<unsigned long long>(pr.T)};
+    const unsigned long long strides[4] = {d * 2, hd * d * 2, static_cast<unsigned long long>(pr.W) * hd * d * 2,
+                                           static_cast<unsigned long long>(pr.H) * pr.W * hd * d * 2};
+    const unsigned box_q[5] = {64, 1, kFwTX, kFwTY, kFwTT};
+    const unsigned box_k[5] = {64, 1, static_cast<unsigned>(kFwTX + kw - 1), static_cast<unsigned>(kFwTY + kh - 1),
+                               static_cast<unsigned>(kFwTT + kt - 1)};
+    const unsigned box_v[5] = {128, 1, box_k[2], box_k[3], box_k[4]};
+    return encode_tensor_map_bf16(mq, q, 5, dims, strides, box_q, true) &&
+           encode_tensor_map_bf16(mk, k, 5, dims, strides, box_k, true) &&
+           encode_tensor_map_bf16(mv, v, 5, dims, strides, box_v, false);
+}
+
+template <int KT, int KH, int KW>
+cudaError_t launch(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, void* out, float* lse,
+                   const Problem& pr, int* flag, cudaStream_t stream) {
+    const int tiles_x = (pr.W + kFwTX - 1) / kFwTX, tiles_y = (pr.H + kFwTY - 1) / kFwTY,
+              tiles_t = (pr.T + kFwTT - 1) / kFwTT;
+    const size_t smem = sizeof(FwSmem) + 1024;
+    auto kern = fixed_window_forward_kernel<KT, KH, KW>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    const dim3 grid(static_cast<unsigned>(tiles_x * tiles_y * tiles_t), static_cast<unsigned>(pr.heads));
+    kern<<<grid, kFwThreads, smem, stream>>>(mq, mk, mv, static_cast<__nv_bfloat16*>(out), lse, pr.T, pr.H, pr.W, pr.heads,
+                                             tiles_x, tiles_y, flag);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool try_fixed_window_forward(const void* q, const void* k, const void* v, void* out, float* lse, const Problem& pr,
+                              cudaStream_t stream, cudaError_t* err) {
+    *err = cudaSuccess;
+    if (pr.d != kFwD || pr.heads > 65535) return false;
+    const bool w333 = pr.kt == 3 && pr.kh == 3 && pr.kw == 3, w222 = pr.kt == 2 && pr.kh == 2 && pr.kw == 2;
+    if (!w333 && !w222) return false;
+    const long long tiles = static_cast<long long>((pr.W + kFwTX - 1) / kFwTX) * ((pr.H + kFwTY - 1) / kFwTY) *
+                            ((pr.T + kFwTT - 1) / kFwTT);
+    if (tiles > 0x7fffffffLL) return false;
+    int* flag = timeout_flag_device_address();
+    CUtensorMap mq, mk, mv;
+    if (!flag || !make_maps(q, k, v, pr, pr.kt, pr.kh, pr.kw, &mq, &mk, &mv)) return false;
+    *err = w333 ? launch<3, 3, 3>(mq, mk, mv, out, lse, pr, flag, stream)
+                : launch<2, 2, 2>(mq, mk, mv, out, lse, pr, flag, stream);
+    return true;
+}
+
+}  // namespace dsa3d

@@ -17,6 +17,8 @@
 
 namespace dsa3d {
 
+__device__ const float kZeroOffset[3] = {0.0f, 0.0f, 0.0f};     // stands in for a NULL offsets tensor
+
 #ifndef DSA3D_FWD_MINBLOCKS
 #define DSA3D_FWD_MINBLOCKS 3
 #endif
@@ -65,7 +67,8 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
     for (int pb = 0; pb < pr.P; pb += LPR) {
         Sample mine;
         mine.base = 0; mine.mask = 0u; mine.ft = mine.fy = mine.fx = 0.0f;
-        if (pb + gl < pr.P) mine = to_sample(pr, make_cell(pr, t, y, x, pb + gl, off_row + (pb + gl) * 3));
+        if (pb + gl < pr.P)
+            mine = to_sample(pr, make_cell(pr, t, y, x, pb + gl, offsets ? off_row + (pb + gl) * 3 : kZeroOffset));
         const int cnt = min(LPR, pr.P - pb);
         if constexpr (LPR >= 8) {
             // Fixed-window regime: every sample of this chunk (in every group of the warp) sits

@@ -1,5 +1,6 @@
 // Internal launch interface between the C-ABI layer and the kernels.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
 
@@ -43,5 +44,21 @@ int backward_impl(const void* q, const void* k, const void* v, const float* offs
                   const void* dout, int T, int H, int W, int heads, int d, const int window[3], void* dq,
                   void* dk, void* dv, float* doffsets, void* workspace, size_t workspace_bytes, int dtype,
                   void* stream, bool tiled);
+
+// Host side of the TMA kernels (dsa3d_producer.cu).  encode_tensor_map_bf16: a tiled map over
+// a bf16 tensor of `rank` dimensions (innermost first; strides_bytes has rank-1 entries, the
+// innermost stride being 2), zero fill outside the tensor, 128-byte swizzle or none.
+bool encode_tensor_map_bf16(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
+                            const unsigned long long* strides_bytes, const unsigned* box, bool swizzle128);
+
+// Device address of the flag a tensor-core kernel raises when one of its bounded waits runs
+// out (read by dsa3d_device_timeout_flag); NULL if it cannot be looked up.
+int* timeout_flag_device_address();
+
+// Fixed-window forward on the tensor cores (dsa3d_fixed_window.cu).  Returns false when the
+// shape is not one it covers (the caller then uses the general kernel with zero offsets);
+// *err receives a launch error.
+bool try_fixed_window_forward(const void* q, const void* k, const void* v, void* out, float* lse, const Problem& pr,
+                              cudaStream_t stream, cudaError_t* err);
 
 }  // namespace dsa3d

@@ -1,0 +1,79 @@
+"""GPU parity of the fixed-window forward (all offsets zero, no offsets tensor): the
+tensor-core tile kernel for bf16 / 128 channels / windows (3,3,3) and (2,2,2), the general
+kernel with a NULL offsets tensor for everything else.  The oracle is run with an all-zero
+offsets tensor."""
+import os
+
+import pytest
+import torch
+
+import oracle
+from paper_2607_22696_b200 import binding, inputs
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+BF16, F32 = torch.bfloat16, torch.float32
+
+
+def _case(shape, window, dtype, seed, sigma_q=1.0):
+    T, H, W, heads, d = shape
+    q, k, v = (inputs.normal(shape, seed, i, sigma_q if i == 0 else 1.0, dtype) for i in range(3))
+    P = window[0] * window[1] * window[2]
+    zeros = torch.zeros(T * H * W, heads, P, 3, dtype=F32)
+    ref_out, ref_lse = oracle.forward(q.view(-1, heads, d), k, v, zeros, T, H, W, heads, d, window)
+    out = torch.full(shape, float("nan"), dtype=dtype, device="cuda")
+    lse = torch.full((T, H, W, heads), float("nan"), dtype=F32, device="cuda")
+    guard = torch.full((64,), 5.0, dtype=F32, device="cuda")
+    binding.dsa3d_forward_fixed_window(q.cuda(), k.cuda(), v.cuda(), T, H, W, heads, d, window, out, lse)
+    torch.cuda.synchronize()
+    assert binding.dsa3d_device_timeout_flag() == 0
+    pu.assert_close("out", out, ref_out.view(shape), dtype)
+    pu.assert_close("lse", lse, ref_lse.view(T, H, W, heads), dtype)
+    assert torch.equal(guard.cpu(), torch.full((64,), 5.0))
+    return q, k, v, out, lse
+
+
+@pytest.mark.parametrize("shape", [(6, 9, 13, 2, 128), (4, 4, 8, 1, 128), (1, 1, 1, 1, 128), (9, 5, 17, 3, 128),
+                                   (2, 13, 7, 2, 128)])
+@pytest.mark.parametrize("window", [(3, 3, 3), (2, 2, 2)])
+def test_tensor_core_tile_kernel_matches_the_oracle(shape, window):
+    """Grids that are not multiples of the 4 x 4 x 8 tile, a grid smaller than one tile, a
+    single token (every window cell but the centre is a dead sample with logit 0)."""
+    _case(shape, window, BF16, 140)
+
+
+def test_sharp_softmax_and_border_samples():
+    """Large logits (one key dominates) next to rows at the border whose dead samples hold
+    logit 0 in the softmax."""
+    _case((5, 6, 9, 2, 128), (3, 3, 3), BF16, 141, sigma_q=6.0)
+
+
+@pytest.mark.parametrize("shape,window,dtype", [((4, 6, 7, 2, 64), (3, 3, 3), BF16), ((3, 5, 6, 2, 32), (3, 3, 3), F32),
+                                                ((4, 6, 9, 2, 128), (3, 5, 5), BF16), ((4, 6, 9, 2, 128), (1, 3, 3), BF16)])
+def test_other_shapes_run_the_general_kernel_without_an_offsets_tensor(shape, window, dtype):
+    _case(shape, window, dtype, 142)
+
+
+def test_tile_kernel_agrees_with_the_general_kernel_on_zero_offsets():
+    """Same problem through the tile kernel, through the general kernel forced by the
+    environment switch, and through dsa3d_forward with a zero offsets tensor."""
+    shape, window = (8, 10, 20, 3, 128), (3, 3, 3)
+    T, H, W, heads, d = shape
+    q, k, v, out_tc, lse_tc = _case(shape, window, BF16, 143)
+    dq, dk, dv = q.cuda(), k.cuda(), v.cuda()
+    os.environ["DSA3D_NO_TENSOR_FIXED_WINDOW"] = "1"
+    try:
+        out_g, lse_g = torch.empty_like(out_tc), torch.empty_like(lse_tc)
+        binding.dsa3d_forward_fixed_window(dq, dk, dv, T, H, W, heads, d, window, out_g, lse_g)
+    finally:
+        del os.environ["DSA3D_NO_TENSOR_FIXED_WINDOW"]
+    zeros = torch.zeros(T, H, W, heads, 27, 3, dtype=F32, device="cuda")
+    out_z, lse_z = torch.empty_like(out_tc), torch.empty_like(lse_tc)
+    binding.dsa3d_forward(dq, dk, dv, zeros, T, H, W, heads, d, window, out_z, lse_z)
+    torch.cuda.synchronize()
+    assert torch.equal(out_g, out_z) and torch.equal(lse_g, lse_z)          # same kernel, same arithmetic
+    assert float((lse_tc - lse_z).abs().max()) <= 1e-4
+    ulp = (out_z.float().abs() * 2.0 ** -7).clamp_min(1e-3)
+    assert bool(((out_tc.float() - out_z.float()).abs() <= ulp).all())      # within one bf16 step of each other
