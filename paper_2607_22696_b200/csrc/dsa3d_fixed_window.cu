@@ -16,8 +16,9 @@
 //      bank), each thread picks the P entries of its window, does the softmax in registers
 //      (dead samples keep logit 0, as in the general kernel) and leaves normalised weights
 //      in shared memory.
-//   4. All 8 warps form the output: a half-warp per query, 8 channels per lane, P rows of V
-//      read from shared memory, fp32 coefficients (no rounding of the weights).
+//   4. All 8 warps form the output: a half-warp per x-row of 8 queries, 8 channels per lane;
+//      each V row of the x-row's reach is read from shared memory and widened once and added
+//      into every query whose window holds it, with fp32 weights (no rounding of the weights).
 // Waits on mbarriers are bounded and raise the library's timeout flag.
 #include <cuda_bf16.h>
 
@@ -158,8 +159,12 @@ fixed_window_forward_kernel(const __grid_constant__ CUtensorMap map_q, const __g
 #pragma unroll
             for (int p = 0; p < P; ++p) { sc[p] = exp2f(sc[p] - mx); sum += sc[p]; }
             const float inv = 1.0f / sum;
+            // weights of an x-row of 8 queries together: [row of the tile][u, v][lx][w]
+            float* wrow = wts + (warp * kFwTY + ly) * (KT * KH * kFwTX * KW) + lx * KW;
 #pragma unroll
-            for (int p = 0; p < P; ++p) wts[r * P + p] = sc[p] * inv;
+            for (int uv = 0; uv < KT * KH; ++uv)
+#pragma unroll
+                for (int ww = 0; ww < KW; ++ww) wrow[uv * (kFwTX * KW) + ww] = sc[uv * KW + ww] * inv;
             const int t = t0 + lt, y = y0 + ly, x = x0 + lx;
             if (t < T && y < H && x < W) {
                 const long long n = (static_cast<long long>(t) * H + y) * W + x;
@@ -174,37 +179,56 @@ fixed_window_forward_kernel(const __grid_constant__ CUtensorMap map_q, const __g
     }
     __syncthreads();
 
-    // ---- 4. output: half-warp per query, 8 channels per lane
+    // ---- 4. output: a half-warp per x-row of 8 queries, 8 channels per lane.  Neighbouring
+    //         queries share most of their window, so each V row of the x-row's reach is read
+    //         and widened once and added into every query whose window holds it.
     {
-        const int hw = tid >> 4, hl = tid & 15;
-        for (int qi = hw; qi < kFwQ; qi += kFwThreads / 16) {
-            const int lt = qi >> 5, ly = (qi >> 3) & 3, lx = qi & 7;
-            const int t = t0 + lt, y = y0 + ly, x = x0 + lx;
-            float acc[8];
+        const int hw = tid >> 4, hl = tid & 15;                   // 16 half-warps = the 4 x 4 x-rows of the tile
+        const int lt = hw >> 2, ly = hw & 3;
+        float acc[kFwTX][8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
+        for (int qx = 0; qx < kFwTX; ++qx)
 #pragma unroll
-            for (int u = 0; u < KT; ++u)
+            for (int e = 0; e < 8; ++e) acc[qx][e] = 0.0f;
+        const float* wrow = wts + hw * (KT * KH * kFwTX * KW);
+#pragma unroll 1
+        for (int uv = 0; uv < KT * KH; ++uv) {
+            const int u = uv / KH, vv = uv - u * KH;
+            float wq[kFwTX * KW];                                 // the 8 queries' KW weights of this kernel row
 #pragma unroll
-                for (int vv = 0; vv < KH; ++vv)
+            for (int i = 0; i < kFwTX * KW; i += 4) {
+                const float4 w4 = *reinterpret_cast<const float4*>(wrow + uv * (kFwTX * KW) + i);
+                wq[i] = w4.x; wq[i + 1] = w4.y; wq[i + 2] = w4.z; wq[i + 3] = w4.w;
+            }
+            const unsigned char* vrow = s.v + (((lt + u) * RY + ly + vv) * RX) * 256 + hl * 16;
 #pragma unroll
-                    for (int ww = 0; ww < KW; ++ww) {
-                        const int j = ((lt + u) * RY + ly + vv) * RX + lx + ww;
-                        const float c = wts[qi * P + (u * KH + vv) * KW + ww];
-                        const uint4 row = *reinterpret_cast<const uint4*>(s.v + j * 256 + hl * 16);
-                        const uint32_t w4[4] = {row.x, row.y, row.z, row.w};
+            for (int xx = 0; xx < RX; ++xx) {
+                const uint4 row = *reinterpret_cast<const uint4*>(vrow + xx * 256);
+                float f[8];
+                f[0] = __uint_as_float(row.x << 16); f[1] = __uint_as_float(row.x & 0xffff0000u);
+                f[2] = __uint_as_float(row.y << 16); f[3] = __uint_as_float(row.y & 0xffff0000u);
+                f[4] = __uint_as_float(row.z << 16); f[5] = __uint_as_float(row.z & 0xffff0000u);
+                f[6] = __uint_as_float(row.w << 16); f[7] = __uint_as_float(row.w & 0xffff0000u);
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            acc[2 * i] = fmaf(c, __uint_as_float(w4[i] << 16), acc[2 * i]);
-                            acc[2 * i + 1] = fmaf(c, __uint_as_float(w4[i] & 0xffff0000u), acc[2 * i + 1]);
-                        }
-                    }
-            if (ok && t < T && y < H && x < W) {
+                for (int ww = 0; ww < KW; ++ww) {
+                    const int qx = xx - ww;                       // the query whose window cell ww is position xx
+                    if (qx < 0 || qx >= kFwTX) continue;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[qx][e] = fmaf(wq[qx * KW + ww], f[e], acc[qx][e]);
+                }
+            }
+        }
+        const int t = t0 + lt, y = y0 + ly;
+        if (ok && t < T && y < H) {
+#pragma unroll
+            for (int qx = 0; qx < kFwTX; ++qx) {
+                const int x = x0 + qx;
+                if (x >= W) continue;
                 const long long n = (static_cast<long long>(t) * H + y) * W + x;
                 uint32_t o[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
+                    const __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[qx][2 * i], acc[qx][2 * i + 1]);
                     o[i] = *reinterpret_cast<const uint32_t*>(&h2);
                 }
                 *reinterpret_cast<uint4*>(out + (n * heads + m) * kFwD + hl * 8) = make_uint4(o[0], o[1], o[2], o[3]);
