@@ -33,14 +33,14 @@ constexpr int kFwTT = 4, kFwTY = 4, kFwTX = 8, kFwQ = kFwTT * kFwTY * kFwTX;   /
 constexpr int kFwD = 128;
 constexpr int kFwThreads = 256;
 constexpr int kFwMaxRows = 368;                   // region rows held per K half / V (multiple of 16)
-constexpr int kFwStageCols = 64;                  // score columns of one region plane staged per warp
 
 struct __align__(1024) FwSmem {
-    unsigned char q[2][kFwQ * 128];               // two 64-channel halves, 128-byte rows; later the score staging
-    unsigned char k[2][kFwMaxRows * 128];         // two halves; later the softmax weights
+    unsigned char q[2][kFwQ * 128];               // two 64-channel halves, 128-byte rows; later score staging + weights
+    unsigned char k[2][kFwMaxRows * 128];         // two 64-channel halves
     unsigned char v[kFwMaxRows * 256];            // full 256-byte rows
-    uint64_t bar_qk, bar_v, bar_mma;
+    uint64_t bar_q, bar_k, bar_v, bar_mma;
     uint32_t tmem_base;
+    uint32_t abort;                               // set by the issuing thread when one of its waits ran out
 };
 
 template <int KT, int KH, int KW>
@@ -48,30 +48,28 @@ __global__ void __launch_bounds__(kFwThreads, 1)
 fixed_window_forward_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                             const __grid_constant__ CUtensorMap map_v, __nv_bfloat16* __restrict__ out,
                             float* __restrict__ lse, int T, int H, int W, int heads, int tiles_x, int tiles_y,
-                            int* timeout_flag) {
+                            long long total, int* timeout_flag) {
     constexpr int P = KT * KH * KW;
     constexpr int RT = kFwTT + KT - 1, RY = kFwTY + KH - 1, RX = kFwTX + KW - 1;
     constexpr int PS = RY * RX;                                   // rows of one region plane
     constexpr int R = RT * PS;                                    // region rows
     constexpr int RP = (R + 15) / 16 * 16;                        // padded to the MMA's N granularity
     constexpr int N1 = RP <= 192 ? RP : 192, N2 = RP - N1;
-    static_assert(RP <= kFwMaxRows && PS <= kFwStageCols && N2 <= 256 && P <= 32, "shape not covered");
-    static_assert((RT - 1) * PS + kFwStageCols <= 512, "staged columns must stay inside the TMEM allocation");
+    constexpr int kChunks = (PS + 31) / 32;                       // 32-column pieces of a region plane
+    static_assert(RP <= kFwMaxRows && N2 <= 256 && P <= 32, "shape not covered");
+    static_assert((RT - 1) * PS + kChunks * 32 <= 512, "staged columns must stay inside the TMEM allocation");
+    static_assert(16 * KT * KH * kFwTX * KW * 4 <= 16 * 1024, "the weights must fit the upper half of the Q buffer");
 
     extern __shared__ unsigned char raw[];
     FwSmem& s = *reinterpret_cast<FwSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int m = blockIdx.y;
-    int tile = blockIdx.x;
-    const int tx = tile % tiles_x; tile /= tiles_x;
-    const int ty = tile % tiles_y;
-    const int tt = tile / tiles_y;
-    const int t0 = tt * kFwTT, y0 = ty * kFwTY, x0 = tx * kFwTX;
 
     if (tid == 0) {
-        mbar_init(smem_u32(&s.bar_qk), 1);
+        mbar_init(smem_u32(&s.bar_q), 1);
+        mbar_init(smem_u32(&s.bar_k), 1);
         mbar_init(smem_u32(&s.bar_v), 1);
         mbar_init(smem_u32(&s.bar_mma), 1);
+        s.abort = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -85,155 +83,207 @@ fixed_window_forward_kernel(const __grid_constant__ CUtensorMap map_q, const __g
     const uint32_t tmem = s.tmem_base;
     bool ok = true;
 
-    // ---- 1. loads, 2. score tile
-    if (tid == 0) {
-        const int kx = x0 - KW / 2, ky = y0 - KH / 2, kt0 = t0 - KT / 2;
-        mbar_expect_tx(smem_u32(&s.bar_qk), 2u * kFwQ * 128u + 2u * R * 128u);
-        for (int h = 0; h < 2; ++h) {
-            tma_load_5d(smem_u32(s.q[h]), &map_q, smem_u32(&s.bar_qk), h * 64, m, x0, y0, t0);
-            tma_load_5d(smem_u32(s.k[h]), &map_k, smem_u32(&s.bar_qk), h * 64, m, kx, ky, kt0);
-        }
+    // Work item -> (head, tile origin); tiles of one head are neighbours in the launch order.
+    const long long tiles_per_head = total / heads;
+    auto locate = [&](long long item, int& m, int& t0, int& y0, int& x0) {
+        m = static_cast<int>(item / tiles_per_head);
+        int tile = static_cast<int>(item - m * tiles_per_head);
+        x0 = (tile % tiles_x) * kFwTX; tile /= tiles_x;
+        y0 = (tile % tiles_y) * kFwTY;
+        t0 = (tile / tiles_y) * kFwTT;
+    };
+    auto load_q = [&](int m, int t0, int y0, int x0) {
+        mbar_expect_tx(smem_u32(&s.bar_q), 2u * kFwQ * 128u);
+        for (int h = 0; h < 2; ++h) tma_load_5d(smem_u32(s.q[h]), &map_q, smem_u32(&s.bar_q), h * 64, m, x0, y0, t0);
+    };
+    auto load_k = [&](int m, int t0, int y0, int x0) {
+        mbar_expect_tx(smem_u32(&s.bar_k), 2u * R * 128u);
+        for (int h = 0; h < 2; ++h)
+            tma_load_5d(smem_u32(s.k[h]), &map_k, smem_u32(&s.bar_k), h * 64, m, x0 - KW / 2, y0 - KH / 2, t0 - KT / 2);
+    };
+    auto load_v = [&](int m, int t0, int y0, int x0) {
         mbar_expect_tx(smem_u32(&s.bar_v), static_cast<uint32_t>(R) * 256u);
-        tma_load_5d(smem_u32(s.v), &map_v, smem_u32(&s.bar_v), 0, m, kx, ky, kt0);
+        tma_load_5d(smem_u32(s.v), &map_v, smem_u32(&s.bar_v), 0, m, x0 - KW / 2, y0 - KH / 2, t0 - KT / 2);
+    };
 
-        if (mbar_wait(smem_u32(&s.bar_qk), 0)) {
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            constexpr uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kFwQ >> 4) << 24);
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const uint64_t da = smem_desc(smem_u32(s.q[h]));
-                const uint64_t db1 = smem_desc(smem_u32(s.k[h]));
-                const uint64_t db2 = smem_desc(smem_u32(s.k[h]) + N1 * 128);       // N1 rows = a multiple of 8
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {                                   // 16 channels = 32 bytes per step
-                    umma_bf16(tmem, da + 2 * kk, db1 + 2 * kk, idesc_base | (static_cast<uint32_t>(N1 >> 3) << 17),
-                              (h | kk) ? 1u : 0u);
-                    if (N2 > 0)
-                        umma_bf16(tmem + N1, da + 2 * kk, db2 + 2 * kk,
-                                  idesc_base | (static_cast<uint32_t>(N2 >> 3) << 17), (h | kk) ? 1u : 0u);
-                }
-            }
-        } else {
-            atomicExch(timeout_flag, 5);
-        }
-        umma_commit(smem_u32(&s.bar_mma));
+    float* stage = reinterpret_cast<float*>(s.q[0]);              // [32 columns][128 threads]: lower half of the Q buffer
+    float* wts = reinterpret_cast<float*>(s.q[1]);                // softmax weights: upper half of the Q buffer
+
+    if (tid == 0 && static_cast<long long>(blockIdx.x) < total) {
+        int m, t0, y0, x0;
+        locate(blockIdx.x, m, t0, y0, x0);
+        load_q(m, t0, y0, x0);
+        load_k(m, t0, y0, x0);
+        load_v(m, t0, y0, x0);
     }
 
-    // ---- 3. window extraction and softmax: warps 0-3, one query per thread
-    float* stage = reinterpret_cast<float*>(s.q);                 // [64 columns][128 threads], free once the MMAs are done
-    float* wts = reinterpret_cast<float*>(s.k);                   // [128 queries][P], free once the MMAs are done
-    if (warp < 4) {
-        if (!mbar_wait(smem_u32(&s.bar_mma), 0)) {
-            if (lane == 0) atomicExch(timeout_flag, 6);
+    uint32_t parity = 0;
+    for (long long item = blockIdx.x; item < total && ok; item += gridDim.x, parity ^= 1u) {
+        int m, t0, y0, x0;
+        locate(item, m, t0, y0, x0);
+        const long long next = item + gridDim.x;
+
+        // ---- 2. score tile, then the next tile's K into the buffer the MMAs have finished with
+        if (tid == 0) {
+            if (mbar_wait(smem_u32(&s.bar_q), parity) && mbar_wait(smem_u32(&s.bar_k), parity)) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                constexpr uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kFwQ >> 4) << 24);
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint64_t da = smem_desc(smem_u32(s.q[h]));
+                    const uint64_t db1 = smem_desc(smem_u32(s.k[h]));
+                    const uint64_t db2 = smem_desc(smem_u32(s.k[h]) + N1 * 128);       // N1 rows = a multiple of 8
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {                                   // 16 channels = 32 bytes per step
+                        umma_bf16(tmem, da + 2 * kk, db1 + 2 * kk, idesc_base | (static_cast<uint32_t>(N1 >> 3) << 17),
+                                  (h | kk) ? 1u : 0u);
+                        if (N2 > 0)
+                            umma_bf16(tmem + N1, da + 2 * kk, db2 + 2 * kk,
+                                      idesc_base | (static_cast<uint32_t>(N2 >> 3) << 17), (h | kk) ? 1u : 0u);
+                    }
+                }
+            } else {
+                atomicExch(timeout_flag, 5);
+                *reinterpret_cast<volatile uint32_t*>(&s.abort) = 1u;
+            }
+            umma_commit(smem_u32(&s.bar_mma));
+            if (next < total && mbar_wait(smem_u32(&s.bar_mma), parity)) {
+                int m2, t2, y2, x2;
+                locate(next, m2, t2, y2, x2);
+                load_k(m2, t2, y2, x2);
+            }
+        }
+
+        // ---- 3. window extraction and softmax: warps 0-3, one query per thread
+        if (warp < 4) {
+            if (!mbar_wait(smem_u32(&s.bar_mma), parity)) {
+                if (lane == 0) atomicExch(timeout_flag, 6);
+                ok = false;
+            }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            __syncwarp();
+            const int r = tid;                                    // query row = TMEM lane
+            const int lt = warp, ly = lane >> 3, lx = lane & 7;   // box order of the Q load: x fastest, then y, then t
+            float sc[P];
+            if (ok) {
+#pragma unroll
+                for (int u = 0; u < KT; ++u) {
+                    // columns of region plane lt + u, 32 at a time, through shared memory:
+                    // stage[column][thread], one bank per thread
+#pragma unroll
+                    for (int ch = 0; ch < kChunks; ++ch) {
+                        uint32_t regs[32];
+                        tmem_load_32(tmem + (static_cast<uint32_t>(warp * 32) << 16) + (lt + u) * PS + ch * 32, regs);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) stage[i * kFwQ + r] = __uint_as_float(regs[i]);
+                        __syncwarp();
+#pragma unroll
+                        for (int vv = 0; vv < KH; ++vv)
+#pragma unroll
+                            for (int ww = 0; ww < KW; ++ww) {
+                                const int idx = (ly + vv) * RX + lx + ww - ch * 32;
+                                if (idx >= 0 && idx < 32) sc[(u * KH + vv) * KW + ww] = stage[idx * kFwQ + r];
+                            }
+                        __syncwarp();
+                    }
+                }
+                const float lscale = rsqrtf(static_cast<float>(kFwD)) * kLog2e;
+                float mx = -INFINITY;
+#pragma unroll
+                for (int p = 0; p < P; ++p) { sc[p] *= lscale; mx = fmaxf(mx, sc[p]); }
+                float sum = 0.0f;
+#pragma unroll
+                for (int p = 0; p < P; ++p) { sc[p] = exp2f(sc[p] - mx); sum += sc[p]; }
+                const float inv = 1.0f / sum;
+                // weights of an x-row of 8 queries together: [row of the tile][u, v][lx][w]
+                float* wrow = wts + (warp * kFwTY + ly) * (KT * KH * kFwTX * KW) + lx * KW;
+#pragma unroll
+                for (int uv = 0; uv < KT * KH; ++uv)
+#pragma unroll
+                    for (int ww = 0; ww < KW; ++ww) wrow[uv * (kFwTX * KW) + ww] = sc[uv * KW + ww] * inv;
+                const int t = t0 + lt, y = y0 + ly, x = x0 + lx;
+                if (t < T && y < H && x < W) {
+                    const long long n = (static_cast<long long>(t) * H + y) * W + x;
+                    lse[n * heads + m] = (mx + log2f(sum)) * kLn2;
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        }
+        if (!mbar_wait(smem_u32(&s.bar_v), parity)) {
+            if (tid == 0) atomicExch(timeout_flag, 7);
             ok = false;
         }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        __syncwarp();
-        const int r = tid;                                        // query row = TMEM lane
-        const int lt = warp, ly = lane >> 3, lx = lane & 7;       // box order of the Q load: x fastest, then y, then t
-        float sc[P];
-        if (ok) {
-#pragma unroll
-            for (int u = 0; u < KT; ++u) {
-                // columns of region plane lt + u, 32 at a time, to shared memory: stage[column][thread]
-#pragma unroll
-                for (int c0 = 0; c0 < kFwStageCols; c0 += 32) {
-                    uint32_t regs[32];
-                    tmem_load_32(tmem + (static_cast<uint32_t>(warp * 32) << 16) + (lt + u) * PS + c0, regs);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) stage[(c0 + i) * kFwQ + r] = __uint_as_float(regs[i]);
-                }
-                __syncwarp();
-#pragma unroll
-                for (int vv = 0; vv < KH; ++vv)
-#pragma unroll
-                    for (int ww = 0; ww < KW; ++ww)
-                        sc[(u * KH + vv) * KW + ww] = stage[((ly + vv) * RX + lx + ww) * kFwQ + r];
-                __syncwarp();
-            }
-            const float lscale = rsqrtf(static_cast<float>(kFwD)) * kLog2e;
-            float mx = -INFINITY;
-#pragma unroll
-            for (int p = 0; p < P; ++p) { sc[p] *= lscale; mx = fmaxf(mx, sc[p]); }
-            float sum = 0.0f;
-#pragma unroll
-            for (int p = 0; p < P; ++p) { sc[p] = exp2f(sc[p] - mx); sum += sc[p]; }
-            const float inv = 1.0f / sum;
-            // weights of an x-row of 8 queries together: [row of the tile][u, v][lx][w]
-            float* wrow = wts + (warp * kFwTY + ly) * (KT * KH * kFwTX * KW) + lx * KW;
-#pragma unroll
-            for (int uv = 0; uv < KT * KH; ++uv)
-#pragma unroll
-                for (int ww = 0; ww < KW; ++ww) wrow[uv * (kFwTX * KW) + ww] = sc[uv * KW + ww] * inv;
-            const int t = t0 + lt, y = y0 + ly, x = x0 + lx;
-            if (t < T && y < H && x < W) {
-                const long long n = (static_cast<long long>(t) * H + y) * W + x;
-                lse[n * heads + m] = (mx + log2f(sum)) * kLn2;
-            }
-        }
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    }
-    if (!mbar_wait(smem_u32(&s.bar_v), 0)) {
-        if (tid == 0) atomicExch(timeout_flag, 7);
-        ok = false;
-    }
-    __syncthreads();
+        if (*reinterpret_cast<volatile uint32_t*>(&s.abort)) ok = false;
+        ok = __syncthreads_and(ok);       // every thread takes the same decision to go on or to stop
 
-    // ---- 4. output: a half-warp per x-row of 8 queries, 8 channels per lane.  Neighbouring
-    //         queries share most of their window, so each V row of the x-row's reach is read
-    //         and widened once and added into every query whose window holds it.
-    {
-        const int hw = tid >> 4, hl = tid & 15;                   // 16 half-warps = the 4 x 4 x-rows of the tile
-        const int lt = hw >> 2, ly = hw & 3;
-        float acc[kFwTX][8];
+        // ---- 4. output: a half-warp per x-row of 8 queries, 8 channels per lane.  Neighbouring
+        //         queries share most of their window, so each V row of the x-row's reach is read
+        //         and widened once and added into every query whose window holds it.
+        {
+            const int hw = tid >> 4, hl = tid & 15;               // 16 half-warps = the 4 x 4 x-rows of the tile
+            const int lt = hw >> 2, ly = hw & 3;
+            float acc[kFwTX][8];
 #pragma unroll
-        for (int qx = 0; qx < kFwTX; ++qx)
+            for (int qx = 0; qx < kFwTX; ++qx)
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[qx][e] = 0.0f;
-        const float* wrow = wts + hw * (KT * KH * kFwTX * KW);
+                for (int e = 0; e < 8; ++e) acc[qx][e] = 0.0f;
+            const float* wrow = wts + hw * (KT * KH * kFwTX * KW);
 #pragma unroll 1
-        for (int uv = 0; uv < KT * KH; ++uv) {
-            const int u = uv / KH, vv = uv - u * KH;
-            float wq[kFwTX * KW];                                 // the 8 queries' KW weights of this kernel row
+            for (int uv = 0; uv < KT * KH; ++uv) {
+                const int u = uv / KH, vv = uv - u * KH;
+                float wq[kFwTX * KW];                             // the 8 queries' KW weights of this kernel row
 #pragma unroll
-            for (int i = 0; i < kFwTX * KW; i += 4) {
-                const float4 w4 = *reinterpret_cast<const float4*>(wrow + uv * (kFwTX * KW) + i);
-                wq[i] = w4.x; wq[i + 1] = w4.y; wq[i + 2] = w4.z; wq[i + 3] = w4.w;
+                for (int i = 0; i < kFwTX * KW; i += 4) {
+                    const float4 w4 = *reinterpret_cast<const float4*>(wrow + uv * (kFwTX * KW) + i);
+                    wq[i] = w4.x; wq[i + 1] = w4.y; wq[i + 2] = w4.z; wq[i + 3] = w4.w;
+                }
+                const unsigned char* vrow = s.v + (((lt + u) * RY + ly + vv) * RX) * 256 + hl * 16;
+#pragma unroll
+                for (int xx = 0; xx < RX; ++xx) {
+                    const uint4 row = *reinterpret_cast<const uint4*>(vrow + xx * 256);
+                    float f[8];
+                    f[0] = __uint_as_float(row.x << 16); f[1] = __uint_as_float(row.x & 0xffff0000u);
+                    f[2] = __uint_as_float(row.y << 16); f[3] = __uint_as_float(row.y & 0xffff0000u);
+                    f[4] = __uint_as_float(row.z << 16); f[5] = __uint_as_float(row.z & 0xffff0000u);
+                    f[6] = __uint_as_float(row.w << 16); f[7] = __uint_as_float(row.w & 0xffff0000u);
+#pragma unroll
+                    for (int ww = 0; ww < KW; ++ww) {
+                        const int qx = xx - ww;                   // the query whose window cell ww is position xx
+                        if (qx < 0 || qx >= kFwTX) continue;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[qx][e] = fmaf(wq[qx * KW + ww], f[e], acc[qx][e]);
+                    }
+                }
             }
-            const unsigned char* vrow = s.v + (((lt + u) * RY + ly + vv) * RX) * 256 + hl * 16;
+            const int t = t0 + lt, y = y0 + ly;
+            if (ok && t < T && y < H) {
 #pragma unroll
-            for (int xx = 0; xx < RX; ++xx) {
-                const uint4 row = *reinterpret_cast<const uint4*>(vrow + xx * 256);
-                float f[8];
-                f[0] = __uint_as_float(row.x << 16); f[1] = __uint_as_float(row.x & 0xffff0000u);
-                f[2] = __uint_as_float(row.y << 16); f[3] = __uint_as_float(row.y & 0xffff0000u);
-                f[4] = __uint_as_float(row.z << 16); f[5] = __uint_as_float(row.z & 0xffff0000u);
-                f[6] = __uint_as_float(row.w << 16); f[7] = __uint_as_float(row.w & 0xffff0000u);
+                for (int qx = 0; qx < kFwTX; ++qx) {
+                    const int x = x0 + qx;
+                    if (x >= W) continue;
+                    const long long n = (static_cast<long long>(t) * H + y) * W + x;
+                    uint32_t o[4];
 #pragma unroll
-                for (int ww = 0; ww < KW; ++ww) {
-                    const int qx = xx - ww;                       // the query whose window cell ww is position xx
-                    if (qx < 0 || qx >= kFwTX) continue;
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) acc[qx][e] = fmaf(wq[qx * KW + ww], f[e], acc[qx][e]);
+                    for (int i = 0; i < 4; ++i) {
+                        const __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[qx][2 * i], acc[qx][2 * i + 1]);
+                        o[i] = *reinterpret_cast<const uint32_t*>(&h2);
+                    }
+                    *reinterpret_cast<uint4*>(out + (n * heads + m) * kFwD + hl * 8) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
             }
         }
-        const int t = t0 + lt, y = y0 + ly;
-        if (ok && t < T && y < H) {
-#pragma unroll
-            for (int qx = 0; qx < kFwTX; ++qx) {
-                const int x = x0 + qx;
-                if (x >= W) continue;
-                const long long n = (static_cast<long long>(t) * H + y) * W + x;
-                uint32_t o[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[qx][2 * i], acc[qx][2 * i + 1]);
-                    o[i] = *reinterpret_cast<const uint32_t*>(&h2);
-                }
-                *reinterpret_cast<uint4*>(out + (n * heads + m) * kFwD + hl * 8) = make_uint4(o[0], o[1], o[2], o[3]);
-            }
+        __syncthreads();              // the weights (Q buffer) and V have been read: refill both
+        if (tid == 0 && next < total) {
+            int m2, t2, y2, x2;
+            locate(next, m2, t2, y2, x2);
+            load_q(m2, t2, y2, x2);
+            load_v(m2, t2, y2, x2);
         }
+    }
+    if (!ok && tid == 0) {            // stopped early: give loads still in flight a bounded time to land
+        mbar_wait(smem_u32(&s.bar_k), parity);
+        mbar_wait(smem_u32(&s.bar_q), parity);
+        mbar_wait(smem_u32(&s.bar_v), parity);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -265,9 +315,15 @@ cudaError_t launch(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorM
     auto kern = fixed_window_forward_kernel<KT, KH, KW>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
-    const dim3 grid(static_cast<unsigned>(tiles_x * tiles_y * tiles_t), static_cast<unsigned>(pr.heads));
+    const long long total = static_cast<long long>(tiles_x) * tiles_y * tiles_t * pr.heads;
+    int dev = 0, sms = 0;
+    e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    const unsigned grid = static_cast<unsigned>(total < sms ? total : sms);     // persistent: one CTA per SM
     kern<<<grid, kFwThreads, smem, stream>>>(mq, mk, mv, static_cast<__nv_bfloat16*>(out), lse, pr.T, pr.H, pr.W, pr.heads,
-                                             tiles_x, tiles_y, flag);
+                                             tiles_x, tiles_y, total, flag);
     return cudaGetLastError();
 }
 
