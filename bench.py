@@ -335,7 +335,10 @@ def run_ours(args, wl):
             binding.dsa3d_forward_fixed_window(t["q"], t["k"], t["v"], *dims, wl.window, b["out"], b["lse"])
         else:
             binding.dsa3d_forward(t["q"], t["k"], t["v"], t["offsets"], *dims, wl.window, b["out"], b["lse"])
-        if wl.backward:
+        if wl.backward and fixed_window:
+            binding.dsa3d_backward_fixed_window(t["q"], t["k"], t["v"], b["lse"], t["dout"], *dims, wl.window,
+                                                b["dq"], b["dk"], b["dv"], b["doff"], b["ws"])
+        elif wl.backward:
             binding.dsa3d_backward(t["q"], t["k"], t["v"], t["offsets"], b["lse"], t["dout"], *dims,
                                    wl.window, b["dq"], b["dk"], b["dv"], b["doff"], b["ws"])
 
@@ -365,7 +368,8 @@ def run_ours(args, wl):
     step_ms = ev[0][0].elapsed_time(ev[K - 1][1]) / K
     fwd_ms = sum(ev[i][2].elapsed_time(ev[i][3]) for i in range(K)) / K
     bwd_ms = sum(ev[i][4].elapsed_time(ev[i][5]) for i in range(K)) / K if wl.backward else 0.0
-    tiled = wl.backward and wl.dtype == torch.bfloat16 and os.environ.get("DSA3D_TILE", "") != "0"
+    tiled = (wl.backward and wl.dtype == torch.bfloat16 and os.environ.get("DSA3D_TILE", "") != "0"
+             and not fixed_window)
     sct_ms = sum(ev[i][6].elapsed_time(ev[i][7]) for i in range(K)) / K if tiled else 0.0
     step_ms = max_ranks(step_ms)
     fwd_ms, bwd_ms, sct_ms = max_ranks(fwd_ms), max_ranks(bwd_ms), max_ranks(sct_ms)
@@ -396,14 +400,17 @@ def run_ours(args, wl):
     # The backward's algorithmic bytes belong to its two kernels together (gather: dQ,
     # dOffsets; tile scatter: dK, dV), so they are set against the sum of the two durations.
     bwd_pair_ms = bwd_ms + sct_ms
-    bwd_gbs = wl.bwd_bytes() / (bwd_pair_ms * 1e-3) / 1e9 if wl.backward else None
+    bwd_bytes = wl.bwd_bytes() - (wl.N * wl.heads * 12 * wl.P if fixed_window else 0)
+    bwd_gbs = bwd_bytes / (bwd_pair_ms * 1e-3) / 1e9 if wl.backward else None
     dominant_bwd = wl.backward and bwd_pair_ms >= fwd_ms
-    dom = {"kernel": ("backward_kernel + scatter_tile_kernel" if tiled else "backward_kernel")
+    dom = {"kernel": ("backward_kernel + scatter_tile_kernel" if tiled else
+                      "fixed_window_backward_query_kernel + fixed_window_backward_key_kernel" if fixed_window
+                      else "backward_kernel")
                      if dominant_bwd else ("fixed_window_forward_kernel" if fixed_window else "forward_kernel"),
            "achieved": bwd_gbs if dominant_bwd else fwd_gbs,
            "ms": bwd_pair_ms if dominant_bwd else fwd_ms,
-           "bytes": wl.bwd_bytes() if dominant_bwd else fwd_bytes}
-    step_bytes = fwd_bytes + (wl.bwd_bytes() if wl.backward else 0)
+           "bytes": bwd_bytes if dominant_bwd else fwd_bytes}
+    step_bytes = fwd_bytes + (bwd_bytes if wl.backward else 0)
     # Fractions of the ceilings that actually bind (the path is on-chip bound, not HBM bound)
     ceil = measure_ceilings(dev)
     items_all = wl.N * wl.heads
@@ -422,7 +429,7 @@ def run_ours(args, wl):
                 red_gbs = items_all * NCU_RED_BYTES_PER_ITEM["scatter_tile_kernel"] / (sct_ms * 1e-3) / 1e9
                 onchip["scatter_tile_kernel"].update(red_gbs=red_gbs, red_frac=red_gbs / ceil["l2_red_v4_f32_gbs"])
     traffic = None
-    if wl.dtype == torch.bfloat16 and wl.d == 128 and wl.P == 27:
+    if wl.dtype == torch.bfloat16 and wl.d == 128 and wl.P == 27 and not fixed_window:
         items = wl.N * wl.heads
         per_item = (NCU_DRAM_BYTES_PER_ITEM["backward_kernel"] + (NCU_DRAM_BYTES_PER_ITEM["scatter_tile_kernel"]
                     if tiled else 0.0)) if dominant_bwd else NCU_DRAM_BYTES_PER_ITEM["forward_kernel"]
@@ -435,6 +442,8 @@ def run_ours(args, wl):
                    "d": wl.d, "window": list(wl.window), "storage": str(wl.dtype).replace("torch.", ""),
                    "offsets": f"{wl.offsets} sigma={wl.sigma}", "batch_per_gpu": 1,
                    "forward_entry": "dsa3d_forward_fixed_window" if fixed_window else "dsa3d_forward",
+                   "backward_entry": ("dsa3d_backward_fixed_window" if fixed_window else "dsa3d_backward")
+                                     if wl.backward else None,
                    "parallelism": f"independent videos x{world}",
                    "l2": "inputs (tens of GB) exceed the 126 MB L2; no flush needed"},
         "roofline": {"bound": "hbm", "kernel": dom["kernel"], "achieved": dom["achieved"], "peak": peak,
@@ -449,7 +458,8 @@ def run_ours(args, wl):
                      "whole_step": {"bytes": step_bytes, "achieved": step_bytes / (step_ms * 1e-3) / 1e9,
                                     "frac": step_bytes / (step_ms * 1e-3) / 1e9 / peak}},
         "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks, "producer": producer,
-        "gpu_launches": K * ((5 if tiled else 4) if (wl.backward and wl.dtype == torch.bfloat16)
+        "gpu_launches": K * (3 if (fixed_window and wl.backward) else
+                             (5 if tiled else 4) if (wl.backward and wl.dtype == torch.bfloat16)
                              else 2 if wl.backward else 1),
     }
     print(json.dumps(line), flush=True)

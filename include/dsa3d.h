@@ -264,6 +264,22 @@ int dsa3d_forward_residual(const void* q, const void* k, const void* v, const fl
 int dsa3d_forward_fixed_window(const void* q, const void* k, const void* v, int T, int H, int W, int heads, int d,
                                const int window[3], void* out, float* lse, int dtype, void* stream);
 
+/*
+ * dsa3d_backward_fixed_window: backward of the operator with every offset equal to zero, without
+ * an offsets tensor: dq, dk, dv (and doffsets, the gradient with respect to the offsets at zero,
+ * unless it is NULL) equal those of dsa3d_backward on an all-zero offsets tensor up to fp32
+ * summation order.  With a fixed window the contributions to a key's dK/dV come from the P
+ * queries around it, so they are gathered instead of scattered: no atomics, results bitwise
+ * deterministic, dk/dv written once in `dtype`.  `lse` is the forward's.  `workspace`:
+ * dsa3d_backward_fixed_window_workspace_bytes(...) bytes (two fp32 coefficients per sample),
+ * 16-byte aligned, contents undefined afterwards.  All supported dtypes, head sizes and windows.
+ */
+int dsa3d_backward_fixed_window(const void* q, const void* k, const void* v, const float* lse, const void* dout, int T,
+                                int H, int W, int heads, int d, const int window[3], void* dq, void* dk, void* dv,
+                                float* doffsets, void* workspace, size_t workspace_bytes, int dtype, void* stream);
+size_t dsa3d_backward_fixed_window_workspace_bytes(int T, int H, int W, int heads, int d, const int window[3],
+                                                   int dtype);
+
 /* Static, NUL-terminated description of a status code. */
 const char* dsa3d_status_string(int status);
 

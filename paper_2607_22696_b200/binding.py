@@ -79,6 +79,10 @@ def load():
     lib.dsa3d_forward_residual.argtypes = [p, p, p, p, p, i, i, i, i, i, win, p, p, i, p]
     lib.dsa3d_forward_fixed_window.restype = i
     lib.dsa3d_forward_fixed_window.argtypes = [p, p, p, i, i, i, i, i, win, p, p, i, p]
+    lib.dsa3d_backward_fixed_window.restype = i
+    lib.dsa3d_backward_fixed_window.argtypes = [p, p, p, p, p, i, i, i, i, i, win, p, p, p, p, p, sz, i, p]
+    lib.dsa3d_backward_fixed_window_workspace_bytes.restype = sz
+    lib.dsa3d_backward_fixed_window_workspace_bytes.argtypes = [i, i, i, i, i, win, i]
     lib.dsa3d_status_string.restype = ctypes.c_char_p
     lib.dsa3d_status_string.argtypes = [i]
     lib.dsa3d_last_cuda_error.restype = i
@@ -176,6 +180,26 @@ def dsa3d_forward_fixed_window(q, k, v, T, H, W, heads, d, window, out, lse, dty
     _check(lib.dsa3d_forward_fixed_window(
         _ptr(q, "q", n * d), _ptr(k, "k", n * d), _ptr(v, "v", n * d), T, H, W, heads, d, _window(window),
         _ptr(out, "out", n * d), _ptr(lse, "lse", n, torch.float32), code, _stream(stream)))
+
+
+def dsa3d_backward_fixed_window_workspace_bytes(T, H, W, heads, d, window, dtype) -> int:
+    code = _DTYPES[dtype] if isinstance(dtype, torch.dtype) else int(dtype)
+    return int(load().dsa3d_backward_fixed_window_workspace_bytes(T, H, W, heads, d, _window(window), code))
+
+
+def dsa3d_backward_fixed_window(q, k, v, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets, workspace,
+                                dtype=None, stream=None) -> None:
+    """dq, dk, dv (and doffsets unless None) <- backward with all offsets zero; see include/dsa3d.h."""
+    lib = load()
+    dt = q.dtype if dtype is None else dtype
+    code = _DTYPES[dt] if isinstance(dt, torch.dtype) else int(dt)
+    n = T * H * W * heads
+    P = int(window[0]) * int(window[1]) * int(window[2])
+    _check(lib.dsa3d_backward_fixed_window(
+        _ptr(q, "q", n * d), _ptr(k, "k", n * d), _ptr(v, "v", n * d), _ptr(lse, "lse", n, torch.float32),
+        _ptr(dout, "dout", n * d), T, H, W, heads, d, _window(window), _ptr(dq, "dq", n * d), _ptr(dk, "dk", n * d),
+        _ptr(dv, "dv", n * d), _ptr(doffsets, "doffsets", n * P * 3, torch.float32), _ptr(workspace, "workspace"),
+        workspace.numel() * workspace.element_size(), code, _stream(stream)))
 
 
 def dsa3d_dwconv3d_forward(x, weight, bias, T, H, W, C, kernel, y, dtype=None, stream=None) -> None:

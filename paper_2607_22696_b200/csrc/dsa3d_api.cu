@@ -152,6 +152,36 @@ int dsa3d_forward_fixed_window(const void* q, const void* k, const void* v, int 
     return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
 }
 
+size_t dsa3d_backward_fixed_window_workspace_bytes(int T, int H, int W, int heads, int d, const int window[3],
+                                                   int dtype) {
+    dsa3d::Problem pr;
+    if (make_problem(T, H, W, heads, d, window, dtype, pr) != DSA3D_OK) return 0;
+    return (static_cast<size_t>(pr.items) * pr.P * sizeof(float2) + 255) & ~static_cast<size_t>(255);
+}
+
+int dsa3d_backward_fixed_window(const void* q, const void* k, const void* v, const float* lse, const void* dout, int T,
+                                int H, int W, int heads, int d, const int window[3], void* dq, void* dk, void* dv,
+                                float* doffsets, void* workspace, size_t workspace_bytes, int dtype, void* stream) {
+    if (!q || !k || !v || !lse || !dout || !dq || !dk || !dv) return DSA3D_ERR_NULL_POINTER;
+    dsa3d::Problem pr;
+    const int rc = make_problem(T, H, W, heads, d, window, dtype, pr);
+    if (rc != DSA3D_OK) return rc;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(lse) || !aligned16(dout) || !aligned16(dq) ||
+        !aligned16(dk) || !aligned16(dv) || (doffsets && !aligned16(doffsets)))
+        return DSA3D_ERR_MISALIGNED;
+    const size_t need = dsa3d_backward_fixed_window_workspace_bytes(T, H, W, heads, d, window, dtype);
+    if (!workspace || workspace_bytes < need) return DSA3D_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return DSA3D_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = record(2, st);
+    if (e != cudaSuccess) return cuda_failed(e);
+    e = dsa3d::launch_fixed_window_backward(q, k, v, lse, dout, dq, dk, dv, doffsets, static_cast<float2*>(workspace), pr,
+                                            dtype == DSA3D_BF16, st);
+    if (e != cudaSuccess) return cuda_failed(e);
+    e = record(3, st);
+    return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
+}
+
 int dsa3d_forward_residual(const void* q, const void* k, const void* v, const float* offsets, const void* residual,
                            int T, int H, int W, int heads, int d, const int window[3], void* out, float* lse,
                            int dtype, void* stream) {

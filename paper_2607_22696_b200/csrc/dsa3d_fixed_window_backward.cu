@@ -1,0 +1,243 @@
+// Backward of the fixed-window variant (all offsets zero).  Every sample sits exactly on the
+// grid position query + b(p), so nothing is interpolated and nothing needs an atomic:
+//
+//   fixed_window_backward_query_kernel   one group of lanes per (query, head).  The dot products
+//       a = q.K_j and b = dO.V_j are taken once for every position j of the box the window and
+//       its +1 neighbours span ((kt+1)(kh+1)(kw+1) positions, 54 of them used for 3x3x3; only
+//       the window itself when dOffsets is not wanted), eight positions per transposed
+//       reduction, into a small table in shared memory.  From the table: alpha_p, g_p, delta,
+//       dS_p; dOffsets by the one-sided derivative of the trilinear weights at an integer
+//       position, dDelta_a = score(j + e_a) - score(j) with score = scale dS_p a + alpha_p b
+//       and positions outside the grid counting 0; the two coefficients scale dS_p and
+//       alpha_p of every sample go to the workspace; dQ = sum_p scale dS_p K_j in a second
+//       visit of the window's K rows.
+//   fixed_window_backward_key_kernel     one group per (key, head): with a fixed window the
+//       contributions to dK_j and dV_j come from the P queries j - b(p), so they are gathered:
+//       dK_j = sum_p coefK[j - b(p), p] q_{j - b(p)},  dV_j = sum_p coefV[j - b(p), p] dO_{j - b(p)},
+//       and written once in the storage type - no fp32 accumulators, no atomics, bitwise
+//       deterministic.
+#include "dsa3d_common.cuh"
+#include "dsa3d_kernels.h"
+
+namespace dsa3d {
+namespace {
+
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+                                   const float* __restrict__ lse, const T* __restrict__ dout, T* __restrict__ dq,
+                                   float* __restrict__ doffsets, float2* __restrict__ coef, const Problem pr) {
+    using E = Elt<T, 1>;
+    using Row = typename E::Row;
+    constexpr int VEC = E::VEC;
+    constexpr int LPR = D / VEC;
+    extern __shared__ float smem[];
+    const int lane = threadIdx.x & 31;
+    const int gl = lane & (LPR - 1);
+    constexpr unsigned gmask = kFullMask;
+    long long item = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) / LPR;
+    const long long warp_first = (static_cast<long long>(blockIdx.x) * blockDim.x + (threadIdx.x & ~31)) / LPR;
+    if (warp_first >= pr.items) return;
+    const bool active = item < pr.items;                 // a trailing group repeats the last item, stores off
+    if (!active) item = pr.items - 1;
+
+    const bool want_doff = doffsets != nullptr;
+    const int BT = pr.kt + (want_doff ? 1 : 0), BY = pr.kh + (want_doff ? 1 : 0), BX = pr.kw + (want_doff ? 1 : 0);
+    const int NB = BT * BY * BX;
+    const int NB8 = (NB + 7) & ~7;
+    // per group: ta[NB8], tb[NB8] (dot products per box position), sa[P] (alpha), sk[P] (scale dS)
+    float* ta = smem + static_cast<size_t>(threadIdx.x / LPR) * (2 * NB8 + 2 * pr.P);
+    float* tb = ta + NB8;
+    float* sa = tb + NB8;
+    float* sk = sa + pr.P;
+
+    const int m = static_cast<int>(item / pr.q_count);
+    const long long n = pr.q_begin + (item - static_cast<long long>(m) * pr.q_count);
+    const int x = static_cast<int>(n % pr.W);
+    const int y = static_cast<int>((n / pr.W) % pr.H);
+    const int t = static_cast<int>(n / (static_cast<long long>(pr.W) * pr.H));
+    const long long row = n * pr.heads + m;
+    const int ch = gl * VEC;
+    const float scale = rsqrtf(static_cast<float>(D));
+    const long long tok_stride = static_cast<long long>(pr.heads) * D;
+    const T* kh = k + static_cast<long long>(m) * D + ch;
+    const long long v_minus_k = v - k;
+    const int ot = t - pr.kt / 2, oy = y - pr.kh / 2, ox = x - pr.kw / 2;      // box origin
+
+    const Row qr = E::load(q + row * D + ch);
+    const Row dor = E::load(dout + row * D + ch);
+    const float lse2 = __ldg(lse + row) * kLog2e;
+
+    // ---- dot products over the box, eight positions per reduction
+    for (int c8 = 0; c8 < NB8; c8 += 8) {
+        float a8[8], b8[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int idx = c8 + i;
+            const int bw = idx % BX, bv = (idx / BX) % BY, bu = idx / (BX * BY);
+            const int pt = ot + bu, py = oy + bv, px = ox + bw;
+            // used: a window cell, or the +1 neighbour of one along exactly one axis
+            const int far = (bu == pr.kt) + (bv == pr.kh) + (bw == pr.kw);
+            const bool inside = idx < NB && far <= 1 && pt >= 0 && pt < pr.T && py >= 0 && py < pr.H && px >= 0 && px < pr.W;
+            a8[i] = b8[i] = 0.0f;
+            if (inside) {
+                const T* pk = kh + ((static_cast<long long>(pt) * pr.H + py) * pr.W + px) * tok_stride;
+                const Row kk = E::load(pk);
+                const Row vv = E::load(pk + v_minus_k);
+                a8[i] = E::dot(qr, kk, 0.0f);
+                b8[i] = E::dot(dor, vv, 0.0f);
+            }
+        }
+        if constexpr (LPR >= 8) {
+            group_reduce8<LPR>(a8, gl, gmask);
+            group_reduce8<LPR>(b8, gl, gmask);
+            const int which = reduce8_index<LPR>(gl);
+            if (gl == reduce8_lane<LPR>(which)) {
+                ta[c8 + which] = a8[0];
+                tb[c8 + which] = b8[0];
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                a8[i] = group_sum<LPR>(a8[i], gmask);
+                b8[i] = group_sum<LPR>(b8[i], gmask);
+            }
+            if (gl == 0) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) { ta[c8 + i] = a8[i]; tb[c8 + i] = b8[i]; }
+            }
+        }
+    }
+    __syncwarp();
+
+    // ---- softmax weights, delta
+    float delta = 0.0f;
+    for (int p = gl; p < pr.P; p += LPR) {
+        const int w = p % pr.kw, vv = (p / pr.kw) % pr.kh, u = p / (pr.kw * pr.kh);
+        const int idx = (u * BY + vv) * BX + w;
+        const float alpha = exp2f(fmaf(ta[idx], scale * kLog2e, -lse2));     // a position outside the grid: logit 0
+        sa[p] = alpha;
+        delta = fmaf(alpha, tb[idx], delta);
+    }
+    delta = group_sum<LPR>(delta, gmask);
+
+    // ---- dS, coefficients, dOffsets
+    for (int p = gl; p < pr.P; p += LPR) {
+        const int w = p % pr.kw, vv = (p / pr.kw) % pr.kh, u = p / (pr.kw * pr.kh);
+        const int idx = (u * BY + vv) * BX + w;
+        const float alpha = sa[p];
+        const float ck = scale * alpha * (tb[idx] - delta);
+        sk[p] = ck;
+        if (active) {
+            coef[row * pr.P + p] = make_float2(ck, alpha);
+            if (want_doff) {
+                const float s0 = fmaf(ck, ta[idx], alpha * tb[idx]);
+                float* dst = doffsets + (row * pr.P + p) * 3;
+                dst[0] = fmaf(ck, ta[idx + BY * BX], alpha * tb[idx + BY * BX]) - s0;
+                dst[1] = fmaf(ck, ta[idx + BX], alpha * tb[idx + BX]) - s0;
+                dst[2] = fmaf(ck, ta[idx + 1], alpha * tb[idx + 1]) - s0;
+            }
+        }
+    }
+    __syncwarp();
+
+    // ---- dQ = sum_p (scale dS_p) K_j over the window cells inside the grid
+    float dqv[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) dqv[e] = 0.0f;
+    for (int p = 0; p < pr.P; ++p) {
+        const int w = p % pr.kw, vv = (p / pr.kw) % pr.kh, u = p / (pr.kw * pr.kh);
+        const int pt = ot + u, py = oy + vv, px = ox + w;
+        if (pt < 0 || pt >= pr.T || py < 0 || py >= pr.H || px < 0 || px >= pr.W) continue;
+        const Row kk = E::load(kh + ((static_cast<long long>(pt) * pr.H + py) * pr.W + px) * tok_stride);
+        E::axpy(sk[p], kk, dqv);
+    }
+    if (active) E::store(dq + row * D + ch, dqv);
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+fixed_window_backward_key_kernel(const T* __restrict__ q, const T* __restrict__ dout, const float2* __restrict__ coef,
+                                 T* __restrict__ dk, T* __restrict__ dv, const Problem pr) {
+    using E = Elt<T, 1>;
+    using Row = typename E::Row;
+    constexpr int VEC = E::VEC;
+    constexpr int LPR = D / VEC;
+    const int gl = threadIdx.x & (LPR - 1);
+    const long long item = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) / LPR;
+    if (item >= pr.items) return;
+    const int m = static_cast<int>(item / pr.q_count);
+    const long long n = item - static_cast<long long>(m) * pr.q_count;
+    const int x = static_cast<int>(n % pr.W);
+    const int y = static_cast<int>((n / pr.W) % pr.H);
+    const int t = static_cast<int>(n / (static_cast<long long>(pr.W) * pr.H));
+    const int ch = gl * VEC;
+    float ak[VEC], av[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) ak[e] = av[e] = 0.0f;
+    int p = 0;
+    for (int u = 0; u < pr.kt; ++u)
+        for (int vv = 0; vv < pr.kh; ++vv)
+            for (int w = 0; w < pr.kw; ++w, ++p) {
+                // the query whose window cell p is this key
+                const int qt = t - (u - pr.kt / 2), qy = y - (vv - pr.kh / 2), qx = x - (w - pr.kw / 2);
+                if (qt < 0 || qt >= pr.T || qy < 0 || qy >= pr.H || qx < 0 || qx >= pr.W) continue;
+                const long long qrow = ((static_cast<long long>(qt) * pr.H + qy) * pr.W + qx) * pr.heads + m;
+                const float2 c = __ldg(coef + qrow * pr.P + p);
+                const Row qr = E::load(q + qrow * D + ch);
+                const Row dr = E::load(dout + qrow * D + ch);
+                E::axpy(c.x, qr, ak);
+                E::axpy(c.y, dr, av);
+            }
+    const long long row = n * pr.heads + m;
+    E::store(dk + row * D + ch, ak);
+    E::store(dv + row * D + ch, av);
+}
+
+template <typename T, int D>
+cudaError_t launch_t(const void* q, const void* k, const void* v, const float* lse, const void* dout, void* dq,
+                     void* dk, void* dv, float* doffsets, float2* coef, const Problem& pr, cudaStream_t stream) {
+    constexpr int LPR = D / Elt<T, 1>::VEC;
+    const int box = doffsets ? (pr.kt + 1) * (pr.kh + 1) * (pr.kw + 1) : pr.P;
+    const size_t per_group = (2 * static_cast<size_t>((box + 7) & ~7) + 2 * pr.P) * sizeof(float);
+    int threads = 256;
+    while (threads > 32 && static_cast<size_t>(threads / LPR) * per_group > 64 * 1024) threads /= 2;
+    const size_t smem = static_cast<size_t>(threads / LPR) * per_group;
+    auto qk = fixed_window_backward_query_kernel<T, D>;
+    if (smem > 48 * 1024) {
+        const cudaError_t e = cudaFuncSetAttribute(qk, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+    }
+    long long groups = threads / LPR;
+    long long blocks = (pr.items + groups - 1) / groups;
+    qk<<<static_cast<unsigned>(blocks), threads, smem, stream>>>(
+        static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), lse, static_cast<const T*>(dout),
+        static_cast<T*>(dq), doffsets, coef, pr);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    groups = 256 / LPR;
+    blocks = (pr.items + groups - 1) / groups;
+    fixed_window_backward_key_kernel<T, D><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
+        static_cast<const T*>(q), static_cast<const T*>(dout), coef, static_cast<T*>(dk), static_cast<T*>(dv), pr);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_fixed_window_backward(const void* q, const void* k, const void* v, const float* lse,
+                                         const void* dout, void* dq, void* dk, void* dv, float* doffsets,
+                                         float2* coef, const Problem& pr, bool bf16, cudaStream_t stream) {
+#define DSA3D_CASE(DD)                                                                                          \
+    case DD:                                                                                                    \
+        return bf16 ? launch_t<__nv_bfloat16, DD>(q, k, v, lse, dout, dq, dk, dv, doffsets, coef, pr, stream)   \
+                    : launch_t<float, DD>(q, k, v, lse, dout, dq, dk, dv, doffsets, coef, pr, stream);
+    switch (pr.d) {
+        DSA3D_CASE(32)
+        DSA3D_CASE(64)
+        DSA3D_CASE(128)
+    }
+#undef DSA3D_CASE
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace dsa3d

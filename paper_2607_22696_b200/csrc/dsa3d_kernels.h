@@ -45,6 +45,12 @@ int backward_impl(const void* q, const void* k, const void* v, const float* offs
                   void* dk, void* dv, float* doffsets, void* workspace, size_t workspace_bytes, int dtype,
                   void* stream, bool tiled);
 
+// Backward of the fixed-window variant (dsa3d_fixed_window_backward.cu): dq, dk, dv in the storage
+// type, doffsets (may be NULL), coef [N*heads, P] scratch.
+cudaError_t launch_fixed_window_backward(const void* q, const void* k, const void* v, const float* lse,
+                                         const void* dout, void* dq, void* dk, void* dv, float* doffsets,
+                                         float2* coef, const Problem& pr, bool bf16, cudaStream_t stream);
+
 // Host side of the TMA kernels (dsa3d_producer.cu).  encode_tensor_map_bf16: a tiled map over
 // a bf16 tensor of `rank` dimensions (innermost first; strides_bytes has rank-1 entries, the
 // innermost stride being 2), zero fill outside the tensor, 128-byte swizzle or none.

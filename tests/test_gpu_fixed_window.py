@@ -77,3 +77,76 @@ def test_tile_kernel_agrees_with_the_general_kernel_on_zero_offsets():
     assert float((lse_tc - lse_z).abs().max()) <= 1e-4
     ulp = (out_z.float().abs() * 2.0 ** -7).clamp_min(1e-3)
     assert bool(((out_tc.float() - out_z.float()).abs() <= ulp).all())      # within one bf16 step of each other
+
+
+# ------------------------------------------------------------------ fixed-window backward
+
+def _backward_case(shape, window, dtype, seed, with_doffsets=True):
+    T, H, W, heads, d = shape
+    P = window[0] * window[1] * window[2]
+    q, k, v = (inputs.normal(shape, seed, i, 1.0, dtype) for i in range(3))
+    dout = inputs.normal(shape, seed, 4, 1.0, dtype)
+    zeros = torch.zeros(T * H * W, heads, P, 3, dtype=F32)
+    _, ref_lse = oracle.forward(q.view(-1, heads, d), k, v, zeros, T, H, W, heads, d, window)
+    ref = oracle.backward(q.view(-1, heads, d), k, v, zeros, dout.view(-1, heads, d), T, H, W, heads, d, window)
+    dq_, dk_, dv_, dout_ = (z.cuda() for z in (q, k, v, dout))
+    out = torch.empty(shape, dtype=dtype, device="cuda")
+    lse = torch.empty((T, H, W, heads), dtype=F32, device="cuda")
+    binding.dsa3d_forward_fixed_window(dq_, dk_, dv_, T, H, W, heads, d, window, out, lse)
+    g = [torch.full(shape, float("nan"), dtype=dtype, device="cuda") for _ in range(3)]
+    doff = torch.full((T, H, W, heads, P, 3), float("nan"), dtype=F32, device="cuda") if with_doffsets else None
+    ws = torch.full((binding.dsa3d_backward_fixed_window_workspace_bytes(T, H, W, heads, d, window, dtype),), 0xFF,
+                    dtype=torch.uint8, device="cuda")
+    guard = torch.full((64,), 9.0, dtype=F32, device="cuda")
+    binding.dsa3d_backward_fixed_window(dq_, dk_, dv_, lse, dout_, T, H, W, heads, d, window, g[0], g[1], g[2], doff, ws)
+    torch.cuda.synchronize()
+    pu.assert_close("lse", lse, ref_lse.view(T, H, W, heads), dtype)
+    for name, got, want in zip(("dq", "dk", "dv"), g, ref[:3]):
+        pu.assert_close(name, got, want.view(shape), dtype, backward=True)
+    if with_doffsets:
+        pu.assert_close("doffsets", doff, ref[3].view(T, H, W, heads, P, 3), dtype, backward=True)
+    assert torch.equal(guard.cpu(), torch.full((64,), 9.0))
+    return (dq_, dk_, dv_, dout_, lse), g, doff
+
+
+@pytest.mark.parametrize("shape,window,dtype", [
+    ((6, 9, 13, 2, 128), (3, 3, 3), BF16), ((4, 5, 6, 2, 64), (3, 3, 3), BF16), ((3, 5, 6, 2, 32), (3, 3, 3), F32),
+    ((5, 6, 7, 2, 128), (2, 2, 2), BF16), ((4, 6, 9, 1, 64), (3, 5, 5), BF16), ((1, 1, 1, 1, 32), (3, 3, 3), F32),
+    ((2, 3, 4, 2, 32), (1, 1, 1), BF16), ((3, 8, 9, 2, 64), (1, 7, 7), F32), ((4, 4, 5, 3, 128), (5, 3, 1), F32)])
+def test_fixed_window_backward_matches_the_oracle(shape, window, dtype):
+    """Against the oracle on an all-zero offsets tensor: odd and even windows, windows that reach
+    two positions outside the grid (dead samples), a single token, every dtype and head size."""
+    _backward_case(shape, window, dtype, 150)
+
+
+def test_fixed_window_backward_without_doffsets_and_determinism():
+    """doffsets may be NULL (only the window's own positions are visited then); dk and dv are
+    gathered, not accumulated with atomics, so two runs agree bit for bit."""
+    shape, window = (5, 7, 9, 2, 128), (3, 3, 3)
+    T, H, W, heads, d = shape
+    (q, k, v, dout, lse), g1, doff = _backward_case(shape, window, BF16, 151)
+    (_, _, _, _, _), g0, none = _backward_case(shape, window, BF16, 151, with_doffsets=False)
+    assert none is None
+    for a, b in zip(g0, g1):
+        assert torch.equal(a, b)
+    g2 = [torch.empty_like(z) for z in g1]
+    ws = torch.empty((binding.dsa3d_backward_fixed_window_workspace_bytes(T, H, W, heads, d, window, BF16),),
+                     dtype=torch.uint8, device="cuda")
+    doff2 = torch.empty_like(doff)
+    binding.dsa3d_backward_fixed_window(q, k, v, lse, dout, T, H, W, heads, d, window, g2[0], g2[1], g2[2], doff2, ws)
+    torch.cuda.synchronize()
+    for a, b in zip(g1, g2):
+        assert torch.equal(a, b)
+    assert torch.equal(doff, doff2)
+
+
+def test_fixed_window_backward_agrees_with_the_general_backward_on_zero_offsets():
+    shape, window = (6, 8, 12, 2, 128), (3, 3, 3)
+    T, H, W, heads, d = shape
+    (q, k, v, dout, lse), g, doff = _backward_case(shape, window, BF16, 152)
+    zeros = torch.zeros(T, H, W, heads, 27, 3, dtype=F32, device="cuda")
+    gg = pu.gpu_backward(q, k, v, zeros, lse, dout, shape, window)
+    for name, a, b in zip(("dq", "dk", "dv"), g, gg[:3]):
+        step = (b.float().abs() * 2.0 ** -7).clamp_min(2e-3)
+        assert bool(((a.float() - b.float()).abs() <= step).all()), name
+    assert float((doff - gg[3]).abs().max()) <= 1e-4 * max(1.0, float(gg[3].abs().max()))
