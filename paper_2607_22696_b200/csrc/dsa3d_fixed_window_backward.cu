@@ -37,7 +37,7 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
     constexpr unsigned gmask = kFullMask;
     long long item = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) / LPR;
     const long long warp_first = (static_cast<long long>(blockIdx.x) * blockDim.x + (threadIdx.x & ~31)) / LPR;
-    if (warp_first >= pr.items) return;
+    const bool whole_warp_idle = warp_first >= pr.items;   // leaves after the block-wide table is built
     const bool active = item < pr.items;                 // a trailing group repeats the last item, stores off
     if (!active) item = pr.items - 1;
 
@@ -45,8 +45,25 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
     const int BT = pr.kt + (want_doff ? 1 : 0), BY = pr.kh + (want_doff ? 1 : 0), BX = pr.kw + (want_doff ? 1 : 0);
     const int NB = BT * BY * BX;
     const int NB8 = (NB + 7) & ~7;
+    // per block: box_tab[NB8] = displacement of box position idx from the box origin and whether
+    // it is used (a window cell, or the +1 neighbour of one along exactly one axis);
+    // samp_tab[P] = box index of sample p's own position
+    int4* box_tab = reinterpret_cast<int4*>(smem);
+    int* samp_tab = reinterpret_cast<int*>(box_tab + NB8);
+    float* group0 = reinterpret_cast<float*>(samp_tab + ((pr.P + 3) & ~3));
+    for (int idx = threadIdx.x; idx < NB8; idx += blockDim.x) {
+        const int bw = idx % BX, bv = (idx / BX) % BY, bu = idx / (BX * BY);
+        const int far = (bu == pr.kt) + (bv == pr.kh) + (bw == pr.kw);
+        box_tab[idx] = make_int4(bu, bv, bw, (idx < NB && far <= 1) ? 1 : 0);
+    }
+    for (int p = threadIdx.x; p < pr.P; p += blockDim.x) {
+        const int w = p % pr.kw, vv = (p / pr.kw) % pr.kh, u = p / (pr.kw * pr.kh);
+        samp_tab[p] = (u * BY + vv) * BX + w;
+    }
+    __syncthreads();
+    if (whole_warp_idle) return;
     // per group: ta[NB8], tb[NB8] (dot products per box position), sa[P] (alpha), sk[P] (scale dS)
-    float* ta = smem + static_cast<size_t>(threadIdx.x / LPR) * (2 * NB8 + 2 * pr.P);
+    float* ta = group0 + static_cast<size_t>(threadIdx.x / LPR) * (2 * NB8 + 2 * pr.P);
     float* tb = ta + NB8;
     float* sa = tb + NB8;
     float* sk = sa + pr.P;
@@ -68,25 +85,28 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
     const Row dor = E::load(dout + row * D + ch);
     const float lse2 = __ldg(lse + row) * kLog2e;
 
-    // ---- dot products over the box, eight positions per reduction
+    // ---- dot products over the box, eight positions per reduction: all 16 row loads of a chunk
+    //      are issued before the first dot product
     for (int c8 = 0; c8 < NB8; c8 += 8) {
+        Row kk[8], vv[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int4 bt = box_tab[c8 + i];
+            const int pt = ot + bt.x, py = oy + bt.y, px = ox + bt.z;
+            const bool inside = bt.w && pt >= 0 && pt < pr.T && py >= 0 && py < pr.H && px >= 0 && px < pr.W;
+            kk[i] = E::zero();
+            vv[i] = E::zero();
+            if (inside) {
+                const T* pk = kh + ((static_cast<long long>(pt) * pr.H + py) * pr.W + px) * tok_stride;
+                kk[i] = E::load(pk);
+                vv[i] = E::load(pk + v_minus_k);
+            }
+        }
         float a8[8], b8[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            const int idx = c8 + i;
-            const int bw = idx % BX, bv = (idx / BX) % BY, bu = idx / (BX * BY);
-            const int pt = ot + bu, py = oy + bv, px = ox + bw;
-            // used: a window cell, or the +1 neighbour of one along exactly one axis
-            const int far = (bu == pr.kt) + (bv == pr.kh) + (bw == pr.kw);
-            const bool inside = idx < NB && far <= 1 && pt >= 0 && pt < pr.T && py >= 0 && py < pr.H && px >= 0 && px < pr.W;
-            a8[i] = b8[i] = 0.0f;
-            if (inside) {
-                const T* pk = kh + ((static_cast<long long>(pt) * pr.H + py) * pr.W + px) * tok_stride;
-                const Row kk = E::load(pk);
-                const Row vv = E::load(pk + v_minus_k);
-                a8[i] = E::dot(qr, kk, 0.0f);
-                b8[i] = E::dot(dor, vv, 0.0f);
-            }
+            a8[i] = E::dot(qr, kk[i], 0.0f);
+            b8[i] = E::dot(dor, vv[i], 0.0f);
         }
         if constexpr (LPR >= 8) {
             group_reduce8<LPR>(a8, gl, gmask);
@@ -113,8 +133,7 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
     // ---- softmax weights, delta
     float delta = 0.0f;
     for (int p = gl; p < pr.P; p += LPR) {
-        const int w = p % pr.kw, vv = (p / pr.kw) % pr.kh, u = p / (pr.kw * pr.kh);
-        const int idx = (u * BY + vv) * BX + w;
+        const int idx = samp_tab[p];
         const float alpha = exp2f(fmaf(ta[idx], scale * kLog2e, -lse2));     // a position outside the grid: logit 0
         sa[p] = alpha;
         delta = fmaf(alpha, tb[idx], delta);
@@ -123,8 +142,7 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
 
     // ---- dS, coefficients, dOffsets
     for (int p = gl; p < pr.P; p += LPR) {
-        const int w = p % pr.kw, vv = (p / pr.kw) % pr.kh, u = p / (pr.kw * pr.kh);
-        const int idx = (u * BY + vv) * BX + w;
+        const int idx = samp_tab[p];
         const float alpha = sa[p];
         const float ck = scale * alpha * (tb[idx] - delta);
         sk[p] = ck;
@@ -145,12 +163,24 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
     float dqv[VEC];
 #pragma unroll
     for (int e = 0; e < VEC; ++e) dqv[e] = 0.0f;
-    for (int p = 0; p < pr.P; ++p) {
-        const int w = p % pr.kw, vv = (p / pr.kw) % pr.kh, u = p / (pr.kw * pr.kh);
-        const int pt = ot + u, py = oy + vv, px = ox + w;
-        if (pt < 0 || pt >= pr.T || py < 0 || py >= pr.H || px < 0 || px >= pr.W) continue;
-        const Row kk = E::load(kh + ((static_cast<long long>(pt) * pr.H + py) * pr.W + px) * tok_stride);
-        E::axpy(sk[p], kk, dqv);
+    for (int p0 = 0; p0 < pr.P; p0 += 8) {
+        Row kk[8];
+        float cks[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            kk[i] = E::zero();
+            cks[i] = 0.0f;
+            if (p0 + i < pr.P) {
+                const int4 bt = box_tab[samp_tab[p0 + i]];
+                const int pt = ot + bt.x, py = oy + bt.y, px = ox + bt.z;
+                if (pt >= 0 && pt < pr.T && py >= 0 && py < pr.H && px >= 0 && px < pr.W) {
+                    kk[i] = E::load(kh + ((static_cast<long long>(pt) * pr.H + py) * pr.W + px) * tok_stride);
+                    cks[i] = sk[p0 + i];
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) E::axpy(cks[i], kk[i], dqv);
     }
     if (active) E::store(dq + row * D + ch, dqv);
 }
@@ -199,10 +229,12 @@ cudaError_t launch_t(const void* q, const void* k, const void* v, const float* l
                      void* dk, void* dv, float* doffsets, float2* coef, const Problem& pr, cudaStream_t stream) {
     constexpr int LPR = D / Elt<T, 1>::VEC;
     const int box = doffsets ? (pr.kt + 1) * (pr.kh + 1) * (pr.kw + 1) : pr.P;
-    const size_t per_group = (2 * static_cast<size_t>((box + 7) & ~7) + 2 * pr.P) * sizeof(float);
+    const size_t box8 = static_cast<size_t>((box + 7) & ~7);
+    const size_t per_group = (2 * box8 + 2 * pr.P) * sizeof(float);
+    const size_t tables = box8 * sizeof(int4) + static_cast<size_t>((pr.P + 3) & ~3) * sizeof(int);
     int threads = 256;
-    while (threads > 32 && static_cast<size_t>(threads / LPR) * per_group > 64 * 1024) threads /= 2;
-    const size_t smem = static_cast<size_t>(threads / LPR) * per_group;
+    while (threads > 32 && tables + static_cast<size_t>(threads / LPR) * per_group > 64 * 1024) threads /= 2;
+    const size_t smem = tables + static_cast<size_t>(threads / LPR) * per_group;
     auto qk = fixed_window_backward_query_kernel<T, D>;
     if (smem > 48 * 1024) {
         const cudaError_t e = cudaFuncSetAttribute(qk, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
