@@ -150,3 +150,30 @@ def test_fixed_window_backward_agrees_with_the_general_backward_on_zero_offsets(
         step = (b.float().abs() * 2.0 ** -7).clamp_min(2e-3)
         assert bool(((a.float() - b.float()).abs() <= step).all()), name
     assert float((doff - gg[3]).abs().max()) <= 1e-4 * max(1.0, float(gg[3].abs().max()))
+
+
+def test_fixed_window_entry_points_agree_with_the_general_kernels_at_a_larger_size():
+    """57,600 tokens x 4 heads (450 tiles per head, several per persistent CTA, ragged in y):
+    forward and backward through the fixed-window entry points against the general kernels on
+    a zero offsets tensor; every element within one bf16 step."""
+    shape, window = (16, 45, 80, 4, 128), (3, 3, 3)
+    T, H, W, heads, d = shape
+    q, k, v = (inputs.normal(shape, 160, i, 1.0, BF16, device="cuda") for i in range(3))
+    dout = inputs.normal(shape, 160, 4, 1.0, BF16, device="cuda")
+    zeros = torch.zeros(T, H, W, heads, 27, 3, dtype=F32, device="cuda")
+    out_g, lse_g = pu.gpu_forward(q, k, v, zeros, shape, window)
+    g_g = pu.gpu_backward(q, k, v, zeros, lse_g, dout, shape, window)
+    out_f, lse_f = torch.empty_like(out_g), torch.empty_like(lse_g)
+    binding.dsa3d_forward_fixed_window(q, k, v, T, H, W, heads, d, window, out_f, lse_f)
+    g_f = [torch.empty_like(q) for _ in range(3)]
+    doff_f = torch.empty_like(zeros)
+    ws = torch.empty((binding.dsa3d_backward_fixed_window_workspace_bytes(T, H, W, heads, d, window, BF16),),
+                     dtype=torch.uint8, device="cuda")
+    binding.dsa3d_backward_fixed_window(q, k, v, lse_f, dout, T, H, W, heads, d, window, g_f[0], g_f[1], g_f[2], doff_f, ws)
+    torch.cuda.synchronize()
+    assert binding.dsa3d_device_timeout_flag() == 0
+    assert float((lse_f - lse_g).abs().max()) <= 1e-4
+    for name, a, b in zip(("out", "dq", "dk", "dv"), [out_f] + g_f, [out_g] + list(g_g[:3])):
+        step = (b.float().abs() * 2.0 ** -7).clamp_min(4e-3)
+        assert bool(((a.float() - b.float()).abs() <= step).all()), name
+    assert float((doff_f - g_g[3]).abs().max()) <= 2e-4 * max(1.0, float(g_g[3].abs().max()))
