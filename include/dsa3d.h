@@ -254,7 +254,7 @@ int dsa3d_forward_residual(const void* q, const void* k, const void* v, const fl
  * dsa3d_forward_fixed_window: the operator with every offset equal to zero (the fixed local
  * window of the ablation on the effect of offsets) without an offsets tensor: same out and
  * lse as dsa3d_forward on an all-zero offsets tensor, up to fp32 summation order.  For bf16,
- * d = 128 and windows (3,3,3) or (2,2,2) it runs as dense tile attention on the tensor cores
+ * d = 64 or 128 and windows (3,3,3) or (2,2,2) it runs as dense tile attention on the tensor cores
  * (scores of a 4x4x8 query tile against its halo region by tcgen05, window mask, softmax,
  * weighted sum from shared memory); every other supported shape runs the general kernel
  * with zero offsets.  The environment variable DSA3D_NO_TENSOR_FIXED_WINDOW forces the

@@ -4,7 +4,7 @@
 // of the dense product  Q_tile . K_region^T  over the tile's halo region, and the window is a
 // mask on that score tile.
 //
-// One CTA per (tile of 4 x 4 x 8 queries, head), bf16, 128 channels:
+// Persistent CTAs, a work item = (tile of 4 x 4 x 8 queries, head); bf16, 64 or 128 channels:
 //   1. TMA 5-D boxes bring the tile's Q rows (128 x 128), the K rows of the region
 //      (tile + kt-1, kh-1, kw-1 halo; zero rows outside the grid, which is exactly the
 //      zero-padded key of a sample outside the grid) in the 128-byte-swizzled K-major layout,
@@ -30,26 +30,29 @@ namespace dsa3d {
 namespace {
 
 constexpr int kFwTT = 4, kFwTY = 4, kFwTX = 8, kFwQ = kFwTT * kFwTY * kFwTX;   // 128 queries per tile
-constexpr int kFwD = 128;
 constexpr int kFwThreads = 256;
 constexpr int kFwMaxRows = 368;                   // region rows held per K half / V (multiple of 16)
 
+template <int D>
 struct __align__(1024) FwSmem {
-    unsigned char q[2][kFwQ * 128];               // two 64-channel halves, 128-byte rows; later score staging + weights
-    unsigned char k[2][kFwMaxRows * 128];         // two 64-channel halves
-    unsigned char v[kFwMaxRows * 256];            // full 256-byte rows
+    unsigned char q[D / 64][kFwQ * 128];          // 64-channel halves, 128-byte rows; later score staging + weights
+    unsigned char k[D / 64][kFwMaxRows * 128];    // 64-channel halves
+    unsigned char v[kFwMaxRows * D * 2];          // full rows
+    unsigned char w[D == 64 ? 16 * 1024 : 16];    // 64 channels: the softmax weights (the Q buffer is only 16 KB)
     uint64_t bar_q, bar_k, bar_v, bar_mma;
     uint32_t tmem_base;
     uint32_t abort;                               // set by the issuing thread when one of its waits ran out
 };
 
-template <int KT, int KH, int KW>
+template <int D, int KT, int KH, int KW>
 __global__ void __launch_bounds__(kFwThreads, 1)
 fixed_window_forward_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                             const __grid_constant__ CUtensorMap map_v, __nv_bfloat16* __restrict__ out,
                             float* __restrict__ lse, int T, int H, int W, int heads, int tiles_x, int tiles_y,
                             long long total, int* timeout_flag) {
     constexpr int P = KT * KH * KW;
+    constexpr int NH = D / 64;                                    // 64-channel halves of a row
+    constexpr int CPL = D / 16;                                   // channels per lane in the output phase
     constexpr int RT = kFwTT + KT - 1, RY = kFwTY + KH - 1, RX = kFwTX + KW - 1;
     constexpr int PS = RY * RX;                                   // rows of one region plane
     constexpr int R = RT * PS;                                    // region rows
@@ -58,10 +61,10 @@ fixed_window_forward_kernel(const __grid_constant__ CUtensorMap map_q, const __g
     constexpr int kChunks = (PS + 31) / 32;                       // 32-column pieces of a region plane
     static_assert(RP <= kFwMaxRows && N2 <= 256 && P <= 32, "shape not covered");
     static_assert((RT - 1) * PS + kChunks * 32 <= 512, "staged columns must stay inside the TMEM allocation");
-    static_assert(16 * KT * KH * kFwTX * KW * 4 <= 16 * 1024, "the weights must fit the upper half of the Q buffer");
+    static_assert(16 * KT * KH * kFwTX * KW * 4 <= 16 * 1024, "the weights must fit their 16 KB");
 
     extern __shared__ unsigned char raw[];
-    FwSmem& s = *reinterpret_cast<FwSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
+    FwSmem<D>& s = *reinterpret_cast<FwSmem<D>*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
@@ -93,21 +96,22 @@ fixed_window_forward_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         t0 = (tile / tiles_y) * kFwTT;
     };
     auto load_q = [&](int m, int t0, int y0, int x0) {
-        mbar_expect_tx(smem_u32(&s.bar_q), 2u * kFwQ * 128u);
-        for (int h = 0; h < 2; ++h) tma_load_5d(smem_u32(s.q[h]), &map_q, smem_u32(&s.bar_q), h * 64, m, x0, y0, t0);
+        mbar_expect_tx(smem_u32(&s.bar_q), static_cast<uint32_t>(NH) * kFwQ * 128u);
+        for (int h = 0; h < NH; ++h) tma_load_5d(smem_u32(s.q[h]), &map_q, smem_u32(&s.bar_q), h * 64, m, x0, y0, t0);
     };
     auto load_k = [&](int m, int t0, int y0, int x0) {
-        mbar_expect_tx(smem_u32(&s.bar_k), 2u * R * 128u);
-        for (int h = 0; h < 2; ++h)
+        mbar_expect_tx(smem_u32(&s.bar_k), static_cast<uint32_t>(NH) * R * 128u);
+        for (int h = 0; h < NH; ++h)
             tma_load_5d(smem_u32(s.k[h]), &map_k, smem_u32(&s.bar_k), h * 64, m, x0 - KW / 2, y0 - KH / 2, t0 - KT / 2);
     };
     auto load_v = [&](int m, int t0, int y0, int x0) {
-        mbar_expect_tx(smem_u32(&s.bar_v), static_cast<uint32_t>(R) * 256u);
+        mbar_expect_tx(smem_u32(&s.bar_v), static_cast<uint32_t>(R) * D * 2u);
         tma_load_5d(smem_u32(s.v), &map_v, smem_u32(&s.bar_v), 0, m, x0 - KW / 2, y0 - KH / 2, t0 - KT / 2);
     };
 
     float* stage = reinterpret_cast<float*>(s.q[0]);              // [32 columns][128 threads]: lower half of the Q buffer
-    float* wts = reinterpret_cast<float*>(s.q[1]);                // softmax weights: upper half of the Q buffer
+    // softmax weights: the second 16 KB of the Q buffer (128 channels) or their own array (64)
+    float* wts = reinterpret_cast<float*>(NH == 1 ? s.w : s.q[0] + 16 * 1024);
 
     if (tid == 0 && static_cast<long long>(blockIdx.x) < total) {
         int m, t0, y0, x0;
@@ -129,7 +133,7 @@ fixed_window_forward_kernel(const __grid_constant__ CUtensorMap map_q, const __g
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 constexpr uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kFwQ >> 4) << 24);
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
+                for (int h = 0; h < NH; ++h) {
                     const uint64_t da = smem_desc(smem_u32(s.q[h]));
                     const uint64_t db1 = smem_desc(smem_u32(s.k[h]));
                     const uint64_t db2 = smem_desc(smem_u32(s.k[h]) + N1 * 128);       // N1 rows = a multiple of 8
@@ -187,7 +191,7 @@ fixed_window_forward_kernel(const __grid_constant__ CUtensorMap map_q, const __g
                         __syncwarp();
                     }
                 }
-                const float lscale = rsqrtf(static_cast<float>(kFwD)) * kLog2e;
+                const float lscale = rsqrtf(static_cast<float>(D)) * kLog2e;
                 float mx = -INFINITY;
 #pragma unroll
                 for (int p = 0; p < P; ++p) { sc[p] *= lscale; mx = fmaxf(mx, sc[p]); }
@@ -222,11 +226,11 @@ fixed_window_forward_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         {
             const int hw = tid >> 4, hl = tid & 15;               // 16 half-warps = the 4 x 4 x-rows of the tile
             const int lt = hw >> 2, ly = hw & 3;
-            float acc[kFwTX][8];
+            float acc[kFwTX][CPL];
 #pragma unroll
             for (int qx = 0; qx < kFwTX; ++qx)
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[qx][e] = 0.0f;
+                for (int e = 0; e < CPL; ++e) acc[qx][e] = 0.0f;
             const float* wrow = wts + hw * (KT * KH * kFwTX * KW);
 #pragma unroll 1
             for (int uv = 0; uv < KT * KH; ++uv) {
@@ -237,21 +241,29 @@ fixed_window_forward_kernel(const __grid_constant__ CUtensorMap map_q, const __g
                     const float4 w4 = *reinterpret_cast<const float4*>(wrow + uv * (kFwTX * KW) + i);
                     wq[i] = w4.x; wq[i + 1] = w4.y; wq[i + 2] = w4.z; wq[i + 3] = w4.w;
                 }
-                const unsigned char* vrow = s.v + (((lt + u) * RY + ly + vv) * RX) * 256 + hl * 16;
+                const unsigned char* vrow = s.v + (((lt + u) * RY + ly + vv) * RX) * (D * 2) + hl * (CPL * 2);
 #pragma unroll
                 for (int xx = 0; xx < RX; ++xx) {
-                    const uint4 row = *reinterpret_cast<const uint4*>(vrow + xx * 256);
-                    float f[8];
-                    f[0] = __uint_as_float(row.x << 16); f[1] = __uint_as_float(row.x & 0xffff0000u);
-                    f[2] = __uint_as_float(row.y << 16); f[3] = __uint_as_float(row.y & 0xffff0000u);
-                    f[4] = __uint_as_float(row.z << 16); f[5] = __uint_as_float(row.z & 0xffff0000u);
-                    f[6] = __uint_as_float(row.w << 16); f[7] = __uint_as_float(row.w & 0xffff0000u);
+                    uint32_t words[CPL / 2];
+                    if constexpr (CPL == 8) {
+                        const uint4 row = *reinterpret_cast<const uint4*>(vrow + xx * (D * 2));
+                        words[0] = row.x; words[1] = row.y; words[2] = row.z; words[3] = row.w;
+                    } else {
+                        const uint2 row = *reinterpret_cast<const uint2*>(vrow + xx * (D * 2));
+                        words[0] = row.x; words[1] = row.y;
+                    }
+                    float f[CPL];
+#pragma unroll
+                    for (int i = 0; i < CPL / 2; ++i) {
+                        f[2 * i] = __uint_as_float(words[i] << 16);
+                        f[2 * i + 1] = __uint_as_float(words[i] & 0xffff0000u);
+                    }
 #pragma unroll
                     for (int ww = 0; ww < KW; ++ww) {
                         const int qx = xx - ww;                   // the query whose window cell ww is position xx
                         if (qx < 0 || qx >= kFwTX) continue;
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) acc[qx][e] = fmaf(wq[qx * KW + ww], f[e], acc[qx][e]);
+                        for (int e = 0; e < CPL; ++e) acc[qx][e] = fmaf(wq[qx * KW + ww], f[e], acc[qx][e]);
                     }
                 }
             }
@@ -262,13 +274,15 @@ fixed_window_forward_kernel(const __grid_constant__ CUtensorMap map_q, const __g
                     const int x = x0 + qx;
                     if (x >= W) continue;
                     const long long n = (static_cast<long long>(t) * H + y) * W + x;
-                    uint32_t o[4];
+                    uint32_t o[CPL / 2];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
+                    for (int i = 0; i < CPL / 2; ++i) {
                         const __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[qx][2 * i], acc[qx][2 * i + 1]);
                         o[i] = *reinterpret_cast<const uint32_t*>(&h2);
                     }
-                    *reinterpret_cast<uint4*>(out + (n * heads + m) * kFwD + hl * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                    __nv_bfloat16* dst = out + (n * heads + m) * D + hl * CPL;
+                    if constexpr (CPL == 8) *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+                    else *reinterpret_cast<uint2*>(dst) = make_uint2(o[0], o[1]);
                 }
             }
         }
@@ -300,19 +314,19 @@ bool make_maps(const void* q, const void* k, const void* v, const Problem& pr, i
     const unsigned box_q[5] = {64, 1, kFwTX, kFwTY, kFwTT};
     const unsigned box_k[5] = {64, 1, static_cast<unsigned>(kFwTX + kw - 1), static_cast<unsigned>(kFwTY + kh - 1),
                                static_cast<unsigned>(kFwTT + kt - 1)};
-    const unsigned box_v[5] = {128, 1, box_k[2], box_k[3], box_k[4]};
+    const unsigned box_v[5] = {static_cast<unsigned>(pr.d), 1, box_k[2], box_k[3], box_k[4]};
     return encode_tensor_map_bf16(mq, q, 5, dims, strides, box_q, true) &&
            encode_tensor_map_bf16(mk, k, 5, dims, strides, box_k, true) &&
            encode_tensor_map_bf16(mv, v, 5, dims, strides, box_v, false);
 }
 
-template <int KT, int KH, int KW>
+template <int D, int KT, int KH, int KW>
 cudaError_t launch(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, void* out, float* lse,
                    const Problem& pr, int* flag, cudaStream_t stream) {
     const int tiles_x = (pr.W + kFwTX - 1) / kFwTX, tiles_y = (pr.H + kFwTY - 1) / kFwTY,
               tiles_t = (pr.T + kFwTT - 1) / kFwTT;
-    const size_t smem = sizeof(FwSmem) + 1024;
-    auto kern = fixed_window_forward_kernel<KT, KH, KW>;
+    const size_t smem = sizeof(FwSmem<D>) + 1024;
+    auto kern = fixed_window_forward_kernel<D, KT, KH, KW>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
     const long long total = static_cast<long long>(tiles_x) * tiles_y * tiles_t * pr.heads;
@@ -332,7 +346,7 @@ cudaError_t launch(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorM
 bool try_fixed_window_forward(const void* q, const void* k, const void* v, void* out, float* lse, const Problem& pr,
                               cudaStream_t stream, cudaError_t* err) {
     *err = cudaSuccess;
-    if (pr.d != kFwD || pr.heads > 65535) return false;
+    if (pr.d != 128 && pr.d != 64) return false;
     const bool w333 = pr.kt == 3 && pr.kh == 3 && pr.kw == 3, w222 = pr.kt == 2 && pr.kh == 2 && pr.kw == 2;
     if (!w333 && !w222) return false;
     const long long tiles = static_cast<long long>((pr.W + kFwTX - 1) / kFwTX) * ((pr.H + kFwTY - 1) / kFwTY) *
@@ -341,8 +355,12 @@ bool try_fixed_window_forward(const void* q, const void* k, const void* v, void*
     int* flag = timeout_flag_device_address();
     CUtensorMap mq, mk, mv;
     if (!flag || !make_maps(q, k, v, pr, pr.kt, pr.kh, pr.kw, &mq, &mk, &mv)) return false;
-    *err = w333 ? launch<3, 3, 3>(mq, mk, mv, out, lse, pr, flag, stream)
-                : launch<2, 2, 2>(mq, mk, mv, out, lse, pr, flag, stream);
+    if (pr.d == 128)
+        *err = w333 ? launch<128, 3, 3, 3>(mq, mk, mv, out, lse, pr, flag, stream)
+                    : launch<128, 2, 2, 2>(mq, mk, mv, out, lse, pr, flag, stream);
+    else
+        *err = w333 ? launch<64, 3, 3, 3>(mq, mk, mv, out, lse, pr, flag, stream)
+                    : launch<64, 2, 2, 2>(mq, mk, mv, out, lse, pr, flag, stream);
     return true;
 }
 
