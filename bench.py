@@ -310,6 +310,17 @@ def run_ours(args, wl):
         return max_over_ranks(x, world, dev)
 
     binding.load()
+    # --shard heads: ONE video over all ranks, rank r taking heads [r*h/G, (r+1)*h/G) of every
+    # token (no exchange inside the operator: heads are independent) - strong scaling.  Default:
+    # every rank its own video - weak scaling.
+    sharded = args.shard == "heads" and world > 1
+    if sharded:
+        from paper_2607_22696_b200 import sharding
+        lo, hi = sharding.head_range(wl.heads, world, rank)
+        if hi == lo:
+            raise RuntimeError("more ranks than heads")
+        wl = inputs.dataclasses.replace(wl, heads=hi - lo)
+    videos = 1 if sharded else world
     dims = (wl.T, wl.H, wl.W, wl.heads, wl.d)
     producer = None
     if args.producer and rank == 0 and wl.dtype == torch.bfloat16:
@@ -373,14 +384,14 @@ def run_ours(args, wl):
     sct_ms = sum(ev[i][6].elapsed_time(ev[i][7]) for i in range(K)) / K if tiled else 0.0
     step_ms = max_ranks(step_ms)
     fwd_ms, bwd_ms, sct_ms = max_ranks(fwd_ms), max_ranks(bwd_ms), max_ranks(sct_ms)
-    value = aggregate_mtokens_per_s(wl, world, step_ms)
+    value = aggregate_mtokens_per_s(wl, videos, step_ms)
 
     # ---------------------------------------------------------------- end to end (host)
     e2e = None
     b.clear()                           # the end-to-end leg brings its own device arena
     torch.cuda.empty_cache()
     if not args.no_e2e:
-        e2e = run_e2e(args, wl, t, dims, dev, barrier, max_ranks, world)
+        e2e = run_e2e(args, wl, t, dims, dev, barrier, max_ranks, world, videos)
     # --------------------------------------------------------------------- CPU baseline
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -436,7 +447,8 @@ def run_ours(args, wl):
         traffic = items * per_item
     line = {
         "metric": metric_name(wl), "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
-        "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": step_ms, "higher_is_better": True, "scaling": "strong" if sharded else "weak",
+        "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": wl.name, "grid": [wl.T, wl.H, wl.W], "tokens": wl.N, "heads": wl.heads,
                    "d": wl.d, "window": list(wl.window), "storage": str(wl.dtype).replace("torch.", ""),
@@ -444,7 +456,8 @@ def run_ours(args, wl):
                    "forward_entry": "dsa3d_forward_fixed_window" if fixed_window else "dsa3d_forward",
                    "backward_entry": ("dsa3d_backward_fixed_window" if fixed_window else "dsa3d_backward")
                                      if wl.backward else None,
-                   "parallelism": f"independent videos x{world}",
+                   "parallelism": (f"one video, heads sharded over {world} ranks (heads of rank 0: {wl.heads})"
+                                   if sharded else f"independent videos x{world}"),
                    "l2": "inputs (tens of GB) exceed the 126 MB L2; no flush needed"},
         "roofline": {"bound": "hbm", "kernel": dom["kernel"], "achieved": dom["achieved"], "peak": peak,
                      "unit": "GB/s", "frac": dom["achieved"] / peak, "traffic": traffic,
@@ -489,7 +502,7 @@ def host_memory_available() -> int:
     return avail if avail is not None else 0
 
 
-def run_e2e(args, wl, t, dims, dev, barrier, max_ranks, world):
+def run_e2e(args, wl, t, dims, dev, barrier, max_ranks, world, videos=None):
     """Forward + backward through dsa3d_step_host: inputs start in pinned host memory and
     every output ends in pinned host memory, each step."""
     from paper_2607_22696_b200 import binding
@@ -542,7 +555,8 @@ def run_e2e(args, wl, t, dims, dev, barrier, max_ranks, world):
     ms = max_ranks(e0.elapsed_time(e1) / steps)
     h2d = sum(h.numel() * h.element_size() for h in host_in.values())
     d2h = sum(h.numel() * h.element_size() for h in host_out.values())
-    return {"value": aggregate_mtokens_per_s(wl, world, ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
+    return {"value": aggregate_mtokens_per_s(wl, world if videos is None else videos, ms), "unit": UNIT,
+            "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": ms, "wall_ms_per_step": wall * 1e3, "steps": steps,
             "entry_point": "dsa3d_step_host"}
 
@@ -558,6 +572,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--shard", default="videos", choices=["videos", "heads"],
+                    help="N > 1: every rank its own video (weak scaling, default) or one video with its heads "
+                         "split over the ranks (strong scaling)")
     ap.add_argument("--no-fixed-window", action="store_true",
                     help="zero-offset workloads: use dsa3d_forward on the zero tensor instead of dsa3d_forward_fixed_window")
     ap.add_argument("--producer", action="store_true",

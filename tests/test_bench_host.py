@@ -62,3 +62,49 @@ def test_two_gloo_ranks_take_different_videos_and_report_the_slowest_time():
     assert r0[2] != r1[2]                               # different data
     assert r0[3] == r1[3] == 15.0                       # max over ranks, seen by both
     assert abs(r0[4] - 2 * 256 / 15e-3 / 1e6) < 1e-12   # whole-job tokens / slowest time
+
+
+def _head_shard_main(rank, world, port, results):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import oracle
+    from paper_2607_22696_b200 import inputs, sharding
+    T, H, W, heads, d, window = 3, 4, 5, 3, 32, (3, 3, 3)            # 3 heads over 2 ranks: 2 + 1
+    shape = (T, H, W, heads, d)
+    q, k, v = (inputs.normal(shape, 200, i, 1.0, torch.float32) for i in range(3))
+    off = inputs.normal((T, H, W, heads, 27, 3), 200, 3, 1.0, torch.float32)
+    lo, hi = sharding.head_range(heads, world, rank)
+    mine = [sharding.shard_heads(z, world, rank) for z in (q, k, v, off)]
+    h = hi - lo
+    out, lse = oracle.forward(mine[0].view(-1, h, d), mine[1], mine[2], mine[3].view(-1, h, 27, 3), T, H, W, h, d, window)
+    out = out.view(T, H, W, h, d).contiguous()
+    # gather every rank's slice (ranks hold different head counts: pad to the largest)
+    hmax = sharding.head_range(heads, world, 0)[1]
+    padded = torch.zeros(T, H, W, hmax, d, dtype=out.dtype)
+    padded[:, :, :, :h] = out
+    bufs = [torch.zeros_like(padded) for _ in range(world)]
+    dist.all_gather(bufs, padded)
+    parts = []
+    for r in range(world):
+        rlo, rhi = sharding.head_range(heads, world, r)
+        parts.append(bufs[r][:, :, :, :rhi - rlo])
+    full = sharding.unshard_heads(parts)
+    ref, _ = oracle.forward(q.view(-1, heads, d), k, v, off.view(-1, heads, 27, 3), T, H, W, heads, d, window)
+    results[rank] = ((lo, hi), float((full - ref.view(shape)).abs().max()))
+    dist.destroy_process_group()
+
+
+def test_head_sharding_over_two_gloo_ranks_reproduces_the_unsharded_result():
+    """Heads are independent, so the operator shards over heads with no exchange: each rank
+    runs its slice (here through the CPU oracle) and the concatenation along the head axis
+    equals the unsharded result exactly."""
+    from paper_2607_22696_b200 import sharding
+    assert [sharding.head_range(16, 8, r) for r in (0, 7)] == [(0, 2), (14, 16)]
+    assert [sharding.head_range(5, 3, r) for r in range(3)] == [(0, 2), (2, 4), (4, 5)]
+    world, port = 2, 29531
+    with mp.Manager() as manager:
+        results = manager.dict()
+        mp.spawn(_head_shard_main, args=(world, port, results), nprocs=world, join=True)
+        r0, r1 = results[0], results[1]
+    assert r0[0] == (0, 2) and r1[0] == (2, 3)
+    assert r0[1] == 0.0 and r1[1] == 0.0
