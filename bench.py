@@ -506,7 +506,8 @@ def run_e2e(args, wl, t, dims, dev, barrier, max_ranks, world, videos=None):
     """Forward + backward through dsa3d_step_host: inputs start in pinned host memory and
     every output ends in pinned host memory, each step."""
     from paper_2607_22696_b200 import binding
-    names_in = ["q", "k", "v", "offsets", "dout"]
+    # a forward-only workload goes through the forward-only host entry point
+    names_in = ["q", "k", "v", "offsets", "dout"] if wl.backward else ["q", "k", "v", "offsets"]
     # The step keeps every input and every output in page-locked host memory (about twice the
     # input bytes per rank).  Page-locking more than the host can spare takes the machine
     # down, so the leg is skipped, on all ranks together, unless every rank's share fits
@@ -527,13 +528,20 @@ def run_e2e(args, wl, t, dims, dev, barrier, max_ranks, world, videos=None):
     torch.cuda.synchronize()
     torch.cuda.empty_cache()
     row_shape, row_dtype = shapes["q"]
-    host_out = {n: torch.empty(row_shape, dtype=row_dtype, pin_memory=True) for n in ("out", "dq", "dk", "dv")}
+    out_names = ("out", "dq", "dk", "dv") if wl.backward else ("out",)
+    host_out = {n: torch.empty(row_shape, dtype=row_dtype, pin_memory=True) for n in out_names}
     host_out["lse"] = torch.empty(dims[:4], dtype=torch.float32, pin_memory=True)
-    host_out["doffsets"] = torch.empty(shapes["offsets"][0], dtype=torch.float32, pin_memory=True)
-    arena_bytes = binding.dsa3d_step_host_arena_bytes(*dims, wl.window, wl.dtype)
+    if wl.backward:
+        host_out["doffsets"] = torch.empty(shapes["offsets"][0], dtype=torch.float32, pin_memory=True)
+    arena_bytes = (binding.dsa3d_step_host_arena_bytes if wl.backward else
+                   binding.dsa3d_forward_host_arena_bytes)(*dims, wl.window, wl.dtype)
     arena = torch.empty(arena_bytes, dtype=torch.uint8, device=dev)
 
     def step():
+        if not wl.backward:
+            binding.dsa3d_forward_host(host_in["q"], host_in["k"], host_in["v"], host_in["offsets"], *dims, wl.window,
+                                       host_out["out"], host_out["lse"], arena)
+            return
         binding.dsa3d_step_host(host_in["q"], host_in["k"], host_in["v"], host_in["offsets"], host_in["dout"],
                                 *dims, wl.window, host_out["out"], host_out["lse"], host_out["dq"],
                                 host_out["dk"], host_out["dv"], host_out["doffsets"], arena)
@@ -558,7 +566,7 @@ def run_e2e(args, wl, t, dims, dev, barrier, max_ranks, world, videos=None):
     return {"value": aggregate_mtokens_per_s(wl, world if videos is None else videos, ms), "unit": UNIT,
             "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": ms, "wall_ms_per_step": wall * 1e3, "steps": steps,
-            "entry_point": "dsa3d_step_host"}
+            "entry_point": "dsa3d_step_host" if wl.backward else "dsa3d_forward_host"}
 
 
 def main():

@@ -139,6 +139,19 @@ size_t dsa3d_step_host_arena_bytes(int T, int H, int W, int heads, int d, const 
                                    int dtype);
 
 /*
+ * dsa3d_forward_host: the forward alone on HOST buffers (sampling / inference): q, k, v,
+ * offsets in, out and lse back, pipelined over slabs of frames like dsa3d_step_host (K and V
+ * go up first; a slab's q and offsets go up while earlier slabs compute and its out and lse
+ * come back while later slabs compute).  `arena`: caller-owned DEVICE scratch of at least
+ * dsa3d_forward_host_arena_bytes(...) bytes, 256-byte aligned.  Same side streams, ordering
+ * and capture restriction as dsa3d_step_host.
+ */
+int dsa3d_forward_host(const void* q_h, const void* k_h, const void* v_h, const float* offsets_h, int T, int H, int W,
+                       int heads, int d, const int window[3], void* out_h, float* lse_h, void* arena,
+                       size_t arena_bytes, int dtype, void* stream);
+size_t dsa3d_forward_host_arena_bytes(int T, int H, int W, int heads, int d, const int window[3], int dtype);
+
+/*
  * Backward without any caller-provided or allocated scratch (the paper has no counterpart;
  * this exists for deployment reasons only).  Meant for callers that cannot give the
  * library a workspace: code running where all device memory was planned ahead of time,

@@ -83,6 +83,10 @@ def load():
     lib.dsa3d_backward_fixed_window.argtypes = [p, p, p, p, p, i, i, i, i, i, win, p, p, p, p, p, sz, i, p]
     lib.dsa3d_backward_fixed_window_workspace_bytes.restype = sz
     lib.dsa3d_backward_fixed_window_workspace_bytes.argtypes = [i, i, i, i, i, win, i]
+    lib.dsa3d_forward_host.restype = i
+    lib.dsa3d_forward_host.argtypes = [p, p, p, p, i, i, i, i, i, win, p, p, p, sz, i, p]
+    lib.dsa3d_forward_host_arena_bytes.restype = sz
+    lib.dsa3d_forward_host_arena_bytes.argtypes = [i, i, i, i, i, win, i]
     lib.dsa3d_status_string.restype = ctypes.c_char_p
     lib.dsa3d_status_string.argtypes = [i]
     lib.dsa3d_last_cuda_error.restype = i
@@ -277,6 +281,26 @@ def dsa3d_step_host(q_h, k_h, v_h, offsets_h, dout_h, T, H, W, heads, d, window,
         _host_ptr(out_h, "out_h", n * d, dt), _host_ptr(lse_h, "lse_h", n, f32),
         _host_ptr(dq_h, "dq_h", n * d, dt), _host_ptr(dk_h, "dk_h", n * d, dt),
         _host_ptr(dv_h, "dv_h", n * d, dt), _host_ptr(doffsets_h, "doffsets_h", n * P * 3, f32),
+        _ptr(arena, "arena"), arena.numel() * arena.element_size(), _DTYPES[dt], _stream(stream)))
+
+
+def dsa3d_forward_host_arena_bytes(T, H, W, heads, d, window, dtype) -> int:
+    code = _DTYPES[dtype] if isinstance(dtype, torch.dtype) else int(dtype)
+    return int(load().dsa3d_forward_host_arena_bytes(T, H, W, heads, d, _window(window), code))
+
+
+def dsa3d_forward_host(q_h, k_h, v_h, offsets_h, T, H, W, heads, d, window, out_h, lse_h, arena, stream=None) -> None:
+    """Forward from HOST tensors (pinned for speed) through a caller-owned device arena; see
+    include/dsa3d.h.  Asynchronous on `stream`."""
+    lib = load()
+    dt = q_h.dtype
+    n = T * H * W * heads
+    P = int(window[0]) * int(window[1]) * int(window[2])
+    f32 = torch.float32
+    _check(lib.dsa3d_forward_host(
+        _host_ptr(q_h, "q_h", n * d, dt), _host_ptr(k_h, "k_h", n * d, dt), _host_ptr(v_h, "v_h", n * d, dt),
+        _host_ptr(offsets_h, "offsets_h", n * P * 3, f32), T, H, W, heads, d, _window(window),
+        _host_ptr(out_h, "out_h", n * d, dt), _host_ptr(lse_h, "lse_h", n, f32),
         _ptr(arena, "arena"), arena.numel() * arena.element_size(), _DTYPES[dt], _stream(stream)))
 
 

@@ -539,6 +539,88 @@ int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const flo
     return DSA3D_OK;
 }
 
+// Forward only on host buffers (inference / sampling): device arena = q, k, v, out rows,
+// offsets, lse.
+size_t dsa3d_forward_host_arena_bytes(int T, int H, int W, int heads, int d, const int window[3], int dtype) {
+    dsa3d::Problem pr;
+    if (make_problem(T, H, W, heads, d, window, dtype, pr) != DSA3D_OK) return 0;
+    const size_t elt = dtype == DSA3D_BF16 ? 2 : 4;
+    const size_t rows = round256(static_cast<size_t>(pr.items) * pr.d * elt);
+    return 4 * rows + round256(static_cast<size_t>(pr.items) * pr.P * 3 * sizeof(float)) +
+           round256(static_cast<size_t>(pr.items) * sizeof(float));
+}
+
+int dsa3d_forward_host(const void* q_h, const void* k_h, const void* v_h, const float* offsets_h, int T, int H, int W,
+                       int heads, int d, const int window[3], void* out_h, float* lse_h, void* arena,
+                       size_t arena_bytes, int dtype, void* stream_) {
+    if (!q_h || !k_h || !v_h || !offsets_h || !out_h || !lse_h || !arena) return DSA3D_ERR_NULL_POINTER;
+    dsa3d::Problem pr;
+    const int rc = make_problem(T, H, W, heads, d, window, dtype, pr);
+    if (rc != DSA3D_OK) return rc;
+    if ((reinterpret_cast<uintptr_t>(arena) & 255u) != 0) return DSA3D_ERR_MISALIGNED;
+    if (arena_bytes < dsa3d_forward_host_arena_bytes(T, H, W, heads, d, window, dtype)) return DSA3D_ERR_WORKSPACE;
+    const bool bf16 = dtype == DSA3D_BF16;
+    const size_t elt = bf16 ? 2 : 4;
+    const size_t row_bytes = static_cast<size_t>(pr.items) * pr.d * elt;
+    const size_t rows = round256(row_bytes);
+    char* base = static_cast<char*>(arena);
+    char *q_d = base, *k_d = base + rows, *v_d = base + 2 * rows, *out_d = base + 3 * rows;
+    char* off_d = base + 4 * rows;
+    char* lse_d = off_d + round256(static_cast<size_t>(pr.items) * pr.P * 3 * sizeof(float));
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    HostStep* hs = host_step_resources();
+    if (!hs) return cuda_failed(cudaGetLastError());
+    cudaError_t e;
+#define DSA3D_TRY(call)                         \
+    do {                                        \
+        e = (call);                             \
+        if (e != cudaSuccess) return cuda_failed(e); \
+    } while (0)
+    // K and V first (every query needs all of them), then slabs of frames: a slab's q and offsets
+    // go up on one side stream while earlier slabs compute, its out and lse come back on the other.
+    int slab_frames = (T + kMaxSlabs - 1) / kMaxSlabs;
+    const int slabs = (T + slab_frames - 1) / slab_frames;
+    const size_t frame_rows = static_cast<size_t>(H) * W * heads;
+    const size_t frame_row_bytes = frame_rows * d * elt;
+    const size_t frame_off_bytes = frame_rows * pr.P * 3 * sizeof(float);
+    const size_t frame_lse_bytes = frame_rows * sizeof(float);
+    DSA3D_TRY(cudaEventRecord(hs->start, stream));
+    DSA3D_TRY(cudaStreamWaitEvent(hs->in, hs->start, 0));
+    DSA3D_TRY(cudaStreamWaitEvent(hs->out, hs->start, 0));
+    DSA3D_TRY(cudaMemcpyAsync(k_d, k_h, row_bytes, cudaMemcpyHostToDevice, hs->in));
+    DSA3D_TRY(cudaMemcpyAsync(v_d, v_h, row_bytes, cudaMemcpyHostToDevice, hs->in));
+    DSA3D_TRY(cudaEventRecord(hs->kv_ready, hs->in));
+    for (int s = 0; s < slabs; ++s) {
+        const int f0 = s * slab_frames, f1 = f0 + slab_frames < T ? f0 + slab_frames : T;
+        const size_t nf = static_cast<size_t>(f1 - f0);
+        DSA3D_TRY(cudaMemcpyAsync(q_d + f0 * frame_row_bytes, static_cast<const char*>(q_h) + f0 * frame_row_bytes,
+                                  nf * frame_row_bytes, cudaMemcpyHostToDevice, hs->in));
+        DSA3D_TRY(cudaMemcpyAsync(off_d + f0 * frame_off_bytes,
+                                  reinterpret_cast<const char*>(offsets_h) + f0 * frame_off_bytes, nf * frame_off_bytes,
+                                  cudaMemcpyHostToDevice, hs->in));
+        DSA3D_TRY(cudaEventRecord(hs->q_ready[s], hs->in));
+    }
+    DSA3D_TRY(cudaStreamWaitEvent(stream, hs->kv_ready, 0));
+    for (int s = 0; s < slabs; ++s) {
+        const int f0 = s * slab_frames, f1 = f0 + slab_frames < T ? f0 + slab_frames : T;
+        const size_t nf = static_cast<size_t>(f1 - f0);
+        DSA3D_TRY(cudaStreamWaitEvent(stream, hs->q_ready[s], 0));
+        const int st = forward_frames(pr, q_d, k_d, v_d, reinterpret_cast<const float*>(off_d), out_d,
+                                      reinterpret_cast<float*>(lse_d), bf16, f0, f1, stream);
+        if (st != DSA3D_OK) return st;
+        DSA3D_TRY(cudaEventRecord(hs->fwd_done[s], stream));
+        DSA3D_TRY(cudaStreamWaitEvent(hs->out, hs->fwd_done[s], 0));
+        DSA3D_TRY(cudaMemcpyAsync(static_cast<char*>(out_h) + f0 * frame_row_bytes, out_d + f0 * frame_row_bytes,
+                                  nf * frame_row_bytes, cudaMemcpyDeviceToHost, hs->out));
+        DSA3D_TRY(cudaMemcpyAsync(reinterpret_cast<char*>(lse_h) + f0 * frame_lse_bytes, lse_d + f0 * frame_lse_bytes,
+                                  nf * frame_lse_bytes, cudaMemcpyDeviceToHost, hs->out));
+    }
+    DSA3D_TRY(cudaEventRecord(hs->out_done, hs->out));
+    DSA3D_TRY(cudaStreamWaitEvent(stream, hs->out_done, 0));     // the call is over when `stream` is
+#undef DSA3D_TRY
+    return DSA3D_OK;
+}
+
 int dsa3d_set_profile_events(void* fwd_start, void* fwd_stop, void* bwd_start, void* bwd_stop,
                              void* scatter_start, void* scatter_stop) {
     g_events[0] = static_cast<cudaEvent_t>(fwd_start);

@@ -347,3 +347,23 @@ def test_forward_and_backward_can_be_captured_in_a_cuda_graph(dtype):
         for got, ref in ((dk, g_e[1]), (dv, g_e[2])):
             ref = ref.float()
             assert float((got.float() - ref).abs().max()) <= 2e-2 * float(ref.abs().max())
+
+
+@pytest.mark.parametrize("dtype,shape", [(BF16, (19, 9, 10, 2, 128)), (F32, (11, 5, 6, 2, 32)), (BF16, (1, 7, 9, 2, 64))])
+def test_forward_host_matches_the_device_forward(dtype, shape):
+    """dsa3d_forward_host (host buffers in and out, slabs of frames pipelined over two side
+    streams) returns exactly what dsa3d_forward returns on device buffers; twice in a row."""
+    q, k, v, off, _ = small_problem(*shape, (3, 3, 3), dtype, 1.3, 61)
+    dims = tuple(q.shape)
+    out_d, lse_d = pu.gpu_forward(q.cuda(), k.cuda(), v.cuda(), off.cuda(), dims, (3, 3, 3))
+    pin = lambda z: z.clone().pin_memory()
+    hq, hk, hv, hoff = pin(q), pin(k), pin(v), pin(off)
+    out_h = torch.full_like(q, float("nan")).pin_memory()
+    lse_h = torch.full(dims[:4], float("nan")).pin_memory()
+    arena = torch.empty(binding.dsa3d_forward_host_arena_bytes(*dims, (3, 3, 3), dtype), dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        binding.dsa3d_forward_host(hq, hk, hv, hoff, *dims, (3, 3, 3), out_h, lse_h, arena)
+        torch.cuda.synchronize()
+        assert torch.equal(out_h, out_d.cpu()) and torch.equal(lse_h, lse_d.cpu())
+        out_h.fill_(float("nan"))
+        lse_h.fill_(float("nan"))
