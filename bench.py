@@ -51,6 +51,10 @@ NCU_DRAM_BYTES_PER_ITEM = {"forward_kernel": 1525.0, "backward_kernel": 2991.0, 
 # of the same capture / items): what is left of the 110,592 gathered bytes after L1 hits.
 NCU_L2_TO_SM_BYTES_PER_ITEM = {"forward_kernel": 82380.0, "backward_kernel": 95482.0}
 NCU_RED_BYTES_PER_ITEM = {"scatter_tile_kernel": 23470.0}      # lts red sectors x 32 B / items
+# Warp instructions executed per item (smsp__inst_executed.sum of the same captures / items):
+# against the issue rate of 4 warp instructions per clock and SM they say how full the
+# schedulers are, which is what bounds the two backward kernels.
+NCU_WARP_INSTRUCTIONS_PER_ITEM = {"forward_kernel": 5402.0, "backward_kernel": 6532.0, "scatter_tile_kernel": 6999.0}
 
 
 def measure_ceilings(dev):
@@ -439,6 +443,15 @@ def run_ours(args, wl):
             if wl.d == 128 and wl.P == 27:
                 red_gbs = items_all * NCU_RED_BYTES_PER_ITEM["scatter_tile_kernel"] / (sct_ms * 1e-3) / 1e9
                 onchip["scatter_tile_kernel"].update(red_gbs=red_gbs, red_frac=red_gbs / ceil["l2_red_v4_f32_gbs"])
+    if wl.dtype == torch.bfloat16 and wl.d == 128 and wl.P == 27 and not fixed_window:
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        mhz = (clocks or {}).get("sm_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
+        issue_peak = 4.0 * sms * mhz * 1e6                      # warp instructions per second
+        onchip["issue_rate_peak_ginst"] = issue_peak / 1e9
+        for name, ms in (("forward_kernel", fwd_ms), ("backward_kernel", bwd_ms), ("scatter_tile_kernel", sct_ms)):
+            if name in onchip and ms > 0:
+                onchip[name]["issue_frac"] = (items_all * NCU_WARP_INSTRUCTIONS_PER_ITEM[name] / (ms * 1e-3)
+                                              / issue_peak)
     traffic = None
     if wl.dtype == torch.bfloat16 and wl.d == 128 and wl.P == 27 and not fixed_window:
         items = wl.N * wl.heads
