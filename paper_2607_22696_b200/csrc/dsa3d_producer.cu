@@ -7,7 +7,8 @@
 //                          TMEM -> bias + fp32 stores.  Persistent, one CTA per SM, warp-
 //                          specialised (TMA producer, MMA issuer, four epilogue warps), four
 //                          shared-memory stages, two TMEM accumulator buffers so the epilogue of
-//                          one tile overlaps the contraction of the next.
+//                          one tile overlaps the contraction of the next.  By default pairs of CTAs
+//                          share a 256-row tile (offsets_gemm_pair_kernel, cta_group::2).
 //   offsets_linear_f32_kernel  the same layer in plain fp32 FMAs for fp32 storage.
 // Every wait on an mbarrier is bounded; a wait that runs out raises a device flag (readable
 // with dsa3d_device_timeout_flag) and the roles drain and free TMEM instead of spinning.
@@ -16,6 +17,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <cstdlib>
 #include <mutex>
 
 #include "../../include/dsa3d.h"
@@ -435,6 +437,137 @@ dwconv3d_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* __re
     }
 }
 
+// The same contraction by pairs of CTAs (a cluster of two SMs on one 256 x BN tile,
+// tcgen05.mma.cta_group::2): each CTA loads its own 128 rows of u and HALF of the w tile, the
+// leader's single MMA thread multiplies both CTAs' operands and its commits arrive on the
+// barriers of both, each CTA drains its own 128 accumulator rows.  Halving the w traffic per SM
+// takes the operand stream under the 64 B/clk an SM can pull from L2 (the one-CTA tiling needs
+// 93 B/clk at full tensor rate).
+constexpr int kPairStages = 6;
+struct __align__(1024) GemmPairSmem {
+    __nv_bfloat16 a[kPairStages][BM * BK];
+    __nv_bfloat16 b[kPairStages][(kMaxBN / 2) * BK];
+    uint64_t full[kPairStages], empty[kPairStages], acc_full[2], acc_empty[2];
+    uint32_t tmem_base;
+};
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_constant__ CUtensorMap map_w,
+                         const float* __restrict__ bias, float* __restrict__ out, long long M, int N, int K, int BN,
+                         long long m_tiles, int n_tiles) {
+    extern __shared__ unsigned char raw[];
+    GemmPairSmem& s = *reinterpret_cast<GemmPairSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();                       // 0: leader (issues the MMAs)
+    const int kblocks = (K + BK - 1) / BK;
+    const long long tiles = m_tiles * n_tiles;                  // m_tiles counts 256-row tiles here
+    const long long pair = blockIdx.x / 2, pairs = gridDim.x / 2;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kPairStages; ++i) { mbar_init(smem_u32(&s.full[i]), 1); mbar_init(smem_u32(&s.empty[i]), 1); }
+        // acc_empty of the leader collects the four epilogue warps of both CTAs
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&s.acc_full[i]), 1); mbar_init(smem_u32(&s.acc_empty[i]), 8); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&s.tmem_base)), "r"(2 * kMaxBN));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    cluster_sync_all();                                          // both CTAs' barriers exist from here on
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = s.tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            for (long long tile = pair; tile < tiles; tile += pairs) {
+                const int n0 = static_cast<int>(tile % n_tiles) * BN;
+                const long long m0 = (tile / n_tiles) * (2 * BM);
+                bool ok = true;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int st = it % kPairStages;
+                    if (!mbar_wait(smem_u32(&s.empty[st]), ((it / kPairStages) & 1) ^ 1)) { ok = false; break; }
+                    const uint32_t full_leader = map_to_cta(smem_u32(&s.full[st]), 0);
+                    if (rank == 0)                               // the bytes of both CTAs land on the leader's barrier
+                        mbar_expect_tx(smem_u32(&s.full[st]), static_cast<uint32_t>(2 * (BM + BN / 2) * BK * 2));
+                    tma_load_2d_pair(smem_u32(s.a[st]), &map_u, full_leader, kb * BK,
+                                     static_cast<int>(m0) + static_cast<int>(rank) * BM);
+                    tma_load_2d_pair(smem_u32(s.b[st]), &map_w, full_leader, kb * BK, n0 + static_cast<int>(rank) * (BN / 2));
+                }
+                if (!ok) { atomicExch(&g_timeout_flag, 8); break; }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
+                                   (static_cast<uint32_t>((2 * BM) >> 4) << 24);
+            uint32_t it = 0, local = 0;
+            bool ok = true;
+            for (long long tile = pair; tile < tiles && ok; tile += pairs, ++local) {
+                const uint32_t buf = local & 1;
+                if (!mbar_wait(smem_u32(&s.acc_empty[buf]), ((local >> 1) & 1) ^ 1)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t d_tmem = tmem + buf * kMaxBN;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int st = it % kPairStages;
+                    if (!mbar_wait(smem_u32(&s.full[st]), (it / kPairStages) & 1)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint64_t da = smem_desc(smem_u32(s.a[st])), db = smem_desc(smem_u32(s.b[st]));
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        umma_bf16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) ? 1u : 0u);
+                    umma_commit_pair(smem_u32(&s.empty[st]));          // frees the stage in both CTAs
+                }
+                umma_commit_pair(smem_u32(&s.acc_full[buf]));
+            }
+            if (!ok) atomicExch(&g_timeout_flag, 9);
+        }
+    } else {
+        const int quarter = warp & 3;
+        uint32_t local = 0;
+        for (long long tile = pair; tile < tiles; tile += pairs, ++local) {
+            const uint32_t buf = local & 1;
+            const int n0 = static_cast<int>(tile % n_tiles) * BN;
+            const long long row = (tile / n_tiles) * (2 * BM) + rank * BM + quarter * 32 + lane;
+            if (!mbar_wait(smem_u32(&s.acc_full[buf]), (local >> 1) & 1)) {
+                if (lane == 0) atomicExch(&g_timeout_flag, 10);
+                break;
+            }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                tmem_load_32(tmem + (static_cast<uint32_t>(quarter * 32) << 16) + buf * kMaxBN + c0, r);
+                if (row < M) {
+                    float* dst = out + row * N + n0 + c0;
+                    if (n0 + c0 + 32 <= N && (N & 3) == 0) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const float4 b4 = __ldg(reinterpret_cast<const float4*>(bias + n0 + c0 + j));
+                            *reinterpret_cast<float4*>(dst + j) =
+                                make_float4(__uint_as_float(r[j]) + b4.x, __uint_as_float(r[j + 1]) + b4.y,
+                                            __uint_as_float(r[j + 2]) + b4.z, __uint_as_float(r[j + 3]) + b4.w);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (n0 + c0 + j < N) dst[j] = __uint_as_float(r[j]) + __ldg(bias + n0 + c0 + j);
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&s.acc_empty[buf]), 0));
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    cluster_sync_all();                                          // neither CTA leaves while its peer may still signal it
+    if (warp == 2) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(2 * kMaxBN));
+}
+
 // fp32 storage: one thread per output, plain fp32 FMAs in channel order.
 __global__ void __launch_bounds__(256)
 offsets_linear_f32_kernel(const float* __restrict__ u, const float* __restrict__ w, const float* __restrict__ bias,
@@ -610,17 +743,46 @@ int dsa3d_offsets_linear_forward(const void* u, const void* w, const float* bias
     // column tiles of equal width, a multiple of 32 columns, at most 256
     const int n_tiles = (O + kMaxBN - 1) / kMaxBN;
     const int BN = ((O + n_tiles - 1) / n_tiles + 31) / 32 * 32;
-    const long long m_tiles = (tokens + BM - 1) / BM;
-    CUtensorMap map_u, map_w;
-    if (!make_map(&map_u, u, static_cast<unsigned long long>(tokens), static_cast<unsigned long long>(C), BM) ||
-        !make_map(&map_w, w, static_cast<unsigned long long>(O), static_cast<unsigned long long>(C),
-                  static_cast<unsigned>(BN)))
-        return DSA3D_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_failed(e);
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return cuda_failed(e);
+    CUtensorMap map_u, map_w;
+    const bool pair = sms >= 2 && !std::getenv("DSA3D_GEMM_ONE_CTA");     // pairs of CTAs unless switched off
+    if (pair) {
+        const long long m_tiles = (tokens + 2 * BM - 1) / (2 * BM);
+        if (!make_map(&map_u, u, static_cast<unsigned long long>(tokens), static_cast<unsigned long long>(C), BM) ||
+            !make_map(&map_w, w, static_cast<unsigned long long>(O), static_cast<unsigned long long>(C),
+                      static_cast<unsigned>(BN / 2)))
+            return DSA3D_ERR_UNSUPPORTED;
+        const size_t smem = sizeof(GemmPairSmem) + 1024;
+        e = cudaFuncSetAttribute(offsets_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem));
+        if (e != cudaSuccess) return cuda_failed(e);
+        const long long tiles = m_tiles * n_tiles;
+        const long long want = 2 * (tiles < sms / 2 ? tiles : sms / 2);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(want));
+        cfg.blockDim = dim3(kGemmThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, offsets_gemm_pair_kernel, map_u, map_w, bias, offsets, tokens, O, C, BN, m_tiles,
+                               n_tiles);
+        return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
+    }
+    const long long m_tiles = (tokens + BM - 1) / BM;
+    if (!make_map(&map_u, u, static_cast<unsigned long long>(tokens), static_cast<unsigned long long>(C), BM) ||
+        !make_map(&map_w, w, static_cast<unsigned long long>(O), static_cast<unsigned long long>(C),
+                  static_cast<unsigned>(BN)))
+        return DSA3D_ERR_UNSUPPORTED;
     const size_t smem = sizeof(GemmSmem) + 1024;
     e = cudaFuncSetAttribute(offsets_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return cuda_failed(e);

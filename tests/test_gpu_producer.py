@@ -64,9 +64,20 @@ def test_dwconv3d_staged_kernel_matches_the_oracle(shape, kernel):
     assert torch.equal(guard.cpu(), torch.full((64,), 3.0))
 
 
+@pytest.fixture(params=["pair", "one_cta"])
+def gemm_variant(request):
+    """Both tilings of the tensor-core linear layer: pairs of CTAs (the default) and one CTA
+    per tile (forced by an environment switch read at every call)."""
+    import os
+    if request.param == "one_cta":
+        os.environ["DSA3D_GEMM_ONE_CTA"] = "1"
+    yield request.param
+    os.environ.pop("DSA3D_GEMM_ONE_CTA", None)
+
+
 @pytest.mark.parametrize("tokens,C,O", [(300, 192, 162), (128, 64, 32), (1000, 256, 1296), (77, 200, 40),
                                         (513, 128, 520), (1, 8, 1), (260, 2048, 81)])
-def test_offsets_linear_bf16_on_tensor_cores(tokens, C, O):
+def test_offsets_linear_bf16_on_tensor_cores(tokens, C, O, gemm_variant):
     """Ragged token counts, channel counts that are not a multiple of the 64-channel stage
     (zero-filled by the tile loads), one to six column tiles of 32 to 256 columns.  The
     products are exact and the accumulation is fp32 in the tensor core's own order, so the
@@ -88,7 +99,7 @@ def test_offsets_linear_bf16_on_tensor_cores(tokens, C, O):
     assert torch.equal(guard.cpu(), torch.full((64,), 7.0))
 
 
-def test_offsets_linear_twice_in_a_row_and_large():
+def test_offsets_linear_twice_in_a_row_and_large(gemm_variant):
     """Two launches back to back on one stream (barrier phases and TMEM are per launch), on a
     problem with more tiles than SMs so that every CTA loops over several tiles and both
     accumulator buffers."""
