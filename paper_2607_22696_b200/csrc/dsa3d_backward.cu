@@ -418,12 +418,21 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                         const uint4 a = *reinterpret_cast<const uint4*>(my_rows + off);
                         const uint4 b = *reinterpret_cast<const uint4*>(my_rows + off + VPR * 16);
                         const unsigned aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+                        // two fp32 FMAs per instruction (fma.rn.f32x2): same arithmetic, fewer issue slots
+                        unsigned long long ckk, cvv;
+                        asm("mov.b64 %0, {%1, %1};" : "=l"(ckk) : "f"(ck));
+                        asm("mov.b64 %0, {%1, %1};" : "=l"(cvv) : "f"(cv));
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
-                            ak[2 * i] = fmaf(ck, __uint_as_float(aw[i] << 16), ak[2 * i]);
-                            ak[2 * i + 1] = fmaf(ck, __uint_as_float(aw[i] & 0xffff0000u), ak[2 * i + 1]);
-                            av[2 * i] = fmaf(cv, __uint_as_float(bw[i] << 16), av[2 * i]);
-                            av[2 * i + 1] = fmaf(cv, __uint_as_float(bw[i] & 0xffff0000u), av[2 * i + 1]);
+                            unsigned long long xa, xb, pa, pb;
+                            asm("mov.b64 %0, {%1, %2};" : "=l"(xa) : "r"(aw[i] << 16), "r"(aw[i] & 0xffff0000u));
+                            asm("mov.b64 %0, {%1, %2};" : "=l"(xb) : "r"(bw[i] << 16), "r"(bw[i] & 0xffff0000u));
+                            asm("mov.b64 %0, {%1, %2};" : "=l"(pa) : "f"(ak[2 * i]), "f"(ak[2 * i + 1]));
+                            asm("mov.b64 %0, {%1, %2};" : "=l"(pb) : "f"(av[2 * i]), "f"(av[2 * i + 1]));
+                            asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(pa) : "l"(ckk), "l"(xa));
+                            asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(pb) : "l"(cvv), "l"(xb));
+                            asm("mov.b64 {%0, %1}, %2;" : "=f"(ak[2 * i]), "=f"(ak[2 * i + 1]) : "l"(pa));
+                            asm("mov.b64 {%0, %1}, %2;" : "=f"(av[2 * i]), "=f"(av[2 * i + 1]) : "l"(pb));
                         }
                     }
                 }

@@ -80,6 +80,18 @@ template <int NV> struct Elt<float, NV> {
     }
 };
 
+// Two independent fp32 FMAs in one instruction (sm_100 fma.rn.f32x2): a0 += x0*y0, a1 += x1*y1,
+// each rounded exactly as fmaf would.  Pays where a loop is bound by issue slots and most of its
+// instructions are FMAs.
+__device__ __forceinline__ void fma2(float& a0, float& a1, float x0, float x1, float y0, float y1) {
+    unsigned long long acc, x, y;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(acc) : "f"(a0), "f"(a1));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(x) : "f"(x0), "f"(x1));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(y) : "f"(y0), "f"(y1));
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(x), "l"(y));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(acc));
+}
+
 __device__ __forceinline__ float fma_bf16(unsigned short a, unsigned short b, float c) {
     float d;
     asm("fma.rn.f32.bf16 %0, %1, %2, %3;" : "=f"(d) : "h"(a), "h"(b), "f"(c));

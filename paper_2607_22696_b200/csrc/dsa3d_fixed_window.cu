@@ -263,7 +263,8 @@ fixed_window_forward_kernel(const __grid_constant__ CUtensorMap map_q, const __g
                         const int qx = xx - ww;                   // the query whose window cell ww is position xx
                         if (qx < 0 || qx >= kFwTX) continue;
 #pragma unroll
-                        for (int e = 0; e < CPL; ++e) acc[qx][e] = fmaf(wq[qx * KW + ww], f[e], acc[qx][e]);
+                        for (int e = 0; e < CPL; e += 2)                  // two FMAs per instruction
+                            fma2(acc[qx][e], acc[qx][e + 1], wq[qx * KW + ww], wq[qx * KW + ww], f[e], f[e + 1]);
                     }
                 }
             }

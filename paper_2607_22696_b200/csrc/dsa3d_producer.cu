@@ -21,6 +21,7 @@
 #include <mutex>
 
 #include "../../include/dsa3d.h"
+#include "dsa3d_common.cuh"
 #include "dsa3d_kernels.h"
 #include "dsa3d_tcgen05.cuh"
 
