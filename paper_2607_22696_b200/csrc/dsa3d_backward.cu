@@ -165,10 +165,18 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
             const float alpha = exp2f(fmaf(sdot, scale * kLog2e, -lse2));
             const float ag = alpha * g;
             delta += ag;
+            if constexpr (NV == 2) {
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) {
-                u_acc[e] = fmaf(ag, kp[e], u_acc[e]);
-                kbar[e] = fmaf(alpha, kp[e], kbar[e]);
+                for (int e = 0; e < VEC; e += 2) {
+                    fma2(u_acc[e], u_acc[e + 1], ag, ag, kp[e], kp[e + 1]);
+                    fma2(kbar[e], kbar[e + 1], alpha, alpha, kp[e], kp[e + 1]);
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) {
+                    u_acc[e] = fmaf(ag, kp[e], u_acc[e]);
+                    kbar[e] = fmaf(alpha, kp[e], kbar[e]);
+                }
             }
             float* sts = stats + (pb + j) * kStats;
             if constexpr (LPR >= 8) {
