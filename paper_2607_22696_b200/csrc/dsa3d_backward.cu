@@ -277,6 +277,9 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     uint4* rows = reinterpret_cast<uint4*>(smem_raw);                                   // [TQ][2][VPR]
     unsigned* cursor = reinterpret_cast<unsigned*>(smem_raw + static_cast<size_t>(TQ) * kPairBytes);   // [NB]
     __shared__ unsigned warp_sums[kTileThreads / 32];
+#ifndef DSA3D_BF16_COEF
+    __shared__ uint4 ent_stage[kTileThreads];          // one entry per lane, read back by every lane of its group
+#endif
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kWarps = kTileThreads / 32;
@@ -395,7 +398,7 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
             constexpr int GW = VPR;                          // lanes per key row
             constexpr int kGroups = 32 / GW;
             const int grp = lane / GW, hl = lane & (GW - 1);
-            const int lane0 = lane & ~(GW - 1);              // first lane of this group
+            [[maybe_unused]] const int lane0 = lane & ~(GW - 1);              // first lane of this group
             const unsigned char* my_rows = smem_raw + hl * 16;
             for (int firstbin = warp * kGroups; firstbin < NB; firstbin += kWarps * kGroups) {
                 const int bin = firstbin + grp;
@@ -417,12 +420,17 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                     uint4 ent = make_uint4(0u, 0u, 0u, 0u);               // offset 0, coefficients 0
                     if (base + hl < cnt_mine) ent = __ldcg(my_scratch + start + base + hl);
                     const int steps = static_cast<int>(min(static_cast<unsigned>(GW), cnt_max - base));
+                    // the group's entries go through shared memory: one broadcast read per step
+                    // instead of three shuffles
+                    __syncwarp();
+                    ent_stage[tid] = ent;
+                    __syncwarp();
+                    const uint4* grp_ent = ent_stage + (tid & ~(GW - 1));
 #pragma unroll 4
                     for (int j = 0; j < steps; ++j) {
-                        const int src = lane0 | j;
-                        const unsigned off = __shfl_sync(kFull, ent.x, src);
-                        const float ck = __uint_as_float(__shfl_sync(kFull, ent.y, src));
-                        const float cv = __uint_as_float(__shfl_sync(kFull, ent.z, src));
+                        const uint4 ej = grp_ent[j];
+                        const unsigned off = ej.x;
+                        const float ck = __uint_as_float(ej.y), cv = __uint_as_float(ej.z);
                         const uint4 a = *reinterpret_cast<const uint4*>(my_rows + off);
                         const uint4 b = *reinterpret_cast<const uint4*>(my_rows + off + VPR * 16);
                         const unsigned aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
