@@ -51,3 +51,40 @@ def offsets_linear(u: torch.Tensor, w: torch.Tensor, bias) -> torch.Tensor:
     if bias is not None:
         out = out + bias.to(torch.float64)
     return out
+
+
+def dwconv3d_backward(x: torch.Tensor, weight: torch.Tensor, dy: torch.Tensor, kernel):
+    """Gradients of L = sum(dy * dwconv3d(x, weight, bias)) with respect to x, weight and
+    bias, written from the definition: tap (i, j, l) couples output position s with input
+    position s + disp, so dx[s + disp] += w[tap] * dy[s], dw[tap] = sum_s x[s + disp] * dy[s]
+    over the output positions whose displaced position lies inside the grid, and
+    dbias[c] = sum_s dy[s, c].  Returns fp64 (dx [T, H, W, C], dw [taps, C], dbias [C])."""
+    kt, kh, kw = (int(s) for s in kernel)
+    T, H, W, C = x.shape
+    xd = x.to(torch.float64)
+    wd = weight.to(torch.float64)
+    g = dy.to(torch.float64)
+    dx = torch.zeros(T, H, W, C, dtype=torch.float64)
+    dw = torch.zeros(kt * kh * kw, C, dtype=torch.float64)
+    for i in range(kt):
+        for j in range(kh):
+            for l in range(kw):
+                dt, dyy, dxx = i - kt // 2, j - kh // 2, l - kw // 2
+                t0, t1 = max(0, -dt), min(T, T - dt)
+                y0, y1 = max(0, -dyy), min(H, H - dyy)
+                x0, x1 = max(0, -dxx), min(W, W - dxx)
+                if t0 >= t1 or y0 >= y1 or x0 >= x1:
+                    continue
+                tap = (i * kh + j) * kw + l
+                gs = g[t0:t1, y0:y1, x0:x1]
+                dx[t0 + dt:t1 + dt, y0 + dyy:y1 + dyy, x0 + dxx:x1 + dxx] += wd[tap] * gs
+                dw[tap] = (xd[t0 + dt:t1 + dt, y0 + dyy:y1 + dyy, x0 + dxx:x1 + dxx] * gs).sum(dim=(0, 1, 2))
+    return dx, dw, g.sum(dim=(0, 1, 2))
+
+
+def offsets_linear_backward(u: torch.Tensor, w: torch.Tensor, doffsets: torch.Tensor):
+    """Gradients of L = sum(doffsets * offsets_linear(u, w, bias)): du[n, c] = sum_o
+    doffsets[n, o] w[o, c]; dw[o, c] = sum_n doffsets[n, o] u[n, c]; dbias[o] = sum_n
+    doffsets[n, o].  Returns fp64 (du [N, C], dw [O, C], dbias [O])."""
+    g = doffsets.to(torch.float64)
+    return g @ w.to(torch.float64), g.t() @ u.to(torch.float64), g.sum(dim=0)
