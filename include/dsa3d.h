@@ -247,6 +247,44 @@ int dsa3d_dwconv3d_forward(const void* x, const float* weight, const float* bias
 int dsa3d_offsets_linear_forward(const void* u, const void* w, const float* bias, long long tokens, int C, int O,
                                  float* offsets, int dtype, void* stream);
 
+/*
+ * Backward of the two layers above (gradients of a scalar loss L; the paper gives no formulas
+ * for them: they follow from the definitions of the two forwards by the chain rule).
+ *
+ * dsa3d_dwconv3d_backward: with dy = dL/dy [T,H,W,C] in `dtype`,
+ *   dx[s]        = sum over taps of weight[tap][c] * dy[s - displacement(tap)]   ([T,H,W,C], `dtype`),
+ *   dweight[tap] = sum over positions s of x[s + displacement(tap)] * dy[s]      (fp32 [kt*kh*kw, C]),
+ *   dbias[c]     = sum over positions of dy[s][c]                                 (fp32 [C]),
+ * zero outside the grid as in the forward.  dx, dweight and dbias may each be NULL (not
+ * computed; dbias needs dweight); x is read only for dweight, weight only for dx.  dx is one
+ * fp32 accumulation in tap order and one rounding; dweight and dbias are fp32 sums whose order
+ * varies from run to run (atomic adds of per-warp partial sums).  workspace: device memory of
+ * dsa3d_dwconv3d_backward_workspace_bytes(C, kernel) bytes (needed for dx only), contents
+ * undefined afterwards.  dx must not alias dy.
+ */
+size_t dsa3d_dwconv3d_backward_workspace_bytes(int C, const int kernel[3]);
+int dsa3d_dwconv3d_backward(const void* x, const float* weight, const void* dy, int T, int H, int W, int C,
+                            const int kernel[3], void* dx, float* dweight, float* dbias, void* workspace,
+                            size_t workspace_bytes, int dtype, void* stream);
+
+/*
+ * dsa3d_offsets_linear_backward: with doffsets = dL/doffsets (fp32 [tokens, O], e.g. the
+ * doffsets of dsa3d_backward),
+ *   du[n][c] = sum_o doffsets[n][o] * w[o][c]     ([tokens, C] in `dtype`),
+ *   dw[o][c] = sum_n doffsets[n][o] * u[n][c]     (fp32 [O, C]),
+ *   dbias[o] = sum_n doffsets[n][o]               (fp32 [O]).
+ * Each output may be NULL (not computed).  bf16: doffsets is rounded to bf16 once and both
+ * contractions run on the tensor cores with fp32 accumulation (slabs of 262144 tokens, dw
+ * accumulated over slabs and k-ranges with fp32 atomic adds, so its summation order varies);
+ * dbias is summed from the fp32 doffsets.  fp32: plain fp32 FMAs.  workspace: device memory of
+ * dsa3d_offsets_linear_backward_workspace_bytes(...) bytes (0 for fp32), contents undefined
+ * afterwards.  Bounded waits as in the forward (dsa3d_device_timeout_flag).
+ */
+size_t dsa3d_offsets_linear_backward_workspace_bytes(long long tokens, int C, int O, int dtype);
+int dsa3d_offsets_linear_backward(const void* u, const void* w, const float* doffsets, long long tokens, int C, int O,
+                                  void* du, float* dw, float* dbias, void* workspace, size_t workspace_bytes, int dtype,
+                                  void* stream);
+
 /* Synchronises with the device and returns the flag described above (0: no wait ever ran
  * out; -1: the flag could not be read). */
 int dsa3d_device_timeout_flag(void);

@@ -73,6 +73,14 @@ def load():
     lib.dsa3d_dwconv3d_forward.argtypes = [p, p, p, i, i, i, i, win, p, i, p]
     lib.dsa3d_offsets_linear_forward.restype = i
     lib.dsa3d_offsets_linear_forward.argtypes = [p, p, p, ctypes.c_longlong, i, i, p, i, p]
+    lib.dsa3d_dwconv3d_backward.restype = i
+    lib.dsa3d_dwconv3d_backward.argtypes = [p, p, p, i, i, i, i, win, p, p, p, p, sz, i, p]
+    lib.dsa3d_dwconv3d_backward_workspace_bytes.restype = sz
+    lib.dsa3d_dwconv3d_backward_workspace_bytes.argtypes = [i, win]
+    lib.dsa3d_offsets_linear_backward.restype = i
+    lib.dsa3d_offsets_linear_backward.argtypes = [p, p, p, ctypes.c_longlong, i, i, p, p, p, p, sz, i, p]
+    lib.dsa3d_offsets_linear_backward_workspace_bytes.restype = sz
+    lib.dsa3d_offsets_linear_backward_workspace_bytes.argtypes = [ctypes.c_longlong, i, i, i]
     lib.dsa3d_device_timeout_flag.restype = i
     lib.dsa3d_device_timeout_flag.argtypes = []
     lib.dsa3d_forward_residual.restype = i
@@ -226,6 +234,49 @@ def dsa3d_offsets_linear_forward(u, w, bias, tokens, C, O, offsets, dtype=None, 
     _check(lib.dsa3d_offsets_linear_forward(
         _ptr(u, "u", tokens * C), _ptr(w, "w", O * C), _ptr(bias, "bias", O, torch.float32), tokens, C, O,
         _ptr(offsets, "offsets", tokens * O, torch.float32), code, _stream(stream)))
+
+
+def _nbytes(t: Optional[torch.Tensor]) -> int:
+    return 0 if t is None else t.numel() * t.element_size()
+
+
+def dsa3d_dwconv3d_backward_workspace_bytes(C, kernel) -> int:
+    return int(load().dsa3d_dwconv3d_backward_workspace_bytes(C, _window(kernel)))
+
+
+def dsa3d_dwconv3d_backward(x, weight, dy, T, H, W, C, kernel, dx, dweight, dbias, workspace, dtype=None,
+                            stream=None) -> None:
+    """dx, dweight, dbias <- gradients of the depthwise convolution (each may be None); see
+    include/dsa3d.h."""
+    lib = load()
+    dt = dy.dtype if dtype is None else dtype
+    code = _DTYPES[dt] if isinstance(dt, torch.dtype) else int(dt)
+    taps = int(kernel[0]) * int(kernel[1]) * int(kernel[2])
+    n = T * H * W * C
+    _check(lib.dsa3d_dwconv3d_backward(
+        _ptr(x, "x", n), _ptr(weight, "weight", taps * C, torch.float32), _ptr(dy, "dy", n), T, H, W, C,
+        _window(kernel), _ptr(dx, "dx", n), _ptr(dweight, "dweight", taps * C, torch.float32),
+        _ptr(dbias, "dbias", C, torch.float32), _ptr(workspace, "workspace"), _nbytes(workspace), code,
+        _stream(stream)))
+
+
+def dsa3d_offsets_linear_backward_workspace_bytes(tokens, C, O, dtype) -> int:
+    code = _DTYPES[dtype] if isinstance(dtype, torch.dtype) else int(dtype)
+    return int(load().dsa3d_offsets_linear_backward_workspace_bytes(tokens, C, O, code))
+
+
+def dsa3d_offsets_linear_backward(u, w, doffsets, tokens, C, O, du, dw, dbias, workspace, dtype=None,
+                                  stream=None) -> None:
+    """du, dw, dbias <- gradients of the offset-producing linear layer (each may be None);
+    see include/dsa3d.h."""
+    lib = load()
+    dt = (u if u is not None else w).dtype if dtype is None else dtype
+    code = _DTYPES[dt] if isinstance(dt, torch.dtype) else int(dt)
+    _check(lib.dsa3d_offsets_linear_backward(
+        _ptr(u, "u", tokens * C), _ptr(w, "w", O * C), _ptr(doffsets, "doffsets", tokens * O, torch.float32),
+        tokens, C, O, _ptr(du, "du", tokens * C), _ptr(dw, "dw", O * C, torch.float32),
+        _ptr(dbias, "dbias", O, torch.float32), _ptr(workspace, "workspace"), _nbytes(workspace), code,
+        _stream(stream)))
 
 
 def dsa3d_device_timeout_flag() -> int:

@@ -94,7 +94,7 @@ template <> struct Vec8<float> {
 template <typename T, int KW>
 __global__ void __launch_bounds__(256)
 dwconv3d_kernel(const T* __restrict__ x, const float* __restrict__ weight, const float* __restrict__ bias,
-                T* __restrict__ y, int Tn, int H, int W, int C, int kt, int kh, int kw_rt) {
+                T* __restrict__ y, int Tn, int H, int W, int C, int kt, int kh, int kw_rt, int ct, int chh, int cw) {
     const int kw = KW > 0 ? KW : kw_rt;
     const int cvecs = C / 8;
     const int xruns = (W + kConvRX - 1) / kConvRX;
@@ -115,10 +115,10 @@ dwconv3d_kernel(const T* __restrict__ x, const float* __restrict__ weight, const
         for (int e = 0; e < 8; ++e) acc[r][e] = bias ? __ldg(bias + c0 + e) : 0.0f;
 
     for (int i = 0; i < kt; ++i) {
-        const int st = tt + i - kt / 2;
+        const int st = tt + i - ct;
         if (st < 0 || st >= Tn) continue;
         for (int j = 0; j < kh; ++j) {
-            const int sy = yy + j - kh / 2;
+            const int sy = yy + j - chh;
             if (sy < 0 || sy >= H) continue;
             const T* row = x + (static_cast<long long>(st) * H + sy) * W * C + c0;
             const float* wrow = weight + static_cast<long long>((i * kh + j) * kw) * C + c0;
@@ -136,7 +136,7 @@ dwconv3d_kernel(const T* __restrict__ x, const float* __restrict__ weight, const
                 typename Vec8<T>::Raw raw[KW + kConvRX - 1];
 #pragma unroll
                 for (int s = 0; s < KW + kConvRX - 1; ++s) {
-                    const int sx = x0 + s - KW / 2;
+                    const int sx = x0 + s - cw;
                     raw[s] = (sx >= 0 && sx < W) ? Vec8<T>::load_raw(row + static_cast<long long>(sx) * C)
                                                  : Vec8<T>::zero_raw();
                 }
@@ -154,7 +154,7 @@ dwconv3d_kernel(const T* __restrict__ x, const float* __restrict__ weight, const
                 }
             } else {
                 for (int s = 0; s < kw + kConvRX - 1; ++s) {
-                    const int sx = x0 + s - kw / 2;
+                    const int sx = x0 + s - cw;
                     if (sx < 0 || sx >= W) continue;
                     float in[8];
                     Vec8<T>::load(row + static_cast<long long>(sx) * C, in);
@@ -181,17 +181,19 @@ dwconv3d_kernel(const T* __restrict__ x, const float* __restrict__ weight, const
 
 template <typename T>
 void launch_dwconv(const void* x, const float* weight, const float* bias, void* y, int T_, int H, int W, int C,
-                   const int kernel[3], unsigned blocks, cudaStream_t st) {
+                   const int kernel[3], const int centre[3], unsigned blocks, cudaStream_t st) {
     const T* xp = static_cast<const T*>(x);
     T* yp = static_cast<T*>(y);
 #define DSA3D_CONV_CASE(KW) \
-    case KW: dwconv3d_kernel<T, KW><<<blocks, 256, 0, st>>>(xp, weight, bias, yp, T_, H, W, C, kernel[0], kernel[1], KW); break;
+    case KW: dwconv3d_kernel<T, KW><<<blocks, 256, 0, st>>>(xp, weight, bias, yp, T_, H, W, C, kernel[0], kernel[1], KW, \
+                                                            centre[0], centre[1], centre[2]); break;
     switch (kernel[2]) {
         DSA3D_CONV_CASE(1)
         DSA3D_CONV_CASE(3)
         DSA3D_CONV_CASE(5)
         DSA3D_CONV_CASE(7)
-        default: dwconv3d_kernel<T, 0><<<blocks, 256, 0, st>>>(xp, weight, bias, yp, T_, H, W, C, kernel[0], kernel[1], kernel[2]);
+        default: dwconv3d_kernel<T, 0><<<blocks, 256, 0, st>>>(xp, weight, bias, yp, T_, H, W, C, kernel[0], kernel[1], kernel[2],
+                                                               centre[0], centre[1], centre[2]);
     }
 #undef DSA3D_CONV_CASE
 }
@@ -332,7 +334,7 @@ template <int KW>
 __global__ void __launch_bounds__(kCvThreads)
 dwconv3d_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* __restrict__ weight,
                     const float* __restrict__ bias, __nv_bfloat16* __restrict__ y, int Tn, int H, int W, int C,
-                    int kt, int kh, int t_chunk) {
+                    int kt, int kh, int t_chunk, int ct, int chh, int cw) {
     extern __shared__ unsigned char raw_smem[];
     unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(raw_smem) + 127) & ~uintptr_t(127));
     const int ring = kt + 1;
@@ -347,7 +349,7 @@ dwconv3d_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* __re
     const int tiles_x = (W + kCvTX - 1) / kCvTX;
     const int x0 = (blockIdx.y % tiles_x) * kCvTX, y0 = (blockIdx.y / tiles_x) * kCvTY;
     const int t_begin = blockIdx.z * t_chunk, t_end = min(Tn, t_begin + t_chunk);
-    const int lo = kt / 2;                                              // planes t-lo .. t-lo+kt-1 feed output t
+    const int lo = ct;                                                  // planes t-lo .. t-lo+kt-1 feed output t
 
     // per tap: the first four channels of every 8-channel vector, then the last four, so that
     // the 8 lanes of a quarter-warp read 128 contiguous bytes (no bank conflicts)
@@ -367,7 +369,7 @@ dwconv3d_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* __re
         const int p = t_begin - lo + n, slot = n % ring;
         mbar_expect_tx(smem_u32(&bars[slot]), plane_bytes);
         tma_load_4d(smem_u32(base + static_cast<size_t>(slot) * plane_bytes), &map_x, smem_u32(&bars[slot]), c0,
-                    x0 - KW / 2, y0 - kh / 2, p);
+                    x0 - cw, y0 - chh, p);
     };
     if (tid == 0)
         for (int n = 0; n < kt; ++n) issue(n);
@@ -445,6 +447,8 @@ dwconv3d_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* __re
 // takes the operand stream under the 64 B/clk an SM can pull from L2 (the one-CTA tiling needs
 // 93 B/clk at full tensor rate).
 constexpr int kPairStages = 6;
+// what the epilogue does with the fp32 accumulators: out = acc + bias in fp32; out = acc in bf16; out += acc
+constexpr int kGemmStoreF32 = 0, kGemmStoreBf16 = 1, kGemmAddF32 = 2;
 struct __align__(1024) GemmPairSmem {
     __nv_bfloat16 a[kPairStages][BM * BK];
     __nv_bfloat16 b[kPairStages][(kMaxBN / 2) * BK];
@@ -454,14 +458,21 @@ struct __align__(1024) GemmPairSmem {
 
 __global__ void __launch_bounds__(kGemmThreads, 1)
 offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_constant__ CUtensorMap map_w,
-                         const float* __restrict__ bias, float* __restrict__ out, long long M, int N, int K, int BN,
-                         long long m_tiles, int n_tiles) {
+                         const float* __restrict__ bias, void* __restrict__ out_raw, long long M, int N, int K, int BN,
+                         long long m_tiles, int n_tiles, int mode, int ksplits) {
     extern __shared__ unsigned char raw[];
     GemmPairSmem& s = *reinterpret_cast<GemmPairSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_rank();                       // 0: leader (issues the MMAs)
     const int kblocks = (K + BK - 1) / BK;
-    const long long tiles = m_tiles * n_tiles;                  // m_tiles counts 256-row tiles here
+    // a work unit is one 256 x BN output tile (m_tiles counts 256-row tiles) times one of
+    // `ksplits` equal ranges of k-blocks; units of a tile are neighbours so they share operands in L2
+    const long long tiles = m_tiles * n_tiles * ksplits;
+    auto k_range = [&](long long unit, int& kb0, int& kb1) {
+        const int ks = static_cast<int>(unit % ksplits);
+        kb0 = static_cast<int>(static_cast<long long>(kblocks) * ks / ksplits);
+        kb1 = static_cast<int>(static_cast<long long>(kblocks) * (ks + 1) / ksplits);
+    };
     const long long pair = blockIdx.x / 2, pairs = gridDim.x / 2;
 
     if (threadIdx.x == 0) {
@@ -484,11 +495,14 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
     if (warp == 0) {
         if (lane == 0) {
             uint32_t it = 0;
-            for (long long tile = pair; tile < tiles; tile += pairs) {
+            for (long long unit = pair; unit < tiles; unit += pairs) {
+                const long long tile = unit / ksplits;
                 const int n0 = static_cast<int>(tile % n_tiles) * BN;
                 const long long m0 = (tile / n_tiles) * (2 * BM);
+                int kb0, kb1;
+                k_range(unit, kb0, kb1);
                 bool ok = true;
-                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const int st = it % kPairStages;
                     if (!mbar_wait(smem_u32(&s.empty[st]), ((it / kPairStages) & 1) ^ 1)) { ok = false; break; }
                     const uint32_t full_leader = map_to_cta(smem_u32(&s.full[st]), 0);
@@ -507,19 +521,21 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
                                    (static_cast<uint32_t>((2 * BM) >> 4) << 24);
             uint32_t it = 0, local = 0;
             bool ok = true;
-            for (long long tile = pair; tile < tiles && ok; tile += pairs, ++local) {
+            for (long long unit = pair; unit < tiles && ok; unit += pairs, ++local) {
                 const uint32_t buf = local & 1;
+                int kb0, kb1;
+                k_range(unit, kb0, kb1);
                 if (!mbar_wait(smem_u32(&s.acc_empty[buf]), ((local >> 1) & 1) ^ 1)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem + buf * kMaxBN;
-                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const int st = it % kPairStages;
                     if (!mbar_wait(smem_u32(&s.full[st]), (it / kPairStages) & 1)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint64_t da = smem_desc(smem_u32(s.a[st])), db = smem_desc(smem_u32(s.b[st]));
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)
-                        umma_bf16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) ? 1u : 0u);
+                        umma_bf16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, ((kb - kb0) | k) ? 1u : 0u);
                     umma_commit_pair(smem_u32(&s.empty[st]));          // frees the stage in both CTAs
                 }
                 umma_commit_pair(smem_u32(&s.acc_full[buf]));
@@ -529,8 +545,9 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
     } else {
         const int quarter = warp & 3;
         uint32_t local = 0;
-        for (long long tile = pair; tile < tiles; tile += pairs, ++local) {
+        for (long long unit = pair; unit < tiles; unit += pairs, ++local) {
             const uint32_t buf = local & 1;
+            const long long tile = unit / ksplits;
             const int n0 = static_cast<int>(tile % n_tiles) * BN;
             const long long row = (tile / n_tiles) * (2 * BM) + rank * BM + quarter * 32 + lane;
             if (!mbar_wait(smem_u32(&s.acc_full[buf]), (local >> 1) & 1)) {
@@ -541,12 +558,15 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
                 tmem_load_32(tmem + (static_cast<uint32_t>(quarter * 32) << 16) + buf * kMaxBN + c0, r);
-                if (row < M) {
-                    float* dst = out + row * N + n0 + c0;
-                    if (n0 + c0 + 32 <= N && (N & 3) == 0) {
+                if (row >= M) continue;
+                const bool whole = n0 + c0 + 32 <= N;
+                if (mode == kGemmStoreF32) {
+                    float* dst = static_cast<float*>(out_raw) + row * N + n0 + c0;
+                    if (whole && (N & 3) == 0) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
-                            const float4 b4 = __ldg(reinterpret_cast<const float4*>(bias + n0 + c0 + j));
+                            const float4 b4 = bias ? __ldg(reinterpret_cast<const float4*>(bias + n0 + c0 + j))
+                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
                             *reinterpret_cast<float4*>(dst + j) =
                                 make_float4(__uint_as_float(r[j]) + b4.x, __uint_as_float(r[j + 1]) + b4.y,
                                             __uint_as_float(r[j + 2]) + b4.z, __uint_as_float(r[j + 3]) + b4.w);
@@ -554,7 +574,40 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
-                            if (n0 + c0 + j < N) dst[j] = __uint_as_float(r[j]) + __ldg(bias + n0 + c0 + j);
+                            if (n0 + c0 + j < N) dst[j] = __uint_as_float(r[j]) + (bias ? __ldg(bias + n0 + c0 + j) : 0.0f);
+                    }
+                } else if (mode == kGemmStoreBf16) {
+                    __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(out_raw) + row * N + n0 + c0;
+                    if (whole && (N & 7) == 0) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[j + 2 * e]),
+                                                                               __uint_as_float(r[j + 2 * e + 1]));
+                                w[e] = *reinterpret_cast<const uint32_t*>(&h);
+                            }
+                            *reinterpret_cast<uint4*>(dst + j) = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (n0 + c0 + j < N) dst[j] = __float2bfloat16_rn(__uint_as_float(r[j]));
+                    }
+                } else {                                     // kGemmAddF32: partial sums of a k-range
+                    float* dst = static_cast<float*>(out_raw) + row * N + n0 + c0;
+                    if (whole && (N & 3) == 0) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + j),
+                                         "f"(__uint_as_float(r[j])), "f"(__uint_as_float(r[j + 1])),
+                                         "f"(__uint_as_float(r[j + 2])), "f"(__uint_as_float(r[j + 3]))
+                                         : "memory");
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (n0 + c0 + j < N) atomicAdd(dst + j, __uint_as_float(r[j]));
                     }
                 }
             }
@@ -603,16 +656,56 @@ EncodeTiledFn encode_tiled() {
 
 // Row-major [rows, cols] bf16 matrix, tiles of box_rows x 64 columns, 128-byte swizzle, zero fill
 // outside the matrix.
-bool make_map(CUtensorMap* map, const void* ptr, unsigned long long rows, unsigned long long cols, unsigned box_rows) {
+bool make_map(CUtensorMap* map, const void* ptr, unsigned long long rows, unsigned long long cols, unsigned box_rows,
+              unsigned long long ld = 0) {
     EncodeTiledFn enc = encode_tiled();
     if (!enc) return false;
     const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint64_t strides[1] = {(ld ? ld : cols) * 2};          // row pitch in bytes (a multiple of 16)
     const cuuint32_t box[2] = {BK, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// out[M, N] = A[M, K] . B[N, K]^T on pairs of CTAs; A and B row-major bf16 with row pitches lda, ldb
+// (elements, multiples of 8).  mode: what the epilogue does; ksplits: equal ranges of k-blocks per
+// output tile (> 1 only with kGemmAddF32).  Column tiles of equal width, a multiple of 32, at most 256.
+cudaError_t launch_pair_gemm(const void* A, unsigned long long lda, const void* B, unsigned long long ldb,
+                             const float* bias, void* out, long long M, int N, int K, int mode, int ksplits, int sms,
+                             cudaStream_t st, bool* unsupported) {
+    *unsupported = false;
+    const int n_tiles = (N + kMaxBN - 1) / kMaxBN;
+    const int BN = ((N + n_tiles - 1) / n_tiles + 31) / 32 * 32;
+    const long long m_tiles = (M + 2 * BM - 1) / (2 * BM);
+    CUtensorMap map_a, map_b;
+    if (!make_map(&map_a, A, static_cast<unsigned long long>(M), static_cast<unsigned long long>(K), BM, lda) ||
+        !make_map(&map_b, B, static_cast<unsigned long long>(N), static_cast<unsigned long long>(K),
+                  static_cast<unsigned>(BN / 2), ldb)) {
+        *unsupported = true;
+        return cudaSuccess;
+    }
+    const size_t smem = sizeof(GemmPairSmem) + 1024;
+    cudaError_t e = cudaFuncSetAttribute(offsets_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    const long long units = m_tiles * n_tiles * ksplits;
+    const long long want = 2 * (units < sms / 2 ? units : sms / 2);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(want));
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, offsets_gemm_pair_kernel, map_a, map_b, bias, out, M, N, K, BN, m_tiles, n_tiles, mode,
+                              ksplits);
 }
 
 // Channels-last activations [T, H, W, C] bf16 as a 4-D map with boxes of 64 channels x pw x ph x 1.
@@ -633,7 +726,7 @@ bool make_map_activations(CUtensorMap* map, const void* ptr, int T, int H, int W
 // Launch the staged kernel if the shape suits it; returns false when the caller should use the
 // plain kernel instead (fp32, odd channel counts, wide kernels).  *err receives a launch error.
 bool try_dwconv_tma(const void* x, const float* weight, const float* bias, void* y, int T, int H, int W, int C,
-                    const int kernel[3], cudaStream_t st, cudaError_t* err) {
+                    const int kernel[3], const int centre[3], cudaStream_t st, cudaError_t* err) {
     *err = cudaSuccess;
     const int kt = kernel[0], kh = kernel[1], kw = kernel[2];
     if (C % kCvCh || kt > kCvMaxKt || (kw != 1 && kw != 3 && kw != 5 && kw != 7)) return false;
@@ -659,7 +752,8 @@ bool try_dwconv_tma(const void* x, const float* weight, const float* bias, void*
                                     static_cast<int>(smem));                                                       \
         if (*err == cudaSuccess) {                                                                                 \
             dwconv3d_tma_kernel<KW><<<grid, kCvThreads, smem, st>>>(map, weight, bias, static_cast<__nv_bfloat16*>(y), \
-                                                                    T, H, W, C, kt, kh, t_chunk);                  \
+                                                                    T, H, W, C, kt, kh, t_chunk, centre[0],        \
+                                                                    centre[1], centre[2]);                         \
             *err = cudaGetLastError();                                                                             \
         }                                                                                                          \
         break;
@@ -671,6 +765,230 @@ bool try_dwconv_tma(const void* x, const float* weight, const float* bias, void*
     }
 #undef DSA3D_CONV_TMA_CASE
     return true;
+}
+
+
+// ------------------------------------------------------------------------------------------
+// Backward of the two layers.
+//   convolution:  dx = correlation of dy with the flipped kernel (the same kernels as the
+//                 forward, centre kt-1-kt/2 etc.); dweight[tap, c] = sum_s x[s + disp] dy[s, c]
+//                 and dbias by dwconv3d_wgrad_kernel.
+//   linear layer: du = doffsets . w and dw = doffsets^T . u as two tensor-core contractions
+//                 (bf16 operands: doffsets is rounded to bf16 once, w and u are transposed
+//                 copies so that every operand is K-major), token slab by token slab; dbias
+//                 from the fp32 doffsets.
+// ------------------------------------------------------------------------------------------
+__global__ void flip_weight_kernel(const float* __restrict__ w, float* __restrict__ wf, int taps, int C) {
+    const long long id = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (id >= static_cast<long long>(taps) * C) return;
+    const int tap = static_cast<int>(id / C), c = static_cast<int>(id % C);
+    wf[static_cast<long long>(taps - 1 - tap) * C + c] = w[id];
+}
+
+template <typename T> struct Pair2;
+template <> struct Pair2<__nv_bfloat16> {
+    static __device__ __forceinline__ float2 load(const __nv_bfloat16* p) {
+        const uint32_t r = __ldg(reinterpret_cast<const uint32_t*>(p));
+        return make_float2(__uint_as_float(r << 16), __uint_as_float(r & 0xffff0000u));
+    }
+};
+template <> struct Pair2<float> {
+    static __device__ __forceinline__ float2 load(const float* p) { return __ldg(reinterpret_cast<const float2*>(p)); }
+};
+
+// One warp per (kernel row (i, j), chunk of grid rows); lane = a pair of neighbouring channels
+// of a 64-channel group.  The warp marches along x over the input columns of its rows: one x
+// vector per column feeds the kw taps of the kernel row against a sliding window of kw dy
+// vectors held in registers.  The partial sums of a warp go to dweight with one atomic per
+// (tap, channel); warps of a block are the kernel rows of the same grid rows, so they share
+// their loads through L1.
+constexpr int kWgradRows = 32;                  // grid rows (t, y) per warp
+template <typename T, int KW>
+__global__ void __launch_bounds__(1024)
+dwconv3d_wgrad_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ dweight,
+                      float* __restrict__ dbias, int Tn, int H, int W, int C, int kt, int kh, int kw_rt) {
+    constexpr int MAXW = KW > 0 ? KW : kConvMaxKw;
+    const int kw = KW > 0 ? KW : kw_rt;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
+    const int c = blockIdx.x * 64 + lane * 2;
+    if (c >= C) return;                                    // C is even: a pair is inside or outside
+    const long long rows = static_cast<long long>(Tn) * H;
+    const long long r0 = static_cast<long long>(blockIdx.y) * kWgradRows;
+    const long long r1 = r0 + kWgradRows < rows ? r0 + kWgradRows : rows;
+    const int ct = kt / 2, chh = kh / 2, cw = kw / 2;
+
+    for (int ij = warp; ij < kt * kh; ij += warps) {
+        const int i = ij / kh, j = ij % kh;
+        float2 acc[MAXW];
+#pragma unroll
+        for (int l = 0; l < MAXW; ++l) acc[l] = make_float2(0.f, 0.f);
+        float2 bsum = make_float2(0.f, 0.f);
+        for (long long r = r0; r < r1; ++r) {
+            const int tt = static_cast<int>(r / H), yy = static_cast<int>(r % H);
+            const T* gy = dy + r * W * C + c;
+            if (ij == 0 && dbias)
+                for (int ox = 0; ox < W; ++ox) {
+                    const float2 g = Pair2<T>::load(gy + static_cast<long long>(ox) * C);
+                    bsum.x += g.x;
+                    bsum.y += g.y;
+                }
+            const int st = tt + i - ct, sy = yy + j - chh;
+            if (st < 0 || st >= Tn || sy < 0 || sy >= H) continue;
+            const T* xr = x + (static_cast<long long>(st) * H + sy) * W * C + c;
+            // window[l] = dy at output column sx + cw - l (zero outside the row)
+            float2 win[MAXW];
+#pragma unroll
+            for (int l = 0; l < MAXW; ++l) win[l] = make_float2(0.f, 0.f);
+            // before input column 0: outputs cw-l for l = 1 .. (shifted in below)
+#pragma unroll
+            for (int l = 1; l < MAXW; ++l) {
+                const int ox = cw - l;                      // output column seen by tap l at sx = 0, minus the shift
+                if (l < kw && ox >= 0 && ox < W) win[l] = Pair2<T>::load(gy + static_cast<long long>(ox) * C);
+            }
+            for (int sx = 0; sx < W; ++sx) {
+                const int ox0 = sx + cw;                    // newest output column (tap 0)
+                win[0] = (ox0 < W) ? Pair2<T>::load(gy + static_cast<long long>(ox0) * C) : make_float2(0.f, 0.f);
+                const float2 xv = Pair2<T>::load(xr + static_cast<long long>(sx) * C);
+#pragma unroll
+                for (int l = 0; l < MAXW; ++l) {
+                    acc[l].x = fmaf(xv.x, win[l].x, acc[l].x);
+                    acc[l].y = fmaf(xv.y, win[l].y, acc[l].y);
+                }
+#pragma unroll
+                for (int l = MAXW - 1; l > 0; --l) win[l] = win[l - 1];
+            }
+        }
+#pragma unroll
+        for (int l = 0; l < MAXW; ++l)
+            if (l < kw) {
+                float* dst = dweight + static_cast<long long>(ij * kw + l) * C + c;
+                atomicAdd(dst, acc[l].x);
+                atomicAdd(dst + 1, acc[l].y);
+            }
+        if (ij == 0 && dbias) {
+            atomicAdd(dbias + c, bsum.x);
+            atomicAdd(dbias + c + 1, bsum.y);
+        }
+    }
+}
+
+template <typename T>
+cudaError_t launch_wgrad(const void* x, const void* dy, float* dweight, float* dbias, int Tn, int H, int W, int C,
+                         const int kernel[3], cudaStream_t st) {
+    const long long rows = static_cast<long long>(Tn) * H;
+    const long long chunks = (rows + kWgradRows - 1) / kWgradRows;
+    if (chunks > 65535) return cudaErrorInvalidConfiguration;
+    int warps = kernel[0] * kernel[1];
+    if (warps > 32) warps = 32;
+    const dim3 grid((C + 63) / 64, static_cast<unsigned>(chunks));
+    const T* xp = static_cast<const T*>(x);
+    const T* gp = static_cast<const T*>(dy);
+#define DSA3D_WGRAD_CASE(KW) \
+    case KW: dwconv3d_wgrad_kernel<T, KW><<<grid, warps * 32, 0, st>>>(xp, gp, dweight, dbias, Tn, H, W, C, kernel[0], kernel[1], KW); break;
+    switch (kernel[2]) {
+        DSA3D_WGRAD_CASE(1)
+        DSA3D_WGRAD_CASE(3)
+        DSA3D_WGRAD_CASE(5)
+        DSA3D_WGRAD_CASE(7)
+        default: dwconv3d_wgrad_kernel<T, 0><<<grid, warps * 32, 0, st>>>(xp, gp, dweight, dbias, Tn, H, W, C, kernel[0], kernel[1], kernel[2]);
+    }
+#undef DSA3D_WGRAD_CASE
+    return cudaGetLastError();
+}
+
+// src [rows, cols] (row pitch lds) -> dstT [cols, rows] bf16 (row pitch ldt); when `dst` is given
+// also the untransposed bf16 copy (row pitch ldd), and when `colsum` is given the fp32 column
+// sums of src (one atomic per column and block).  A block owns a 64-column strip of up to
+// kTrRowsPerBlock rows and walks it in 64 x 64 tiles through shared memory.
+constexpr int kTrRowsPerBlock = 1024;
+template <typename S>
+__global__ void __launch_bounds__(256)
+transpose_to_bf16_kernel(const S* __restrict__ src, long long lds, long long rows, int cols,
+                         __nv_bfloat16* __restrict__ dstT, long long ldt, __nv_bfloat16* __restrict__ dst, long long ldd,
+                         float* __restrict__ colsum) {
+    __shared__ unsigned short tile[64][66];
+    __shared__ float sums[4][64];
+    const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;           // 64 columns x 4 row phases
+    const int c0 = blockIdx.x * 64;
+    const long long rb = static_cast<long long>(blockIdx.y) * kTrRowsPerBlock;
+    const long long re = rb + kTrRowsPerBlock < rows ? rb + kTrRowsPerBlock : rows;
+    float csum = 0.0f;
+    for (long long t0 = rb; t0 < re; t0 += 64) {
+        for (int r = ty; r < 64; r += 4) {
+            const long long row = t0 + r;
+            float v = 0.0f;
+            if (row < re && c0 + tx < cols) v = static_cast<float>(src[row * lds + c0 + tx]);
+            csum += v;
+            const __nv_bfloat16 h = __float2bfloat16_rn(v);
+            tile[r][tx] = *reinterpret_cast<const unsigned short*>(&h);
+            if (dst && row < re && c0 + tx < cols) dst[row * ldd + c0 + tx] = h;
+        }
+        __syncthreads();
+        for (int cc = ty; cc < 64; cc += 4) {
+            const long long row = t0 + tx;
+            if (row < re && c0 + cc < cols) {
+                const unsigned short u = tile[tx][cc];
+                dstT[static_cast<long long>(c0 + cc) * ldt + row] = *reinterpret_cast<const __nv_bfloat16*>(&u);
+            }
+        }
+        __syncthreads();
+    }
+    if (colsum) {
+        sums[ty][tx] = csum;
+        __syncthreads();
+        if (ty == 0 && c0 + tx < cols) atomicAdd(colsum + c0 + tx, sums[0][tx] + sums[1][tx] + sums[2][tx] + sums[3][tx]);
+    }
+}
+
+// fp32 storage: plain loops, one thread per output element.
+__global__ void __launch_bounds__(256)
+linear_du_f32_kernel(const float* __restrict__ g, const float* __restrict__ w, float* __restrict__ du, long long M, int C,
+                     int O) {
+    const long long id = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (id >= M * C) return;
+    const long long n = id / C;
+    const int c = static_cast<int>(id - n * C);
+    float acc = 0.0f;
+    for (int o = 0; o < O; ++o) acc = fmaf(__ldg(g + n * O + o), __ldg(w + static_cast<long long>(o) * C + c), acc);
+    du[id] = acc;
+}
+
+__global__ void __launch_bounds__(256)
+linear_dw_f32_kernel(const float* __restrict__ g, const float* __restrict__ u, float* __restrict__ dw,
+                     float* __restrict__ dbias, long long M, int C, int O) {
+    const long long id = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (id >= static_cast<long long>(O) * C) return;
+    const int o = static_cast<int>(id / C), c = static_cast<int>(id % C);
+    float acc = 0.0f, bs = 0.0f;
+    for (long long n = 0; n < M; ++n) {
+        const float gv = __ldg(g + n * O + o);
+        acc = fmaf(gv, __ldg(u + n * C + c), acc);
+        bs += gv;
+    }
+    if (dw) dw[id] = acc;
+    if (dbias && c == 0) dbias[o] = bs;
+}
+
+long long round_up8(long long v) { return (v + 7) / 8 * 8; }
+size_t round_up256(size_t v) { return (v + 255) / 256 * 256; }
+constexpr long long kLinearSlabTokens = 262144;          // tokens per pass of the linear layer's backward
+
+struct LinearBackwardPlan {
+    long long slab, ld_o, ld_s;
+    size_t off_wt, off_g, off_gt, off_ut, total;
+};
+LinearBackwardPlan linear_backward_plan(long long tokens, int C, int O) {
+    LinearBackwardPlan p;
+    p.slab = tokens < kLinearSlabTokens ? tokens : kLinearSlabTokens;
+    p.ld_o = round_up8(O);
+    p.ld_s = round_up8(p.slab);
+    size_t at = 0;
+    p.off_wt = at; at += round_up256(static_cast<size_t>(C) * p.ld_o * 2);          // w^T  [C, O]
+    p.off_g = at;  at += round_up256(static_cast<size_t>(p.slab) * p.ld_o * 2);     // doffsets in bf16 [slab, O]
+    p.off_gt = at; at += round_up256(static_cast<size_t>(O) * p.ld_s * 2);          // its transpose   [O, slab]
+    p.off_ut = at; at += round_up256(static_cast<size_t>(C) * p.ld_s * 2);          // u^T  [C, slab]
+    p.total = at;
+    return p;
 }
 
 }  // namespace
@@ -697,12 +1015,10 @@ namespace {
 
 int cuda_failed(cudaError_t e) { return dsa3d::note_cuda_error(e); }
 
-}  // namespace
-
-extern "C" {
-
-int dsa3d_dwconv3d_forward(const void* x, const float* weight, const float* bias, int T, int H, int W, int C,
-                           const int kernel[3], void* y, int dtype, void* stream) {
+// y = cross-correlation of x with weight; tap (i, j, l) reads the input at displacement
+// (i - centre[0], j - centre[1], l - centre[2]).
+int conv_entry(const void* x, const float* weight, const float* bias, int T, int H, int W, int C, const int kernel[3],
+               const int centre[3], void* y, int dtype, void* stream) {
     if (!x || !weight || !y || !kernel) return DSA3D_ERR_NULL_POINTER;
     if (T < 1 || H < 1 || W < 1 || C < 8 || C % 8) return DSA3D_ERR_BAD_SHAPE;
     if (kernel[0] < 1 || kernel[1] < 1 || kernel[2] < 1 || kernel[2] > kConvMaxKw || kernel[0] > 15 || kernel[1] > 15)
@@ -715,15 +1031,26 @@ int dsa3d_dwconv3d_forward(const void* x, const float* weight, const float* bias
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (dtype == DSA3D_BF16) {
         cudaError_t te;
-        if (try_dwconv_tma(x, weight, bias, y, T, H, W, C, kernel, st, &te))
+        if (try_dwconv_tma(x, weight, bias, y, T, H, W, C, kernel, centre, st, &te))
             return te == cudaSuccess ? DSA3D_OK : cuda_failed(te);
     }
     if (dtype == DSA3D_BF16)
-        launch_dwconv<__nv_bfloat16>(x, weight, bias, y, T, H, W, C, kernel, static_cast<unsigned>(blocks), st);
+        launch_dwconv<__nv_bfloat16>(x, weight, bias, y, T, H, W, C, kernel, centre, static_cast<unsigned>(blocks), st);
     else
-        launch_dwconv<float>(x, weight, bias, y, T, H, W, C, kernel, static_cast<unsigned>(blocks), st);
+        launch_dwconv<float>(x, weight, bias, y, T, H, W, C, kernel, centre, static_cast<unsigned>(blocks), st);
     const cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
+}
+
+}  // namespace
+
+extern "C" {
+
+int dsa3d_dwconv3d_forward(const void* x, const float* weight, const float* bias, int T, int H, int W, int C,
+                           const int kernel[3], void* y, int dtype, void* stream) {
+    if (!kernel) return DSA3D_ERR_NULL_POINTER;
+    const int centre[3] = {kernel[0] / 2, kernel[1] / 2, kernel[2] / 2};
+    return conv_entry(x, weight, bias, T, H, W, C, kernel, centre, y, dtype, stream);
 }
 
 int dsa3d_offsets_linear_forward(const void* u, const void* w, const float* bias, long long tokens, int C, int O,
@@ -752,31 +1079,10 @@ int dsa3d_offsets_linear_forward(const void* u, const void* w, const float* bias
     CUtensorMap map_u, map_w;
     const bool pair = sms >= 2 && !std::getenv("DSA3D_GEMM_ONE_CTA");     // pairs of CTAs unless switched off
     if (pair) {
-        const long long m_tiles = (tokens + 2 * BM - 1) / (2 * BM);
-        if (!make_map(&map_u, u, static_cast<unsigned long long>(tokens), static_cast<unsigned long long>(C), BM) ||
-            !make_map(&map_w, w, static_cast<unsigned long long>(O), static_cast<unsigned long long>(C),
-                      static_cast<unsigned>(BN / 2)))
-            return DSA3D_ERR_UNSUPPORTED;
-        const size_t smem = sizeof(GemmPairSmem) + 1024;
-        e = cudaFuncSetAttribute(offsets_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(smem));
-        if (e != cudaSuccess) return cuda_failed(e);
-        const long long tiles = m_tiles * n_tiles;
-        const long long want = 2 * (tiles < sms / 2 ? tiles : sms / 2);
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(static_cast<unsigned>(want));
-        cfg.blockDim = dim3(kGemmThreads);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        e = cudaLaunchKernelEx(&cfg, offsets_gemm_pair_kernel, map_u, map_w, bias, offsets, tokens, O, C, BN, m_tiles,
-                               n_tiles);
+        bool unsupported = false;
+        e = launch_pair_gemm(u, static_cast<unsigned long long>(C), w, static_cast<unsigned long long>(C), bias, offsets,
+                             tokens, O, C, kGemmStoreF32, 1, sms, st, &unsupported);
+        if (unsupported) return DSA3D_ERR_UNSUPPORTED;
         return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
     }
     const long long m_tiles = (tokens + BM - 1) / BM;
@@ -793,6 +1099,143 @@ int dsa3d_offsets_linear_forward(const void* u, const void* w, const float* bias
                                                            n_tiles);
     e = cudaGetLastError();
     return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
+}
+
+size_t dsa3d_dwconv3d_backward_workspace_bytes(int C, const int kernel[3]) {
+    if (!kernel || C < 1 || kernel[0] < 1 || kernel[1] < 1 || kernel[2] < 1) return 0;
+    return round_up256(static_cast<size_t>(kernel[0]) * kernel[1] * kernel[2] * C * sizeof(float));
+}
+
+int dsa3d_dwconv3d_backward(const void* x, const float* weight, const void* dy, int T, int H, int W, int C,
+                            const int kernel[3], void* dx, float* dweight, float* dbias, void* workspace,
+                            size_t workspace_bytes, int dtype, void* stream) {
+    if (!dy || !kernel || (dx && (!weight || !workspace)) || (dweight && !x) || (dbias && !dweight))
+        return DSA3D_ERR_NULL_POINTER;
+    if (T < 1 || H < 1 || W < 1 || C < 8 || C % 8) return DSA3D_ERR_BAD_SHAPE;
+    if (kernel[0] < 1 || kernel[1] < 1 || kernel[2] < 1 || kernel[2] > kConvMaxKw || kernel[0] > 15 || kernel[1] > 15)
+        return DSA3D_ERR_BAD_SHAPE;
+    if (dtype != DSA3D_F32 && dtype != DSA3D_BF16) return DSA3D_ERR_UNSUPPORTED;
+    if (!aligned16(dy) || (x && !aligned16(x)) || (dx && !aligned16(dx)) || (dweight && !aligned16(dweight)) ||
+        (workspace && !aligned16(workspace)))
+        return DSA3D_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int taps = kernel[0] * kernel[1] * kernel[2];
+    if (dx) {
+        if (workspace_bytes < dsa3d_dwconv3d_backward_workspace_bytes(C, kernel)) return DSA3D_ERR_WORKSPACE;
+        float* wf = static_cast<float*>(workspace);
+        const long long n = static_cast<long long>(taps) * C;
+        flip_weight_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(weight, wf, taps, C);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_failed(e);
+        // flipped tap i' = kt-1-i reads dy at displacement i' - (kt-1-kt/2)
+        const int centre[3] = {kernel[0] - 1 - kernel[0] / 2, kernel[1] - 1 - kernel[1] / 2, kernel[2] - 1 - kernel[2] / 2};
+        const int rc = conv_entry(dy, wf, nullptr, T, H, W, C, kernel, centre, dx, dtype, stream);
+        if (rc != DSA3D_OK) return rc;
+    }
+    if (dweight) {
+        cudaError_t e = cudaMemsetAsync(dweight, 0, static_cast<size_t>(taps) * C * sizeof(float), st);
+        if (e != cudaSuccess) return cuda_failed(e);
+        if (dbias) {
+            e = cudaMemsetAsync(dbias, 0, static_cast<size_t>(C) * sizeof(float), st);
+            if (e != cudaSuccess) return cuda_failed(e);
+        }
+        e = dtype == DSA3D_BF16 ? launch_wgrad<__nv_bfloat16>(x, dy, dweight, dbias, T, H, W, C, kernel, st)
+                                : launch_wgrad<float>(x, dy, dweight, dbias, T, H, W, C, kernel, st);
+        if (e != cudaSuccess) return cuda_failed(e);
+    }
+    return DSA3D_OK;
+}
+
+size_t dsa3d_offsets_linear_backward_workspace_bytes(long long tokens, int C, int O, int dtype) {
+    if (tokens < 1 || C < 1 || O < 1 || dtype != DSA3D_BF16) return 0;
+    return linear_backward_plan(tokens, C, O).total;
+}
+
+int dsa3d_offsets_linear_backward(const void* u, const void* w, const float* doffsets, long long tokens, int C, int O,
+                                  void* du, float* dw, float* dbias, void* workspace, size_t workspace_bytes, int dtype,
+                                  void* stream) {
+    if (!doffsets || (du && !w) || (dw && !u)) return DSA3D_ERR_NULL_POINTER;
+    if (tokens < 1 || C < 8 || C % 8 || O < 1 || tokens > 0x7fffffffLL) return DSA3D_ERR_BAD_SHAPE;
+    if (dtype != DSA3D_F32 && dtype != DSA3D_BF16) return DSA3D_ERR_UNSUPPORTED;
+    if (!aligned16(doffsets) || (u && !aligned16(u)) || (w && !aligned16(w)) || (du && !aligned16(du)) ||
+        (dw && !aligned16(dw)) || (workspace && !aligned16(workspace)))
+        return DSA3D_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if (dtype == DSA3D_F32) {
+        if (du) {
+            const long long blocks = (tokens * C + 255) / 256;
+            if (blocks > 0x7fffffffLL) return DSA3D_ERR_BAD_SHAPE;
+            linear_du_f32_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(
+                doffsets, static_cast<const float*>(w), static_cast<float*>(du), tokens, C, O);
+            if ((e = cudaGetLastError()) != cudaSuccess) return cuda_failed(e);
+        }
+        if (dw || dbias) {
+            if (!u) return DSA3D_ERR_NULL_POINTER;
+            const long long blocks = (static_cast<long long>(O) * C + 255) / 256;
+            linear_dw_f32_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(doffsets, static_cast<const float*>(u), dw,
+                                                                                 dbias, tokens, C, O);
+            if ((e = cudaGetLastError()) != cudaSuccess) return cuda_failed(e);
+        }
+        return DSA3D_OK;
+    }
+    if (!du && !dw && !dbias) return DSA3D_OK;
+    if (!workspace) return DSA3D_ERR_NULL_POINTER;
+    const LinearBackwardPlan plan = linear_backward_plan(tokens, C, O);
+    if (workspace_bytes < plan.total) return DSA3D_ERR_WORKSPACE;
+    int dev = 0, sms = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return cuda_failed(e);
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return cuda_failed(e);
+    if (sms < 2) return DSA3D_ERR_UNSUPPORTED;
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    __nv_bfloat16* wt = reinterpret_cast<__nv_bfloat16*>(ws + plan.off_wt);
+    __nv_bfloat16* g = reinterpret_cast<__nv_bfloat16*>(ws + plan.off_g);
+    __nv_bfloat16* gt = reinterpret_cast<__nv_bfloat16*>(ws + plan.off_gt);
+    __nv_bfloat16* ut = reinterpret_cast<__nv_bfloat16*>(ws + plan.off_ut);
+    const __nv_bfloat16* ub = static_cast<const __nv_bfloat16*>(u);
+    if (dw && (e = cudaMemsetAsync(dw, 0, static_cast<size_t>(O) * C * sizeof(float), st)) != cudaSuccess) return cuda_failed(e);
+    if (dbias && (e = cudaMemsetAsync(dbias, 0, static_cast<size_t>(O) * sizeof(float), st)) != cudaSuccess) return cuda_failed(e);
+    if (du) {                                                        // w [O, C] -> w^T [C, O]
+        const dim3 grid((C + 63) / 64, static_cast<unsigned>((O + kTrRowsPerBlock - 1) / kTrRowsPerBlock));
+        transpose_to_bf16_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(w), C, O, C, wt,
+                                                                      plan.ld_o, nullptr, 0, nullptr);
+        if ((e = cudaGetLastError()) != cudaSuccess) return cuda_failed(e);
+    }
+    bool unsupported = false;
+    for (long long s0 = 0; s0 < tokens; s0 += plan.slab) {
+        const long long ns = tokens - s0 < plan.slab ? tokens - s0 : plan.slab;
+        const unsigned row_blocks = static_cast<unsigned>((ns + kTrRowsPerBlock - 1) / kTrRowsPerBlock);
+        {   // doffsets slab -> bf16 copy, bf16 transpose, column sums
+            const dim3 grid((O + 63) / 64, row_blocks);
+            transpose_to_bf16_kernel<float><<<grid, 256, 0, st>>>(doffsets + s0 * O, O, ns, O, gt, plan.ld_s,
+                                                                  du ? g : nullptr, plan.ld_o, dbias);
+            if ((e = cudaGetLastError()) != cudaSuccess) return cuda_failed(e);
+        }
+        if (du) {                                                    // du[slab] = g . (w^T)^T
+            e = launch_pair_gemm(g, static_cast<unsigned long long>(plan.ld_o), wt, static_cast<unsigned long long>(plan.ld_o),
+                                 nullptr, static_cast<__nv_bfloat16*>(du) + s0 * C, ns, C, O, kGemmStoreBf16, 1, sms, st,
+                                 &unsupported);
+            if (unsupported) return DSA3D_ERR_UNSUPPORTED;
+            if (e != cudaSuccess) return cuda_failed(e);
+        }
+        if (dw) {                                                    // dw += g^T . (u^T)^T over this slab's tokens
+            const dim3 grid((C + 63) / 64, row_blocks);
+            transpose_to_bf16_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(ub + s0 * C, C, ns, C, ut, plan.ld_s, nullptr, 0,
+                                                                          nullptr);
+            if ((e = cudaGetLastError()) != cudaSuccess) return cuda_failed(e);
+            const long long tiles = ((O + 2 * BM - 1) / (2 * BM)) * static_cast<long long>((C + kMaxBN - 1) / kMaxBN);
+            const long long kblocks = (ns + BK - 1) / BK;
+            long long ksplits = (2LL * (sms / 2) + tiles - 1) / tiles;        // about two waves of work units
+            if (ksplits > kblocks) ksplits = kblocks;
+            if (ksplits < 1) ksplits = 1;
+            e = launch_pair_gemm(gt, static_cast<unsigned long long>(plan.ld_s), ut, static_cast<unsigned long long>(plan.ld_s),
+                                 nullptr, dw, O, C, static_cast<int>(ns), kGemmAddF32, static_cast<int>(ksplits), sms, st,
+                                 &unsupported);
+            if (unsupported) return DSA3D_ERR_UNSUPPORTED;
+            if (e != cudaSuccess) return cuda_failed(e);
+        }
+    }
+    return DSA3D_OK;
 }
 
 int dsa3d_device_timeout_flag(void) {
