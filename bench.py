@@ -268,6 +268,23 @@ def measure_producer(wl, dev, reps: int = 5):
 
     conv_ms = timed(lambda: binding.dsa3d_dwconv3d_forward(x, wc, None, T, H, W, C, (3, 3, 3), u))
     gemm_ms = timed(lambda: binding.dsa3d_offsets_linear_forward(u, wlin, blin, N, C, O, off))
+    # backward of both layers: dy of the convolution = the activations themselves (any tensor of
+    # that shape and dtype does), doffsets of the linear layer = the offsets it just produced
+    dxc = torch.empty_like(x)
+    dwc = torch.empty((27, C), dtype=torch.float32, device=dev)
+    dbc = torch.empty((C,), dtype=torch.float32, device=dev)
+    wsc = torch.empty(binding.dsa3d_dwconv3d_backward_workspace_bytes(C, (3, 3, 3)), dtype=torch.uint8, device=dev)
+    conv_dx_ms = timed(lambda: binding.dsa3d_dwconv3d_backward(None, wc, u, T, H, W, C, (3, 3, 3), dxc, None, None, wsc))
+    conv_dw_ms = timed(lambda: binding.dsa3d_dwconv3d_backward(x, None, u, T, H, W, C, (3, 3, 3), None, dwc, dbc, None))
+    del dxc, wsc
+    du = torch.empty_like(u)
+    dwl = torch.empty((O, C), dtype=torch.float32, device=dev)
+    dbl = torch.empty((O,), dtype=torch.float32, device=dev)
+    wsl = torch.empty(binding.dsa3d_offsets_linear_backward_workspace_bytes(N, C, O, wl.dtype), dtype=torch.uint8,
+                      device=dev)
+    lin_du_ms = timed(lambda: binding.dsa3d_offsets_linear_backward(None, wlin, off, N, C, O, du, None, None, wsl))
+    lin_dw_ms = timed(lambda: binding.dsa3d_offsets_linear_backward(u, None, off, N, C, O, None, dwl, dbl, wsl))
+    del du, dwl, dbl, wsl
     flag = binding.dsa3d_device_timeout_flag()
     elt = wl.elt
     peaks = {}
@@ -286,7 +303,12 @@ def measure_producer(wl, dev, reps: int = 5):
            "offsets_linear": {"ms": gemm_ms, "bound": "tensor", "achieved": gemm_tf, "peak": tf_peak,
                               "unit": "TFLOP/s", "frac": gemm_tf / tf_peak, "dtype": "bf16 x bf16 -> f32",
                               "peak_source": "measured burst (MEASURED_PEAKS.json bf16_tflops)" if peaks else "fallback"},
-           "per_layer_ms": 2 * conv_ms + gemm_ms}
+           "per_layer_ms": 2 * conv_ms + gemm_ms,
+           "backward": {"dwconv3d_dx_ms": conv_dx_ms, "dwconv3d_dweight_dbias_ms": conv_dw_ms,
+                        "offsets_linear_du_ms": lin_du_ms, "offsets_linear_dw_dbias_ms": lin_dw_ms,
+                        "offsets_linear_tflops": {"du": 2.0 * N * C * O / (lin_du_ms * 1e-3) / 1e12,
+                                                  "dw": 2.0 * N * C * O / (lin_dw_ms * 1e-3) / 1e12},
+                        "note": "linear-layer times include the bf16 conversion and transposes of doffsets and u"}}
     del x, wc, wlin, blin, u, off
     torch.cuda.empty_cache()
     return res

@@ -456,10 +456,13 @@ struct __align__(1024) GemmPairSmem {
     uint32_t tmem_base;
 };
 
+// MN_MAJOR: the operands are given as [K, M] and [K, N] row-major matrices (the contraction index
+// is the row), fetched as boxes of 64 columns x BK rows; BN is 256 then.
+template <int MODE, bool MN_MAJOR>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_constant__ CUtensorMap map_w,
                          const float* __restrict__ bias, void* __restrict__ out_raw, long long M, int N, int K, int BN,
-                         long long m_tiles, int n_tiles, int mode, int ksplits) {
+                         long long m_tiles, int n_tiles, int ksplits) {
     extern __shared__ unsigned char raw[];
     GemmPairSmem& s = *reinterpret_cast<GemmPairSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -508,9 +511,22 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
                     const uint32_t full_leader = map_to_cta(smem_u32(&s.full[st]), 0);
                     if (rank == 0)                               // the bytes of both CTAs land on the leader's barrier
                         mbar_expect_tx(smem_u32(&s.full[st]), static_cast<uint32_t>(2 * (BM + BN / 2) * BK * 2));
-                    tma_load_2d_pair(smem_u32(s.a[st]), &map_u, full_leader, kb * BK,
-                                     static_cast<int>(m0) + static_cast<int>(rank) * BM);
-                    tma_load_2d_pair(smem_u32(s.b[st]), &map_w, full_leader, kb * BK, n0 + static_cast<int>(rank) * (BN / 2));
+                    if constexpr (MN_MAJOR) {
+                        const int ma = static_cast<int>(m0) + static_cast<int>(rank) * BM;
+                        const int nb = n0 + static_cast<int>(rank) * (kMaxBN / 2);
+#pragma unroll
+                        for (int atom = 0; atom < 2; ++atom) {
+                            tma_load_2d_pair(smem_u32(s.a[st]) + atom * (64 * BK * 2), &map_u, full_leader, ma + atom * 64,
+                                             kb * BK);
+                            tma_load_2d_pair(smem_u32(s.b[st]) + atom * (64 * BK * 2), &map_w, full_leader, nb + atom * 64,
+                                             kb * BK);
+                        }
+                    } else {
+                        tma_load_2d_pair(smem_u32(s.a[st]), &map_u, full_leader, kb * BK,
+                                         static_cast<int>(m0) + static_cast<int>(rank) * BM);
+                        tma_load_2d_pair(smem_u32(s.b[st]), &map_w, full_leader, kb * BK,
+                                         n0 + static_cast<int>(rank) * (BN / 2));
+                    }
                 }
                 if (!ok) { atomicExch(&g_timeout_flag, 8); break; }
             }
@@ -518,7 +534,8 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
-                                   (static_cast<uint32_t>((2 * BM) >> 4) << 24);
+                                   (static_cast<uint32_t>((2 * BM) >> 4) << 24) |
+                                   (MN_MAJOR ? (1u << 15) | (1u << 16) : 0u);       // both operands MN-major
             uint32_t it = 0, local = 0;
             bool ok = true;
             for (long long unit = pair; unit < tiles && ok; unit += pairs, ++local) {
@@ -532,10 +549,19 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
                     const int st = it % kPairStages;
                     if (!mbar_wait(smem_u32(&s.full[st]), (it / kPairStages) & 1)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint64_t da = smem_desc(smem_u32(s.a[st])), db = smem_desc(smem_u32(s.b[st]));
+                    if constexpr (MN_MAJOR) {
+                        // 16 rows of 128 bytes per step: 2048 bytes = 128 in the descriptor's 16-byte units
+                        const uint64_t da = smem_desc_mn(smem_u32(s.a[st]), 64 * BK * 2),
+                                       db = smem_desc_mn(smem_u32(s.b[st]), 64 * BK * 2);
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
-                        umma_bf16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, ((kb - kb0) | k) ? 1u : 0u);
+                        for (int k = 0; k < BK / 16; ++k)
+                            umma_bf16_pair(d_tmem, da + 128 * k, db + 128 * k, idesc, ((kb - kb0) | k) ? 1u : 0u);
+                    } else {
+                        const uint64_t da = smem_desc(smem_u32(s.a[st])), db = smem_desc(smem_u32(s.b[st]));
+#pragma unroll
+                        for (int k = 0; k < BK / 16; ++k)
+                            umma_bf16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, ((kb - kb0) | k) ? 1u : 0u);
+                    }
                     umma_commit_pair(smem_u32(&s.empty[st]));          // frees the stage in both CTAs
                 }
                 umma_commit_pair(smem_u32(&s.acc_full[buf]));
@@ -560,7 +586,7 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
                 tmem_load_32(tmem + (static_cast<uint32_t>(quarter * 32) << 16) + buf * kMaxBN + c0, r);
                 if (row >= M) continue;
                 const bool whole = n0 + c0 + 32 <= N;
-                if (mode == kGemmStoreF32) {
+                if constexpr (MODE == kGemmStoreF32) {
                     float* dst = static_cast<float*>(out_raw) + row * N + n0 + c0;
                     if (whole && (N & 3) == 0) {
 #pragma unroll
@@ -576,7 +602,7 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
                         for (int j = 0; j < 32; ++j)
                             if (n0 + c0 + j < N) dst[j] = __uint_as_float(r[j]) + (bias ? __ldg(bias + n0 + c0 + j) : 0.0f);
                     }
-                } else if (mode == kGemmStoreBf16) {
+                } else if constexpr (MODE == kGemmStoreBf16) {
                     __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(out_raw) + row * N + n0 + c0;
                     if (whole && (N & 7) == 0) {
 #pragma unroll
@@ -674,22 +700,24 @@ bool make_map(CUtensorMap* map, const void* ptr, unsigned long long rows, unsign
 // output tile (> 1 only with kGemmAddF32).  Column tiles of equal width, a multiple of 32, at most 256.
 cudaError_t launch_pair_gemm(const void* A, unsigned long long lda, const void* B, unsigned long long ldb,
                              const float* bias, void* out, long long M, int N, int K, int mode, int ksplits, int sms,
-                             cudaStream_t st, bool* unsupported) {
+                             cudaStream_t st, bool* unsupported, bool mn_major = false) {
     *unsupported = false;
     const int n_tiles = (N + kMaxBN - 1) / kMaxBN;
-    const int BN = ((N + n_tiles - 1) / n_tiles + 31) / 32 * 32;
+    const int BN = mn_major ? kMaxBN : ((N + n_tiles - 1) / n_tiles + 31) / 32 * 32;
     const long long m_tiles = (M + 2 * BM - 1) / (2 * BM);
     CUtensorMap map_a, map_b;
-    if (!make_map(&map_a, A, static_cast<unsigned long long>(M), static_cast<unsigned long long>(K), BM, lda) ||
-        !make_map(&map_b, B, static_cast<unsigned long long>(N), static_cast<unsigned long long>(K),
-                  static_cast<unsigned>(BN / 2), ldb)) {
+    // MN-major: A is [K, M] and B is [K, N] in memory, fetched as boxes of 64 columns x BK rows
+    const bool ok = mn_major
+        ? make_map(&map_a, A, static_cast<unsigned long long>(K), static_cast<unsigned long long>(M), BK, lda) &&
+          make_map(&map_b, B, static_cast<unsigned long long>(K), static_cast<unsigned long long>(N), BK, ldb)
+        : make_map(&map_a, A, static_cast<unsigned long long>(M), static_cast<unsigned long long>(K), BM, lda) &&
+          make_map(&map_b, B, static_cast<unsigned long long>(N), static_cast<unsigned long long>(K),
+                   static_cast<unsigned>(BN / 2), ldb);
+    if (!ok || (mn_major && mode != kGemmAddF32)) {
         *unsupported = true;
         return cudaSuccess;
     }
     const size_t smem = sizeof(GemmPairSmem) + 1024;
-    cudaError_t e = cudaFuncSetAttribute(offsets_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
     const long long units = m_tiles * n_tiles * ksplits;
     const long long want = 2 * (units < sms / 2 ? units : sms / 2);
     cudaLaunchConfig_t cfg = {};
@@ -704,8 +732,15 @@ cudaError_t launch_pair_gemm(const void* A, unsigned long long lda, const void* 
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, offsets_gemm_pair_kernel, map_a, map_b, bias, out, M, N, K, BN, m_tiles, n_tiles, mode,
-                              ksplits);
+    auto launch = [&](auto kernel) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+        return cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, bias, out, M, N, K, BN, m_tiles, n_tiles, ksplits);
+    };
+    if (mn_major) return launch(offsets_gemm_pair_kernel<kGemmAddF32, true>);
+    if (mode == kGemmStoreF32) return launch(offsets_gemm_pair_kernel<kGemmStoreF32, false>);
+    if (mode == kGemmStoreBf16) return launch(offsets_gemm_pair_kernel<kGemmStoreBf16, false>);
+    return launch(offsets_gemm_pair_kernel<kGemmAddF32, false>);
 }
 
 // Channels-last activations [T, H, W, C] bf16 as a 4-D map with boxes of 64 channels x pw x ph x 1.
@@ -774,9 +809,10 @@ bool try_dwconv_tma(const void* x, const float* weight, const float* bias, void*
 //                 forward, centre kt-1-kt/2 etc.); dweight[tap, c] = sum_s x[s + disp] dy[s, c]
 //                 and dbias by dwconv3d_wgrad_kernel.
 //   linear layer: du = doffsets . w and dw = doffsets^T . u as two tensor-core contractions
-//                 (bf16 operands: doffsets is rounded to bf16 once, w and u are transposed
-//                 copies so that every operand is K-major), token slab by token slab; dbias
-//                 from the fp32 doffsets.
+//                 (bf16 operands: doffsets is rounded to bf16 once; the first takes a transposed
+//                 copy of w so that both operands are K-major, the second reads doffsets and u
+//                 as MN-major operands, the token index being their row), token slab by token
+//                 slab; dbias from the fp32 doffsets.
 // ------------------------------------------------------------------------------------------
 __global__ void flip_weight_kernel(const float* __restrict__ w, float* __restrict__ wf, int taps, int C) {
     const long long id = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -845,6 +881,7 @@ dwconv3d_wgrad_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* 
                 const int ox = cw - l;                      // output column seen by tap l at sx = 0, minus the shift
                 if (l < kw && ox >= 0 && ox < W) win[l] = Pair2<T>::load(gy + static_cast<long long>(ox) * C);
             }
+#pragma unroll 4
             for (int sx = 0; sx < W; ++sx) {
                 const int ox0 = sx + cw;                    // newest output column (tap 0)
                 win[0] = (ox0 < W) ? Pair2<T>::load(gy + static_cast<long long>(ox0) * C) : make_float2(0.f, 0.f);
@@ -896,47 +933,87 @@ cudaError_t launch_wgrad(const void* x, const void* dy, float* dweight, float* d
     return cudaGetLastError();
 }
 
-// src [rows, cols] (row pitch lds) -> dstT [cols, rows] bf16 (row pitch ldt); when `dst` is given
-// also the untransposed bf16 copy (row pitch ldd), and when `colsum` is given the fp32 column
-// sums of src (one atomic per column and block).  A block owns a 64-column strip of up to
-// kTrRowsPerBlock rows and walks it in 64 x 64 tiles through shared memory.
+// src [rows, cols] (row pitch lds) -> dstT [cols, rows] bf16 (row pitch ldt, a multiple of 8); when
+// `dst` is given also the untransposed bf16 copy (row pitch ldd, a multiple of 8: whole words are
+// written, the padding columns included), and when `colsum` is given the fp32 column sums of src
+// (one atomic per column and block).  A block owns a 64-column strip of up to kTrRowsPerBlock
+// rows and walks it in 64 x 64 tiles through shared memory; a thread moves pairs: two
+// neighbouring columns on the way in, two neighbouring rows on the way out, so every warp
+// access is 128 contiguous bytes (256 for fp32 sources).
 constexpr int kTrRowsPerBlock = 1024;
+template <typename S> struct SrcPair;
+template <> struct SrcPair<float> {
+    static __device__ __forceinline__ float2 load(const float* p, bool vec, bool second) {
+        if (vec) return __ldg(reinterpret_cast<const float2*>(p));
+        return make_float2(__ldg(p), second ? __ldg(p + 1) : 0.0f);
+    }
+};
+template <> struct SrcPair<__nv_bfloat16> {
+    static __device__ __forceinline__ float2 load(const __nv_bfloat16* p, bool vec, bool second) {
+        if (vec) {
+            const uint32_t r = __ldg(reinterpret_cast<const uint32_t*>(p));
+            return make_float2(__uint_as_float(r << 16), __uint_as_float(r & 0xffff0000u));
+        }
+        return make_float2(__bfloat162float(p[0]), second ? __bfloat162float(p[1]) : 0.0f);
+    }
+};
+
 template <typename S>
 __global__ void __launch_bounds__(256)
 transpose_to_bf16_kernel(const S* __restrict__ src, long long lds, long long rows, int cols,
                          __nv_bfloat16* __restrict__ dstT, long long ldt, __nv_bfloat16* __restrict__ dst, long long ldd,
                          float* __restrict__ colsum) {
-    __shared__ unsigned short tile[64][66];
-    __shared__ float sums[4][64];
-    const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;           // 64 columns x 4 row phases
+    __shared__ uint32_t tile[64][33];                                // [row][column pair]
+    __shared__ float sums[8][64];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;          // 32 pairs x 8 phases
     const int c0 = blockIdx.x * 64;
     const long long rb = static_cast<long long>(blockIdx.y) * kTrRowsPerBlock;
     const long long re = rb + kTrRowsPerBlock < rows ? rb + kTrRowsPerBlock : rows;
-    float csum = 0.0f;
+    const int c = c0 + 2 * tx;
+    const bool in0 = c < cols, in1 = c + 1 < cols;
+    // a pair is one aligned vector when the row pitch keeps pairs aligned and both columns exist
+    const bool vec = in1 && (lds & 1) == 0 && (reinterpret_cast<uintptr_t>(src) & (2 * sizeof(S) - 1)) == 0;
+    float s0 = 0.0f, s1 = 0.0f;
     for (long long t0 = rb; t0 < re; t0 += 64) {
-        for (int r = ty; r < 64; r += 4) {
+#pragma unroll
+        for (int r = ty; r < 64; r += 8) {
             const long long row = t0 + r;
-            float v = 0.0f;
-            if (row < re && c0 + tx < cols) v = static_cast<float>(src[row * lds + c0 + tx]);
-            csum += v;
-            const __nv_bfloat16 h = __float2bfloat16_rn(v);
-            tile[r][tx] = *reinterpret_cast<const unsigned short*>(&h);
-            if (dst && row < re && c0 + tx < cols) dst[row * ldd + c0 + tx] = h;
+            float2 v = make_float2(0.0f, 0.0f);
+            if (row < re && in0) v = SrcPair<S>::load(src + row * lds + c, vec, in1);
+            s0 += v.x;
+            s1 += v.y;
+            const __nv_bfloat162 h = __floats2bfloat162_rn(v.x, v.y);
+            const uint32_t word = *reinterpret_cast<const uint32_t*>(&h);
+            if (dstT) tile[r][tx] = word;
+            if (dst && row < re && c < ldd) *reinterpret_cast<uint32_t*>(dst + row * ldd + c) = word;
         }
+        if (!dstT) continue;                                         // copy and column sums only (uniform)
         __syncthreads();
-        for (int cc = ty; cc < 64; cc += 4) {
-            const long long row = t0 + tx;
-            if (row < re && c0 + cc < cols) {
-                const unsigned short u = tile[tx][cc];
-                dstT[static_cast<long long>(c0 + cc) * ldt + row] = *reinterpret_cast<const __nv_bfloat16*>(&u);
+        // rows 2tx, 2tx+1 of column pair j: one word per column, each the two rows' values
+        const long long row = t0 + 2 * tx;
+#pragma unroll
+        for (int j = ty; j < 32; j += 8) {
+            const uint32_t a = tile[2 * tx][j], b = tile[2 * tx + 1][j];
+            const int cc = c0 + 2 * j;
+            if (row < re) {                                          // row + 1 < ldt: the pitch is even
+                if (cc < cols)
+                    *reinterpret_cast<uint32_t*>(dstT + static_cast<long long>(cc) * ldt + row) = __byte_perm(a, b, 0x5410);
+                if (cc + 1 < cols)
+                    *reinterpret_cast<uint32_t*>(dstT + static_cast<long long>(cc + 1) * ldt + row) = __byte_perm(a, b, 0x7632);
             }
         }
         __syncthreads();
     }
     if (colsum) {
-        sums[ty][tx] = csum;
+        sums[ty][2 * tx] = s0;
+        sums[ty][2 * tx + 1] = s1;
         __syncthreads();
-        if (ty == 0 && c0 + tx < cols) atomicAdd(colsum + c0 + tx, sums[0][tx] + sums[1][tx] + sums[2][tx] + sums[3][tx]);
+        if (threadIdx.x < 64 && c0 + threadIdx.x < cols) {
+            float t = 0.0f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) t += sums[k][threadIdx.x];
+            atomicAdd(colsum + c0 + threadIdx.x, t);
+        }
     }
 }
 
@@ -974,19 +1051,16 @@ size_t round_up256(size_t v) { return (v + 255) / 256 * 256; }
 constexpr long long kLinearSlabTokens = 262144;          // tokens per pass of the linear layer's backward
 
 struct LinearBackwardPlan {
-    long long slab, ld_o, ld_s;
-    size_t off_wt, off_g, off_gt, off_ut, total;
+    long long slab, ld_o;
+    size_t off_wt, off_g, total;
 };
 LinearBackwardPlan linear_backward_plan(long long tokens, int C, int O) {
     LinearBackwardPlan p;
     p.slab = tokens < kLinearSlabTokens ? tokens : kLinearSlabTokens;
     p.ld_o = round_up8(O);
-    p.ld_s = round_up8(p.slab);
     size_t at = 0;
     p.off_wt = at; at += round_up256(static_cast<size_t>(C) * p.ld_o * 2);          // w^T  [C, O]
     p.off_g = at;  at += round_up256(static_cast<size_t>(p.slab) * p.ld_o * 2);     // doffsets in bf16 [slab, O]
-    p.off_gt = at; at += round_up256(static_cast<size_t>(O) * p.ld_s * 2);          // its transpose   [O, slab]
-    p.off_ut = at; at += round_up256(static_cast<size_t>(C) * p.ld_s * 2);          // u^T  [C, slab]
     p.total = at;
     return p;
 }
@@ -1190,8 +1264,6 @@ int dsa3d_offsets_linear_backward(const void* u, const void* w, const float* dof
     unsigned char* ws = static_cast<unsigned char*>(workspace);
     __nv_bfloat16* wt = reinterpret_cast<__nv_bfloat16*>(ws + plan.off_wt);
     __nv_bfloat16* g = reinterpret_cast<__nv_bfloat16*>(ws + plan.off_g);
-    __nv_bfloat16* gt = reinterpret_cast<__nv_bfloat16*>(ws + plan.off_gt);
-    __nv_bfloat16* ut = reinterpret_cast<__nv_bfloat16*>(ws + plan.off_ut);
     const __nv_bfloat16* ub = static_cast<const __nv_bfloat16*>(u);
     if (dw && (e = cudaMemsetAsync(dw, 0, static_cast<size_t>(O) * C * sizeof(float), st)) != cudaSuccess) return cuda_failed(e);
     if (dbias && (e = cudaMemsetAsync(dbias, 0, static_cast<size_t>(O) * sizeof(float), st)) != cudaSuccess) return cuda_failed(e);
@@ -1205,10 +1277,10 @@ int dsa3d_offsets_linear_backward(const void* u, const void* w, const float* dof
     for (long long s0 = 0; s0 < tokens; s0 += plan.slab) {
         const long long ns = tokens - s0 < plan.slab ? tokens - s0 : plan.slab;
         const unsigned row_blocks = static_cast<unsigned>((ns + kTrRowsPerBlock - 1) / kTrRowsPerBlock);
-        {   // doffsets slab -> bf16 copy, bf16 transpose, column sums
+        {   // doffsets slab -> bf16 copy and column sums
             const dim3 grid((O + 63) / 64, row_blocks);
-            transpose_to_bf16_kernel<float><<<grid, 256, 0, st>>>(doffsets + s0 * O, O, ns, O, gt, plan.ld_s,
-                                                                  du ? g : nullptr, plan.ld_o, dbias);
+            transpose_to_bf16_kernel<float><<<grid, 256, 0, st>>>(doffsets + s0 * O, O, ns, O, nullptr, 0,
+                                                                  (du || dw) ? g : nullptr, plan.ld_o, dbias);
             if ((e = cudaGetLastError()) != cudaSuccess) return cuda_failed(e);
         }
         if (du) {                                                    // du[slab] = g . (w^T)^T
@@ -1218,19 +1290,15 @@ int dsa3d_offsets_linear_backward(const void* u, const void* w, const float* dof
             if (unsupported) return DSA3D_ERR_UNSUPPORTED;
             if (e != cudaSuccess) return cuda_failed(e);
         }
-        if (dw) {                                                    // dw += g^T . (u^T)^T over this slab's tokens
-            const dim3 grid((C + 63) / 64, row_blocks);
-            transpose_to_bf16_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(ub + s0 * C, C, ns, C, ut, plan.ld_s, nullptr, 0,
-                                                                          nullptr);
-            if ((e = cudaGetLastError()) != cudaSuccess) return cuda_failed(e);
+        if (dw) {       // dw += g^T . u over this slab's tokens: both operands have the contraction index as rows
             const long long tiles = ((O + 2 * BM - 1) / (2 * BM)) * static_cast<long long>((C + kMaxBN - 1) / kMaxBN);
             const long long kblocks = (ns + BK - 1) / BK;
             long long ksplits = (2LL * (sms / 2) + tiles - 1) / tiles;        // about two waves of work units
             if (ksplits > kblocks) ksplits = kblocks;
             if (ksplits < 1) ksplits = 1;
-            e = launch_pair_gemm(gt, static_cast<unsigned long long>(plan.ld_s), ut, static_cast<unsigned long long>(plan.ld_s),
+            e = launch_pair_gemm(g, static_cast<unsigned long long>(plan.ld_o), ub + s0 * C, static_cast<unsigned long long>(C),
                                  nullptr, dw, O, C, static_cast<int>(ns), kGemmAddF32, static_cast<int>(ksplits), sms, st,
-                                 &unsupported);
+                                 &unsupported, true);
             if (unsupported) return DSA3D_ERR_UNSUPPORTED;
             if (e != cudaSuccess) return cuda_failed(e);
         }

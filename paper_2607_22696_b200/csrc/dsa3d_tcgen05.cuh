@@ -51,6 +51,18 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
     d |= static_cast<uint64_t>(2) << 61;            // 128-byte swizzle
     return d;
 }
+// The same for an MN-major tile: the operand's M (or N) index runs along the 128-byte rows, 64
+// elements per swizzle atom, and its K index along the rows; 8-row groups 1024 bytes apart
+// (stride byte offset), atoms of 64 further M/N elements `atom_stride` bytes apart (leading
+// byte offset) - one TMA box of 64 columns x BK rows per atom.
+__device__ __forceinline__ uint64_t smem_desc_mn(uint32_t saddr, uint32_t atom_stride) {
+    uint64_t d = static_cast<uint64_t>((saddr >> 4) & 0x3fff);
+    d |= static_cast<uint64_t>((atom_stride >> 4) & 0x3fff) << 16;
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    d |= static_cast<uint64_t>(2) << 61;
+    return d;
+}
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
