@@ -19,6 +19,7 @@
 #include <cstdint>
 #include <cstdlib>
 #include <mutex>
+#include <type_traits>
 
 #include "../../include/dsa3d.h"
 #include "dsa3d_common.cuh"
@@ -909,10 +910,152 @@ dwconv3d_wgrad_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* 
     }
 }
 
+// The 3 x 3 x 3 kernel in bf16, staged like dwconv3d_tma_kernel: a CTA owns a column of
+// 4 x 16 positions x 64 channels and marches along t; the x planes (with their halo) sit in a
+// ring of 4 shared-memory slots and the dy planes in a ring of 2, each fetched by TMA one step
+// ahead.  A lane owns a pair of channels, a warp one row of 16 positions: per kernel row it
+// slides over 18 x words against the row's 16 dy words, all 27 x 2 sums in registers (packed
+// fp32 FMAs).  The four warps reduce in shared memory; one vector atomic per four channels
+// and tap goes to dweight.
+constexpr int kWgTY = 4, kWgTX = 16, kWgXRing = 4, kWgYRing = 2;
+constexpr int kWgXPlane = (kWgTY + 2) * (kWgTX + 2) * kCvCh * 2;        // 13824 bytes
+constexpr int kWgYPlane = kWgTY * kWgTX * kCvCh * 2;                    // 8192 bytes
+struct __align__(128) WgradSmem {
+    unsigned char xp[kWgXRing][kWgXPlane];
+    unsigned char yp[kWgYRing][kWgYPlane];
+    float red[28][kCvCh];
+    uint64_t xbar[kWgXRing], ybar[kWgYRing];
+};
+
+__global__ void __launch_bounds__(128)
+dwconv3d_wgrad333_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_dy,
+                             float* __restrict__ dweight, float* __restrict__ dbias, int Tn, int H, int W, int C,
+                             int t_chunk) {
+    extern __shared__ unsigned char raw_smem[];
+    WgradSmem& s = *reinterpret_cast<WgradSmem*>((reinterpret_cast<uintptr_t>(raw_smem) + 127) & ~uintptr_t(127));
+    const int tid = threadIdx.x, lane = tid & 31, yl = tid >> 5;
+    const int c0 = blockIdx.x * kCvCh;
+    const int tiles_x = (W + kWgTX - 1) / kWgTX;
+    const int x0 = (blockIdx.y % tiles_x) * kWgTX, y0 = (blockIdx.y / tiles_x) * kWgTY;
+    const int t_begin = blockIdx.z * t_chunk, t_end = min(Tn, t_begin + t_chunk);
+
+    for (int i = tid; i < 28 * kCvCh; i += 128) (&s.red[0][0])[i] = 0.0f;
+    if (tid == 0) {
+        for (int i = 0; i < kWgXRing; ++i) mbar_init(smem_u32(&s.xbar[i]), 1);
+        for (int i = 0; i < kWgYRing; ++i) mbar_init(smem_u32(&s.ybar[i]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    // x plane n is frame t_begin - 1 + n (slot n % 4); dy plane m is frame t_begin + m (slot m % 2)
+    auto issue_x = [&](int n) {
+        const int slot = n % kWgXRing;
+        mbar_expect_tx(smem_u32(&s.xbar[slot]), kWgXPlane);
+        tma_load_4d(smem_u32(s.xp[slot]), &map_x, smem_u32(&s.xbar[slot]), c0, x0 - 1, y0 - 1, t_begin - 1 + n);
+    };
+    auto issue_y = [&](int m) {
+        const int slot = m % kWgYRing;
+        mbar_expect_tx(smem_u32(&s.ybar[slot]), kWgYPlane);
+        tma_load_4d(smem_u32(s.yp[slot]), &map_dy, smem_u32(&s.ybar[slot]), c0, x0, y0, t_begin + m);
+    };
+    if (tid == 0) {
+        for (int n = 0; n < 3; ++n) issue_x(n);
+        issue_y(0);
+    }
+
+    float2 acc[27];
+#pragma unroll
+    for (int k = 0; k < 27; ++k) acc[k] = make_float2(0.f, 0.f);
+    float2 bsum = make_float2(0.f, 0.f);
+    bool ok = true;
+
+    for (int t = t_begin; t < t_end && ok; ++t) {
+        const int m = t - t_begin;                                      // dy plane; x planes m, m+1, m+2
+        if (tid == 0 && t + 1 < t_end) {                                // slots last read by step t-1
+            issue_x(m + 3);
+            issue_y(m + 1);
+        }
+        for (int n = (m == 0 ? 0 : m + 2); n <= m + 2; ++n)
+            if (!mbar_wait(smem_u32(&s.xbar[n % kWgXRing]), (n / kWgXRing) & 1)) ok = false;
+        if (!mbar_wait(smem_u32(&s.ybar[m % kWgYRing]), (m / kWgYRing) & 1)) ok = false;
+        if (!ok) {
+            atomicExch(&g_timeout_flag, 11);
+            break;
+        }
+        // this warp's row of dy: 16 words per lane
+        const uint32_t* gy = reinterpret_cast<const uint32_t*>(s.yp[m % kWgYRing]) + (yl * kWgTX) * (kCvCh / 2) + lane;
+        float2 g[kWgTX];
+#pragma unroll
+        for (int ox = 0; ox < kWgTX; ++ox) {
+            const uint32_t r = gy[ox * (kCvCh / 2)];
+            g[ox] = make_float2(__uint_as_float(r << 16), __uint_as_float(r & 0xffff0000u));
+            bsum.x += g[ox].x;
+            bsum.y += g[ox].y;
+        }
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+            const uint32_t* plane = reinterpret_cast<const uint32_t*>(s.xp[(m + i) % kWgXRing]);
+#pragma unroll
+            for (int j = 0; j < 3; ++j) {
+                const uint32_t* xrow = plane + ((yl + j) * (kWgTX + 2)) * (kCvCh / 2) + lane;
+#pragma unroll
+                for (int sx = 0; sx < kWgTX + 2; ++sx) {                // input column x0 - 1 + sx
+                    const uint32_t r = xrow[sx * (kCvCh / 2)];
+                    const float x_lo = __uint_as_float(r << 16), x_hi = __uint_as_float(r & 0xffff0000u);
+#pragma unroll
+                    for (int l = 0; l < 3; ++l) {
+                        const int ox = sx - l;                          // output column that tap l pairs with it
+                        if (ox < 0 || ox >= kWgTX) continue;
+                        float2& a = acc[(i * 3 + j) * 3 + l];
+                        fma2(a.x, a.y, x_lo, x_hi, g[ox].x, g[ox].y);
+                    }
+                }
+            }
+        }
+        __syncthreads();                                                // the oldest x slot and this dy slot are free
+    }
+    // rows of the tile beyond the grid carry zeros (TMA fill), so no masking is needed
+#pragma unroll
+    for (int k = 0; k < 27; ++k) {
+        atomicAdd(&s.red[k][lane * 2], acc[k].x);
+        atomicAdd(&s.red[k][lane * 2 + 1], acc[k].y);
+    }
+    atomicAdd(&s.red[27][lane * 2], bsum.x);
+    atomicAdd(&s.red[27][lane * 2 + 1], bsum.y);
+    __syncthreads();
+    for (int i = tid; i < 28 * (kCvCh / 4); i += 128) {
+        const int k = i / (kCvCh / 4), q = (i % (kCvCh / 4)) * 4;
+        float* dst = k < 27 ? dweight + static_cast<long long>(k) * C + c0 + q : (dbias ? dbias + c0 + q : nullptr);
+        if (dst)
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(s.red[k][q]), "f"(s.red[k][q + 1]),
+                         "f"(s.red[k][q + 2]), "f"(s.red[k][q + 3])
+                         : "memory");
+    }
+}
+
 template <typename T>
 cudaError_t launch_wgrad(const void* x, const void* dy, float* dweight, float* dbias, int Tn, int H, int W, int C,
                          const int kernel[3], cudaStream_t st) {
     const long long rows = static_cast<long long>(Tn) * H;
+    if (std::is_same<T, __nv_bfloat16>::value && kernel[0] == 3 && kernel[1] == 3 && kernel[2] == 3 && C % kCvCh == 0 &&
+        !std::getenv("DSA3D_WGRAD_PLAIN")) {
+        const int tiles = ((W + kWgTX - 1) / kWgTX) * ((H + kWgTY - 1) / kWgTY);
+        CUtensorMap map_x, map_dy;
+        if (tiles <= 65535 && make_map_activations(&map_x, x, Tn, H, W, C, kWgTX + 2, kWgTY + 2) &&
+            make_map_activations(&map_dy, dy, Tn, H, W, C, kWgTX, kWgTY)) {
+            int splits = 1;                                  // as in the forward: fill the GPU, keep chunks long
+            const long long columns = static_cast<long long>(C / kCvCh) * tiles;
+            while (columns * splits < 148 * 8 && Tn / (splits * 2) >= 12) splits *= 2;
+            const int t_chunk = (Tn + splits - 1) / splits;
+            const size_t smem = sizeof(WgradSmem) + 128;
+            cudaError_t e = cudaFuncSetAttribute(dwconv3d_wgrad333_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 static_cast<int>(smem));
+            if (e != cudaSuccess) return e;
+            const dim3 grid(C / kCvCh, tiles, (Tn + t_chunk - 1) / t_chunk);
+            dwconv3d_wgrad333_tma_kernel<<<grid, 128, smem, st>>>(map_x, map_dy, dweight, dbias, Tn, H, W, C, t_chunk);
+            return cudaGetLastError();
+        }
+    }
     const long long chunks = (rows + kWgradRows - 1) / kWgradRows;
     if (chunks > 65535) return cudaErrorInvalidConfiguration;
     int warps = kernel[0] * kernel[1];

@@ -38,11 +38,15 @@ def _workspace(nbytes):
                                           ((1, 1, 1, 8), (3, 3, 3)), ((2, 3, 2, 8), (5, 1, 7)),
                                           ((3, 4, 5, 72), (2, 4, 6)),
                                           ((6, 7, 19, 64), (3, 3, 3)), ((40, 6, 17, 64), (2, 4, 3)),
-                                          ((5, 9, 33, 128), (3, 7, 7)), ((70, 3, 5, 64), (3, 3, 1))])
+                                          ((5, 9, 33, 128), (3, 7, 7)), ((70, 3, 5, 64), (3, 3, 1)),
+                                          ((48, 4, 16, 64), (3, 3, 3)), ((9, 10, 35, 128), (3, 3, 3)),
+                                          ((1, 1, 1, 64), (3, 3, 3)), ((2, 5, 17, 192), (3, 3, 3))])
 def test_dwconv3d_backward_matches_the_oracle(dtype, shape, kernel):
     """Odd, even and mixed kernel sizes (the flipped kernel's centre differs from the forward's
     for even sizes), widths with and without a compiled-in slide, channel counts that take the
-    staged kernel for dx (bf16, multiples of 64) and ones that do not, more grid rows than one
+    staged kernels (bf16, multiples of 64 channels; the 3 x 3 x 3 weight gradient has one of its
+    own, here with grids that are not multiples of its 4 x 16 tile, a single frame, and enough
+    frames that the march is cut into chunks) and ones that do not, more grid rows than one
     warp's chunk."""
     T, H, W, C = shape
     taps = kernel[0] * kernel[1] * kernel[2]
