@@ -4,6 +4,7 @@ import pytest
 import torch
 
 import oracle
+from oracle import producer
 from paper_2607_22696_b200 import autograd as ops, inputs
 
 import parity_util as pu
@@ -46,3 +47,39 @@ def test_fixed_window_autograd_wrapper_matches_the_oracle():
     pu.assert_close("out", out, o_ref.view(shape), BF16)
     for name, leaf, ref in zip(("dq", "dk", "dv"), leaves, refs):
         pu.assert_close(name, leaf.grad, ref.view(shape), BF16, backward=True)
+
+
+@pytest.mark.parametrize("dtype", [BF16, F32])
+def test_producer_autograd_wrappers_match_the_oracle(dtype):
+    """Gradients of the convolution and of the linear layer through loss.backward()."""
+    T, H, W, C, kernel = 4, 5, 18, 64, (3, 3, 3)
+    x = inputs.normal((T, H, W, C), 172, 0, 1.0, dtype)
+    wc = inputs.normal((27, C), 172, 1, 0.3, F32)
+    bc = inputs.normal((C,), 172, 2, 0.5, F32)
+    dy = inputs.normal((T, H, W, C), 172, 3, 1.0, dtype)
+    leaves = [z.cuda().requires_grad_(True) for z in (x, wc, bc)]
+    y = ops.dwconv3d(*leaves, kernel)
+    y.backward(dy.cuda())
+    torch.cuda.synchronize()
+    pu.assert_close("y", y, producer.dwconv3d(x, wc, bc, kernel), dtype)
+    dx, dw, db = producer.dwconv3d_backward(x, wc, dy, kernel)
+    pu.assert_close("dx", leaves[0].grad, dx, dtype, backward=True)
+    for name, got, ref in (("dweight", leaves[1].grad, dw), ("dbias", leaves[2].grad, db)):
+        assert float((got.cpu().double() - ref).abs().max()) <= 1e-4 * max(float(ref.pow(2).mean().sqrt()), 1.0), name
+
+    tokens, O = 300, 54
+    u = inputs.normal((tokens, C), 173, 0, 1.0, dtype)
+    wl = inputs.normal((O, C), 173, 1, 0.2, dtype)
+    bl = inputs.normal((O,), 173, 2, 1.0, F32)
+    g = inputs.normal((tokens, O), 173, 3, 0.5, F32)
+    leaves = [z.cuda().requires_grad_(True) for z in (u, wl, bl)]
+    off = ops.offsets_linear(*leaves)
+    off.backward(g.cuda())
+    torch.cuda.synchronize()
+    ref = producer.offsets_linear(u, wl, bl)
+    assert float((off.detach().cpu().double() - ref).abs().max()) <= 1e-3 * max(float(ref.pow(2).mean().sqrt()), 1.0)
+    du, dwl, dbl = producer.offsets_linear_backward(u, wl, g)
+    pu.assert_close("du", leaves[0].grad, du, dtype, backward=True)
+    pu.assert_close("dw", leaves[1].grad, dwl, dtype, backward=True)
+    assert leaves[1].grad.dtype == dtype
+    assert float((leaves[2].grad.cpu().double() - dbl).abs().max()) <= 1e-4 * max(float(dbl.abs().max()), 1.0)
