@@ -1160,6 +1160,36 @@ transpose_to_bf16_kernel(const S* __restrict__ src, long long lds, long long row
     }
 }
 
+// fp32 [rows, cols] -> bf16 copy (row pitch ldd) plus fp32 column sums, for cols a multiple of 4:
+// a thread owns four neighbouring columns and walks down kCvtRows rows, so a block reads whole
+// rows front to back (one contiguous stream per block) and issues one atomic per column.
+constexpr int kCvtRows = 512;
+__global__ void __launch_bounds__(1024)
+convert_rows_bf16_kernel(const float* __restrict__ src, long long rows, int cols, __nv_bfloat16* __restrict__ dst,
+                         long long ldd, float* __restrict__ colsum) {
+    const long long rb = static_cast<long long>(blockIdx.x) * kCvtRows;
+    const long long re = rb + kCvtRows < rows ? rb + kCvtRows : rows;
+    for (int c = threadIdx.x * 4; c < cols; c += blockDim.x * 4) {
+        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float* sp = src + rb * cols + c;
+        __nv_bfloat16* dp = dst + rb * ldd + c;
+#pragma unroll 4
+        for (long long r = rb; r < re; ++r, sp += cols, dp += ldd) {
+            const float4 v = __ldg(reinterpret_cast<const float4*>(sp));
+            sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+            *reinterpret_cast<uint2*>(dp) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo),
+                                                       *reinterpret_cast<const uint32_t*>(&hi));
+        }
+        if (colsum) {
+            atomicAdd(colsum + c, sum.x);
+            atomicAdd(colsum + c + 1, sum.y);
+            atomicAdd(colsum + c + 2, sum.z);
+            atomicAdd(colsum + c + 3, sum.w);
+        }
+    }
+}
+
 // fp32 storage: plain loops, one thread per output element.
 __global__ void __launch_bounds__(256)
 linear_du_f32_kernel(const float* __restrict__ g, const float* __restrict__ w, float* __restrict__ du, long long M, int C,
@@ -1420,10 +1450,16 @@ int dsa3d_offsets_linear_backward(const void* u, const void* w, const float* dof
     for (long long s0 = 0; s0 < tokens; s0 += plan.slab) {
         const long long ns = tokens - s0 < plan.slab ? tokens - s0 : plan.slab;
         const unsigned row_blocks = static_cast<unsigned>((ns + kTrRowsPerBlock - 1) / kTrRowsPerBlock);
-        {   // doffsets slab -> bf16 copy and column sums
+        if (O % 4 == 0) {   // doffsets slab -> bf16 copy and column sums
+            int threads = ((O / 4 + 31) / 32) * 32;
+            if (threads > 1024) threads = 1024;
+            convert_rows_bf16_kernel<<<static_cast<unsigned>((ns + kCvtRows - 1) / kCvtRows), threads, 0, st>>>(
+                doffsets + s0 * O, ns, O, g, plan.ld_o, dbias);
+            if ((e = cudaGetLastError()) != cudaSuccess) return cuda_failed(e);
+        } else {            // rows that do not start on a 16-byte boundary: the pairwise kernel
             const dim3 grid((O + 63) / 64, row_blocks);
-            transpose_to_bf16_kernel<float><<<grid, 256, 0, st>>>(doffsets + s0 * O, O, ns, O, nullptr, 0,
-                                                                  (du || dw) ? g : nullptr, plan.ld_o, dbias);
+            transpose_to_bf16_kernel<float><<<grid, 256, 0, st>>>(doffsets + s0 * O, O, ns, O, nullptr, 0, g, plan.ld_o,
+                                                                  dbias);
             if ((e = cudaGetLastError()) != cudaSuccess) return cuda_failed(e);
         }
         if (du) {                                                    // du[slab] = g . (w^T)^T
