@@ -149,3 +149,49 @@ def test_producer_entry_points_reject_bad_arguments_without_launching(lib):
     assert res(a, a, a, a, None, 4, 8, 8, 2, 32, win, a, a, 0, None) == 1  # the term itself is required
     assert res(a, a, a, a, a + 2, 4, 8, 8, 2, 32, win, a, a, 0, None) == 4
     assert res(a, a, a, a, a, 4, 8, 8, 2, 48, win, a, a, 0, None) == 3     # head size not supported
+
+
+def test_producer_backward_entry_points_reject_bad_arguments_without_launching(lib):
+    """Gradients of the convolution and of the linear layer: every check runs before the first
+    launch or copy (fake aligned addresses, never dereferenced), and the workspace queries need
+    no device."""
+    a = 4096
+    win = (ctypes.c_int * 3)(3, 3, 3)
+    vp, ci, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    lib.dsa3d_dwconv3d_backward_workspace_bytes.restype = sz
+    lib.dsa3d_dwconv3d_backward_workspace_bytes.argtypes = [ci, ctypes.POINTER(ci)]
+    assert lib.dsa3d_dwconv3d_backward_workspace_bytes(64, win) >= 27 * 64 * 4
+    assert lib.dsa3d_dwconv3d_backward_workspace_bytes(0, win) == 0
+    lib.dsa3d_dwconv3d_backward.restype = ci
+    lib.dsa3d_dwconv3d_backward.argtypes = [vp, vp, vp, ci, ci, ci, ci, ctypes.POINTER(ci), vp, vp, vp, vp, sz, ci, vp]
+    conv = lambda *args: lib.dsa3d_dwconv3d_backward(*args)
+    assert conv(a, a, None, 2, 2, 2, 8, win, a, a, None, a, 1 << 20, 1, None) == 1      # dy is required
+    assert conv(a, a, a, 2, 2, 2, 8, win, a, None, None, None, 0, 1, None) == 1         # dx needs a workspace
+    assert conv(a, a, a, 2, 2, 2, 8, win, None, None, a, None, 0, 1, None) == 1         # dbias needs dweight
+    assert conv(None, a, a, 2, 2, 2, 8, win, None, a, None, None, 0, 1, None) == 1      # dweight needs x
+    assert conv(a, a, a, 2, 2, 2, 12, win, a, a, None, a, 1 << 20, 1, None) == 2        # channels
+    assert conv(a, a, a, 2, 2, 2, 8, (ctypes.c_int * 3)(3, 16, 3), a, a, None, a, 1 << 20, 1, None) == 2
+    assert conv(a, a, a, 2, 2, 2, 8, win, a, a, None, a, 1 << 20, 9, None) == 3         # dtype
+    assert conv(a, a, a + 8, 2, 2, 2, 8, win, a, a, None, a, 1 << 20, 1, None) == 4     # misaligned dy
+    assert conv(a, a, a, 2, 2, 2, 8, win, a, None, None, a, 16, 1, None) == 5           # workspace too small
+
+    lib.dsa3d_offsets_linear_backward_workspace_bytes.restype = sz
+    lib.dsa3d_offsets_linear_backward_workspace_bytes.argtypes = [ctypes.c_longlong, ci, ci, ci]
+    need = lib.dsa3d_offsets_linear_backward_workspace_bytes(1000, 64, 81, 1)
+    assert need >= 64 * 88 * 2 + 1000 * 88 * 2            # w^T and the bf16 copy, rows padded to 8 columns
+    assert lib.dsa3d_offsets_linear_backward_workspace_bytes(1000, 64, 81, 0) == 0      # fp32 needs none
+    # the slab bounds the workspace: beyond 262144 tokens it no longer grows
+    assert lib.dsa3d_offsets_linear_backward_workspace_bytes(10 ** 7, 64, 81, 1) == \
+        lib.dsa3d_offsets_linear_backward_workspace_bytes(262144, 64, 81, 1)
+    lib.dsa3d_offsets_linear_backward.restype = ci
+    lib.dsa3d_offsets_linear_backward.argtypes = [vp, vp, vp, ctypes.c_longlong, ci, ci, vp, vp, vp, vp, sz, ci, vp]
+    lin = lambda *args: lib.dsa3d_offsets_linear_backward(*args)
+    assert lin(a, a, None, 16, 64, 81, a, a, a, a, need, 1, None) == 1                  # doffsets is required
+    assert lin(a, None, a, 16, 64, 81, a, None, None, a, need, 1, None) == 1            # du needs w
+    assert lin(None, a, a, 16, 64, 81, None, a, None, a, need, 1, None) == 1            # dw needs u
+    assert lin(a, a, a, 0, 64, 81, a, a, a, a, need, 1, None) == 2
+    assert lin(a, a, a, 16, 60, 81, a, a, a, a, need, 1, None) == 2
+    assert lin(a, a, a, 16, 64, 81, a, a, a, a, need, 4, None) == 3
+    assert lin(a, a, a + 4, 16, 64, 81, a, a, a, a, need, 1, None) == 4
+    assert lin(a, a, a, 16, 64, 81, a, a, a, None, 0, 1, None) == 1                     # bf16 needs its workspace
+    assert lin(a, a, a, 16, 64, 81, a, a, a, a, 64, 1, None) == 5                       # too small
