@@ -448,7 +448,8 @@ dwconv3d_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* __re
 // takes the operand stream under the 64 B/clk an SM can pull from L2 (the one-CTA tiling needs
 // 93 B/clk at full tensor rate).
 constexpr int kPairStages = 6;
-// what the epilogue does with the fp32 accumulators: out = acc + bias in fp32; out = acc in bf16; out += acc
+// what the epilogue does with the fp32 accumulators: out = acc + bias in fp32 (bias required);
+// out = acc in bf16; out += acc
 constexpr int kGemmStoreF32 = 0, kGemmStoreBf16 = 1, kGemmAddF32 = 2;
 struct __align__(1024) GemmPairSmem {
     __nv_bfloat16 a[kPairStages][BM * BK];
@@ -592,8 +593,7 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
                     if (whole && (N & 3) == 0) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
-                            const float4 b4 = bias ? __ldg(reinterpret_cast<const float4*>(bias + n0 + c0 + j))
-                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+                            const float4 b4 = __ldg(reinterpret_cast<const float4*>(bias + n0 + c0 + j));
                             *reinterpret_cast<float4*>(dst + j) =
                                 make_float4(__uint_as_float(r[j]) + b4.x, __uint_as_float(r[j + 1]) + b4.y,
                                             __uint_as_float(r[j + 2]) + b4.z, __uint_as_float(r[j + 3]) + b4.w);
@@ -601,7 +601,7 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
-                            if (n0 + c0 + j < N) dst[j] = __uint_as_float(r[j]) + (bias ? __ldg(bias + n0 + c0 + j) : 0.0f);
+                            if (n0 + c0 + j < N) dst[j] = __uint_as_float(r[j]) + __ldg(bias + n0 + c0 + j);
                     }
                 } else if constexpr (MODE == kGemmStoreBf16) {
                     __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(out_raw) + row * N + n0 + c0;
