@@ -134,6 +134,28 @@ int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const flo
                     void* out_h, float* lse_h, void* dq_h, void* dk_h, void* dv_h, float* doffsets_h,
                     void* arena, size_t arena_bytes, int dtype, void* stream);
 
+/*
+ * dsa3d_step_host_pipelined: the same step, for a sequence of steps on one arena.  It differs
+ * in ordering only: its uploads do not wait for the work already in `stream` but only for the
+ * device buffers they overwrite, and nothing at its end makes `stream` wait for the downloads.
+ * The next call's K and V (the arena holds two copies of each) and first slabs therefore go up
+ * while this call's kernels run, and this call's dk and dv come down while the next call's
+ * forward runs - the two transfers a single step cannot hide.  The host INPUT buffers must be
+ * complete on the host when the call is made (no ordering with earlier work in `stream` is
+ * implied for them); all host buffers of a call must stay untouched until
+ * dsa3d_step_host_flush(stream) has been called and `stream` has completed, or until a later
+ * pipelined call has been flushed.  Results of call i are final on the host no later than that.
+ * A call whose arena, shape or dtype differs from the previous one first waits for all of the
+ * previous call.  dsa3d_step_host is this call followed by the flush, with the uploads ordered
+ * after `stream`.  dsa3d_step_host_flush makes `stream` wait for every transfer the calling
+ * thread's earlier steps queued.
+ */
+int dsa3d_step_host_pipelined(const void* q_h, const void* k_h, const void* v_h, const float* offsets_h,
+                              const void* dout_h, int T, int H, int W, int heads, int d, const int window[3],
+                              void* out_h, float* lse_h, void* dq_h, void* dk_h, void* dv_h, float* doffsets_h,
+                              void* arena, size_t arena_bytes, int dtype, void* stream);
+int dsa3d_step_host_flush(void* stream);
+
 /* Device scratch bytes dsa3d_step_host needs (0 for arguments the library would reject). */
 size_t dsa3d_step_host_arena_bytes(int T, int H, int W, int heads, int d, const int window[3],
                                    int dtype);

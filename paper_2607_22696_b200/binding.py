@@ -48,6 +48,10 @@ def load():
     lib.dsa3d_backward_workspace_bytes.argtypes = [i, i, i, i, i, win, i]
     lib.dsa3d_step_host.restype = i
     lib.dsa3d_step_host.argtypes = [p, p, p, p, p, i, i, i, i, i, win, p, p, p, p, p, p, p, sz, i, p]
+    lib.dsa3d_step_host_pipelined.restype = i
+    lib.dsa3d_step_host_pipelined.argtypes = [p, p, p, p, p, i, i, i, i, i, win, p, p, p, p, p, p, p, sz, i, p]
+    lib.dsa3d_step_host_flush.restype = i
+    lib.dsa3d_step_host_flush.argtypes = [p]
     lib.dsa3d_step_host_arena_bytes.restype = sz
     lib.dsa3d_step_host_arena_bytes.argtypes = [i, i, i, i, i, win, i]
     lib.dsa3d_set_profile_events.restype = i
@@ -316,16 +320,13 @@ def dsa3d_step_host_arena_bytes(T, H, W, heads, d, window, dtype) -> int:
     return int(load().dsa3d_step_host_arena_bytes(T, H, W, heads, d, _window(window), code))
 
 
-def dsa3d_step_host(q_h, k_h, v_h, offsets_h, dout_h, T, H, W, heads, d, window,
-                    out_h, lse_h, dq_h, dk_h, dv_h, doffsets_h, arena, stream=None) -> None:
-    """Forward + backward from HOST tensors (pinned for speed) through a caller-owned
-    device arena (a CUDA uint8 tensor); see include/dsa3d.h.  Asynchronous on `stream`."""
-    lib = load()
+def _step_host(fn, q_h, k_h, v_h, offsets_h, dout_h, T, H, W, heads, d, window,
+               out_h, lse_h, dq_h, dk_h, dv_h, doffsets_h, arena, stream) -> None:
     dt = q_h.dtype
     n = T * H * W * heads
     P = int(window[0]) * int(window[1]) * int(window[2])
     f32 = torch.float32
-    _check(lib.dsa3d_step_host(
+    _check(fn(
         _host_ptr(q_h, "q_h", n * d, dt), _host_ptr(k_h, "k_h", n * d, dt), _host_ptr(v_h, "v_h", n * d, dt),
         _host_ptr(offsets_h, "offsets_h", n * P * 3, f32), _host_ptr(dout_h, "dout_h", n * d, dt),
         T, H, W, heads, d, _window(window),
@@ -333,6 +334,26 @@ def dsa3d_step_host(q_h, k_h, v_h, offsets_h, dout_h, T, H, W, heads, d, window,
         _host_ptr(dq_h, "dq_h", n * d, dt), _host_ptr(dk_h, "dk_h", n * d, dt),
         _host_ptr(dv_h, "dv_h", n * d, dt), _host_ptr(doffsets_h, "doffsets_h", n * P * 3, f32),
         _ptr(arena, "arena"), arena.numel() * arena.element_size(), _DTYPES[dt], _stream(stream)))
+
+
+def dsa3d_step_host(q_h, k_h, v_h, offsets_h, dout_h, T, H, W, heads, d, window,
+                    out_h, lse_h, dq_h, dk_h, dv_h, doffsets_h, arena, stream=None) -> None:
+    """Forward + backward from HOST tensors (pinned for speed) through a caller-owned
+    device arena (a CUDA uint8 tensor); see include/dsa3d.h.  Asynchronous on `stream`."""
+    _step_host(load().dsa3d_step_host, q_h, k_h, v_h, offsets_h, dout_h, T, H, W, heads, d, window,
+               out_h, lse_h, dq_h, dk_h, dv_h, doffsets_h, arena, stream)
+
+
+def dsa3d_step_host_pipelined(q_h, k_h, v_h, offsets_h, dout_h, T, H, W, heads, d, window,
+                              out_h, lse_h, dq_h, dk_h, dv_h, doffsets_h, arena, stream=None) -> None:
+    """The same step for a sequence of steps on one arena: transfers overlap the neighbouring
+    calls' kernels; results are final after dsa3d_step_host_flush + stream completion."""
+    _step_host(load().dsa3d_step_host_pipelined, q_h, k_h, v_h, offsets_h, dout_h, T, H, W, heads, d, window,
+               out_h, lse_h, dq_h, dk_h, dv_h, doffsets_h, arena, stream)
+
+
+def dsa3d_step_host_flush(stream=None) -> None:
+    _check(load().dsa3d_step_host_flush(_stream(stream)))
 
 
 def dsa3d_forward_host_arena_bytes(T, H, W, heads, d, window, dtype) -> int:

@@ -361,7 +361,7 @@ size_t round256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
 // Layout of the device arena of dsa3d_step_host: offsets of each buffer, total in `total`.
 struct Arena {
-    size_t q, k, v, dout, out, dq, dk, dv, offsets, doffsets, lse, workspace, total;
+    size_t q, k, v, k2, v2, dout, out, dq, dk, dv, offsets, doffsets, lse, workspace, total;
     size_t row_bytes, off_bytes, lse_bytes, ws_bytes;
 };
 
@@ -377,7 +377,8 @@ Arena arena_layout(const dsa3d::Problem& pr, int dtype) {
         a.ws_bytes = backward_workspace(tiled, dtype, true).total;
     }
     size_t at = 0;
-    size_t* rows[8] = {&a.q, &a.k, &a.v, &a.dout, &a.out, &a.dq, &a.dk, &a.dv};
+    // K and V twice: the pipelined step uploads the next call's K/V while this call's kernels read theirs
+    size_t* rows[10] = {&a.q, &a.k, &a.v, &a.k2, &a.v2, &a.dout, &a.out, &a.dq, &a.dk, &a.dv};
     for (size_t* r : rows) { *r = at; at += round256(a.row_bytes); }
     a.offsets = at; at += round256(a.off_bytes);
     a.doffsets = at; at += round256(a.off_bytes);
@@ -396,6 +397,16 @@ struct HostStep {
     cudaEvent_t start = nullptr, kv_ready = nullptr, out_done = nullptr;
     cudaEvent_t q_ready[kMaxSlabs] = {}, dout_ready[kMaxSlabs] = {}, fwd_done[kMaxSlabs] = {},
                 gather_done[kMaxSlabs] = {};
+    // ordering between one call and the next (a wait on an event never recorded is a no-op):
+    cudaEvent_t kv_free[2] = {};               // main: last kernel that reads K/V buffer b has run
+    cudaEvent_t slab_in_free[kMaxSlabs] = {};  // main: q/offsets/dout of slab s consumed
+    cudaEvent_t slab_dl_done[kMaxSlabs] = {};  // out: out/lse/dq/doffsets of slab s are on the host
+    cudaEvent_t finish_done = nullptr;         // main: dk/dv final on the device
+    cudaEvent_t dkdv_dl_done = nullptr;        // out: dk/dv are on the host
+    cudaEvent_t main_done = nullptr;           // main: end of the call's kernels
+    int kv_index = 0;                          // K/V buffer of the next call
+    const void* last_arena = nullptr;
+    long long last_shape[7] = {0, 0, 0, 0, 0, 0, 0};
 };
 thread_local HostStep g_host_step[8];
 
@@ -410,10 +421,12 @@ HostStep* host_step_resources() {
     if (!slot) return nullptr;                          // more than 8 devices used from one thread
     if (cudaStreamCreateWithFlags(&slot->in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
     if (cudaStreamCreateWithFlags(&slot->out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-    cudaEvent_t* single[3] = {&slot->start, &slot->kv_ready, &slot->out_done};
+    cudaEvent_t* single[8] = {&slot->start, &slot->kv_ready, &slot->out_done, &slot->finish_done, &slot->dkdv_dl_done,
+                              &slot->main_done, &slot->kv_free[0], &slot->kv_free[1]};
     for (cudaEvent_t* ev : single)
         if (cudaEventCreateWithFlags(ev, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-    cudaEvent_t* per_slab[4] = {slot->q_ready, slot->dout_ready, slot->fwd_done, slot->gather_done};
+    cudaEvent_t* per_slab[6] = {slot->q_ready, slot->dout_ready, slot->fwd_done, slot->gather_done, slot->slab_in_free,
+                                slot->slab_dl_done};
     for (cudaEvent_t* arr : per_slab)
         for (int i = 0; i < kMaxSlabs; ++i)
             if (cudaEventCreateWithFlags(&arr[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
@@ -429,10 +442,15 @@ size_t dsa3d_step_host_arena_bytes(int T, int H, int W, int heads, int d, const 
     return arena_layout(pr, dtype).total;
 }
 
-int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const float* offsets_h,
-                    const void* dout_h, int T, int H, int W, int heads, int d, const int window[3],
-                    void* out_h, float* lse_h, void* dq_h, void* dk_h, void* dv_h, float* doffsets_h,
-                    void* arena, size_t arena_bytes, int dtype, void* stream_) {
+namespace {
+
+// One step enqueued on `stream_` and the two side streams.  ordered_start: uploads wait for the
+// work already on the stream (the plain entry point); otherwise only for the buffers they
+// overwrite, so that they overlap the previous call's kernels (the pipelined entry point).
+int step_host_body(const void* q_h, const void* k_h, const void* v_h, const float* offsets_h,
+                   const void* dout_h, int T, int H, int W, int heads, int d, const int window[3],
+                   void* out_h, float* lse_h, void* dq_h, void* dk_h, void* dv_h, float* doffsets_h,
+                   void* arena, size_t arena_bytes, int dtype, void* stream_, bool ordered_start) {
     if (!q_h || !k_h || !v_h || !offsets_h || !dout_h || !out_h || !lse_h || !dq_h || !dk_h || !dv_h ||
         !doffsets_h || !arena)
         return DSA3D_ERR_NULL_POINTER;
@@ -476,15 +494,35 @@ int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const flo
     const char* off_hb = reinterpret_cast<const char*>(offsets_h);
     const char* dout_hb = static_cast<const char*>(dout_h);
 
-    DSA3D_TRY(cudaEventRecord(hs->start, stream));
-    DSA3D_TRY(cudaStreamWaitEvent(hs->in, hs->start, 0));
-    DSA3D_TRY(cudaStreamWaitEvent(hs->out, hs->start, 0));
-    DSA3D_TRY(cudaMemcpyAsync(base + a.k, k_h, a.row_bytes, cudaMemcpyHostToDevice, hs->in));
-    DSA3D_TRY(cudaMemcpyAsync(base + a.v, v_h, a.row_bytes, cudaMemcpyHostToDevice, hs->in));
+    // A call with another arena or shape than the previous one shares no per-slab ordering with
+    // it: wait for all of the previous call first.
+    const long long shape[7] = {T, H, W, heads, d, dtype, static_cast<long long>(window[0]) * 10000 + window[1] * 100 + window[2]};
+    bool same = hs->last_arena == arena;
+    for (int i = 0; i < 7; ++i) same = same && hs->last_shape[i] == shape[i];
+    if (!same) {
+        DSA3D_TRY(cudaStreamWaitEvent(hs->in, hs->main_done, 0));
+        DSA3D_TRY(cudaStreamWaitEvent(hs->in, hs->out_done, 0));
+        DSA3D_TRY(cudaStreamWaitEvent(stream, hs->out_done, 0));
+        hs->last_arena = arena;
+        for (int i = 0; i < 7; ++i) hs->last_shape[i] = shape[i];
+    }
+    if (ordered_start) {
+        DSA3D_TRY(cudaEventRecord(hs->start, stream));
+        DSA3D_TRY(cudaStreamWaitEvent(hs->in, hs->start, 0));
+        DSA3D_TRY(cudaStreamWaitEvent(hs->out, hs->start, 0));
+    }
+    const int kvb = hs->kv_index;
+    hs->kv_index ^= 1;
+    char* k_d = base + (kvb ? a.k2 : a.k);
+    char* v_d = base + (kvb ? a.v2 : a.v);
+    DSA3D_TRY(cudaStreamWaitEvent(hs->in, hs->kv_free[kvb], 0));
+    DSA3D_TRY(cudaMemcpyAsync(k_d, k_h, a.row_bytes, cudaMemcpyHostToDevice, hs->in));
+    DSA3D_TRY(cudaMemcpyAsync(v_d, v_h, a.row_bytes, cudaMemcpyHostToDevice, hs->in));
     DSA3D_TRY(cudaEventRecord(hs->kv_ready, hs->in));
     for (int s = 0; s < slabs; ++s) {
         const int f0 = s * slab_frames, f1 = f0 + slab_frames < T ? f0 + slab_frames : T;
         const size_t nf = static_cast<size_t>(f1 - f0);
+        DSA3D_TRY(cudaStreamWaitEvent(hs->in, hs->slab_in_free[s], 0));     // the previous call's use of this slab
         DSA3D_TRY(cudaMemcpyAsync(base + a.q + f0 * frame_row_bytes, q_hb + f0 * frame_row_bytes,
                                   nf * frame_row_bytes, cudaMemcpyHostToDevice, hs->in));
         DSA3D_TRY(cudaMemcpyAsync(base + a.offsets + f0 * frame_off_bytes, off_hb + f0 * frame_off_bytes,
@@ -495,6 +533,9 @@ int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const flo
         DSA3D_TRY(cudaEventRecord(hs->dout_ready[s], hs->in));
     }
 
+    // fp32 storage accumulates dk/dv in place: the previous call's download of them comes first.
+    // (bf16 accumulates in the workspace; its dk/dv are only written by backward_finish below.)
+    if (!bf16) DSA3D_TRY(cudaStreamWaitEvent(stream, hs->dkdv_dl_done, 0));
     st = backward_clear(plan, stream);
     if (st != DSA3D_OK) return st;
     DSA3D_TRY(cudaStreamWaitEvent(stream, hs->kv_ready, 0));
@@ -505,8 +546,8 @@ int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const flo
         const int f0 = s * slab_frames, f1 = f0 + slab_frames < T ? f0 + slab_frames : T;
         const size_t nf = static_cast<size_t>(f1 - f0);
         DSA3D_TRY(cudaStreamWaitEvent(stream, hs->q_ready[s], 0));
-        st = forward_frames(pr, base + a.q, base + a.k, base + a.v, off_d, base + a.out, lse_d, bf16, f0, f1,
-                            stream);
+        DSA3D_TRY(cudaStreamWaitEvent(stream, hs->slab_dl_done[s], 0));     // the previous call's results of this slab
+        st = forward_frames(pr, base + a.q, k_d, v_d, off_d, base + a.out, lse_d, bf16, f0, f1, stream);
         if (st != DSA3D_OK) return st;
         DSA3D_TRY(cudaEventRecord(hs->fwd_done[s], stream));
         DSA3D_TRY(cudaStreamWaitEvent(hs->out, hs->fwd_done[s], 0));
@@ -518,9 +559,10 @@ int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const flo
                                   cudaMemcpyDeviceToHost, hs->out));
 
         DSA3D_TRY(cudaStreamWaitEvent(stream, hs->dout_ready[s], 0));
-        st = backward_frames(plan, base + a.q, base + a.k, base + a.v, off_d, lse_d, base + a.dout, base + a.dq,
+        st = backward_frames(plan, base + a.q, k_d, v_d, off_d, lse_d, base + a.dout, base + a.dq,
                              doff_d, f0, f1, stream, hs->gather_done[s]);
         if (st != DSA3D_OK) return st;
+        DSA3D_TRY(cudaEventRecord(hs->slab_in_free[s], stream));
         DSA3D_TRY(cudaStreamWaitEvent(hs->out, hs->gather_done[s], 0));
         DSA3D_TRY(cudaMemcpyAsync(static_cast<char*>(dq_h) + f0 * frame_row_bytes,
                                   base + a.dq + f0 * frame_row_bytes, nf * frame_row_bytes,
@@ -528,15 +570,48 @@ int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const flo
         DSA3D_TRY(cudaMemcpyAsync(reinterpret_cast<char*>(doffsets_h) + f0 * frame_off_bytes,
                                   base + a.doffsets + f0 * frame_off_bytes, nf * frame_off_bytes,
                                   cudaMemcpyDeviceToHost, hs->out));
+        DSA3D_TRY(cudaEventRecord(hs->slab_dl_done[s], hs->out));
     }
-    DSA3D_TRY(cudaEventRecord(hs->out_done, hs->out));
+    DSA3D_TRY(cudaEventRecord(hs->kv_free[kvb], stream));                 // no later kernel of this call reads K/V
+    DSA3D_TRY(cudaStreamWaitEvent(stream, hs->dkdv_dl_done, 0));          // the previous call's dk/dv are on the host
     st = backward_finish(plan, base + a.dk, base + a.dv, stream);
     if (st != DSA3D_OK) return st;
-    DSA3D_TRY(cudaMemcpyAsync(dk_h, base + a.dk, a.row_bytes, cudaMemcpyDeviceToHost, stream));
-    DSA3D_TRY(cudaMemcpyAsync(dv_h, base + a.dv, a.row_bytes, cudaMemcpyDeviceToHost, stream));
-    DSA3D_TRY(cudaStreamWaitEvent(stream, hs->out_done, 0));     // the step is over when `stream` is
+    DSA3D_TRY(cudaEventRecord(hs->finish_done, stream));
+    DSA3D_TRY(cudaEventRecord(hs->main_done, stream));
+    DSA3D_TRY(cudaStreamWaitEvent(hs->out, hs->finish_done, 0));
+    DSA3D_TRY(cudaMemcpyAsync(dk_h, base + a.dk, a.row_bytes, cudaMemcpyDeviceToHost, hs->out));
+    DSA3D_TRY(cudaMemcpyAsync(dv_h, base + a.dv, a.row_bytes, cudaMemcpyDeviceToHost, hs->out));
+    DSA3D_TRY(cudaEventRecord(hs->dkdv_dl_done, hs->out));
+    DSA3D_TRY(cudaEventRecord(hs->out_done, hs->out));
 #undef DSA3D_TRY
     return DSA3D_OK;
+}
+
+}  // namespace
+
+int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const float* offsets_h,
+                    const void* dout_h, int T, int H, int W, int heads, int d, const int window[3],
+                    void* out_h, float* lse_h, void* dq_h, void* dk_h, void* dv_h, float* doffsets_h,
+                    void* arena, size_t arena_bytes, int dtype, void* stream) {
+    const int rc = step_host_body(q_h, k_h, v_h, offsets_h, dout_h, T, H, W, heads, d, window, out_h, lse_h, dq_h, dk_h,
+                                  dv_h, doffsets_h, arena, arena_bytes, dtype, stream, true);
+    if (rc != DSA3D_OK) return rc;
+    return dsa3d_step_host_flush(stream);                        // the step is over when `stream` is
+}
+
+int dsa3d_step_host_pipelined(const void* q_h, const void* k_h, const void* v_h, const float* offsets_h,
+                              const void* dout_h, int T, int H, int W, int heads, int d, const int window[3],
+                              void* out_h, float* lse_h, void* dq_h, void* dk_h, void* dv_h, float* doffsets_h,
+                              void* arena, size_t arena_bytes, int dtype, void* stream) {
+    return step_host_body(q_h, k_h, v_h, offsets_h, dout_h, T, H, W, heads, d, window, out_h, lse_h, dq_h, dk_h, dv_h,
+                          doffsets_h, arena, arena_bytes, dtype, stream, false);
+}
+
+int dsa3d_step_host_flush(void* stream) {
+    HostStep* hs = host_step_resources();
+    if (!hs) return cuda_failed(cudaGetLastError());
+    const cudaError_t e = cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), hs->out_done, 0);
+    return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
 }
 
 // Forward only on host buffers (inference / sampling): device arena = q, k, v, out rows,

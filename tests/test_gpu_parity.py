@@ -228,6 +228,94 @@ def test_step_host_matches_the_device_entry_points(dtype, shape):
             z.fill_(float("nan"))
 
 
+@pytest.mark.parametrize("dtype,shape", [(BF16, (19, 9, 10, 2, 128)), (F32, (6, 10, 12, 3, 64)), (BF16, (1, 7, 9, 2, 64))])
+def test_pipelined_host_steps_match_the_device_entry_points(dtype, shape):
+    """A sequence of dsa3d_step_host_pipelined calls on one arena - different inputs per step,
+    each with its own host buffers - queued without waiting, then one flush: every step's results
+    must equal dsa3d_forward + dsa3d_backward on its own inputs (the next call's uploads overlap
+    this call's kernels, so a missing ordering between calls shows up as another step's data).
+    Then a call with another shape on the same arena (which must wait for the whole previous
+    call), and the plain entry point after pipelined ones."""
+    window = (3, 3, 3)
+    pin = lambda z: z.clone().pin_memory()
+
+    def make(shape_, seed):
+        q, k, v, off, dout = small_problem(*shape_, window, dtype, 1.3, seed)
+        dims = tuple(q.shape)
+        dev = [z.cuda() for z in (q, k, v, off, dout)]
+        out_d, lse_d = pu.gpu_forward(*dev[:4], dims, window)
+        g_d = pu.gpu_backward(*dev[:4], lse_d, dev[4], dims, window)
+        hout = {n: torch.full_like(q, float("nan")).pin_memory() for n in ("out", "dq", "dk", "dv")}
+        hout["lse"] = torch.full(dims[:4], float("nan")).pin_memory()
+        hout["doff"] = torch.full_like(off, float("nan")).pin_memory()
+        return dims, [pin(z) for z in (q, k, v, off, dout)], hout, (out_d.cpu(), lse_d.cpu(), [g.cpu() for g in g_d])
+
+    def check(hout, ref):
+        out_d, lse_d, g_d = ref
+        assert torch.equal(hout["out"], out_d) and torch.equal(hout["lse"], lse_d)
+        assert torch.equal(hout["dq"], g_d[0]) and torch.equal(hout["doff"], g_d[3])
+        for got, r in ((hout["dk"], g_d[1]), (hout["dv"], g_d[2])):
+            assert float((got.float() - r.float()).abs().max()) <= 2e-2 * float(r.float().abs().max())
+
+    other = (shape[0] + 2, shape[1], shape[2] + 1, shape[3], shape[4])
+    steps = [make(shape, 600 + i) for i in range(4)] + [make(other, 610)] + [make(shape, 611)]
+    nbytes = max(binding.dsa3d_step_host_arena_bytes(*st[0], window, dtype) for st in steps)
+    arena = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    for dims, hin, hout, _ in steps:
+        binding.dsa3d_step_host_pipelined(*hin, *dims, window, hout["out"], hout["lse"], hout["dq"], hout["dk"],
+                                          hout["dv"], hout["doff"], arena)
+    binding.dsa3d_step_host_flush()
+    torch.cuda.synchronize()
+    for _, _, hout, ref in steps:
+        check(hout, ref)
+    # the plain entry point right after pipelined calls, without a flush in between
+    dims, hin, hout, ref = make(shape, 620)
+    binding.dsa3d_step_host_pipelined(*steps[0][1], *steps[0][0], window, *(steps[0][2][n] for n in
+                                      ("out", "lse", "dq", "dk", "dv", "doff")), arena)
+    binding.dsa3d_step_host(*hin, *dims, window, hout["out"], hout["lse"], hout["dq"], hout["dk"], hout["dv"],
+                            hout["doff"], arena)
+    torch.cuda.synchronize()
+    check(hout, ref)
+    check(steps[0][2], steps[0][3])
+
+
+def test_pipelined_host_steps_with_transfers_long_enough_to_overlap():
+    """Three pipelined steps with different inputs at a size where each transfer and each kernel
+    takes of the order of a millisecond (40 MB per tensor, 8 slabs), so that uploads of step i+1
+    and downloads of step i really run beside kernels: per-query results must still be bitwise
+    those of the device entry points."""
+    shape, window = (16, 40, 60, 4, 128), (3, 3, 3)
+    T, H, W, heads, d = shape
+    n = T * H * W * heads
+    steps = []
+    for i in range(3):
+        q, k, v, dout = (inputs.normal(shape, 630 + i, j, 1.0, BF16) for j in range(4))
+        off = inputs.normal((T, H, W, heads, 27, 3), 630 + i, 4, 1.5, F32)
+        dev = [z.cuda() for z in (q, k, v, off, dout)]
+        out_d, lse_d = pu.gpu_forward(*dev[:4], shape, window)
+        g_d = pu.gpu_backward(*dev[:4], lse_d, dev[4], shape, window)
+        hout = {nm: torch.full(shape, float("nan"), dtype=BF16).pin_memory() for nm in ("out", "dq", "dk", "dv")}
+        hout["lse"] = torch.full(shape[:4], float("nan")).pin_memory()
+        hout["doff"] = torch.full(off.shape, float("nan")).pin_memory()
+        steps.append(([z.pin_memory() for z in (q, k, v, off, dout)], hout,
+                      (out_d.cpu(), lse_d.cpu(), [g.cpu() for g in g_d])))
+        del dev, out_d, lse_d, g_d
+    arena = torch.empty(binding.dsa3d_step_host_arena_bytes(*shape, window, BF16), dtype=torch.uint8, device="cuda")
+    for rounds in range(2):                                   # the second round reuses events and both K/V buffers
+        for hin, hout, _ in steps:
+            binding.dsa3d_step_host_pipelined(*hin, *shape, window, hout["out"], hout["lse"], hout["dq"], hout["dk"],
+                                              hout["dv"], hout["doff"], arena)
+        binding.dsa3d_step_host_flush()
+        torch.cuda.synchronize()
+        for _, hout, (out_d, lse_d, g_d) in steps:
+            assert torch.equal(hout["out"], out_d) and torch.equal(hout["lse"], lse_d)
+            assert torch.equal(hout["dq"], g_d[0]) and torch.equal(hout["doff"], g_d[3])
+            for got, r in ((hout["dk"], g_d[1]), (hout["dv"], g_d[2])):
+                assert float((got.float() - r.float()).abs().max()) <= 2e-2 * float(r.float().abs().max())
+            for z in hout.values():
+                z.fill_(float("nan"))
+
+
 @pytest.mark.parametrize("dtype,d", [(BF16, 128), (BF16, 64), (F32, 32)])
 def test_integer_positions_mixed_with_real_ones(dtype, d):
     """The forward takes chunks of samples that all sit on grid positions through a batched
