@@ -454,6 +454,7 @@ constexpr int kGemmStoreF32 = 0, kGemmStoreBf16 = 1, kGemmAddF32 = 2;
 struct __align__(1024) GemmPairSmem {
     __nv_bfloat16 a[kPairStages][BM * BK];
     __nv_bfloat16 b[kPairStages][(kMaxBN / 2) * BK];
+    float stage_out[4][2][32 * 32];        // per epilogue warp: two 32 x 32 fp32 boxes for TMA stores
     uint64_t full[kPairStages], empty[kPairStages], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
 };
@@ -463,6 +464,7 @@ struct __align__(1024) GemmPairSmem {
 template <int MODE, bool MN_MAJOR>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_constant__ CUtensorMap map_w,
+                         const __grid_constant__ CUtensorMap map_out, int tma_store,
                          const float* __restrict__ bias, void* __restrict__ out_raw, long long M, int N, int K, int BN,
                          long long m_tiles, int n_tiles, int ksplits) {
     extern __shared__ unsigned char raw[];
@@ -572,7 +574,7 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
         }
     } else {
         const int quarter = warp & 3;
-        uint32_t local = 0;
+        uint32_t local = 0, boxes = 0;
         for (long long unit = pair; unit < tiles; unit += pairs, ++local) {
             const uint32_t buf = local & 1;
             const long long tile = unit / ksplits;
@@ -586,9 +588,38 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
                 tmem_load_32(tmem + (static_cast<uint32_t>(quarter * 32) << 16) + buf * kMaxBN + c0, r);
-                if (row >= M) continue;
                 const bool whole = n0 + c0 + 32 <= N;
                 if constexpr (MODE == kGemmStoreF32) {
+                    if (tma_store) {
+                        // the warp's 32 x 32 block goes through shared memory (128-byte rows, 16-byte
+                        // chunks swizzled by the row as the tensor map expects) and out as one TMA box:
+                        // whole 128-byte lines per row instead of 32 scattered 16-byte pieces per store
+                        if (n0 + c0 >= N || row - lane >= M) continue;      // nothing of this box is inside
+                        unsigned char* stg = reinterpret_cast<unsigned char*>(s.stage_out[quarter][boxes & 1]);
+                        if (lane == 0) tma_store_wait_read<1>();           // the box before last has left this buffer
+                        __syncwarp();
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            float4 b4;
+                            if (whole) {
+                                b4 = __ldg(reinterpret_cast<const float4*>(bias + n0 + c0 + 4 * j));
+                            } else {
+                                const int cb = n0 + c0 + 4 * j;
+                                b4 = make_float4(cb < N ? __ldg(bias + cb) : 0.f, cb + 1 < N ? __ldg(bias + cb + 1) : 0.f,
+                                                 cb + 2 < N ? __ldg(bias + cb + 2) : 0.f, cb + 3 < N ? __ldg(bias + cb + 3) : 0.f);
+                            }
+                            *reinterpret_cast<float4*>(stg + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                                make_float4(__uint_as_float(r[4 * j]) + b4.x, __uint_as_float(r[4 * j + 1]) + b4.y,
+                                            __uint_as_float(r[4 * j + 2]) + b4.z, __uint_as_float(r[4 * j + 3]) + b4.w);
+                        }
+                        fence_async_smem();
+                        __syncwarp();
+                        if (lane == 0)
+                            tma_store_2d(&map_out, smem_u32(stg), n0 + c0, static_cast<int>(row - lane));
+                        ++boxes;
+                        continue;
+                    }
+                    if (row >= M) continue;
                     float* dst = static_cast<float*>(out_raw) + row * N + n0 + c0;
                     if (whole && (N & 3) == 0) {
 #pragma unroll
@@ -604,6 +635,7 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
                             if (n0 + c0 + j < N) dst[j] = __uint_as_float(r[j]) + __ldg(bias + n0 + c0 + j);
                     }
                 } else if constexpr (MODE == kGemmStoreBf16) {
+                    if (row >= M) continue;
                     __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(out_raw) + row * N + n0 + c0;
                     if (whole && (N & 7) == 0) {
 #pragma unroll
@@ -623,6 +655,7 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
                             if (n0 + c0 + j < N) dst[j] = __float2bfloat16_rn(__uint_as_float(r[j]));
                     }
                 } else {                                     // kGemmAddF32: partial sums of a k-range
+                    if (row >= M) continue;
                     float* dst = static_cast<float*>(out_raw) + row * N + n0 + c0;
                     if (whole && (N & 3) == 0) {
 #pragma unroll
@@ -642,6 +675,7 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&s.acc_empty[buf]), 0));
         }
+        if (MODE == kGemmStoreF32 && tma_store && lane == 0) tma_store_wait_all();   // shared memory is read, stores done
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -696,6 +730,19 @@ bool make_map(CUtensorMap* map, const void* ptr, unsigned long long rows, unsign
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Row-major fp32 [rows, cols] output, boxes of 32 x 32, 128-byte swizzle (cols a multiple of 4).
+bool make_map_out_f32(CUtensorMap* map, void* ptr, unsigned long long rows, unsigned long long cols) {
+    EncodeTiledFn enc = encode_tiled();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 4};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // out[M, N] = A[M, K] . B[N, K]^T on pairs of CTAs; A and B row-major bf16 with row pitches lda, ldb
 // (elements, multiples of 8).  mode: what the epilogue does; ksplits: equal ranges of k-blocks per
 // output tile (> 1 only with kGemmAddF32).  Column tiles of equal width, a multiple of 32, at most 256.
@@ -733,10 +780,17 @@ cudaError_t launch_pair_gemm(const void* A, unsigned long long lda, const void* 
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    // fp32 + bias epilogue: 32 x 32 boxes by TMA when the rows of the output are 16-byte multiples
+    CUtensorMap map_out = map_a;
+    int tma_store = 0;
+    if (mode == kGemmStoreF32 && (N & 3) == 0 && !std::getenv("DSA3D_GEMM_PLAIN_STORES") &&
+        make_map_out_f32(&map_out, out, static_cast<unsigned long long>(M), static_cast<unsigned long long>(N)))
+        tma_store = 1;
     auto launch = [&](auto kernel) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
-        return cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, bias, out, M, N, K, BN, m_tiles, n_tiles, ksplits);
+        return cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_out, tma_store, bias, out, M, N, K, BN, m_tiles, n_tiles,
+                                  ksplits);
     };
     if (mn_major) return launch(offsets_gemm_pair_kernel<kGemmAddF32, true>);
     if (mode == kGemmStoreF32) return launch(offsets_gemm_pair_kernel<kGemmStoreF32, false>);

@@ -51,6 +51,21 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
     d |= static_cast<uint64_t>(2) << 61;            // 128-byte swizzle
     return d;
 }
+// TMA store of a 2-D box from shared memory (bulk async-group of the issuing thread); rows and
+// columns beyond the tensor's extent are clipped.  The caller makes its shared-memory writes
+// visible to the async proxy first (fence_async_smem) and must not reuse the buffer before
+// tma_store_wait_read lets it.
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+template <int N> __device__ __forceinline__ void tma_store_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 // The same for an MN-major tile: the operand's M (or N) index runs along the 128-byte rows, 64
 // elements per swizzle atom, and its K index along the rows; 8-row groups 1024 bytes apart
 // (stride byte offset), atoms of 64 further M/N elements `atom_stride` bytes apart (leading
