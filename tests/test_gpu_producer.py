@@ -64,15 +64,19 @@ def test_dwconv3d_staged_kernel_matches_the_oracle(shape, kernel):
     assert torch.equal(guard.cpu(), torch.full((64,), 3.0))
 
 
-@pytest.fixture(params=["pair", "one_cta"])
+@pytest.fixture(params=["pair", "pair_plain_stores", "one_cta"])
 def gemm_variant(request):
-    """Both tilings of the tensor-core linear layer: pairs of CTAs (the default) and one CTA
-    per tile (forced by an environment switch read at every call)."""
+    """The tilings of the tensor-core linear layer: pairs of CTAs with the epilogue leaving by
+    TMA stores (the default; output counts that are not a multiple of 4 take plain stores by
+    themselves), the same with plain stores forced, and one CTA per tile (environment switches
+    read at every call)."""
     import os
-    if request.param == "one_cta":
-        os.environ["DSA3D_GEMM_ONE_CTA"] = "1"
+    switch = {"one_cta": "DSA3D_GEMM_ONE_CTA", "pair_plain_stores": "DSA3D_GEMM_PLAIN_STORES"}.get(request.param)
+    if switch:
+        os.environ[switch] = "1"
     yield request.param
-    os.environ.pop("DSA3D_GEMM_ONE_CTA", None)
+    if switch:
+        os.environ.pop(switch, None)
 
 
 @pytest.mark.parametrize("tokens,C,O", [(300, 192, 162), (128, 64, 32), (1000, 256, 1296), (77, 200, 40),
