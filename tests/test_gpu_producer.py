@@ -38,11 +38,23 @@ def test_dwconv3d_matches_the_oracle(dtype, shape, kernel):
         pu.assert_close("dwconv3d", y, ref, dtype)
 
 
+@pytest.fixture(params=["default", "general"])
+def conv_variant(request):
+    """3 x 3 x 3 kernels take a kernel of their own by default (weights in registers); the
+    general staged kernel is forced by an environment switch read at every call."""
+    import os
+    if request.param == "general":
+        os.environ["DSA3D_CONV_GENERAL"] = "1"
+    yield request.param
+    os.environ.pop("DSA3D_CONV_GENERAL", None)
+
+
 @pytest.mark.parametrize("shape,kernel", [((6, 7, 19, 64), (3, 3, 3)), ((48, 4, 16, 64), (3, 3, 3)),
+                                          ((1, 1, 1, 64), (3, 3, 3)), ((9, 10, 35, 128), (3, 3, 3)),
                                           ((5, 9, 33, 128), (3, 7, 7)), ((4, 5, 6, 64), (1, 1, 1)),
                                           ((9, 3, 40, 192), (5, 3, 5)), ((2, 1, 1, 64), (7, 5, 7)),
                                           ((40, 6, 17, 64), (2, 4, 3))])
-def test_dwconv3d_staged_kernel_matches_the_oracle(shape, kernel):
+def test_dwconv3d_staged_kernel_matches_the_oracle(shape, kernel, conv_variant):
     """bf16 with a multiple of 64 channels takes the kernel that stages planes in shared
     memory with TMA and marches along t: grids that are not multiples of the 4 x 16 tile,
     fewer frames than kernel taps, even kernel sizes, and grids small enough that the march
