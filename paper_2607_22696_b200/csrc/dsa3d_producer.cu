@@ -1173,7 +1173,12 @@ dwconv3d_333_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
                         const int ox = sx - l;                          // output that tap l maps this input to
                         if (ox < 0 || ox >= kWgTX) continue;
                         const float2 w2 = wv[(i * 3 + j) * 3 + l];
+#ifdef DSA3D_CONV3_PLAIN_FMA
+                        acc[ox].x = fmaf(x_lo, w2.x, acc[ox].x);
+                        acc[ox].y = fmaf(x_hi, w2.y, acc[ox].y);
+#else
                         fma2(acc[ox].x, acc[ox].y, x_lo, x_hi, w2.x, w2.y);
+#endif
                     }
                 }
             }
