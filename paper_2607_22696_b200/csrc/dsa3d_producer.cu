@@ -635,6 +635,32 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
                             if (n0 + c0 + j < N) dst[j] = __uint_as_float(r[j]) + __ldg(bias + n0 + c0 + j);
                     }
                 } else if constexpr (MODE == kGemmStoreBf16) {
+                    if (tma_store) {
+                        // 32 rows x 64 bytes through shared memory (64-byte swizzle: the 16-byte chunk index
+                        // is XORed with bits 1-2 of the row) and out as one TMA box
+                        if (n0 + c0 >= N || row - lane >= M) continue;
+                        unsigned char* stg = reinterpret_cast<unsigned char*>(s.stage_out[quarter][boxes & 1]);
+                        if (lane == 0) tma_store_wait_read<1>();
+                        __syncwarp();
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * j + 2 * e]),
+                                                                               __uint_as_float(r[8 * j + 2 * e + 1]));
+                                w[e] = *reinterpret_cast<const uint32_t*>(&h);
+                            }
+                            *reinterpret_cast<uint4*>(stg + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4)) =
+                                make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                        fence_async_smem();
+                        __syncwarp();
+                        if (lane == 0)
+                            tma_store_2d(&map_out, smem_u32(stg), n0 + c0, static_cast<int>(row - lane));
+                        ++boxes;
+                        continue;
+                    }
                     if (row >= M) continue;
                     __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(out_raw) + row * N + n0 + c0;
                     if (whole && (N & 7) == 0) {
@@ -675,7 +701,7 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&s.acc_empty[buf]), 0));
         }
-        if (MODE == kGemmStoreF32 && tma_store && lane == 0) tma_store_wait_all();   // shared memory is read, stores done
+        if (MODE != kGemmAddF32 && tma_store && lane == 0) tma_store_wait_all();     // shared memory is read, stores done
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -743,6 +769,19 @@ bool make_map_out_f32(CUtensorMap* map, void* ptr, unsigned long long rows, unsi
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Row-major bf16 [rows, cols] output, boxes of 32 x 32 (64-byte rows), 64-byte swizzle (cols a multiple of 8).
+bool make_map_out_bf16(CUtensorMap* map, void* ptr, unsigned long long rows, unsigned long long cols) {
+    EncodeTiledFn enc = encode_tiled();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // out[M, N] = A[M, K] . B[N, K]^T on pairs of CTAs; A and B row-major bf16 with row pitches lda, ldb
 // (elements, multiples of 8).  mode: what the epilogue does; ksplits: equal ranges of k-blocks per
 // output tile (> 1 only with kGemmAddF32).  Column tiles of equal width, a multiple of 32, at most 256.
@@ -785,6 +824,9 @@ cudaError_t launch_pair_gemm(const void* A, unsigned long long lda, const void* 
     int tma_store = 0;
     if (mode == kGemmStoreF32 && (N & 3) == 0 && !std::getenv("DSA3D_GEMM_PLAIN_STORES") &&
         make_map_out_f32(&map_out, out, static_cast<unsigned long long>(M), static_cast<unsigned long long>(N)))
+        tma_store = 1;
+    if (mode == kGemmStoreBf16 && (N & 7) == 0 && !std::getenv("DSA3D_GEMM_PLAIN_STORES") &&
+        make_map_out_bf16(&map_out, out, static_cast<unsigned long long>(M), static_cast<unsigned long long>(N)))
         tma_store = 1;
     auto launch = [&](auto kernel) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));

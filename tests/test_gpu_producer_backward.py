@@ -76,9 +76,20 @@ def test_dwconv3d_backward_matches_the_oracle(dtype, shape, kernel):
     assert torch.equal(dx2, dx)
 
 
+@pytest.fixture(params=["tma_stores", "plain_stores"])
+def store_variant(request):
+    """du leaves the contraction by TMA stores (default) or by plain stores (environment switch
+    read at every call)."""
+    import os
+    if request.param == "plain_stores":
+        os.environ["DSA3D_GEMM_PLAIN_STORES"] = "1"
+    yield request.param
+    os.environ.pop("DSA3D_GEMM_PLAIN_STORES", None)
+
+
 @pytest.mark.parametrize("tokens,C,O", [(300, 192, 162), (128, 64, 32), (1000, 256, 1296), (77, 200, 40),
                                         (513, 128, 520), (1, 8, 1), (260, 2048, 81), (2500, 72, 300)])
-def test_offsets_linear_backward_bf16_on_tensor_cores(tokens, C, O):
+def test_offsets_linear_backward_bf16_on_tensor_cores(tokens, C, O, store_variant):
     """Ragged sizes on every axis: output counts that are not a multiple of 8 (padded row
     pitch of the transposed copies), token counts that are not a multiple of the 64-token
     k-block, one and several column tiles, k-ranges split over several CTA pairs.  doffsets is
