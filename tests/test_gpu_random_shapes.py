@@ -66,3 +66,70 @@ def test_random_small_problems_match_the_oracle(seed):
         for name, got, want in zip(("dq", "dk", "dv"), g, refs[:3]):
             pu.assert_close(name, got, want.view(shape), dtype, backward=True)
         pu.assert_close("doffsets", doff, refs[3].view(T, H, W, heads, P, 3), dtype, backward=True)
+
+
+def _sum_close(name, got, ref, rel):
+    got = got.detach().cpu().double()
+    assert torch.isfinite(got).all(), name
+    worst = float((got - ref).abs().max())
+    bound = rel * max(float(ref.pow(2).mean().sqrt()), 1.0)
+    assert worst <= bound, f"{name}: max abs error {worst:.3e} > {bound:.3e}"
+
+
+@pytest.mark.parametrize("seed", [3, 4])
+def test_random_layers_around_the_operator_match_the_oracle(seed):
+    """The convolution and the linear layer, forward and backward, on random shapes: grids with
+    extents of 1, channel counts that are and are not multiples of 64 (staged and plain kernels),
+    kernel sizes with and without kernels of their own, token and output counts that are ragged
+    against every tile size of the contractions."""
+    from oracle import producer
+    rng = random.Random(seed)
+    for it in range(30):
+        dtype = rng.choice([BF16, BF16, F32])
+        T, H, W = rng.randint(1, 10), rng.randint(1, 9), rng.randint(1, 37)
+        C = rng.choice([8, 16, 24, 64, 64, 128, 192])
+        kernel = rng.choice([(3, 3, 3), (3, 3, 3), (1, 1, 1), (2, 2, 2), (3, 5, 5), (1, 3, 7), (5, 3, 1), (2, 3, 4)])
+        taps = kernel[0] * kernel[1] * kernel[2]
+        s = 2000 + 100 * seed + it
+        x = inputs.normal((T, H, W, C), s, 0, 1.0, dtype)
+        wc = inputs.normal((taps, C), s, 1, 0.3, F32)
+        bc = inputs.normal((C,), s, 2, 0.5, F32) if rng.random() < 0.7 else None
+        dy = inputs.normal((T, H, W, C), s, 3, 1.0, dtype)
+        xd, wd, dyd = x.cuda(), wc.cuda(), dy.cuda()
+        y = torch.full((T, H, W, C), float("nan"), dtype=dtype, device="cuda")
+        binding.dsa3d_dwconv3d_forward(xd, wd, None if bc is None else bc.cuda(), T, H, W, C, kernel, y)
+        dx = torch.full((T, H, W, C), float("nan"), dtype=dtype, device="cuda")
+        dw = torch.full((taps, C), float("nan"), dtype=F32, device="cuda")
+        db = torch.full((C,), float("nan"), dtype=F32, device="cuda")
+        ws = torch.empty(max(binding.dsa3d_dwconv3d_backward_workspace_bytes(C, kernel), 16), dtype=torch.uint8, device="cuda")
+        binding.dsa3d_dwconv3d_backward(xd, wd, dyd, T, H, W, C, kernel, dx, dw, db, ws)
+        torch.cuda.synchronize()
+        tag = f"case {it}: {dtype} grid {(T, H, W)} C {C} kernel {kernel}"
+        pu.assert_close(tag + " y", y, producer.dwconv3d(x, wc, bc, kernel), dtype)
+        r_dx, r_dw, r_db = producer.dwconv3d_backward(x, wc, dy, kernel)
+        pu.assert_close(tag + " dx", dx, r_dx, dtype, backward=True)
+        _sum_close(tag + " dweight", dw, r_dw, 1e-4)
+        _sum_close(tag + " dbias", db, r_db, 1e-4)
+
+        tokens, O = rng.randint(1, 700), rng.choice([1, 3, 27, 40, 81, 162, 300, 648])
+        u = inputs.normal((tokens, C), s, 4, 1.0, dtype)
+        wl = inputs.normal((O, C), s, 5, 0.2, dtype)
+        bl = inputs.normal((O,), s, 6, 1.0, F32)
+        g = inputs.normal((tokens, O), s, 7, 0.5, F32)
+        ud, wld, gd = u.cuda(), wl.cuda(), g.cuda()
+        off = torch.full((tokens, O), float("nan"), dtype=F32, device="cuda")
+        binding.dsa3d_offsets_linear_forward(ud, wld, bl.cuda(), tokens, C, O, off)
+        du = torch.full((tokens, C), float("nan"), dtype=dtype, device="cuda")
+        dwl = torch.full((O, C), float("nan"), dtype=F32, device="cuda")
+        dbl = torch.full((O,), float("nan"), dtype=F32, device="cuda")
+        wsl = torch.empty(max(binding.dsa3d_offsets_linear_backward_workspace_bytes(tokens, C, O, dtype), 16),
+                          dtype=torch.uint8, device="cuda")
+        binding.dsa3d_offsets_linear_backward(ud, wld, gd, tokens, C, O, du, dwl, dbl, wsl)
+        torch.cuda.synchronize()
+        assert binding.dsa3d_device_timeout_flag() == 0
+        tag = f"case {it}: {dtype} tokens {tokens} C {C} O {O}"
+        _sum_close(tag + " offsets", off, producer.offsets_linear(u, wl, bl), 1e-3 if dtype == BF16 else 1e-5)
+        r_du, r_dwl, r_dbl = producer.offsets_linear_backward(u, wl, g)
+        pu.assert_close(tag + " du", du, r_du, dtype, backward=True)
+        pu.assert_close(tag + " dw", dwl, r_dwl, dtype, backward=True)
+        _sum_close(tag + " dbias", dbl, r_dbl, 1e-5)
