@@ -145,6 +145,7 @@ int dsa3d_step_host(const void* q_h, const void* k_h, const void* v_h, const flo
  * implied for them); all host buffers of a call must stay untouched until
  * dsa3d_step_host_flush(stream) has been called and `stream` has completed, or until a later
  * pipelined call has been flushed.  Results of call i are final on the host no later than that.
+ * The arena must not be in use by other work queued in `stream` (the uploads do not wait for it).
  * A call whose arena, shape or dtype differs from the previous one first waits for all of the
  * previous call.  dsa3d_step_host is this call followed by the flush, with the uploads ordered
  * after `stream`.  dsa3d_step_host_flush makes `stream` wait for every transfer the calling

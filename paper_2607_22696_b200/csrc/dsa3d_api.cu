@@ -659,6 +659,10 @@ int dsa3d_forward_host(const void* q_h, const void* k_h, const void* v_h, const 
     const size_t frame_row_bytes = frame_rows * d * elt;
     const size_t frame_off_bytes = frame_rows * pr.P * 3 * sizeof(float);
     const size_t frame_lse_bytes = frame_rows * sizeof(float);
+    // transfers that pipelined steps may still have in flight on the side streams come first
+    // (this call may reuse their arena), and a later step shares no per-slab ordering with it
+    DSA3D_TRY(cudaStreamWaitEvent(stream, hs->out_done, 0));
+    hs->last_arena = nullptr;
     DSA3D_TRY(cudaEventRecord(hs->start, stream));
     DSA3D_TRY(cudaStreamWaitEvent(hs->in, hs->start, 0));
     DSA3D_TRY(cudaStreamWaitEvent(hs->out, hs->start, 0));
