@@ -83,3 +83,67 @@ def test_producer_autograd_wrappers_match_the_oracle(dtype):
     pu.assert_close("dw", leaves[1].grad, dwl, dtype, backward=True)
     assert leaves[1].grad.dtype == dtype
     assert float((leaves[2].grad.cpu().double() - dbl).abs().max()) <= 1e-4 * max(float(dbl.abs().max()), 1.0)
+
+
+def test_layer_module_equals_its_parts_and_its_gradients_follow_the_loss():
+    """The Eq. 1 module only chains the wrappers: its output equals the entry points called by
+    hand on the same tensors (bitwise), every parameter and input receives a finite gradient,
+    and output and gradients equal the same chain evaluated stage by stage in the fp64 oracle."""
+    from paper_2607_22696_b200 import binding
+    from paper_2607_22696_b200.layer import DeformableSlideAttention3D
+    T, H, W, heads, d, window = 4, 5, 6, 2, 32, (3, 3, 3)
+    hidden, N = heads * d, T * H * W
+    layer = DeformableSlideAttention3D(heads, d, window, (3, 3, 3), dtype=F32, seed=5)
+    with torch.no_grad():          # leave the zero start: offsets of a fraction of a cell, off the lattice
+        layer.offset_weight.copy_(inputs.normal(tuple(layer.offset_weight.shape), 180, 0, 0.05, F32).cuda())
+        layer.offset_bias.copy_(inputs.normal(tuple(layer.offset_bias.shape), 180, 1, 0.3, F32).cuda())
+    x = inputs.normal((T, H, W, hidden), 181, 0, 1.0, F32).cuda().requires_grad_(True)
+    q, k, v = (inputs.normal((T, H, W, heads, d), 181, i, 1.0, F32).cuda().requires_grad_(True) for i in (1, 2, 3))
+    probe = inputs.normal((T, H, W, heads, d), 181, 4, 1.0, F32).cuda()
+
+    out = layer(x, q, k, v)
+    # by hand through the binding
+    u = torch.empty_like(x)
+    binding.dsa3d_dwconv3d_forward(x.detach(), layer.offset_conv_weight.detach(), layer.offset_conv_bias.detach(),
+                                   T, H, W, hidden, (3, 3, 3), u)
+    off = torch.empty((N, heads * 27 * 3), dtype=F32, device="cuda")
+    binding.dsa3d_offsets_linear_forward(u, layer.offset_weight.detach(), layer.offset_bias.detach(), N, hidden,
+                                         heads * 27 * 3, off)
+    term = torch.empty_like(x)
+    binding.dsa3d_dwconv3d_forward(x.detach(), layer.term_conv_weight.detach(), layer.term_conv_bias.detach(),
+                                   T, H, W, hidden, (3, 3, 3), term)
+    ref = torch.empty_like(out)
+    lse = torch.empty((T, H, W, heads), dtype=F32, device="cuda")
+    binding.dsa3d_forward_residual(q.detach(), k.detach(), v.detach(), off, term, T, H, W, heads, d, window, ref, lse)
+    torch.cuda.synchronize()
+    assert torch.equal(out.detach(), ref)
+
+    (out * probe).sum().backward()
+    torch.cuda.synchronize()
+    leaves = dict(layer.named_parameters(), x=x, q=q, k=k, v=v)
+    for name, leaf in leaves.items():
+        assert leaf.grad is not None and torch.isfinite(leaf.grad).all(), name
+        assert float(leaf.grad.abs().max()) > 0, name
+
+    # the same chain in the fp64 oracle, stage by stage on its own intermediate results (fp32
+    # storage keeps the GPU's offsets within 1e-6 of the oracle's, so no sample changes cell)
+    par = {n: p.detach().cpu() for n, p in layer.named_parameters()}
+    xc, qc, kc, vc, pc = (z.detach().cpu() for z in (x, q, k, v, probe))
+    u_o = producer.dwconv3d(xc, par["offset_conv_weight"], par["offset_conv_bias"], (3, 3, 3))
+    off_o = producer.offsets_linear(u_o.view(N, hidden), par["offset_weight"], par["offset_bias"])
+    term_o = producer.dwconv3d(xc, par["term_conv_weight"], par["term_conv_bias"], (3, 3, 3))
+    off4 = off_o.view(N, heads, 27, 3).float()            # the operator takes its offsets in fp32
+    o_ref, _ = oracle.forward(qc.view(-1, heads, d), kc, vc, off4, T, H, W, heads, d, window)
+    pu.assert_close("layer output", out, o_ref.view(T, H, W, heads, d) + term_o.view(T, H, W, heads, d), F32)
+    dq_o, dk_o, dv_o, doff_o = oracle.backward(qc.view(-1, heads, d), kc, vc, off4, pc.view(-1, heads, d),
+                                               T, H, W, heads, d, window)
+    du_o, dwl_o, dbl_o = producer.offsets_linear_backward(u_o.view(N, hidden), par["offset_weight"], doff_o.view(N, -1))
+    dx1, dwc1, dbc1 = producer.dwconv3d_backward(xc, par["offset_conv_weight"], du_o.view(T, H, W, hidden), (3, 3, 3))
+    dx2, dwc2, dbc2 = producer.dwconv3d_backward(xc, par["term_conv_weight"], pc.view(T, H, W, hidden), (3, 3, 3))
+    want = {"offset_conv_weight": dwc1, "offset_conv_bias": dbc1, "term_conv_weight": dwc2, "term_conv_bias": dbc2,
+            "offset_weight": dwl_o, "offset_bias": dbl_o, "x": dx1 + dx2, "q": dq_o, "k": dk_o, "v": dv_o}
+    for name, ref in want.items():
+        got = leaves[name].grad.detach().cpu().double().reshape(-1)
+        ref = ref.reshape(-1)
+        bound = 1e-4 * max(float(ref.abs().max()), 1.0)
+        assert float((got - ref).abs().max()) <= bound, (name, float((got - ref).abs().max()), bound)
