@@ -473,10 +473,12 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
     const uint32_t rank = cluster_rank();                       // 0: leader (issues the MMAs)
     const int kblocks = (K + BK - 1) / BK;
     // a work unit is one 256 x BN output tile (m_tiles counts 256-row tiles) times one of
-    // `ksplits` equal ranges of k-blocks; units of a tile are neighbours so they share operands in L2
+    // `ksplits` equal ranges of k-blocks; the k-range is the slow index, so the units in flight at any
+    // time are different tiles walking through the same k-range: each operand block is fetched from
+    // DRAM once and found in L2 by the other tiles of its row or column
     const long long tiles = m_tiles * n_tiles * ksplits;
     auto k_range = [&](long long unit, int& kb0, int& kb1) {
-        const int ks = static_cast<int>(unit % ksplits);
+        const int ks = static_cast<int>(unit / (m_tiles * n_tiles));
         kb0 = static_cast<int>(static_cast<long long>(kblocks) * ks / ksplits);
         kb1 = static_cast<int>(static_cast<long long>(kblocks) * (ks + 1) / ksplits);
     };
@@ -503,7 +505,7 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
         if (lane == 0) {
             uint32_t it = 0;
             for (long long unit = pair; unit < tiles; unit += pairs) {
-                const long long tile = unit / ksplits;
+                const long long tile = unit % (m_tiles * n_tiles);
                 const int n0 = static_cast<int>(tile % n_tiles) * BN;
                 const long long m0 = (tile / n_tiles) * (2 * BM);
                 int kb0, kb1;
@@ -577,7 +579,7 @@ offsets_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_u, const __grid
         uint32_t local = 0, boxes = 0;
         for (long long unit = pair; unit < tiles; unit += pairs, ++local) {
             const uint32_t buf = local & 1;
-            const long long tile = unit / ksplits;
+            const long long tile = unit % (m_tiles * n_tiles);
             const int n0 = static_cast<int>(tile % n_tiles) * BN;
             const long long row = (tile / n_tiles) * (2 * BM) + rank * BM + quarter * 32 + lane;
             if (!mbar_wait(smem_u32(&s.acc_full[buf]), (local >> 1) & 1)) {
