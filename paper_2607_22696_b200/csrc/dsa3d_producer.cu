@@ -391,6 +391,7 @@ dwconv3d_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* __re
                 ok = false;
                 break;
             }
+        ok = __syncthreads_and(ok);                                     // all threads stop together or not at all
         float acc[kCvRX][8];
 #pragma unroll
         for (int r = 0; r < kCvRX; ++r)
@@ -1086,10 +1087,9 @@ dwconv3d_wgrad333_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __
         for (int n = (m == 0 ? 0 : m + 2); n <= m + 2; ++n)
             if (!mbar_wait(smem_u32(&s.xbar[n % kWgXRing]), (n / kWgXRing) & 1)) ok = false;
         if (!mbar_wait(smem_u32(&s.ybar[m % kWgYRing]), (m / kWgYRing) & 1)) ok = false;
-        if (!ok) {
-            atomicExch(&g_timeout_flag, 11);
-            break;
-        }
+        if (!ok) atomicExch(&g_timeout_flag, 11);
+        ok = __syncthreads_and(ok);                                     // all threads stop together or not at all
+        if (!ok) break;
         // this warp's row of dy: 16 words per lane
         const uint32_t* gy = reinterpret_cast<const uint32_t*>(s.yp[m % kWgYRing]) + (yl * kWgTX) * (kCvCh / 2) + lane;
         float2 g[kWgTX];
@@ -1195,10 +1195,9 @@ dwconv3d_333_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
         if (tid == 0 && m + kCv3Ring - 1 < planes) issue_x(m + kCv3Ring - 1);   // its slot was last read by output t-1
         for (int n = (m == 0 ? 0 : m + 2); n <= m + 2; ++n)
             if (!mbar_wait(smem_u32(&s.xbar[n % kCv3Ring]), (n / kCv3Ring) & 1)) ok = false;
-        if (!ok) {
-            atomicExch(&g_timeout_flag, 12);
-            break;
-        }
+        if (!ok) atomicExch(&g_timeout_flag, 12);
+        ok = __syncthreads_and(ok);                                     // all threads stop together or not at all
+        if (!ok) break;
         float2 acc[kWgTX];
 #pragma unroll
         for (int ox = 0; ox < kWgTX; ++ox) acc[ox] = bv;
