@@ -139,29 +139,31 @@ class ClockSampler:
 
 # ------------------------------------------------------------------- CPU oracle sampling
 
-def oracle_sample(wl, rows: int, device_for_generation):
+def oracle_sample(wl, rows: int, device_for_generation, frames: int = 1):
     """A bounded, exact sample of the workload for the CPU oracle: the first `rows` grid rows
-    of the middle frame as queries, evaluated on the crop of frames that their samples can
-    reach (exact, because no sample leaves the crop: |offset_t| is bounded by the largest
-    offset actually drawn for these queries).  Returns the cropped problem as CPU tensors."""
+    of `frames` consecutive frames from the middle one on as queries, evaluated on the crop of
+    frames that their samples can reach (exact, because no sample leaves the crop: |offset_t|
+    is bounded by the largest offset actually drawn for these queries).  Returns the cropped
+    problem as CPU tensors."""
     tq = wl.T // 2
     rows = max(1, min(rows, wl.H))
-    off_q = inputs.make_offsets(wl, device_for_generation, frames=(tq, tq + 1))[:, :rows].contiguous()
+    nf = max(1, min(frames, wl.T - tq))
+    off_q = inputs.make_offsets(wl, device_for_generation, frames=(tq, tq + nf))[:, :rows].contiguous()
     finite = off_q[torch.isfinite(off_q)]
     reach = int(math.floor(2 + wl.window[0] // 2 + (float(finite.abs().max()) if finite.numel() else 0.0)))
-    t0, t1 = max(0, tq - reach), min(wl.T, tq + reach + 1)
+    t0, t1 = max(0, tq - reach), min(wl.T, tq + nf - 1 + reach + 1)
     k = inputs.make_rows(wl, "k", device_for_generation, frames=(t0, t1)).cpu()
     v = inputs.make_rows(wl, "v", device_for_generation, frames=(t0, t1)).cpu()
-    q = inputs.make_rows(wl, "q", device_for_generation, frames=(tq, tq + 1))[:, :rows].contiguous().cpu()
-    dout = inputs.make_rows(wl, "dout", device_for_generation, frames=(tq, tq + 1))[:, :rows].contiguous().cpu()
+    q = inputs.make_rows(wl, "q", device_for_generation, frames=(tq, tq + nf))[:, :rows].contiguous().cpu()
+    dout = inputs.make_rows(wl, "dout", device_for_generation, frames=(tq, tq + nf))[:, :rows].contiguous().cpu()
     Tc = t1 - t0
-    qtok = ((tq - t0) * wl.H * wl.W + torch.arange(rows * wl.W)).to(torch.int64)
+    qtok = torch.cat([((tq + f - t0) * wl.H * wl.W + torch.arange(rows * wl.W)) for f in range(nf)]).to(torch.int64)
     return dict(q=q.view(-1, wl.heads, wl.d), k=k, v=v, offsets=off_q.cpu().view(-1, wl.heads, wl.P, 3),
                 dout=dout.view(-1, wl.heads, wl.d), qtok=qtok, dims=(Tc, wl.H, wl.W, wl.heads, wl.d),
-                tokens=rows * wl.W,
-                desc=f"{rows} grid rows ({rows * wl.W} query tokens, all {wl.heads} heads) of frame {tq}, "
-                     f"{'fwd+bwd incl. dK/dV' if wl.backward else 'forward only'}, on the exact {Tc}-frame "
-                     f"crop their samples reach")
+                tokens=nf * rows * wl.W,
+                desc=f"{rows} grid rows of each of {nf} frame(s) from frame {tq} on ({nf * rows * wl.W} query tokens, "
+                     f"all {wl.heads} heads), {'fwd+bwd incl. dK/dV' if wl.backward else 'forward only'}, on the exact "
+                     f"{Tc}-frame crop their samples reach")
 
 
 def time_oracle(sample, wl, backward=True):
@@ -421,7 +423,7 @@ def run_ours(args, wl):
     # --------------------------------------------------------------------- CPU baseline
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
-        sample = oracle_sample(wl, args.cpu_rows, dev)
+        sample = oracle_sample(wl, args.cpu_rows, dev, args.cpu_frames)
         dt, threads = time_oracle(sample, wl, wl.backward)
         cpu = {"value": sample["tokens"] / dt / 1e6, "unit": UNIT, "cores": threads, "kind": "oracle",
                "sample": sample["desc"], "seconds": dt}
@@ -634,7 +636,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="1080p_256f_bf16", choices=sorted(inputs.WORKLOADS))
-    ap.add_argument("--cpu-rows", type=int, default=32, help="grid rows of one frame the CPU baseline processes")
+    ap.add_argument("--cpu-rows", type=int, default=68, help="grid rows per frame the CPU baseline processes")
+    ap.add_argument("--cpu-frames", type=int, default=4, help="consecutive frames the CPU baseline takes its rows from")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

@@ -108,3 +108,41 @@ def test_head_sharding_over_two_gloo_ranks_reproduces_the_unsharded_result():
         r0, r1 = results[0], results[1]
     assert r0[0] == (0, 2) and r1[0] == (2, 3)
     assert r0[1] == 0.0 and r1[1] == 0.0
+
+
+def test_cpu_baseline_sample_is_an_exact_crop_of_the_workload():
+    """bench.py times the oracle on a crop of the workload (some rows of some frames as queries,
+    the frames their samples can reach as keys).  The crop must compute what the full problem
+    computes for those queries: same outputs, same query-side gradients."""
+    import importlib.util
+    import dataclasses
+    import oracle
+    from paper_2607_22696_b200 import inputs
+    spec = importlib.util.spec_from_file_location("bench_module", os.path.join(ROOT, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    wl = dataclasses.replace(inputs.WORKLOADS["tiny_f32"], T=12, H=5, W=6, sigma=0.8, seed=77)
+    sample = bench.oracle_sample(wl, 3, "cpu", frames=2)
+    Tc, H, W, heads, d = sample["dims"]
+    assert sample["tokens"] == 2 * 3 * W and Tc < wl.T
+    out_c, lse_c = oracle.forward(sample["q"], sample["k"], sample["v"], sample["offsets"], Tc, H, W, heads, d, wl.window,
+                                  qtok=sample["qtok"])
+    dq_c, _, _, doff_c = oracle.backward(sample["q"], sample["k"], sample["v"], sample["offsets"], sample["dout"],
+                                         Tc, H, W, heads, d, wl.window, qtok=sample["qtok"])
+    # the whole problem
+    q = inputs.make_rows(wl, "q", "cpu")
+    k = inputs.make_rows(wl, "k", "cpu")
+    v = inputs.make_rows(wl, "v", "cpu")
+    dout = inputs.make_rows(wl, "dout", "cpu")
+    off = inputs.make_offsets(wl, "cpu")
+    P = wl.window[0] * wl.window[1] * wl.window[2]
+    out_f, lse_f = oracle.forward(q.view(-1, heads, d), k, v, off.view(-1, heads, P, 3), wl.T, H, W, heads, d, wl.window)
+    dq_f, _, _, doff_f = oracle.backward(q.view(-1, heads, d), k, v, off.view(-1, heads, P, 3), dout.view(-1, heads, d),
+                                         wl.T, H, W, heads, d, wl.window)
+    tq = wl.T // 2
+    tok = torch.cat([(tq + f) * H * W + torch.arange(3 * W) for f in range(2)])
+    # positions are formed in fp32 from the frame index, so a frame index shifted by the crop moves
+    # the fractional parts by an ulp of the position: equal up to that, not bitwise
+    for name, got, ref in (("out", out_c, out_f.view(-1, heads, d)[tok]), ("lse", lse_c, lse_f.view(-1, heads)[tok]),
+                           ("dq", dq_c, dq_f.view(-1, heads, d)[tok]), ("doffsets", doff_c, doff_f.view(-1, heads, P, 3)[tok])):
+        assert float((got - ref).abs().max()) <= 1e-5 * max(float(ref.abs().max()), 1.0), name
