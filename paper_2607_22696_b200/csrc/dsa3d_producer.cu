@@ -1589,7 +1589,7 @@ int dsa3d_dwconv3d_backward(const void* x, const float* weight, const void* dy, 
         return DSA3D_ERR_BAD_SHAPE;
     if (dtype != DSA3D_F32 && dtype != DSA3D_BF16) return DSA3D_ERR_UNSUPPORTED;
     if (!aligned16(dy) || (x && !aligned16(x)) || (dx && !aligned16(dx)) || (dweight && !aligned16(dweight)) ||
-        (workspace && !aligned16(workspace)))
+        (dbias && !aligned16(dbias)) || (weight && !aligned16(weight)) || (workspace && !aligned16(workspace)))
         return DSA3D_ERR_MISALIGNED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int taps = kernel[0] * kernel[1] * kernel[2];

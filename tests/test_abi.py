@@ -173,6 +173,7 @@ def test_producer_backward_entry_points_reject_bad_arguments_without_launching(l
     assert conv(a, a, a, 2, 2, 2, 8, (ctypes.c_int * 3)(3, 16, 3), a, a, None, a, 1 << 20, 1, None) == 2
     assert conv(a, a, a, 2, 2, 2, 8, win, a, a, None, a, 1 << 20, 9, None) == 3         # dtype
     assert conv(a, a, a + 8, 2, 2, 2, 8, win, a, a, None, a, 1 << 20, 1, None) == 4     # misaligned dy
+    assert conv(a, a, a, 2, 2, 2, 8, win, None, a, a + 4, None, 0, 1, None) == 4        # misaligned dbias
     assert conv(a, a, a, 2, 2, 2, 8, win, a, None, None, a, 16, 1, None) == 5           # workspace too small
 
     lib.dsa3d_offsets_linear_backward_workspace_bytes.restype = sz
