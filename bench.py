@@ -43,10 +43,13 @@ UNIT = "Mtokens/s"
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes per (token, head) item, dram__bytes_read.sum + dram__bytes_write.sum of one ncu
-# capture per kernel on the profile_small_bf16 workload (profiles/*_profile_small_bf16.md).
-# Every kernel's traffic is proportional to the number of items, so a launch on another
-# workload with the same d and window is reported as items x these figures.
+# capture per kernel on the profile_small_bf16 workload (profiles/*_profile_small_bf16.md); a
+# launch on another workload with the same d and window is reported as items x these figures.
 NCU_DRAM_BYTES_PER_ITEM = {"forward_kernel": 1525.0, "backward_kernel": 2991.0, "scatter_tile_kernel": 12902.0}
+# The same two counters captured at the full size of the default workload (one pass per launch,
+# profiles/dram_traffic_1080p_256f_bf16.md).  Traffic does NOT grow in proportion to the items:
+# the small case's K/V and accumulator working sets fit the 126 MB L2, the full grid's do not.
+NCU_DRAM_BYTES_PER_LAUNCH_1080P = {"forward_kernel": 87.02e9, "backward_kernel": 160.31e9, "scatter_tile_kernel": 784.87e9}
 # L2 -> SM bytes per item of the forward's corner gathers (l1tex__m_xbar2l1tex_read_bytes.sum
 # of the same capture / items): what is left of the 110,592 gathered bytes after L1 hits.
 NCU_L2_TO_SM_BYTES_PER_ITEM = {"forward_kernel": 82380.0, "backward_kernel": 95482.0}
@@ -476,12 +479,18 @@ def run_ours(args, wl):
             if name in onchip and ms > 0:
                 onchip[name]["issue_frac"] = (items_all * NCU_WARP_INSTRUCTIONS_PER_ITEM[name] / (ms * 1e-3)
                                               / issue_peak)
-    traffic = None
+    traffic, traffic_source = None, None
     if wl.dtype == torch.bfloat16 and wl.d == 128 and wl.P == 27 and not fixed_window:
         items = wl.N * wl.heads
         per_item = (NCU_DRAM_BYTES_PER_ITEM["backward_kernel"] + (NCU_DRAM_BYTES_PER_ITEM["scatter_tile_kernel"]
                     if tiled else 0.0)) if dominant_bwd else NCU_DRAM_BYTES_PER_ITEM["forward_kernel"]
         traffic = items * per_item
+        traffic_source = "ncu dram bytes per item on profile_small_bf16 x items of this launch"
+        if wl.name == "1080p_256f_bf16" and world == 1 and not sharded:
+            full = NCU_DRAM_BYTES_PER_LAUNCH_1080P
+            traffic = (full["backward_kernel"] + (full["scatter_tile_kernel"] if tiled else 0.0)) if dominant_bwd \
+                else full["forward_kernel"]
+            traffic_source = "ncu dram__bytes_read.sum + dram__bytes_write.sum of this kernel at this workload's full size"
     line = {
         "metric": metric_name(wl), "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
         "ms_per_step": step_ms, "higher_is_better": True, "scaling": "strong" if sharded else "weak",
@@ -498,7 +507,7 @@ def run_ours(args, wl):
                    "l2": "inputs (tens of GB) exceed the 126 MB L2; no flush needed"},
         "roofline": {"bound": "hbm", "kernel": dom["kernel"], "achieved": dom["achieved"], "peak": peak,
                      "unit": "GB/s", "frac": dom["achieved"] / peak, "traffic": traffic,
-                     "traffic_source": "ncu dram bytes per item on profile_small_bf16 x items of this launch",
+                     "traffic_source": traffic_source,
                      "peak_source": peak_src, "algorithmic_bytes_per_launch": dom["bytes"],
                      "kernel_ms": dom["ms"],
                      "forward_kernel": {"ms": fwd_ms, "achieved": fwd_gbs, "frac": fwd_gbs / peak},
