@@ -486,7 +486,7 @@ def run_ours(args, wl):
                     if tiled else 0.0)) if dominant_bwd else NCU_DRAM_BYTES_PER_ITEM["forward_kernel"]
         traffic = items * per_item
         traffic_source = "ncu dram bytes per item on profile_small_bf16 x items of this launch"
-        if wl.name == "1080p_256f_bf16" and world == 1 and not sharded:
+        if wl.name == "1080p_256f_bf16" and not sharded:          # per launch, i.e. per rank
             full = NCU_DRAM_BYTES_PER_LAUNCH_1080P
             traffic = (full["backward_kernel"] + (full["scatter_tile_kernel"] if tiled else 0.0)) if dominant_bwd \
                 else full["forward_kernel"]
