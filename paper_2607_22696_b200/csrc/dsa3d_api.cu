@@ -506,6 +506,9 @@ int step_host_body(const void* q_h, const void* k_h, const void* v_h, const floa
         hs->last_arena = arena;
         for (int i = 0; i < 7; ++i) hs->last_shape[i] = shape[i];
     }
+    // the previous call's kernels come first even if it was queued on another stream (they share the
+    // workspace and the result buffers; on the same stream this wait is already satisfied)
+    DSA3D_TRY(cudaStreamWaitEvent(stream, hs->main_done, 0));
     if (ordered_start) {
         DSA3D_TRY(cudaEventRecord(hs->start, stream));
         DSA3D_TRY(cudaStreamWaitEvent(hs->in, hs->start, 0));
