@@ -665,6 +665,7 @@ int dsa3d_forward_host(const void* q_h, const void* k_h, const void* v_h, const 
     // transfers that pipelined steps may still have in flight on the side streams come first
     // (this call may reuse their arena), and a later step shares no per-slab ordering with it
     DSA3D_TRY(cudaStreamWaitEvent(stream, hs->out_done, 0));
+    DSA3D_TRY(cudaStreamWaitEvent(stream, hs->main_done, 0));      // their kernels too, if queued on another stream
     hs->last_arena = nullptr;
     DSA3D_TRY(cudaEventRecord(hs->start, stream));
     DSA3D_TRY(cudaStreamWaitEvent(hs->in, hs->start, 0));
