@@ -54,7 +54,8 @@ typedef enum {
     DSA3D_ERR_UNSUPPORTED = 3,    /* dtype, head dimension or window outside the supported set */
     DSA3D_ERR_MISALIGNED = 4,     /* a pointer is not 16-byte aligned */
     DSA3D_ERR_WORKSPACE = 5,      /* workspace missing or smaller than required */
-    DSA3D_ERR_CUDA = 6            /* a CUDA runtime call failed; see dsa3d_last_cuda_error */
+    DSA3D_ERR_CUDA = 6,           /* a CUDA runtime call failed; see dsa3d_last_cuda_error */
+    DSA3D_ERR_DEVICE_TIMEOUT = 7  /* a bounded wait inside a kernel ran out (dsa3d_check_device_timeout) */
 } dsa3d_status;
 
 typedef enum { DSA3D_F32 = 0, DSA3D_BF16 = 1 } dsa3d_dtype;
@@ -311,6 +312,10 @@ int dsa3d_offsets_linear_backward(const void* u, const void* w, const float* dof
 /* Synchronises with the device and returns the flag described above (0: no wait ever ran
  * out; -1: the flag could not be read). */
 int dsa3d_device_timeout_flag(void);
+/* The same check as a status: synchronises with the device and returns DSA3D_OK, or
+ * DSA3D_ERR_DEVICE_TIMEOUT if any kernel of the library launched so far gave up a bounded wait
+ * (its outputs are then incomplete), or DSA3D_ERR_CUDA if the flag could not be read. */
+int dsa3d_check_device_timeout(void);
 
 /*
  * dsa3d_forward_residual: Eq. 1 with its first term: out = residual + attention output,

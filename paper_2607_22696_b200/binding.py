@@ -87,6 +87,8 @@ def load():
     lib.dsa3d_offsets_linear_backward_workspace_bytes.argtypes = [ctypes.c_longlong, i, i, i]
     lib.dsa3d_device_timeout_flag.restype = i
     lib.dsa3d_device_timeout_flag.argtypes = []
+    lib.dsa3d_check_device_timeout.restype = i
+    lib.dsa3d_check_device_timeout.argtypes = []
     lib.dsa3d_forward_residual.restype = i
     lib.dsa3d_forward_residual.argtypes = [p, p, p, p, p, i, i, i, i, i, win, p, p, i, p]
     lib.dsa3d_forward_fixed_window.restype = i
@@ -285,6 +287,11 @@ def dsa3d_offsets_linear_backward(u, w, doffsets, tokens, C, O, du, dw, dbias, w
 
 def dsa3d_device_timeout_flag() -> int:
     return int(load().dsa3d_device_timeout_flag())
+
+
+def dsa3d_check_device_timeout() -> None:
+    """Raises Dsa3dError (status 7) if a kernel of the library gave up a bounded wait."""
+    _check(load().dsa3d_check_device_timeout())
 
 
 def dsa3d_backward(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets,

@@ -771,6 +771,7 @@ const char* dsa3d_status_string(int status) {
         case DSA3D_ERR_MISALIGNED: return "a pointer is not 16-byte aligned";
         case DSA3D_ERR_WORKSPACE: return "workspace missing or too small";
         case DSA3D_ERR_CUDA: return "a CUDA runtime call failed";
+        case DSA3D_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
         default: return "unknown status";
     }
 }

@@ -1717,4 +1717,10 @@ int dsa3d_device_timeout_flag(void) {
     return flag;
 }
 
+int dsa3d_check_device_timeout(void) {
+    const int flag = dsa3d_device_timeout_flag();
+    if (flag < 0) return cuda_failed(cudaGetLastError());
+    return flag == 0 ? DSA3D_OK : DSA3D_ERR_DEVICE_TIMEOUT;
+}
+
 }  // extern "C"

@@ -36,7 +36,7 @@ def test_library_exports_every_declared_symbol(lib):
 
 def test_status_strings(lib):
     assert lib.dsa3d_status_string(0) == b"success"
-    for code in range(1, 7):
+    for code in range(1, 8):
         s = lib.dsa3d_status_string(code)
         assert s and s != b"unknown status"
     assert lib.dsa3d_status_string(99) == b"unknown status"

@@ -108,6 +108,7 @@ def test_offsets_linear_bf16_on_tensor_cores(tokens, C, O, gemm_variant):
     binding.dsa3d_offsets_linear_forward(u.cuda(), w.cuda(), bias.cuda(), tokens, C, O, out)
     torch.cuda.synchronize()
     assert binding.dsa3d_device_timeout_flag() == 0
+    binding.dsa3d_check_device_timeout()                       # the same as a status: raises on a timeout
     got = out.cpu().double()
     assert torch.isfinite(got).all()
     scale = float(ref.pow(2).mean().sqrt())
