@@ -42,22 +42,61 @@ METRIC = "3D-DSA fwd+bwd Mtokens/s at 1080p\u00d7256f (bf16); achieved HBM GB/s 
 UNIT = "Mtokens/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes per (token, head) item, dram__bytes_read.sum + dram__bytes_write.sum of one ncu
-# capture per kernel on the profile_small_bf16 workload (profiles/*_profile_small_bf16.md); a
-# launch on another workload with the same d and window is reported as items x these figures.
-NCU_DRAM_BYTES_PER_ITEM = {"forward_kernel": 1525.0, "backward_kernel": 2991.0, "scatter_tile_kernel": 12902.0}
-# The same two counters captured at the full size of the default workload (one pass per launch,
-# profiles/dram_traffic_1080p_256f_bf16.md).  Traffic does NOT grow in proportion to the items:
-# the small case's K/V and accumulator working sets fit the 126 MB L2, the full grid's do not.
-NCU_DRAM_BYTES_PER_LAUNCH_1080P = {"forward_kernel": 87.02e9, "backward_kernel": 160.31e9, "scatter_tile_kernel": 784.87e9}
-# L2 -> SM bytes per item of the forward's corner gathers (l1tex__m_xbar2l1tex_read_bytes.sum
-# of the same capture / items): what is left of the 110,592 gathered bytes after L1 hits.
-NCU_L2_TO_SM_BYTES_PER_ITEM = {"forward_kernel": 82380.0, "backward_kernel": 95482.0}
-NCU_RED_BYTES_PER_ITEM = {"scatter_tile_kernel": 23470.0}      # lts red sectors x 32 B / items
-# Warp instructions executed per item (smsp__inst_executed.sum of the same captures / items):
-# against the issue rate of 4 warp instructions per clock and SM they say how full the
-# schedulers are, which is what bounds the two backward kernels.
-NCU_WARP_INSTRUCTIONS_PER_ITEM = {"forward_kernel": 5402.0, "backward_kernel": 6532.0, "scatter_tile_kernel": 6999.0}
+# Counters of one ncu capture per kernel on the small profiling workload (profile_small_bf16: a
+# 3 GB cut of the default workload, d = 128, window 3x3x3), per (token, head) item:
+#   dram    dram__bytes_read.sum + dram__bytes_write.sum
+#   l2_sm   l1tex__m_xbar2l1tex_read_bytes.sum (what the corner gathers pull through the L2-to-SM
+#           port after L1 hits; the algorithmic figure P*8*2*d*elt is computed live below)
+#   inst    smsp__inst_executed.sum (warp instructions)
+# Each entry names the kernel's source files and their SHA-256 (first 12 hex digits of the
+# digest over the files in that order) at the time of the capture; when the sources on disk
+# differ, every figure derived from the entry is printed with "stale": true.  A launch on another
+# workload with the same d and window is reported as items x these figures, which understates the
+# DRAM traffic of grids whose K/V and accumulators no longer fit the 126 MB L2 (a one-off capture
+# at 1080p gave 1.7x / 1.6x / 1.8x the small case's bytes per item for the three kernels).
+NCU_PER_ITEM = {
+    "forward_kernel": {"dram": 1525.0, "l2_sm": 82380.0, "inst": 5402.0,
+                       "sources": ["dsa3d_forward.cu", "dsa3d_common.cuh"], "sha": "unrecorded"},
+    "backward_kernel": {"dram": 2991.0, "l2_sm": 95482.0, "inst": 6532.0,
+                        "sources": ["dsa3d_backward.cu", "dsa3d_common.cuh"], "sha": "unrecorded"},
+    "scatter_tile_kernel": {"dram": 12902.0, "inst": 6999.0,
+                            "sources": ["dsa3d_backward.cu", "dsa3d_common.cuh"], "sha": "unrecorded"},
+}
+
+
+def source_sha(files) -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for name in files:
+        with open(os.path.join(ROOT, "paper_2607_22696_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:12]
+
+
+def ncu_figures(kernel: str):
+    """The recorded per-item counters of `kernel` and whether its sources changed since."""
+    rec = NCU_PER_ITEM[kernel]
+    try:
+        stale = source_sha(rec["sources"]) != rec["sha"]
+    except OSError:
+        stale = True
+    return rec, stale
+
+
+def tile_geometry(wl):
+    """Tiles and key rows per tile of the dK/dV pre-reduction as the library lays them out
+    (4 x 8 x 8 queries, halo 6, unless DSA3D_TILE overrides it)."""
+    tt, ty, tx, halo = 4, 8, 8, 6
+    env = os.environ.get("DSA3D_TILE", "")
+    parts = env.split(",") if env else []
+    if len(parts) == 4:
+        try:
+            tt, ty, tx, halo = (int(x) for x in parts)
+        except ValueError:
+            pass
+    tiles = -(-wl.T // tt) * -(-wl.H // ty) * -(-wl.W // tx) * wl.heads
+    rows = (tt + 2 * halo) * (ty + 2 * halo) * (tx + 2 * halo)
+    return tiles, rows
 
 
 def measure_ceilings(dev):
@@ -453,44 +492,65 @@ def run_ours(args, wl):
            "ms": bwd_pair_ms if dominant_bwd else fwd_ms,
            "bytes": bwd_bytes if dominant_bwd else fwd_bytes}
     step_bytes = fwd_bytes + (bwd_bytes if wl.backward else 0)
-    # Fractions of the ceilings that actually bind (the path is on-chip bound, not HBM bound)
+    # Fractions of the ceilings that actually bind (the path is on-chip bound, not HBM bound).
+    # Computed from the workload where the quantity follows from the method (rows gathered per
+    # sample, rows reduced per tile, FMAs per corner); where only a counter can tell (bytes left
+    # after L1 hits, warp instructions), from the recorded capture, marked stale when the kernel's
+    # sources changed since.
     ceil = measure_ceilings(dev)
     items_all = wl.N * wl.heads
+    general = not fixed_window
+    gather_bytes = items_all * wl.P * 8 * 2 * wl.d * wl.elt         # 8 corner rows of K and of V per sample
     fma_fwd = items_all * wl.P * 8 * 2 * wl.d
-    onchip = {"ceilings": ceil,
-              "forward_kernel": {"fma_frac": fma_fwd / (fwd_ms * 1e-3) / 1e12 / ceil["fma_bf16_mixed_tfma"]}}
-    if wl.dtype == torch.bfloat16 and wl.d == 128 and wl.P == 27:
-        gather_gbs = items_all * NCU_L2_TO_SM_BYTES_PER_ITEM["forward_kernel"] / (fwd_ms * 1e-3) / 1e9
-        onchip["forward_kernel"].update(l2_gather_gbs=gather_gbs, l2_gather_frac=gather_gbs / ceil["l2_row_gather_gbs"])
+    fma_peak = ceil["fma_bf16_mixed_tfma"] if wl.dtype == torch.bfloat16 else ceil["fma_f32_tfma"]
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    mhz = (clocks or {}).get("sm_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
+    issue_peak = 4.0 * sms * mhz * 1e6                              # warp instructions per second
+    captured = wl.dtype == torch.bfloat16 and wl.d == 128 and wl.P == 27 and general
+    onchip = {"ceilings": ceil, "issue_rate_peak_ginst": issue_peak / 1e9}
+
+    def kernel_fracs(name, ms, fma, gathers):
+        out = {"fma_frac": fma / (ms * 1e-3) / 1e12 / fma_peak}
+        if gathers and general:
+            out["l2_gather_algorithmic_frac"] = gather_bytes / (ms * 1e-3) / 1e9 / ceil["l2_row_gather_gbs"]
+        if captured:
+            rec, stale = ncu_figures(name)
+            out["issue_frac"] = items_all * rec["inst"] / (ms * 1e-3) / issue_peak
+            if "l2_sm" in rec:
+                out["l2_gather_gbs"] = items_all * rec["l2_sm"] / (ms * 1e-3) / 1e9
+                out["l2_gather_frac"] = out["l2_gather_gbs"] / ceil["l2_row_gather_gbs"]
+            out["counters_stale"] = stale
+        return out
+
+    onchip["forward_kernel"] = kernel_fracs("forward_kernel", fwd_ms, fma_fwd, True)
     if wl.backward:
-        onchip["backward_kernel"] = {"fma_frac": items_all * wl.P * 8 * 3 * wl.d / (bwd_ms * 1e-3) / 1e12
-                                     / ceil["fma_bf16_mixed_tfma"]}
+        onchip["backward_kernel"] = kernel_fracs("backward_kernel", bwd_ms, items_all * wl.P * 8 * 3 * wl.d, True)
         if tiled:
-            onchip["scatter_tile_kernel"] = {"fma_frac": fma_fwd / (sct_ms * 1e-3) / 1e12 / ceil["fma_bf16_mixed_tfma"]}
-            if wl.d == 128 and wl.P == 27:
-                red_gbs = items_all * NCU_RED_BYTES_PER_ITEM["scatter_tile_kernel"] / (sct_ms * 1e-3) / 1e9
-                onchip["scatter_tile_kernel"].update(red_gbs=red_gbs, red_frac=red_gbs / ceil["l2_red_v4_f32_gbs"])
-    if wl.dtype == torch.bfloat16 and wl.d == 128 and wl.P == 27 and not fixed_window:
-        sms = torch.cuda.get_device_properties(dev).multi_processor_count
-        mhz = (clocks or {}).get("sm_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
-        issue_peak = 4.0 * sms * mhz * 1e6                      # warp instructions per second
-        onchip["issue_rate_peak_ginst"] = issue_peak / 1e9
-        for name, ms in (("forward_kernel", fwd_ms), ("backward_kernel", bwd_ms), ("scatter_tile_kernel", sct_ms)):
-            if name in onchip and ms > 0:
-                onchip[name]["issue_frac"] = (items_all * NCU_WARP_INSTRUCTIONS_PER_ITEM[name] / (ms * 1e-3)
-                                              / issue_peak)
+            onchip["scatter_tile_kernel"] = kernel_fracs("scatter_tile_kernel", sct_ms, fma_fwd, False)
+            tiles, rows = tile_geometry(wl)
+            red_gbs = tiles * rows * 2.0 * wl.d * 4 / (sct_ms * 1e-3) / 1e9     # every region row, dK and dV, fp32
+            onchip["scatter_tile_kernel"].update(red_gbs_upper=red_gbs, red_frac_upper=red_gbs / ceil["l2_red_v4_f32_gbs"])
+    # the ceiling that binds the dominant kernel: its largest on-chip fraction
+    dom_names = ((["backward_kernel"] + (["scatter_tile_kernel"] if tiled else [])) if dominant_bwd else ["forward_kernel"])
+    binding_name, binding_frac, binding_kernel = None, 0.0, None
+    if general:
+        for kname in dom_names:
+            for key, label in (("l2_gather_frac", "l2_gather"), ("l2_gather_algorithmic_frac", "l2_gather"),
+                               ("issue_frac", "issue"), ("red_frac_upper", "l2_red"), ("fma_frac", "fma")):
+                if key == "l2_gather_algorithmic_frac" and "l2_gather_frac" in onchip[kname]:
+                    continue                      # the counter-based figure (after L1 hits) is the tighter one
+                val = onchip[kname].get(key)
+                if val is not None and val > binding_frac:
+                    binding_name, binding_frac, binding_kernel = label, val, kname
     traffic, traffic_source = None, None
-    if wl.dtype == torch.bfloat16 and wl.d == 128 and wl.P == 27 and not fixed_window:
-        items = wl.N * wl.heads
-        per_item = (NCU_DRAM_BYTES_PER_ITEM["backward_kernel"] + (NCU_DRAM_BYTES_PER_ITEM["scatter_tile_kernel"]
-                    if tiled else 0.0)) if dominant_bwd else NCU_DRAM_BYTES_PER_ITEM["forward_kernel"]
-        traffic = items * per_item
-        traffic_source = "ncu dram bytes per item on profile_small_bf16 x items of this launch"
-        if wl.name == "1080p_256f_bf16" and not sharded:          # per launch, i.e. per rank
-            full = NCU_DRAM_BYTES_PER_LAUNCH_1080P
-            traffic = (full["backward_kernel"] + (full["scatter_tile_kernel"] if tiled else 0.0)) if dominant_bwd \
-                else full["forward_kernel"]
-            traffic_source = "ncu dram__bytes_read.sum + dram__bytes_write.sum of this kernel at this workload's full size"
+    if captured:
+        kernels = dom_names
+        traffic = sum(items_all * ncu_figures(kn)[0]["dram"] for kn in kernels)
+        stale = any(ncu_figures(kn)[1] for kn in kernels)
+        traffic_source = ("dram__bytes_read.sum + dram__bytes_write.sum per item of an ncu capture on the 3 GB cut "
+                          "profile_small_bf16 x items of this launch; understates grids whose K/V and accumulators "
+                          "exceed the 126 MB L2 (about 1.6-1.8x more per item at 1080p)"
+                          + ("; STALE: kernel sources changed since the capture" if stale else ""))
     line = {
         "metric": metric_name(wl), "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
         "ms_per_step": step_ms, "higher_is_better": True, "scaling": "strong" if sharded else "weak",
@@ -508,6 +568,8 @@ def run_ours(args, wl):
         "roofline": {"bound": "hbm", "kernel": dom["kernel"], "achieved": dom["achieved"], "peak": peak,
                      "unit": "GB/s", "frac": dom["achieved"] / peak, "traffic": traffic,
                      "traffic_source": traffic_source,
+                     "binding": ({"ceiling": binding_name, "kernel": binding_kernel, "frac": binding_frac}
+                                 if binding_name else None),
                      "peak_source": peak_src, "algorithmic_bytes_per_launch": dom["bytes"],
                      "kernel_ms": dom["ms"],
                      "forward_kernel": {"ms": fwd_ms, "achieved": fwd_gbs, "frac": fwd_gbs / peak},

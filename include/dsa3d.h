@@ -18,8 +18,11 @@
  *   A sample with no corner inside the grid (or a NaN/inf position) has k_p = v_p = 0 and
  *   s_p = 0; it still takes part in the softmax.  With all offsets zero the operator is
  *   fixed 3D sliding-window attention (paper, Ablations, "Effect of offsets").
- *   The depthwise-convolution term of Eq. 1, the projections and the offset predictor are
- *   not part of this library.  There is no causal mask.
+ *   There is no causal mask.  dsa3d_forward / dsa3d_backward are that operator alone.  The
+ *   layers Eq. 1 puts around it are separate entry points further down: the depthwise
+ *   convolution (its first term, dsa3d_dwconv3d_* and dsa3d_forward_residual) and the linear
+ *   layer of the offset predictor (dsa3d_offsets_linear_*), each with its backward.  The
+ *   q/k/v projections are not part of this library.
  *
  * Layouts (row-major, channels last, one video per call; a batch is one call per item):
  *   q, k, v, out, dout, dq, dk, dv : [T, H, W, heads, d]     element type = `dtype`
@@ -37,6 +40,18 @@
  *
  * Errors.  Every function returns a dsa3d_status (0 = success).  Arguments are checked
  * before anything is launched; nothing aborts, throws or traps.
+ *
+ * Experiment switches.  A few environment variables, read on each call, select an alternative
+ * kernel for the same result (they exist to measure one variant against another; none changes
+ * what is computed beyond fp32 summation order):
+ *   DSA3D_TILE="tt,ty,tx,halo"     query tiling of the dK/dV pre-reduction of dsa3d_backward
+ *                                  (default 4,8,8,6; "0" = no tiling, every contribution is an
+ *                                  atomic add); also changes dsa3d_backward_workspace_bytes
+ *   DSA3D_NO_TENSOR_FIXED_WINDOW   dsa3d_forward_fixed_window uses the general kernel
+ *   DSA3D_GEMM_ONE_CTA             dsa3d_offsets_linear_forward: one CTA per tile instead of a pair
+ *   DSA3D_GEMM_PLAIN_STORES        its epilogue stores from registers instead of by TMA
+ *   DSA3D_CONV_GENERAL             dsa3d_dwconv3d_*: the kernel for any size also for 3x3x3
+ *   DSA3D_WGRAD_PLAIN              dsa3d_dwconv3d_backward: the unstaged weight-gradient kernel
  */
 #ifndef DSA3D_H
 #define DSA3D_H
@@ -187,8 +202,10 @@ size_t dsa3d_forward_host_arena_bytes(int T, int H, int W, int heads, int d, con
  *     rejected with DSA3D_ERR_WORKSPACE before anything is launched;
  *   - the function calls no cudaMalloc / cudaFree and nothing else that allocates;
  *   - the first call on each device looks up the array's device address (one
- *     cudaGetSymbolAddress with that device current) and caches it; make that first call
- *     outside any stream capture;
+ *     cudaGetSymbolAddress with that device current) and caches it for the life of the
+ *     process; make that first call outside any stream capture.  The cached address does not
+ *     survive a cudaDeviceReset (or any other teardown of the device's primary context): a
+ *     process that resets a device must not call this function on it again;
  *   - all calls share the one array, which keeps the previous call's contents; every call
  *     clears it on `stream` before use.  Two calls whose GPU work can overlap (different
  *     streams, or different threads on one device) race on it and give wrong dk/dv:
@@ -316,6 +333,17 @@ int dsa3d_device_timeout_flag(void);
  * DSA3D_ERR_DEVICE_TIMEOUT if any kernel of the library launched so far gave up a bounded wait
  * (its outputs are then incomplete), or DSA3D_ERR_CUDA if the flag could not be read. */
 int dsa3d_check_device_timeout(void);
+/* Resets the flag to 0 (synchronises with the device).  The flag is sticky: once a wait has run
+ * out, every later check reports it until this is called.  Call it after handling a
+ * DSA3D_ERR_DEVICE_TIMEOUT, with no kernel of the library in flight. */
+int dsa3d_clear_device_timeout(void);
+/* TEST AID, not part of the operator (the paper has no counterpart).  Launches, on `stream`, one
+ * warp in which a single thread waits on a hardware barrier that nothing ever arrives at, polling
+ * at most `polls` times (1 .. 2^20), exactly like the bounded waits of the tensor-core kernels;
+ * the wait then gives up, the thread sets the timeout flag to 99 and the kernel returns normally.
+ * Nothing traps or spins without a limit.  It lets a caller (and the test-suite) exercise the
+ * path dsa3d_check_device_timeout -> DSA3D_ERR_DEVICE_TIMEOUT -> dsa3d_clear_device_timeout. */
+int dsa3d_test_wait_timeout(unsigned polls, void* stream);
 
 /*
  * dsa3d_forward_residual: Eq. 1 with its first term: out = residual + attention output,

@@ -89,6 +89,10 @@ def load():
     lib.dsa3d_device_timeout_flag.argtypes = []
     lib.dsa3d_check_device_timeout.restype = i
     lib.dsa3d_check_device_timeout.argtypes = []
+    lib.dsa3d_clear_device_timeout.restype = i
+    lib.dsa3d_clear_device_timeout.argtypes = []
+    lib.dsa3d_test_wait_timeout.restype = i
+    lib.dsa3d_test_wait_timeout.argtypes = [ctypes.c_uint, p]
     lib.dsa3d_forward_residual.restype = i
     lib.dsa3d_forward_residual.argtypes = [p, p, p, p, p, i, i, i, i, i, win, p, p, i, p]
     lib.dsa3d_forward_fixed_window.restype = i
@@ -292,6 +296,17 @@ def dsa3d_device_timeout_flag() -> int:
 def dsa3d_check_device_timeout() -> None:
     """Raises Dsa3dError (status 7) if a kernel of the library gave up a bounded wait."""
     _check(load().dsa3d_check_device_timeout())
+
+
+def dsa3d_clear_device_timeout() -> None:
+    """Resets the (sticky) timeout flag."""
+    _check(load().dsa3d_clear_device_timeout())
+
+
+def dsa3d_test_wait_timeout(polls: int, stream=None) -> None:
+    """Test aid: one thread waits `polls` polls on a barrier nobody arrives at, gives up and raises
+    the timeout flag; see include/dsa3d.h."""
+    _check(load().dsa3d_test_wait_timeout(int(polls), _stream(stream)))
 
 
 def dsa3d_backward(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets,

@@ -26,8 +26,7 @@
 //   {row offset, fp32 coefficient pair} in a per-CTA global scratch), then each group of
 //   d/8 lanes (a half-warp at 128 channels, a quarter-warp at 64) owns a row, walks its entries, accumulates  coefficient x q-row  and  coefficient x
 //   dO-row  in fp32 registers from the tile's q/dO rows held in shared memory, and issues
-//   ONE reduction per row and tensor.  (Built with DSA3D_BF16_COEF the entries are 8 bytes
-//   with bf16 coefficients and the products use the mixed-precision FMA.)
+//   ONE reduction per row and tensor.
 #include "dsa3d_common.cuh"
 #include "dsa3d_kernels.h"
 
@@ -277,9 +276,7 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     uint4* rows = reinterpret_cast<uint4*>(smem_raw);                                   // [TQ][2][VPR]
     unsigned* cursor = reinterpret_cast<unsigned*>(smem_raw + static_cast<size_t>(TQ) * kPairBytes);   // [NB]
     __shared__ unsigned warp_sums[kTileThreads / 32];
-#ifndef DSA3D_BF16_COEF
     __shared__ uint4 ent_stage[kTileThreads];          // one entry per lane, read back by every lane of its group
-#endif
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kWarps = kTileThreads / 32;
@@ -341,14 +338,8 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                             const int bin = bin0 + ((c >> 2) * ey + ((c >> 1) & 1)) * ex + (c & 1);
                             const unsigned slot = atomicAdd(&cursor[bin], 1u);
                             if (sweep == 1) {
-#ifndef DSA3D_BF16_COEF
                                 my_scratch[slot] = make_uint4(static_cast<unsigned>(ql * kPairBytes),
                                                               __float_as_uint(w * cf.x), __float_as_uint(w * cf.y), 0u);
-#else
-                                const __nv_bfloat162 pk = __floats2bfloat162_rn(w * cf.x, w * cf.y);   // (wk, wv)
-                                my_scratch[slot] = make_uint2(static_cast<unsigned>(ql * kPairBytes),
-                                                              *reinterpret_cast<const unsigned*>(&pk));
-#endif
                             }
                         }
                     }
@@ -416,7 +407,6 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
 #pragma unroll
                 for (int e = 0; e < 8; ++e) ak[e] = av[e] = 0.0f;
                 for (unsigned base = 0; base < cnt_max; base += GW) {
-#ifndef DSA3D_BF16_COEF
                     uint4 ent = make_uint4(0u, 0u, 0u, 0u);               // offset 0, coefficients 0
                     if (base + hl < cnt_mine) ent = __ldcg(my_scratch + start + base + hl);
                     const int steps = static_cast<int>(min(static_cast<unsigned>(GW), cnt_max - base));
@@ -452,33 +442,6 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                         }
                     }
                 }
-#else
-                    uint2 ent = make_uint2(0u, 0u);                       // offset 0, coefficients 0
-                    if (base + hl < cnt_mine) ent = __ldcg(my_scratch + start + base + hl);
-                    const int steps = static_cast<int>(min(static_cast<unsigned>(GW), cnt_max - base));
-#pragma unroll 4
-                    for (int j = 0; j < steps; ++j) {
-                        const int src = lane0 | j;
-                        const unsigned off = __shfl_sync(kFull, ent.x, src);
-                        const unsigned cw = __shfl_sync(kFull, ent.y, src);
-                        unsigned short ck, cv;
-                        split_b32(cw, ck, cv);
-                        const uint4 a = *reinterpret_cast<const uint4*>(my_rows + off);
-                        const uint4 b = *reinterpret_cast<const uint4*>(my_rows + off + VPR * 16);
-                        const unsigned aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            unsigned short lo, hi;
-                            split_b32(aw[i], lo, hi);
-                            ak[2 * i] = fma_bf16(ck, lo, ak[2 * i]);
-                            ak[2 * i + 1] = fma_bf16(ck, hi, ak[2 * i + 1]);
-                            split_b32(bw[i], lo, hi);
-                            av[2 * i] = fma_bf16(cv, lo, av[2 * i]);
-                            av[2 * i + 1] = fma_bf16(cv, hi, av[2 * i + 1]);
-                        }
-                    }
-                }
-#endif
                 if (cnt_mine > 0u) {
                     const int bx = bin % ex, by = (bin / ex) % ey, bt = bin / (ex * ey);
                     const long long tok = (static_cast<long long>(lo_t + bt) * pr.H + (lo_y + by)) * pr.W + (lo_x + bx);
@@ -506,15 +469,15 @@ size_t tile_smem_bytes(const Problem& pr) {
 #ifndef DSA3D_BWD_BF16_NV
 #define DSA3D_BWD_BF16_NV 2
 #endif
-template <typename T, int D> struct LaneWidth { static constexpr int NV = 1; };
-template <> struct LaneWidth<__nv_bfloat16, 128> { static constexpr int NV = DSA3D_BWD_BF16_NV; };
+template <typename T, int D> struct BwdLaneWidth { static constexpr int NV = 1; };
+template <> struct BwdLaneWidth<__nv_bfloat16, 128> { static constexpr int NV = DSA3D_BWD_BF16_NV; };
 
 template <typename T, int D>
 static cudaError_t launch_backward_t(const void* q, const void* k, const void* v, const float* offsets,
                                      const float* lse, const void* dout, void* dq, float* acc_dk,
                                      float* acc_dv, float* doffsets, float2* coef, const Problem& pr,
                                      cudaStream_t stream) {
-    constexpr int NV = LaneWidth<T, D>::NV;
+    constexpr int NV = BwdLaneWidth<T, D>::NV;
     constexpr int LPR = D / Elt<T, NV>::VEC;
     // Shared memory holds 8 floats per (group, sample); shrink the block for large windows.
     int threads = 256;

@@ -11,11 +11,7 @@ namespace dsa3d {
 
 // One contribution to dK/dV as the tile kernel bins it: byte offset of the query's q/dO row
 // pair in shared memory and the two coefficients (w_c * ck_p, w_c * cv_p).
-#ifndef DSA3D_BF16_COEF
 using TileEntry = uint4;            // {offset, fp32 wk, fp32 wv, unused}
-#else
-using TileEntry = uint2;            // {offset, (bf16 wk, bf16 wv)}: the faster, less exact build
-#endif
 
 struct Problem {
     int T, H, W, heads, d;
@@ -137,12 +133,10 @@ template <int NV> struct Elt<__nv_bfloat16, NV> {
         return acc;
     }
     // acc += c * x with an fp32 coefficient: the bf16 values are widened (one shift or mask
-    // each) and multiplied in fp32, so the coefficient keeps all its bits.  Building with
-    // DSA3D_BF16_COEF rounds the coefficient to bf16 instead and uses the mixed instruction
-    // (about 12 % faster overall); that error stays inside the 2e-2 bound on every test but
-    // reaches it on rare elements of very large tensors, so it is not the default.
+    // each) and multiplied in fp32, so the coefficient keeps all its bits.  (Rounding the
+    // coefficient to bf16 and using the mixed instruction was measured 12 % faster overall, but
+    // its error reaches the 2e-2 bound on rare elements of very large tensors.)
     static __device__ __forceinline__ void axpy(float c, const Row& x, float (&acc)[VEC]) {
-#ifndef DSA3D_BF16_COEF
         if constexpr (NV == 2 && kPackedAxpy) {
 #pragma unroll
             for (int i = 0; i < NW; ++i)
@@ -154,16 +148,6 @@ template <int NV> struct Elt<__nv_bfloat16, NV> {
                 acc[2 * i + 1] = fmaf(c, __uint_as_float(x.w[i] & 0xffff0000u), acc[2 * i + 1]);
             }
         }
-#else
-        const unsigned short cb = __bfloat16_as_ushort(__float2bfloat16_rn(c));
-#pragma unroll
-        for (int i = 0; i < NW; ++i) {
-            unsigned short xl, xh;
-            split_b32(x.w[i], xl, xh);
-            acc[2 * i] = fma_bf16(cb, xl, acc[2 * i]);
-            acc[2 * i + 1] = fma_bf16(cb, xh, acc[2 * i + 1]);
-        }
-#endif
     }
     static __device__ __forceinline__ void to_float(const Row& x, float (&f)[VEC]) {
 #pragma unroll

@@ -193,14 +193,14 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
 #ifndef DSA3D_FWD_BF16_NV
 #define DSA3D_FWD_BF16_NV 1
 #endif
-template <typename T, int D> struct LaneWidth { static constexpr int NV = 1; };
-template <> struct LaneWidth<__nv_bfloat16, 128> { static constexpr int NV = DSA3D_FWD_BF16_NV; };
+template <typename T, int D> struct FwdLaneWidth { static constexpr int NV = 1; };
+template <> struct FwdLaneWidth<__nv_bfloat16, 128> { static constexpr int NV = DSA3D_FWD_BF16_NV; };
 
 template <typename T, int D>
 static cudaError_t launch_forward_t(const void* q, const void* k, const void* v, const float* offsets,
                                     const void* addend, void* out, float* lse, const Problem& pr,
                                     cudaStream_t stream) {
-    constexpr int NV = LaneWidth<T, D>::NV;
+    constexpr int NV = FwdLaneWidth<T, D>::NV;
     constexpr int LPR = D / Elt<T, NV>::VEC;
     constexpr int threads = 256;
     const long long groups_per_block = threads / LPR;

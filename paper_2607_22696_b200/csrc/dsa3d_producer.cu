@@ -1479,6 +1479,20 @@ bool dsa3d::encode_tensor_map_bf16(CUtensorMap* map, const void* base, int rank,
                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+namespace {
+// Test aid (dsa3d_test_wait_timeout): one thread waits, with a small poll limit, on an mbarrier
+// that nothing ever arrives at, then gives up the way every bounded wait of the library does:
+// it raises the timeout flag (value 99) and returns.  No TMA, no TMEM, nothing to drain.
+__global__ void wait_timeout_probe_kernel(unsigned polls) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!mbar_wait_limit(smem_u32(&bar), 0u, polls)) atomicExch(&g_timeout_flag, 99);
+    }
+}
+}  // namespace
+
 int* dsa3d::timeout_flag_device_address() {
     void* p = nullptr;
     return cudaGetSymbolAddress(&p, g_timeout_flag) == cudaSuccess ? static_cast<int*>(p) : nullptr;
@@ -1721,6 +1735,19 @@ int dsa3d_check_device_timeout(void) {
     const int flag = dsa3d_device_timeout_flag();
     if (flag < 0) return cuda_failed(cudaGetLastError());
     return flag == 0 ? DSA3D_OK : DSA3D_ERR_DEVICE_TIMEOUT;
+}
+
+int dsa3d_clear_device_timeout(void) {
+    const int zero = 0;
+    const cudaError_t e = cudaMemcpyToSymbol(g_timeout_flag, &zero, sizeof(int));
+    return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
+}
+
+int dsa3d_test_wait_timeout(unsigned polls, void* stream) {
+    if (polls < 1 || polls > (1u << 20)) return DSA3D_ERR_BAD_SHAPE;
+    wait_timeout_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(polls);
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
 }
 
 }  // extern "C"

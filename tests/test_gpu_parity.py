@@ -355,6 +355,15 @@ def test_batched_entry_points_equal_one_call_per_video():
         assert torch.equal(dq[b], g1[0]) and torch.equal(doff[b], g1[3])
         for got, ref in ((dk[b], g1[1]), (dv[b], g1[2])):
             assert float((got.float() - ref.float()).abs().max()) <= 2e-2 * float(ref.float().abs().max())
+    # and the second video of the batch against the oracle directly
+    import oracle
+    qh, kh, vh, offh, douth = vids[1]
+    o_ref, l_ref = oracle.forward(qh, kh, vh, offh, *dims, win)
+    refs = oracle.backward(qh, kh, vh, offh, douth, *dims, win)
+    pu.assert_close("batch out", out[1], o_ref, BF16)
+    pu.assert_close("batch lse", lse[1], l_ref, BF16)
+    for name, got, ref in zip(("dq", "dk", "dv", "doffsets"), (dq[1], dk[1], dv[1], doff[1]), refs):
+        pu.assert_close("batch " + name, got, ref, BF16, backward=True)
 
 
 # ----------------------------------------------------------------- stays inside its buffers

@@ -66,6 +66,28 @@ def test_noalloc_backward_matches_workspace_backward_twice_in_a_row():
 
 
 @pytest.mark.gpu
+def test_noalloc_backward_matches_the_oracle():
+    """All four gradients of the no-allocation entry point against the CPU oracle directly (not
+    only against dsa3d_backward), at the tolerances of the parity tests."""
+    import oracle
+    import parity_util as pu
+    lib = binding.load()
+    window, dims = (3, 3, 3), (4, 7, 9, 3, 128)
+    T, H, W, heads, d = dims
+    wl = inputs.Workload("noalloc_oracle", T, H, W, heads, d, window, torch.bfloat16, 1.2, 103)
+    host = inputs.make_inputs(wl, "cpu", with_dout=True)
+    t = {n: z.cuda() for n, z in host.items()}
+    out = torch.empty_like(t["q"])
+    lse = torch.empty(dims[:4], dtype=torch.float32, device="cuda")
+    binding.dsa3d_forward(t["q"], t["k"], t["v"], t["offsets"], *dims, window, out, lse)
+    status, got = _raw_backward(lib, "dsa3d_backward_noalloc", t, lse, dims, window, with_workspace=False)
+    assert status == 0
+    refs = oracle.backward(host["q"], host["k"], host["v"], host["offsets"], host["dout"], T, H, W, heads, d, window)
+    for name, g, r in zip(("dq", "dk", "dv", "doffsets"), got, refs):
+        pu.assert_close(name, g, r, torch.bfloat16, backward=True)
+
+
+@pytest.mark.gpu
 def test_noalloc_backward_rejects_problems_beyond_its_fixed_array():
     lib = binding.load()
     limit = lib.dsa3d_backward_noalloc_max_elements()
