@@ -142,6 +142,7 @@ int dsa3d_forward_fixed_window(const void* q, const void* k, const void* v, int 
     bool done = false;
     if (dtype == DSA3D_BF16 && !std::getenv("DSA3D_NO_TENSOR_FIXED_WINDOW")) {
         done = dsa3d::try_fixed_window_forward(q, k, v, out, lse, pr, st, &e);
+        if (!done) done = dsa3d::try_fixed_window_forward_planes(q, k, v, out, lse, pr, st, &e);
         if (done && e != cudaSuccess) return cuda_failed(e);
     }
     if (!done) {                      // general kernel, a NULL offsets tensor reads as all zeros

@@ -43,8 +43,15 @@ constexpr int kStats = 8;   // per sample: alpha, g, A_t, A_y, A_x, B_t, B_y, B_
 #define DSA3D_BWD_MINBLOCKS 3
 #endif
 
+#ifndef DSA3D_BWD_THREADS_NV2
+#define DSA3D_BWD_THREADS_NV2 256
+#endif
+#ifndef DSA3D_BWD_MINBLOCKS_NV2
+#define DSA3D_BWD_MINBLOCKS_NV2 2
+#endif
+
 template <typename T, int D, int NV>
-__global__ void __launch_bounds__(256, NV == 2 ? 2 : DSA3D_BWD_MINBLOCKS)
+__global__ void __launch_bounds__(NV == 2 ? DSA3D_BWD_THREADS_NV2 : 256, NV == 2 ? DSA3D_BWD_MINBLOCKS_NV2 : DSA3D_BWD_MINBLOCKS)
 backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                 const float* __restrict__ offsets, const float* __restrict__ lse,
                 const T* __restrict__ dout, T* __restrict__ dq, float* __restrict__ acc_dk,
@@ -92,10 +99,23 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
     float delta = 0.0f;
 
     // ---------------------------------------------------------------- pass 1: gather
+#ifdef DSA3D_BWD_PREFETCH_OFF
+    // the offsets of the next chunk of samples are requested one chunk ahead
+    float nxt_t = 0.0f, nxt_y = 0.0f, nxt_x = 0.0f;
+    if (gl < pr.P) { nxt_t = __ldg(off_row + gl * 3); nxt_y = __ldg(off_row + gl * 3 + 1); nxt_x = __ldg(off_row + gl * 3 + 2); }
+#endif
     for (int pb = 0; pb < pr.P; pb += LPR) {
         Sample mine;
         mine.base = 0; mine.mask = 0u; mine.ft = mine.fy = mine.fx = 0.0f;
+#ifdef DSA3D_BWD_PREFETCH_OFF
+        if (pb + gl < pr.P) mine = to_sample(pr, make_cell_values(pr, t, y, x, pb + gl, nxt_t, nxt_y, nxt_x));
+        if (pb + LPR + gl < pr.P) {
+            const float* o3 = off_row + (pb + LPR + gl) * 3;
+            nxt_t = __ldg(o3); nxt_y = __ldg(o3 + 1); nxt_x = __ldg(o3 + 2);
+        }
+#else
         if (pb + gl < pr.P) mine = to_sample(pr, make_cell(pr, t, y, x, pb + gl, off_row + (pb + gl) * 3));
+#endif
         const int cnt = min(LPR, pr.P - pb);
         for (int j = 0; j < cnt; ++j) {
             const Sample s = group_bcast<LPR>(mine, j, gmask);
@@ -480,7 +500,7 @@ static cudaError_t launch_backward_t(const void* q, const void* k, const void* v
     constexpr int NV = BwdLaneWidth<T, D>::NV;
     constexpr int LPR = D / Elt<T, NV>::VEC;
     // Shared memory holds 8 floats per (group, sample); shrink the block for large windows.
-    int threads = 256;
+    int threads = NV == 2 ? DSA3D_BWD_THREADS_NV2 : 256;
     while (threads > 32 && static_cast<size_t>(threads / LPR) * pr.P * kStats * sizeof(float) > 64 * 1024)
         threads /= 2;
     const size_t smem = static_cast<size_t>(threads / LPR) * pr.P * kStats * sizeof(float);

@@ -215,6 +215,27 @@ __device__ __forceinline__ unsigned corner_mask(int rt, int ry, int rx, int et, 
     return (t0 ? yx : 0u) | (t1 ? (yx << 4) : 0u);
 }
 
+// The same from the three offset components already loaded.
+__device__ __forceinline__ Cell make_cell_values(const Problem& pr, int t, int y, int x, int p, float ot, float oy,
+                                                 float ox) {
+    const int w = p % pr.kw;
+    const int v = (p / pr.kw) % pr.kh;
+    const int u = p / (pr.kw * pr.kh);
+    Cell c;
+    c.it = c.iy = c.ix = 0;
+    c.mask = 0u;
+    c.ft = c.fy = c.fx = 0.0f;
+    int it, iy, ix;
+    float ft, fy, fx;
+    if (!axis_cell(t + u - pr.kt / 2, ot, pr.T, it, ft)) return c;
+    if (!axis_cell(y + v - pr.kh / 2, oy, pr.H, iy, fy)) return c;
+    if (!axis_cell(x + w - pr.kw / 2, ox, pr.W, ix, fx)) return c;
+    c.it = it; c.iy = iy; c.ix = ix;
+    c.ft = ft; c.fy = fy; c.fx = fx;
+    c.mask = corner_mask(it, iy, ix, pr.T, pr.H, pr.W);
+    return c;
+}
+
 __device__ __forceinline__ Cell make_cell(const Problem& pr, int t, int y, int x, int p,
                                           const float* __restrict__ off3) {
     const int w = p % pr.kw;

@@ -67,4 +67,9 @@ int* timeout_flag_device_address();
 bool try_fixed_window_forward(const void* q, const void* k, const void* v, void* out, float* lse, const Problem& pr,
                               cudaStream_t stream, cudaError_t* err);
 
+// The same for windows (3,5,5) and (3,7,7) (dsa3d_fixed_window_planes.cu): both contractions on the
+// tensor cores, the halo region taken one plane at a time.
+bool try_fixed_window_forward_planes(const void* q, const void* k, const void* v, void* out, float* lse,
+                                     const Problem& pr, cudaStream_t stream, cudaError_t* err);
+
 }  // namespace dsa3d

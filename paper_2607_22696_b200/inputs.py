@@ -154,6 +154,10 @@ WORKLOADS: Dict[str, Workload] = {w.name: w for w in [
     Workload(f"sweep_w{kt}{kh}{kw}_{kind}", 64, 45, 80, 16, 128, (kt, kh, kw), _BF16,
              3.0 if kind == "normal" else 0.0, 4, offsets=kind)
     for (kt, kh, kw) in [(2, 2, 2), (3, 3, 3), (3, 5, 5)] for kind in ["zero", "int", "normal"]
+] + [
+    # not a BASELINE config: the fixed-window variant of the paper's ablation on the effect of offsets
+    # (window (3,7,7), all offsets zero) on the grid of the sweep
+    Workload("sweep_w377_zero", 64, 45, 80, 16, 128, (3, 7, 7), _BF16, 0.0, 4, offsets="zero"),
 ]}
 
 

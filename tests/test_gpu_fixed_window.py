@@ -1,6 +1,7 @@
 """GPU parity of the fixed-window forward (all offsets zero, no offsets tensor): the
-tensor-core tile kernel for bf16 / 128 channels / windows (3,3,3) and (2,2,2), the general
-kernel with a NULL offsets tensor for everything else.  The oracle is run with an all-zero
+tensor-core tile kernels for bf16 with 64 or 128 channels (windows (3,3,3) and (2,2,2) in one
+score tile; (3,5,5) and (3,7,7) plane by plane), the general kernel with a NULL offsets tensor
+for everything else.  The oracle is run with an all-zero
 offsets tensor."""
 import os
 
@@ -44,6 +45,36 @@ def test_tensor_core_tile_kernel_matches_the_oracle(shape, window):
     _case(shape, window, BF16, 140)
 
 
+@pytest.mark.parametrize("shape", [(6, 9, 13, 2, 128), (4, 4, 8, 1, 128), (1, 1, 1, 1, 128), (9, 5, 17, 3, 128),
+                                   (2, 13, 7, 2, 128), (8, 8, 16, 2, 64), (5, 4, 19, 3, 64), (1, 2, 3, 1, 64)])
+@pytest.mark.parametrize("window", [(3, 5, 5), (3, 7, 7)])
+def test_plane_by_plane_tensor_core_kernel_matches_the_oracle(shape, window):
+    """Windows (3,5,5) and the paper's (3,7,7): scores and weighted sum both on the tensor cores,
+    the halo region taken one plane at a time.  Grids that are not multiples of the tile, smaller
+    than one tile, a single token (all but the centre cell dead), several tiles per CTA."""
+    _case(shape, window, BF16, 144)
+
+
+@pytest.mark.parametrize("window", [(3, 5, 5), (3, 7, 7)])
+def test_plane_kernel_sharp_softmax_many_tiles_and_agreement_with_the_general_kernel(window):
+    """One dominant key per query (weights close to 1 and close to 0 next to each other: the bf16
+    head/remainder split of the weights must hold), on a grid of several hundred tiles so that
+    every CTA walks through many of them; then the same problem through the general kernel."""
+    shape = (12, 20, 40, 4, 128)
+    T, H, W, heads, d = shape
+    q, k, v, out_tc, lse_tc = _case(shape, window, BF16, 145, sigma_q=5.0)
+    os.environ["DSA3D_NO_TENSOR_FIXED_WINDOW"] = "1"
+    try:
+        out_g, lse_g = torch.empty_like(out_tc), torch.empty_like(lse_tc)
+        binding.dsa3d_forward_fixed_window(q.cuda(), k.cuda(), v.cuda(), T, H, W, heads, d, window, out_g, lse_g)
+        torch.cuda.synchronize()
+    finally:
+        del os.environ["DSA3D_NO_TENSOR_FIXED_WINDOW"]
+    assert float((lse_tc - lse_g).abs().max()) <= 1e-4
+    ulp = (out_g.float().abs() * 2.0 ** -7).clamp_min(2e-3)
+    assert bool(((out_tc.float() - out_g.float()).abs() <= ulp).all())      # within one bf16 step of each other
+
+
 def test_sharp_softmax_and_border_samples():
     """Large logits (one key dominates) next to rows at the border whose dead samples hold
     logit 0 in the softmax."""
@@ -51,7 +82,8 @@ def test_sharp_softmax_and_border_samples():
 
 
 @pytest.mark.parametrize("shape,window,dtype", [((4, 6, 7, 2, 32), (3, 3, 3), BF16), ((3, 5, 6, 2, 32), (3, 3, 3), F32),
-                                                ((4, 6, 9, 2, 128), (3, 5, 5), BF16), ((4, 6, 9, 2, 128), (1, 3, 3), BF16)])
+                                                ((4, 6, 9, 2, 128), (5, 5, 5), BF16), ((4, 6, 9, 2, 128), (1, 3, 3), BF16),
+                                                ((4, 6, 9, 2, 32), (3, 5, 5), BF16)])
 def test_other_shapes_run_the_general_kernel_without_an_offsets_tensor(shape, window, dtype):
     _case(shape, window, dtype, 142)
 
