@@ -11,20 +11,24 @@
 //
 //   pass 1, plane by plane:  K plane by TMA (zero rows outside the grid = the zero-padded key of
 //     a dead sample) -> S_plane = Q . K_plane^T by tcgen05.mma into one of two TMEM buffers ->
-//     the two warps that share a TMEM quadrant copy the plane's score columns to shared memory,
-//     every thread picks the window cells of its query that lie in this plane (static register
-//     indices).  Two threads serve a query (the window's kernel rows are split between them).
+//     the two warps that share a TMEM quadrant (= the 32 queries of one tile plane) copy the
+//     plane's score columns to shared memory, every thread picks the window cells of its query
+//     that lie in this plane (static register indices).  Two threads serve a query (the window's
+//     kernel rows are split between them).
 //   softmax in registers; the pair of threads exchanges max and sum through shared memory; lse out.
 //   pass 2, plane by plane:  V plane by TMA into the same ring of buffers; every thread writes its
-//     query's row of P_plane into shared memory in the 128-byte-swizzled K-major layout, each
-//     fp32 weight split into a bf16 head and a bf16 remainder (relative error of the pair 2^-17,
-//     far inside the rounding of the output); two chains of tcgen05.mma (head and remainder, V as
-//     an MN-major operand) accumulate  O += P_plane . V_plane  in TMEM.
+//     cells into its query's row of P_plane in shared memory (128-byte-swizzled K-major layout),
+//     each fp32 weight split into a bf16 head and a bf16 remainder (relative error of the pair
+//     2^-17, far inside the rounding of the output), as two matrices; two chains of tcgen05.mma
+//     (V as an MN-major operand) accumulate  O += P_plane . V_plane  in TMEM.  While the chain of
+//     one matrix runs, the other matrix is being written.
 //   epilogue: O from TMEM, one rounding to bf16, out.
 //
-// One thread issues every TMA load and every MMA.  Loads run two planes ahead through a ring of
-// two plane buffers.  Every wait on an mbarrier is bounded; a wait that runs out raises the
-// library's timeout flag and the CTA stops after draining its loads and freeing its TMEM.
+// Roles: warps 0-7 are the workers described above; warp 8 holds the one thread that issues every
+// TMA load and every MMA.  Nothing but mbarriers (and a barrier per pair of worker warps) orders the
+// roles inside a tile, so a quadrant only stops at the planes its own queries see.  Every wait on
+// an mbarrier is bounded; a wait that runs out raises the library's timeout flag, the CTA walks
+// through the rest of its tile without waiting, drains its loads and frees its TMEM.
 #include <cuda_bf16.h>
 
 #include "dsa3d_common.cuh"
@@ -35,7 +39,8 @@ namespace dsa3d {
 namespace {
 
 constexpr int kPlTT = 4, kPlTY = 4, kPlTX = 8, kPlQ = kPlTT * kPlTY * kPlTX;    // 128 queries per tile
-constexpr int kPlThreads = 256;
+constexpr int kPlWorkers = 256, kPlThreads = kPlWorkers + 64;      // + loading warp + MMA warp
+constexpr int kPlMaxSlots = 4;
 
 template <int D, int KT, int KH, int KW>
 struct PlaneShape {
@@ -46,30 +51,56 @@ struct PlaneShape {
     static constexpr int KB = (PSP + 63) / 64;                      // 64-column blocks of a P row
     static constexpr int PIECES = (PS + 31) / 32;                   // 32-column pieces of a score plane
     static constexpr int VH = (KH + 1) / 2;                         // kernel rows of the first thread of a pair
-    static constexpr int SBUF = (PIECES * 32 + 31) / 32 * 32;       // TMEM columns set aside per score buffer
+    static constexpr int SBUF = PIECES * 32;                        // TMEM columns set aside per score buffer
     static constexpr int S0 = D, S1 = D + SBUF;                     // TMEM: O at 0, two score buffers behind it
     static constexpr int P_BYTES = KB * kPlQ * 128;                 // one P matrix (head or remainder)
     static constexpr int STAGE_BYTES = PIECES * 32 * kPlQ * 4;      // a score plane as [column][query] floats
-    static constexpr int WORK_BYTES = (2 * P_BYTES > STAGE_BYTES ? 2 * P_BYTES : STAGE_BYTES);
+    static constexpr int Q_BYTES = NH * kPlQ * 128;
     static constexpr int SLOT_HALF = PSP * 128;                     // one 64-channel half of a plane buffer
+    static constexpr int SLOT_BYTES = NH * SLOT_HALF;
+    static constexpr int SMALL_BYTES = 2 * kPlWorkers * 4 + 256 + 2048;   // pair arrays, barriers, alignment slack
+    static constexpr int BUDGET = 227 * 1024;
+    // Work area: the score staging of pass 1 and the two P matrices of pass 2 share their bytes.
+    // Q has its own buffer (so the next tile's Q arrives during pass 2) unless giving it up buys
+    // a third plane buffer: then it sits behind the staging area, on top of the tail of P.
+    static constexpr int WORK_OWN = (2 * P_BYTES > STAGE_BYTES ? 2 * P_BYTES : STAGE_BYTES);
+    static constexpr int NS_OWN = (BUDGET - SMALL_BYTES - Q_BYTES - WORK_OWN) / SLOT_BYTES;
+    static constexpr int WORK_SHARED = (2 * P_BYTES > STAGE_BYTES + Q_BYTES ? 2 * P_BYTES : STAGE_BYTES + Q_BYTES);
+    static constexpr int NS_SHARED = (BUDGET - SMALL_BYTES - WORK_SHARED) / SLOT_BYTES;
+    static constexpr bool Q_SHARED = NS_OWN < 3 && NS_SHARED > NS_OWN;
+    static constexpr int NS_RAW = Q_SHARED ? NS_SHARED : NS_OWN;
+    static constexpr int NS = NS_RAW > kPlMaxSlots ? kPlMaxSlots : NS_RAW;
+    static constexpr int WORK_BYTES = Q_SHARED ? WORK_SHARED : WORK_OWN;
+    static constexpr int Q_OFFSET = STAGE_BYTES;                    // of Q inside the work area when shared
     static_assert(PSP <= 256, "a region plane must fit one MMA (N <= 256)");
     static_assert(D + 2 * SBUF <= 512, "TMEM columns");
-    static_assert(SLOT_HALF % 1024 == 0 || true, "");
+    static_assert(SLOT_HALF % 1024 == 0 && STAGE_BYTES % 1024 == 0, "buffers keep the 1024-byte alignment of the swizzle");
+    static_assert(NS >= 2, "at least two plane buffers");
 };
 
 template <int D, int KT, int KH, int KW>
 struct __align__(1024) PlSmem {
     using S = PlaneShape<D, KT, KH, KW>;
-    unsigned char q[S::NH][kPlQ * 128];                             // 64-channel halves, swizzled 128-byte rows
-    unsigned char slot[2][S::NH][(S::SLOT_HALF + 1023) / 1024 * 1024];   // K or V plane, same image for both uses
-    unsigned char work[(S::WORK_BYTES + 1023) / 1024 * 1024];       // score staging (pass 1), P head + remainder (pass 2)
-    float pair_max[kPlThreads], pair_sum[kPlThreads];
-    uint64_t bar_q, bar_full[2], bar_s[2], bar_pv;
+    unsigned char work[S::WORK_BYTES];                              // staging (pass 1) / P head + remainder (pass 2) [/ Q]
+    unsigned char slot[S::NS][S::NH][S::SLOT_HALF];                 // ring of K or V planes, same image for both uses
+    unsigned char q_own[S::Q_SHARED ? 1024 : S::Q_BYTES];           // 64-channel halves, swizzled 128-byte rows
+    float pair_max[kPlWorkers], pair_sum[kPlWorkers];
+    uint64_t bar_q, bar_full[kPlMaxSlots], bar_slot_free[kPlMaxSlots];
+    uint64_t bar_s[2], bar_s_free[2], bar_p_full[2], bar_p_free[2], bar_o;
     uint32_t tmem_base;
+    uint32_t abort;                                                 // a wait ran out somewhere: nobody waits any more
 };
 
 __device__ __forceinline__ void named_barrier_sync(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+// Barrier 6 of the workers and the MMA warp at the end of a tile; returns the OR of `flag` over them.
+__device__ __forceinline__ bool tile_barrier_or(bool flag) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, 6, %2, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out) : "r"(static_cast<uint32_t>(flag)), "r"(kPlWorkers + 32) : "memory");
+    return out != 0u;
 }
 
 template <int D, int KT, int KH, int KW>
@@ -77,23 +108,29 @@ __global__ void __launch_bounds__(kPlThreads, 1)
 fixed_window_planes_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                            const __grid_constant__ CUtensorMap map_v, __nv_bfloat16* __restrict__ out,
                            float* __restrict__ lse, int T, int H, int W, int heads, int tiles_x, int tiles_y,
-                           long long total, int* timeout_flag) {
+                           int total, int* timeout_flag) {
     using S = PlaneShape<D, KT, KH, KW>;
-    constexpr int NH = S::NH, RT = S::RT, RX = S::RX, PS = S::PS, PSP = S::PSP, VH = S::VH;
+    constexpr int NH = S::NH, RT = S::RT, RX = S::RX, PS = S::PS, PSP = S::PSP, VH = S::VH, NS = S::NS;
     constexpr int JOBS = 2 * RT;                                      // plane loads per tile: RT of K, then RT of V
     extern __shared__ unsigned char raw[];
     PlSmem<D, KT, KH, KW>& s =
         *reinterpret_cast<PlSmem<D, KT, KH, KW>*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int lt = warp & 3, half = warp >> 2;                        // query plane of the tile; which thread of the pair
-    const int ly = lane >> 3, lx = lane & 7;                          // box order of the Q load: x fastest, then y, then t
-    const int r = lt * 32 + lane;                                     // query row of the tile = TMEM lane
-    const uint32_t lane_base = static_cast<uint32_t>(lt * 32) << 16;
+    unsigned char* q_buf = S::Q_SHARED ? s.work + S::Q_OFFSET : s.q_own;
+    unsigned char* p_head = s.work;
+    unsigned char* p_rest = s.work + S::P_BYTES;
 
     if (tid == 0) {
         mbar_init(smem_u32(&s.bar_q), 1);
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&s.bar_full[i]), 1); mbar_init(smem_u32(&s.bar_s[i]), 1); }
-        mbar_init(smem_u32(&s.bar_pv), 1);
+        for (int i = 0; i < kPlMaxSlots; ++i) { mbar_init(smem_u32(&s.bar_full[i]), 1); mbar_init(smem_u32(&s.bar_slot_free[i]), 1); }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&s.bar_s[i]), 1);
+            mbar_init(smem_u32(&s.bar_s_free[i]), kPlWorkers / 32);   // lane 0 of every worker warp
+            mbar_init(smem_u32(&s.bar_p_full[i]), kPlWorkers / 32);   // lane 0 of every worker warp
+            mbar_init(smem_u32(&s.bar_p_free[i]), 1);
+        }
+        mbar_init(smem_u32(&s.bar_o), 1);
+        s.abort = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -104,7 +141,7 @@ fixed_window_planes_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
     // rows PS .. PSP-1 of the plane buffers are never written by a load: they must read as zero
     // (as V rows they are multiplied by the zero columns of P; anything non-finite would spoil O)
     if constexpr (PSP > PS) {
-        for (int i = tid; i < 2 * NH * (PSP - PS) * 8; i += kPlThreads) {
+        for (int i = tid; i < NS * NH * (PSP - PS) * 8; i += kPlThreads) {
             const int chunk = i & 7, row = PS + (i >> 3) % (PSP - PS), which = (i >> 3) / (PSP - PS);
             *reinterpret_cast<uint4*>(&s.slot[which / NH][which % NH][row * 128 + chunk * 16]) = make_uint4(0u, 0u, 0u, 0u);
         }
@@ -114,265 +151,328 @@ fixed_window_planes_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = s.tmem_base;
+    volatile uint32_t* abort_flag = &s.abort;
 
-    const long long tiles_per_head = total / heads;
-    auto locate = [&](long long item, int& m, int& t0, int& y0, int& x0) {
-        m = static_cast<int>(item / tiles_per_head);
-        int tile = static_cast<int>(item - m * tiles_per_head);
+    // A wait of this kernel: skipped once somebody has given up (the tile is then walked through
+    // without waiting and thrown away); a wait that runs out raises the flags itself.
+    auto wait = [&](uint64_t* bar, uint32_t parity, int code) -> bool {
+        if (*abort_flag) return false;
+        if (mbar_wait(smem_u32(bar), parity)) return true;
+        atomicExch(timeout_flag, code);
+        *abort_flag = 1u;
+        return false;
+    };
+
+    const int tiles_per_head = total / heads;                        // 32-bit throughout: the host checks the counts fit
+    auto locate = [&](int item, int& m, int& t0, int& y0, int& x0) {
+        m = item / tiles_per_head;
+        int tile = item - m * tiles_per_head;
         x0 = (tile % tiles_x) * kPlTX; tile /= tiles_x;
         y0 = (tile % tiles_y) * kPlTY;
         t0 = (tile / tiles_y) * kPlTT;
     };
-    // plane load number g of this CTA: tile g / JOBS, K plane (g % JOBS) or V plane (g % JOBS - RT)
-    auto issue_load = [&](long long g) {
-        const long long item = blockIdx.x + (g / JOBS) * static_cast<long long>(gridDim.x);
-        if (item >= total) return;
-        const int j = static_cast<int>(g % JOBS), sl = static_cast<int>(g & 1);
-        int m, t0, y0, x0;
-        locate(item, m, t0, y0, x0);
-        const uint32_t bar = smem_u32(&s.bar_full[sl]);
-        mbar_expect_tx(bar, static_cast<uint32_t>(NH) * PS * 128u);
-        const CUtensorMap* map = j < RT ? &map_k : &map_v;
-        for (int h = 0; h < NH; ++h)
-            tma_load_5d(smem_u32(s.slot[sl][h]), map, bar, h * 64, m, x0 - KW / 2, y0 - KH / 2, t0 - KT / 2 + j % RT);
-    };
-    auto issue_q = [&](long long item) {
-        if (item >= total) return;
-        int m, t0, y0, x0;
-        locate(item, m, t0, y0, x0);
-        mbar_expect_tx(smem_u32(&s.bar_q), static_cast<uint32_t>(NH) * kPlQ * 128u);
-        for (int h = 0; h < NH; ++h) tma_load_5d(smem_u32(s.q[h]), &map_q, smem_u32(&s.bar_q), h * 64, m, x0, y0, t0);
-    };
-    auto full_wait = [&](long long g) { return mbar_wait(smem_u32(&s.bar_full[g & 1]), static_cast<uint32_t>((g >> 1) & 1)); };
+    const int my_tiles = static_cast<int>(blockIdx.x) < total ? (total - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x) : 0;
 
-    constexpr uint32_t idesc_common = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kPlQ >> 4) << 24);
-    // score plane number sp (counted over the CTA's life) -> TMEM buffer sp & 1
-    auto issue_scores = [&](long long g, long long sp, bool first_of_tile, uint32_t q_parity) {
-        bool ready = full_wait(g);
-        if (ready && first_of_tile) ready = mbar_wait(smem_u32(&s.bar_q), q_parity);
-        if (ready) {
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t d_tmem = tmem + ((sp & 1) ? S::S1 : S::S0);
-#pragma unroll
-            for (int h = 0; h < NH; ++h) {
-                const uint64_t da = smem_desc(smem_u32(s.q[h])), db = smem_desc(smem_u32(s.slot[g & 1][h]));
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-                    umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc_common | (static_cast<uint32_t>(PSP >> 3) << 17),
-                              (h | kk) ? 1u : 0u);
-            }
-        } else {
-            atomicExch(timeout_flag, 13);
-        }
-        umma_commit(smem_u32(&s.bar_s[sp & 1]));                      // arrives at once if nothing was issued
-        return ready;
-    };
-
-    if (tid == 0 && static_cast<long long>(blockIdx.x) < total) {
-        issue_q(blockIdx.x);
-        issue_load(0);
-        issue_load(1);
-    }
-
-    float* stage = reinterpret_cast<float*>(s.work);                 // [column][query]
-    unsigned char* p_head = s.work;
-    unsigned char* p_rest = s.work + S::P_BYTES;
-    const float lscale = rsqrtf(static_cast<float>(D)) * kLog2e;
-    bool ok = true;
-    long long it = 0;
-    for (long long item = blockIdx.x; item < total && ok; item += gridDim.x, ++it) {
-        int m, t0, y0, x0;
-        locate(item, m, t0, y0, x0);
-        const long long g0 = it * JOBS, sp0 = it * RT;
-        float sc[KT][VH][KW];
-#pragma unroll
-        for (int u = 0; u < KT; ++u)
-#pragma unroll
-            for (int vi = 0; vi < VH; ++vi)
-#pragma unroll
-                for (int ww = 0; ww < KW; ++ww) sc[u][vi][ww] = -INFINITY;
-
-        // ------------------------------------------------------------ pass 1: scores, plane by plane
-        if (tid == 0 && !issue_scores(g0, sp0, true, static_cast<uint32_t>(it & 1))) ok = false;
-        for (int pl = 0; pl < RT; ++pl) {
-            const long long g = g0 + pl, sp = sp0 + pl;
-            if (tid == 0 && pl + 1 < RT && ok && !issue_scores(g + 1, sp + 1, false, 0u)) ok = false;
-            if (!mbar_wait(smem_u32(&s.bar_s[sp & 1]), static_cast<uint32_t>((sp >> 1) & 1))) {
-                if (lane == 0) atomicExch(timeout_flag, 14);
-                ok = false;
-            }
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (tid == 0 && ok) {                                     // this plane's buffer is free: two planes ahead
-                issue_load(g + 2);
-                if (pl == RT - 1) issue_q(item + gridDim.x);          // all score MMAs of the tile have read Q
-            }
-            const int u_rt = pl - lt;                                 // the kernel plane this region plane is to the warp's queries
-            if (u_rt >= 0 && u_rt < KT) {
-                const uint32_t sbuf = tmem + lane_base + ((sp & 1) ? S::S1 : S::S0);
-                for (int piece = half; piece < S::PIECES; piece += 2) {
-                    uint32_t regs[32];
-                    tmem_load_32(sbuf + piece * 32, regs);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) stage[(piece * 32 + i) * kPlQ + r] = __uint_as_float(regs[i]);
+    if (warp == kPlWorkers / 32) {
+        // ==================================================================== loading thread (lane 0)
+        // Walks the CTA's stream of plane loads (tile after tile: RT planes of K, RT planes of V) as
+        // far ahead as the ring of plane buffers allows, and puts the Q loads in between.  It takes no
+        // part in the per-tile barrier of the other roles.
+        if (lane == 0 && my_tiles > 0) {
+            const int jobs_total = my_tiles * JOBS;
+            int tile_index = 0, j = 0;                               // tile and plane load within it of load g
+            int m, t0, y0, x0;
+            auto locate_tile = [&](int ti) { locate(static_cast<int>(blockIdx.x) + ti * static_cast<int>(gridDim.x), m, t0, y0, x0); };
+            auto load_q = [&](int ti) {
+                int qm, qt0, qy0, qx0;
+                locate(static_cast<int>(blockIdx.x) + ti * static_cast<int>(gridDim.x), qm, qt0, qy0, qx0);
+                mbar_expect_tx(smem_u32(&s.bar_q), static_cast<uint32_t>(NH) * kPlQ * 128u);
+                for (int h = 0; h < NH; ++h)
+                    tma_load_5d(smem_u32(q_buf + h * (kPlQ * 128)), &map_q, smem_u32(&s.bar_q), h * 64, qm, qx0, qy0, qt0);
+            };
+            // Q of tile ti + 1 may be loaded once the MMAs of plane load `q_free_job` of tile ti have run:
+            // the tile's last score plane, or - when Q lies on the tail of P - its last P.V plane.
+            constexpr int q_free_job = S::Q_SHARED ? JOBS - 1 : RT - 1;
+            locate_tile(0);
+            load_q(0);
+            for (int g = 0; g < jobs_total; ++g) {
+                const int sl = g % NS;
+                if (g >= NS) {
+                    if (!wait(&s.bar_slot_free[sl], static_cast<uint32_t>((g / NS - 1) & 1), 13)) break;
+                    // the MMAs of load g - NS have run
+                    const int done = g - NS, done_tile = done / JOBS;
+                    if (done - done_tile * JOBS == q_free_job && done_tile + 1 < my_tiles) load_q(done_tile + 1);
                 }
-                named_barrier_sync(1 + lt, 64);                       // the two warps of this quadrant
-#pragma unroll
-                for (int u = 0; u < KT; ++u) {
-                    if (u != u_rt) continue;
-#pragma unroll
-                    for (int vi = 0; vi < VH; ++vi) {
-                        const int vv = vi + half * VH;
-                        if (vv >= KH) continue;
-#pragma unroll
-                        for (int ww = 0; ww < KW; ++ww)
-                            sc[u][vi][ww] = stage[((ly + vv) * RX + lx + ww) * kPlQ + r] * lscale;
+                const uint32_t bar = smem_u32(&s.bar_full[sl]);
+                mbar_expect_tx(bar, static_cast<uint32_t>(NH) * PS * 128u);
+                const CUtensorMap* map = j < RT ? &map_k : &map_v;
+                const int plane = j < RT ? j : j - RT;
+                for (int h = 0; h < NH; ++h)
+                    tma_load_5d(smem_u32(s.slot[sl][h]), map, bar, h * 64, m, x0 - KW / 2, y0 - KH / 2, t0 - KT / 2 + plane);
+                if (++j == JOBS) {
+                    j = 0;
+                    if (++tile_index < my_tiles) locate_tile(tile_index);
+                }
+            }
+            // Q loads whose trigger lies within the last NS plane loads of the stream
+            if (!*abort_flag) {
+                for (int done = jobs_total - NS < 0 ? 0 : jobs_total - NS; done < jobs_total; ++done) {
+                    const int done_tile = done / JOBS;
+                    if (done - done_tile * JOBS == q_free_job && done_tile + 1 < my_tiles) {
+                        if (wait(&s.bar_slot_free[done % NS], static_cast<uint32_t>((done / NS) & 1), 13)) load_q(done_tile + 1);
                     }
                 }
             }
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            ok = __syncthreads_and(ok);                               // staging area and score buffer are free again
-            if (!ok) break;
         }
-        if (!ok) break;
-
-        // ------------------------------------------------------------ softmax over the window (two threads per query)
-        float mx = -INFINITY;
+    } else if (warp == kPlWorkers / 32 + 1) {
+        // ==================================================================== MMA thread (lane 0)
+        constexpr uint32_t idesc_common = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kPlQ >> 4) << 24);
+        constexpr uint32_t idesc_s = idesc_common | (static_cast<uint32_t>(PSP >> 3) << 17);
+        constexpr uint32_t idesc_pv = idesc_common | (1u << 16) | (static_cast<uint32_t>(D >> 3) << 17);     // B = V, MN-major
+        // descriptors of plane buffer 0; buffer i lies i * SLOT_BYTES further (the address field counts 16 bytes)
+        uint64_t desc_q[NH], desc_slot_k[NH], desc_p[2][S::KB];
+        constexpr uint64_t slot_step = S::SLOT_BYTES >> 4;
+        for (int h = 0; h < NH; ++h) {
+            desc_q[h] = smem_desc(smem_u32(q_buf + h * (kPlQ * 128)));
+            desc_slot_k[h] = smem_desc(smem_u32(s.slot[0][h]));
+        }
+        const uint64_t desc_slot_v = smem_desc_mn(smem_u32(s.slot[0][0]), static_cast<uint32_t>(S::SLOT_HALF));
+        for (int part = 0; part < 2; ++part)
+            for (int b = 0; b < S::KB; ++b) desc_p[part][b] = smem_desc(smem_u32((part ? p_rest : p_head) + b * (kPlQ * 128)));
+        int g = 0, sl = 0, sp = 0, pvc = 0;                          // plane load, its buffer, score plane, P.V plane counters
+        uint32_t full_parity = 0;                                    // of bar_full[sl] for load g
+        for (int it = 0; it < my_tiles; ++it) {
+            if (lane == 0) {
+                // ---- pass 1: S_plane = Q . K_plane^T
+                for (int pl = 0; pl < RT; ++pl, ++g, ++sp) {
+                    bool ready = wait(&s.bar_full[sl], full_parity, 14);
+                    if (ready && pl == 0) ready = wait(&s.bar_q, static_cast<uint32_t>(it & 1), 15);
+                    // the workers have taken plane sp - 2 out of this score buffer
+                    if (ready && sp >= 2) ready = wait(&s.bar_s_free[sp & 1], static_cast<uint32_t>(((sp >> 1) - 1) & 1), 16);
+                    if (ready) {
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        const uint32_t d_tmem = tmem + ((sp & 1) ? S::S1 : S::S0);
 #pragma unroll
-        for (int u = 0; u < KT; ++u)
+                        for (int h = 0; h < NH; ++h)
 #pragma unroll
-            for (int vi = 0; vi < VH; ++vi)
+                            for (int kk = 0; kk < 4; ++kk)
+                                umma_bf16(d_tmem, desc_q[h] + 2 * kk, desc_slot_k[h] + sl * slot_step + 2 * kk, idesc_s, (h | kk) ? 1u : 0u);
+                    }
+                    umma_commit(smem_u32(&s.bar_s[sp & 1]));          // arrives at once if nothing was issued
+                    umma_commit(smem_u32(&s.bar_slot_free[sl]));
+                    if (++sl == NS) { sl = 0; full_parity ^= 1u; }
+                }
+                // ---- pass 2: O += P_plane . V_plane, the head and the remainder of P as two chains
+                for (int pl = 0; pl < RT; ++pl, ++g, ++pvc) {
+                    bool ready = wait(&s.bar_full[sl], full_parity, 18);
 #pragma unroll
-                for (int ww = 0; ww < KW; ++ww) mx = fmaxf(mx, sc[u][vi][ww]);
-        s.pair_max[tid] = mx;
-        named_barrier_sync(1 + lt, 64);
-        mx = fmaxf(mx, s.pair_max[tid ^ 128]);
-        float sum = 0.0f;
+                    for (int part = 0; part < 2; ++part) {
+                        if (ready) ready = wait(&s.bar_p_full[part], static_cast<uint32_t>(pvc & 1), 19);
+                        if (ready) {
+                            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-        for (int u = 0; u < KT; ++u)
+                            for (int ks = 0; ks < PSP / 16; ++ks)
+                                umma_bf16(tmem, desc_p[part][ks >> 2] + 2 * (ks & 3), desc_slot_v + sl * slot_step + 128 * ks, idesc_pv,
+                                          (pl | part | ks) ? 1u : 0u);
+                        }
+                        umma_commit(smem_u32(&s.bar_p_free[part]));
+                    }
+                    umma_commit(smem_u32(&s.bar_slot_free[sl]));
+                    if (pl == RT - 1) umma_commit(smem_u32(&s.bar_o));
+                    if (++sl == NS) { sl = 0; full_parity ^= 1u; }
+                }
+            }
+            // the workers' epilogue reads O; the next tile's first P.V chain starts beyond the barrier below
+            __syncwarp();
+            if (tile_barrier_or(*abort_flag != 0u)) break;           // the same decision in every thread
+        }
+    } else {
+        // ==================================================================== workers
+        const int lt = warp & 3, half = warp >> 2;                    // query plane of the tile; which thread of the pair
+        const int ly = lane >> 3, lx = lane & 7;                      // box order of the Q load: x fastest, then y, then t
+        const int r = lt * 32 + lane;                                 // query row of the tile = TMEM lane
+        const uint32_t lane_base = static_cast<uint32_t>(lt * 32) << 16;
+        const uint32_t row_off = static_cast<uint32_t>(r) * 128u, rx = static_cast<uint32_t>(r & 7);
+        float* stage = reinterpret_cast<float*>(s.work);             // [column][query]
+        const float lscale = rsqrtf(static_cast<float>(D)) * kLog2e;
+        // Where this thread's window cells sit is the same for every plane and every tile: kept in
+        // registers when the window is small enough, recomputed otherwise.
+        constexpr bool kCacheCells = VH * KW <= 16;
+        uint32_t cell_stage[kCacheCells ? VH : 1][kCacheCells ? KW : 1];   // element of `stage` holding the cell's score
+        uint32_t cell_p[kCacheCells ? VH : 1][kCacheCells ? KW : 1];       // byte offset of the cell inside a P matrix
+        auto stage_index = [&](int vv, int ww) { return static_cast<uint32_t>((ly + vv) * RX + lx + ww) * kPlQ + r; };
+        auto p_offset = [&](int vv, int ww) {
+            const uint32_t col = static_cast<uint32_t>((ly + vv) * RX + lx + ww);
+            return (col >> 6) * (kPlQ * 128) + row_off + ((((col & 63) >> 3) ^ rx) << 4) + (col & 7) * 2;
+        };
+        if constexpr (kCacheCells) {
 #pragma unroll
             for (int vi = 0; vi < VH; ++vi)
 #pragma unroll
                 for (int ww = 0; ww < KW; ++ww) {
-                    sc[u][vi][ww] = exp2f(sc[u][vi][ww] - mx);            // cells this thread does not own: exp2(-inf) = 0
-                    sum += sc[u][vi][ww];
+                    const int vv = vi + half * VH < KH ? vi + half * VH : 0;
+                    cell_stage[vi][ww] = stage_index(vv, ww);
+                    cell_p[vi][ww] = p_offset(vv, ww);
                 }
-        s.pair_sum[tid] = sum;
-        named_barrier_sync(1 + lt, 64);
-        sum += s.pair_sum[tid ^ 128];
-        const float inv = 1.0f / sum;
-        const int qt = t0 + lt, qy = y0 + ly, qx = x0 + lx;
-        const bool in_grid = qt < T && qy < H && qx < W;
-        const long long n = (static_cast<long long>(qt) * H + qy) * W + qx;
-        if (half == 0 && in_grid) lse[n * heads + m] = (mx + log2f(sum)) * kLn2;
+        }
+        for (int it = 0; it < my_tiles; ++it) {
+            int m, t0, y0, x0;
+            locate(static_cast<int>(blockIdx.x) + it * static_cast<int>(gridDim.x), m, t0, y0, x0);
+            const int sp0 = it * RT;
+            float sc[KT][VH][KW];
+#pragma unroll
+            for (int u = 0; u < KT; ++u)
+#pragma unroll
+                for (int vi = 0; vi < VH; ++vi)
+#pragma unroll
+                    for (int ww = 0; ww < KW; ++ww) sc[u][vi][ww] = -INFINITY;
 
-        // ------------------------------------------------------------ pass 2: O += P_plane . V_plane
-        // A thread's cells sit at the same columns of P in each of its KT planes, so its row only has
-        // to be cleared before the first plane (the buffer held scores) and after its last one.
-        const uint32_t row_off = static_cast<uint32_t>(r) * 128u, rx = static_cast<uint32_t>(r & 7);
-        for (int pl = 0; pl < RT; ++pl) {
-            const long long g = g0 + RT + pl, pvc = it * RT + pl;
-            if (pl > 0) {
-                if (!mbar_wait(smem_u32(&s.bar_pv), static_cast<uint32_t>((pvc - 1) & 1))) {
-                    if (lane == 0) atomicExch(timeout_flag, 15);
-                    ok = false;
+            // ---------------------------------------------------------- pass 1: the window's scores, plane by plane
+            for (int pl = 0; pl < RT; ++pl) {
+                const int sp = sp0 + pl;
+                wait(&s.bar_s[sp & 1], static_cast<uint32_t>((sp >> 1) & 1), 21);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const int u_rt = pl - lt;                             // the kernel plane this region plane is to the warp's queries
+                if (u_rt >= 0 && u_rt < KT) {
+                    const uint32_t sbuf = tmem + lane_base + ((sp & 1) ? S::S1 : S::S0);
+                    for (int piece = half; piece < S::PIECES; piece += 2) {
+                        uint32_t regs[32];
+                        tmem_load_32(sbuf + piece * 32, regs);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) stage[(piece * 32 + i) * kPlQ + r] = __uint_as_float(regs[i]);
+                    }
+                    named_barrier_sync(1 + lt, 64);                   // the two warps of this quadrant: plane staged
+#pragma unroll
+                    for (int u = 0; u < KT; ++u) {
+                        if (u != u_rt) continue;
+#pragma unroll
+                        for (int vi = 0; vi < VH; ++vi) {
+                            const int vv = vi + half * VH;
+                            if (vv >= KH) continue;
+#pragma unroll
+                            for (int ww = 0; ww < KW; ++ww)
+                                sc[u][vi][ww] = stage[kCacheCells ? cell_stage[kCacheCells ? vi : 0][kCacheCells ? ww : 0] : stage_index(vv, ww)] * lscale;
+                        }
+                    }
+                    named_barrier_sync(1 + lt, 64);                   // both have picked: the staging rows may be refilled
                 }
-                if (tid == 0 && ok) issue_load(g + 1);                // the plane before this one has been multiplied
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&s.bar_s_free[sp & 1]));
             }
-            const int u_rt = pl - lt;
-            const bool mine = u_rt >= 0 && u_rt < KT;
-            if (pl == 0 || (!mine && u_rt == KT)) {                   // clear the row (one thread of the pair per matrix)
-                unsigned char* dst = (half ? p_rest : p_head) + row_off;
+
+            // ---------------------------------------------------------- softmax over the window (two threads per query)
+            float mx = -INFINITY;
 #pragma unroll
-                for (int c = 0; c < PSP / 8; ++c)
-                    *reinterpret_cast<uint4*>(dst + (c >> 3) * (kPlQ * 128) + (((c & 7) ^ rx) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+            for (int u = 0; u < KT; ++u)
+#pragma unroll
+                for (int vi = 0; vi < VH; ++vi)
+#pragma unroll
+                    for (int ww = 0; ww < KW; ++ww) mx = fmaxf(mx, sc[u][vi][ww]);
+            s.pair_max[tid] = mx;
+            named_barrier_sync(1 + lt, 64);
+            mx = fmaxf(mx, s.pair_max[tid ^ 128]);
+            float sum = 0.0f;
+#pragma unroll
+            for (int u = 0; u < KT; ++u)
+#pragma unroll
+                for (int vi = 0; vi < VH; ++vi)
+#pragma unroll
+                    for (int ww = 0; ww < KW; ++ww) {
+                        sc[u][vi][ww] = exp2f(sc[u][vi][ww] - mx);        // cells this thread does not own: exp2(-inf) = 0
+                        sum += sc[u][vi][ww];
+                    }
+            s.pair_sum[tid] = sum;
+            named_barrier_sync(1 + lt, 64);
+            sum += s.pair_sum[tid ^ 128];
+            const float inv = 1.0f / sum;
+            const int qt = t0 + lt, qy = y0 + ly, qx = x0 + lx;
+            const bool in_grid = qt < T && qy < H && qx < W;
+            const long long n = (static_cast<long long>(qt) * H + qy) * W + qx;
+            if (half == 0 && in_grid) lse[n * heads + m] = (mx + log2f(sum)) * kLn2;
+
+            // ---------------------------------------------------------- pass 2: this query's row of P, plane by plane
+            // A thread's cells sit at the same columns of P in each of its KT planes: the row is cleared
+            // once per tile (the area held scores), the cells are overwritten plane after plane and
+            // written as zeros for the plane after the last.
+            for (int pl = 0; pl < RT; ++pl) {
+                const int pvc = it * RT + pl;
+                const int u_rt = pl - lt;
+                const bool mine = u_rt >= 0 && u_rt < KT;
+                if (pl == 0) {
+                    // the chains of the previous tile have run (its epilogue waited for them); all staging
+                    // reads of this tile are done once every worker is here
+                    named_barrier_sync(5, kPlWorkers);
+                    unsigned char* dst = (half ? p_rest : p_head) + row_off;
+#pragma unroll
+                    for (int c = 0; c < PSP / 8; ++c)
+                        *reinterpret_cast<uint4*>(dst + (c >> 3) * (kPlQ * 128) + (((c & 7) ^ rx) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+                    named_barrier_sync(1 + lt, 64);                   // both matrices of the row are clear before cells land
+                }
+#pragma unroll
+                for (int part = 0; part < 2; ++part) {
+                    if (pl > 0) wait(&s.bar_p_free[part], static_cast<uint32_t>((pvc - 1) & 1), 22);   // the chain of the plane before
+                    if (mine || u_rt == KT) {
+                        unsigned char* dst = part ? p_rest : p_head;
+#pragma unroll
+                        for (int u = 0; u <= KT; ++u) {
+                            if (u != u_rt) continue;
+#pragma unroll
+                            for (int vi = 0; vi < VH; ++vi) {
+                                const int vv = vi + half * VH;
+                                if (vv >= KH) continue;
+#pragma unroll
+                                for (int ww = 0; ww < KW; ++ww) {
+                                    float p = 0.0f;
+                                    if (u < KT) p = sc[u < KT ? u : 0][vi][ww] * inv;
+                                    __nv_bfloat16 val = __float2bfloat16_rn(p);
+                                    if (part) val = __float2bfloat16_rn(p - __bfloat162float(val));
+                                    *reinterpret_cast<__nv_bfloat16*>(dst + (kCacheCells ? cell_p[kCacheCells ? vi : 0][kCacheCells ? ww : 0] : p_offset(vv, ww))) = val;
+                                }
+                            }
+                        }
+                    }
+                    fence_async_smem();                               // the MMAs read P through the async proxy
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&s.bar_p_full[part]));
+                }
             }
-            if (pl == 0) named_barrier_sync(1 + lt, 64);              // both matrices of the row are clear before cells land
-            if (mine) {
+
+            // ---------------------------------------------------------- epilogue: the pair splits the channels
+            wait(&s.bar_o, static_cast<uint32_t>(it & 1), 23);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            {
+                constexpr int CH = D / 2;                             // channels per thread of the pair
 #pragma unroll
-                for (int u = 0; u < KT; ++u) {
-                    if (u != u_rt) continue;
+                for (int c0 = 0; c0 < CH; c0 += 32) {
+                    uint32_t regs[32];
+                    tmem_load_32(tmem + lane_base + half * CH + c0, regs);
+                    if (in_grid && !*abort_flag) {
+                        uint4* dst = reinterpret_cast<uint4*>(out + (n * heads + m) * D + half * CH + c0);
 #pragma unroll
-                    for (int vi = 0; vi < VH; ++vi) {
-                        const int vv = vi + half * VH;
-                        if (vv >= KH) continue;
+                        for (int i = 0; i < 4; ++i) {
+                            uint32_t o[4];
 #pragma unroll
-                        for (int ww = 0; ww < KW; ++ww) {
-                            const float p = sc[u][vi][ww] * inv;
-                            const __nv_bfloat16 hd = __float2bfloat16_rn(p);
-                            const __nv_bfloat16 rs = __float2bfloat16_rn(p - __bfloat162float(hd));
-                            const uint32_t col = static_cast<uint32_t>((ly + vv) * RX + lx + ww);
-                            const uint32_t off = (col >> 6) * (kPlQ * 128) + row_off + ((((col & 63) >> 3) ^ rx) << 4) + (col & 7) * 2;
-                            *reinterpret_cast<__nv_bfloat16*>(p_head + off) = hd;
-                            *reinterpret_cast<__nv_bfloat16*>(p_rest + off) = rs;
+                            for (int j = 0; j < 4; ++j) {
+                                const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(regs[8 * i + 2 * j]),
+                                                                                __uint_as_float(regs[8 * i + 2 * j + 1]));
+                                o[j] = *reinterpret_cast<const uint32_t*>(&h2);
+                            }
+                            dst[i] = make_uint4(o[0], o[1], o[2], o[3]);
                         }
                     }
                 }
             }
-            fence_async_smem();                                       // the MMAs read P through the async proxy
-            ok = __syncthreads_and(ok);
-            if (!ok) break;
-            if (tid == 0) {
-                if (full_wait(g)) {
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    constexpr uint32_t idesc = idesc_common | (1u << 16) | (static_cast<uint32_t>(D >> 3) << 17);   // B = V, MN-major
-                    const uint64_t db = smem_desc_mn(smem_u32(s.slot[g & 1][0]), static_cast<uint32_t>(sizeof(s.slot[0][0])));
-#pragma unroll
-                    for (int part = 0; part < 2; ++part) {
-                        const uint32_t pa = smem_u32(part ? p_rest : p_head);
-#pragma unroll
-                        for (int ks = 0; ks < PSP / 16; ++ks)
-                            umma_bf16(tmem, smem_desc(pa + (ks >> 2) * (kPlQ * 128)) + 2 * (ks & 3), db + 128 * ks, idesc,
-                                      (pl | part | ks) ? 1u : 0u);
-                    }
-                } else {
-                    atomicExch(timeout_flag, 16);
-                    ok = false;
-                }
-                umma_commit(smem_u32(&s.bar_pv));
-            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            if (tile_barrier_or(*abort_flag != 0u)) break;           // O is free for the next tile's chains
         }
-        ok = __syncthreads_and(ok);                                   // thread 0 may have given up on the last plane
-        if (!ok) break;
-        if (!mbar_wait(smem_u32(&s.bar_pv), static_cast<uint32_t>((it * RT + RT - 1) & 1))) {
-            if (lane == 0) atomicExch(timeout_flag, 17);
-            ok = false;
-        }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        ok = __syncthreads_and(ok);
-        if (!ok) break;
-        if (tid == 0) issue_load(g0 + JOBS + 1);                      // second plane of the next tile
-
-        // ------------------------------------------------------------ epilogue: the pair splits the channels
-        if (ok) {
-            constexpr int CH = D / 2;                                 // channels per thread of the pair
-#pragma unroll
-            for (int c0 = 0; c0 < CH; c0 += 32) {
-                uint32_t regs[32];
-                tmem_load_32(tmem + lane_base + half * CH + c0, regs);
-                if (in_grid) {
-                    uint4* dst = reinterpret_cast<uint4*>(out + (n * heads + m) * D + half * CH + c0);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        uint32_t o[4];
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(regs[8 * i + 2 * j]),
-                                                                            __uint_as_float(regs[8 * i + 2 * j + 1]));
-                            o[j] = *reinterpret_cast<const uint32_t*>(&h2);
-                        }
-                        dst[i] = make_uint4(o[0], o[1], o[2], o[3]);
-                    }
-                }
-            }
-        }
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        ok = __syncthreads_and(ok);                                   // O and the work area are free for the next tile
     }
-    if (!ok && tid == 0) {            // stopped early: give loads still in flight a bounded time to land
-        mbar_wait_limit(smem_u32(&s.bar_full[0]), 0u, 1u << 16);
-        mbar_wait_limit(smem_u32(&s.bar_full[1]), 0u, 1u << 16);
-        mbar_wait_limit(smem_u32(&s.bar_full[0]), 1u, 1u << 16);
-        mbar_wait_limit(smem_u32(&s.bar_full[1]), 1u, 1u << 16);
+    // Gave up: loads may still be in flight towards this CTA's shared memory; give them a bounded time.
+    if (*abort_flag && tid == kPlWorkers) {
+        for (int i = 0; i < NS; ++i) {
+            mbar_wait_limit(smem_u32(&s.bar_full[i]), 0u, 1u << 16);
+            mbar_wait_limit(smem_u32(&s.bar_full[i]), 1u, 1u << 16);
+        }
         mbar_wait_limit(smem_u32(&s.bar_q), 0u, 1u << 16);
         mbar_wait_limit(smem_u32(&s.bar_q), 1u, 1u << 16);
     }
@@ -405,6 +505,7 @@ cudaError_t launch_planes(const CUtensorMap& mq, const CUtensorMap& mk, const CU
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
     const long long total = static_cast<long long>(tiles_x) * tiles_y * tiles_t * pr.heads;
+    if (total * (2 * (kPlTT + KT - 1)) >= (1LL << 31)) return cudaErrorInvalidValue;   // the kernel counts planes in 32 bits
     int dev = 0, sms = 0;
     e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -412,7 +513,7 @@ cudaError_t launch_planes(const CUtensorMap& mq, const CUtensorMap& mk, const CU
     if (e != cudaSuccess) return e;
     const unsigned grid = static_cast<unsigned>(total < sms ? total : sms);     // persistent: one CTA per SM
     kern<<<grid, kPlThreads, smem, stream>>>(mq, mk, mv, static_cast<__nv_bfloat16*>(out), lse, pr.T, pr.H, pr.W, pr.heads,
-                                             tiles_x, tiles_y, total, flag);
+                                             tiles_x, tiles_y, static_cast<int>(total), flag);
     return cudaGetLastError();
 }
 
@@ -426,7 +527,7 @@ bool try_fixed_window_forward_planes(const void* q, const void* k, const void* v
     if (!w355 && !w377) return false;
     const long long tiles = static_cast<long long>((pr.W + kPlTX - 1) / kPlTX) * ((pr.H + kPlTY - 1) / kPlTY) *
                             ((pr.T + kPlTT - 1) / kPlTT);
-    if (tiles > 0x7fffffffLL) return false;
+    if (tiles * pr.heads * 2 * (kPlTT + pr.kt - 1) >= (1LL << 31)) return false;     // the kernel counts planes in 32 bits
     int* flag = timeout_flag_device_address();
     CUtensorMap mq, mk, mv;
     if (!flag || !make_plane_maps(q, k, v, pr, pr.kh, pr.kw, &mq, &mk, &mv)) return false;
