@@ -361,10 +361,12 @@ int dsa3d_forward_residual(const void* q, const void* k, const void* v, const fl
  * dsa3d_forward_fixed_window: the operator with every offset equal to zero (the fixed local
  * window of the ablation on the effect of offsets) without an offsets tensor: same out and
  * lse as dsa3d_forward on an all-zero offsets tensor, up to fp32 summation order.  For bf16,
- * d = 64 or 128 and windows (3,3,3) or (2,2,2) it runs as dense tile attention on the tensor cores
- * (scores of a 4x4x8 query tile against its halo region by tcgen05, window mask, softmax,
- * weighted sum from shared memory); every other supported shape runs the general kernel
- * with zero offsets.  The environment variable DSA3D_NO_TENSOR_FIXED_WINDOW forces the
+ * d = 64 or 128 it runs as dense tile attention on the tensor cores: windows (3,3,3) and (2,2,2)
+ * with the scores of a 4x4x8 query tile against its whole halo region in one tcgen05 tile, window
+ * mask, softmax and the weighted sum from shared memory; windows (3,5,5) and (3,7,7) (the paper's
+ * own) one region plane at a time with the weighted sum on the tensor cores too, each fp32 weight
+ * entering as a bf16 head plus a bf16 remainder.  Every other supported shape runs the general
+ * kernel with zero offsets.  The environment variable DSA3D_NO_TENSOR_FIXED_WINDOW forces the
  * general kernel.  The backward of this variant is dsa3d_backward with a zero offsets
  * tensor.  Bounded waits as in dsa3d_offsets_linear_forward (dsa3d_device_timeout_flag).
  */
@@ -378,8 +380,13 @@ int dsa3d_forward_fixed_window(const void* q, const void* k, const void* v, int 
  * summation order.  With a fixed window the contributions to a key's dK/dV come from the P
  * queries around it, so they are gathered instead of scattered: no atomics, results bitwise
  * deterministic, dk/dv written once in `dtype`.  `lse` is the forward's.  `workspace`:
- * dsa3d_backward_fixed_window_workspace_bytes(...) bytes (two fp32 coefficients per sample),
- * 16-byte aligned, contents undefined afterwards.  All supported dtypes, head sizes and windows.
+ * dsa3d_backward_fixed_window_workspace_bytes(...) bytes (two fp32 coefficients per sample, plus,
+ * for bf16 with d = 64 or 128 and windows (3,3,3) or (2,2,2), a table of the dot products q.K_j and
+ * dO.V_j of every query's window and its +1 neighbours, which a tcgen05 kernel fills from dense
+ * Q.K^T and dO.V^T tiles so that the gradient kernel gathers no K/V rows for them), 16-byte aligned,
+ * contents undefined afterwards.  All supported dtypes, head sizes and windows.  The environment
+ * variable DSA3D_NO_TENSOR_FIXED_WINDOW switches the table kernel off.  Bounded waits as in
+ * dsa3d_offsets_linear_forward (dsa3d_device_timeout_flag).
  */
 int dsa3d_backward_fixed_window(const void* q, const void* k, const void* v, const float* lse, const void* dout, int T,
                                 int H, int W, int heads, int d, const int window[3], void* dq, void* dk, void* dv,

@@ -157,7 +157,11 @@ size_t dsa3d_backward_fixed_window_workspace_bytes(int T, int H, int W, int head
                                                    int dtype) {
     dsa3d::Problem pr;
     if (make_problem(T, H, W, heads, d, window, dtype, pr) != DSA3D_OK) return 0;
-    return (static_cast<size_t>(pr.items) * pr.P * sizeof(float2) + 255) & ~static_cast<size_t>(255);
+    // two fp32 coefficients per sample, then (where the tensor-core table kernel covers the shape)
+    // the dot-product tables of every query's box
+    const size_t coef = (static_cast<size_t>(pr.items) * pr.P * sizeof(float2) + 255) & ~static_cast<size_t>(255);
+    const size_t table = static_cast<size_t>(pr.items) * dsa3d::fixed_window_table_floats(pr, dtype == DSA3D_BF16) * sizeof(float);
+    return coef + table;
 }
 
 int dsa3d_backward_fixed_window(const void* q, const void* k, const void* v, const float* lse, const void* dout, int T,
@@ -176,8 +180,17 @@ int dsa3d_backward_fixed_window(const void* q, const void* k, const void* v, con
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = record(2, st);
     if (e != cudaSuccess) return cuda_failed(e);
-    e = dsa3d::launch_fixed_window_backward(q, k, v, lse, dout, dq, dk, dv, doffsets, static_cast<float2*>(workspace), pr,
-                                            dtype == DSA3D_BF16, st);
+    const float* table = nullptr;
+    if (dsa3d::fixed_window_table_floats(pr, dtype == DSA3D_BF16) > 0 && !std::getenv("DSA3D_NO_TENSOR_FIXED_WINDOW")) {
+        const size_t coef_bytes = (static_cast<size_t>(pr.items) * pr.P * sizeof(float2) + 255) & ~static_cast<size_t>(255);
+        float* tab = reinterpret_cast<float*>(static_cast<char*>(workspace) + coef_bytes);
+        if (dsa3d::try_fixed_window_tables(q, k, v, dout, tab, pr, st, &e)) {
+            if (e != cudaSuccess) return cuda_failed(e);
+            table = tab;
+        }
+    }
+    e = dsa3d::launch_fixed_window_backward(q, k, v, lse, dout, dq, dk, dv, doffsets, static_cast<float2*>(workspace), table,
+                                            pr, dtype == DSA3D_BF16, st);
     if (e != cudaSuccess) return cuda_failed(e);
     e = record(3, st);
     return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);

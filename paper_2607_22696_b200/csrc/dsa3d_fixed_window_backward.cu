@@ -22,11 +22,15 @@
 namespace dsa3d {
 namespace {
 
-template <typename T, int D>
-__global__ void __launch_bounds__(256)
+#ifndef DSA3D_FWB_TABLE_BLOCKS
+#define DSA3D_FWB_TABLE_BLOCKS 3
+#endif
+template <typename T, int D, bool TABLE>
+__global__ void __launch_bounds__(256, TABLE ? DSA3D_FWB_TABLE_BLOCKS : 1)
 fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                                    const float* __restrict__ lse, const T* __restrict__ dout, T* __restrict__ dq,
-                                   float* __restrict__ doffsets, float2* __restrict__ coef, const Problem pr) {
+                                   float* __restrict__ doffsets, float2* __restrict__ coef,
+                                   const float* __restrict__ table, const Problem pr) {
     using E = Elt<T, 1>;
     using Row = typename E::Row;
     constexpr int VEC = E::VEC;
@@ -42,7 +46,9 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
     if (!active) item = pr.items - 1;
 
     const bool want_doff = doffsets != nullptr;
-    const int BT = pr.kt + (want_doff ? 1 : 0), BY = pr.kh + (want_doff ? 1 : 0), BX = pr.kw + (want_doff ? 1 : 0);
+    // with a table the box always has the +1 neighbours (that is how the table is laid out)
+    const bool wide = want_doff || TABLE;
+    const int BT = pr.kt + (wide ? 1 : 0), BY = pr.kh + (wide ? 1 : 0), BX = pr.kw + (wide ? 1 : 0);
     const int NB = BT * BY * BX;
     const int NB8 = (NB + 7) & ~7;
     // per block: box_tab[NB8] = displacement of box position idx from the box origin and whether
@@ -81,10 +87,18 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
     const long long v_minus_k = v - k;
     const int ot = t - pr.kt / 2, oy = y - pr.kh / 2, ox = x - pr.kw / 2;      // box origin
 
-    const Row qr = E::load(q + row * D + ch);
-    const Row dor = E::load(dout + row * D + ch);
     const float lse2 = __ldg(lse + row) * kLog2e;
 
+    if constexpr (TABLE) {
+        // ---- dot products from the table the tensor cores wrote: [item][a, b][NB8]
+        const float* mine = table + row * (2 * NB8);
+        for (int i = gl; i < NB8; i += LPR) {
+            ta[i] = __ldg(mine + i);
+            tb[i] = __ldg(mine + NB8 + i);
+        }
+    } else {
+    const Row qr = E::load(q + row * D + ch);
+    const Row dor = E::load(dout + row * D + ch);
     // ---- dot products over the box, eight positions per reduction: all 16 row loads of a chunk
     //      are issued before the first dot product
     for (int c8 = 0; c8 < NB8; c8 += 8) {
@@ -127,6 +141,7 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
                 for (int i = 0; i < 8; ++i) { ta[c8 + i] = a8[i]; tb[c8 + i] = b8[i]; }
             }
         }
+    }
     }
     __syncwarp();
 
@@ -226,16 +241,17 @@ fixed_window_backward_key_kernel(const T* __restrict__ q, const T* __restrict__ 
 
 template <typename T, int D>
 cudaError_t launch_t(const void* q, const void* k, const void* v, const float* lse, const void* dout, void* dq,
-                     void* dk, void* dv, float* doffsets, float2* coef, const Problem& pr, cudaStream_t stream) {
+                     void* dk, void* dv, float* doffsets, float2* coef, const float* table, const Problem& pr,
+                     cudaStream_t stream) {
     constexpr int LPR = D / Elt<T, 1>::VEC;
-    const int box = doffsets ? (pr.kt + 1) * (pr.kh + 1) * (pr.kw + 1) : pr.P;
+    const int box = (doffsets || table) ? (pr.kt + 1) * (pr.kh + 1) * (pr.kw + 1) : pr.P;
     const size_t box8 = static_cast<size_t>((box + 7) & ~7);
     const size_t per_group = (2 * box8 + 2 * pr.P) * sizeof(float);
     const size_t tables = box8 * sizeof(int4) + static_cast<size_t>((pr.P + 3) & ~3) * sizeof(int);
     int threads = 256;
     while (threads > 32 && tables + static_cast<size_t>(threads / LPR) * per_group > 64 * 1024) threads /= 2;
     const size_t smem = tables + static_cast<size_t>(threads / LPR) * per_group;
-    auto qk = fixed_window_backward_query_kernel<T, D>;
+    auto qk = table ? fixed_window_backward_query_kernel<T, D, true> : fixed_window_backward_query_kernel<T, D, false>;
     if (smem > 48 * 1024) {
         const cudaError_t e = cudaFuncSetAttribute(qk, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
@@ -244,7 +260,7 @@ cudaError_t launch_t(const void* q, const void* k, const void* v, const float* l
     long long blocks = (pr.items + groups - 1) / groups;
     qk<<<static_cast<unsigned>(blocks), threads, smem, stream>>>(
         static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), lse, static_cast<const T*>(dout),
-        static_cast<T*>(dq), doffsets, coef, pr);
+        static_cast<T*>(dq), doffsets, coef, table, pr);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     groups = 256 / LPR;
@@ -258,11 +274,12 @@ cudaError_t launch_t(const void* q, const void* k, const void* v, const float* l
 
 cudaError_t launch_fixed_window_backward(const void* q, const void* k, const void* v, const float* lse,
                                          const void* dout, void* dq, void* dk, void* dv, float* doffsets,
-                                         float2* coef, const Problem& pr, bool bf16, cudaStream_t stream) {
-#define DSA3D_CASE(DD)                                                                                          \
-    case DD:                                                                                                    \
-        return bf16 ? launch_t<__nv_bfloat16, DD>(q, k, v, lse, dout, dq, dk, dv, doffsets, coef, pr, stream)   \
-                    : launch_t<float, DD>(q, k, v, lse, dout, dq, dk, dv, doffsets, coef, pr, stream);
+                                         float2* coef, const float* table, const Problem& pr, bool bf16,
+                                         cudaStream_t stream) {
+#define DSA3D_CASE(DD)                                                                                                 \
+    case DD:                                                                                                           \
+        return bf16 ? launch_t<__nv_bfloat16, DD>(q, k, v, lse, dout, dq, dk, dv, doffsets, coef, table, pr, stream)   \
+                    : launch_t<float, DD>(q, k, v, lse, dout, dq, dk, dv, doffsets, coef, table, pr, stream);
     switch (pr.d) {
         DSA3D_CASE(32)
         DSA3D_CASE(64)

@@ -46,10 +46,20 @@ int backward_impl(const void* q, const void* k, const void* v, const float* offs
                   void* stream, bool tiled);
 
 // Backward of the fixed-window variant (dsa3d_fixed_window_backward.cu): dq, dk, dv in the storage
-// type, doffsets (may be NULL), coef [N*heads, P] scratch.
+// type, doffsets (may be NULL), coef [N*heads, P] scratch.  `table` (or NULL): the dot products
+// q.K_j and dO.V_j of every query's box as try_fixed_window_tables leaves them; the kernel then
+// reads them instead of gathering K and V rows for them.
 cudaError_t launch_fixed_window_backward(const void* q, const void* k, const void* v, const float* lse,
                                          const void* dout, void* dq, void* dk, void* dv, float* doffsets,
-                                         float2* coef, const Problem& pr, bool bf16, cudaStream_t stream);
+                                         float2* coef, const float* table, const Problem& pr, bool bf16,
+                                         cudaStream_t stream);
+
+// Dot-product tables of the fixed-window backward on the tensor cores (dsa3d_fixed_window_tables.cu).
+// fixed_window_table_floats: floats per (token, head) item, 0 when the shape is not covered.
+// try_fixed_window_tables: false when the shape is not covered (nothing launched).
+int fixed_window_table_floats(const Problem& pr, bool bf16);
+bool try_fixed_window_tables(const void* q, const void* k, const void* v, const void* dout, float* table,
+                             const Problem& pr, cudaStream_t stream, cudaError_t* err);
 
 // Host side of the TMA kernels (dsa3d_producer.cu).  encode_tensor_map_bf16: a tiled map over
 // a bf16 tensor of `rank` dimensions (innermost first; strides_bytes has rank-1 entries, the
