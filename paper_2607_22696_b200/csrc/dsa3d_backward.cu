@@ -27,6 +27,8 @@
 //   d/8 lanes (a half-warp at 128 channels, a quarter-warp at 64) owns a row, walks its entries, accumulates  coefficient x q-row  and  coefficient x
 //   dO-row  in fp32 registers from the tile's q/dO rows held in shared memory, and issues
 //   ONE reduction per row and tensor.
+#include <type_traits>
+
 #include "dsa3d_common.cuh"
 #include "dsa3d_kernels.h"
 
@@ -99,115 +101,133 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
     float delta = 0.0f;
 
     // ---------------------------------------------------------------- pass 1: gather
-#ifdef DSA3D_BWD_PREFETCH_OFF
-    // the offsets of the next chunk of samples are requested one chunk ahead
-    float nxt_t = 0.0f, nxt_y = 0.0f, nxt_x = 0.0f;
-    if (gl < pr.P) { nxt_t = __ldg(off_row + gl * 3); nxt_y = __ldg(off_row + gl * 3 + 1); nxt_x = __ldg(off_row + gl * 3 + 2); }
-#endif
-    for (int pb = 0; pb < pr.P; pb += LPR) {
-        Sample mine;
-        mine.base = 0; mine.mask = 0u; mine.ft = mine.fy = mine.fx = 0.0f;
-#ifdef DSA3D_BWD_PREFETCH_OFF
-        if (pb + gl < pr.P) mine = to_sample(pr, make_cell_values(pr, t, y, x, pb + gl, nxt_t, nxt_y, nxt_x));
-        if (pb + LPR + gl < pr.P) {
-            const float* o3 = off_row + (pb + LPR + gl) * 3;
-            nxt_t = __ldg(o3); nxt_y = __ldg(o3 + 1); nxt_x = __ldg(o3 + 2);
-        }
-#else
-        if (pb + gl < pr.P) mine = to_sample(pr, make_cell(pr, t, y, x, pb + gl, off_row + (pb + gl) * 3));
-#endif
-        const int cnt = min(LPR, pr.P - pb);
-        for (int j = 0; j < cnt; ++j) {
-            const Sample s = group_bcast<LPR>(mine, j, gmask);
-            const float wt[2] = {1.0f - s.ft, s.ft}, wy[2] = {1.0f - s.fy, s.fy}, wx[2] = {1.0f - s.fx, s.fx};
-            const T* kp4[4];             // corner row pointers per (ct, cy); cx = 1 is one token further
-            kp4[0] = kh + s.base * tok_stride;
-            kp4[1] = kp4[0] + sy;
-            kp4[2] = kp4[0] + st;
-            kp4[3] = kp4[2] + sy;
-            float w[8];
-            {
-                const float wty[4] = {wt[0] * wy[0], wt[0] * wy[1], wt[1] * wy[0], wt[1] * wy[1]};
-#pragma unroll
-                for (int c = 0; c < 8; ++c) w[c] = wty[c >> 1] * wx[c & 1];
-            }
-            float a[8], b[8];            // lane partials of q.K_c and dO.V_c (0 for corners not loaded)
-            float kp[VEC];
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) kp[e] = 0.0f;
-            const bool full = s.mask == 0xffu && s.ft != 0.0f && s.fy != 0.0f && s.fx != 0.0f;
-            if (full) {                    // every corner inside the grid and needed: 16 loads back to back
-                Row kk[8], vv[8];
-#pragma unroll
-                for (int c = 0; c < 8; ++c) kk[c] = E::load(kp4[c >> 1] + (c & 1) * sx);
-#pragma unroll
-                for (int c = 0; c < 8; ++c) vv[c] = E::load(kp4[c >> 1] + (c & 1) * sx + v_minus_k);
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    a[c] = E::dot(qr, kk[c], 0.0f);
-                    b[c] = E::dot(dor, vv[c], 0.0f);
-                    E::axpy(w[c], kk[c], kp);
+    // Integer-offset regime: when every sample of every item of this warp sits exactly on a grid position
+    // (one look at the offsets decides), a sample's value needs corner (0,0,0) alone and its one-sided
+    // derivatives the +1 neighbour along each axis: four rows of K and of V, loaded back to back, instead
+    // of eight.  The two regimes are two instances of the same loop, so that neither pays for the other's
+    // registers.
+    bool warp_on_lattice = true;
+    for (int p = gl; p < pr.P; p += LPR) {
+        const float* o3 = off_row + p * 3;
+        const float ot = __ldg(o3), oy = __ldg(o3 + 1), ox = __ldg(o3 + 2);
+        warp_on_lattice = warp_on_lattice && ot == floorf(ot) && oy == floorf(oy) && ox == floorf(ox);
+    }
+    warp_on_lattice = __all_sync(kFullMask, warp_on_lattice);
+    auto pass1 = [&](auto lattice_tag) {
+        constexpr bool lattice_chunk = decltype(lattice_tag)::value;
+        for (int pb = 0; pb < pr.P; pb += LPR) {
+            Sample mine;
+            mine.base = 0; mine.mask = 0u; mine.ft = mine.fy = mine.fx = 0.0f;
+            if (pb + gl < pr.P) mine = to_sample(pr, make_cell(pr, t, y, x, pb + gl, off_row + (pb + gl) * 3));
+            const int cnt = min(LPR, pr.P - pb);
+            for (int j = 0; j < cnt; ++j) {
+                const Sample s = group_bcast<LPR>(mine, j, gmask);
+                const float wt[2] = {1.0f - s.ft, s.ft}, wy[2] = {1.0f - s.fy, s.fy}, wx[2] = {1.0f - s.fx, s.fx};
+                const T* kp4[4];             // corner row pointers per (ct, cy); cx = 1 is one token further
+                kp4[0] = kh + s.base * tok_stride;
+                kp4[1] = kp4[0] + sy;
+                kp4[2] = kp4[0] + st;
+                kp4[3] = kp4[2] + sy;
+                float w[8];
+                {
+                    const float wty[4] = {wt[0] * wy[0], wt[0] * wy[1], wt[1] * wy[0], wt[1] * wy[1]};
+    #pragma unroll
+                    for (int c = 0; c < 8; ++c) w[c] = wty[c >> 1] * wx[c & 1];
                 }
-            } else {
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const int ct = c >> 2, cy = (c >> 1) & 1, cx = c & 1;
-                    // a corner matters if its weight or one of its weight derivatives is non-zero
-                    const bool needed = (w[c] != 0.0f) | (wy[cy] * wx[cx] != 0.0f) | (wt[ct] * wx[cx] != 0.0f) |
-                                        (wt[ct] * wy[cy] != 0.0f);
-                    a[c] = b[c] = 0.0f;
-                    if (((s.mask >> c) & 1u) && needed) {
-                        const T* pk = kp4[c >> 1] + cx * sx;
-                        const Row kk = E::load(pk);
-                        const Row vv = E::load(pk + v_minus_k);
-                        a[c] = E::dot(qr, kk, 0.0f);
-                        b[c] = E::dot(dor, vv, 0.0f);
-                        E::axpy(w[c], kk, kp);
+                float a[8], b[8];            // lane partials of q.K_c and dO.V_c (0 for corners not loaded)
+                float kp[VEC];
+    #pragma unroll
+                for (int e = 0; e < VEC; ++e) kp[e] = 0.0f;
+                const bool full = !lattice_chunk && s.mask == 0xffu && s.ft != 0.0f && s.fy != 0.0f && s.fx != 0.0f;
+                if (full) {                    // every corner inside the grid and needed: 16 loads back to back
+                    Row kk[8], vv[8];
+    #pragma unroll
+                    for (int c = 0; c < 8; ++c) kk[c] = E::load(kp4[c >> 1] + (c & 1) * sx);
+    #pragma unroll
+                    for (int c = 0; c < 8; ++c) vv[c] = E::load(kp4[c >> 1] + (c & 1) * sx + v_minus_k);
+    #pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        a[c] = E::dot(qr, kk[c], 0.0f);
+                        b[c] = E::dot(dor, vv[c], 0.0f);
+                        E::axpy(w[c], kk[c], kp);
+                    }
+                } else if (lattice_chunk) {
+                    // corners 0, 1 (x+1), 2 (y+1), 4 (t+1)
+                    Row k0 = E::zero(), k1 = E::zero(), k2 = E::zero(), k4 = E::zero();
+                    Row v0 = E::zero(), v1 = E::zero(), v2 = E::zero(), v4 = E::zero();
+                    if (s.mask & 1u) { k0 = E::load(kp4[0]); v0 = E::load(kp4[0] + v_minus_k); }
+                    if (s.mask & 2u) { k1 = E::load(kp4[0] + sx); v1 = E::load(kp4[0] + sx + v_minus_k); }
+                    if (s.mask & 4u) { k2 = E::load(kp4[1]); v2 = E::load(kp4[1] + v_minus_k); }
+                    if (s.mask & 16u) { k4 = E::load(kp4[2]); v4 = E::load(kp4[2] + v_minus_k); }
+                    a[0] = E::dot(qr, k0, 0.0f); b[0] = E::dot(dor, v0, 0.0f);
+                    a[1] = E::dot(qr, k1, 0.0f); b[1] = E::dot(dor, v1, 0.0f);
+                    a[2] = E::dot(qr, k2, 0.0f); b[2] = E::dot(dor, v2, 0.0f);
+                    a[4] = E::dot(qr, k4, 0.0f); b[4] = E::dot(dor, v4, 0.0f);
+                    a[3] = b[3] = a[5] = b[5] = a[6] = b[6] = a[7] = b[7] = 0.0f;
+                    E::to_float(k0, kp);                                  // weight 1 on corner (0,0,0), 0 on the others
+                } else {
+    #pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const int ct = c >> 2, cy = (c >> 1) & 1, cx = c & 1;
+                        // a corner matters if its weight or one of its weight derivatives is non-zero
+                        const bool needed = (w[c] != 0.0f) | (wy[cy] * wx[cx] != 0.0f) | (wt[ct] * wx[cx] != 0.0f) |
+                                            (wt[ct] * wy[cy] != 0.0f);
+                        a[c] = b[c] = 0.0f;
+                        if (((s.mask >> c) & 1u) && needed) {
+                            const T* pk = kp4[c >> 1] + cx * sx;
+                            const Row kk = E::load(pk);
+                            const Row vv = E::load(pk + v_minus_k);
+                            a[c] = E::dot(qr, kk, 0.0f);
+                            b[c] = E::dot(dor, vv, 0.0f);
+                            E::axpy(w[c], kk, kp);
+                        }
                     }
                 }
-            }
-            // r = (s, g, A_t, A_y, A_x, B_t, B_y, B_x) as lane partials, then summed over the group
-            float r[kStats];
-            trilerp_grad(a, s.ft, s.fy, s.fx, r[0], r[2], r[3], r[4]);
-            trilerp_grad(b, s.ft, s.fy, s.fx, r[1], r[5], r[6], r[7]);
-            float sdot, g;
-            if constexpr (LPR >= 8) {
-                group_reduce8<LPR>(r, gl, gmask);
-                sdot = __shfl_sync(gmask, r[0], reduce8_lane<LPR>(0), LPR);
-                g = __shfl_sync(gmask, r[0], reduce8_lane<LPR>(1), LPR);
-            } else {
-#pragma unroll
-                for (int i = 0; i < kStats; ++i) r[i] = group_sum<LPR>(r[i], gmask);
-                sdot = r[0];
-                g = r[1];
-            }
-            const float alpha = exp2f(fmaf(sdot, scale * kLog2e, -lse2));
-            const float ag = alpha * g;
-            delta += ag;
-            if constexpr (NV == 2) {
-#pragma unroll
-                for (int e = 0; e < VEC; e += 2) {
-                    fma2(u_acc[e], u_acc[e + 1], ag, ag, kp[e], kp[e + 1]);
-                    fma2(kbar[e], kbar[e + 1], alpha, alpha, kp[e], kp[e + 1]);
+                // r = (s, g, A_t, A_y, A_x, B_t, B_y, B_x) as lane partials, then summed over the group
+                float r[kStats];
+                trilerp_grad(a, s.ft, s.fy, s.fx, r[0], r[2], r[3], r[4]);
+                trilerp_grad(b, s.ft, s.fy, s.fx, r[1], r[5], r[6], r[7]);
+                float sdot, g;
+                if constexpr (LPR >= 8) {
+                    group_reduce8<LPR>(r, gl, gmask);
+                    sdot = __shfl_sync(gmask, r[0], reduce8_lane<LPR>(0), LPR);
+                    g = __shfl_sync(gmask, r[0], reduce8_lane<LPR>(1), LPR);
+                } else {
+    #pragma unroll
+                    for (int i = 0; i < kStats; ++i) r[i] = group_sum<LPR>(r[i], gmask);
+                    sdot = r[0];
+                    g = r[1];
                 }
-            } else {
-#pragma unroll
-                for (int e = 0; e < VEC; ++e) {
-                    u_acc[e] = fmaf(ag, kp[e], u_acc[e]);
-                    kbar[e] = fmaf(alpha, kp[e], kbar[e]);
+                const float alpha = exp2f(fmaf(sdot, scale * kLog2e, -lse2));
+                const float ag = alpha * g;
+                delta += ag;
+                if constexpr (NV == 2) {
+    #pragma unroll
+                    for (int e = 0; e < VEC; e += 2) {
+                        fma2(u_acc[e], u_acc[e + 1], ag, ag, kp[e], kp[e + 1]);
+                        fma2(kbar[e], kbar[e + 1], alpha, alpha, kp[e], kp[e + 1]);
+                    }
+                } else {
+    #pragma unroll
+                    for (int e = 0; e < VEC; ++e) {
+                        u_acc[e] = fmaf(ag, kp[e], u_acc[e]);
+                        kbar[e] = fmaf(alpha, kp[e], kbar[e]);
+                    }
                 }
-            }
-            float* sts = stats + (pb + j) * kStats;
-            if constexpr (LPR >= 8) {
-                const int idx = reduce8_index<LPR>(gl);
-                if (gl == reduce8_lane<LPR>(idx)) sts[idx] = idx == 0 ? alpha : r[0];   // slot 1 keeps g
-            } else if (gl == 0) {
-                sts[0] = alpha; sts[1] = g;
-#pragma unroll
-                for (int i = 2; i < kStats; ++i) sts[i] = r[i];
+                float* sts = stats + (pb + j) * kStats;
+                if constexpr (LPR >= 8) {
+                    const int idx = reduce8_index<LPR>(gl);
+                    if (gl == reduce8_lane<LPR>(idx)) sts[idx] = idx == 0 ? alpha : r[0];   // slot 1 keeps g
+                } else if (gl == 0) {
+                    sts[0] = alpha; sts[1] = g;
+    #pragma unroll
+                    for (int i = 2; i < kStats; ++i) sts[i] = r[i];
+                }
             }
         }
-    }
+    };
+    if (warp_on_lattice) pass1(std::true_type{});
+    else pass1(std::false_type{});
     {
         float dqv[VEC];
 #pragma unroll
