@@ -394,6 +394,26 @@ int dsa3d_backward_fixed_window(const void* q, const void* k, const void* v, con
 size_t dsa3d_backward_fixed_window_workspace_bytes(int T, int H, int W, int heads, int d, const int window[3],
                                                    int dtype);
 
+/*
+ * Checked build (a debugging aid; the paper has no counterpart).  A library compiled with
+ * -DDSA3D_DEBUG (paper_2607_22696_b200.build.build(debug=True) writes it to libdsa3d_debug.so) tests,
+ * in dsa3d_forward and dsa3d_backward, every K/V row a sample is about to read, every dK/dV row a
+ * contribution is about to be added to and every bin and scratch slot of the dK/dV pre-reduction
+ * against the extent of its tensor before the access; the first index out of range is recorded in a
+ * device word and that access is skipped - nothing traps, asserts or aborts.  (The tensor-core kernels
+ * address memory through TMA tensor maps, whose bounds the hardware enforces.)
+ *   dsa3d_debug_build            1 if this library was built with the checks, else 0
+ *   dsa3d_debug_first_violation  synchronises with the device; *code = 0 if no violation was recorded
+ *                                (always, in a normal build), else the site (1-3 forward gathers, 4-6
+ *                                backward gathers, 7 direct dK/dV scatter, 8 bin, 9 scratch slot, 10
+ *                                pre-reduced dK/dV row) and *offset = the offending element offset,
+ *                                bin, slot or token.  Both HOST pointers.
+ *   dsa3d_debug_clear            resets the record
+ */
+int dsa3d_debug_build(void);
+int dsa3d_debug_first_violation(int* code, long long* offset);
+int dsa3d_debug_clear(void);
+
 /* Static, NUL-terminated description of a status code. */
 const char* dsa3d_status_string(int status);
 

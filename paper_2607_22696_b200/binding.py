@@ -38,6 +38,22 @@ def load():
             f"{LIB_PATH} is missing: build it with `python -m paper_2607_22696_b200.build`; "
             "there is no CPU or PyTorch fallback for this operator")
     lib = ctypes.CDLL(LIB_PATH)
+    _declare(lib)
+    _lib = lib
+    return lib
+
+
+def load_checked_build():
+    """The bounds-checked build of the library (libdsa3d_debug.so, see include/dsa3d.h) as a ctypes
+    handle of its own with the same prototypes; the functions of this module keep using the normal
+    build.  Built on first use."""
+    from . import build as _build
+    lib = ctypes.CDLL(_build.build(debug=True))
+    _declare(lib)
+    return lib
+
+
+def _declare(lib) -> None:
     p, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
     win = ctypes.POINTER(ctypes.c_int)
     lib.dsa3d_forward.restype = i
@@ -109,8 +125,12 @@ def load():
     lib.dsa3d_status_string.argtypes = [i]
     lib.dsa3d_last_cuda_error.restype = i
     lib.dsa3d_last_cuda_error.argtypes = []
-    _lib = lib
-    return lib
+    lib.dsa3d_debug_build.restype = i
+    lib.dsa3d_debug_build.argtypes = []
+    lib.dsa3d_debug_first_violation.restype = i
+    lib.dsa3d_debug_first_violation.argtypes = [ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_longlong)]
+    lib.dsa3d_debug_clear.restype = i
+    lib.dsa3d_debug_clear.argtypes = []
 
 
 def _window(window: Sequence[int]):

@@ -21,6 +21,17 @@ int cuda_failed(cudaError_t e) { return dsa3d::note_cuda_error(e); }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Checked build: the word the kernels record their first out-of-range index in.
+#ifdef DSA3D_DEBUG
+__device__ unsigned long long g_debug_word = 0ull;
+unsigned long long* debug_word_address() {
+    void* p = nullptr;
+    return cudaGetSymbolAddress(&p, g_debug_word) == cudaSuccess ? static_cast<unsigned long long*>(p) : nullptr;
+}
+#else
+unsigned long long* debug_word_address() { return nullptr; }
+#endif
+
 // Fills `pr`; returns DSA3D_OK or the reason the shape is rejected.
 int make_problem(int T, int H, int W, int heads, int d, const int* window, int dtype, dsa3d::Problem& pr) {
     if (!window) return DSA3D_ERR_NULL_POINTER;
@@ -47,6 +58,7 @@ int make_problem(int T, int H, int W, int heads, int d, const int* window, int d
     pr.halo = 0;
     pr.tiles_t = pr.tiles_y = pr.tiles_x = 0;
     pr.tt_begin = pr.tt_count = 0;
+    pr.debug_word = debug_word_address();
     return DSA3D_OK;
 }
 
@@ -773,6 +785,39 @@ int dsa3d_backward_batch(const void* q, const void* k, const void* v, const floa
             workspace_bytes, dtype, stream);
         if (st != DSA3D_OK) return st;
     }
+    return DSA3D_OK;
+}
+
+int dsa3d_debug_build(void) {
+#ifdef DSA3D_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+int dsa3d_debug_first_violation(int* code, long long* offset) {
+    if (!code || !offset) return DSA3D_ERR_NULL_POINTER;
+    *code = 0;
+    *offset = 0;
+#ifdef DSA3D_DEBUG
+    unsigned long long word = 0ull;
+    const cudaError_t e = cudaMemcpyFromSymbol(&word, g_debug_word, sizeof(word));     // synchronises with the device
+    if (e != cudaSuccess) return cuda_failed(e);
+    *code = static_cast<int>(word >> 56);
+    long long off = static_cast<long long>(word & ((1ull << 56) - 1));
+    if (off & (1LL << 55)) off -= (1LL << 56);                                          // sign of the 56-bit field
+    *offset = off;
+#endif
+    return DSA3D_OK;
+}
+
+int dsa3d_debug_clear(void) {
+#ifdef DSA3D_DEBUG
+    const unsigned long long zero = 0ull;
+    const cudaError_t e = cudaMemcpyToSymbol(g_debug_word, &zero, sizeof(zero));
+    if (e != cudaSuccess) return cuda_failed(e);
+#endif
     return DSA3D_OK;
 }
 

@@ -94,6 +94,7 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
     const long long head_off = static_cast<long long>(m) * D + ch;
     const T* kh = k + head_off;
     const long long v_minus_k = v - k;                       // same layout: V row = K row + this
+    [[maybe_unused]] const long long kv_extent = pr.N * pr.heads * D;      // elements of K, V, dK, dV: checked build
 
     float u_acc[VEC], kbar[VEC];
 #pragma unroll
@@ -155,10 +156,10 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
                     // corners 0, 1 (x+1), 2 (y+1), 4 (t+1)
                     Row k0 = E::zero(), k1 = E::zero(), k2 = E::zero(), k4 = E::zero();
                     Row v0 = E::zero(), v1 = E::zero(), v2 = E::zero(), v4 = E::zero();
-                    if (s.mask & 1u) { k0 = E::load(kp4[0]); v0 = E::load(kp4[0] + v_minus_k); }
-                    if (s.mask & 2u) { k1 = E::load(kp4[0] + sx); v1 = E::load(kp4[0] + sx + v_minus_k); }
-                    if (s.mask & 4u) { k2 = E::load(kp4[1]); v2 = E::load(kp4[1] + v_minus_k); }
-                    if (s.mask & 16u) { k4 = E::load(kp4[2]); v4 = E::load(kp4[2] + v_minus_k); }
+                    if ((s.mask & 1u) && DSA3D_IN_RANGE(pr, kp4[0] - k, kv_extent, 5)) { k0 = E::load(kp4[0]); v0 = E::load(kp4[0] + v_minus_k); }
+                    if ((s.mask & 2u) && DSA3D_IN_RANGE(pr, kp4[0] + sx - k, kv_extent, 5)) { k1 = E::load(kp4[0] + sx); v1 = E::load(kp4[0] + sx + v_minus_k); }
+                    if ((s.mask & 4u) && DSA3D_IN_RANGE(pr, kp4[1] - k, kv_extent, 5)) { k2 = E::load(kp4[1]); v2 = E::load(kp4[1] + v_minus_k); }
+                    if ((s.mask & 16u) && DSA3D_IN_RANGE(pr, kp4[2] - k, kv_extent, 5)) { k4 = E::load(kp4[2]); v4 = E::load(kp4[2] + v_minus_k); }
                     a[0] = E::dot(qr, k0, 0.0f); b[0] = E::dot(dor, v0, 0.0f);
                     a[1] = E::dot(qr, k1, 0.0f); b[1] = E::dot(dor, v1, 0.0f);
                     a[2] = E::dot(qr, k2, 0.0f); b[2] = E::dot(dor, v2, 0.0f);
@@ -173,7 +174,7 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
                         const bool needed = (w[c] != 0.0f) | (wy[cy] * wx[cx] != 0.0f) | (wt[ct] * wx[cx] != 0.0f) |
                                             (wt[ct] * wy[cy] != 0.0f);
                         a[c] = b[c] = 0.0f;
-                        if (((s.mask >> c) & 1u) && needed) {
+                        if (((s.mask >> c) & 1u) && needed && DSA3D_IN_RANGE(pr, kp4[c >> 1] + cx * sx - k, kv_extent, 6)) {
                             const T* pk = kp4[c >> 1] + cx * sx;
                             const Row kk = E::load(pk);
                             const Row vv = E::load(pk + v_minus_k);
@@ -276,7 +277,8 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const float w = wt[c >> 2] * wy[(c >> 1) & 1] * wx[c & 1];
-                if (((s.mask >> c) & 1u) && w != 0.0f) {
+                if (((s.mask >> c) & 1u) && w != 0.0f &&
+                    DSA3D_IN_RANGE(pr, head_off + s.base * tok_stride + ((c >> 2) * st + ((c >> 1) & 1) * sy + (c & 1) * sx), kv_extent, 7)) {
                     const long long o = s.base * tok_stride + ((c >> 2) * st + ((c >> 1) & 1) * sy + (c & 1) * sx);
                     const float wk = w * ck, wv = w * cv;
                     float* pk = dk_h + o;
@@ -376,8 +378,9 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                         const float w = wt[c >> 2] * wy[(c >> 1) & 1] * wx[c & 1];
                         if (((mask >> c) & 1u) && w != 0.0f) {
                             const int bin = bin0 + ((c >> 2) * ey + ((c >> 1) & 1)) * ex + (c & 1);
+                            if (!DSA3D_IN_RANGE(pr, bin, NB, 8)) continue;
                             const unsigned slot = atomicAdd(&cursor[bin], 1u);
-                            if (sweep == 1) {
+                            if (sweep == 1 && DSA3D_IN_RANGE(pr, slot, scratch_entries_per_cta, 9)) {
                                 my_scratch[slot] = make_uint4(static_cast<unsigned>(ql * kPairBytes),
                                                               __float_as_uint(w * cf.x), __float_as_uint(w * cf.y), 0u);
                             }
@@ -486,10 +489,12 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                     const int bx = bin % ex, by = (bin / ex) % ey, bt = bin / (ex * ey);
                     const long long tok = (static_cast<long long>(lo_t + bt) * pr.H + (lo_y + by)) * pr.W + (lo_x + bx);
                     const long long o = tok * tok_stride + static_cast<long long>(m) * D + hl * 8;
+                    if (DSA3D_IN_RANGE(pr, tok, pr.N, 10)) {
                     red_add_v4(acc_dk + o, ak[0], ak[1], ak[2], ak[3]);
                     red_add_v4(acc_dk + o + 4, ak[4], ak[5], ak[6], ak[7]);
                     red_add_v4(acc_dv + o, av[0], av[1], av[2], av[3]);
                     red_add_v4(acc_dv + o + 4, av[4], av[5], av[6], av[7]);
+                    }
                 }
             }
         }

@@ -27,7 +27,27 @@ struct Problem {
     int tile_t, tile_y, tile_x, halo;
     int tiles_t, tiles_y, tiles_x;
     int tt_begin, tt_count;   // tile rows along t that the tile kernel visits (all: 0, tiles_t)
+    // Checked build (-DDSA3D_DEBUG) only: device word that receives the first out-of-range index a
+    // kernel was about to use (0 = none); NULL otherwise.
+    unsigned long long* debug_word;
 };
+
+// Checked build: every row a gather reads and every row or bin a scatter writes is tested against its
+// tensor's extent first; a violation is recorded (first one wins: code in the top 8 bits, the offending
+// element offset in the rest) and the access is skipped - nothing traps.  In the normal build the
+// tests compile to `true`.
+#ifdef DSA3D_DEBUG
+__device__ __forceinline__ bool debug_in_range(const Problem& pr, long long offset, long long extent, int code) {
+    if (offset >= 0 && offset < extent) return true;
+    if (pr.debug_word)
+        atomicCAS(pr.debug_word, 0ull, (static_cast<unsigned long long>(code) << 56) |
+                                           (static_cast<unsigned long long>(offset) & ((1ull << 56) - 1)));
+    return false;
+}
+#define DSA3D_IN_RANGE(pr, offset, extent, code) dsa3d::debug_in_range((pr), (offset), (extent), (code))
+#else
+#define DSA3D_IN_RANGE(pr, offset, extent, code) true
+#endif
 
 // ---------------------------------------------------------------------------------------
 // Element access.  A lane handles NV consecutive 16-byte vectors of a row (8 bf16 or 4 fp32

@@ -58,6 +58,7 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
     const float* off_row = offsets + row * pr.P * 3;
     const T* kh = k + static_cast<long long>(m) * D + ch;    // + tok * heads * D
     const long long v_minus_k = v - k;                       // same layout: V row = K row + this
+    [[maybe_unused]] const long long kv_extent = pr.N * pr.heads * D;      // elements of K (= of V): checked build
 
     float acc[VEC];
 #pragma unroll
@@ -87,8 +88,10 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
                         vv[i] = E::zero();
                         if ((mk & 1u) && jb + i < cnt) {            // corner (0,0,0) inside the grid
                             const T* pk = kh + base * tok_stride;
-                            kk[i] = E::load(pk);
-                            vv[i] = E::load(pk + v_minus_k);
+                            if (DSA3D_IN_RANGE(pr, pk - k, kv_extent, 1)) {
+                                kk[i] = E::load(pk);
+                                vv[i] = E::load(pk + v_minus_k);
+                            }
                         }
                     }
                     float dd[8];
@@ -137,16 +140,18 @@ forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
             if (full) {
                 Row kk[8];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) kk[c] = E::load(kp4[c >> 1] + (c & 1) * sx);
+                for (int c = 0; c < 8; ++c)
+                    kk[c] = DSA3D_IN_RANGE(pr, kp4[c >> 1] + (c & 1) * sx - k, kv_extent, 2) ? E::load(kp4[c >> 1] + (c & 1) * sx) : E::zero();
 #pragma unroll
-                for (int c = 0; c < 8; ++c) vv[c] = E::load(kp4[c >> 1] + (c & 1) * sx + v_minus_k);
+                for (int c = 0; c < 8; ++c)
+                    vv[c] = DSA3D_IN_RANGE(pr, kp4[c >> 1] + (c & 1) * sx - k, kv_extent, 2) ? E::load(kp4[c >> 1] + (c & 1) * sx + v_minus_k) : E::zero();
 #pragma unroll
                 for (int c = 0; c < 8; ++c) sdot = fmaf(w[c], E::dot(qr, kk[c], 0.0f), sdot);
             } else {
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
                     vv[c] = E::zero();
-                    if (((s.mask >> c) & 1u) && w[c] != 0.0f) {
+                    if (((s.mask >> c) & 1u) && w[c] != 0.0f && DSA3D_IN_RANGE(pr, kp4[c >> 1] + (c & 1) * sx - k, kv_extent, 3)) {
                         const T* pk = kp4[c >> 1] + (c & 1) * sx;
                         const Row kk = E::load(pk);
                         vv[c] = E::load(pk + v_minus_k);
