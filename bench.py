@@ -410,10 +410,15 @@ def run_ours(args, wl):
     # the entry point that takes no offsets tensor (tensor-core tile kernel where the shape
     # allows); the backward is the general one on the zero offsets tensor.
     fixed_window = wl.offsets == "zero" and not args.no_fixed_window
+    # offsets below 1 in size: the forward entry point that decides on the device between the tensor-core
+    # tile kernel and the general kernel; the backward is the general one
+    bounded = wl.offsets == "small" and not args.no_fixed_window
 
     def step():
         if fixed_window:
             binding.dsa3d_forward_fixed_window(t["q"], t["k"], t["v"], *dims, wl.window, b["out"], b["lse"])
+        elif bounded:
+            binding.dsa3d_forward_bounded_offsets(t["q"], t["k"], t["v"], t["offsets"], *dims, wl.window, b["out"], b["lse"])
         else:
             binding.dsa3d_forward(t["q"], t["k"], t["v"], t["offsets"], *dims, wl.window, b["out"], b["lse"])
         if wl.backward and fixed_window:
@@ -559,7 +564,8 @@ def run_ours(args, wl):
         "config": {"workload": wl.name, "grid": [wl.T, wl.H, wl.W], "tokens": wl.N, "heads": wl.heads,
                    "d": wl.d, "window": list(wl.window), "storage": str(wl.dtype).replace("torch.", ""),
                    "offsets": f"{wl.offsets} sigma={wl.sigma}", "batch_per_gpu": 1,
-                   "forward_entry": "dsa3d_forward_fixed_window" if fixed_window else "dsa3d_forward",
+                   "forward_entry": ("dsa3d_forward_fixed_window" if fixed_window else
+                                     "dsa3d_forward_bounded_offsets" if bounded else "dsa3d_forward"),
                    "backward_entry": ("dsa3d_backward_fixed_window" if fixed_window else "dsa3d_backward")
                                      if wl.backward else None,
                    "parallelism": (f"one video, heads sharded over {world} ranks (heads of rank 0: {wl.heads})"

@@ -374,6 +374,25 @@ int dsa3d_forward_fixed_window(const void* q, const void* k, const void* v, int 
                                const int window[3], void* out, float* lse, int dtype, void* stream);
 
 /*
+ * dsa3d_forward_bounded_offsets: dsa3d_forward for callers whose learned offsets are small perturbations
+ * of the fixed window (Formulation: the window positions shifted by learned offsets; the ablation on the
+ * effect of offsets compares them with the fixed window).  Same arguments, same out and lse (up to fp32
+ * summation order).  A first kernel checks the offsets tensor; if every component is finite and below 1
+ * in size, every corner of every sample lies in the box "window grown by one position on each side" and
+ * the operator runs as dense tile attention on the tensor cores for bf16, d = 64 or 128 and window (3,3,3):
+ * scores of a 4x4x8 query tile against its region by tcgen05, plane by plane; each logit the trilinear
+ * combination of eight entries of the score tile; the softmax weights times the corner weights summed
+ * per box position; the weighted sum as a second tcgen05 product (weights as bf16 head + remainder).
+ * Otherwise - some offset too large, or another shape - the general kernel runs, so the call is correct
+ * for any offsets; the decision is taken on the device, the call stays asynchronous.  Calls that are in
+ * flight at the same time each use their own gate word (out of 1024).  The environment variable
+ * DSA3D_NO_TENSOR_FIXED_WINDOW forces the general kernel.  Bounded waits as in
+ * dsa3d_offsets_linear_forward (dsa3d_device_timeout_flag).  The backward of such a call is dsa3d_backward.
+ */
+int dsa3d_forward_bounded_offsets(const void* q, const void* k, const void* v, const float* offsets, int T, int H, int W,
+                                  int heads, int d, const int window[3], void* out, float* lse, int dtype, void* stream);
+
+/*
  * dsa3d_backward_fixed_window: backward of the operator with every offset equal to zero, without
  * an offsets tensor: dq, dk, dv (and doffsets, the gradient with respect to the offsets at zero,
  * unless it is NULL) equal those of dsa3d_backward on an all-zero offsets tensor up to fp32

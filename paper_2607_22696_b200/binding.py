@@ -111,6 +111,8 @@ def _declare(lib) -> None:
     lib.dsa3d_test_wait_timeout.argtypes = [ctypes.c_uint, p]
     lib.dsa3d_forward_residual.restype = i
     lib.dsa3d_forward_residual.argtypes = [p, p, p, p, p, i, i, i, i, i, win, p, p, i, p]
+    lib.dsa3d_forward_bounded_offsets.restype = i
+    lib.dsa3d_forward_bounded_offsets.argtypes = [p, p, p, p, i, i, i, i, i, win, p, p, i, p]
     lib.dsa3d_forward_fixed_window.restype = i
     lib.dsa3d_forward_fixed_window.argtypes = [p, p, p, i, i, i, i, i, win, p, p, i, p]
     lib.dsa3d_backward_fixed_window.restype = i
@@ -194,6 +196,20 @@ def dsa3d_forward(q, k, v, offsets, T, H, W, heads, d, window, out, lse, dtype=N
     n = T * H * W * heads
     P = int(window[0]) * int(window[1]) * int(window[2])
     _check(lib.dsa3d_forward(
+        _ptr(q, "q", n * d), _ptr(k, "k", n * d), _ptr(v, "v", n * d),
+        _ptr(offsets, "offsets", n * P * 3, torch.float32), T, H, W, heads, d, _window(window),
+        _ptr(out, "out", n * d), _ptr(lse, "lse", n, torch.float32), code, _stream(stream)))
+
+
+def dsa3d_forward_bounded_offsets(q, k, v, offsets, T, H, W, heads, d, window, out, lse, dtype=None, stream=None) -> None:
+    """dsa3d_forward for offsets that are small perturbations of the window: tensor-core tile kernel when
+    every |offset| < 1 (decided on the device), the general kernel otherwise; see include/dsa3d.h."""
+    lib = load()
+    dt = q.dtype if dtype is None else dtype
+    code = _DTYPES[dt] if isinstance(dt, torch.dtype) else int(dt)
+    n = T * H * W * heads
+    P = int(window[0]) * int(window[1]) * int(window[2])
+    _check(lib.dsa3d_forward_bounded_offsets(
         _ptr(q, "q", n * d), _ptr(k, "k", n * d), _ptr(v, "v", n * d),
         _ptr(offsets, "offsets", n * P * 3, torch.float32), T, H, W, heads, d, _window(window),
         _ptr(out, "out", n * d), _ptr(lse, "lse", n, torch.float32), code, _stream(stream)))

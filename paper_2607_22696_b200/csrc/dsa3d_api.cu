@@ -1,5 +1,6 @@
 // C ABI of the 3D-DSA library: argument validation, workspace layout, launches.
 // Declarations and the contract of every entry point are in include/dsa3d.h.
+#include <atomic>
 #include <cstdlib>
 #include <stdint.h>
 #include <stdio.h>
@@ -159,6 +160,49 @@ int dsa3d_forward_fixed_window(const void* q, const void* k, const void* v, int 
     }
     if (!done) {                      // general kernel, a NULL offsets tensor reads as all zeros
         e = dsa3d::launch_forward(q, k, v, nullptr, nullptr, out, lse, pr, dtype == DSA3D_BF16, st);
+        if (e != cudaSuccess) return cuda_failed(e);
+    }
+    e = record(1, st);
+    return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
+}
+
+namespace {
+// Gate words of dsa3d_forward_bounded_offsets: one per call, taken round-robin, so that calls whose GPU
+// work overlaps (other streams, other threads) do not share one.
+constexpr unsigned kGateWords = 1024;
+__device__ int g_gate_words[kGateWords];
+std::atomic<unsigned> g_next_gate{0};
+}  // namespace
+
+int dsa3d_forward_bounded_offsets(const void* q, const void* k, const void* v, const float* offsets, int T, int H, int W,
+                                  int heads, int d, const int window[3], void* out, float* lse, int dtype, void* stream) {
+    if (!q || !k || !v || !offsets || !out || !lse) return DSA3D_ERR_NULL_POINTER;
+    dsa3d::Problem pr;
+    const int rc = make_problem(T, H, W, heads, d, window, dtype, pr);
+    if (rc != DSA3D_OK) return rc;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(offsets) || !aligned16(out) || !aligned16(lse))
+        return DSA3D_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = record(0, st);
+    if (e != cudaSuccess) return cuda_failed(e);
+    bool tiled = false;
+    if (dsa3d::bounded_offsets_shape_covered(pr, dtype == DSA3D_BF16) && !std::getenv("DSA3D_NO_TENSOR_FIXED_WINDOW")) {
+        void* words = nullptr;
+        e = cudaGetSymbolAddress(&words, g_gate_words);
+        if (e != cudaSuccess) return cuda_failed(e);
+        int* gate = static_cast<int*>(words) + g_next_gate.fetch_add(1u) % kGateWords;
+        e = dsa3d::launch_offsets_bound_check(offsets, pr.items * pr.P * 3, gate, st);
+        if (e != cudaSuccess) return cuda_failed(e);
+        // the tile kernel runs if the check left 0 in the gate, the general kernel if it left 1
+        tiled = dsa3d::try_bounded_offsets_forward(q, k, v, offsets, gate, out, lse, pr, st, &e);
+        if (tiled && e != cudaSuccess) return cuda_failed(e);
+        if (tiled) {
+            e = dsa3d::launch_forward(q, k, v, offsets, nullptr, out, lse, pr, true, st, gate);
+            if (e != cudaSuccess) return cuda_failed(e);
+        }
+    }
+    if (!tiled) {
+        e = dsa3d::launch_forward(q, k, v, offsets, nullptr, out, lse, pr, dtype == DSA3D_BF16, st);
         if (e != cudaSuccess) return cuda_failed(e);
     }
     e = record(1, st);

@@ -42,7 +42,10 @@ constexpr int kPlTT = 4, kPlTY = 4, kPlTX = 8, kPlQ = kPlTT * kPlTY * kPlTX;    
 constexpr int kPlWorkers = 256, kPlThreads = kPlWorkers + 64;      // + loading warp + MMA warp
 constexpr int kPlMaxSlots = 4;
 
-template <int D, int KT, int KH, int KW>
+// BOUNDED = false: fixed window (KT, KH, KW), all offsets zero.  BOUNDED = true: learned offsets with
+// |offset| < 1 on every axis; (KT, KH, KW) is then the BOX of grid positions a query's samples can touch,
+// the window grown by one position on each side, and the window itself is (KT-2, KH-2, KW-2).
+template <int D, int KT, int KH, int KW, bool BOUNDED = false>
 struct PlaneShape {
     static constexpr int NH = D / 64;                               // 64-channel halves of a row
     static constexpr int RT = kPlTT + KT - 1, RY = kPlTY + KH - 1, RX = kPlTX + KW - 1;
@@ -58,7 +61,9 @@ struct PlaneShape {
     static constexpr int Q_BYTES = NH * kPlQ * 128;
     static constexpr int SLOT_HALF = PSP * 128;                     // one 64-channel half of a plane buffer
     static constexpr int SLOT_BYTES = NH * SLOT_HALF;
-    static constexpr int SMALL_BYTES = 2 * kPlWorkers * 4 + 256 + 2048;   // pair arrays, barriers, alignment slack
+    static constexpr int CELLS = KT * KH * KW;
+    static constexpr int BOX_BYTES = BOUNDED ? CELLS * kPlQ * 4 : 0;       // per query: scores, then weights, of its box
+    static constexpr int SMALL_BYTES = 2 * kPlWorkers * 4 + 256 + 2048 + BOX_BYTES;   // pair arrays, barriers, slack, box
     static constexpr int BUDGET = 227 * 1024;
     // Work area: the score staging of pass 1 and the two P matrices of pass 2 share their bytes.
     // Q has its own buffer (so the next tile's Q arrives during pass 2) unless giving it up buys
@@ -78,12 +83,13 @@ struct PlaneShape {
     static_assert(NS >= 2, "at least two plane buffers");
 };
 
-template <int D, int KT, int KH, int KW>
+template <int D, int KT, int KH, int KW, bool BOUNDED = false>
 struct __align__(1024) PlSmem {
-    using S = PlaneShape<D, KT, KH, KW>;
+    using S = PlaneShape<D, KT, KH, KW, BOUNDED>;
     unsigned char work[S::WORK_BYTES];                              // staging (pass 1) / P head + remainder (pass 2) [/ Q]
     unsigned char slot[S::NS][S::NH][S::SLOT_HALF];                 // ring of K or V planes, same image for both uses
     unsigned char q_own[S::Q_SHARED ? 1024 : S::Q_BYTES];           // 64-channel halves, swizzled 128-byte rows
+    float box[BOUNDED ? S::CELLS * kPlQ : 1];                      // [cell][query]
     float pair_max[kPlWorkers], pair_sum[kPlWorkers];
     uint64_t bar_q, bar_full[kPlMaxSlots], bar_slot_free[kPlMaxSlots];
     uint64_t bar_s[2], bar_s_free[2], bar_p_full[2], bar_p_free[2], bar_o;
@@ -103,18 +109,18 @@ __device__ __forceinline__ bool tile_barrier_or(bool flag) {
     return out != 0u;
 }
 
-template <int D, int KT, int KH, int KW>
+template <int D, int KT, int KH, int KW, bool BOUNDED>
 __global__ void __launch_bounds__(kPlThreads, 1)
 fixed_window_planes_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                            const __grid_constant__ CUtensorMap map_v, __nv_bfloat16* __restrict__ out,
                            float* __restrict__ lse, int T, int H, int W, int heads, int tiles_x, int tiles_y,
-                           int total, int* timeout_flag) {
-    using S = PlaneShape<D, KT, KH, KW>;
+                           int total, int* timeout_flag, const float* __restrict__ offsets, const int* __restrict__ gate) {
+    using S = PlaneShape<D, KT, KH, KW, BOUNDED>;
     constexpr int NH = S::NH, RT = S::RT, RX = S::RX, PS = S::PS, PSP = S::PSP, VH = S::VH, NS = S::NS;
     constexpr int JOBS = 2 * RT;                                      // plane loads per tile: RT of K, then RT of V
     extern __shared__ unsigned char raw[];
-    PlSmem<D, KT, KH, KW>& s =
-        *reinterpret_cast<PlSmem<D, KT, KH, KW>*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
+    PlSmem<D, KT, KH, KW, BOUNDED>& s =
+        *reinterpret_cast<PlSmem<D, KT, KH, KW, BOUNDED>*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     unsigned char* q_buf = S::Q_SHARED ? s.work + S::Q_OFFSET : s.q_own;
     unsigned char* p_head = s.work;
@@ -171,7 +177,11 @@ fixed_window_planes_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
         y0 = (tile % tiles_y) * kPlTY;
         t0 = (tile / tiles_y) * kPlTT;
     };
-    const int my_tiles = static_cast<int>(blockIdx.x) < total ? (total - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x) : 0;
+    // BOUNDED: an earlier kernel on the stream left 0 in *gate if every offset is finite and below 1 in size;
+    // otherwise this kernel has nothing to do (the general kernel runs instead)
+    const bool open = !BOUNDED || gate == nullptr || *gate == 0;
+    const int my_tiles = (open && static_cast<int>(blockIdx.x) < total)
+                             ? (total - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x) : 0;
 
     if (warp == kPlWorkers / 32) {
         // ==================================================================== loading thread (lane 0)
@@ -319,13 +329,35 @@ fixed_window_planes_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
             int m, t0, y0, x0;
             locate(static_cast<int>(blockIdx.x) + it * static_cast<int>(gridDim.x), m, t0, y0, x0);
             const int sp0 = it * RT;
-            float sc[KT][VH][KW];
+            float sc[BOUNDED ? 1 : KT][BOUNDED ? 1 : VH][BOUNDED ? 1 : KW];     // fixed window: this thread's window scores
+            if constexpr (!BOUNDED) {
 #pragma unroll
-            for (int u = 0; u < KT; ++u)
+                for (int u = 0; u < KT; ++u)
 #pragma unroll
-                for (int vi = 0; vi < VH; ++vi)
+                    for (int vi = 0; vi < VH; ++vi)
 #pragma unroll
-                    for (int ww = 0; ww < KW; ++ww) sc[u][vi][ww] = -INFINITY;
+                        for (int ww = 0; ww < KW; ++ww) sc[u][vi][ww] = -INFINITY;
+            }
+
+            // BOUNDED: this thread's samples are every other one of the window; their offsets are requested now,
+            // so that they have arrived by the time pass 1 is over
+            constexpr int WT = BOUNDED ? KT - 2 : 1, WH = BOUNDED ? KH - 2 : 1, WW = BOUNDED ? KW - 2 : 1;
+            constexpr int NP = WT * WH * WW, PH = (NP + 1) / 2;
+            const int qt = t0 + lt, qy = y0 + ly, qx = x0 + lx;
+            const bool in_grid = qt < T && qy < H && qx < W;
+            const long long n = (static_cast<long long>(qt) * H + qy) * W + qx;
+            float offv[BOUNDED ? PH : 1][3];
+            if constexpr (BOUNDED) {
+                const float* off_row = offsets + (n * heads + m) * (NP * 3);
+#pragma unroll
+                for (int i = 0; i < PH; ++i) {
+                    const int p = 2 * i + half;
+                    offv[i][0] = offv[i][1] = offv[i][2] = 0.0f;
+                    if (in_grid && p < NP) {
+                        offv[i][0] = __ldg(off_row + p * 3); offv[i][1] = __ldg(off_row + p * 3 + 1); offv[i][2] = __ldg(off_row + p * 3 + 2);
+                    }
+                }
+            }
 
             // ---------------------------------------------------------- pass 1: the window's scores, plane by plane
             for (int pl = 0; pl < RT; ++pl) {
@@ -350,8 +382,11 @@ fixed_window_planes_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                             const int vv = vi + half * VH;
                             if (vv >= KH) continue;
 #pragma unroll
-                            for (int ww = 0; ww < KW; ++ww)
-                                sc[u][vi][ww] = stage[kCacheCells ? cell_stage[kCacheCells ? vi : 0][kCacheCells ? ww : 0] : stage_index(vv, ww)] * lscale;
+                            for (int ww = 0; ww < KW; ++ww) {
+                                const float sv = stage[kCacheCells ? cell_stage[kCacheCells ? vi : 0][kCacheCells ? ww : 0] : stage_index(vv, ww)] * lscale;
+                                if constexpr (BOUNDED) s.box[((u * KH + vv) * KW + ww) * kPlQ + r] = sv;
+                                else sc[u][vi][ww] = sv;
+                            }
                         }
                     }
                     named_barrier_sync(1 + lt, 64);                   // both have picked: the staging rows may be refilled
@@ -361,34 +396,124 @@ fixed_window_planes_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                 if (lane == 0) mbar_arrive(smem_u32(&s.bar_s_free[sp & 1]));
             }
 
-            // ---------------------------------------------------------- softmax over the window (two threads per query)
-            float mx = -INFINITY;
+            float mx, sum, inv;
+            if constexpr (BOUNDED) {
+                // ------------------------------------------------------ learned offsets below 1 in size: the eight corners
+                // of every sample lie in the query's box, whose scores are in shared memory.  The two threads of
+                // a query take every other sample: logit = trilinear combination of the corner scores (positions
+                // outside the grid hold 0: the zero-padded key), softmax, then the weights alpha_p * w_c are summed
+                // into the box cells in place of the scores.
+                named_barrier_sync(1 + lt, 64);                       // the whole box is in place
+                float lg[PH], fr[PH][3];
+                int cellv[PH];
+                // position of a sample relative to the box origin, exactly as the general kernel forms it:
+                // float(coord + b) + offset, floor, difference - all in fp32
 #pragma unroll
-            for (int u = 0; u < KT; ++u)
+                for (int i = 0; i < PH; ++i) {
+                    const int p = 2 * i + half;
+                    const int w = p % WW, v = (p / WW) % WH, u = p / (WW * WH);
+                    const float pt = __fadd_rn(static_cast<float>(qt + u - WT / 2), offv[i][0]),
+                                py = __fadd_rn(static_cast<float>(qy + v - WH / 2), offv[i][1]),
+                                px = __fadd_rn(static_cast<float>(qx + w - WW / 2), offv[i][2]);
+                    const float flt = floorf(pt), fly = floorf(py), flx = floorf(px);
+                    float ft = __fsub_rn(pt, flt), fy = __fsub_rn(py, fly), fx = __fsub_rn(px, flx);
+                    // cell index of corner (0,0,0) inside the box (origin = query - K/2).  An offset just below +1
+                    // can round the fp32 position up to the next integer: the sample then sits exactly on the
+                    // box's last position, which is written as the cell before it with fraction 1.  (The clamps
+                    // also keep a garbage offset from indexing outside the box.)
+                    int ct = max(static_cast<int>(flt) - (qt - KT / 2), 0), cy = max(static_cast<int>(fly) - (qy - KH / 2), 0),
+                        cx = max(static_cast<int>(flx) - (qx - KW / 2), 0);
+                    if (ct > KT - 2) { ct = KT - 2; ft = 1.0f; }
+                    if (cy > KH - 2) { cy = KH - 2; fy = 1.0f; }
+                    if (cx > KW - 2) { cx = KW - 2; fx = 1.0f; }
+                    cellv[i] = ((ct * KH + cy) * KW + cx) * kPlQ + r;
+                    fr[i][0] = ft; fr[i][1] = fy; fr[i][2] = fx;
+                }
+                mx = -INFINITY;
 #pragma unroll
-                for (int vi = 0; vi < VH; ++vi)
+                for (int i = 0; i < PH; ++i) {
+                    const int p = 2 * i + half;
+                    lg[i] = -INFINITY;
+                    if (p < NP) {
+                        const float ft = fr[i][0], fy = fr[i][1], fx = fr[i][2];
+                        const float* bx = s.box + cellv[i];
+                        float a[8];
 #pragma unroll
-                    for (int ww = 0; ww < KW; ++ww) mx = fmaxf(mx, sc[u][vi][ww]);
-            s.pair_max[tid] = mx;
-            named_barrier_sync(1 + lt, 64);
-            mx = fmaxf(mx, s.pair_max[tid ^ 128]);
-            float sum = 0.0f;
-#pragma unroll
-            for (int u = 0; u < KT; ++u)
-#pragma unroll
-                for (int vi = 0; vi < VH; ++vi)
-#pragma unroll
-                    for (int ww = 0; ww < KW; ++ww) {
-                        sc[u][vi][ww] = exp2f(sc[u][vi][ww] - mx);        // cells this thread does not own: exp2(-inf) = 0
-                        sum += sc[u][vi][ww];
+                        for (int c = 0; c < 8; ++c) a[c] = bx[(((c >> 2) * KH + ((c >> 1) & 1)) * KW + (c & 1)) * kPlQ];
+                        const float x0v = fmaf(fx, a[1] - a[0], a[0]), x1v = fmaf(fx, a[3] - a[2], a[2]);
+                        const float x2v = fmaf(fx, a[5] - a[4], a[4]), x3v = fmaf(fx, a[7] - a[6], a[6]);
+                        const float y0v = fmaf(fy, x1v - x0v, x0v), y1v = fmaf(fy, x3v - x2v, x2v);
+                        lg[i] = fmaf(ft, y1v - y0v, y0v);
+                        mx = fmaxf(mx, lg[i]);
                     }
-            s.pair_sum[tid] = sum;
-            named_barrier_sync(1 + lt, 64);
-            sum += s.pair_sum[tid ^ 128];
-            const float inv = 1.0f / sum;
-            const int qt = t0 + lt, qy = y0 + ly, qx = x0 + lx;
-            const bool in_grid = qt < T && qy < H && qx < W;
-            const long long n = (static_cast<long long>(qt) * H + qy) * W + qx;
+                }
+                s.pair_max[tid] = mx;
+                named_barrier_sync(1 + lt, 64);
+                mx = fmaxf(mx, s.pair_max[tid ^ 128]);
+                sum = 0.0f;
+#pragma unroll
+                for (int i = 0; i < PH; ++i) { lg[i] = exp2f(lg[i] - mx); sum += lg[i]; }
+                s.pair_sum[tid] = sum;
+                named_barrier_sync(1 + lt, 64);                       // also: every score of the box has been read
+                sum += s.pair_sum[tid ^ 128];
+                inv = 1.0f / sum;
+                // the box now collects the weights: cleared (each thread its rows), then the two threads add
+                // their samples one after the other (plain read-add-write: no two threads at a cell at once)
+#pragma unroll
+                for (int u = 0; u < KT; ++u)
+#pragma unroll
+                    for (int vi = 0; vi < VH; ++vi) {
+                        const int vv = vi + half * VH;
+                        if (vv >= KH) continue;
+#pragma unroll
+                        for (int ww = 0; ww < KW; ++ww) s.box[((u * KH + vv) * KW + ww) * kPlQ + r] = 0.0f;
+                    }
+                named_barrier_sync(1 + lt, 64);
+#pragma unroll
+                for (int turn = 0; turn < 2; ++turn) {
+                    if (turn == half) {
+#pragma unroll
+                        for (int i = 0; i < PH; ++i) {
+                            const int p = 2 * i + half;
+                            if (p >= NP) continue;
+                            const float ft = fr[i][0], fy = fr[i][1], fx = fr[i][2];
+                            float* bx = s.box + cellv[i];
+                            const float al = lg[i] * inv;
+                            const float wt[2] = {1.0f - ft, ft}, wy[2] = {1.0f - fy, fy}, wx[2] = {1.0f - fx, fx};
+#pragma unroll
+                            for (int c = 0; c < 8; ++c)
+                                bx[(((c >> 2) * KH + ((c >> 1) & 1)) * KW + (c & 1)) * kPlQ] += al * (wt[c >> 2] * wy[(c >> 1) & 1] * wx[c & 1]);
+                        }
+                    }
+                    named_barrier_sync(1 + lt, 64);
+                }
+            } else {
+                // ------------------------------------------------------ softmax over the window (two threads per query)
+                mx = -INFINITY;
+    #pragma unroll
+                for (int u = 0; u < KT; ++u)
+    #pragma unroll
+                    for (int vi = 0; vi < VH; ++vi)
+    #pragma unroll
+                        for (int ww = 0; ww < KW; ++ww) mx = fmaxf(mx, sc[u][vi][ww]);
+                s.pair_max[tid] = mx;
+                named_barrier_sync(1 + lt, 64);
+                mx = fmaxf(mx, s.pair_max[tid ^ 128]);
+                sum = 0.0f;
+    #pragma unroll
+                for (int u = 0; u < KT; ++u)
+    #pragma unroll
+                    for (int vi = 0; vi < VH; ++vi)
+    #pragma unroll
+                        for (int ww = 0; ww < KW; ++ww) {
+                            sc[u][vi][ww] = exp2f(sc[u][vi][ww] - mx);        // cells this thread does not own: exp2(-inf) = 0
+                            sum += sc[u][vi][ww];
+                        }
+                s.pair_sum[tid] = sum;
+                named_barrier_sync(1 + lt, 64);
+                sum += s.pair_sum[tid ^ 128];
+                inv = 1.0f / sum;
+            }
             if (half == 0 && in_grid) lse[n * heads + m] = (mx + log2f(sum)) * kLn2;
 
             // ---------------------------------------------------------- pass 2: this query's row of P, plane by plane
@@ -424,7 +549,11 @@ fixed_window_planes_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
 #pragma unroll
                                 for (int ww = 0; ww < KW; ++ww) {
                                     float p = 0.0f;
-                                    if (u < KT) p = sc[u < KT ? u : 0][vi][ww] * inv;
+                                    if constexpr (BOUNDED) {
+                                        if (u < KT) p = s.box[(((u < KT ? u : 0) * KH + vv) * KW + ww) * kPlQ + r];
+                                    } else {
+                                        if (u < KT) p = sc[u < KT ? u : 0][vi][ww] * inv;
+                                    }
                                     __nv_bfloat16 val = __float2bfloat16_rn(p);
                                     if (part) val = __float2bfloat16_rn(p - __bfloat162float(val));
                                     *reinterpret_cast<__nv_bfloat16*>(dst + (kCacheCells ? cell_p[kCacheCells ? vi : 0][kCacheCells ? ww : 0] : p_offset(vv, ww))) = val;
@@ -495,13 +624,13 @@ bool make_plane_maps(const void* q, const void* k, const void* v, const Problem&
            encode_tensor_map_bf16(mv, v, 5, dims, strides, box_p, true);
 }
 
-template <int D, int KT, int KH, int KW>
+template <int D, int KT, int KH, int KW, bool BOUNDED>
 cudaError_t launch_planes(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, void* out, float* lse,
-                          const Problem& pr, int* flag, cudaStream_t stream) {
+                          const Problem& pr, int* flag, const float* offsets, const int* gate, cudaStream_t stream) {
     const int tiles_x = (pr.W + kPlTX - 1) / kPlTX, tiles_y = (pr.H + kPlTY - 1) / kPlTY,
               tiles_t = (pr.T + kPlTT - 1) / kPlTT;
-    const size_t smem = sizeof(PlSmem<D, KT, KH, KW>) + 1024;
-    auto kern = fixed_window_planes_kernel<D, KT, KH, KW>;
+    const size_t smem = sizeof(PlSmem<D, KT, KH, KW, BOUNDED>) + 1024;
+    auto kern = fixed_window_planes_kernel<D, KT, KH, KW, BOUNDED>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
     const long long total = static_cast<long long>(tiles_x) * tiles_y * tiles_t * pr.heads;
@@ -513,8 +642,23 @@ cudaError_t launch_planes(const CUtensorMap& mq, const CUtensorMap& mk, const CU
     if (e != cudaSuccess) return e;
     const unsigned grid = static_cast<unsigned>(total < sms ? total : sms);     // persistent: one CTA per SM
     kern<<<grid, kPlThreads, smem, stream>>>(mq, mk, mv, static_cast<__nv_bfloat16*>(out), lse, pr.T, pr.H, pr.W, pr.heads,
-                                             tiles_x, tiles_y, static_cast<int>(total), flag);
+                                             tiles_x, tiles_y, static_cast<int>(total), flag, offsets, gate);
     return cudaGetLastError();
+}
+
+// *gate = 1 if some offset component is NaN, infinite or not below 1 in size (plain stores of the same
+// value: no ordering needed).  The caller has set *gate = 0 on the same stream.
+__global__ void __launch_bounds__(256)
+offsets_bound_kernel(const float4* __restrict__ off4, long long count4, const float* __restrict__ tail, int tail_count,
+                     int* __restrict__ gate) {
+    bool bad = false;
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < count4; i += stride) {
+        const float4 o = __ldg(off4 + i);
+        bad = bad || !(fabsf(o.x) < 1.0f) || !(fabsf(o.y) < 1.0f) || !(fabsf(o.z) < 1.0f) || !(fabsf(o.w) < 1.0f);
+    }
+    if (blockIdx.x == 0 && static_cast<int>(threadIdx.x) < tail_count) bad = bad || !(fabsf(tail[threadIdx.x]) < 1.0f);
+    if (__syncthreads_or(bad) && threadIdx.x == 0) *gate = 1;
 }
 
 }  // namespace
@@ -532,11 +676,42 @@ bool try_fixed_window_forward_planes(const void* q, const void* k, const void* v
     CUtensorMap mq, mk, mv;
     if (!flag || !make_plane_maps(q, k, v, pr, pr.kh, pr.kw, &mq, &mk, &mv)) return false;
     if (pr.d == 128)
-        *err = w355 ? launch_planes<128, 3, 5, 5>(mq, mk, mv, out, lse, pr, flag, stream)
-                    : launch_planes<128, 3, 7, 7>(mq, mk, mv, out, lse, pr, flag, stream);
+        *err = w355 ? launch_planes<128, 3, 5, 5, false>(mq, mk, mv, out, lse, pr, flag, nullptr, nullptr, stream)
+                    : launch_planes<128, 3, 7, 7, false>(mq, mk, mv, out, lse, pr, flag, nullptr, nullptr, stream);
     else
-        *err = w355 ? launch_planes<64, 3, 5, 5>(mq, mk, mv, out, lse, pr, flag, stream)
-                    : launch_planes<64, 3, 7, 7>(mq, mk, mv, out, lse, pr, flag, stream);
+        *err = w355 ? launch_planes<64, 3, 5, 5, false>(mq, mk, mv, out, lse, pr, flag, nullptr, nullptr, stream)
+                    : launch_planes<64, 3, 7, 7, false>(mq, mk, mv, out, lse, pr, flag, nullptr, nullptr, stream);
+    return true;
+}
+
+bool bounded_offsets_shape_covered(const Problem& pr, bool bf16) {
+    return bf16 && (pr.d == 128 || pr.d == 64) && pr.kt == 3 && pr.kh == 3 && pr.kw == 3;
+}
+
+cudaError_t launch_offsets_bound_check(const float* offsets, long long count, int* gate, cudaStream_t stream) {
+    cudaError_t e = cudaMemsetAsync(gate, 0, sizeof(int), stream);
+    if (e != cudaSuccess) return e;
+    const long long count4 = count / 4;
+    long long blocks = (count4 + 255) / 256;
+    if (blocks > 148LL * 8) blocks = 148LL * 8;
+    if (blocks < 1) blocks = 1;
+    offsets_bound_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
+        reinterpret_cast<const float4*>(offsets), count4, offsets + count4 * 4, static_cast<int>(count - count4 * 4), gate);
+    return cudaGetLastError();
+}
+
+bool try_bounded_offsets_forward(const void* q, const void* k, const void* v, const float* offsets, const int* gate,
+                                 void* out, float* lse, const Problem& pr, cudaStream_t stream, cudaError_t* err) {
+    *err = cudaSuccess;
+    if (!bounded_offsets_shape_covered(pr, true)) return false;
+    const long long tiles = static_cast<long long>((pr.W + kPlTX - 1) / kPlTX) * ((pr.H + kPlTY - 1) / kPlTY) *
+                            ((pr.T + kPlTT - 1) / kPlTT);
+    if (tiles * pr.heads * 2 * (kPlTT + pr.kt + 2 - 1) >= (1LL << 31)) return false;
+    int* flag = timeout_flag_device_address();
+    CUtensorMap mq, mk, mv;
+    if (!flag || !make_plane_maps(q, k, v, pr, pr.kh + 2, pr.kw + 2, &mq, &mk, &mv)) return false;
+    *err = pr.d == 128 ? launch_planes<128, 5, 5, 5, true>(mq, mk, mv, out, lse, pr, flag, offsets, gate, stream)
+                       : launch_planes<64, 5, 5, 5, true>(mq, mk, mv, out, lse, pr, flag, offsets, gate, stream);
     return true;
 }
 

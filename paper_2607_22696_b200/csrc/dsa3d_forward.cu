@@ -27,7 +27,8 @@ template <typename T, int D, int NV, bool kAdd>
 __global__ void __launch_bounds__(256, NV == 2 ? 2 : DSA3D_FWD_MINBLOCKS)
 forward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                const float* __restrict__ offsets, const T* addend, T* out, float* __restrict__ lse,
-               const Problem pr) {
+               const Problem pr, const int* __restrict__ gate) {
+    if (gate && *gate == 0) return;                      // another kernel takes this call (see launch_forward)
     using E = Elt<T, NV>;
     using Row = typename E::Row;
     constexpr int VEC = E::VEC;
@@ -204,7 +205,7 @@ template <> struct FwdLaneWidth<__nv_bfloat16, 128> { static constexpr int NV = 
 template <typename T, int D>
 static cudaError_t launch_forward_t(const void* q, const void* k, const void* v, const float* offsets,
                                     const void* addend, void* out, float* lse, const Problem& pr,
-                                    cudaStream_t stream) {
+                                    cudaStream_t stream, const int* gate) {
     constexpr int NV = FwdLaneWidth<T, D>::NV;
     constexpr int LPR = D / Elt<T, NV>::VEC;
     constexpr int threads = 256;
@@ -213,20 +214,20 @@ static cudaError_t launch_forward_t(const void* q, const void* k, const void* v,
     if (addend)
         forward_kernel<T, D, NV, true><<<static_cast<unsigned>(blocks), threads, 0, stream>>>(
             static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), offsets,
-            static_cast<const T*>(addend), static_cast<T*>(out), lse, pr);
+            static_cast<const T*>(addend), static_cast<T*>(out), lse, pr, gate);
     else
         forward_kernel<T, D, NV, false><<<static_cast<unsigned>(blocks), threads, 0, stream>>>(
             static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), offsets, nullptr,
-            static_cast<T*>(out), lse, pr);
+            static_cast<T*>(out), lse, pr, gate);
     return cudaGetLastError();
 }
 
 cudaError_t launch_forward(const void* q, const void* k, const void* v, const float* offsets, const void* addend,
-                           void* out, float* lse, const Problem& pr, bool bf16, cudaStream_t stream) {
-#define DSA3D_CASE(DD)                                                                              \
-    case DD:                                                                                        \
-        return bf16 ? launch_forward_t<__nv_bfloat16, DD>(q, k, v, offsets, addend, out, lse, pr, stream)   \
-                    : launch_forward_t<float, DD>(q, k, v, offsets, addend, out, lse, pr, stream);
+                           void* out, float* lse, const Problem& pr, bool bf16, cudaStream_t stream, const int* gate) {
+#define DSA3D_CASE(DD)                                                                                    \
+    case DD:                                                                                              \
+        return bf16 ? launch_forward_t<__nv_bfloat16, DD>(q, k, v, offsets, addend, out, lse, pr, stream, gate)   \
+                    : launch_forward_t<float, DD>(q, k, v, offsets, addend, out, lse, pr, stream, gate);
     switch (pr.d) {
         DSA3D_CASE(32)
         DSA3D_CASE(64)

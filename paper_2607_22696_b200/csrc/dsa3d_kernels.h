@@ -10,8 +10,10 @@ namespace dsa3d {
 
 // `addend` (same layout and type as out, or NULL) is added to the attention output before the
 // single rounding to the storage type: the first term of Eq. 1.
+// `gate` (or NULL): a device word; when given, the kernel does nothing unless it is non-zero.
 cudaError_t launch_forward(const void* q, const void* k, const void* v, const float* offsets, const void* addend,
-                           void* out, float* lse, const Problem& pr, bool bf16, cudaStream_t stream);
+                           void* out, float* lse, const Problem& pr, bool bf16, cudaStream_t stream,
+                           const int* gate = nullptr);
 
 // Remember `e` as the calling thread's last CUDA error (dsa3d_last_cuda_error) and return
 // DSA3D_ERR_CUDA.
@@ -81,5 +83,15 @@ bool try_fixed_window_forward(const void* q, const void* k, const void* v, void*
 // tensor cores, the halo region taken one plane at a time.
 bool try_fixed_window_forward_planes(const void* q, const void* k, const void* v, void* out, float* lse,
                                      const Problem& pr, cudaStream_t stream, cudaError_t* err);
+
+// Forward for learned offsets below 1 in size on every axis (dsa3d_fixed_window_planes.cu): the samples of
+// a query then stay inside the box "window grown by one position", and the operator runs as dense tile
+// attention on the tensor cores.  launch_offsets_bound_check leaves *gate = 0 if all `count` offset
+// components are finite and below 1 in size, else 1; try_bounded_offsets_forward launches the tile kernel,
+// which does nothing unless *gate == 0 (false: shape not covered, nothing launched).
+bool bounded_offsets_shape_covered(const Problem& pr, bool bf16);
+cudaError_t launch_offsets_bound_check(const float* offsets, long long count, int* gate, cudaStream_t stream);
+bool try_bounded_offsets_forward(const void* q, const void* k, const void* v, const float* offsets, const int* gate,
+                                 void* out, float* lse, const Problem& pr, cudaStream_t stream, cudaError_t* err);
 
 }  // namespace dsa3d

@@ -158,6 +158,9 @@ WORKLOADS: Dict[str, Workload] = {w.name: w for w in [
     # not a BASELINE config: the fixed-window variant of the paper's ablation on the effect of offsets
     # (window (3,7,7), all offsets zero) on the grid of the sweep
     Workload("sweep_w377_zero", 64, 45, 80, 16, 128, (3, 7, 7), _BF16, 0.0, 4, offsets="zero"),
+    # not a BASELINE config: offsets as small perturbations of the window (every component below 1 in
+    # size), the regime in which the forward runs as tile attention on the tensor cores
+    Workload("sweep_w333_small", 64, 45, 80, 16, 128, (3, 3, 3), _BF16, 0.4, 4, offsets="small"),
 ]}
 
 
@@ -178,6 +181,9 @@ def make_offsets(wl: Workload, device="cpu", frames=None) -> torch.Tensor:
                      torch.float32, device, first=t0 * wl.H * wl.W * wl.heads * 3)
         jit = normal(shape, wl.seed, TENSOR_IDS["offsets"], 0.3, torch.float32, device, first=first)
         return jit.add_(vel)
+    if wl.offsets == "small":
+        # learned offsets as small perturbations of the fixed window: N(0, sigma^2) cut off below 1 in size
+        return normal(shape, wl.seed, TENSOR_IDS["offsets"], wl.sigma, torch.float32, device, first=first).clamp_(-0.999, 0.999)
     return normal(shape, wl.seed, TENSOR_IDS["offsets"], wl.sigma, torch.float32, device, first=first)
 
 

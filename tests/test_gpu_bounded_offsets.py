@@ -1,0 +1,111 @@
+"""dsa3d_forward_bounded_offsets: the forward for learned offsets that are small perturbations of the
+fixed window.  When every offset component is finite and below 1 in size the operator runs as dense
+tile attention on the tensor cores (logits = trilinear combinations of entries of the Q.K^T tile,
+weighted sum as a second tcgen05 product); otherwise the general kernel runs.  Both roads are
+compared with the CPU oracle on the same offsets, element by element."""
+import os
+
+import pytest
+import torch
+
+import oracle
+import parity_util as pu
+from paper_2607_22696_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+BF16, F32 = torch.bfloat16, torch.float32
+
+
+def _bounded_offsets(shape, seed, kind):
+    """Offsets with |component| < 1: uniform in (-1, 1), tiny, zero, or pushed against the bound."""
+    n = 1
+    for x in shape:
+        n *= x
+    g = torch.Generator().manual_seed(seed)
+    if kind == "uniform":
+        off = torch.rand(n, generator=g, dtype=torch.float64) * 2 - 1
+        off = off.clamp(-0.999999, 0.999999).to(F32)
+    elif kind == "tiny":
+        off = ((torch.rand(n, generator=g, dtype=torch.float64) * 2 - 1) * 1e-3).to(F32)
+    elif kind == "zero":
+        off = torch.zeros(n, dtype=F32)
+    elif kind == "edge":                      # values next to -1, 0 and +1, where the cell of a sample changes
+        pick = torch.randint(0, 6, (n,), generator=g)
+        table = torch.tensor([-0.99999994, -1e-7, 0.0, 1e-7, 0.99999994, 0.5], dtype=F32)
+        off = table[pick]
+    else:
+        raise ValueError(kind)
+    assert float(off.abs().max()) < 1.0
+    return off.view(shape)
+
+
+def _run(shape, window, dtype, seed, offsets, sigma_q=1.0):
+    T, H, W, heads, d = shape
+    q, k, v = (inputs.normal(shape, seed, i, sigma_q if i == 0 else 1.0, dtype) for i in range(3))
+    out = torch.full(shape, float("nan"), dtype=dtype, device="cuda")
+    lse = torch.full((T, H, W, heads), float("nan"), dtype=F32, device="cuda")
+    binding.dsa3d_forward_bounded_offsets(q.cuda(), k.cuda(), v.cuda(), offsets.cuda(), T, H, W, heads, d, window, out, lse)
+    torch.cuda.synchronize()
+    assert binding.dsa3d_device_timeout_flag() == 0
+    P = window[0] * window[1] * window[2]
+    o_ref, l_ref = oracle.forward(q.view(-1, heads, d), k, v, offsets.view(-1, heads, P, 3), T, H, W, heads, d, window)
+    pu.assert_close("out", out, o_ref.view(shape), dtype)
+    pu.assert_close("lse", lse, l_ref.view(T, H, W, heads), dtype)
+    return q, k, v, out, lse
+
+
+@pytest.mark.parametrize("shape", [(6, 9, 13, 2, 128), (4, 4, 8, 1, 128), (1, 1, 1, 1, 128), (9, 5, 17, 3, 128),
+                                   (2, 13, 7, 2, 128), (8, 8, 16, 2, 64), (5, 4, 19, 3, 64)])
+@pytest.mark.parametrize("kind", ["uniform", "edge"])
+def test_tile_kernel_for_offsets_below_one_matches_the_oracle(shape, kind):
+    T, H, W, heads, d = shape
+    off = _bounded_offsets((T, H, W, heads, 27, 3), 700 + T * W, kind)
+    _run(shape, (3, 3, 3), BF16, 170, off)
+
+
+@pytest.mark.parametrize("kind", ["tiny", "zero"])
+def test_tile_kernel_many_tiles_sharp_softmax(kind):
+    shape = (12, 20, 40, 4, 128)
+    T, H, W, heads, d = shape
+    off = _bounded_offsets((T, H, W, heads, 27, 3), 710, kind)
+    _run(shape, (3, 3, 3), BF16, 171, off, sigma_q=5.0)
+
+
+def test_the_two_roads_agree_and_one_large_offset_switches_to_the_general_kernel():
+    """The same bounded problem through the tile kernel and through the general kernel (forced by the
+    environment switch): within one bf16 step of each other.  Then a single offset of size 1.5, a NaN
+    and an infinity: the device-side check must send the whole call to the general kernel, whose result
+    is dsa3d_forward's bit for bit."""
+    shape, window = (8, 10, 20, 3, 128), (3, 3, 3)
+    T, H, W, heads, d = shape
+    off = _bounded_offsets((T, H, W, heads, 27, 3), 720, "uniform")
+    q, k, v, out_tc, lse_tc = _run(shape, window, BF16, 172, off)
+    dq, dk, dv = q.cuda(), k.cuda(), v.cuda()
+    os.environ["DSA3D_NO_TENSOR_FIXED_WINDOW"] = "1"
+    try:
+        out_g, lse_g = torch.empty_like(out_tc), torch.empty_like(lse_tc)
+        binding.dsa3d_forward_bounded_offsets(dq, dk, dv, off.cuda(), T, H, W, heads, d, window, out_g, lse_g)
+        torch.cuda.synchronize()
+    finally:
+        del os.environ["DSA3D_NO_TENSOR_FIXED_WINDOW"]
+    assert float((lse_tc - lse_g).abs().max()) <= 1e-4
+    ulp = (out_g.float().abs() * 2.0 ** -7).clamp_min(2e-3)
+    assert bool(((out_tc.float() - out_g.float()).abs() <= ulp).all())
+    for bad in (1.5, float("nan"), float("inf"), -1.0):
+        off2 = off.clone()
+        off2.view(-1)[off2.numel() // 2 + 1] = bad
+        out_a, lse_a = torch.full_like(out_tc, float("nan")), torch.full_like(lse_tc, float("nan"))
+        out_b, lse_b = torch.empty_like(out_tc), torch.empty_like(lse_tc)
+        binding.dsa3d_forward_bounded_offsets(dq, dk, dv, off2.cuda(), T, H, W, heads, d, window, out_a, lse_a)
+        binding.dsa3d_forward(dq, dk, dv, off2.cuda(), T, H, W, heads, d, window, out_b, lse_b)
+        torch.cuda.synchronize()
+        assert torch.equal(out_a, out_b) and torch.equal(lse_a, lse_b), bad
+
+
+@pytest.mark.parametrize("shape,window,dtype", [((4, 6, 7, 2, 32), (3, 3, 3), BF16), ((3, 5, 6, 2, 32), (3, 3, 3), F32),
+                                                ((4, 6, 9, 2, 128), (2, 2, 2), BF16), ((4, 6, 9, 2, 64), (3, 5, 5), BF16)])
+def test_other_shapes_take_the_general_kernel(shape, window, dtype):
+    T, H, W, heads, d = shape
+    P = window[0] * window[1] * window[2]
+    off = _bounded_offsets((T, H, W, heads, P, 3), 730, "uniform")
+    _run(shape, window, dtype, 173, off)
