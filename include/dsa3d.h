@@ -47,6 +47,12 @@
  *   DSA3D_TILE="tt,ty,tx,halo"     query tiling of the dK/dV pre-reduction of dsa3d_backward
  *                                  (default 4,8,8,6; "0" = no tiling, every contribution is an
  *                                  atomic add); also changes dsa3d_backward_workspace_bytes
+ *   DSA3D_KEY_BLOCKS=1             dsa3d_backward (bf16, d = 64 or 128, extents up to 1022) forms dK/dV per
+ *                                  block of 4 x 8 x 8 keys as tensor-core products (coefficient matrix of the
+ *                                  block against chunks of 32 queries, tcgen05 in tf32: the coefficients lose
+ *                                  the bits below 2^-10 relative, q and dO none) instead of the tile kernel's
+ *                                  binning; slower so far; also changes dsa3d_backward_workspace_bytes; a
+ *                                  non-finite q or dO row then reaches every key whose block it lies near
  *   DSA3D_NO_TENSOR_FIXED_WINDOW   dsa3d_forward_fixed_window uses the general kernel
  *   DSA3D_GEMM_ONE_CTA             dsa3d_offsets_linear_forward: one CTA per tile instead of a pair
  *   DSA3D_GEMM_PLAIN_STORES        its epilogue stores from registers instead of by TMA

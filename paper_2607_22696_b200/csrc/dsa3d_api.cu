@@ -59,6 +59,8 @@ int make_problem(int T, int H, int W, int heads, int d, const int* window, int d
     pr.halo = 0;
     pr.tiles_t = pr.tiles_y = pr.tiles_x = 0;
     pr.tt_begin = pr.tt_count = 0;
+    pr.key_blocks = 0;
+    pr.cell_codes = nullptr;
     pr.debug_word = debug_word_address();
     return DSA3D_OK;
 }
@@ -87,6 +89,10 @@ void set_tiling(dsa3d::Problem& pr) {
     pr.tiles_x = (pr.W + tx - 1) / tx;
     pr.tt_begin = 0;
     pr.tt_count = pr.tiles_t;
+    // DSA3D_KEY_BLOCKS=1 replaces the tile kernel by the tensor-core key-block kernel where that covers the
+    // shape (and no tiling was asked for explicitly): correct and tested, but slower so far.
+    const char* kb = getenv("DSA3D_KEY_BLOCKS");
+    pr.key_blocks = (kb && kb[0] == '1' && !getenv("DSA3D_TILE") && dsa3d::key_blocks_shape_covered(pr)) ? 1 : 0;
 }
 
 struct BackwardWorkspace {
@@ -101,8 +107,13 @@ BackwardWorkspace backward_workspace(const dsa3d::Problem& pr, int dtype, bool t
     if (tiled && pr.tile_t >= 1) {
         // rounded up so that the 16-byte bin entries behind it stay 16-byte aligned
         w.coef_bytes = (static_cast<size_t>(pr.items) * pr.P * sizeof(float2) + 255) & ~static_cast<size_t>(255);
-        w.entries_per_cta = static_cast<long long>(pr.tile_t) * pr.tile_y * pr.tile_x * pr.P * 8;
-        w.scratch_bytes = static_cast<size_t>(kTileSlots) * w.entries_per_cta * sizeof(dsa3d::TileEntry);
+        if (pr.key_blocks) {
+            // one cell code per sample of the whole grid in place of the tile kernel's bin entries
+            w.scratch_bytes = (static_cast<size_t>(pr.N) * pr.heads * pr.P * sizeof(uint32_t) + 255) & ~static_cast<size_t>(255);
+        } else {
+            w.entries_per_cta = static_cast<long long>(pr.tile_t) * pr.tile_y * pr.tile_x * pr.P * 8;
+            w.scratch_bytes = static_cast<size_t>(kTileSlots) * w.entries_per_cta * sizeof(dsa3d::TileEntry);
+        }
     }
     w.total = w.acc_bytes + w.coef_bytes + w.scratch_bytes;
     return w;
@@ -310,6 +321,7 @@ int backward_plan(int T, int H, int W, int heads, int d, const int* window, int 
     plan.acc_dv = plan.bf16 ? reinterpret_cast<float*>(wsp) + plan.count : static_cast<float*>(dv);
     plan.coef = plan.ws.coef_bytes ? reinterpret_cast<float2*>(wsp + plan.ws.acc_bytes) : nullptr;
     plan.scratch = plan.ws.scratch_bytes ? wsp + plan.ws.acc_bytes + plan.ws.coef_bytes : nullptr;
+    if (plan.pr.key_blocks) plan.pr.cell_codes = static_cast<uint32_t*>(plan.scratch);
     if (plan.coef) {
         int dev = 0, sms = 0;
         cudaError_t e = cudaGetDevice(&dev);
@@ -371,8 +383,9 @@ int backward_frames(const BackwardPlan& plan, const void* q, const void* k, cons
     if (plan.coef) {
         e = record(4, stream);
         if (e != cudaSuccess) return cuda_failed(e);
-        e = dsa3d::launch_scatter_tiles(q, dout, offsets, plan.coef, plan.acc_dk, plan.acc_dv, plan.scratch,
-                                        plan.ctas, plan.ws.entries_per_cta, pr, stream);
+        e = pr.key_blocks ? dsa3d::launch_dkdv_blocks(q, dout, offsets, plan.coef, plan.acc_dk, plan.acc_dv, pr, stream)
+                          : dsa3d::launch_scatter_tiles(q, dout, offsets, plan.coef, plan.acc_dk, plan.acc_dv, plan.scratch,
+                                                        plan.ctas, plan.ws.entries_per_cta, pr, stream);
         if (e != cudaSuccess) return cuda_failed(e);
         e = record(5, stream);
         if (e != cudaSuccess) return cuda_failed(e);

@@ -34,11 +34,6 @@
 
 namespace dsa3d {
 
-__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
-                 : "memory");
-}
-
 constexpr int kStats = 8;   // per sample: alpha, g, A_t, A_y, A_x, B_t, B_y, B_x
 
 #ifndef DSA3D_BWD_MINBLOCKS
@@ -254,7 +249,8 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
             const int p = pb + gl;
             const Cell cell = make_cell(pr, t, y, x, p, off_row + p * 3);
             mine = to_sample(pr, cell);
-            mine.mask = cell.mask & ~halo_corner_mask(pr, cell, t, y, x);   // corners the tile kernel does not take
+            // corners the tile kernel (or the key-block kernel) does not take
+            mine.mask = cell.mask & ~(pr.key_blocks ? block_near_mask(cell, t, y, x) : halo_corner_mask(pr, cell, t, y, x));
             if (!active) mine.mask = 0u;
             const float* sts = stats + p * kStats;
             const float alpha = sts[0];
@@ -266,6 +262,7 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
                 doff_row[p * 3 + 1] = fmaf(my_ck, sts[3], alpha * sts[6]);
                 doff_row[p * 3 + 2] = fmaf(my_ck, sts[4], alpha * sts[7]);
                 if (coef) coef[row * pr.P + p] = make_float2(my_ck, my_cv);
+                if (pr.key_blocks) pr.cell_codes[row * pr.P + p] = cell_code(cell);
             }
         }
         const int cnt = min(LPR, pr.P - pb);

@@ -27,6 +27,11 @@ struct Problem {
     int tile_t, tile_y, tile_x, halo;
     int tiles_t, tiles_y, tiles_x;
     int tt_begin, tt_count;   // tile rows along t that the tile kernel visits (all: 0, tiles_t)
+    // Key-block scheme (see block_near_mask below) instead of query tiles: the gather kernel leaves every
+    // sample's cell code in cell_codes [N*heads][P] and scatters only the corners whose query lies outside
+    // the region of the corner's key block.
+    int key_blocks;
+    uint32_t* cell_codes;
     // Checked build (-DDSA3D_DEBUG) only: device word that receives the first out-of-range index a
     // kernel was about to use (0 = none); NULL otherwise.
     unsigned long long* debug_word;
@@ -295,6 +300,39 @@ __device__ __forceinline__ unsigned halo_corner_mask(const Problem& pr, const Ce
                        pr.tile_y + 2 * pr.halo, pr.tile_x + 2 * pr.halo);
 }
 
+// ---------------------------------------------------------------------------------------
+// Key blocks (the tensor-core dK/dV kernel, dsa3d_backward_blocks.cu).  The grid is cut into
+// blocks of 4 x 8 x 8 key positions; the kernel that owns a block sums the contributions of every
+// query in the block's REGION: 16 frames from t0 - 6, 20 rows from y0 - 6 (five strips of 4),
+// 24 columns from x0 - 8 (three strips of 8).  A contribution whose query lies outside the
+// region of its key's block is scattered by the gather kernel itself.
+// ---------------------------------------------------------------------------------------
+constexpr int kKbT = 4, kKbY = 8, kKbX = 8;
+constexpr int kKbLoT = 6, kKbLoY = 6, kKbLoX = 8;             // the region starts this far below the block
+constexpr int kKbRegT = 16, kKbRegY = 20, kKbRegX = 24;       // its extent
+
+// Bit c is set when the query (t, y, x) lies in the region of the key block holding corner c of the cell.
+__device__ __forceinline__ unsigned block_near_mask(const Cell& c, int t, int y, int x) {
+    unsigned nt[2], ny[2], nx[2];
+#pragma unroll
+    for (int a = 0; a < 2; ++a) {
+        nt[a] = static_cast<unsigned>(t - ((c.it + a) & ~(kKbT - 1)) + kKbLoT) < static_cast<unsigned>(kKbRegT);
+        ny[a] = static_cast<unsigned>(y - ((c.iy + a) & ~(kKbY - 1)) + kKbLoY) < static_cast<unsigned>(kKbRegY);
+        nx[a] = static_cast<unsigned>(x - ((c.ix + a) & ~(kKbX - 1)) + kKbLoX) < static_cast<unsigned>(kKbRegX);
+    }
+    const unsigned yx = (ny[0] & nx[0]) | ((ny[0] & nx[1]) << 1) | ((ny[1] & nx[0]) << 2) | ((ny[1] & nx[1]) << 3);
+    return (nt[0] ? yx : 0u) | (nt[1] ? (yx << 4) : 0u);
+}
+
+// A sample's cell as one word for the key-block kernel's scan: (it + 1) | (iy + 1) << 10 | (ix + 1) << 20
+// (extents up to 1022), all ones for a sample with no corner inside the grid.
+constexpr uint32_t kDeadCellCode = 0xffffffffu;
+__device__ __forceinline__ uint32_t cell_code(const Cell& c) {
+    if (c.mask == 0u) return kDeadCellCode;
+    return static_cast<uint32_t>(c.it + 1) | (static_cast<uint32_t>(c.iy + 1) << 10) |
+           (static_cast<uint32_t>(c.ix + 1) << 20);
+}
+
 // Shuffles inside a group of LPR consecutive lanes (LPR a power of two <= 32).
 template <int LPR> __device__ __forceinline__ unsigned group_mask(int lane) {
     if constexpr (LPR == 32) {
@@ -378,6 +416,12 @@ template <int LPR> __device__ __forceinline__ Sample group_bcast(const Sample& s
     r.fy = __shfl_sync(gmask, s.fy, src, LPR);
     r.fx = __shfl_sync(gmask, s.fx, src, LPR);
     return r;
+}
+
+// One 16-byte fp32 reduction into global memory (the dK/dV accumulators).
+__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
+                 : "memory");
 }
 
 constexpr float kLog2e = 1.4426950408889634f;

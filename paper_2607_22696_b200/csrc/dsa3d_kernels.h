@@ -36,6 +36,14 @@ cudaError_t launch_scatter_tiles(const void* q, const void* dout, const float* o
 // Dynamic shared memory of the tile kernel for this problem's tiling.
 size_t tile_smem_bytes(const Problem& pr);
 
+// dK/dV of bf16 problems by key blocks on the tensor cores (dsa3d_backward_blocks.cu) instead of
+// launch_scatter_tiles: adds, for the query tokens of `pr`, every contribution whose query lies in the region
+// of its key's block (block_near_mask) to the accumulators.  Needs the coefficients and the cell codes
+// (pr.cell_codes) the gather kernel wrote with pr.key_blocks set.
+bool key_blocks_shape_covered(const Problem& pr);
+cudaError_t launch_dkdv_blocks(const void* q, const void* dout, const float* offsets, const float2* coef, float* acc_dk,
+                               float* acc_dv, const Problem& pr, cudaStream_t stream);
+
 // fp32 accumulators -> bf16 outputs (round to nearest even).
 cudaError_t launch_convert_bf16(const float* acc, void* dst, long long count, cudaStream_t stream);
 

@@ -58,8 +58,13 @@ CASES = [
 ]
 
 
+@pytest.mark.parametrize("key_blocks", [False, True])
 @pytest.mark.parametrize("dims,window,dtype,sigma,kind", CASES)
-def test_parity_cases_leave_no_violation_in_the_checked_build(dims, window, dtype, sigma, kind):
+def test_parity_cases_leave_no_violation_in_the_checked_build(dims, window, dtype, sigma, kind, key_blocks, monkeypatch):
+    if key_blocks:
+        if dtype != torch.bfloat16 or dims[4] < 64:
+            pytest.skip("the key-block kernel takes bf16 rows of 64 or 128 channels")
+        monkeypatch.setenv("DSA3D_KEY_BLOCKS", "1")       # dK/dV on the tensor cores instead of the tile kernel
     lib = binding.load_checked_build()
     assert lib.dsa3d_debug_build() == 1 and binding.load().dsa3d_debug_build() == 0
     assert lib.dsa3d_debug_clear() == 0
