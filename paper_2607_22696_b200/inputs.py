@@ -161,6 +161,10 @@ WORKLOADS: Dict[str, Workload] = {w.name: w for w in [
     # not a BASELINE config: offsets as small perturbations of the window (every component below 1 in
     # size), the regime in which the forward runs as tile attention on the tensor cores
     Workload("sweep_w333_small", 64, 45, 80, 16, 128, (3, 3, 3), _BF16, 0.4, 4, offsets="small"),
+    # cuts of the fixed-window and small-offset cases for profiler captures (a few GB on the device)
+    Workload("profile_small_w333_zero_bf16", 32, 45, 80, 8, 128, (3, 3, 3), _BF16, 0.0, 5, offsets="zero"),
+    Workload("profile_small_w377_zero_bf16", 16, 45, 80, 8, 128, (3, 7, 7), _BF16, 0.0, 5, offsets="zero"),
+    Workload("profile_small_w333_small_bf16", 32, 45, 80, 8, 128, (3, 3, 3), _BF16, 0.4, 5, offsets="small"),
 ]}
 
 
