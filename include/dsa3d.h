@@ -51,7 +51,8 @@
  *                                  block of 4 x 8 x 8 keys as tensor-core products (coefficient matrix of the
  *                                  block against chunks of 32 queries, tcgen05 in tf32: the coefficients lose
  *                                  the bits below 2^-10 relative, q and dO none) instead of the tile kernel's
- *                                  binning; slower so far; also changes dsa3d_backward_workspace_bytes; a
+ *                                  binning (the gather kernel then lists every sample per key block); slower
+ *                                  so far; also changes dsa3d_backward_workspace_bytes; a
  *                                  non-finite q or dO row then reaches every key whose block it lies near
  *   DSA3D_NO_TENSOR_FIXED_WINDOW   dsa3d_forward_fixed_window uses the general kernel
  *   DSA3D_GEMM_ONE_CTA             dsa3d_offsets_linear_forward: one CTA per tile instead of a pair

@@ -60,7 +60,9 @@ int make_problem(int T, int H, int W, int heads, int d, const int* window, int d
     pr.tiles_t = pr.tiles_y = pr.tiles_x = 0;
     pr.tt_begin = pr.tt_count = 0;
     pr.key_blocks = 0;
-    pr.cell_codes = nullptr;
+    pr.blk_count = nullptr;
+    pr.blk_list = nullptr;
+    pr.blk_cap = 0;
     pr.debug_word = debug_word_address();
     return DSA3D_OK;
 }
@@ -108,8 +110,9 @@ BackwardWorkspace backward_workspace(const dsa3d::Problem& pr, int dtype, bool t
         // rounded up so that the 16-byte bin entries behind it stay 16-byte aligned
         w.coef_bytes = (static_cast<size_t>(pr.items) * pr.P * sizeof(float2) + 255) & ~static_cast<size_t>(255);
         if (pr.key_blocks) {
-            // one cell code per sample of the whole grid in place of the tile kernel's bin entries
-            w.scratch_bytes = (static_cast<size_t>(pr.N) * pr.heads * pr.P * sizeof(uint32_t) + 255) & ~static_cast<size_t>(255);
+            // per-block counters and sample lists, sorted records of the resident CTAs, in place of the bin entries
+            const dsa3d::KeyBlockLayout kb = dsa3d::key_block_layout(pr);
+            w.scratch_bytes = kb.count_bytes + kb.list_bytes + kb.sorted_bytes;
         } else {
             w.entries_per_cta = static_cast<long long>(pr.tile_t) * pr.tile_y * pr.tile_x * pr.P * 8;
             w.scratch_bytes = static_cast<size_t>(kTileSlots) * w.entries_per_cta * sizeof(dsa3d::TileEntry);
@@ -321,7 +324,12 @@ int backward_plan(int T, int H, int W, int heads, int d, const int* window, int 
     plan.acc_dv = plan.bf16 ? reinterpret_cast<float*>(wsp) + plan.count : static_cast<float*>(dv);
     plan.coef = plan.ws.coef_bytes ? reinterpret_cast<float2*>(wsp + plan.ws.acc_bytes) : nullptr;
     plan.scratch = plan.ws.scratch_bytes ? wsp + plan.ws.acc_bytes + plan.ws.coef_bytes : nullptr;
-    if (plan.pr.key_blocks) plan.pr.cell_codes = static_cast<uint32_t*>(plan.scratch);
+    if (plan.pr.key_blocks) {
+        const dsa3d::KeyBlockLayout kb = dsa3d::key_block_layout(plan.pr);
+        plan.pr.blk_count = static_cast<uint32_t*>(plan.scratch);
+        plan.pr.blk_list = reinterpret_cast<uint32_t*>(static_cast<char*>(plan.scratch) + kb.count_bytes);
+        plan.pr.blk_cap = kb.cap;
+    }
     if (plan.coef) {
         int dev = 0, sms = 0;
         cudaError_t e = cudaGetDevice(&dev);
@@ -371,6 +379,10 @@ int backward_frames(const BackwardPlan& plan, const void* q, const void* k, cons
     const dsa3d::Problem pr = frames_of(plan.pr, f0, f1);
     cudaError_t e = record(2, stream);
     if (e != cudaSuccess) return cuda_failed(e);
+    if (pr.key_blocks) {                 // the sample lists of the key blocks start empty for every launch
+        e = cudaMemsetAsync(pr.blk_count, 0, dsa3d::key_block_layout(pr).count_bytes, stream);
+        if (e != cudaSuccess) return cuda_failed(e);
+    }
     e = dsa3d::launch_backward(q, k, v, offsets, lse, dout, dq, plan.acc_dk, plan.acc_dv, doffsets, plan.coef, pr,
                                plan.bf16, stream);
     if (e != cudaSuccess) return cuda_failed(e);

@@ -250,7 +250,8 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
             const Cell cell = make_cell(pr, t, y, x, p, off_row + p * 3);
             mine = to_sample(pr, cell);
             // corners the tile kernel (or the key-block kernel) does not take
-            mine.mask = cell.mask & ~(pr.key_blocks ? block_near_mask(cell, t, y, x) : halo_corner_mask(pr, cell, t, y, x));
+            if (pr.key_blocks) mine.mask = active ? block_lists_append(pr, cell, t, y, x, m, p) : 0u;
+            else mine.mask = cell.mask & ~halo_corner_mask(pr, cell, t, y, x);
             if (!active) mine.mask = 0u;
             const float* sts = stats + p * kStats;
             const float alpha = sts[0];
@@ -262,7 +263,6 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
                 doff_row[p * 3 + 1] = fmaf(my_ck, sts[3], alpha * sts[6]);
                 doff_row[p * 3 + 2] = fmaf(my_ck, sts[4], alpha * sts[7]);
                 if (coef) coef[row * pr.P + p] = make_float2(my_ck, my_cv);
-                if (pr.key_blocks) pr.cell_codes[row * pr.P + p] = cell_code(cell);
             }
         }
         const int cnt = min(LPR, pr.P - pb);

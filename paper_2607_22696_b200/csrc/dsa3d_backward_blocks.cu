@@ -6,20 +6,22 @@
 // of 256 keys (4 x 8 x 8 positions of one head) and the queries around it, that is
 //     dK_block = A_k . Q,   dV_block = A_v . dO,
 // with A[key, query] = sum of the coefficients that query sends to that key: a sparse matrix (a few per
-// cent of its entries), but one whose non-zeros are found without sorting anything, and whose product is
-// a dense contraction the tensor cores take.  The block's result is complete when its queries have been
-// walked, so it leaves the chip once - no per-contribution reductions into global memory.
+// cent of its entries) whose product is a dense contraction the tensor cores take.  The block's result is
+// complete when its queries have been walked, so it leaves the chip once.
 //
-// One persistent CTA per SM walks its blocks; for a block it walks the chunks of the block's query region
-// (32 queries: 4 rows x 8 columns of one frame; 16 x 5 x 3 chunk slots, those outside the grid or the
-// launch's frames skipped).  Roles:
-//   two groups of four warps take the chunks alternately, each with its own pair of A matrices.  For a chunk
-//     a group scans the cell codes the gather kernel left for the chunk's (query, sample) pairs and lists the
-//     samples with a corner inside the block (about 6 % of them); requests their offsets and coefficient
-//     pairs; once the MMAs of its previous chunk are done, puts that chunk's entries of A back to zero from
-//     its list (nothing dense is swept per chunk); then adds each listed sample's up to eight coefficients
-//     into A (fp32 words in shared memory, 128-byte-swizzled K-major rows of 32 queries, shared-memory
-//     atomics) and hands the chunk over;
+// The gather kernel has appended every sample to the list of each key block it touches
+// (block_lists_append).  One persistent CTA per SM walks its blocks; for a block it walks the chunks of
+// the block's query region (32 queries: 4 rows x 8 columns of one frame; 16 x 5 x 3 chunk slots, those
+// outside the grid or the launch's frames skipped).  Roles:
+//   four sorter warps, one block ahead: a counting sort of the block's list by chunk slot, during which they
+//     fetch each sample's offsets and coefficient pair, form its cell once more (make_cell_values: the same
+//     arithmetic as the gather kernel) and write, for every corner of the sample that lies in the block, a
+//     16-byte entry {position in A, w_c ck, w_c cv} to the CTA's scratch in global memory, chunk after chunk;
+//   two groups of four warps take the chunks alternately, each with its own pair of A matrices (fp32 words,
+//     128-byte-swizzled K-major rows of 32 queries): once the MMAs of the group's previous chunk are done its
+//     entries of A go back to zero from a list of positions in shared memory (nothing dense is swept per
+//     chunk), then the chunk's entries - already on their way into registers - are added with shared-memory
+//     atomics and the chunk is handed over;
 //   four warps stage the chunks' q and dO rows, widened to fp32 and transposed, as the K-major B operands
 //     (one row per channel, 32 queries along it), one chunk ahead in registers;
 //   one thread issues, per chunk, 16 tcgen05.mma.kind::tf32 (M = 128 keys, N = channels, K = 8 queries) that
@@ -38,26 +40,32 @@ namespace dsa3d {
 namespace {
 
 constexpr int kBkRows = kKbT * kKbY * kKbX;                            // 256 keys: two MMA row halves
-constexpr int kBkChunkY = 4, kBkChunkX = 8, kBkChunkQ = kBkChunkY * kBkChunkX;
-constexpr int kBkChunksX = kKbRegX / kBkChunkX;                        // 3
-constexpr int kBkChunksPerFrame = (kKbRegY / kBkChunkY) * kBkChunksX;  // 15
+constexpr int kBkChunkY = kKbChunkY, kBkChunkX = kKbChunkX, kBkChunkQ = kBkChunkY * kBkChunkX;
+constexpr int kBkChunksX = kKbChunksX;                                 // 3
+constexpr int kBkChunksPerFrame = kKbChunksPerFrame;                   // 15
 constexpr int kBkSlots = kKbRegT * kBkChunksPerFrame;                  // 240 chunk slots per block
 constexpr int kBkGroup = 128;                                          // threads of a scatter group
 constexpr int kBkStagers = 128;                                        // threads staging the B operands
-constexpr int kBkThreads = 2 * kBkGroup + kBkStagers + 32;             // + the warp that issues the MMAs
-constexpr int kBkListCap = 1024;                                       // listed samples per chunk and pass (32 queries x 32 samples)
-constexpr int kBkHeld = 2;                                             // listed samples a thread holds in registers
-static_assert(kBkRows == 256 && kBkChunkQ == 32, "the index arithmetic below assumes these");
+constexpr int kBkSorters = 128;                                        // threads sorting the next block's list
+constexpr int kBkThreads = 2 * kBkGroup + kBkStagers + kBkSorters + 32;   // + the warp that issues the MMAs
+constexpr int kBkListCap = 2048;                                       // positions of a chunk remembered for the sparse clear
+constexpr int kBkHeld = 4;                                             // entries a thread holds in registers
+constexpr int kBkMaxCtas = 160;                                        // resident CTAs the sorted scratch is sized for
+static_assert(kBkRows == 256 && kBkChunkQ == 32 && kBkSlots <= 256, "the index arithmetic below assumes these");
+
+using BkEntry = uint4;                     // {position in A (bk_a_index), fp32 w*ck, fp32 w*cv, unused}
 
 template <int D>
 struct __align__(1024) BkSmem {
     float a32[2][2][kBkRows * kBkChunkQ];      // [group][dK, dV]: rows of 32 queries (128 bytes), 128-byte swizzle
     float b32[2][2][kBkChunkQ * D];            // [group][q, dO]: rows = channels, 32 queries (128 bytes) each, same swizzle
-    uint32_t list[2][2][kBkListCap];           // [group][chunk parity]: ql | p << 5 | (rt+1) << 13 | (ry+1) << 16 | (rx+1) << 20
-    uint32_t count[2][4];                      // [group][chunk % 3]
+    uint16_t list[2][2][kBkListCap];           // [group][chunk parity]: positions the chunk touched, for the clear
+    uint32_t chunk_start[2][kBkSlots + 1];     // [block parity]: first entry of every chunk slot
+    uint32_t cursor[kBkSlots];                 // the sorters' histogram, then their write positions
+    uint32_t count[2][2];                      // [group][chunk parity]: entries of the chunk
     uint32_t blk_data[2];                      // [block parity]: an MMA has written the block's tiles
     int last_seq[2];                           // [group]: block of the group's last chunk
-    uint64_t bar_a_full[2], bar_b_full[2], bar_done[2];
+    uint64_t bar_a_full[2], bar_b_full[2], bar_done[2], bar_sorted[2], bar_free[2];
     uint32_t tmem_base;
     uint32_t abort;
 };
@@ -71,13 +79,15 @@ struct BkWalk {
 
 struct BkChunk {
     int seq, slot;                  // which of the CTA's blocks, which chunk slot of it
+    int frame, yc, xc;              // the slot as (frame of the region, strip of rows, strip of columns)
     int m, t0, y0, x0;              // head and origin of the key block
     int qt, qy0, qx0;               // frame and origin of the chunk's queries
     bool valid;
 };
 
 __device__ __forceinline__ void bk_start(BkChunk& ch) {
-    ch.seq = -1; ch.slot = kBkSlots; ch.m = ch.t0 = ch.y0 = ch.x0 = ch.qt = ch.qy0 = ch.qx0 = 0; ch.valid = true;
+    ch.seq = -1; ch.slot = kBkSlots; ch.frame = ch.yc = ch.xc = 0;
+    ch.m = ch.t0 = ch.y0 = ch.x0 = ch.qt = ch.qy0 = ch.qx0 = 0; ch.valid = true;
 }
 
 // Head and origin of the CTA's block number `seq`.
@@ -94,18 +104,23 @@ __device__ __forceinline__ void bk_locate(int seq, const BkWalk& wk, int& m, int
 __device__ __forceinline__ void bk_advance(BkChunk& ch, const BkWalk& wk, const Problem& pr) {
     if (!ch.valid) return;
     for (;;) {
-        if (++ch.slot >= kBkSlots) {
+        if (ch.slot >= kBkSlots - 1) {
             if (++ch.seq >= wk.my_blocks) { ch.valid = false; return; }
             bk_locate(ch.seq, wk, ch.m, ch.t0, ch.y0, ch.x0);
-            ch.slot = 0;
+            ch.slot = 0; ch.frame = ch.yc = ch.xc = 0;
+        } else {
+            ++ch.slot;
+            if (++ch.xc == kBkChunksX) { ch.xc = 0; if (++ch.yc == kKbRegY / kBkChunkY) { ch.yc = 0; ++ch.frame; } }
         }
-        const int frame = ch.slot / kBkChunksPerFrame;
-        ch.qt = ch.t0 - kKbLoT + frame;
-        if (ch.qt < wk.f0) { ch.slot = (wk.f0 - (ch.t0 - kKbLoT)) * kBkChunksPerFrame - 1; continue; }
-        if (ch.qt >= wk.f1) { ch.slot = kBkSlots; continue; }
-        const int r = ch.slot - frame * kBkChunksPerFrame;
-        ch.qy0 = ch.y0 - kKbLoY + kBkChunkY * (r / kBkChunksX);
-        ch.qx0 = ch.x0 - kKbLoX + kBkChunkX * (r % kBkChunksX);
+        ch.qt = ch.t0 - kKbLoT + ch.frame;
+        if (ch.qt < wk.f0) {                                          // on to the first frame of the launch
+            ch.frame = wk.f0 - (ch.t0 - kKbLoT);
+            if (ch.frame >= kKbRegT) { ch.slot = kBkSlots - 1; continue; }
+            ch.yc = ch.xc = 0; ch.slot = ch.frame * kBkChunksPerFrame; ch.qt = wk.f0;
+        }
+        if (ch.qt >= wk.f1) { ch.slot = kBkSlots - 1; continue; }
+        ch.qy0 = ch.y0 - kKbLoY + kBkChunkY * ch.yc;
+        ch.qx0 = ch.x0 - kKbLoX + kBkChunkX * ch.xc;
         if (ch.qy0 + kBkChunkY <= 0 || ch.qy0 >= pr.H || ch.qx0 + kBkChunkX <= 0 || ch.qx0 >= pr.W) continue;
         return;
     }
@@ -121,27 +136,31 @@ __device__ __forceinline__ int bk_a_index(int row, int ql) {
     return row * kBkChunkQ + ((((ql >> 2) ^ (row & 7)) << 2) | (ql & 3));
 }
 
-template <int D, bool MULTI>      // MULTI: more than 32 samples per query, taken in passes of 32
+template <int D>
 __global__ void __launch_bounds__(kBkThreads, 1)
 dkdv_block_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ dout,
                   const float* __restrict__ offsets, const float2* __restrict__ coef, float* __restrict__ acc_dk,
-                  float* __restrict__ acc_dv, const int total_blocks, const int blocks_per_head, const int by_count,
-                  const int bx_count, const int tb_begin, const int f0, const int f1, int* timeout_flag,
-                  const Problem pr) {
+                  float* __restrict__ acc_dv, BkEntry* __restrict__ sorted, const int total_blocks,
+                  const int blocks_per_head, const int by_count, const int bx_count, const int tb_begin, const int f0,
+                  const int f1, int* timeout_flag, const Problem pr) {
     extern __shared__ unsigned char raw[];
     BkSmem<D>& s = *reinterpret_cast<BkSmem<D>*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    constexpr int kMmaWarp = (2 * kBkGroup + kBkStagers) / 32;
-    const uint32_t* __restrict__ codes_g = pr.cell_codes;
-    [[maybe_unused]] const long long code_extent = pr.N * pr.heads * pr.P;
+    constexpr int kStagerWarp0 = 2 * kBkGroup / 32, kSorterWarp0 = kStagerWarp0 + kBkStagers / 32,
+                  kMmaWarp = kSorterWarp0 + kBkSorters / 32;
+    [[maybe_unused]] const long long sample_extent = pr.N * pr.heads * pr.P;
     [[maybe_unused]] const long long kv_extent = pr.N * pr.heads * D;
+    // this CTA's two buffers of sorted entries
+    BkEntry* const my_sorted = sorted + static_cast<long long>(blockIdx.x) * 2 * pr.blk_cap * 8;
 
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&s.bar_a_full[i]), kBkGroup / 32);      // lane 0 of every warp of the group
             mbar_init(smem_u32(&s.bar_b_full[i]), kBkStagers / 32);
             mbar_init(smem_u32(&s.bar_done[i]), 1);
-            for (int k = 0; k < 4; ++k) s.count[i][k] = 0u;
+            mbar_init(smem_u32(&s.bar_sorted[i]), kBkSorters / 32);
+            mbar_init(smem_u32(&s.bar_free[i]), 1);
+            s.count[i][0] = s.count[i][1] = 0u;
             s.blk_data[i] = 0u;
             s.last_seq[i] = -1;
         }
@@ -177,6 +196,7 @@ dkdv_block_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __re
                        ? (total_blocks - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x) : 0;
     wk.blocks_per_head = blocks_per_head; wk.by_count = by_count; wk.bx_count = bx_count; wk.tb_begin = tb_begin;
     wk.f0 = f0; wk.f1 = f1;
+    const int bt_n = (pr.T + kKbT - 1) / kKbT;
 
     if (warp == kMmaWarp) {
         // ==================================================================== MMA thread
@@ -202,7 +222,7 @@ dkdv_block_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __re
                 if (ok) ok = wait(&s.bar_b_full[g], static_cast<uint32_t>(i & 1), 35);
                 if (ok) {
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    if (*(volatile uint32_t*)&s.count[g][i % 3] > 0u) {
+                    if (*(volatile uint32_t*)&s.count[g][i & 1] > 0u) {
                         if (fresh) { *(volatile uint32_t*)&s.blk_data[cur & 1] = 1u; __threadfence_block(); }
 #pragma unroll
                         for (int x = 0; x < 2; ++x)
@@ -220,11 +240,104 @@ dkdv_block_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __re
                 bk_advance(ch, wk, pr);
             }
         }
-    } else if (warp >= 2 * kBkGroup / 32) {
+    } else if (warp >= kSorterWarp0) {
+        // ==================================================================== sorters: one block ahead of the groups
+        const int st = tid - kSorterWarp0 * 32;
+        for (int seq = 0; seq < wk.my_blocks; ++seq) {
+            const int buf = seq & 1;
+            // the groups have left block seq - 2, whose records and chunk starts this block replaces
+            if (seq >= 2) wait(&s.bar_free[buf], static_cast<uint32_t>(((seq >> 1) - 1) & 1), 37);
+            int m, t0, y0, x0;
+            bk_locate(seq, wk, m, t0, y0, x0);
+            const long long bid = ((static_cast<long long>(m) * bt_n + t0 / kKbT) * by_count + y0 / kKbY) * bx_count + x0 / kKbX;
+            const int n = static_cast<int>(min(__ldcg(pr.blk_count + bid), static_cast<uint32_t>(pr.blk_cap)));
+            const uint32_t* lst = pr.blk_list + bid * pr.blk_cap;
+            for (int i = st; i < kBkSlots; i += kBkSorters) s.cursor[i] = 0u;
+            bk_named_barrier(4, kBkSorters);
+            // corners of a listed sample that lie in the block and in the grid (what it will add entries for)
+            auto block_corners = [&](uint32_t entry) -> unsigned {
+                const int rt = static_cast<int>((entry >> 21) & 7u) - 1, ry = static_cast<int>((entry >> 24) & 15u) - 1,
+                          rx = static_cast<int>(entry >> 28) - 1;
+                return corner_mask(rt, ry, rx, kKbT, kKbY, kKbX) & corner_mask(t0 + rt, y0 + ry, x0 + rx, pr.T, pr.H, pr.W);
+            };
+            for (int e = st; e < n; e += kBkSorters) {
+                const uint32_t entry = __ldcg(lst + e);
+                atomicAdd(&s.cursor[entry & 255u], static_cast<uint32_t>(__popc(block_corners(entry))));
+            }
+            bk_named_barrier(4, kBkSorters);
+            if (st < 32) {                                             // exclusive prefix of the 240 counts
+                constexpr int PER = (kBkSlots + 31) / 32;
+                uint32_t c[PER], sum = 0u;
+#pragma unroll
+                for (int k = 0; k < PER; ++k) { c[k] = st * PER + k < kBkSlots ? s.cursor[st * PER + k] : 0u; sum += c[k]; }
+                uint32_t incl = sum;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) { const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o); if (st >= o) incl += v; }
+                uint32_t run = incl - sum;
+#pragma unroll
+                for (int k = 0; k < PER; ++k)
+                    if (st * PER + k < kBkSlots) { s.chunk_start[buf][st * PER + k] = run; s.cursor[st * PER + k] = run; run += c[k]; }
+                if (st == 31) s.chunk_start[buf][kBkSlots] = incl;
+            }
+            bk_named_barrier(4, kBkSorters);
+            BkEntry* out = my_sorted + static_cast<long long>(buf) * pr.blk_cap * 8;
+            for (int e0 = st; e0 < n; e0 += 2 * kBkSorters) {
+                uint32_t entry[2];
+                float o[2][3];
+                float2 cf[2];
+                int qt[2], qy[2], qx[2];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int e = e0 + h * kBkSorters;
+                    entry[h] = 0u; o[h][0] = o[h][1] = o[h][2] = 0.0f; cf[h] = make_float2(0.f, 0.f); qt[h] = qy[h] = qx[h] = 0;
+                    if (e < n) {
+                        entry[h] = __ldcg(lst + e);
+                        const int slot = entry[h] & 255u, ql = (entry[h] >> 8) & 31u, p = (entry[h] >> 13) & 255u;
+                        const int frame = slot / kBkChunksPerFrame, r = slot - frame * kBkChunksPerFrame;
+                        qt[h] = t0 - kKbLoT + frame;
+                        qy[h] = y0 - kKbLoY + kBkChunkY * (r / kBkChunksX) + (ql >> 3);
+                        qx[h] = x0 - kKbLoX + kBkChunkX * (r % kBkChunksX) + (ql & 7);
+                        const long long sample = (((static_cast<long long>(qt[h]) * pr.H + qy[h]) * pr.W + qx[h]) * pr.heads + m) * pr.P + p;
+                        if (DSA3D_IN_RANGE(pr, sample, sample_extent, 11)) {
+                            o[h][0] = __ldg(offsets + sample * 3); o[h][1] = __ldg(offsets + sample * 3 + 1); o[h][2] = __ldg(offsets + sample * 3 + 2);
+                            cf[h] = __ldg(coef + sample);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int e = e0 + h * kBkSorters;
+                    if (e < n) {
+                        const Cell cell = make_cell_values(pr, qt[h], qy[h], qx[h], (entry[h] >> 13) & 255u, o[h][0], o[h][1], o[h][2]);
+                        const unsigned corners = block_corners(entry[h]);
+                        const int ql = (entry[h] >> 8) & 31u;
+                        const int rt = static_cast<int>((entry[h] >> 21) & 7u) - 1, ry = static_cast<int>((entry[h] >> 24) & 15u) - 1,
+                                  rx = static_cast<int>(entry[h] >> 28) - 1;
+                        uint32_t at = atomicAdd(&s.cursor[entry[h] & 255u], static_cast<uint32_t>(__popc(corners)));
+                        const float wt[2] = {1.0f - cell.ft, cell.ft}, wy[2] = {1.0f - cell.fy, cell.fy}, wx[2] = {1.0f - cell.fx, cell.fx};
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            if (!((corners >> c) & 1u)) continue;
+                            // a corner the cell does not have (its code and the list entry disagree) adds nothing
+                            const float w = ((cell.mask >> c) & 1u) ? wt[c >> 2] * wy[(c >> 1) & 1] * wx[c & 1] : 0.0f;
+                            const int idx = bk_a_index(((rt + (c >> 2)) * kKbY + ry + ((c >> 1) & 1)) * kKbX + rx + (c & 1), ql);
+                            if (DSA3D_IN_RANGE(pr, at, static_cast<long long>(pr.blk_cap) * 8, 14))
+                                out[at] = make_uint4(static_cast<uint32_t>(idx), __float_as_uint(w * cf[h].x), __float_as_uint(w * cf[h].y), 0u);
+                            ++at;
+                        }
+                    }
+                }
+            }
+            __threadfence_block();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s.bar_sorted[buf]));
+            bk_named_barrier(4, kBkSorters);                            // the cursors are free for the next block
+        }
+    } else if (warp >= kStagerWarp0) {
         // ==================================================================== B operands: lane = query, warp = channel range
         constexpr int CPS = D / (kBkStagers / 32);                    // channels per warp
         constexpr int UPS = CPS / 8;                                  // 16-byte pieces of them
-        const int sw = warp - 2 * kBkGroup / 32;
+        const int sw = warp - kStagerWarp0;
         uint4 rows_q[UPS], rows_d[UPS];
         auto load_rows = [&](const BkChunk& ch) {
             const int qy = ch.qy0 + (lane >> 3), qx = ch.qx0 + (lane & 7);
@@ -272,78 +385,6 @@ dkdv_block_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __re
         const int bar_id = 1 + g;
         float* a_k = &s.a32[g][0][0];
         float* a_v = &s.a32[g][1][0];
-        volatile uint32_t* counts = s.count[g];
-        // a listed sample: its offsets and coefficient pair, then its coefficients into the A matrices
-        auto load_details = [&](uint32_t entry, const BkChunk& ch, float (&o)[3], float2& cf) {
-            const int ql = entry & 31, p = (entry >> 5) & 255;
-            const long long n = (static_cast<long long>(ch.qt) * pr.H + (ch.qy0 + (ql >> 3))) * pr.W + (ch.qx0 + (ql & 7));
-            const long long sample = (n * pr.heads + ch.m) * pr.P + p;
-            o[0] = o[1] = o[2] = 0.0f; cf = make_float2(0.f, 0.f);
-            if (DSA3D_IN_RANGE(pr, sample, code_extent, 11)) {
-                o[0] = __ldg(offsets + sample * 3); o[1] = __ldg(offsets + sample * 3 + 1); o[2] = __ldg(offsets + sample * 3 + 2);
-                cf = __ldg(coef + sample);
-            }
-        };
-        auto scatter = [&](uint32_t entry, const BkChunk& ch, const float (&o)[3], const float2 cf) {
-            const int ql = entry & 31, p = (entry >> 5) & 255;
-            const Cell cell = make_cell_values(pr, ch.qt, ch.qy0 + (ql >> 3), ch.qx0 + (ql & 7), p, o[0], o[1], o[2]);
-            const int rt = cell.it - ch.t0, ry = cell.iy - ch.y0, rx = cell.ix - ch.x0;
-            const float wt[2] = {1.0f - cell.ft, cell.ft}, wy[2] = {1.0f - cell.fy, cell.fy}, wx[2] = {1.0f - cell.fx, cell.fx};
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const int kt_ = rt + (c >> 2), ky_ = ry + ((c >> 1) & 1), kx_ = rx + (c & 1);
-                const float w = wt[c >> 2] * wy[(c >> 1) & 1] * wx[c & 1];
-                if (((cell.mask >> c) & 1u) && w != 0.0f && static_cast<unsigned>(kt_) < static_cast<unsigned>(kKbT) &&
-                    static_cast<unsigned>(ky_) < static_cast<unsigned>(kKbY) && static_cast<unsigned>(kx_) < static_cast<unsigned>(kKbX)) {
-                    const int idx = bk_a_index((kt_ * kKbY + ky_) * kKbX + kx_, ql);
-                    atomicAdd(a_k + idx, w * cf.x);
-                    atomicAdd(a_v + idx, w * cf.y);
-                }
-            }
-        };
-        // the entries of A that the samples of a list may have touched, back to zero
-        auto clear_listed = [&](const uint32_t* lst, int n) {
-            for (int pair = gt; pair < n * 8; pair += kBkGroup) {
-                const uint32_t entry = lst[pair >> 3];
-                const int cc = pair & 7;
-                const int kt_ = static_cast<int>((entry >> 13) & 7u) - 1 + (cc >> 2);
-                const int ky_ = static_cast<int>((entry >> 16) & 15u) - 1 + ((cc >> 1) & 1);
-                const int kx_ = static_cast<int>((entry >> 20) & 15u) - 1 + (cc & 1);
-                if (static_cast<unsigned>(kt_) < static_cast<unsigned>(kKbT) && static_cast<unsigned>(ky_) < static_cast<unsigned>(kKbY) &&
-                    static_cast<unsigned>(kx_) < static_cast<unsigned>(kKbX)) {
-                    const int idx = bk_a_index((kt_ * kKbY + ky_) * kKbX + kx_, static_cast<int>(entry & 31u));
-                    a_k[idx] = 0.0f;
-                    a_v[idx] = 0.0f;
-                }
-            }
-        };
-        // samples of the group's 32 queries x 32 lanes whose cell touches the block -> list
-        auto scan = [&](const uint32_t (&codes)[8], int pi, const BkChunk& ch, uint32_t* lst, uint32_t* counter) {
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const uint32_t code = codes[k];
-                const uint32_t dt = (code & 1023u) - static_cast<uint32_t>(ch.t0);          // corner 0 relative to the block, + 1
-                const uint32_t dy = ((code >> 10) & 1023u) - static_cast<uint32_t>(ch.y0);
-                const uint32_t dx = (code >> 20) - static_cast<uint32_t>(ch.x0);
-                if (code != kDeadCellCode && dt <= static_cast<uint32_t>(kKbT) && dy <= static_cast<uint32_t>(kKbY) &&
-                    dx <= static_cast<uint32_t>(kKbX)) {
-                    const uint32_t at = atomicAdd(counter, 1u);
-                    if (at < static_cast<uint32_t>(kBkListCap))
-                        lst[at] = static_cast<uint32_t>(gw * 8 + k) | (static_cast<uint32_t>(pi * 32 + lane) << 5) | (dt << 13) | (dy << 16) | (dx << 20);
-                }
-            }
-        };
-        auto load_codes = [&](uint32_t (&codes)[8], int pi, const BkChunk& ch) {
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const int ql = gw * 8 + k;
-                const int qy = ch.qy0 + (ql >> 3), qx = ch.qx0 + (ql & 7), p = pi * 32 + lane;
-                const long long at = ((((static_cast<long long>(ch.qt) * pr.H + qy) * pr.W + qx) * pr.heads + ch.m)) * pr.P + p;
-                codes[k] = kDeadCellCode;
-                if (ch.valid && qy >= 0 && qy < pr.H && qx >= 0 && qx < pr.W && p < pr.P && DSA3D_IN_RANGE(pr, at, code_extent, 14))
-                    codes[k] = __ldg(codes_g + at);
-            }
-        };
         // the finished block: its four tiles from TMEM to the accumulators (warp of the group = TMEM lane quarter)
         auto epilogue = [&](int seq) {
             int m, t0, y0, x0;
@@ -371,111 +412,93 @@ dkdv_block_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __re
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         };
+        // where a chunk's entries lie, once its block has been sorted
+        int sorted_seq = -1;
+        auto locate_records = [&](const BkChunk& ch, int& n, const BkEntry*& recs) {
+            n = 0; recs = my_sorted;
+            if (!ch.valid) return;
+            if (ch.seq != sorted_seq) {
+                wait(&s.bar_sorted[ch.seq & 1], static_cast<uint32_t>((ch.seq >> 1) & 1), 38);
+                sorted_seq = ch.seq;
+            }
+            const uint32_t b = *(volatile uint32_t*)&s.chunk_start[ch.seq & 1][ch.slot], e = *(volatile uint32_t*)&s.chunk_start[ch.seq & 1][ch.slot + 1];
+            n = *abort_flag ? 0 : static_cast<int>(e - b);
+            recs = my_sorted + static_cast<long long>(ch.seq & 1) * pr.blk_cap * 8 + b;
+        };
 
         BkChunk ch;
         bk_start(ch);
         bk_advance(ch, wk, pr);
-        int j = 0, prev_seq = -1, last_seq = -1;
+        int j = 0, prev_seq = -1, last_seq = -1, n_prev = 0;
         if (g == 1) {
             if (ch.valid) prev_seq = ch.seq;
             bk_advance(ch, wk, pr);
             j = 1;
         }
-        uint32_t codes[8];
-        if constexpr (!MULTI) load_codes(codes, 0, ch);
-        for (int i = 0; ch.valid; ++i, j += 2) {
-            BkChunk nx = ch;
-            bk_advance(nx, wk, pr);
-            const int mid_seq = nx.valid ? nx.seq : -1;                  // block of the chunk between this one and the group's next
-            bk_advance(nx, wk, pr);
-            uint32_t* lst = s.list[g][i & 1];
-            uint32_t* counter = &s.count[g][i % 3];
-            bool drained = false;
-            if constexpr (!MULTI) {
-                // ---- which samples touch the block; their details requested; the codes of the group's next chunk requested
-                scan(codes, 0, ch, lst, counter);
-                bk_named_barrier(bar_id, kBkGroup);
-                const int n = static_cast<int>(min(counts[i % 3], static_cast<uint32_t>(kBkListCap)));
-                uint32_t ent[kBkHeld];
-                float o[kBkHeld][3];
-                float2 cf[kBkHeld];
+        int n = 0;
+        const BkEntry* recs = my_sorted;
+        BkEntry held[kBkHeld];
+        locate_records(ch, n, recs);
 #pragma unroll
-                for (int h = 0; h < kBkHeld; ++h) {
-                    ent[h] = 0u;
-                    if (gt + h * kBkGroup < n) { ent[h] = lst[gt + h * kBkGroup]; load_details(ent[h], ch, o[h], cf[h]); }
+        for (int h = 0; h < kBkHeld; ++h)
+            if (gt + h * kBkGroup < n) held[h] = __ldcg(recs + gt + h * kBkGroup);
+        for (int i = 0; ch.valid; ++i, j += 2) {
+            bool drained = false;
+            // ---- the group's previous chunk has been multiplied: its entries of A back to zero (and a finished block out)
+            if (i >= 1) wait(&s.bar_done[g], static_cast<uint32_t>((i - 1) & 1), 33);
+            if (j > 0 && ch.seq != prev_seq) {
+                wait(&s.bar_done[g ^ 1], static_cast<uint32_t>(((j - 1) >> 1) & 1), 32);
+                if (*(volatile uint32_t*)&s.blk_data[prev_seq & 1]) epilogue(prev_seq);
+                drained = true;
+            }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (n_prev > kBkListCap) {
+                float4* a = reinterpret_cast<float4*>(a_k);                  // the dK and dV matrices are adjacent
+                for (int e = gt; e < 2 * kBkRows * kBkChunkQ / 4; e += kBkGroup) a[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+            } else {
+                const uint16_t* prev = s.list[g][(i - 1) & 1];
+                for (int e = gt; e < n_prev; e += kBkGroup) { const int idx = prev[e]; a_k[idx] = 0.0f; a_v[idx] = 0.0f; }
+            }
+            bk_named_barrier(bar_id, kBkGroup);
+            if (drained && gt == 0) {
+                *(volatile uint32_t*)&s.blk_data[prev_seq & 1] = 0u;
+                mbar_arrive(smem_u32(&s.bar_free[prev_seq & 1]));          // the sorters may reuse that block's buffers
+            }
+            // ---- this chunk's coefficients into A
+            uint16_t* lst = s.list[g][i & 1];
+#pragma unroll
+            for (int h = 0; h < kBkHeld; ++h)
+                if (gt + h * kBkGroup < n) {
+                    atomicAdd(a_k + held[h].x, __uint_as_float(held[h].y));
+                    atomicAdd(a_v + held[h].x, __uint_as_float(held[h].z));
+                    lst[gt + h * kBkGroup] = static_cast<uint16_t>(held[h].x);
                 }
-                load_codes(codes, 0, nx);
-                if (gt == 0) s.count[g][(i + 1) % 3] = 0u;               // the count of chunk i - 2 is no longer read
-                // ---- the previous chunk has been multiplied: its entries of A back to zero (and a finished block out)
-                if (i >= 1) wait(&s.bar_done[g], static_cast<uint32_t>((i - 1) & 1), 33);
-                if (j > 0 && ch.seq != prev_seq) {
-                    wait(&s.bar_done[g ^ 1], static_cast<uint32_t>(((j - 1) >> 1) & 1), 32);
-                    if (*(volatile uint32_t*)&s.blk_data[prev_seq & 1]) { epilogue(prev_seq); drained = true; }
-                }
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                if (i >= 1) clear_listed(s.list[g][(i - 1) & 1], static_cast<int>(min(counts[(i - 1) % 3], static_cast<uint32_t>(kBkListCap))));
-                bk_named_barrier(bar_id, kBkGroup);
-                if (drained && gt == 0) *(volatile uint32_t*)&s.blk_data[prev_seq & 1] = 0u;
-                // ---- this chunk's coefficients into A
+            for (int base = kBkHeld * kBkGroup; base < n; base += kBkHeld * kBkGroup) {
 #pragma unroll
                 for (int h = 0; h < kBkHeld; ++h)
-                    if (gt + h * kBkGroup < n) scatter(ent[h], ch, o[h], cf[h]);
-                for (int base = kBkHeld * kBkGroup; base < n; base += kBkHeld * kBkGroup) {
+                    if (base + gt + h * kBkGroup < n) held[h] = __ldcg(recs + base + gt + h * kBkGroup);
 #pragma unroll
-                    for (int h = 0; h < kBkHeld; ++h) {
-                        ent[h] = 0u;
-                        if (base + gt + h * kBkGroup < n) { ent[h] = lst[base + gt + h * kBkGroup]; load_details(ent[h], ch, o[h], cf[h]); }
+                for (int h = 0; h < kBkHeld; ++h)
+                    if (base + gt + h * kBkGroup < n) {
+                        atomicAdd(a_k + held[h].x, __uint_as_float(held[h].y));
+                        atomicAdd(a_v + held[h].x, __uint_as_float(held[h].z));
+                        if (base + gt + h * kBkGroup < kBkListCap) lst[base + gt + h * kBkGroup] = static_cast<uint16_t>(held[h].x);
                     }
-#pragma unroll
-                    for (int h = 0; h < kBkHeld; ++h)
-                        if (base + gt + h * kBkGroup < n) scatter(ent[h], ch, o[h], cf[h]);
-                }
-            } else {
-                // ---- more than 32 samples per query: the previous chunk's A cleared whole, then one pass per 32 samples
-                if (gt == 0) { s.count[g][(i + 1) % 3] = 0u; }
-                if (i >= 1) wait(&s.bar_done[g], static_cast<uint32_t>((i - 1) & 1), 33);
-                if (j > 0 && ch.seq != prev_seq) {
-                    wait(&s.bar_done[g ^ 1], static_cast<uint32_t>(((j - 1) >> 1) & 1), 32);
-                    if (*(volatile uint32_t*)&s.blk_data[prev_seq & 1]) { epilogue(prev_seq); drained = true; }
-                }
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                if (i >= 1) {
-                    float4* a = reinterpret_cast<float4*>(a_k);              // dK and dV matrices are adjacent
-                    for (int e = gt; e < 2 * kBkRows * kBkChunkQ / 4; e += kBkGroup) a[e] = make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-                uint32_t* pass_counter = &s.count[g][3];
-                const int passes = (pr.P + 31) / 32;
-                for (int pi = 0; pi < passes; ++pi) {
-                    if (gt == 0) *pass_counter = 0u;
-                    load_codes(codes, pi, ch);
-                    bk_named_barrier(bar_id, kBkGroup);
-                    if (drained && gt == 0 && pi == 0) *(volatile uint32_t*)&s.blk_data[prev_seq & 1] = 0u;
-                    scan(codes, pi, ch, lst, pass_counter);
-                    bk_named_barrier(bar_id, kBkGroup);
-                    const int n = static_cast<int>(min(counts[3], static_cast<uint32_t>(kBkListCap)));
-                    if (gt == 0) *counter += static_cast<uint32_t>(n);
-                    for (int base = 0; base < n; base += kBkHeld * kBkGroup) {
-                        uint32_t ent[kBkHeld];
-                        float o[kBkHeld][3];
-                        float2 cf[kBkHeld];
-#pragma unroll
-                        for (int h = 0; h < kBkHeld; ++h) {
-                            ent[h] = 0u;
-                            if (base + gt + h * kBkGroup < n) { ent[h] = lst[base + gt + h * kBkGroup]; load_details(ent[h], ch, o[h], cf[h]); }
-                        }
-#pragma unroll
-                        for (int h = 0; h < kBkHeld; ++h)
-                            if (base + gt + h * kBkGroup < n) scatter(ent[h], ch, o[h], cf[h]);
-                    }
-                    bk_named_barrier(bar_id, kBkGroup);
-                }
             }
+            if (gt == 0) *(volatile uint32_t*)&s.count[g][i & 1] = static_cast<uint32_t>(n);
             fence_async_smem();                                       // the MMAs read A through the async proxy
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&s.bar_a_full[g]));
+            // ---- the group's next chunk: its entries on their way
             last_seq = ch.seq;
-            prev_seq = mid_seq;
-            ch = nx;
+            n_prev = n;
+            bk_advance(ch, wk, pr);
+            prev_seq = ch.valid ? ch.seq : -1;                        // block of the chunk between this one and the group's next
+            bk_advance(ch, wk, pr);
+            locate_records(ch, n, recs);
+#pragma unroll
+            for (int h = 0; h < kBkHeld; ++h)
+                if (gt + h * kBkGroup < n) held[h] = __ldcg(recs + gt + h * kBkGroup);
         }
         // ---- the last block: every MMA done, then group 0 takes it out
         {
@@ -497,11 +520,11 @@ dkdv_block_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __re
     if (warp == kMmaWarp) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(4 * D));
 }
 
-template <int D, bool MULTI>
+template <int D>
 cudaError_t launch_blocks_t(const void* q, const void* dout, const float* offsets, const float2* coef, float* acc_dk,
-                            float* acc_dv, int total, int per_head, int by_count, int bx_count, int tb_begin, int f0, int f1,
-                            int* flag, const Problem& pr, cudaStream_t stream) {
-    auto kern = dkdv_block_kernel<D, MULTI>;
+                            float* acc_dv, BkEntry* sorted, int total, int per_head, int by_count, int bx_count, int tb_begin,
+                            int f0, int f1, int* flag, const Problem& pr, cudaStream_t stream) {
+    auto kern = dkdv_block_kernel<D>;
     const size_t smem = sizeof(BkSmem<D>) + 1024;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
@@ -510,18 +533,31 @@ cudaError_t launch_blocks_t(const void* q, const void* dout, const float* offset
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
+    if (sms > kBkMaxCtas) sms = kBkMaxCtas;
     const unsigned grid = static_cast<unsigned>(total < sms ? total : sms);     // persistent: one CTA per SM
     kern<<<grid, kBkThreads, smem, stream>>>(static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(dout),
-                                             offsets, coef, acc_dk, acc_dv, total, per_head, by_count, bx_count, tb_begin,
-                                             f0, f1, flag, pr);
+                                             offsets, coef, acc_dk, acc_dv, sorted, total, per_head, by_count, bx_count,
+                                             tb_begin, f0, f1, flag, pr);
     return cudaGetLastError();
 }
 
 }  // namespace
 
+KeyBlockLayout key_block_layout(const Problem& pr) {
+    KeyBlockLayout kb{};
+    kb.blocks = static_cast<long long>((pr.T + kKbT - 1) / kKbT) * ((pr.H + kKbY - 1) / kKbY) * ((pr.W + kKbX - 1) / kKbX) * pr.heads;
+    // a block of 256 keys is touched by 256 * P samples, each counted for about 1.6 blocks; the rest of the
+    // room is for the blocks that get more than their share (a sample that finds a list full is scattered directly)
+    kb.cap = (kBkRows * pr.P * 9 / 5 + 255) / 256 * 256;
+    kb.count_bytes = (static_cast<size_t>(kb.blocks) * sizeof(uint32_t) + 255) & ~static_cast<size_t>(255);
+    kb.list_bytes = static_cast<size_t>(kb.blocks) * kb.cap * sizeof(uint32_t);
+    kb.sorted_bytes = static_cast<size_t>(kBkMaxCtas) * 2 * kb.cap * 8 * sizeof(BkEntry);       // up to eight entries per listed sample
+    return kb;
+}
+
 bool key_blocks_shape_covered(const Problem& pr) {
     if (pr.d != 128 && pr.d != 64) return false;
-    if (pr.T > 1022 || pr.H > 1022 || pr.W > 1022 || pr.P > 256) return false;       // 10-bit fields of the cell codes
+    if (pr.P > 256) return false;                                                     // 8-bit sample field of a list entry
     const long long blocks = static_cast<long long>((pr.T + kKbT - 1) / kKbT) * ((pr.H + kKbY - 1) / kKbY) *
                              ((pr.W + kKbX - 1) / kKbX) * pr.heads;
     return blocks < (1LL << 30);
@@ -529,7 +565,7 @@ bool key_blocks_shape_covered(const Problem& pr) {
 
 cudaError_t launch_dkdv_blocks(const void* q, const void* dout, const float* offsets, const float2* coef, float* acc_dk,
                                float* acc_dv, const Problem& pr, cudaStream_t stream) {
-    if (!key_blocks_shape_covered(pr) || !pr.cell_codes) return cudaErrorInvalidValue;
+    if (!key_blocks_shape_covered(pr) || !pr.blk_count || !pr.blk_list) return cudaErrorInvalidValue;
     int* flag = timeout_flag_device_address();
     if (!flag) return cudaErrorInvalidValue;
     const long long per_frame = static_cast<long long>(pr.H) * pr.W;
@@ -544,10 +580,11 @@ cudaError_t launch_dkdv_blocks(const void* q, const void* dout, const float* off
     const int by_count = (pr.H + kKbY - 1) / kKbY, bx_count = (pr.W + kKbX - 1) / kKbX;
     const int per_head = (tb_end - tb_begin + 1) * by_count * bx_count;
     const int total = per_head * pr.heads;
-#define DSA3D_BK(DD, MM) launch_blocks_t<DD, MM>(q, dout, offsets, coef, acc_dk, acc_dv, total, per_head, by_count, bx_count, \
-                                                 tb_begin, f0, f1, flag, pr, stream)
-    if (pr.d == 128) return pr.P <= 32 ? DSA3D_BK(128, false) : DSA3D_BK(128, true);
-    return pr.P <= 32 ? DSA3D_BK(64, false) : DSA3D_BK(64, true);
+    const KeyBlockLayout kb = key_block_layout(pr);
+    BkEntry* sorted = reinterpret_cast<BkEntry*>(reinterpret_cast<char*>(pr.blk_list) + kb.list_bytes);
+#define DSA3D_BK(DD) launch_blocks_t<DD>(q, dout, offsets, coef, acc_dk, acc_dv, sorted, total, per_head, by_count, bx_count, \
+                                         tb_begin, f0, f1, flag, pr, stream)
+    return pr.d == 128 ? DSA3D_BK(128) : DSA3D_BK(64);
 #undef DSA3D_BK
 }
 

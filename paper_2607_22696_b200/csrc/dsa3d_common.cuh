@@ -27,11 +27,15 @@ struct Problem {
     int tile_t, tile_y, tile_x, halo;
     int tiles_t, tiles_y, tiles_x;
     int tt_begin, tt_count;   // tile rows along t that the tile kernel visits (all: 0, tiles_t)
-    // Key-block scheme (see block_near_mask below) instead of query tiles: the gather kernel leaves every
-    // sample's cell code in cell_codes [N*heads][P] and scatters only the corners whose query lies outside
-    // the region of the corner's key block.
+    // Key-block scheme (see block_near_mask below) instead of query tiles: the gather kernel appends every
+    // sample to the list of each key block one of its corners lies in (blk_list [blocks][blk_cap] of packed
+    // entries, blk_count [blocks], blocks numbered ((head * tb + bt) * by + by_) * bx + bx_ over the whole
+    // grid) and scatters only the corners whose query lies outside the region of the corner's key block - or
+    // whose block's list was full.
     int key_blocks;
-    uint32_t* cell_codes;
+    uint32_t* blk_count;
+    uint32_t* blk_list;
+    int blk_cap;
     // Checked build (-DDSA3D_DEBUG) only: device word that receives the first out-of-range index a
     // kernel was about to use (0 = none); NULL otherwise.
     unsigned long long* debug_word;
@@ -324,13 +328,45 @@ __device__ __forceinline__ unsigned block_near_mask(const Cell& c, int t, int y,
     return (nt[0] ? yx : 0u) | (nt[1] ? (yx << 4) : 0u);
 }
 
-// A sample's cell as one word for the key-block kernel's scan: (it + 1) | (iy + 1) << 10 | (ix + 1) << 20
-// (extents up to 1022), all ones for a sample with no corner inside the grid.
-constexpr uint32_t kDeadCellCode = 0xffffffffu;
-__device__ __forceinline__ uint32_t cell_code(const Cell& c) {
-    if (c.mask == 0u) return kDeadCellCode;
-    return static_cast<uint32_t>(c.it + 1) | (static_cast<uint32_t>(c.iy + 1) << 10) |
-           (static_cast<uint32_t>(c.ix + 1) << 20);
+// Entry of a key block's sample list: chunk slot of the query in the block's region (8 bits), query inside the
+// chunk (5), sample (8), corner (0,0,0) of the cell relative to the block + 1 (3 + 4 + 4 bits).
+__device__ __forceinline__ uint32_t block_entry(int slot, int ql, int p, int rt1, int ry1, int rx1) {
+    return static_cast<uint32_t>(slot) | (static_cast<uint32_t>(ql) << 8) | (static_cast<uint32_t>(p) << 13) |
+           (static_cast<uint32_t>(rt1) << 21) | (static_cast<uint32_t>(ry1) << 24) | (static_cast<uint32_t>(rx1) << 28);
+}
+constexpr int kKbChunkY = 4, kKbChunkX = 8;                    // a chunk of the region: 4 rows x 8 columns of one frame
+constexpr int kKbChunksX = kKbRegX / kKbChunkX, kKbChunksPerFrame = (kKbRegY / kKbChunkY) * kKbChunksX;   // 3, 15
+
+// The gather kernel's side of the key-block scheme for one sample: append it to the list of every block that
+// holds one of its corners and whose region holds the query; return the corners left for the direct scatter.
+__device__ __forceinline__ unsigned block_lists_append(const Problem& pr, const Cell& c, int t, int y, int x, int m, int p) {
+    const unsigned near = block_near_mask(c, t, y, x) & c.mask;
+    unsigned far = c.mask & ~near;
+    if (near == 0u) return far;
+    const int bt_n = (pr.T + kKbT - 1) / kKbT, by_n = (pr.H + kKbY - 1) / kKbY, bx_n = (pr.W + kKbX - 1) / kKbX;
+    // along an axis the two corners lie in different blocks only when the second one starts a block
+    const unsigned cross = (((c.it + 1) & (kKbT - 1)) == 0 ? 1u : 0u) | (((c.iy + 1) & (kKbY - 1)) == 0 ? 2u : 0u) |
+                           (((c.ix + 1) & (kKbX - 1)) == 0 ? 4u : 0u);
+    for (unsigned sel = 0; sel < 8u; ++sel) {
+        if (sel & ~cross) continue;
+        // corners of this block: second corner along the crossing axes chosen by `sel`, both along the others
+        unsigned sub = 0xffu;
+        if (cross & 1u) sub &= (sel & 1u) ? 0xf0u : 0x0fu;
+        if (cross & 2u) sub &= (sel & 2u) ? 0xccu : 0x33u;
+        if (cross & 4u) sub &= (sel & 4u) ? 0xaau : 0x55u;
+        sub &= near;
+        if (sub == 0u) continue;
+        const int t0 = (c.it + static_cast<int>(sel & 1u)) & ~(kKbT - 1), y0 = (c.iy + static_cast<int>((sel >> 1) & 1u)) & ~(kKbY - 1),
+                  x0 = (c.ix + static_cast<int>((sel >> 2) & 1u)) & ~(kKbX - 1);
+        const long long bid = ((static_cast<long long>(m) * bt_n + t0 / kKbT) * by_n + y0 / kKbY) * bx_n + x0 / kKbX;
+        const int dy = y - (y0 - kKbLoY), dx = x - (x0 - kKbLoX);
+        const int slot = ((t - (t0 - kKbLoT)) * (kKbRegY / kKbChunkY) + dy / kKbChunkY) * kKbChunksX + dx / kKbChunkX;
+        const uint32_t entry = block_entry(slot, (dy % kKbChunkY) * kKbChunkX + dx % kKbChunkX, p, c.it - t0 + 1, c.iy - y0 + 1, c.ix - x0 + 1);
+        const uint32_t at = atomicAdd(pr.blk_count + bid, 1u);
+        if (at < static_cast<uint32_t>(pr.blk_cap)) pr.blk_list[bid * pr.blk_cap + at] = entry;
+        else far |= sub;                                      // list full: these corners go the direct way
+    }
+    return far;
 }
 
 // Shuffles inside a group of LPR consecutive lanes (LPR a power of two <= 32).

@@ -37,9 +37,12 @@ cudaError_t launch_scatter_tiles(const void* q, const void* dout, const float* o
 size_t tile_smem_bytes(const Problem& pr);
 
 // dK/dV of bf16 problems by key blocks on the tensor cores (dsa3d_backward_blocks.cu) instead of
-// launch_scatter_tiles: adds, for the query tokens of `pr`, every contribution whose query lies in the region
-// of its key's block (block_near_mask) to the accumulators.  Needs the coefficients and the cell codes
-// (pr.cell_codes) the gather kernel wrote with pr.key_blocks set.
+// launch_scatter_tiles: adds, for the query tokens of `pr`, every contribution the gather kernel listed for a
+// key block (block_lists_append, with pr.key_blocks set and the counters cleared before its launch) to the
+// accumulators.  key_block_layout: sizes of the counters, the per-block lists (pr.blk_count, pr.blk_list follow
+// each other in one buffer) and the sorted records of the resident CTAs behind them.
+struct KeyBlockLayout { size_t count_bytes, list_bytes, sorted_bytes; int cap; long long blocks; };
+KeyBlockLayout key_block_layout(const Problem& pr);
 bool key_blocks_shape_covered(const Problem& pr);
 cudaError_t launch_dkdv_blocks(const void* q, const void* dout, const float* offsets, const float2* coef, float* acc_dk,
                                float* acc_dv, const Problem& pr, cudaStream_t stream);
