@@ -47,7 +47,7 @@
  *   DSA3D_TILE="tt,ty,tx,halo"     query tiling of the dK/dV pre-reduction of dsa3d_backward
  *                                  (default 4,8,8,6; "0" = no tiling, every contribution is an
  *                                  atomic add); also changes dsa3d_backward_workspace_bytes
- *   DSA3D_KEY_BLOCKS=1             dsa3d_backward (bf16, d = 64 or 128, extents up to 1022) forms dK/dV per
+ *   DSA3D_KEY_BLOCKS=1             dsa3d_backward (bf16, d = 64 or 128) forms dK/dV per
  *                                  block of 4 x 8 x 8 keys as tensor-core products (coefficient matrix of the
  *                                  block against chunks of 32 queries, tcgen05 in tf32: the coefficients lose
  *                                  the bits below 2^-10 relative, q and dO none) instead of the tile kernel's

@@ -29,8 +29,8 @@ namespace {
 constexpr int kTbTT = 4, kTbTY = 4, kTbTX = 8, kTbQ = kTbTT * kTbTY * kTbTX;    // 128 queries per tile
 constexpr int kTbSplit = 2;                                                   // worker warps per TMEM quadrant
 constexpr int kTbWorkers = 128 * kTbSplit, kTbThreads = kTbWorkers + 96;      // + loading warp + two MMA warps
-constexpr int kTbSlots = 4;
-constexpr int kTbScoreBufs = 4;                                               // score planes in flight in TMEM
+constexpr int kTbSlots = 4;                                                   // plane buffers, at most
+constexpr int kTbScoreBufs = 4;                                               // score planes in flight in TMEM, at most
 
 template <int D, int KT, int KH, int KW>
 struct TableShape {
@@ -45,7 +45,12 @@ struct TableShape {
     static constexpr int SLOT_HALF = PSP * 128;
     static constexpr int STAGE_BYTES = PIECES * 32 * kTbQ * 4;
     static constexpr int A_BYTES = NH * kTbQ * 128;                 // Q or dO rows of the tile
-    static_assert(PSP <= 256 && kTbScoreBufs * SBUF <= 512, "plane too large");
+    static constexpr int SLOT_BYTES = NH * ((SLOT_HALF + 1023) / 1024 * 1024);
+    // as many score planes in TMEM and plane buffers in shared memory as fit, up to four each
+    static constexpr int NB = 512 / SBUF < kTbScoreBufs ? 512 / SBUF : kTbScoreBufs;
+    static constexpr int NS_FIT = (227 * 1024 - 4096 - 2 * A_BYTES - STAGE_BYTES) / SLOT_BYTES;
+    static constexpr int NS = NS_FIT > kTbSlots ? kTbSlots : NS_FIT;
+    static_assert(PSP <= 256 && NB >= 2 && NS >= 2, "plane too large");
     static_assert(SLOT_HALF % 1024 == 0 || PSP % 8 == 0, "");
 };
 
@@ -53,7 +58,7 @@ template <int D, int KT, int KH, int KW>
 struct __align__(1024) TbSmem {
     using S = TableShape<D, KT, KH, KW>;
     unsigned char a[2][S::A_BYTES];                                 // Q, dO: 64-channel halves, swizzled 128-byte rows
-    unsigned char slot[kTbSlots][S::NH][(S::SLOT_HALF + 1023) / 1024 * 1024];
+    unsigned char slot[S::NS][S::NH][(S::SLOT_HALF + 1023) / 1024 * 1024];
     unsigned char stage[S::STAGE_BYTES];                            // a score plane as [column][query] floats
     uint64_t bar_a[2], bar_full[kTbSlots], bar_slot_free[kTbSlots], bar_s[kTbScoreBufs], bar_s_free[kTbScoreBufs];
     uint32_t tmem_base;
@@ -70,10 +75,10 @@ fixed_window_tables_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                            float* __restrict__ table, int T, int H, int W, int heads, int tiles_x, int tiles_y, int total,
                            int* timeout_flag) {
     using S = TableShape<D, KT, KH, KW>;
-    constexpr int NH = S::NH, RT = S::RT, RX = S::RX, PS = S::PS, PSP = S::PSP, VH = S::VH, NS = kTbSlots;
+    constexpr int NH = S::NH, RT = S::RT, RX = S::RX, PS = S::PS, PSP = S::PSP, VH = S::VH, NS = S::NS;
     constexpr int BT = S::BT, BY = S::BY, BX = S::BX;
     constexpr int JOBS = 2 * RT;                                      // per tile: RT planes of K (against Q), RT of V (against dO)
-    constexpr int NB = kTbScoreBufs;
+    constexpr int NB = S::NB;
     constexpr int TMEM_COLS = NB * S::SBUF <= 128 ? 128 : (NB * S::SBUF <= 256 ? 256 : 512);
     extern __shared__ unsigned char raw[];
     TbSmem<D, KT, KH, KW>& s =
@@ -327,6 +332,7 @@ int fixed_window_table_floats(const Problem& pr, bool bf16) {
     if (!bf16 || (pr.d != 128 && pr.d != 64)) return 0;
     if (pr.kt == 3 && pr.kh == 3 && pr.kw == 3) return 2 * TableShape<128, 3, 3, 3>::CELLS8;
     if (pr.kt == 2 && pr.kh == 2 && pr.kw == 2) return 2 * TableShape<128, 2, 2, 2>::CELLS8;
+    if (pr.kt == 3 && pr.kh == 5 && pr.kw == 5) return 2 * TableShape<128, 3, 5, 5>::CELLS8;
     return 0;
 }
 
@@ -337,12 +343,14 @@ bool try_fixed_window_tables(const void* q, const void* k, const void* v, const 
     int* flag = timeout_flag_device_address();
     if (!flag) return false;
     bool unsupported = false;
-    const bool w333 = pr.kt == 3;
+    const bool w333 = pr.kt == 3 && pr.kh == 3, w355 = pr.kt == 3 && pr.kh == 5;
     if (pr.d == 128)
         *err = w333 ? launch_tables<128, 3, 3, 3>(q, k, v, dout, table, pr, flag, stream, &unsupported)
+             : w355 ? launch_tables<128, 3, 5, 5>(q, k, v, dout, table, pr, flag, stream, &unsupported)
                     : launch_tables<128, 2, 2, 2>(q, k, v, dout, table, pr, flag, stream, &unsupported);
     else
         *err = w333 ? launch_tables<64, 3, 3, 3>(q, k, v, dout, table, pr, flag, stream, &unsupported)
+             : w355 ? launch_tables<64, 3, 5, 5>(q, k, v, dout, table, pr, flag, stream, &unsupported)
                     : launch_tables<64, 2, 2, 2>(q, k, v, dout, table, pr, flag, stream, &unsupported);
     return !unsupported;
 }
