@@ -48,6 +48,8 @@ int make_problem(int T, int H, int W, int heads, int d, const int* window, int d
     if (N * heads / 8 >= (1LL << 31) - 1) return DSA3D_ERR_BAD_SHAPE;
     pr.T = T; pr.H = H; pr.W = W; pr.heads = heads; pr.d = d;
     pr.kt = window[0]; pr.kh = window[1]; pr.kw = window[2];
+    pr.inv_kw = ((1u << 20) + static_cast<unsigned>(pr.kw) - 1u) / static_cast<unsigned>(pr.kw);
+    pr.inv_kh = ((1u << 20) + static_cast<unsigned>(pr.kh) - 1u) / static_cast<unsigned>(pr.kh);
     // one frame of rows must be addressable with 32-bit element offsets
     if (static_cast<long long>(H) * W * heads * d >= (1LL << 31)) return DSA3D_ERR_BAD_SHAPE;
     pr.P = static_cast<int>(P);

@@ -16,6 +16,9 @@ using TileEntry = uint4;            // {offset, fp32 wk, fp32 wv, unused}
 struct Problem {
     int T, H, W, heads, d;
     int kt, kh, kw, P;
+    // ceil(2^20 / kw) and ceil(2^20 / kh): p / kw = (p * inv_kw) >> 20 exactly for p < 2^8 (P <= 256), so that
+    // a sample's window cell needs no integer division
+    unsigned inv_kw, inv_kh;
     long long N;       // T*H*W
     long long items;   // work items of this launch: one per (query token, head) = q_count*heads
     // Query tokens [q_begin, q_begin + q_count) are processed (the whole grid unless a caller
@@ -247,9 +250,10 @@ __device__ __forceinline__ unsigned corner_mask(int rt, int ry, int rx, int et, 
 // The same from the three offset components already loaded.
 __device__ __forceinline__ Cell make_cell_values(const Problem& pr, int t, int y, int x, int p, float ot, float oy,
                                                  float ox) {
-    const int w = p % pr.kw;
-    const int v = (p / pr.kw) % pr.kh;
-    const int u = p / (pr.kw * pr.kh);
+    const int pk = static_cast<int>((static_cast<unsigned>(p) * pr.inv_kw) >> 20);      // p / kw
+    const int w = p - pk * pr.kw;
+    const int u = static_cast<int>((static_cast<unsigned>(pk) * pr.inv_kh) >> 20);     // p / (kw * kh)
+    const int v = pk - u * pr.kh;
     Cell c;
     c.it = c.iy = c.ix = 0;
     c.mask = 0u;
@@ -267,9 +271,10 @@ __device__ __forceinline__ Cell make_cell_values(const Problem& pr, int t, int y
 
 __device__ __forceinline__ Cell make_cell(const Problem& pr, int t, int y, int x, int p,
                                           const float* __restrict__ off3) {
-    const int w = p % pr.kw;
-    const int v = (p / pr.kw) % pr.kh;
-    const int u = p / (pr.kw * pr.kh);
+    const int pk = static_cast<int>((static_cast<unsigned>(p) * pr.inv_kw) >> 20);      // p / kw
+    const int w = p - pk * pr.kw;
+    const int u = static_cast<int>((static_cast<unsigned>(pk) * pr.inv_kh) >> 20);     // p / (kw * kh)
+    const int v = pk - u * pr.kh;
     Cell c;
     c.it = c.iy = c.ix = 0;
     c.mask = 0u;
