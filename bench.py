@@ -400,6 +400,8 @@ def run_ours(args, wl):
     wl_rank = rank_workload(wl, rank)
     t = inputs.make_inputs(wl_rank, dev, with_dout=True)
     ws_bytes = binding.dsa3d_backward_workspace_bytes(*dims, wl.window, wl.dtype)
+    if wl.offsets == "zero" and wl.backward:        # the fixed-window backward keeps its dot-product tables there
+        ws_bytes = max(ws_bytes, binding.dsa3d_backward_fixed_window_workspace_bytes(*dims, wl.window, wl.dtype))
     b = {"out": torch.empty_like(t["q"]),
          "lse": torch.empty(wl.T, wl.H, wl.W, wl.heads, dtype=torch.float32, device=dev),
          "dq": torch.empty_like(t["q"]), "dk": torch.empty_like(t["q"]), "dv": torch.empty_like(t["q"]),

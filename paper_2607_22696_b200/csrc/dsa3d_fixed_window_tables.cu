@@ -43,7 +43,9 @@ struct TableShape {
     static constexpr int VH = (BY + kTbSplit - 1) / kTbSplit;        // consecutive box rows along y per thread of a query's group
     static constexpr int SBUF = PIECES * 32;
     static constexpr int SLOT_HALF = PSP * 128;
-    static constexpr int STAGE_BYTES = PIECES * 32 * kTbQ * 4;
+    // a large score plane is staged and picked from in two halves of its columns
+    static constexpr int SUBS = PIECES > 4 ? 2 : 1, PPS = (PIECES + SUBS - 1) / SUBS;
+    static constexpr int STAGE_BYTES = PPS * 32 * kTbQ * 4;
     static constexpr int A_BYTES = NH * kTbQ * 128;                 // Q or dO rows of the tile
     static constexpr int SLOT_BYTES = NH * ((SLOT_HALF + 1023) / 1024 * 1024);
     // as many score planes in TMEM and plane buffers in shared memory as fit, up to four each
@@ -228,26 +230,36 @@ fixed_window_tables_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                     const int u_rt = pl - lt;                         // the box plane this region plane is to the warp's queries
                     if (u_rt >= 0 && u_rt < BT) {
                         const uint32_t sbuf = tmem + lane_base + (sp % NB) * S::SBUF;
-                        for (int piece = half; piece < S::PIECES; piece += kTbSplit) {
-                            uint32_t regs[32];
-                            tmem_load_32(sbuf + piece * 32, regs);
+                        // this thread's rows of the box plane are neighbours (vv = half * VH ...), so its cells
+                        // are one contiguous run of the table: written as 16-byte pieces when BX = 4 (a warp's
+                        // stores then fill whole 32-byte sectors instead of touching each one eight times)
+                        float* dst = my_table + which * S::CELLS8 + u_rt * (BY * BX) + half * VH * BX;
+                        float cells[VH * BX];
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) stage[(piece * 32 + i) * kTbQ + r] = __uint_as_float(regs[i]);
+                        for (int i = 0; i < VH * BX; ++i) cells[i] = 0.0f;
+#pragma unroll
+                        for (int sub = 0; sub < S::SUBS; ++sub) {
+                            constexpr int PPS = S::PPS;
+                            for (int piece = sub * PPS + half; piece < (sub + 1) * PPS && piece < S::PIECES; piece += kTbSplit) {
+                                uint32_t regs[32];
+                                tmem_load_32(sbuf + piece * 32, regs);
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) stage[((piece - sub * PPS) * 32 + i) * kTbQ + r] = __uint_as_float(regs[i]);
+                            }
+                            pair_barrier(1 + lt);                     // the plane (or this half of its columns) is staged
+                            if (in_grid && !*abort_flag) {
+#pragma unroll
+                                for (int vi = 0; vi < VH; ++vi)
+#pragma unroll
+                                    for (int ww = 0; ww < BX; ++ww) {
+                                        const int vv = vi + half * VH;
+                                        const int col = (ly + vv) * RX + lx + ww - sub * PPS * 32;
+                                        if (vv < BY && (S::SUBS == 1 || (col >= 0 && col < PPS * 32))) cells[vi * BX + ww] = stage[col * kTbQ + r];
+                                    }
+                            }
+                            pair_barrier(1 + lt);                     // both have copied: the staging rows may be refilled
                         }
-                        pair_barrier(1 + lt);                         // the plane is staged
                         if (in_grid && !*abort_flag) {
-                            // this thread's rows of the box plane are neighbours (vv = half * VH ...), so its cells
-                            // are one contiguous run of the table: written as 16-byte pieces when BX = 4 (a warp's
-                            // stores then fill whole 32-byte sectors instead of touching each one eight times)
-                            float* dst = my_table + which * S::CELLS8 + u_rt * (BY * BX) + half * VH * BX;
-                            float cells[VH * BX];
-#pragma unroll
-                            for (int vi = 0; vi < VH; ++vi)
-#pragma unroll
-                                for (int ww = 0; ww < BX; ++ww) {
-                                    const int vv = vi + half * VH;
-                                    cells[vi * BX + ww] = vv < BY ? stage[((ly + vv) * RX + lx + ww) * kTbQ + r] : 0.0f;
-                                }
                             if constexpr (BX == 4 && (BY * BX) % 4 == 0 && S::CELLS8 % 4 == 0) {
 #pragma unroll
                                 for (int vi = 0; vi < VH; ++vi)
@@ -259,7 +271,6 @@ fixed_window_tables_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                                     if (i / BX + half * VH < BY) dst[i] = cells[i];
                             }
                         }
-                        pair_barrier(1 + lt);                         // both have copied: the staging rows may be refilled
                     }
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                     __syncwarp();
@@ -333,6 +344,7 @@ int fixed_window_table_floats(const Problem& pr, bool bf16) {
     if (pr.kt == 3 && pr.kh == 3 && pr.kw == 3) return 2 * TableShape<128, 3, 3, 3>::CELLS8;
     if (pr.kt == 2 && pr.kh == 2 && pr.kw == 2) return 2 * TableShape<128, 2, 2, 2>::CELLS8;
     if (pr.kt == 3 && pr.kh == 5 && pr.kw == 5) return 2 * TableShape<128, 3, 5, 5>::CELLS8;
+    if (pr.kt == 3 && pr.kh == 7 && pr.kw == 7) return 2 * TableShape<128, 3, 7, 7>::CELLS8;
     return 0;
 }
 
@@ -343,14 +355,16 @@ bool try_fixed_window_tables(const void* q, const void* k, const void* v, const 
     int* flag = timeout_flag_device_address();
     if (!flag) return false;
     bool unsupported = false;
-    const bool w333 = pr.kt == 3 && pr.kh == 3, w355 = pr.kt == 3 && pr.kh == 5;
+    const bool w333 = pr.kt == 3 && pr.kh == 3, w355 = pr.kt == 3 && pr.kh == 5, w377 = pr.kt == 3 && pr.kh == 7;
     if (pr.d == 128)
         *err = w333 ? launch_tables<128, 3, 3, 3>(q, k, v, dout, table, pr, flag, stream, &unsupported)
              : w355 ? launch_tables<128, 3, 5, 5>(q, k, v, dout, table, pr, flag, stream, &unsupported)
+             : w377 ? launch_tables<128, 3, 7, 7>(q, k, v, dout, table, pr, flag, stream, &unsupported)
                     : launch_tables<128, 2, 2, 2>(q, k, v, dout, table, pr, flag, stream, &unsupported);
     else
         *err = w333 ? launch_tables<64, 3, 3, 3>(q, k, v, dout, table, pr, flag, stream, &unsupported)
              : w355 ? launch_tables<64, 3, 5, 5>(q, k, v, dout, table, pr, flag, stream, &unsupported)
+             : w377 ? launch_tables<64, 3, 7, 7>(q, k, v, dout, table, pr, flag, stream, &unsupported)
                     : launch_tables<64, 2, 2, 2>(q, k, v, dout, table, pr, flag, stream, &unsupported);
     return !unsupported;
 }

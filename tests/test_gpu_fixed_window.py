@@ -145,6 +145,8 @@ def _backward_case(shape, window, dtype, seed, with_doffsets=True):
     ((6, 9, 13, 2, 128), (3, 3, 3), BF16), ((4, 5, 6, 2, 64), (3, 3, 3), BF16), ((3, 5, 6, 2, 32), (3, 3, 3), F32),
     ((5, 6, 7, 2, 128), (2, 2, 2), BF16), ((4, 6, 9, 1, 64), (3, 5, 5), BF16), ((1, 1, 1, 1, 32), (3, 3, 3), F32),
     ((9, 10, 19, 2, 128), (3, 5, 5), BF16), ((4, 4, 8, 1, 128), (3, 5, 5), BF16), ((6, 13, 9, 3, 64), (3, 5, 5), BF16),
+    ((9, 10, 19, 2, 128), (3, 7, 7), BF16), ((4, 4, 8, 1, 128), (3, 7, 7), BF16), ((6, 13, 9, 3, 64), (3, 7, 7), BF16),
+    ((1, 2, 3, 1, 64), (3, 7, 7), BF16),
     ((2, 3, 4, 2, 32), (1, 1, 1), BF16), ((3, 8, 9, 2, 64), (1, 7, 7), F32), ((4, 4, 5, 3, 128), (5, 3, 1), F32)])
 def test_fixed_window_backward_matches_the_oracle(shape, window, dtype):
     """Against the oracle on an all-zero offsets tensor: odd and even windows, windows that reach
