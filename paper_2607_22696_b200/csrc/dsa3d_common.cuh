@@ -113,6 +113,7 @@ template <int NV> struct Elt<float, NV> {
 #pragma unroll
         for (int e = 0; e < VEC; ++e) acc[e] = fmaf(c, x.v[e], acc[e]);
     }
+    static __device__ __forceinline__ void axpy_paired(float c, const Row& x, float (&acc)[VEC]) { axpy(c, x, acc); }
     static __device__ __forceinline__ void to_float(const Row& x, float (&f)[VEC]) {
 #pragma unroll
         for (int e = 0; e < VEC; ++e) f[e] = x.v[e];
@@ -180,6 +181,12 @@ template <int NV> struct Elt<__nv_bfloat16, NV> {
                 acc[2 * i + 1] = fmaf(c, __uint_as_float(x.w[i] & 0xffff0000u), acc[2 * i + 1]);
             }
         }
+    }
+    // The same with two FMAs per instruction whatever the lane width (for loops that are bound by issue slots).
+    static __device__ __forceinline__ void axpy_paired(float c, const Row& x, float (&acc)[VEC]) {
+#pragma unroll
+        for (int i = 0; i < NW; ++i)
+            fma2(acc[2 * i], acc[2 * i + 1], c, c, __uint_as_float(x.w[i] << 16), __uint_as_float(x.w[i] & 0xffff0000u));
     }
     static __device__ __forceinline__ void to_float(const Row& x, float (&f)[VEC]) {
 #pragma unroll

@@ -195,7 +195,7 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
             }
         }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) E::axpy(cks[i], kk[i], dqv);
+        for (int i = 0; i < 8; ++i) E::axpy_paired(cks[i], kk[i], dqv);
     }
     if (active) E::store(dq + row * D + ch, dqv);
 }
@@ -220,20 +220,33 @@ fixed_window_backward_key_kernel(const T* __restrict__ q, const T* __restrict__ 
     float ak[VEC], av[VEC];
 #pragma unroll
     for (int e = 0; e < VEC; ++e) ak[e] = av[e] = 0.0f;
-    int p = 0;
-    for (int u = 0; u < pr.kt; ++u)
-        for (int vv = 0; vv < pr.kh; ++vv)
-            for (int w = 0; w < pr.kw; ++w, ++p) {
-                // the query whose window cell p is this key
-                const int qt = t - (u - pr.kt / 2), qy = y - (vv - pr.kh / 2), qx = x - (w - pr.kw / 2);
-                if (qt < 0 || qt >= pr.T || qy < 0 || qy >= pr.H || qx < 0 || qx >= pr.W) continue;
-                const long long qrow = ((static_cast<long long>(qt) * pr.H + qy) * pr.W + qx) * pr.heads + m;
-                const float2 c = __ldg(coef + qrow * pr.P + p);
-                const Row qr = E::load(q + qrow * D + ch);
-                const Row dr = E::load(dout + qrow * D + ch);
-                E::axpy(c.x, qr, ak);
-                E::axpy(c.y, dr, av);
+    // The query whose window cell p = (u, vv, w) is this key sits at key - b(p): walking w moves it one token
+    // back, so the row and coefficient pointers are stepped instead of recomputed, and the range tests are
+    // taken once per loop level.
+    const long long tok = static_cast<long long>(pr.heads) * D;              // elements from one token to the next
+    const long long coef_tok = static_cast<long long>(pr.heads) * pr.P;
+    for (int u = 0; u < pr.kt; ++u) {
+        const int qt = t - (u - pr.kt / 2);
+        if (qt < 0 || qt >= pr.T) continue;
+        for (int vv = 0; vv < pr.kh; ++vv) {
+            const int qy = y - (vv - pr.kh / 2);
+            if (qy < 0 || qy >= pr.H) continue;
+            const int qx0 = x + pr.kw / 2;                                   // the query of w = 0; w steps it down
+            const long long qrow0 = ((static_cast<long long>(qt) * pr.H + qy) * pr.W + qx0) * pr.heads + m;
+            const T* qp = q + qrow0 * D + ch;
+            const T* dp = dout + qrow0 * D + ch;
+            const float2* cp = coef + qrow0 * pr.P + (u * pr.kh + vv) * pr.kw;
+            for (int w = 0; w < pr.kw; ++w, qp -= tok, dp -= tok, cp -= coef_tok - 1) {
+                const int qx = qx0 - w;
+                if (qx < 0 || qx >= pr.W) continue;
+                const float2 c = __ldg(cp);
+                const Row qr = E::load(qp);
+                const Row dr = E::load(dp);
+                E::axpy_paired(c.x, qr, ak);
+                E::axpy_paired(c.y, dr, av);
             }
+        }
+    }
     const long long row = n * pr.heads + m;
     E::store(dk + row * D + ch, ak);
     E::store(dv + row * D + ch, av);
