@@ -262,7 +262,7 @@ int dsa3d_backward_fixed_window(const void* q, const void* k, const void* v, con
         }
     }
     e = dsa3d::launch_fixed_window_backward(q, k, v, lse, dout, dq, dk, dv, doffsets, static_cast<float2*>(workspace), table,
-                                            pr, dtype == DSA3D_BF16, st);
+                                            pr, dtype == DSA3D_BF16, !std::getenv("DSA3D_NO_TENSOR_FIXED_WINDOW"), st);
     if (e != cudaSuccess) return cuda_failed(e);
     e = record(3, st);
     return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);

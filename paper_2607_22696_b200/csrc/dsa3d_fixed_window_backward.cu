@@ -16,6 +16,8 @@
 //       dK_j = sum_p coefK[j - b(p), p] q_{j - b(p)},  dV_j = sum_p coefV[j - b(p), p] dO_{j - b(p)},
 //       and written once in the storage type - no fp32 accumulators, no atomics, bitwise
 //       deterministic.
+#include <type_traits>
+
 #include "dsa3d_common.cuh"
 #include "dsa3d_kernels.h"
 
@@ -174,7 +176,8 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
     }
     __syncwarp();
 
-    // ---- dQ = sum_p (scale dS_p) K_j over the window cells inside the grid
+    // ---- dQ = sum_p (scale dS_p) K_j over the window cells inside the grid (unless the tile kernel forms it)
+    if (dq == nullptr) return;
     float dqv[VEC];
 #pragma unroll
     for (int e = 0; e < VEC; ++e) dqv[e] = 0.0f;
@@ -255,7 +258,7 @@ fixed_window_backward_key_kernel(const T* __restrict__ q, const T* __restrict__ 
 template <typename T, int D>
 cudaError_t launch_t(const void* q, const void* k, const void* v, const float* lse, const void* dout, void* dq,
                      void* dk, void* dv, float* doffsets, float2* coef, const float* table, const Problem& pr,
-                     cudaStream_t stream) {
+                     bool tile_grad, cudaStream_t stream) {
     constexpr int LPR = D / Elt<T, 1>::VEC;
     const int box = (doffsets || table) ? (pr.kt + 1) * (pr.kh + 1) * (pr.kw + 1) : pr.P;
     const size_t box8 = static_cast<size_t>((box + 7) & ~7);
@@ -271,11 +274,22 @@ cudaError_t launch_t(const void* q, const void* k, const void* v, const float* l
     }
     long long groups = threads / LPR;
     long long blocks = (pr.items + groups - 1) / groups;
+    // bf16, small windows: dQ, dK and dV per tile from regions in shared memory, after the coefficients are out
+    const bool tiled = std::is_same<T, __nv_bfloat16>::value && tile_grad && fixed_window_tile_grad_covers(pr, true);
     qk<<<static_cast<unsigned>(blocks), threads, smem, stream>>>(
         static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), lse, static_cast<const T*>(dout),
-        static_cast<T*>(dq), doffsets, coef, table, pr);
+        tiled ? nullptr : static_cast<T*>(dq), doffsets, coef, table, pr);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    if (tiled) {
+        if (try_fixed_window_tile_grad(q, k, dout, coef, dq, dk, dv, pr, stream, &e)) return e;
+        // could not be launched after all: the query kernel once more, this time with its dQ
+        qk<<<static_cast<unsigned>(blocks), threads, smem, stream>>>(
+            static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), lse, static_cast<const T*>(dout),
+            static_cast<T*>(dq), doffsets, coef, table, pr);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
     groups = 256 / LPR;
     blocks = (pr.items + groups - 1) / groups;
     fixed_window_backward_key_kernel<T, D><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
@@ -288,11 +302,11 @@ cudaError_t launch_t(const void* q, const void* k, const void* v, const float* l
 cudaError_t launch_fixed_window_backward(const void* q, const void* k, const void* v, const float* lse,
                                          const void* dout, void* dq, void* dk, void* dv, float* doffsets,
                                          float2* coef, const float* table, const Problem& pr, bool bf16,
-                                         cudaStream_t stream) {
+                                         bool tile_grad, cudaStream_t stream) {
 #define DSA3D_CASE(DD)                                                                                                 \
     case DD:                                                                                                           \
-        return bf16 ? launch_t<__nv_bfloat16, DD>(q, k, v, lse, dout, dq, dk, dv, doffsets, coef, table, pr, stream)   \
-                    : launch_t<float, DD>(q, k, v, lse, dout, dq, dk, dv, doffsets, coef, table, pr, stream);
+        return bf16 ? launch_t<__nv_bfloat16, DD>(q, k, v, lse, dout, dq, dk, dv, doffsets, coef, table, pr, tile_grad, stream)   \
+                    : launch_t<float, DD>(q, k, v, lse, dout, dq, dk, dv, doffsets, coef, table, pr, tile_grad, stream);
     switch (pr.d) {
         DSA3D_CASE(32)
         DSA3D_CASE(64)

@@ -61,16 +61,25 @@ int backward_impl(const void* q, const void* k, const void* v, const float* offs
 // Backward of the fixed-window variant (dsa3d_fixed_window_backward.cu): dq, dk, dv in the storage
 // type, doffsets (may be NULL), coef [N*heads, P] scratch.  `table` (or NULL): the dot products
 // q.K_j and dO.V_j of every query's box as try_fixed_window_tables leaves them; the kernel then
-// reads them instead of gathering K and V rows for them.
+// reads them instead of gathering K and V rows for them.  `tile_grad`: let the tile kernel of
+// dsa3d_fixed_window_tile_grad.cu form dq, dk and dv where it covers the shape.
 cudaError_t launch_fixed_window_backward(const void* q, const void* k, const void* v, const float* lse,
                                          const void* dout, void* dq, void* dk, void* dv, float* doffsets,
                                          float2* coef, const float* table, const Problem& pr, bool bf16,
-                                         cudaStream_t stream);
+                                         bool tile_grad, cudaStream_t stream);
 
 // Dot-product tables of the fixed-window backward on the tensor cores (dsa3d_fixed_window_tables.cu).
 // fixed_window_table_floats: floats per (token, head) item, 0 when the shape is not covered.
 // try_fixed_window_tables: false when the shape is not covered (nothing launched).
 int fixed_window_table_floats(const Problem& pr, bool bf16);
+
+// The three weighted row sums of the fixed-window backward (dQ over the K region, dK over the q region, dV over
+// the dO region) per tile of 4 x 4 x 8 outputs with the region in shared memory (dsa3d_fixed_window_tile_grad.cu),
+// from the coefficient pairs the query kernel left.  covers: bf16, 64 or 128 channels, windows (3,3,3), (2,2,2).
+// try_...: false when nothing was launched (shape not covered, or the tensor maps could not be made).
+bool fixed_window_tile_grad_covers(const Problem& pr, bool bf16);
+bool try_fixed_window_tile_grad(const void* q, const void* k, const void* dout, const float2* coef, void* dq, void* dk,
+                                void* dv, const Problem& pr, cudaStream_t stream, cudaError_t* err);
 bool try_fixed_window_tables(const void* q, const void* k, const void* v, const void* dout, float* table,
                              const Problem& pr, cudaStream_t stream, cudaError_t* err);
 
