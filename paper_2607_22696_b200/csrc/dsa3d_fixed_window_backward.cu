@@ -274,8 +274,10 @@ cudaError_t launch_t(const void* q, const void* k, const void* v, const float* l
     }
     long long groups = threads / LPR;
     long long blocks = (pr.items + groups - 1) / groups;
-    // bf16, small windows: dQ, dK and dV per tile from regions in shared memory, after the coefficients are out
-    const bool tiled = std::is_same<T, __nv_bfloat16>::value && tile_grad && fixed_window_tile_grad_covers(pr, true);
+    // bf16: dQ, dK and dV per tile, after the coefficients are out - from regions in shared memory for the
+    // small windows, as plane-by-plane products on the tensor cores for the larger ones
+    const bool tiled = std::is_same<T, __nv_bfloat16>::value && tile_grad &&
+                       (fixed_window_tile_grad_covers(pr, true) || fixed_window_planes_grad_covers(pr, true));
     qk<<<static_cast<unsigned>(blocks), threads, smem, stream>>>(
         static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), lse, static_cast<const T*>(dout),
         tiled ? nullptr : static_cast<T*>(dq), doffsets, coef, table, pr);
@@ -283,6 +285,7 @@ cudaError_t launch_t(const void* q, const void* k, const void* v, const float* l
     if (e != cudaSuccess) return e;
     if (tiled) {
         if (try_fixed_window_tile_grad(q, k, dout, coef, dq, dk, dv, pr, stream, &e)) return e;
+        if (try_fixed_window_planes_grad(q, k, dout, coef, dq, dk, dv, pr, stream, &e)) return e;
         // could not be launched after all: the query kernel once more, this time with its dQ
         qk<<<static_cast<unsigned>(blocks), threads, smem, stream>>>(
             static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), lse, static_cast<const T*>(dout),
