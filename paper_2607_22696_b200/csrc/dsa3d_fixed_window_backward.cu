@@ -32,7 +32,7 @@ __global__ void __launch_bounds__(256, TABLE ? DSA3D_FWB_TABLE_BLOCKS : 1)
 fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                                    const float* __restrict__ lse, const T* __restrict__ dout, T* __restrict__ dq,
                                    float* __restrict__ doffsets, float2* __restrict__ coef,
-                                   const float* __restrict__ table, const Problem pr) {
+                                   const float* __restrict__ table, const bool coef_planes, const Problem pr) {
     using E = Elt<T, 1>;
     using Row = typename E::Row;
     constexpr int VEC = E::VEC;
@@ -164,7 +164,16 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
         const float ck = scale * alpha * (tb[idx] - delta);
         sk[p] = ck;
         if (active) {
-            coef[row * pr.P + p] = make_float2(ck, alpha);
+            if (coef_planes) {
+                // for the plane-by-plane tile kernel: one plane of ck and one of cv, each [head][sample][token],
+                // so that the outputs of a tile row find the coefficients of one window cell side by side
+                float* planes = reinterpret_cast<float*>(coef);
+                const long long at = (static_cast<long long>(m) * pr.P + p) * pr.N + n;
+                planes[at] = ck;
+                planes[pr.N * pr.heads * pr.P + at] = alpha;
+            } else {
+                coef[row * pr.P + p] = make_float2(ck, alpha);
+            }
             if (want_doff) {
                 const float s0 = fmaf(ck, ta[idx], alpha * tb[idx]);
                 float* dst = doffsets + (row * pr.P + p) * 3;
@@ -276,20 +285,22 @@ cudaError_t launch_t(const void* q, const void* k, const void* v, const float* l
     long long blocks = (pr.items + groups - 1) / groups;
     // bf16: dQ, dK and dV per tile, after the coefficients are out - from regions in shared memory for the
     // small windows, as plane-by-plane products on the tensor cores for the larger ones
-    const bool tiled = std::is_same<T, __nv_bfloat16>::value && tile_grad &&
-                       (fixed_window_tile_grad_covers(pr, true) || fixed_window_planes_grad_covers(pr, true));
+    const bool planes = std::is_same<T, __nv_bfloat16>::value && tile_grad && fixed_window_planes_grad_covers(pr, true);
+    const bool tiled = planes || (std::is_same<T, __nv_bfloat16>::value && tile_grad && fixed_window_tile_grad_covers(pr, true));
     qk<<<static_cast<unsigned>(blocks), threads, smem, stream>>>(
         static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), lse, static_cast<const T*>(dout),
-        tiled ? nullptr : static_cast<T*>(dq), doffsets, coef, table, pr);
+        tiled ? nullptr : static_cast<T*>(dq), doffsets, coef, table, planes, pr);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (tiled) {
-        if (try_fixed_window_tile_grad(q, k, dout, coef, dq, dk, dv, pr, stream, &e)) return e;
-        if (try_fixed_window_planes_grad(q, k, dout, coef, dq, dk, dv, pr, stream, &e)) return e;
-        // could not be launched after all: the query kernel once more, this time with its dQ
+        if (planes ? try_fixed_window_planes_grad(q, k, dout, reinterpret_cast<const float*>(coef), dq, dk, dv, pr, stream, &e)
+                   : try_fixed_window_tile_grad(q, k, dout, coef, dq, dk, dv, pr, stream, &e))
+            return e;
+        // could not be launched after all: the query kernel once more, this time with its dQ (and the
+        // coefficients in the order the key kernel reads them)
         qk<<<static_cast<unsigned>(blocks), threads, smem, stream>>>(
             static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), lse, static_cast<const T*>(dout),
-            static_cast<T*>(dq), doffsets, coef, table, pr);
+            static_cast<T*>(dq), doffsets, coef, table, false, pr);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }

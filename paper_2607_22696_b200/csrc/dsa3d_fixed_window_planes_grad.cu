@@ -17,9 +17,9 @@
 //   The coefficients a thread needs for a plane are requested one plane ahead, with unconditional
 //   loads from a clamped position (a load under a condition is waited for where it is issued).
 //
-// Roles: warps 0-7 are the workers (two threads per output row, the window's kernel rows split
-// between them), warp 8 holds the thread that issues every TMA load, warp 9 the thread that issues
-// every MMA.  Nothing but mbarriers orders the roles.  Every wait is bounded; a wait that runs out
+// Roles: warps 0-15 are the workers (four threads per output row, the window's kernel rows split
+// between them: what bounds the kernel is the length of a worker's instruction stream per plane),
+// warp 16 holds the thread that issues every TMA load, warp 17 the thread that issues every MMA.  Nothing but mbarriers orders the roles.  Every wait is bounded; a wait that runs out
 // raises the library's timeout flag, after which nobody waits any more: the CTA walks through the
 // rest of its work, drains its loads and frees its TMEM.
 #include <cuda_bf16.h>
@@ -32,7 +32,8 @@ namespace dsa3d {
 namespace {
 
 constexpr int kPgTT = 4, kPgTY = 4, kPgTX = 8, kPgRows = kPgTT * kPgTY * kPgTX;    // 128 outputs per tile
-constexpr int kPgWorkers = 256, kPgThreads = kPgWorkers + 64;
+constexpr int kPgSplit = 4;                                       // worker threads per output row (the window's kernel rows split between them)
+constexpr int kPgWorkers = kPgSplit * kPgRows, kPgThreads = kPgWorkers + 64;
 constexpr int kPgMaxSlots = 4;
 
 template <int D, int KT, int KH, int KW>
@@ -42,7 +43,7 @@ struct PgShape {
     static constexpr int PS = RY * RX;                              // rows of one region plane
     static constexpr int PSP = (PS + 15) / 16 * 16;                 // padded to the MMA granularity
     static constexpr int KB = (PSP + 63) / 64;                      // 64-column blocks of a C row
-    static constexpr int VH = (KH + 1) / 2;                         // kernel rows of the first thread of a pair
+    static constexpr int VH = (KH + kPgSplit - 1) / kPgSplit;       // kernel rows per worker thread, at most
     static constexpr int C_BYTES = KB * kPgRows * 128;              // one coefficient matrix (head or remainder)
     static constexpr int SLOT_HALF = PSP * 128;                     // one 64-channel half of a plane buffer
     static constexpr int SLOT_BYTES = NH * SLOT_HALF;
@@ -51,7 +52,11 @@ struct PgShape {
     // target (dK, dV) reaches k - 1 - k/2 back
     static constexpr int FT = KT / 2, FY = KH / 2, FX = KW / 2;
     static constexpr int BT = KT - 1 - KT / 2, BY = KH - 1 - KH / 2, BX = KW - 1 - KW / 2;
-    static constexpr int NS_RAW = (227 * 1024 - 2048 - 2 * C_BYTES) / SLOT_BYTES;
+    // The coefficient matrices of successive (plane, head | remainder) units rotate through NC buffers, so
+    // the workers write up to NC - 1 units ahead of the chain that is running.
+    static constexpr int BUDGET = 227 * 1024 - 2048;
+    static constexpr int NC = BUDGET - 3 * SLOT_BYTES >= 4 * C_BYTES ? 4 : 3;
+    static constexpr int NS_RAW = (BUDGET - NC * C_BYTES) / SLOT_BYTES;
     static constexpr int NS = NS_RAW > kPgMaxSlots ? kPgMaxSlots : NS_RAW;
     static_assert(PSP <= 256 && 3 * D <= 512, "a plane is one MMA's K extent; three accumulators in TMEM");
     static_assert(SLOT_HALF % 1024 == 0, "plane buffers keep the 1024-byte alignment of the swizzle");
@@ -62,10 +67,10 @@ struct PgShape {
 template <int D, int KT, int KH, int KW>
 struct __align__(1024) PgSmem {
     using S = PgShape<D, KT, KH, KW>;
-    unsigned char c[2][S::C_BYTES];                                 // coefficient matrix: head, remainder
+    unsigned char c[S::NC][S::C_BYTES];                             // coefficient matrices in rotation
     unsigned char slot[S::NS][S::NH][S::SLOT_HALF];                 // ring of region planes
     uint64_t bar_full[kPgMaxSlots], bar_slot_free[kPgMaxSlots];
-    uint64_t bar_c_full[2], bar_c_free[2], bar_o[3];
+    uint64_t bar_c_full[4], bar_c_free[4], bar_o[3];
     uint32_t tmem_base;
     uint32_t abort;                                                 // a wait ran out somewhere: nobody waits any more
 };
@@ -73,11 +78,11 @@ struct __align__(1024) PgSmem {
 template <int D, int KT, int KH, int KW>
 __global__ void __launch_bounds__(kPgThreads, 1)
 fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_q,
-                                const __grid_constant__ CUtensorMap map_do, const float2* __restrict__ coef,
+                                const __grid_constant__ CUtensorMap map_do, const float* __restrict__ coef,
                                 __nv_bfloat16* __restrict__ dq, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
                                 int T, int H, int W, int heads, int tiles_x, int tiles_y, int total, int* timeout_flag) {
     using S = PgShape<D, KT, KH, KW>;
-    constexpr int NH = S::NH, RT = S::RT, RX = S::RX, PS = S::PS, PSP = S::PSP, VH = S::VH, NS = S::NS, P = S::P;
+    constexpr int NH = S::NH, RT = S::RT, RX = S::RX, PS = S::PS, PSP = S::PSP, VH = S::VH, NS = S::NS, NC = S::NC, P = S::P;
     constexpr int JOBS = 3 * RT;                                      // plane loads per tile
     extern __shared__ unsigned char raw[];
     PgSmem<D, KT, KH, KW>& s =
@@ -86,7 +91,7 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
 
     if (tid == 0) {
         for (int i = 0; i < kPgMaxSlots; ++i) { mbar_init(smem_u32(&s.bar_full[i]), 1); mbar_init(smem_u32(&s.bar_slot_free[i]), 1); }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < 4; ++i) {
             mbar_init(smem_u32(&s.bar_c_full[i]), kPgWorkers / 32);   // lane 0 of every worker warp
             mbar_init(smem_u32(&s.bar_c_free[i]), 1);
         }
@@ -102,7 +107,7 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
     // the coefficient matrices start as zeros (a thread only ever writes its own cells, and writes them
     // back to zero after its last plane); rows PS .. PSP-1 of the plane buffers are never written by a
     // load and are multiplied by zero columns of C: they must not hold anything non-finite
-    for (int i = tid; i < 2 * S::C_BYTES / 16; i += kPgThreads) reinterpret_cast<uint4*>(&s.c[0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = tid; i < S::NC * S::C_BYTES / 16; i += kPgThreads) reinterpret_cast<uint4*>(&s.c[0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
     if constexpr (PSP > PS) {
         for (int i = tid; i < NS * NH * (PSP - PS) * 8; i += kPgThreads) {
             const int chunk = i & 7, row = PS + (i >> 3) % (PSP - PS), which = (i >> 3) / (PSP - PS);
@@ -165,28 +170,37 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
             constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (static_cast<uint32_t>(D >> 3) << 17) |
                                        (static_cast<uint32_t>(kPgRows >> 4) << 24);
             constexpr uint64_t slot_step = S::SLOT_BYTES >> 4;
-            uint64_t desc_c[2][S::KB];
-            for (int part = 0; part < 2; ++part)
-                for (int b = 0; b < S::KB; ++b) desc_c[part][b] = smem_desc(smem_u32(&s.c[part][b * (kPgRows * 128)]));
+            uint64_t desc_c[NC][S::KB];
+            for (int buf = 0; buf < NC; ++buf)
+                for (int b = 0; b < S::KB; ++b) desc_c[buf][b] = smem_desc(smem_u32(&s.c[buf][b * (kPgRows * 128)]));
             const uint64_t desc_slot = smem_desc_mn(smem_u32(s.slot[0][0]), static_cast<uint32_t>(S::SLOT_HALF));
-            int sl = 0, pc = 0;                                       // plane buffer, plane counter of the CTA
-            uint32_t full_parity = 0;
+            int sl = 0, buf = 0;                                      // plane buffer; coefficient buffer of the next unit
+            uint32_t full_parity = 0, c_parity = 0;
             for (int it = 0; it < my_tiles; ++it) {
                 for (int sweep = 0; sweep < 3; ++sweep) {
                     const uint32_t acc = tmem + static_cast<uint32_t>(sweep * D);
-                    for (int pl = 0; pl < RT; ++pl, ++pc) {
+                    for (int pl = 0; pl < RT; ++pl) {
                         bool ready = wait(&s.bar_full[sl], full_parity, 52);
 #pragma unroll
                         for (int part = 0; part < 2; ++part) {
-                            if (ready) ready = wait(&s.bar_c_full[part], static_cast<uint32_t>(pc & 1), 53);
+                            if (ready) ready = wait(&s.bar_c_full[buf], c_parity, 53);
                             if (ready) {
                                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                                // one of NC descriptor sets; chosen by comparisons so that the array stays in registers
+                                uint64_t dc[S::KB];
+#pragma unroll
+                                for (int b = 0; b < S::KB; ++b) {
+                                    dc[b] = desc_c[0][b];
+#pragma unroll
+                                    for (int i = 1; i < NC; ++i) if (buf == i) dc[b] = desc_c[i][b];
+                                }
 #pragma unroll
                                 for (int ks = 0; ks < PSP / 16; ++ks)
-                                    umma_bf16(acc, desc_c[part][ks >> 2] + 2 * (ks & 3), desc_slot + sl * slot_step + 128 * ks, idesc,
+                                    umma_bf16(acc, dc[ks >> 2] + 2 * (ks & 3), desc_slot + sl * slot_step + 128 * ks, idesc,
                                               (pl | part | ks) ? 1u : 0u);
                             }
-                            umma_commit(smem_u32(&s.bar_c_free[part]));   // arrives at once if nothing was issued
+                            umma_commit(smem_u32(&s.bar_c_free[buf]));    // arrives at once if nothing was issued
+                            if (++buf == NC) { buf = 0; c_parity ^= 1u; }
                         }
                         umma_commit(smem_u32(&s.bar_slot_free[sl]));
                         if (pl == RT - 1) umma_commit(smem_u32(&s.bar_o[sweep]));
@@ -197,139 +211,213 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
         }
     } else {
         // ==================================================================== workers
-        const int lt = warp & 3, half = warp >> 2;                    // output plane of the tile; which thread of the pair
+        const int lt = warp & 3, sub = warp >> 2;                     // output plane of the tile; which thread of the row's four
         const int ly = lane >> 3, lx = lane & 7;
         const int r = lt * 32 + lane;                                 // output row of the tile = TMEM lane
         const uint32_t lane_base = static_cast<uint32_t>(lt * 32) << 16;
         const uint32_t row_off = static_cast<uint32_t>(r) * 128u, rx = static_cast<uint32_t>(r & 7);
-        // byte offset, inside a coefficient matrix, of this row's cell at kernel row vv, column ww
-        auto c_offset = [&](int vv, int ww) {
-            const uint32_t col = static_cast<uint32_t>((ly + vv) * RX + lx + ww);
-            return (col >> 6) * (kPgRows * 128) + row_off + ((((col & 63) >> 3) ^ rx) << 4) + (col & 7) * 2;
+        const int v0 = (sub * KH) / kPgSplit, nv = ((sub + 1) * KH) / kPgSplit - v0;    // this thread's kernel rows (warp-uniform)
+        // The cells of one kernel row are KW neighbouring columns of the output's row of C: they are written as
+        // whole 16-byte chunks of 8 columns (one chunk, or two when the cells straddle a chunk boundary).
+        // The other columns of those chunks belong to no cell of this output row - the neighbouring kernel
+        // rows lie 8 + KW - 1 columns away - so writing them as zeros is right.  Where the chunks lie and by
+        // how many columns the cells are shifted inside them is the same for every plane and tile:
+        // bits 0-11 / 12-23 the byte offsets of the two chunks (in 16-byte units), bits 24-26 the shift.
+        static_assert(S::C_BYTES <= 65536 && KW <= 7 && RX >= KW + 7, "chunk offsets in 12 bits; a kernel row's chunks touch no other row's cells");
+        constexpr int CELLS = VH * KW;
+        uint32_t row_geo[VH];
+#pragma unroll
+        for (int vi = 0; vi < VH; ++vi) {
+            const int vv = vi < nv ? v0 + vi : v0;
+            const uint32_t col0 = static_cast<uint32_t>((ly + vv) * RX + lx);
+            auto chunk_off = [&](uint32_t col) { return (col >> 6) * (kPgRows * 128) + row_off + ((((col & 63) >> 3) ^ rx) << 4); };
+            row_geo[vi] = (chunk_off(col0) >> 4) | ((chunk_off(col0 + 8) >> 4) << 12) | ((col0 & 7u) << 24);
+        }
+        // KW bf16 values, packed in pairs (w[3] unused beyond KW), to their places in the row's two chunks
+        auto store_row = [&](unsigned char* dst, uint32_t geo, const uint32_t (&w)[4]) {
+            const bool s1 = (geo >> 24) & 1u, s2 = (geo >> 25) & 1u, s4 = (geo >> 26) & 1u;
+            uint32_t a[5], b[6], c[8];
+            a[0] = s1 ? w[0] << 16 : w[0];
+#pragma unroll
+            for (int i = 1; i < 4; ++i) a[i] = s1 ? __funnelshift_l(w[i - 1], w[i], 16) : w[i];
+            a[4] = s1 ? w[3] >> 16 : 0u;
+            b[0] = s2 ? 0u : a[0];
+#pragma unroll
+            for (int i = 1; i < 5; ++i) b[i] = s2 ? a[i - 1] : a[i];
+            b[5] = s2 ? a[4] : 0u;
+            c[0] = s4 ? 0u : b[0];
+            c[1] = s4 ? 0u : b[1];
+#pragma unroll
+            for (int i = 2; i < 6; ++i) c[i] = s4 ? b[i - 2] : b[i];
+            c[6] = s4 ? b[4] : 0u;
+            c[7] = s4 ? b[5] : 0u;
+            *reinterpret_cast<uint4*>(dst + ((geo & 0xfffu) << 4)) = make_uint4(c[0], c[1], c[2], c[3]);
+            if (((geo >> 24) & 7u) + KW > 8u) *reinterpret_cast<uint4*>(dst + (((geo >> 12) & 0xfffu) << 4)) = make_uint4(c[4], c[5], c[6], c[7]);
         };
-        const float* cf = reinterpret_cast<const float*>(coef);
+        const int n_step = T * H * W;                                 // tokens: the step from one sample's plane to the next
+        const float* plane_ck = coef;                                 // [head][sample][token]
+        const float* plane_cv = coef + static_cast<long long>(heads) * P * n_step;
         // Step q of this thread = (tile, sweep, kernel plane u) in the order they come: the coefficients of
-        // the row's cells (this thread's kernel rows, every column) in that plane.
+        // the row's cells (this thread's kernel rows, every column) in that plane.  What depends on the
+        // tile alone is worked out at the tile's first step: positions inside a coefficient plane (they
+        // fit 32 bits, the host checks) and which source queries exist.
         const int steps = my_tiles * 3 * KT;
-        auto fetch = [&](int q, float (&wv)[VH][KW], uint32_t& dead) {
+        int g_a0 = 0, g_a1 = 0;
+        uint32_t g_tmask = 0u, g_ymask = 0u, g_xmask = 0u, g_own = 0u;
+        auto fetch = [&](int q, float (&wv)[CELLS], uint32_t& dead) {
             const int ti = q / (3 * KT), rem = q - ti * (3 * KT), sweep = rem / KT, u = rem - sweep * KT;
-            int m, t0, y0, x0;
-            locate(ti, m, t0, y0, x0);
-            const int ot = t0 + lt, oy = y0 + ly, ox = x0 + lx;       // the output position
-            dead = 0u;
-            long long base;                                           // index of the cell (first kernel row of this thread, column 0)
-            int step_v, step_w;                                       // index steps to the next kernel row / column
-            int st, sy0, sx0;                                         // the query the cell's coefficient belongs to
-            if (sweep == 0) {                                         // output = the query itself, cell (u, vv, ww)
-                st = ot; sy0 = oy; sx0 = ox;
-                base = (((static_cast<long long>(ot) * H + oy) * W + ox) * heads + m) * P + (u * KH + half * VH) * KW;
-                step_v = KW; step_w = 1;
-            } else {                                                  // output = a key; the query at region offset (u, vv, ww) of it
-                st = ot - S::BT + u; sy0 = oy - S::BY + half * VH; sx0 = ox - S::BX;
-                base = (((static_cast<long long>(st) * H + sy0) * W + sx0) * heads + m) * P +
-                       ((KT - 1 - u) * KH + (KH - 1 - half * VH)) * KW + (KW - 1);
-                step_v = W * heads * P - KW; step_w = heads * P - 1;
+            if (rem == 0) {
+                int m, t0, y0, x0;
+                locate(ti, m, t0, y0, x0);
+                const int ot = t0 + lt, oy = y0 + ly, ox = x0 + lx;   // the output position
+                const int n_out = (ot * H + oy) * W + ox;
+                g_a0 = m * P * n_step + n_out;                        // sample 0 of the output's own query
+                g_a1 = (m * P + P - 1) * n_step + n_out - ((S::BT * H + S::BY) * W + S::BX);   // last sample of the first source query
+                g_own = (ot < T && oy < H && ox < W) ? (1u << KW) - 1u : 0u;
+                g_tmask = g_ymask = g_xmask = 0u;
+#pragma unroll
+                for (int i = 0; i < KT; ++i) if (ot - S::BT + i >= 0 && ot - S::BT + i < T) g_tmask |= 1u << i;
+#pragma unroll
+                for (int i = 0; i < VH; ++i) if (i < nv && oy - S::BY + v0 + i >= 0 && oy - S::BY + v0 + i < H) g_ymask |= 1u << i;
+#pragma unroll
+                for (int i = 0; i < KW; ++i) if (ox - S::BX + i >= 0 && ox - S::BX + i < W) g_xmask |= 1u << i;
             }
-            const bool t_ok = st >= 0 && st < T;
-            const float* src = cf + (sweep == 2 ? 1 : 0);
+            // sweep 0: the output is the query itself, cell (u, v0 + vi, ww) = sample index, own token;
+            // sweeps 1, 2: the output is a key, the cell at region offset (u, v0 + vi, ww) belongs to the query
+            // at that offset from (key - B) and is its sample mirrored in the window
+            int base, step_v, step_w;
+            uint32_t alive = 0u;
+            if (sweep == 0) {
+                base = g_a0 + (u * KH + v0) * KW * n_step;
+                step_v = KW * n_step; step_w = n_step;
 #pragma unroll
-            for (int vi = 0; vi < VH; ++vi) {
-                if (vi + half * VH >= KH) continue;                   // warp-uniform: the second thread of a pair has one row less
-                const int sy = sweep == 0 ? sy0 : sy0 + vi;
-                const bool ty_ok = t_ok && sy >= 0 && sy < H;
+                for (int vi = 0; vi < VH; ++vi) if (vi < nv) alive |= g_own << (vi * KW);
+            } else {
+                base = g_a1 + u * (H * W - KH * KW * n_step) + v0 * (W - KW * n_step);
+                step_v = W - KW * n_step; step_w = 1 - n_step;
+                if ((g_tmask >> u) & 1u) {
 #pragma unroll
-                for (int ww = 0; ww < KW; ++ww) {
-                    const int sx = sweep == 0 ? sx0 : sx0 + ww;
-                    const bool exists = ty_ok && sx >= 0 && sx < W;
-                    const long long at = exists ? base + vi * step_v + ww * step_w : 0;
-                    wv[vi][ww] = __ldg(src + 2 * at);
-                    if (!exists) dead |= 1u << (vi * KW + ww);
+                    for (int vi = 0; vi < VH; ++vi) if ((g_ymask >> vi) & 1u) alive |= g_xmask << (vi * KW);
                 }
             }
+            const float* plane = sweep == 2 ? plane_cv : plane_ck;
+#pragma unroll
+            for (int i = 0; i < CELLS; ++i) {
+                const int vi = i / KW, ww = i - vi * KW;
+                const int at = ((alive >> i) & 1u) ? base + vi * step_v + ww * step_w : 0;    // a cell that does not exist reads word 0
+                wv[i] = __ldg(plane + at);
+            }
+            dead = ~alive;
         };
-
-        float wnext[VH][KW], wcur[VH][KW];
-        uint32_t dnext = 0u, dcur = 0u;
+        float wnext[CELLS];
+        uint32_t dnext = 0u;
 #pragma unroll
-        for (int vi = 0; vi < VH; ++vi)
-#pragma unroll
-            for (int ww = 0; ww < KW; ++ww) wnext[vi][ww] = wcur[vi][ww] = 0.0f;
+        for (int i = 0; i < CELLS; ++i) wnext[i] = 0.0f;
         int q = 0;                                                    // the step whose coefficients wnext holds
         if (steps > 0) fetch(0, wnext, dnext);
-        int pc = 0;
-        for (int it = 0; it < my_tiles; ++it) {
+        int buf = 0, clear_left = 0;                                  // coefficient buffer of the next unit; units still to clear
+        uint32_t c_parity = 0;
+        bool first_round = true;                                      // the first NC units find their buffers free
+        // Epilogue of sweep `sweep` of this CTA's tile `it`: the row's threads split the channels.
+        auto epilogue = [&](int it, int sweep) {
             int m, t0, y0, x0;
             locate(it, m, t0, y0, x0);
             const int ot = t0 + lt, oy = y0 + ly, ox = x0 + lx;
             const bool in_grid = ot < T && oy < H && ox < W;
             const long long n = (static_cast<long long>(ot) * H + oy) * W + ox;
-            for (int sweep = 0; sweep < 3; ++sweep) {
-                for (int pl = 0; pl < RT; ++pl, ++pc) {
-                    const int u_rt = pl - lt;                         // the kernel plane this region plane is to the warp's outputs
-                    const bool mine = u_rt >= 0 && u_rt < KT;
-                    // cells go back to zero on the plane after the last; the last output plane of the tile has no
-                    // such plane and clears its cells on the first plane of the next sweep instead
-                    const bool clear = u_rt == KT || (lt == kPgTT - 1 && pl == 0);
-                    if (mine) {
+            wait(&s.bar_o[sweep], static_cast<uint32_t>(it & 1), 55);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (sub * 32 < D) {
+                __nv_bfloat16* out = sweep == 0 ? dq : sweep == 1 ? dk : dv;
+                uint32_t regs[32];
+                tmem_load_32(tmem + lane_base + static_cast<uint32_t>(sweep * D + sub * 32), regs);
+                if (in_grid && !*abort_flag) {
+                    uint4* dst = reinterpret_cast<uint4*>(out + (n * heads + m) * D + sub * 32);
 #pragma unroll
-                        for (int vi = 0; vi < VH; ++vi)
+                    for (int i = 0; i < 4; ++i) {
+                        uint32_t o[4];
 #pragma unroll
-                            for (int ww = 0; ww < KW; ++ww) wcur[vi][ww] = wnext[vi][ww];
-                        dcur = dnext;
-                        if (++q < steps) fetch(q, wnext, dnext);
-                    }
-#pragma unroll
-                    for (int part = 0; part < 2; ++part) {
-                        if (pc > 0) wait(&s.bar_c_free[part], static_cast<uint32_t>((pc - 1) & 1), 54);   // the chain of the plane before
-                        if (mine || clear) {
-                            unsigned char* dst = s.c[part];
-#pragma unroll
-                            for (int vi = 0; vi < VH; ++vi) {
-                                const int vv = vi + half * VH;
-                                if (vv >= KH) continue;
-#pragma unroll
-                                for (int ww = 0; ww < KW; ++ww) {
-                                    const float p = (mine && !((dcur >> (vi * KW + ww)) & 1u)) ? wcur[vi][ww] : 0.0f;
-                                    __nv_bfloat16 val = __float2bfloat16_rn(p);
-                                    if (part) val = __float2bfloat16_rn(p - __bfloat162float(val));
-                                    *reinterpret_cast<__nv_bfloat16*>(dst + c_offset(vv, ww)) = val;
-                                }
-                            }
+                        for (int j = 0; j < 4; ++j) {
+                            const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(regs[8 * i + 2 * j]),
+                                                                            __uint_as_float(regs[8 * i + 2 * j + 1]));
+                            o[j] = *reinterpret_cast<const uint32_t*>(&h2);
                         }
-                        fence_async_smem();                           // the MMAs read C through the async proxy
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&s.bar_c_full[part]));
+                        dst[i] = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 }
-                // ------------------------------------------------------ epilogue of this sweep: the pair splits the channels
-                wait(&s.bar_o[sweep], static_cast<uint32_t>(it & 1), 55);
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                {
-                    constexpr int CH = D / 2;
-                    __nv_bfloat16* out = sweep == 0 ? dq : sweep == 1 ? dk : dv;
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        };
+        // The planes of the CTA's tiles and sweeps form one stream.  The epilogue of a sweep is taken after
+        // the first plane of the next sweep has been written, so that the MMA thread has that plane's chains
+        // to run meanwhile (each sweep has its own accumulator; by then the sweep's last chain is usually done).
+        for (int pj = 0, it = 0, sweep = 0, pl = 0; it < my_tiles; ++pj) {
+            const int u_rt = pl - lt;                         // the kernel plane this region plane is to the warp's outputs
+            const bool mine = u_rt >= 0 && u_rt < KT;
+            // A thread's cells are the same columns in every unit.  After its last plane of a sweep it
+            // writes them back to zero in the NC units that follow (one per buffer).
+            const bool writes = mine || clear_left > 0;
+            uint32_t rest[VH][4];                             // bf16 remainders of this plane's coefficients, packed in pairs
+            // ---- head
+            if (!first_round) wait(&s.bar_c_free[buf], c_parity ^ 1u, 54);       // the chain of the unit NC before this one
+            if (writes) {
+                unsigned char* dst = s.c[buf];
 #pragma unroll
-                    for (int c0 = 0; c0 < CH; c0 += 32) {
-                        uint32_t regs[32];
-                        tmem_load_32(tmem + lane_base + static_cast<uint32_t>(sweep * D + half * CH + c0), regs);
-                        if (in_grid && !*abort_flag) {
-                            uint4* dst = reinterpret_cast<uint4*>(out + (n * heads + m) * D + half * CH + c0);
+                for (int vi = 0; vi < VH; ++vi) {
+                    if (vi >= nv) continue;
+                    uint32_t head[4];
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                uint32_t o[4];
+                    for (int j = 0; j < 4; ++j) {
+                        // cells 2j and 2j + 1 of the kernel row (0 beyond KW, for a query that does not exist, and when clearing)
+                        float p[2];
 #pragma unroll
-                                for (int j = 0; j < 4; ++j) {
-                                    const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(regs[8 * i + 2 * j]),
-                                                                                    __uint_as_float(regs[8 * i + 2 * j + 1]));
-                                    o[j] = *reinterpret_cast<const uint32_t*>(&h2);
-                                }
-                                dst[i] = make_uint4(o[0], o[1], o[2], o[3]);
-                            }
+                        for (int e = 0; e < 2; ++e) {
+                            const int ww = 2 * j + e, i = vi * KW + ww;
+                            p[e] = (ww < KW && mine && !((dnext >> (ww < KW ? i : 0)) & 1u)) ? wnext[ww < KW ? i : 0] : 0.0f;
                         }
+                        const __nv_bfloat162 hd = __floats2bfloat162_rn(p[0], p[1]);
+                        head[j] = *reinterpret_cast<const uint32_t*>(&hd);
+                        const __nv_bfloat162 rm = __floats2bfloat162_rn(p[0] - __uint_as_float(head[j] << 16),
+                                                                        p[1] - __uint_as_float(head[j] & 0xffff0000u));
+                        rest[vi][j] = *reinterpret_cast<const uint32_t*>(&rm);
                     }
+                    store_row(dst, row_geo[vi], head);
                 }
-                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                if (!mine) --clear_left;
+            }
+            fence_async_smem();                               // the MMAs read C through the async proxy
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s.bar_c_full[buf]));
+            if (++buf == NC) { buf = 0; c_parity ^= 1u; first_round = false; }
+            // the next plane's coefficients: requested once the head is out, on their way while the
+            // remainder is written and through the waits of the next plane
+            if (mine && ++q < steps) fetch(q, wnext, dnext);
+            // ---- remainder
+            const bool writes_rest = mine || clear_left > 0;
+            if (!first_round) wait(&s.bar_c_free[buf], c_parity ^ 1u, 54);
+            if (writes_rest) {
+                unsigned char* dst = s.c[buf];
+                const uint32_t zero[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+                for (int vi = 0; vi < VH; ++vi) {
+                    if (vi >= nv) continue;
+                    if (mine) store_row(dst, row_geo[vi], rest[vi]);
+                    else store_row(dst, row_geo[vi], zero);
+                }
+                if (!mine) --clear_left;
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s.bar_c_full[buf]));
+            if (++buf == NC) { buf = 0; c_parity ^= 1u; first_round = false; }
+            if (mine && u_rt == KT - 1) clear_left = NC;
+            if (pl == 0 && pj > 0) epilogue(sweep == 0 ? it - 1 : it, sweep == 0 ? 2 : sweep - 1);
+            if (++pl == RT) {
+                pl = 0;
+                if (++sweep == 3) { sweep = 0; ++it; }
             }
         }
+        if (my_tiles > 0) epilogue(my_tiles - 1, 2);
     }
     // Gave up: loads may still be in flight towards this CTA's shared memory; give them a bounded time.
     if (*abort_flag && tid == kPgWorkers) {
@@ -344,7 +432,7 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
 }
 
 template <int D, int KT, int KH, int KW>
-cudaError_t launch_planes_grad(const void* q, const void* k, const void* dout, const float2* coef, void* dq, void* dk, void* dv,
+cudaError_t launch_planes_grad(const void* q, const void* k, const void* dout, const float* coef, void* dq, void* dk, void* dv,
                                const Problem& pr, int* flag, cudaStream_t stream, bool* unsupported) {
     using S = PgShape<D, KT, KH, KW>;
     const unsigned long long d = static_cast<unsigned long long>(pr.d), hd = static_cast<unsigned long long>(pr.heads);
@@ -361,8 +449,8 @@ cudaError_t launch_planes_grad(const void* q, const void* k, const void* dout, c
     }
     const int tiles_x = (pr.W + kPgTX - 1) / kPgTX, tiles_y = (pr.H + kPgTY - 1) / kPgTY, tiles_t = (pr.T + kPgTT - 1) / kPgTT;
     const long long total = static_cast<long long>(tiles_x) * tiles_y * tiles_t * pr.heads;
-    // the kernel counts planes and coefficient indices relative to a row in 32 bits
-    if (total * 3 * S::RT >= (1LL << 31) || static_cast<long long>(pr.W) * pr.heads * pr.P * (S::VH + 1) >= (1LL << 30)) {
+    // the kernel counts planes, and positions inside a coefficient plane, in 32 bits
+    if (total * 3 * S::RT >= (1LL << 31) || pr.N * pr.heads * pr.P >= (1LL << 31)) {
         *unsupported = true;
         return cudaSuccess;
     }
@@ -389,7 +477,7 @@ bool fixed_window_planes_grad_covers(const Problem& pr, bool bf16) {
     return pr.kt == 3 && ((pr.kh == 5 && pr.kw == 5) || (pr.kh == 7 && pr.kw == 7));
 }
 
-bool try_fixed_window_planes_grad(const void* q, const void* k, const void* dout, const float2* coef, void* dq, void* dk, void* dv,
+bool try_fixed_window_planes_grad(const void* q, const void* k, const void* dout, const float* coef, void* dq, void* dk, void* dv,
                                   const Problem& pr, cudaStream_t stream, cudaError_t* err) {
     *err = cudaSuccess;
     if (!fixed_window_planes_grad_covers(pr, true)) return false;

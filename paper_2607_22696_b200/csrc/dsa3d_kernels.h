@@ -83,7 +83,8 @@ bool try_fixed_window_tile_grad(const void* q, const void* k, const void* dout, 
 // The same three sums for the larger windows ((3,5,5), (3,7,7); bf16, 64 or 128 channels) as products
 //  C_plane . X_plane  on the tensor cores, one region plane at a time (dsa3d_fixed_window_planes_grad.cu).
 bool fixed_window_planes_grad_covers(const Problem& pr, bool bf16);
-bool try_fixed_window_planes_grad(const void* q, const void* k, const void* dout, const float2* coef, void* dq, void* dk,
+// `coef_planes`: the coefficients as one plane of ck and one of cv, each [head][sample][token].
+bool try_fixed_window_planes_grad(const void* q, const void* k, const void* dout, const float* coef_planes, void* dq, void* dk,
                                   void* dv, const Problem& pr, cudaStream_t stream, cudaError_t* err);
 bool try_fixed_window_tables(const void* q, const void* k, const void* v, const void* dout, float* table,
                              const Problem& pr, cudaStream_t stream, cudaError_t* err);

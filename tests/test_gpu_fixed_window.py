@@ -154,6 +154,16 @@ def test_fixed_window_backward_matches_the_oracle(shape, window, dtype):
     _backward_case(shape, window, dtype, 150)
 
 
+@pytest.mark.parametrize("shape,window", [((13, 22, 37, 3, 64), (3, 7, 7)), ((16, 21, 40, 3, 128), (3, 5, 5))])
+def test_plane_gradient_kernel_over_several_tiles_per_block(shape, window):
+    """More (tile, head) items than the GPU has SMs: every persistent block of the plane-by-plane gradient
+    kernel walks several tiles, so its stream of planes, the rotation of its coefficient buffers and the
+    clearing of cells between sweeps carry over from tile to tile."""
+    T, H, W, heads, _ = shape
+    assert ((T + 3) // 4) * ((H + 3) // 4) * ((W + 7) // 8) * heads > 2 * 148
+    _backward_case(shape, window, BF16, 152)
+
+
 def test_fixed_window_backward_without_doffsets_and_determinism():
     """doffsets may be NULL (only the window's own positions are visited then); dk and dv are
     gathered, not accumulated with atomics, so two runs agree bit for bit."""
