@@ -164,16 +164,7 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
         const float ck = scale * alpha * (tb[idx] - delta);
         sk[p] = ck;
         if (active) {
-            if (coef_planes) {
-                // for the plane-by-plane tile kernel: one plane of ck and one of cv, each [head][sample][token],
-                // so that the outputs of a tile row find the coefficients of one window cell side by side
-                float* planes = reinterpret_cast<float*>(coef);
-                const long long at = (static_cast<long long>(m) * pr.P + p) * pr.N + n;
-                planes[at] = ck;
-                planes[pr.N * pr.heads * pr.P + at] = alpha;
-            } else {
-                coef[row * pr.P + p] = make_float2(ck, alpha);
-            }
+            if (!coef_planes) coef[row * pr.P + p] = make_float2(ck, alpha);
             if (want_doff) {
                 const float s0 = fmaf(ck, ta[idx], alpha * tb[idx]);
                 float* dst = doffsets + (row * pr.P + p) * 3;
@@ -184,6 +175,31 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
         }
     }
     __syncwarp();
+
+    if (coef_planes) {
+        // For the plane-by-plane tile kernel the coefficients go out as one plane of ck and one of cv, each
+        // [head][sample][token], so that the outputs of a tile row find the coefficients of one window cell
+        // side by side.  The block's groups hold consecutive tokens: the block writes together, a run of
+        // tokens per sample, from the groups' arrays in shared memory.
+        const int groups = blockDim.x / LPR;
+        long long* group_at = reinterpret_cast<long long*>(group0 + static_cast<size_t>(groups) * (2 * NB8 + 2 * pr.P));
+        if (gl == 0) group_at[threadIdx.x / LPR] = static_cast<long long>(m) * pr.P * pr.N + n;
+        __syncthreads();                                   // warps with no item at all have left: they count as arrived
+        float* planes = reinterpret_cast<float*>(coef);
+        const long long plane_elems = pr.N * pr.heads * pr.P;
+        const long long block_first = static_cast<long long>(blockIdx.x) * groups;     // item of group 0
+        // the threads still here: the warps up to the last one that holds an item
+        const long long lanes_with_items = (pr.items - block_first) * LPR;
+        const int live = lanes_with_items >= blockDim.x ? static_cast<int>(blockDim.x) : static_cast<int>((lanes_with_items + 31) / 32 * 32);
+        for (int i = threadIdx.x; i < groups * pr.P; i += live) {
+            const int g = i % groups, p = i / groups;
+            if (block_first + g >= pr.items) continue;     // a group without an item (its arrays and position are not set)
+            const long long at = group_at[g];
+            const float* ga = group0 + static_cast<size_t>(g) * (2 * NB8 + 2 * pr.P) + 2 * NB8;     // sa, then sk
+            planes[at + p * pr.N] = ga[pr.P + p];
+            planes[plane_elems + at + p * pr.N] = ga[p];
+        }
+    }
 
     // ---- dQ = sum_p (scale dS_p) K_j over the window cells inside the grid (unless the tile kernel forms it)
     if (dq == nullptr) return;
@@ -274,8 +290,8 @@ cudaError_t launch_t(const void* q, const void* k, const void* v, const float* l
     const size_t per_group = (2 * box8 + 2 * pr.P) * sizeof(float);
     const size_t tables = box8 * sizeof(int4) + static_cast<size_t>((pr.P + 3) & ~3) * sizeof(int);
     int threads = 256;
-    while (threads > 32 && tables + static_cast<size_t>(threads / LPR) * per_group > 64 * 1024) threads /= 2;
-    const size_t smem = tables + static_cast<size_t>(threads / LPR) * per_group;
+    while (threads > 32 && tables + static_cast<size_t>(threads / LPR) * (per_group + sizeof(long long)) > 64 * 1024) threads /= 2;
+    const size_t smem = tables + static_cast<size_t>(threads / LPR) * (per_group + sizeof(long long));   // + a position per group
     auto qk = table ? fixed_window_backward_query_kernel<T, D, true> : fixed_window_backward_query_kernel<T, D, false>;
     if (smem > 48 * 1024) {
         const cudaError_t e = cudaFuncSetAttribute(qk, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
