@@ -260,11 +260,16 @@ fixed_window_tables_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                             pair_barrier(1 + lt);                     // both have copied: the staging rows may be refilled
                         }
                         if (in_grid && !*abort_flag) {
-                            if constexpr (BX == 4 && (BY * BX) % 4 == 0 && S::CELLS8 % 4 == 0) {
+                            // the run of VH * BX floats, in the widest pieces its alignment allows
+                            constexpr int RUN = VH * BX;
+                            constexpr bool whole = BY % kTbSplit == 0;     // every thread of the group has all VH rows
+                            if constexpr (whole && RUN % 4 == 0 && (BY * BX) % 4 == 0 && S::CELLS8 % 4 == 0) {
 #pragma unroll
-                                for (int vi = 0; vi < VH; ++vi)
-                                    if (vi + half * VH < BY)
-                                        reinterpret_cast<float4*>(dst)[vi] = make_float4(cells[4 * vi], cells[4 * vi + 1], cells[4 * vi + 2], cells[4 * vi + 3]);
+                                for (int i = 0; i < RUN / 4; ++i)
+                                    reinterpret_cast<float4*>(dst)[i] = make_float4(cells[4 * i], cells[4 * i + 1], cells[4 * i + 2], cells[4 * i + 3]);
+                            } else if constexpr (whole && RUN % 2 == 0 && (BY * BX) % 2 == 0 && S::CELLS8 % 2 == 0) {
+#pragma unroll
+                                for (int i = 0; i < RUN / 2; ++i) reinterpret_cast<float2*>(dst)[i] = make_float2(cells[2 * i], cells[2 * i + 1]);
                             } else {
 #pragma unroll
                                 for (int i = 0; i < VH * BX; ++i)
