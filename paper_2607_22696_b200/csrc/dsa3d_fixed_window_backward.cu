@@ -16,6 +16,8 @@
 //       dK_j = sum_p coefK[j - b(p), p] q_{j - b(p)},  dV_j = sum_p coefV[j - b(p), p] dO_{j - b(p)},
 //       and written once in the storage type - no fp32 accumulators, no atomics, bitwise
 //       deterministic.
+#include <cuda_bf16.h>
+
 #include <type_traits>
 
 #include "dsa3d_common.cuh"
@@ -23,6 +25,14 @@
 
 namespace dsa3d {
 namespace {
+
+// An fp32 value as two bf16 numbers whose sum is the value to 2^-17 relative: the nearest bf16 in the low
+// half of the word, the nearest bf16 of what is left in the high half.
+__device__ __forceinline__ uint32_t split_bf16_pair(float x) {
+    const __nv_bfloat16 head = __float2bfloat16_rn(x);
+    const __nv_bfloat16 rest = __float2bfloat16_rn(x - __bfloat162float(head));
+    return static_cast<uint32_t>(__bfloat16_as_ushort(head)) | (static_cast<uint32_t>(__bfloat16_as_ushort(rest)) << 16);
+}
 
 #ifndef DSA3D_FWB_TABLE_BLOCKS
 #define DSA3D_FWB_TABLE_BLOCKS 3
@@ -179,13 +189,14 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
     if (coef_planes) {
         // For the plane-by-plane tile kernel the coefficients go out as one plane of ck and one of cv, each
         // [head][sample][token], so that the outputs of a tile row find the coefficients of one window cell
-        // side by side.  The block's groups hold consecutive tokens: the block writes together, a run of
+        // side by side - and already as that kernel multiplies them: a bf16 head and the bf16 remainder of
+        // the fp32 value in one word (relative error of the pair 2^-17).  The block's groups hold consecutive tokens: the block writes together, a run of
         // tokens per sample, from the groups' arrays in shared memory.
         const int groups = blockDim.x / LPR;
         long long* group_at = reinterpret_cast<long long*>(group0 + static_cast<size_t>(groups) * (2 * NB8 + 2 * pr.P));
         if (gl == 0) group_at[threadIdx.x / LPR] = static_cast<long long>(m) * pr.P * pr.N + n;
         __syncthreads();                                   // warps with no item at all have left: they count as arrived
-        float* planes = reinterpret_cast<float*>(coef);
+        uint32_t* planes = reinterpret_cast<uint32_t*>(coef);
         const long long plane_elems = pr.N * pr.heads * pr.P;
         const long long block_first = static_cast<long long>(blockIdx.x) * groups;     // item of group 0
         // the threads still here: the warps up to the last one that holds an item
@@ -196,8 +207,8 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
             if (block_first + g >= pr.items) continue;     // a group without an item (its arrays and position are not set)
             const long long at = group_at[g];
             const float* ga = group0 + static_cast<size_t>(g) * (2 * NB8 + 2 * pr.P) + 2 * NB8;     // sa, then sk
-            planes[at + p * pr.N] = ga[pr.P + p];
-            planes[plane_elems + at + p * pr.N] = ga[p];
+            planes[at + p * pr.N] = split_bf16_pair(ga[pr.P + p]);
+            planes[plane_elems + at + p * pr.N] = split_bf16_pair(ga[p]);
         }
     }
 

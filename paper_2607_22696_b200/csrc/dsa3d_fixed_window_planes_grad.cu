@@ -10,10 +10,11 @@
 //   per (tile, head) three sweeps (dQ over K, dK over q, dV over dO), per sweep kt+3 planes:
 //     the plane's rows by TMA into a ring of buffers; every worker thread writes the coefficients of
 //     its output row that fall into this plane into the row of C_plane in shared memory
-//     (128-byte-swizzled K-major), each fp32 coefficient split into a bf16 head and a bf16 remainder
-//     (relative error of the pair 2^-17), as two matrices; two chains of tcgen05.mma (the plane as an
-//     MN-major operand) accumulate  O_sweep += C_plane . X_plane  in TMEM - one accumulator per sweep,
-//     so a sweep's epilogue (TMEM -> bf16 -> global) never holds up the next sweep's products.
+//     (128-byte-swizzled K-major), each fp32 coefficient as a bf16 head and a bf16 remainder (relative
+//     error of the pair 2^-17; the query kernel leaves them split like that), as two matrices; two
+//     chains of tcgen05.mma (the plane as an MN-major operand) accumulate  O_sweep += C_plane . X_plane
+//     in TMEM - one accumulator per sweep, so a sweep's epilogue (TMEM -> bf16 -> global) never holds
+//     up the next sweep's products.
 //   The coefficients a thread needs for a plane are requested one plane ahead, with unconditional
 //   loads from a clamped position (a load under a condition is waited for where it is issued).
 //
@@ -78,7 +79,7 @@ struct __align__(1024) PgSmem {
 template <int D, int KT, int KH, int KW>
 __global__ void __launch_bounds__(kPgThreads, 1)
 fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_q,
-                                const __grid_constant__ CUtensorMap map_do, const float* __restrict__ coef,
+                                const __grid_constant__ CUtensorMap map_do, const uint32_t* __restrict__ coef,
                                 __nv_bfloat16* __restrict__ dq, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
                                 int T, int H, int W, int heads, int tiles_x, int tiles_y, int total, int* timeout_flag) {
     using S = PgShape<D, KT, KH, KW>;
@@ -211,10 +212,15 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
         }
     } else {
         // ==================================================================== workers
-        const int lt = warp & 3, sub = warp >> 2;                     // output plane of the tile; which thread of the row's four
+        // A worker thread has two places.  Writing coefficients it is thread `sub` of the four that share the
+        // output row (lt, lane); the four warps of one lt sit on four different schedulers, so the planes a
+        // row group is busy in load all of them.  Reading an accumulator it can only reach the TMEM lanes of
+        // its warp's quarter (warp % 4): there it takes 32 channels (part warp / 4) of row (warp % 4, lane).
+        const int lt = warp >> 2, sub = warp & 3;                     // output plane of the tile; which thread of the row's four
+        const int lt_acc = warp & 3, part_acc = warp >> 2;
         const int ly = lane >> 3, lx = lane & 7;
         const int r = lt * 32 + lane;                                 // output row of the tile = TMEM lane
-        const uint32_t lane_base = static_cast<uint32_t>(lt * 32) << 16;
+        const uint32_t lane_base = static_cast<uint32_t>(lt_acc * 32) << 16;
         const uint32_t row_off = static_cast<uint32_t>(r) * 128u, rx = static_cast<uint32_t>(r & 7);
         const int v0 = (sub * KH) / kPgSplit, nv = ((sub + 1) * KH) / kPgSplit - v0;    // this thread's kernel rows (warp-uniform)
         // The cells of one kernel row are KW neighbouring columns of the output's row of C: they are written as
@@ -255,8 +261,8 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
             if (((geo >> 24) & 7u) + KW > 8u) *reinterpret_cast<uint4*>(dst + (((geo >> 12) & 0xfffu) << 4)) = make_uint4(c[4], c[5], c[6], c[7]);
         };
         const int n_step = T * H * W;                                 // tokens: the step from one sample's plane to the next
-        const float* plane_ck = coef;                                 // [head][sample][token]
-        const float* plane_cv = coef + static_cast<long long>(heads) * P * n_step;
+        const uint32_t* plane_ck = coef;                              // [head][sample][token], a word = bf16 head | bf16 remainder << 16
+        const uint32_t* plane_cv = coef + static_cast<long long>(heads) * P * n_step;
         // Step q of this thread = (tile, sweep, kernel plane u) in the order they come: the coefficients of
         // the row's cells (this thread's kernel rows, every column) in that plane.  What depends on the
         // tile alone is worked out at the tile's first step: positions inside a coefficient plane (they
@@ -264,7 +270,7 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
         const int steps = my_tiles * 3 * KT;
         int g_a0 = 0, g_a1 = 0;
         uint32_t g_tmask = 0u, g_ymask = 0u, g_xmask = 0u, g_own = 0u;
-        auto fetch = [&](int q, float (&wv)[CELLS], uint32_t& dead) {
+        auto fetch = [&](int q, uint32_t (&wv)[CELLS], uint32_t& dead) {
             const int ti = q / (3 * KT), rem = q - ti * (3 * KT), sweep = rem / KT, u = rem - sweep * KT;
             if (rem == 0) {
                 int m, t0, y0, x0;
@@ -300,7 +306,7 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
                     for (int vi = 0; vi < VH; ++vi) if ((g_ymask >> vi) & 1u) alive |= g_xmask << (vi * KW);
                 }
             }
-            const float* plane = sweep == 2 ? plane_cv : plane_ck;
+            const uint32_t* plane = sweep == 2 ? plane_cv : plane_ck;
 #pragma unroll
             for (int i = 0; i < CELLS; ++i) {
                 const int vi = i / KW, ww = i - vi * KW;
@@ -309,10 +315,10 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
             }
             dead = ~alive;
         };
-        float wnext[CELLS];
+        uint32_t wnext[CELLS];
         uint32_t dnext = 0u;
 #pragma unroll
-        for (int i = 0; i < CELLS; ++i) wnext[i] = 0.0f;
+        for (int i = 0; i < CELLS; ++i) wnext[i] = 0u;
         int q = 0;                                                    // the step whose coefficients wnext holds
         if (steps > 0) fetch(0, wnext, dnext);
         int buf = 0, clear_left = 0;                                  // coefficient buffer of the next unit; units still to clear
@@ -322,17 +328,17 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
         auto epilogue = [&](int it, int sweep) {
             int m, t0, y0, x0;
             locate(it, m, t0, y0, x0);
-            const int ot = t0 + lt, oy = y0 + ly, ox = x0 + lx;
+            const int ot = t0 + lt_acc, oy = y0 + ly, ox = x0 + lx;
             const bool in_grid = ot < T && oy < H && ox < W;
             const long long n = (static_cast<long long>(ot) * H + oy) * W + ox;
             wait(&s.bar_o[sweep], static_cast<uint32_t>(it & 1), 55);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (sub * 32 < D) {
+            if (part_acc * 32 < D) {
                 __nv_bfloat16* out = sweep == 0 ? dq : sweep == 1 ? dk : dv;
                 uint32_t regs[32];
-                tmem_load_32(tmem + lane_base + static_cast<uint32_t>(sweep * D + sub * 32), regs);
+                tmem_load_32(tmem + lane_base + static_cast<uint32_t>(sweep * D + part_acc * 32), regs);
                 if (in_grid && !*abort_flag) {
-                    uint4* dst = reinterpret_cast<uint4*>(out + (n * heads + m) * D + sub * 32);
+                    uint4* dst = reinterpret_cast<uint4*>(out + (n * heads + m) * D + part_acc * 32);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         uint32_t o[4];
@@ -368,18 +374,16 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
                     uint32_t head[4];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        // cells 2j and 2j + 1 of the kernel row (0 beyond KW, for a query that does not exist, and when clearing)
-                        float p[2];
+                        // cells 2j and 2j + 1 of the kernel row (0 beyond KW, for a query that does not exist, and when
+                        // clearing): their heads side by side in one word, their remainders in another
+                        uint32_t w[2];
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
                             const int ww = 2 * j + e, i = vi * KW + ww;
-                            p[e] = (ww < KW && mine && !((dnext >> (ww < KW ? i : 0)) & 1u)) ? wnext[ww < KW ? i : 0] : 0.0f;
+                            w[e] = (ww < KW && mine && !((dnext >> (ww < KW ? i : 0)) & 1u)) ? wnext[ww < KW ? i : 0] : 0u;
                         }
-                        const __nv_bfloat162 hd = __floats2bfloat162_rn(p[0], p[1]);
-                        head[j] = *reinterpret_cast<const uint32_t*>(&hd);
-                        const __nv_bfloat162 rm = __floats2bfloat162_rn(p[0] - __uint_as_float(head[j] << 16),
-                                                                        p[1] - __uint_as_float(head[j] & 0xffff0000u));
-                        rest[vi][j] = *reinterpret_cast<const uint32_t*>(&rm);
+                        head[j] = __byte_perm(w[0], w[1], 0x5410);
+                        rest[vi][j] = __byte_perm(w[0], w[1], 0x7632);
                     }
                     store_row(dst, row_geo[vi], head);
                 }
@@ -432,7 +436,7 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
 }
 
 template <int D, int KT, int KH, int KW>
-cudaError_t launch_planes_grad(const void* q, const void* k, const void* dout, const float* coef, void* dq, void* dk, void* dv,
+cudaError_t launch_planes_grad(const void* q, const void* k, const void* dout, const uint32_t* coef, void* dq, void* dk, void* dv,
                                const Problem& pr, int* flag, cudaStream_t stream, bool* unsupported) {
     using S = PgShape<D, KT, KH, KW>;
     const unsigned long long d = static_cast<unsigned long long>(pr.d), hd = static_cast<unsigned long long>(pr.heads);
@@ -477,13 +481,14 @@ bool fixed_window_planes_grad_covers(const Problem& pr, bool bf16) {
     return pr.kt == 3 && ((pr.kh == 5 && pr.kw == 5) || (pr.kh == 7 && pr.kw == 7));
 }
 
-bool try_fixed_window_planes_grad(const void* q, const void* k, const void* dout, const float* coef, void* dq, void* dk, void* dv,
+bool try_fixed_window_planes_grad(const void* q, const void* k, const void* dout, const float* coef_planes, void* dq, void* dk, void* dv,
                                   const Problem& pr, cudaStream_t stream, cudaError_t* err) {
     *err = cudaSuccess;
     if (!fixed_window_planes_grad_covers(pr, true)) return false;
     int* flag = timeout_flag_device_address();
     if (!flag) return false;
     bool unsupported = false;
+    const uint32_t* coef = reinterpret_cast<const uint32_t*>(coef_planes);
     const bool w355 = pr.kh == 5;
     if (pr.d == 128)
         *err = w355 ? launch_planes_grad<128, 3, 5, 5>(q, k, dout, coef, dq, dk, dv, pr, flag, stream, &unsupported)
