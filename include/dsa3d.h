@@ -54,7 +54,9 @@
  *                                  binning (the gather kernel then lists every sample per key block); slower
  *                                  so far; also changes dsa3d_backward_workspace_bytes; a
  *                                  non-finite q or dO row then reaches every key whose block it lies near
- *   DSA3D_NO_TENSOR_FIXED_WINDOW   dsa3d_forward_fixed_window uses the general kernel
+ *   DSA3D_NO_TENSOR_FIXED_WINDOW   dsa3d_forward_fixed_window and dsa3d_forward_bounded_offsets use the general
+ *                                  kernel; dsa3d_backward_fixed_window uses its per-row CUDA-core kernels only
+ *                                  (no dot-product tables, no tile kernels)
  *   DSA3D_GEMM_ONE_CTA             dsa3d_offsets_linear_forward: one CTA per tile instead of a pair
  *   DSA3D_GEMM_PLAIN_STORES        its epilogue stores from registers instead of by TMA
  *   DSA3D_CONV_GENERAL             dsa3d_dwconv3d_*: the kernel for any size also for 3x3x3
@@ -407,12 +409,15 @@ int dsa3d_forward_bounded_offsets(const void* q, const void* k, const void* v, c
  * queries around it, so they are gathered instead of scattered: no atomics, results bitwise
  * deterministic, dk/dv written once in `dtype`.  `lse` is the forward's.  `workspace`:
  * dsa3d_backward_fixed_window_workspace_bytes(...) bytes (two fp32 coefficients per sample, plus,
- * for bf16 with d = 64 or 128 and windows (3,3,3) or (2,2,2), a table of the dot products q.K_j and
- * dO.V_j of every query's window and its +1 neighbours, which a tcgen05 kernel fills from dense
- * Q.K^T and dO.V^T tiles so that the gradient kernel gathers no K/V rows for them), 16-byte aligned,
- * contents undefined afterwards.  All supported dtypes, head sizes and windows.  The environment
- * variable DSA3D_NO_TENSOR_FIXED_WINDOW switches the table kernel off.  Bounded waits as in
- * dsa3d_offsets_linear_forward (dsa3d_device_timeout_flag).
+ * for bf16 with d = 64 or 128 and windows (2,2,2), (3,3,3), (3,5,5) or (3,7,7), a table of the dot
+ * products q.K_j and dO.V_j of every query's window and its +1 neighbours, which a tcgen05 kernel
+ * fills from dense Q.K^T and dO.V^T tiles so that the gradient kernel gathers no K/V rows for them),
+ * 16-byte aligned, contents undefined afterwards.  All supported dtypes, head sizes and windows.
+ * For those bf16 shapes dq, dk and dv are then formed per tile of 4 x 4 x 8 outputs: from halo
+ * regions in shared memory for the two small windows, as plane-by-plane tcgen05 products for the
+ * two larger ones (coefficients as a bf16 head plus a bf16 remainder, relative error 2^-17).  The
+ * environment variable DSA3D_NO_TENSOR_FIXED_WINDOW switches the table and tile kernels off.
+ * Bounded waits as in dsa3d_offsets_linear_forward (dsa3d_device_timeout_flag).
  */
 int dsa3d_backward_fixed_window(const void* q, const void* k, const void* v, const float* lse, const void* dout, int T,
                                 int H, int W, int heads, int d, const int window[3], void* dq, void* dk, void* dv,
