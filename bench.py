@@ -402,6 +402,8 @@ def run_ours(args, wl):
     ws_bytes = binding.dsa3d_backward_workspace_bytes(*dims, wl.window, wl.dtype)
     if wl.offsets == "zero" and wl.backward:        # the fixed-window backward keeps its dot-product tables there
         ws_bytes = max(ws_bytes, binding.dsa3d_backward_fixed_window_workspace_bytes(*dims, wl.window, wl.dtype))
+    if wl.offsets == "small" and wl.backward:       # tables and coefficient planes of the bounded-offsets backward
+        ws_bytes = max(ws_bytes, binding.dsa3d_backward_bounded_offsets_workspace_bytes(*dims, wl.window, wl.dtype))
     b = {"out": torch.empty_like(t["q"]),
          "lse": torch.empty(wl.T, wl.H, wl.W, wl.heads, dtype=torch.float32, device=dev),
          "dq": torch.empty_like(t["q"]), "dk": torch.empty_like(t["q"]), "dv": torch.empty_like(t["q"]),
@@ -412,8 +414,8 @@ def run_ours(args, wl):
     # the entry point that takes no offsets tensor (tensor-core tile kernel where the shape
     # allows); the backward is the general one on the zero offsets tensor.
     fixed_window = wl.offsets == "zero" and not args.no_fixed_window
-    # offsets below 1 in size: the forward entry point that decides on the device between the tensor-core
-    # tile kernel and the general kernel; the backward is the general one
+    # offsets below 1 in size: the entry points that decide on the device between the tensor-core tile
+    # kernels and the general kernels
     bounded = wl.offsets == "small" and not args.no_fixed_window
 
     def step():
@@ -426,6 +428,9 @@ def run_ours(args, wl):
         if wl.backward and fixed_window:
             binding.dsa3d_backward_fixed_window(t["q"], t["k"], t["v"], b["lse"], t["dout"], *dims, wl.window,
                                                 b["dq"], b["dk"], b["dv"], b["doff"], b["ws"])
+        elif wl.backward and bounded:
+            binding.dsa3d_backward_bounded_offsets(t["q"], t["k"], t["v"], t["offsets"], b["lse"], t["dout"], *dims,
+                                                   wl.window, b["dq"], b["dk"], b["dv"], b["doff"], b["ws"])
         elif wl.backward:
             binding.dsa3d_backward(t["q"], t["k"], t["v"], t["offsets"], b["lse"], t["dout"], *dims,
                                    wl.window, b["dq"], b["dk"], b["dv"], b["doff"], b["ws"])
@@ -568,7 +573,8 @@ def run_ours(args, wl):
                    "offsets": f"{wl.offsets} sigma={wl.sigma}", "batch_per_gpu": 1,
                    "forward_entry": ("dsa3d_forward_fixed_window" if fixed_window else
                                      "dsa3d_forward_bounded_offsets" if bounded else "dsa3d_forward"),
-                   "backward_entry": ("dsa3d_backward_fixed_window" if fixed_window else "dsa3d_backward")
+                   "backward_entry": ("dsa3d_backward_fixed_window" if fixed_window else
+                                      "dsa3d_backward_bounded_offsets" if bounded else "dsa3d_backward")
                                      if wl.backward else None,
                    "parallelism": (f"one video, heads sharded over {world} ranks (heads of rank 0: {wl.heads})"
                                    if sharded else f"independent videos x{world}"),

@@ -55,7 +55,8 @@
  *                                  so far; also changes dsa3d_backward_workspace_bytes; a
  *                                  non-finite q or dO row then reaches every key whose block it lies near
  *   DSA3D_NO_TENSOR_FIXED_WINDOW   dsa3d_forward_fixed_window and dsa3d_forward_bounded_offsets use the general
- *                                  kernel; dsa3d_backward_fixed_window uses its per-row CUDA-core kernels only
+ *                                  kernel, dsa3d_backward_bounded_offsets the kernels of dsa3d_backward;
+ *                                  dsa3d_backward_fixed_window uses its per-row CUDA-core kernels only
  *                                  (no dot-product tables, no tile kernels)
  *   DSA3D_GEMM_ONE_CTA             dsa3d_offsets_linear_forward: one CTA per tile instead of a pair
  *   DSA3D_GEMM_PLAIN_STORES        its epilogue stores from registers instead of by TMA
@@ -396,10 +397,35 @@ int dsa3d_forward_fixed_window(const void* q, const void* k, const void* v, int 
  * for any offsets; the decision is taken on the device, the call stays asynchronous.  Calls that are in
  * flight at the same time each use their own gate word (out of 1024).  The environment variable
  * DSA3D_NO_TENSOR_FIXED_WINDOW forces the general kernel.  Bounded waits as in
- * dsa3d_offsets_linear_forward (dsa3d_device_timeout_flag).  The backward of such a call is dsa3d_backward.
+ * dsa3d_offsets_linear_forward (dsa3d_device_timeout_flag).  The backward of such a call is
+ * dsa3d_backward_bounded_offsets (or dsa3d_backward).
  */
 int dsa3d_forward_bounded_offsets(const void* q, const void* k, const void* v, const float* offsets, int T, int H, int W,
                                   int heads, int d, const int window[3], void* out, float* lse, int dtype, void* stream);
+
+/*
+ * dsa3d_backward_bounded_offsets: dsa3d_backward for the same callers.  Same arguments, same dq, dk, dv and
+ * doffsets (up to fp32 summation order; the coefficients of dq, dk and dv enter their products as a bf16
+ * head plus a bf16 remainder, relative error 2^-17).  The offsets tensor is checked on the device as in
+ * dsa3d_forward_bounded_offsets.  If every component is finite and below 1 in size (bf16, d = 64 or 128,
+ * window (3,3,3)) no row is gathered or scattered one by one: a tcgen05 kernel leaves, per (query, head),
+ * the dot products q.K_j and dO.V_j of the 6 x 6 x 6 grid positions from query - 2; a second kernel forms
+ * every sample's logit, dO.V and their derivatives as trilinear combinations of eight of them (cell and
+ * fractions exactly as dsa3d_backward forms them), alpha from `lse`, delta, dS, doffsets, and sums the
+ * coefficients of the samples' corners per grid position into a 5 x 5 x 5 box; dq, dk and dv are then the
+ * sums of a fixed (5,5,5) window with those coefficients, plane-by-plane tcgen05 products as in
+ * dsa3d_backward_fixed_window.  Otherwise the kernels of dsa3d_backward run (they are queued behind the
+ * others and do nothing when the check passed), so the call is correct for any offsets and stays
+ * asynchronous.  dk and dv of the tile route are written once in `dtype` (no atomics, bitwise deterministic).
+ * `workspace`: dsa3d_backward_bounded_offsets_workspace_bytes(...) bytes, 16-byte aligned, contents undefined
+ * afterwards.  Other shapes and dtypes, and the switches DSA3D_NO_TENSOR_FIXED_WINDOW and DSA3D_KEY_BLOCKS=1,
+ * make it dsa3d_backward.  Bounded waits as in dsa3d_offsets_linear_forward (dsa3d_device_timeout_flag).
+ */
+int dsa3d_backward_bounded_offsets(const void* q, const void* k, const void* v, const float* offsets, const float* lse,
+                                   const void* dout, int T, int H, int W, int heads, int d, const int window[3], void* dq,
+                                   void* dk, void* dv, float* doffsets, void* workspace, size_t workspace_bytes, int dtype,
+                                   void* stream);
+size_t dsa3d_backward_bounded_offsets_workspace_bytes(int T, int H, int W, int heads, int d, const int window[3], int dtype);
 
 /*
  * dsa3d_backward_fixed_window: backward of the operator with every offset equal to zero, without

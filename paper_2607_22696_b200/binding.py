@@ -62,6 +62,10 @@ def _declare(lib) -> None:
     lib.dsa3d_backward.argtypes = [p, p, p, p, p, p, i, i, i, i, i, win, p, p, p, p, p, sz, i, p]
     lib.dsa3d_backward_workspace_bytes.restype = sz
     lib.dsa3d_backward_workspace_bytes.argtypes = [i, i, i, i, i, win, i]
+    lib.dsa3d_backward_bounded_offsets.restype = i
+    lib.dsa3d_backward_bounded_offsets.argtypes = [p, p, p, p, p, p, i, i, i, i, i, win, p, p, p, p, p, sz, i, p]
+    lib.dsa3d_backward_bounded_offsets_workspace_bytes.restype = sz
+    lib.dsa3d_backward_bounded_offsets_workspace_bytes.argtypes = [i, i, i, i, i, win, i]
     lib.dsa3d_step_host.restype = i
     lib.dsa3d_step_host.argtypes = [p, p, p, p, p, i, i, i, i, i, win, p, p, p, p, p, p, p, sz, i, p]
     lib.dsa3d_step_host_pipelined.restype = i
@@ -357,6 +361,31 @@ def dsa3d_backward(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, d
     if workspace_bytes is None:
         workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(lib.dsa3d_backward(
+        _ptr(q, "q", n * d), _ptr(k, "k", n * d), _ptr(v, "v", n * d),
+        _ptr(offsets, "offsets", n * P * 3, torch.float32), _ptr(lse, "lse", n, torch.float32),
+        _ptr(dout, "dout", n * d), T, H, W, heads, d, _window(window),
+        _ptr(dq, "dq", n * d), _ptr(dk, "dk", n * d), _ptr(dv, "dv", n * d),
+        _ptr(doffsets, "doffsets", n * P * 3, torch.float32),
+        _ptr(workspace, "workspace"), int(workspace_bytes), code, _stream(stream)))
+
+
+def dsa3d_backward_bounded_offsets_workspace_bytes(T, H, W, heads, d, window, dtype) -> int:
+    code = _DTYPES[dtype] if isinstance(dtype, torch.dtype) else int(dtype)
+    return int(load().dsa3d_backward_bounded_offsets_workspace_bytes(T, H, W, heads, d, _window(window), code))
+
+
+def dsa3d_backward_bounded_offsets(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets,
+                                   workspace=None, workspace_bytes=None, dtype=None, stream=None) -> None:
+    """dsa3d_backward for offsets that are small perturbations of the window: tensor-core tile kernels when
+    every |offset| < 1 (decided on the device), the general kernels otherwise; see include/dsa3d.h."""
+    lib = load()
+    dt = q.dtype if dtype is None else dtype
+    code = _DTYPES[dt] if isinstance(dt, torch.dtype) else int(dt)
+    n = T * H * W * heads
+    P = int(window[0]) * int(window[1]) * int(window[2])
+    if workspace_bytes is None:
+        workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.dsa3d_backward_bounded_offsets(
         _ptr(q, "q", n * d), _ptr(k, "k", n * d), _ptr(v, "v", n * d),
         _ptr(offsets, "offsets", n * P * 3, torch.float32), _ptr(lse, "lse", n, torch.float32),
         _ptr(dout, "dout", n * d), T, H, W, heads, d, _window(window),

@@ -12,7 +12,7 @@ LIB_DEBUG = os.path.join(HERE, "libdsa3d_debug.so")     # the checked build (-DD
 SOURCES = ["dsa3d_api.cu", "dsa3d_forward.cu", "dsa3d_backward.cu", "dsa3d_backward_blocks.cu", "dsa3d_noalloc.cu", "dsa3d_probes.cu",
            "dsa3d_producer.cu", "dsa3d_fixed_window.cu", "dsa3d_fixed_window_planes.cu", "dsa3d_fixed_window_tables.cu",
            "dsa3d_fixed_window_backward.cu", "dsa3d_fixed_window_tile_grad.cu",
-           "dsa3d_fixed_window_planes_grad.cu"]
+           "dsa3d_fixed_window_planes_grad.cu", "dsa3d_bounded_offsets_backward.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC"]
 

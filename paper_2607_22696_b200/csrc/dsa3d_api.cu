@@ -65,6 +65,7 @@ int make_problem(int T, int H, int W, int heads, int d, const int* window, int d
     pr.blk_count = nullptr;
     pr.blk_list = nullptr;
     pr.blk_cap = 0;
+    pr.gate = nullptr;
     pr.debug_word = debug_word_address();
     return DSA3D_OK;
 }
@@ -225,6 +226,55 @@ int dsa3d_forward_bounded_offsets(const void* q, const void* k, const void* v, c
     return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
 }
 
+namespace {
+bool bounded_backward_tiled(const dsa3d::Problem& pr, int dtype) {
+    const char* kb = std::getenv("DSA3D_KEY_BLOCKS");
+    return dtype == DSA3D_BF16 && dsa3d::bounded_offsets_backward_covers(pr, true) &&
+           !std::getenv("DSA3D_NO_TENSOR_FIXED_WINDOW") && !(kb && kb[0] == '1');
+}
+}  // namespace
+
+size_t dsa3d_backward_bounded_offsets_workspace_bytes(int T, int H, int W, int heads, int d, const int window[3], int dtype) {
+    const size_t general = dsa3d_backward_workspace_bytes(T, H, W, heads, d, window, dtype);
+    dsa3d::Problem pr;
+    if (make_problem(T, H, W, heads, d, window, dtype, pr) != DSA3D_OK) return 0;
+    if (!bounded_backward_tiled(pr, dtype)) return general;
+    const size_t tiled = dsa3d::bounded_offsets_backward_bytes(pr);      // the two routes never hold data at the same time
+    return tiled > general ? tiled : general;
+}
+
+int dsa3d_backward_bounded_offsets(const void* q, const void* k, const void* v, const float* offsets, const float* lse,
+                                   const void* dout, int T, int H, int W, int heads, int d, const int window[3], void* dq,
+                                   void* dk, void* dv, float* doffsets, void* workspace, size_t workspace_bytes, int dtype,
+                                   void* stream) {
+    if (!q || !k || !v || !offsets || !lse || !dout || !dq || !dk || !dv || !doffsets) return DSA3D_ERR_NULL_POINTER;
+    dsa3d::Problem pr;
+    const int rc = make_problem(T, H, W, heads, d, window, dtype, pr);
+    if (rc != DSA3D_OK) return rc;
+    if (!bounded_backward_tiled(pr, dtype))
+        return dsa3d::backward_impl(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets, workspace,
+                                    workspace_bytes, dtype, stream, true);
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(offsets) || !aligned16(lse) || !aligned16(dout) ||
+        !aligned16(dq) || !aligned16(dk) || !aligned16(dv) || !aligned16(doffsets))
+        return DSA3D_ERR_MISALIGNED;
+    if (!workspace || workspace_bytes < dsa3d_backward_bounded_offsets_workspace_bytes(T, H, W, heads, d, window, dtype))
+        return DSA3D_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return DSA3D_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    void* words = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&words, g_gate_words);
+    if (e != cudaSuccess) return cuda_failed(e);
+    int* gate = static_cast<int*>(words) + g_next_gate.fetch_add(1u) % kGateWords;
+    e = dsa3d::launch_offsets_bound_check(offsets, pr.items * pr.P * 3, gate, st);
+    if (e != cudaSuccess) return cuda_failed(e);
+    // the three tile kernels run if the check left 0 in the gate, the general kernels behind them if it left 1
+    const bool tiled = dsa3d::try_bounded_offsets_backward(q, k, v, offsets, lse, dout, dq, dk, dv, doffsets, workspace, gate,
+                                                          pr, st, &e);
+    if (tiled && e != cudaSuccess) return cuda_failed(e);
+    return dsa3d::backward_impl(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets, workspace,
+                                workspace_bytes, dtype, stream, true, tiled ? gate : nullptr);
+}
+
 size_t dsa3d_backward_fixed_window_workspace_bytes(int T, int H, int W, int heads, int d, const int window[3],
                                                    int dtype) {
     dsa3d::Problem pr;
@@ -348,7 +398,8 @@ int backward_plan(int T, int H, int W, int heads, int d, const int* window, int 
 int backward_clear(const BackwardPlan& plan, cudaStream_t stream) {
     cudaError_t e;
     if (plan.bf16) {
-        e = cudaMemsetAsync(plan.workspace, 0, plan.ws.acc_bytes, stream);
+        e = plan.pr.gate ? dsa3d::launch_gated_clear(plan.workspace, plan.ws.acc_bytes, plan.pr.gate, stream)
+                         : cudaMemsetAsync(plan.workspace, 0, plan.ws.acc_bytes, stream);
         if (e != cudaSuccess) return cuda_failed(e);
     } else {
         e = cudaMemsetAsync(plan.acc_dk, 0, plan.count * sizeof(float), stream);
@@ -410,9 +461,9 @@ int backward_frames(const BackwardPlan& plan, const void* q, const void* k, cons
 // Accumulators -> dk, dv (bf16 storage only; fp32 storage accumulated in place).
 int backward_finish(const BackwardPlan& plan, void* dk, void* dv, cudaStream_t stream) {
     if (!plan.bf16) return DSA3D_OK;
-    cudaError_t e = dsa3d::launch_convert_bf16(plan.acc_dk, dk, static_cast<long long>(plan.count), stream);
+    cudaError_t e = dsa3d::launch_convert_bf16(plan.acc_dk, dk, static_cast<long long>(plan.count), stream, plan.pr.gate);
     if (e != cudaSuccess) return cuda_failed(e);
-    e = dsa3d::launch_convert_bf16(plan.acc_dv, dv, static_cast<long long>(plan.count), stream);
+    e = dsa3d::launch_convert_bf16(plan.acc_dv, dv, static_cast<long long>(plan.count), stream, plan.pr.gate);
     if (e != cudaSuccess) return cuda_failed(e);
     return DSA3D_OK;
 }
@@ -433,7 +484,7 @@ int forward_frames(const dsa3d::Problem& full, const void* q, const void* k, con
 int dsa3d::backward_impl(const void* q, const void* k, const void* v, const float* offsets, const float* lse,
                          const void* dout, int T, int H, int W, int heads, int d, const int window[3],
                          void* dq, void* dk, void* dv, float* doffsets, void* workspace,
-                         size_t workspace_bytes, int dtype, void* stream_, bool tiled) {
+                         size_t workspace_bytes, int dtype, void* stream_, bool tiled, const int* gate) {
     if (!q || !k || !v || !offsets || !lse || !dout || !dq || !dk || !dv || !doffsets)
         return DSA3D_ERR_NULL_POINTER;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(offsets) || !aligned16(lse) ||
@@ -442,6 +493,7 @@ int dsa3d::backward_impl(const void* q, const void* k, const void* v, const floa
     BackwardPlan plan;
     int rc = backward_plan(T, H, W, heads, d, window, dtype, tiled, dk, dv, workspace, workspace_bytes, plan);
     if (rc != DSA3D_OK) return rc;
+    plan.pr.gate = gate;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     rc = backward_clear(plan, stream);
     if (rc != DSA3D_OK) return rc;

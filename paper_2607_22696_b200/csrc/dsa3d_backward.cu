@@ -61,6 +61,7 @@ backward_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
     constexpr int VEC = E::VEC;
     constexpr int LPR = D / VEC;
     extern __shared__ float smem[];
+    if (gated_off(pr)) return;
     const int lane = threadIdx.x & 31;
     const int gl = lane & (LPR - 1);
     constexpr unsigned gmask = kFullMask;
@@ -311,6 +312,7 @@ scatter_tile_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     constexpr int kPairBytes = 2 * VPR * 16;         // one query's q row followed by its dO row
     constexpr unsigned kFull = 0xffffffffu;
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    if (gated_off(pr)) return;
     const int TQ = pr.tile_t * pr.tile_y * pr.tile_x;
     const int et = pr.tile_t + 2 * pr.halo, ey = pr.tile_y + 2 * pr.halo, ex = pr.tile_x + 2 * pr.halo;
     const int NB = et * ey * ex;
@@ -596,7 +598,8 @@ cudaError_t launch_scatter_tiles(const void* q, const void* dout, const float* o
 }
 
 __global__ void __launch_bounds__(256)
-convert_bf16_kernel(const float4* __restrict__ acc, uint2* __restrict__ dst, long long count4) {
+convert_bf16_kernel(const float4* __restrict__ acc, uint2* __restrict__ dst, long long count4, const int* __restrict__ gate) {
+    if (gate != nullptr && *gate == 0) return;      // the tile kernels of a bounded-offsets backward wrote dk and dv
     const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
     for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < count4; i += stride) {
         const float4 a = acc[i];
@@ -606,13 +609,32 @@ convert_bf16_kernel(const float4* __restrict__ acc, uint2* __restrict__ dst, lon
     }
 }
 
-cudaError_t launch_convert_bf16(const float* acc, void* dst, long long count, cudaStream_t stream) {
+// Zeroes `count4` 16-byte pieces unless *gate is 0 (a gated backward whose tile kernels took the call needs
+// no accumulators; an unconditional memset would cost it their size in HBM writes).
+__global__ void __launch_bounds__(256)
+gated_clear_kernel(uint4* __restrict__ dst, long long count4, const int* __restrict__ gate) {
+    if (*gate == 0) return;
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < count4; i += stride)
+        dst[i] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+cudaError_t launch_gated_clear(void* dst, size_t bytes, const int* gate, cudaStream_t stream) {
+    const long long count4 = static_cast<long long>(bytes / 16);     // the accumulators are whole rows of d floats
+    long long blocks = (count4 + 255) / 256;
+    if (blocks > 148LL * 16) blocks = 148LL * 16;
+    if (blocks < 1) blocks = 1;
+    gated_clear_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(static_cast<uint4*>(dst), count4, gate);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_convert_bf16(const float* acc, void* dst, long long count, cudaStream_t stream, const int* gate) {
     const long long count4 = count / 4;      // d is a multiple of 32, so count is a multiple of 4
     long long blocks = (count4 + 255) / 256;
     if (blocks > 148LL * 16) blocks = 148LL * 16;
     if (blocks < 1) blocks = 1;
     convert_bf16_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
-        reinterpret_cast<const float4*>(acc), reinterpret_cast<uint2*>(dst), count4);
+        reinterpret_cast<const float4*>(acc), reinterpret_cast<uint2*>(dst), count4, gate);
     return cudaGetLastError();
 }
 

@@ -42,7 +42,13 @@ struct Problem {
     // Checked build (-DDSA3D_DEBUG) only: device word that receives the first out-of-range index a
     // kernel was about to use (0 = none); NULL otherwise.
     unsigned long long* debug_word;
+    // Backward behind a check of the offsets (dsa3d_backward_bounded_offsets): the general kernels run only
+    // if this device word is non-zero (the check found offsets its tile kernels do not cover); NULL: always.
+    const int* gate;
 };
+
+// True when a gated general kernel has nothing to do (see Problem::gate).
+__device__ __forceinline__ bool gated_off(const Problem& pr) { return pr.gate != nullptr && *pr.gate == 0; }
 
 // Checked build: every row a gather reads and every row or bin a scatter writes is tested against its
 // tensor's extent first; a violation is recorded (first one wins: code in the top 8 bits, the offending

@@ -81,7 +81,8 @@ __global__ void __launch_bounds__(kPgThreads, 1)
 fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_q,
                                 const __grid_constant__ CUtensorMap map_do, const uint32_t* __restrict__ coef,
                                 __nv_bfloat16* __restrict__ dq, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
-                                int T, int H, int W, int heads, int tiles_x, int tiles_y, int total, int* timeout_flag) {
+                                int T, int H, int W, int heads, int tiles_x, int tiles_y, int total, int* timeout_flag,
+                                const int* __restrict__ gate) {
     using S = PgShape<D, KT, KH, KW>;
     constexpr int NH = S::NH, RT = S::RT, RX = S::RX, PS = S::PS, PSP = S::PSP, VH = S::VH, NS = S::NS, NC = S::NC, P = S::P;
     constexpr int JOBS = 3 * RT;                                      // plane loads per tile
@@ -139,7 +140,9 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
         y0 = (tile % tiles_y) * kPgTY;
         t0 = (tile / tiles_y) * kPgTT;
     };
-    const int my_tiles = static_cast<int>(blockIdx.x) < total
+    // behind a check of learned offsets: nothing to do unless the check left 0 in *gate
+    const bool open = gate == nullptr || *gate == 0;
+    const int my_tiles = open && static_cast<int>(blockIdx.x) < total
                              ? (total - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x) : 0;
 
     if (warp == kPgWorkers / 32) {
@@ -437,7 +440,7 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
 
 template <int D, int KT, int KH, int KW>
 cudaError_t launch_planes_grad(const void* q, const void* k, const void* dout, const uint32_t* coef, void* dq, void* dk, void* dv,
-                               const Problem& pr, int* flag, cudaStream_t stream, bool* unsupported) {
+                               const Problem& pr, int* flag, cudaStream_t stream, bool* unsupported, const int* gate = nullptr) {
     using S = PgShape<D, KT, KH, KW>;
     const unsigned long long d = static_cast<unsigned long long>(pr.d), hd = static_cast<unsigned long long>(pr.heads);
     const unsigned long long dims[5] = {d, hd, static_cast<unsigned long long>(pr.W), static_cast<unsigned long long>(pr.H),
@@ -454,7 +457,7 @@ cudaError_t launch_planes_grad(const void* q, const void* k, const void* dout, c
     const int tiles_x = (pr.W + kPgTX - 1) / kPgTX, tiles_y = (pr.H + kPgTY - 1) / kPgTY, tiles_t = (pr.T + kPgTT - 1) / kPgTT;
     const long long total = static_cast<long long>(tiles_x) * tiles_y * tiles_t * pr.heads;
     // the kernel counts planes, and positions inside a coefficient plane, in 32 bits
-    if (total * 3 * S::RT >= (1LL << 31) || pr.N * pr.heads * pr.P >= (1LL << 31)) {
+    if (total * 3 * S::RT >= (1LL << 31) || pr.N * pr.heads * S::P >= (1LL << 31)) {
         *unsupported = true;
         return cudaSuccess;
     }
@@ -470,7 +473,7 @@ cudaError_t launch_planes_grad(const void* q, const void* k, const void* dout, c
     const unsigned grid = static_cast<unsigned>(total < sms ? total : sms);     // persistent: one CTA per SM
     kern<<<grid, kPgThreads, smem, stream>>>(mk, mq, mdo, coef, static_cast<__nv_bfloat16*>(dq), static_cast<__nv_bfloat16*>(dk),
                                              static_cast<__nv_bfloat16*>(dv), pr.T, pr.H, pr.W, pr.heads, tiles_x, tiles_y,
-                                             static_cast<int>(total), flag);
+                                             static_cast<int>(total), flag, gate);
     return cudaGetLastError();
 }
 
@@ -496,6 +499,23 @@ bool try_fixed_window_planes_grad(const void* q, const void* k, const void* dout
     else
         *err = w355 ? launch_planes_grad<64, 3, 5, 5>(q, k, dout, coef, dq, dk, dv, pr, flag, stream, &unsupported)
                     : launch_planes_grad<64, 3, 7, 7>(q, k, dout, coef, dq, dk, dv, pr, flag, stream, &unsupported);
+    return !unsupported;
+}
+
+// Learned offsets below 1 in size, window (3,3,3): the coefficients of a query's samples, summed per grid
+// position, fill the box of 5 x 5 x 5 positions around the query; dQ, dK and dV are then the sums of a
+// fixed (5,5,5) window with those coefficients.  `coef_planes`: ck and cv planes [head][125][token].
+bool try_bounded_offsets_planes_grad(const void* q, const void* k, const void* dout, const float* coef_planes, void* dq,
+                                     void* dk, void* dv, const Problem& pr, const int* gate, cudaStream_t stream,
+                                     cudaError_t* err) {
+    *err = cudaSuccess;
+    if ((pr.d != 128 && pr.d != 64) || pr.kt != 3 || pr.kh != 3 || pr.kw != 3) return false;
+    int* flag = timeout_flag_device_address();
+    if (!flag) return false;
+    bool unsupported = false;
+    const uint32_t* coef = reinterpret_cast<const uint32_t*>(coef_planes);
+    *err = pr.d == 128 ? launch_planes_grad<128, 5, 5, 5>(q, k, dout, coef, dq, dk, dv, pr, flag, stream, &unsupported, gate)
+                       : launch_planes_grad<64, 5, 5, 5>(q, k, dout, coef, dq, dk, dv, pr, flag, stream, &unsupported, gate);
     return !unsupported;
 }
 

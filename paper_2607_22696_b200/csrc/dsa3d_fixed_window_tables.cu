@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(kTbThreads, 1)
 fixed_window_tables_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_do,
                            const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                            float* __restrict__ table, int T, int H, int W, int heads, int tiles_x, int tiles_y, int total,
-                           int* timeout_flag) {
+                           int* timeout_flag, const int* __restrict__ gate) {
     using S = TableShape<D, KT, KH, KW>;
     constexpr int NH = S::NH, RT = S::RT, RX = S::RX, PS = S::PS, PSP = S::PSP, VH = S::VH, NS = S::NS;
     constexpr int BT = S::BT, BY = S::BY, BX = S::BX;
@@ -122,7 +122,9 @@ fixed_window_tables_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
         y0 = (tile % tiles_y) * kTbTY;
         t0 = (tile / tiles_y) * kTbTT;
     };
-    const int my_tiles = static_cast<int>(blockIdx.x) < total
+    // behind a check of learned offsets: nothing to do unless the check left 0 in *gate
+    const bool open = gate == nullptr || *gate == 0;
+    const int my_tiles = open && static_cast<int>(blockIdx.x) < total
                              ? (total - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x) : 0;
     auto tile_item = [&](int ti) { return static_cast<int>(blockIdx.x) + ti * static_cast<int>(gridDim.x); };
 
@@ -301,7 +303,7 @@ fixed_window_tables_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
 
 template <int D, int KT, int KH, int KW>
 cudaError_t launch_tables(const void* q, const void* k, const void* v, const void* dout, float* table, const Problem& pr,
-                          int* flag, cudaStream_t stream, bool* unsupported) {
+                          int* flag, cudaStream_t stream, bool* unsupported, const int* gate = nullptr) {
     using S = TableShape<D, KT, KH, KW>;
     const unsigned long long d = static_cast<unsigned long long>(pr.d), hd = static_cast<unsigned long long>(pr.heads);
     const unsigned long long dims[5] = {d, hd, static_cast<unsigned long long>(pr.W), static_cast<unsigned long long>(pr.H),
@@ -336,11 +338,28 @@ cudaError_t launch_tables(const void* q, const void* k, const void* v, const voi
     if (e != cudaSuccess) return e;
     const unsigned grid = static_cast<unsigned>(total < sms ? total : sms);     // persistent: one CTA per SM
     kern<<<grid, kTbThreads, smem, stream>>>(mq, mdo, mk, mv, table, pr.T, pr.H, pr.W, pr.heads, tiles_x, tiles_y,
-                                             static_cast<int>(total), flag);
+                                             static_cast<int>(total), flag, gate);
     return cudaGetLastError();
 }
 
 }  // namespace
+
+// Learned offsets below 1 in size, window (3,3,3): every corner of every sample, and the +1 neighbour a
+// one-sided derivative needs when a position rounds up to a grid position, lie in the box of 6 x 6 x 6
+// positions whose first corner is query - 2: the table of a (5,5,5) window.
+int bounded_offsets_table_floats() { return 2 * TableShape<128, 5, 5, 5>::CELLS8; }
+
+bool try_bounded_offsets_tables(const void* q, const void* k, const void* v, const void* dout, float* table,
+                                const Problem& pr, const int* gate, cudaStream_t stream, cudaError_t* err) {
+    *err = cudaSuccess;
+    if ((pr.d != 128 && pr.d != 64) || pr.kt != 3 || pr.kh != 3 || pr.kw != 3) return false;
+    int* flag = timeout_flag_device_address();
+    if (!flag) return false;
+    bool unsupported = false;
+    *err = pr.d == 128 ? launch_tables<128, 5, 5, 5>(q, k, v, dout, table, pr, flag, stream, &unsupported, gate)
+                       : launch_tables<64, 5, 5, 5>(q, k, v, dout, table, pr, flag, stream, &unsupported, gate);
+    return !unsupported;
+}
 
 // Floats per (token, head) item of the table for this problem, or 0 when the tensor-core table
 // kernel does not cover it (then the backward gathers its dot products itself).

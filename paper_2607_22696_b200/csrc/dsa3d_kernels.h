@@ -48,7 +48,10 @@ cudaError_t launch_dkdv_blocks(const void* q, const void* dout, const float* off
                                float* acc_dv, const Problem& pr, cudaStream_t stream);
 
 // fp32 accumulators -> bf16 outputs (round to nearest even).
-cudaError_t launch_convert_bf16(const float* acc, void* dst, long long count, cudaStream_t stream);
+cudaError_t launch_convert_bf16(const float* acc, void* dst, long long count, cudaStream_t stream,
+                                const int* gate = nullptr);
+// Zeroes `bytes` (a multiple of 16) at `dst` unless *gate is 0.
+cudaError_t launch_gated_clear(void* dst, size_t bytes, const int* gate, cudaStream_t stream);
 
 // Shared implementation of dsa3d_backward.  `tiled` selects the tile pre-reduction of the
 // dK/dV scatter (bf16 only; needs the large workspace); without it the workspace is just the
@@ -56,7 +59,7 @@ cudaError_t launch_convert_bf16(const float* acc, void* dst, long long count, cu
 int backward_impl(const void* q, const void* k, const void* v, const float* offsets, const float* lse,
                   const void* dout, int T, int H, int W, int heads, int d, const int window[3], void* dq,
                   void* dk, void* dv, float* doffsets, void* workspace, size_t workspace_bytes, int dtype,
-                  void* stream, bool tiled);
+                  void* stream, bool tiled, const int* gate = nullptr);
 
 // Backward of the fixed-window variant (dsa3d_fixed_window_backward.cu): dq, dk, dv in the storage
 // type, doffsets (may be NULL), coef [N*heads, P] scratch.  `table` (or NULL): the dot products
@@ -80,6 +83,26 @@ int fixed_window_table_floats(const Problem& pr, bool bf16);
 bool fixed_window_tile_grad_covers(const Problem& pr, bool bf16);
 bool try_fixed_window_tile_grad(const void* q, const void* k, const void* dout, const float2* coef, void* dq, void* dk,
                                 void* dv, const Problem& pr, cudaStream_t stream, cudaError_t* err);
+bool try_bounded_offsets_planes_grad(const void* q, const void* k, const void* dout, const float* coef_planes, void* dq,
+                                     void* dk, void* dv, const Problem& pr, const int* gate, cudaStream_t stream,
+                                     cudaError_t* err);
+
+// Backward for learned offsets below 1 in size, window (3,3,3) (dsa3d_bounded_offsets_backward.cu): tables,
+// per-query arithmetic and the three tile sums, all doing nothing unless *gate is 0.  Returns false when
+// nothing was launched (shape not covered).  `workspace`: bounded_offsets_backward_bytes(pr) bytes.
+bool bounded_offsets_backward_covers(const Problem& pr, bool bf16);
+size_t bounded_offsets_backward_bytes(const Problem& pr);
+bool try_bounded_offsets_backward(const void* q, const void* k, const void* v, const float* offsets, const float* lse,
+                                  const void* dout, void* dq, void* dk, void* dv, float* doffsets, void* workspace,
+                                  const int* gate, const Problem& pr, cudaStream_t stream, cudaError_t* err);
+
+// The dot-product tables of the box a query's samples can touch when every learned offset is below 1 in
+// size (window (3,3,3): 6 x 6 x 6 positions from query - 2, dsa3d_fixed_window_tables.cu); the kernel does
+// nothing unless *gate is 0.
+int bounded_offsets_table_floats();
+bool try_bounded_offsets_tables(const void* q, const void* k, const void* v, const void* dout, float* table,
+                                const Problem& pr, const int* gate, cudaStream_t stream, cudaError_t* err);
+
 // The same three sums for the larger windows ((3,5,5), (3,7,7); bf16, 64 or 128 channels) as products
 //  C_plane . X_plane  on the tensor cores, one region plane at a time (dsa3d_fixed_window_planes_grad.cu).
 bool fixed_window_planes_grad_covers(const Problem& pr, bool bf16);

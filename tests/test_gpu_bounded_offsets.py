@@ -109,3 +109,93 @@ def test_other_shapes_take_the_general_kernel(shape, window, dtype):
     P = window[0] * window[1] * window[2]
     off = _bounded_offsets((T, H, W, heads, P, 3), 730, "uniform")
     _run(shape, window, dtype, 173, off)
+
+
+# ------------------------------------------------------------------------------------------------
+# dsa3d_backward_bounded_offsets: dot-product tables on the tensor cores, per-sample arithmetic from
+# the tables, dq / dk / dv as the sums of a fixed 5 x 5 x 5 window on the tensor cores
+# ------------------------------------------------------------------------------------------------
+def _run_backward(shape, window, dtype, seed, offsets, sigma_q=1.0, entry=None):
+    T, H, W, heads, d = shape
+    P = window[0] * window[1] * window[2]
+    q, k, v, dout = (inputs.normal(shape, seed, i, sigma_q if i == 0 else 1.0, dtype) for i in range(4))
+    dev = [z.cuda() for z in (q, k, v, offsets, dout)]
+    out, lse = pu.gpu_forward(*dev[:4], shape, window)
+    grads = [torch.full(shape, float("nan"), dtype=dtype, device="cuda") for _ in range(3)]
+    doff = torch.full((T, H, W, heads, P, 3), float("nan"), dtype=F32, device="cuda")
+    nbytes = binding.dsa3d_backward_bounded_offsets_workspace_bytes(T, H, W, heads, d, window, dtype)
+    ws = torch.full((nbytes + 64,), 0xA5, dtype=torch.uint8, device="cuda")       # poisoned, with a guard band behind it
+    call = entry or binding.dsa3d_backward_bounded_offsets
+    call(dev[0], dev[1], dev[2], dev[3], lse, dev[4], T, H, W, heads, d, window, grads[0], grads[1], grads[2], doff,
+         ws[:nbytes] if nbytes else None, nbytes)
+    torch.cuda.synchronize()
+    assert binding.dsa3d_device_timeout_flag() == 0
+    assert torch.equal(ws[nbytes:].cpu(), torch.full((64,), 0xA5, dtype=torch.uint8))
+    refs = oracle.backward(q, k, v, offsets, dout, T, H, W, heads, d, window)
+    for name, got, ref in zip(("dq", "dk", "dv", "doffsets"), (*grads, doff), refs):
+        pu.assert_close(name, got, ref, dtype, backward=True)
+    return dev, lse, grads, doff
+
+
+@pytest.mark.parametrize("shape", [(6, 9, 13, 2, 128), (4, 4, 8, 1, 128), (1, 1, 1, 1, 128), (9, 5, 17, 3, 128),
+                                   (2, 13, 7, 2, 128), (8, 8, 16, 2, 64), (5, 4, 19, 3, 64)])
+@pytest.mark.parametrize("kind", ["uniform", "edge"])
+def test_backward_tile_kernels_for_offsets_below_one_match_the_oracle(shape, kind):
+    T, H, W, heads, d = shape
+    off = _bounded_offsets((T, H, W, heads, 27, 3), 740 + T * W, kind)
+    _run_backward(shape, (3, 3, 3), BF16, 174, off)
+
+
+@pytest.mark.parametrize("kind", ["tiny", "zero", "uniform"])
+def test_backward_tile_kernels_many_tiles_per_block(kind):
+    """More (tile, head) items than SMs, a sharp softmax: the persistent blocks walk several tiles."""
+    shape = (12, 20, 40, 4, 128)
+    T, H, W, heads, d = shape
+    off = _bounded_offsets((T, H, W, heads, 27, 3), 750, kind)
+    _run_backward(shape, (3, 3, 3), BF16, 175, off, sigma_q=3.0)
+
+
+def test_backward_roads_agree_and_one_large_offset_switches_to_the_general_kernels():
+    """The bounded problem through the tile kernels and through dsa3d_backward: within a bf16 step of each
+    other.  Then one offset of size 1.5, a NaN, an infinity, exactly -1: the device-side check must hand
+    the whole call to the general kernels (which were queued behind the tile kernels), and dq and doffsets
+    are dsa3d_backward's bit for bit, dk and dv up to the order of its atomic sums."""
+    shape, window = (8, 10, 20, 3, 128), (3, 3, 3)
+    T, H, W, heads, d = shape
+    off = _bounded_offsets((T, H, W, heads, 27, 3), 760, "uniform")
+    dev, lse, g_tc, doff_tc = _run_backward(shape, window, BF16, 176, off)
+    g_gen = pu.gpu_backward(dev[0], dev[1], dev[2], dev[3], lse, dev[4], shape, window)
+    for a, b in zip((*g_tc, doff_tc), g_gen):
+        a, b = a.float(), b.float()
+        step = (b.abs() * 2.0 ** -7).clamp_min(float(b.pow(2).mean().sqrt()) * 2.0 ** -7)
+        assert bool(((a - b).abs() <= step).all())
+    nbytes = binding.dsa3d_backward_bounded_offsets_workspace_bytes(T, H, W, heads, d, window, BF16)
+    ws = torch.empty((nbytes,), dtype=torch.uint8, device="cuda")
+    for bad in (1.5, float("nan"), float("inf"), -1.0):
+        off2 = off.clone()
+        off2.view(-1)[off2.numel() // 2 + 1] = bad
+        o2 = off2.cuda()
+        _, lse2 = pu.gpu_forward(dev[0], dev[1], dev[2], o2, shape, window)
+        ga = [torch.full(shape, float("nan"), dtype=BF16, device="cuda") for _ in range(3)]
+        da = torch.full((T, H, W, heads, 27, 3), float("nan"), dtype=F32, device="cuda")
+        binding.dsa3d_backward_bounded_offsets(dev[0], dev[1], dev[2], o2, lse2, dev[4], T, H, W, heads, d, window,
+                                               ga[0], ga[1], ga[2], da, ws, nbytes)
+        gb = pu.gpu_backward(dev[0], dev[1], dev[2], o2, lse2, dev[4], shape, window)
+        torch.cuda.synchronize()
+        for a, b in ((ga[0], gb[0]), (da, gb[3])):          # per-query results: the same kernel, the same bits
+            assert bool(((a == b) | (torch.isnan(a) & torch.isnan(b))).all()), bad
+        for a, b in ((ga[1], gb[1]), (ga[2], gb[2])):
+            fa, fb = a.float(), b.float()
+            finite = torch.isfinite(fb)
+            assert torch.equal(torch.isfinite(fa), finite)
+            step = (fb[finite].abs() * 2.0 ** -7).clamp_min(2e-3)
+            assert bool(((fa[finite] - fb[finite]).abs() <= step).all()), bad
+
+
+@pytest.mark.parametrize("shape,window,dtype", [((4, 6, 7, 2, 32), (3, 3, 3), BF16), ((3, 5, 6, 2, 32), (3, 3, 3), F32),
+                                                ((4, 6, 9, 2, 128), (2, 2, 2), BF16), ((4, 6, 9, 2, 64), (3, 5, 5), BF16)])
+def test_backward_other_shapes_take_the_general_kernels(shape, window, dtype):
+    T, H, W, heads, d = shape
+    P = window[0] * window[1] * window[2]
+    off = _bounded_offsets((T, H, W, heads, P, 3), 770, "uniform")
+    _run_backward(shape, window, dtype, 177, off)
