@@ -13,10 +13,11 @@
 // fixed_window_backward_query_kernel then takes its dot products from the table instead of
 // gathering K and V rows.
 //
-// Roles as in the plane-by-plane forward: 16 worker warps copy scores (the four warps that share a TMEM
+// Roles as in the plane-by-plane forward: 8 worker warps copy scores (the two warps that share a TMEM
 // quadrant split a plane's columns and the box's rows along y between them), one more warp holds the
-// thread that issues the TMA loads, two more one thread each that issues the MMAs of every other plane; mbarriers order them, every wait is bounded, and a wait that
-// runs out raises the library's timeout flag, after which nobody waits any more.
+// thread that issues the TMA loads, two more one thread each that issues the MMAs of every other plane;
+// mbarriers order them, every wait is bounded, and a wait that runs out raises the library's timeout
+// flag, after which nobody waits any more.
 #include <cuda_bf16.h>
 
 #include "dsa3d_common.cuh"
@@ -269,6 +270,21 @@ fixed_window_tables_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
 #pragma unroll
                                 for (int i = 0; i < RUN / 4; ++i)
                                     reinterpret_cast<float4*>(dst)[i] = make_float4(cells[4 * i], cells[4 * i + 1], cells[4 * i + 2], cells[4 * i + 3]);
+                            } else if constexpr (whole && RUN % 4 == 2 && (BY * BX) % 4 == 0 && S::CELLS8 % 4 == 0) {
+                                // the run starts 16-byte aligned for every other thread of the group and 8 bytes
+                                // off for the others: one 8-byte piece at the far or the near end, 16-byte pieces between
+                                const int lead = (half * RUN) & 3;                  // 0 or 2 floats before the first aligned piece
+                                if (lead) *reinterpret_cast<float2*>(dst) = make_float2(cells[0], cells[1]);
+#pragma unroll
+                                for (int i = 0; i < RUN / 4; ++i) {
+                                    float4 piece;
+                                    piece.x = lead ? cells[4 * i + 2] : cells[4 * i];
+                                    piece.y = lead ? cells[4 * i + 3] : cells[4 * i + 1];
+                                    piece.z = lead ? cells[4 * i + 4] : cells[4 * i + 2];
+                                    piece.w = lead ? cells[4 * i + 5] : cells[4 * i + 3];
+                                    *reinterpret_cast<float4*>(dst + lead + 4 * i) = piece;
+                                }
+                                if (!lead) *reinterpret_cast<float2*>(dst + RUN - 2) = make_float2(cells[RUN - 2], cells[RUN - 1]);
                             } else if constexpr (whole && RUN % 2 == 0 && (BY * BX) % 2 == 0 && S::CELLS8 % 2 == 0) {
 #pragma unroll
                                 for (int i = 0; i < RUN / 2; ++i) reinterpret_cast<float2*>(dst)[i] = make_float2(cells[2 * i], cells[2 * i + 1]);
