@@ -55,12 +55,12 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of grids whose K/V and accumulators no longer fit the 126 MB L2 (a one-off capture
 # at 1080p gave 1.7x / 1.6x / 1.8x the small case's bytes per item for the three kernels).
 NCU_PER_ITEM = {
-    "forward_kernel": {"dram": 1525.0, "l2_sm": 83800.0, "inst": 5509.0,
-                       "sources": ["dsa3d_forward.cu", "dsa3d_common.cuh"], "sha": "d5e2be99de83"},
-    "backward_kernel": {"dram": 3002.0, "l2_sm": 92036.0, "inst": 5900.0,
-                        "sources": ["dsa3d_backward.cu", "dsa3d_common.cuh"], "sha": "19c61e43dd9d"},
-    "scatter_tile_kernel": {"dram": 13025.0, "inst": 6025.0,
-                            "sources": ["dsa3d_backward.cu", "dsa3d_common.cuh"], "sha": "19c61e43dd9d"},
+    "forward_kernel": {"dram": 1525.0, "l2_sm": 83815.0, "inst": 5509.0,
+                       "sources": ["dsa3d_forward.cu", "dsa3d_common.cuh"], "sha": "a335f85dc533"},
+    "backward_kernel": {"dram": 3003.0, "l2_sm": 92009.0, "inst": 5901.0,
+                        "sources": ["dsa3d_backward.cu", "dsa3d_common.cuh"], "sha": "ac74993402dc"},
+    "scatter_tile_kernel": {"dram": 13000.0, "inst": 5980.0,
+                            "sources": ["dsa3d_backward.cu", "dsa3d_common.cuh"], "sha": "ac74993402dc"},
 }
 
 
