@@ -417,9 +417,10 @@ int dsa3d_forward_bounded_offsets(const void* q, const void* k, const void* v, c
  * dsa3d_backward_fixed_window.  Otherwise the kernels of dsa3d_backward run (they are queued behind the
  * others and do nothing when the check passed), so the call is correct for any offsets and stays
  * asynchronous.  dk and dv of the tile route are written once in `dtype` (no atomics, bitwise deterministic).
- * `workspace`: dsa3d_backward_bounded_offsets_workspace_bytes(...) bytes, 16-byte aligned, contents undefined
- * afterwards.  Other shapes and dtypes, and the switches DSA3D_NO_TENSOR_FIXED_WINDOW and DSA3D_KEY_BLOCKS=1,
- * make it dsa3d_backward.  Bounded waits as in dsa3d_offsets_linear_forward (dsa3d_device_timeout_flag).
+ * `workspace`: dsa3d_backward_bounded_offsets_workspace_bytes(...) bytes (for the tile route 2.7 KB per
+ * (token, head): the tables and the coefficient boxes), 16-byte aligned, contents undefined afterwards.
+ * Other shapes and dtypes, grids of 2^31 / (125 heads) tokens or more, and the switches
+ * DSA3D_NO_TENSOR_FIXED_WINDOW and DSA3D_KEY_BLOCKS=1, make it dsa3d_backward.  Bounded waits as in dsa3d_offsets_linear_forward (dsa3d_device_timeout_flag).
  */
 int dsa3d_backward_bounded_offsets(const void* q, const void* k, const void* v, const float* offsets, const float* lse,
                                    const void* dout, int T, int H, int W, int heads, int d, const int window[3], void* dq,

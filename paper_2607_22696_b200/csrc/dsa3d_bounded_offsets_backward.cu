@@ -175,8 +175,11 @@ bounded_offsets_backward_query_kernel(const float* __restrict__ offsets, const f
 }  // namespace
 
 bool bounded_offsets_backward_covers(const Problem& pr, bool bf16) {
-    return bf16 && (pr.d == 128 || pr.d == 64) && pr.kt == 3 && pr.kh == 3 && pr.kw == 3 &&
-           pr.q_begin == 0 && pr.q_count == pr.N;
+    if (!bf16 || (pr.d != 128 && pr.d != 64) || pr.kt != 3 || pr.kh != 3 || pr.kw != 3) return false;
+    if (pr.q_begin != 0 || pr.q_count != pr.N) return false;
+    // what the tile kernels count in 32 bits: positions inside a coefficient plane, planes walked
+    const long long tiles = static_cast<long long>((pr.W + 7) / 8) * ((pr.H + 3) / 4) * ((pr.T + 3) / 4) * pr.heads;
+    return pr.N * pr.heads * kBoBoxCells < (1LL << 31) && tiles * 3 * 9 < (1LL << 31);
 }
 
 // Bytes of workspace of the three kernels: the tables, then the two coefficient planes.
