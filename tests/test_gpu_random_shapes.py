@@ -1,6 +1,7 @@
 """Seeded random sweep over small problems: grid extents (including 1), head counts, head sizes,
 storage types, windows and offset kinds are drawn at random and every entry point that applies
-(general forward/backward; the fixed-window pair when the offsets are zero) is compared with the
+(general forward/backward; the fixed-window pair when the offsets are zero; the bounded-offsets pair on
+offsets below 1 in size) is compared with the
 oracle.  Catches indexing slips that hand-picked shapes miss; the draws are fixed by the seed."""
 import random
 
@@ -66,6 +67,44 @@ def test_random_small_problems_match_the_oracle(seed):
         for name, got, want in zip(("dq", "dk", "dv"), g, refs[:3]):
             pu.assert_close(name, got, want.view(shape), dtype, backward=True)
         pu.assert_close("doffsets", doff, refs[3].view(T, H, W, heads, P, 3), dtype, backward=True)
+
+
+@pytest.mark.parametrize("seed", [3])
+def test_random_small_offset_problems_match_the_oracle(seed):
+    """The pair of entry points for learned offsets below 1 in size (window (3,3,3), bf16) on random small
+    grids: offsets uniform in (-1, 1), or drawn from values next to -1, 0 and +1 where a sample changes cell."""
+    rng = random.Random(seed)
+    window, P = (3, 3, 3), 27
+    edge = torch.tensor([-0.99999994, -1e-7, 0.0, 1e-7, 0.99999994, 0.5, -0.5], dtype=F32)
+    for it in range(24):
+        shape = (rng.randint(1, 9), rng.randint(1, 11), rng.randint(1, 19), rng.randint(1, 3), rng.choice([64, 128]))
+        T, H, W, heads, d = shape
+        s = 2000 + it
+        q, k, v, dout = (inputs.normal(shape, s, i, rng.choice([1.0, 3.0]) if i == 0 else 1.0, BF16) for i in range(4))
+        gen = torch.Generator().manual_seed(s)
+        if rng.random() < 0.5:
+            off = (torch.rand((T, H, W, heads, P, 3), generator=gen, dtype=torch.float64) * 2 - 1).clamp(-0.999999, 0.999999).to(F32)
+        else:
+            off = edge[torch.randint(0, edge.numel(), (T, H, W, heads, P, 3), generator=gen)]
+        o_ref, l_ref = oracle.forward(q.view(-1, heads, d), k, v, off.view(-1, heads, P, 3), T, H, W, heads, d, window)
+        refs = oracle.backward(q.view(-1, heads, d), k, v, off.view(-1, heads, P, 3), dout.view(-1, heads, d),
+                               T, H, W, heads, d, window)
+        qd, kd, vd, od, dd = (z.cuda() for z in (q, k, v, off, dout))
+        out = torch.full(shape, float("nan"), dtype=BF16, device="cuda")
+        lse = torch.full((T, H, W, heads), float("nan"), dtype=F32, device="cuda")
+        binding.dsa3d_forward_bounded_offsets(qd, kd, vd, od, T, H, W, heads, d, window, out, lse)
+        g = [torch.full(shape, float("nan"), dtype=BF16, device="cuda") for _ in range(3)]
+        doff = torch.full((T, H, W, heads, P, 3), float("nan"), dtype=F32, device="cuda")
+        ws = torch.empty((binding.dsa3d_backward_bounded_offsets_workspace_bytes(T, H, W, heads, d, window, BF16),),
+                         dtype=torch.uint8, device="cuda")
+        binding.dsa3d_backward_bounded_offsets(qd, kd, vd, od, lse, dd, T, H, W, heads, d, window, g[0], g[1], g[2], doff, ws)
+        torch.cuda.synchronize()
+        assert binding.dsa3d_device_timeout_flag() == 0
+        pu.assert_close("out", out, o_ref.view(shape), BF16)
+        pu.assert_close("lse", lse, l_ref.view(T, H, W, heads), BF16)
+        for name, got, want in zip(("dq", "dk", "dv"), g, refs[:3]):
+            pu.assert_close(name, got, want.view(shape), BF16, backward=True)
+        pu.assert_close("doffsets", doff, refs[3].view(T, H, W, heads, P, 3), BF16, backward=True)
 
 
 def _sum_close(name, got, ref, rel):
