@@ -118,14 +118,39 @@ def test_binding_reports_library_errors():
 
 # ------------------------------------------------- BASELINE configs 3, 4, 5 at full size
 
-def run_large(name, heads_sel, key_boxes, n_random=1024, backward=True):
+def _tile_route(t, dims, window, fixed_window):
+    """The pair of entry points `bench.py` times for workloads with zero offsets (fixed-window pair) or
+    offsets below 1 in size (bounded-offsets pair)."""
+    T, H, W, heads, d = dims
+    out, lse = torch.full_like(t["q"], float("nan")), torch.full((T, H, W, heads), float("nan"), device="cuda")
+    grads = [torch.full_like(t["q"], float("nan")) for _ in range(3)] + [torch.full_like(t["offsets"], float("nan"))]
+    sizes = binding.dsa3d_backward_fixed_window_workspace_bytes if fixed_window else binding.dsa3d_backward_bounded_offsets_workspace_bytes
+    ws = torch.full((max(sizes(T, H, W, heads, d, window, t["q"].dtype), 16),), 0xFF, dtype=torch.uint8, device="cuda")
+    if fixed_window:
+        binding.dsa3d_forward_fixed_window(t["q"], t["k"], t["v"], T, H, W, heads, d, window, out, lse)
+        binding.dsa3d_backward_fixed_window(t["q"], t["k"], t["v"], lse, t["dout"], T, H, W, heads, d, window, *grads, ws)
+    else:
+        binding.dsa3d_forward_bounded_offsets(t["q"], t["k"], t["v"], t["offsets"], T, H, W, heads, d, window, out, lse)
+        binding.dsa3d_backward_bounded_offsets(t["q"], t["k"], t["v"], t["offsets"], lse, t["dout"], T, H, W, heads, d,
+                                               window, *grads, ws)
+    torch.cuda.synchronize()
+    assert binding.dsa3d_device_timeout_flag() == 0
+    return out, lse, tuple(grads)
+
+
+def run_large(name, heads_sel, key_boxes, n_random=1024, backward=True, route="general"):
     wl = inputs.WORKLOADS[name]
     dims = (wl.T, wl.H, wl.W, wl.heads, wl.d)
-    t = inputs.make_inputs(wl, "cuda")
-    out, lse = pu.gpu_forward(t["q"], t["k"], t["v"], t["offsets"], dims, wl.window)
-    t["out"] = out
+    t = inputs.make_inputs(wl, "cuda", with_dout=True) if route != "general" else inputs.make_inputs(wl, "cuda")
     grads = None
-    if backward:
+    if route != "general":
+        out, lse, grads = _tile_route(t, dims, wl.window, route == "fixed_window")
+        t["out"] = out
+        pu.assert_bilinearity_invariants(t, out, grads)
+    else:
+        out, lse = pu.gpu_forward(t["q"], t["k"], t["v"], t["offsets"], dims, wl.window)
+        t["out"] = out
+    if backward and route == "general":
         grads = pu.gpu_backward(t["q"], t["k"], t["v"], t["offsets"], lse, t["dout"], dims, wl.window)
         pu.assert_bilinearity_invariants(t, out, grads)
     pu.sampled_parity(t, dims, wl.window, lse, grads, heads_sel, n_random=n_random, key_boxes=key_boxes)
@@ -173,6 +198,17 @@ def test_paper_window_3x7x7_on_the_1080p_grid():
 def test_config_sweep_720p_grid(window, kind):
     boxes = [((0, 0, 0), (1, 2, 2)), ((32, 22, 40), (33, 23, 42))]
     run_large(f"sweep_w{window}_{kind}", [0, 15], boxes, n_random=512)
+
+
+@pytest.mark.parametrize("name,route", [("sweep_w222_zero", "fixed_window"), ("sweep_w333_zero", "fixed_window"),
+                                        ("sweep_w355_zero", "fixed_window"), ("sweep_w377_zero", "fixed_window"),
+                                        ("sweep_w333_small", "bounded")])
+def test_sweep_grid_through_the_entry_points_the_bench_times(name, route):
+    """Zero offsets and offsets below 1 in size at the sweep's full grid, through the entry points
+    `bench.py` uses for them (tensor-core tile kernels): sampled queries and key boxes against the oracle,
+    whole-tensor invariants."""
+    boxes = [((0, 0, 0), (1, 2, 2)), ((32, 22, 40), (33, 23, 42)), ((63, 44, 78), (64, 45, 80))]
+    run_large(name, [0, 15], boxes, n_random=512, route=route)
 
 
 # ------------------------------------------------- tilings of the backward dK/dV scatter
