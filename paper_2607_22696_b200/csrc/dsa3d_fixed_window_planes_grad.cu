@@ -53,10 +53,13 @@ struct PgShape {
     // target (dK, dV) reaches k - 1 - k/2 back
     static constexpr int FT = KT / 2, FY = KH / 2, FX = KW / 2;
     static constexpr int BT = KT - 1 - KT / 2, BY = KH - 1 - KH / 2, BX = KW - 1 - KW / 2;
-    // The coefficient matrices of successive (plane, head | remainder) units rotate through NC buffers, so
-    // the workers write up to NC - 1 units ahead of the chain that is running.
+    // The coefficient matrices of successive (plane, head | remainder) units rotate through NC buffers: the
+    // workers write unit k + NC - 1 while the chain of unit k runs.  Two (head in one, remainder in the other)
+    // measured best: every further buffer is one more unit in which a thread has to write its cells back to
+    // zero after its last plane (3x5x5 backward 12.4 / 12.8 / 13.0 ms with 2 / 3 / 4), and leaves less room
+    // for plane buffers.
     static constexpr int BUDGET = 227 * 1024 - 2048;
-    static constexpr int NC = BUDGET - 3 * SLOT_BYTES >= 4 * C_BYTES ? 4 : 3;
+    static constexpr int NC = 2;
     static constexpr int NS_RAW = (BUDGET - NC * C_BYTES) / SLOT_BYTES;
     static constexpr int NS = NS_RAW > kPgMaxSlots ? kPgMaxSlots : NS_RAW;
     static_assert(PSP <= 256 && 3 * D <= 512, "a plane is one MMA's K extent; three accumulators in TMEM");
