@@ -38,6 +38,12 @@
  * Supported: dtype DSA3D_F32 or DSA3D_BF16; d in {32, 64, 128}; 1 <= P <= 256;
  * T, H, W, heads >= 1; T*H*W < 2^31.  Arithmetic is fp32 whatever the storage type.
  *
+ * Non-finite values.  dsa3d_forward and dsa3d_backward confine a NaN or infinity in a row of q, k, v or dout to
+ * the results that row enters by the definition above.  The tile kernels behind the fixed-window and
+ * bounded-offsets entry points form dense products over the region of a 4 x 4 x 8 tile, in which such a row is
+ * multiplied by zero weights as well: there it can reach every output of the tiles whose region holds the row.
+ * Finite inputs are not affected.
+ *
  * Errors.  Every function returns a dsa3d_status (0 = success).  Arguments are checked
  * before anything is launched; nothing aborts, throws or traps.
  *
