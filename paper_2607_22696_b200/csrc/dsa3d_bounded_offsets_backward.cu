@@ -35,10 +35,12 @@ constexpr int kBoBox = 5, kBoBoxCells = kBoBox * kBoBox * kBoBox;      // coeffi
 constexpr int kBoRounds = (kBoP + kBoLanes - 1) / kBoLanes;
 
 struct BoGroup {
-    float tab_a[kBoTabCells], tab_b[kBoTabCells];
-    float box_ck[kBoBoxCells], box_cv[kBoBoxCells];
+    union {                                  // the tables are read for the last time before the box is first written
+        struct { float tab_a[kBoTabCells], tab_b[kBoTabCells]; };
+        struct { float box_ck[kBoBoxCells], box_cv[kBoBoxCells]; };
+    };
     float s_ck[kBoP], s_cv[kBoP], s_ft[kBoP], s_fy[kBoP], s_fx[kBoP];
-    int s_cell[kBoP];                        // (bt * 5 + by) * 5 + bx of corner (0,0,0) in the coefficient box, -1: dead sample
+    int s_cell[kBoP];                        // bt | by << 3 | bx << 6 of corner (0,0,0) in the coefficient box, -1: dead sample
 };
 
 // An fp32 value as two bf16 numbers whose sum is the value to 2^-17 relative: the nearest bf16 in the low
@@ -77,7 +79,6 @@ bounded_offsets_backward_query_kernel(const float* __restrict__ offsets, const f
             g.tab_a[i] = __ldg(mine + i);
             g.tab_b[i] = __ldg(mine + kBoTabCells + i);
         }
-        for (int i = gl; i < kBoBoxCells; i += kBoLanes) g.box_ck[i] = g.box_cv[i] = 0.0f;
     }
     __syncwarp();
 
@@ -109,7 +110,7 @@ bounded_offsets_backward_query_kernel(const float* __restrict__ offsets, const f
             }
             trilerp_grad(a, cell.ft, cell.fy, cell.fx, sdot, da[r][0], da[r][1], da[r][2]);
             trilerp_grad(b, cell.ft, cell.fy, cell.fx, gp[r], db[r][0], db[r][1], db[r][2]);
-            code = (bt * kBoBox + by) * kBoBox + bx;
+            code = bt | (by << 3) | (bx << 6);
         }
         alpha[r] = exp2f(fmaf(sdot, scale * kLog2e, -lse2));   // a dead sample stays in the softmax with logit 0
         delta = fmaf(alpha[r], gp[r], delta);
@@ -133,26 +134,29 @@ bounded_offsets_backward_query_kernel(const float* __restrict__ offsets, const f
             dst[2] = fmaf(ck, da[r][2], alpha[r] * db[r][2]);
         }
     }
+    __syncwarp();                                          // every table read of the group is done: the box takes their place
+    for (int i = gl; i < kBoBoxCells; i += kBoLanes) g.box_ck[i] = g.box_cv[i] = 0.0f;
     __syncwarp();
 
-    // ---- the coefficient box: sample after sample, the eight lanes taking the eight corners (distinct
-    //      positions, so plain read-add-write; the order of the sums is fixed)
+    // ---- the coefficient box: sample after sample, the eight lanes taking the eight corners.  A lane takes
+    //      the corner whose box position has the lane's parity pattern (t, y, x parities = the lane's three
+    //      bits): the eight corners of a cell have the eight patterns once each, so a box position is only
+    //      ever touched by one lane - plain read-add-write, no ordering between lanes, sums in sample order.
     {
-        const int ct = gl >> 2, cy = (gl >> 1) & 1, cx = gl & 1;
+#pragma unroll 3
         for (int p = 0; p < kBoP; ++p) {
             const int code = g.s_cell[p];
-            if (code >= 0) {
-                const float ft = g.s_ft[p], fy = g.s_fy[p], fx = g.s_fx[p];
-                const float w = (ct ? ft : 1.0f - ft) * (cy ? fy : 1.0f - fy) * (cx ? fx : 1.0f - fx);
-                const int bx = code % kBoBox, by = (code / kBoBox) % kBoBox, bt = code / (kBoBox * kBoBox);
-                // a corner beyond the box can only carry weight 0 (a position rounded up to the box's last plane)
-                if (w != 0.0f && bt + ct < kBoBox && by + cy < kBoBox && bx + cx < kBoBox) {
-                    const int i = code + (ct * kBoBox + cy) * kBoBox + cx;
-                    g.box_ck[i] = fmaf(g.s_ck[p], w, g.box_ck[i]);
-                    g.box_cv[i] = fmaf(g.s_cv[p], w, g.box_cv[i]);
-                }
+            if (code < 0) continue;
+            const int bt = code & 7, by = (code >> 3) & 7, bx = code >> 6;
+            const int ct = (gl >> 2) ^ (bt & 1), cy = ((gl >> 1) & 1) ^ (by & 1), cx = (gl & 1) ^ (bx & 1);
+            const float ft = g.s_ft[p], fy = g.s_fy[p], fx = g.s_fx[p];
+            const float w = (ct ? ft : 1.0f - ft) * (cy ? fy : 1.0f - fy) * (cx ? fx : 1.0f - fx);
+            // a corner beyond the box can only carry weight 0 (a position rounded up to the box's last plane)
+            if (w != 0.0f && bt + ct < kBoBox && by + cy < kBoBox && bx + cx < kBoBox) {
+                const int i = ((bt + ct) * kBoBox + by + cy) * kBoBox + bx + cx;
+                g.box_ck[i] = fmaf(g.s_ck[p], w, g.box_ck[i]);
+                g.box_cv[i] = fmaf(g.s_cv[p], w, g.box_cv[i]);
             }
-            __syncwarp();
         }
     }
 
