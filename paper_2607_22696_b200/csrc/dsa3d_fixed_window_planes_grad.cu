@@ -245,26 +245,30 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
             auto chunk_off = [&](uint32_t col) { return (col >> 6) * (kPgRows * 128) + row_off + ((((col & 63) >> 3) ^ rx) << 4); };
             row_geo[vi] = (chunk_off(col0) >> 4) | ((chunk_off(col0 + 8) >> 4) << 12) | ((col0 & 7u) << 24);
         }
-        // KW bf16 values, packed in pairs (w[3] unused beyond KW), to their places in the row's two chunks
-        auto store_row = [&](unsigned char* dst, uint32_t geo, const uint32_t (&w)[4]) {
+        // The KW cells of a kernel row (a word each: bf16 head | bf16 remainder << 16) moved to their places among
+        // the 16 columns of the row's two chunks - one network of selects for head and remainder together, the
+        // shift (0 .. 7 columns) being the thread's own - then parted into the words of the head matrix and of
+        // the remainder matrix (two columns per word).
+        auto align_row = [&](uint32_t geo, const uint32_t (&cell)[8], uint32_t (&head)[8], uint32_t (&rest)[8]) {
             const bool s1 = (geo >> 24) & 1u, s2 = (geo >> 25) & 1u, s4 = (geo >> 26) & 1u;
-            uint32_t a[5], b[6], c[8];
-            a[0] = s1 ? w[0] << 16 : w[0];
+            uint32_t a[8], b[10], c[14];
+            a[0] = s1 ? 0u : cell[0];
 #pragma unroll
-            for (int i = 1; i < 4; ++i) a[i] = s1 ? __funnelshift_l(w[i - 1], w[i], 16) : w[i];
-            a[4] = s1 ? w[3] >> 16 : 0u;
-            b[0] = s2 ? 0u : a[0];
+            for (int i = 1; i < 8; ++i) a[i] = s1 ? cell[i - 1] : cell[i];              // cell[7] is always 0 (KW <= 7)
 #pragma unroll
-            for (int i = 1; i < 5; ++i) b[i] = s2 ? a[i - 1] : a[i];
-            b[5] = s2 ? a[4] : 0u;
-            c[0] = s4 ? 0u : b[0];
-            c[1] = s4 ? 0u : b[1];
+            for (int i = 0; i < 10; ++i) b[i] = s2 ? (i >= 2 ? a[i - 2] : 0u) : (i < 8 ? a[i] : 0u);
 #pragma unroll
-            for (int i = 2; i < 6; ++i) c[i] = s4 ? b[i - 2] : b[i];
-            c[6] = s4 ? b[4] : 0u;
-            c[7] = s4 ? b[5] : 0u;
-            *reinterpret_cast<uint4*>(dst + ((geo & 0xfffu) << 4)) = make_uint4(c[0], c[1], c[2], c[3]);
-            if (((geo >> 24) & 7u) + KW > 8u) *reinterpret_cast<uint4*>(dst + (((geo >> 12) & 0xfffu) << 4)) = make_uint4(c[4], c[5], c[6], c[7]);
+            for (int i = 0; i < 14; ++i) c[i] = s4 ? (i >= 4 ? b[i - 4] : 0u) : (i < 10 ? b[i] : 0u);
+#pragma unroll
+            for (int j = 0; j < 7; ++j) {
+                head[j] = __byte_perm(c[2 * j], c[2 * j + 1], 0x5410);
+                rest[j] = __byte_perm(c[2 * j], c[2 * j + 1], 0x7632);
+            }
+            head[7] = rest[7] = 0u;
+        };
+        auto store_chunks = [&](unsigned char* dst, uint32_t geo, const uint32_t (&w)[8]) {
+            *reinterpret_cast<uint4*>(dst + ((geo & 0xfffu) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+            if (((geo >> 24) & 7u) + KW > 8u) *reinterpret_cast<uint4*>(dst + (((geo >> 12) & 0xfffu) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
         };
         const int n_step = T * H * W;                                 // tokens: the step from one sample's plane to the next
         const uint32_t* plane_ck = coef;                              // [head][sample][token], a word = bf16 head | bf16 remainder << 16
@@ -369,7 +373,7 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
             // A thread's cells are the same columns in every unit.  After its last plane of a sweep it
             // writes them back to zero in the NC units that follow (one per buffer).
             const bool writes = mine || clear_left > 0;
-            uint32_t rest[VH][4];                             // bf16 remainders of this plane's coefficients, packed in pairs
+            uint32_t rest[VH][8];                             // remainder words of this plane's rows, already in place
             // ---- head
             if (!first_round) wait(&s.bar_c_free[buf], c_parity ^ 1u, 54);       // the chain of the unit NC before this one
             if (writes) {
@@ -377,21 +381,15 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
 #pragma unroll
                 for (int vi = 0; vi < VH; ++vi) {
                     if (vi >= nv) continue;
-                    uint32_t head[4];
+                    // the row's cells: 0 beyond KW, for a query that does not exist, and when clearing
+                    uint32_t cell[8], head[8];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        // cells 2j and 2j + 1 of the kernel row (0 beyond KW, for a query that does not exist, and when
-                        // clearing): their heads side by side in one word, their remainders in another
-                        uint32_t w[2];
-#pragma unroll
-                        for (int e = 0; e < 2; ++e) {
-                            const int ww = 2 * j + e, i = vi * KW + ww;
-                            w[e] = (ww < KW && mine && !((dnext >> (ww < KW ? i : 0)) & 1u)) ? wnext[ww < KW ? i : 0] : 0u;
-                        }
-                        head[j] = __byte_perm(w[0], w[1], 0x5410);
-                        rest[vi][j] = __byte_perm(w[0], w[1], 0x7632);
+                    for (int ww = 0; ww < 8; ++ww) {
+                        const int i = vi * KW + (ww < KW ? ww : 0);
+                        cell[ww] = (ww < KW && mine && !((dnext >> i) & 1u)) ? wnext[i] : 0u;
                     }
-                    store_row(dst, row_geo[vi], head);
+                    align_row(row_geo[vi], cell, head, rest[vi]);
+                    store_chunks(dst, row_geo[vi], head);
                 }
                 if (!mine) --clear_left;
             }
@@ -407,12 +405,12 @@ fixed_window_planes_grad_kernel(const __grid_constant__ CUtensorMap map_k, const
             if (!first_round) wait(&s.bar_c_free[buf], c_parity ^ 1u, 54);
             if (writes_rest) {
                 unsigned char* dst = s.c[buf];
-                const uint32_t zero[4] = {0u, 0u, 0u, 0u};
+                const uint32_t zero[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
 #pragma unroll
                 for (int vi = 0; vi < VH; ++vi) {
                     if (vi >= nv) continue;
-                    if (mine) store_row(dst, row_geo[vi], rest[vi]);
-                    else store_row(dst, row_geo[vi], zero);
+                    if (mine) store_chunks(dst, row_geo[vi], rest[vi]);
+                    else store_chunks(dst, row_geo[vi], zero);
                 }
                 if (!mine) --clear_left;
             }
