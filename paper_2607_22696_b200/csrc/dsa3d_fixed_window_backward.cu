@@ -37,7 +37,9 @@ __device__ __forceinline__ uint32_t split_bf16_pair(float x) {
 #ifndef DSA3D_FWB_TABLE_BLOCKS
 #define DSA3D_FWB_TABLE_BLOCKS 3
 #endif
-template <typename T, int D, bool TABLE>
+// KT, KH, KW: the window when it is known at compile time (the shapes the table kernel covers: loop bounds,
+// strides and the box layout then fold into the code), 0, 0, 0 = taken from the problem.
+template <typename T, int D, bool TABLE, int KT = 0, int KH = 0, int KW = 0>
 __global__ void __launch_bounds__(256, TABLE ? DSA3D_FWB_TABLE_BLOCKS : 1)
 fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                                    const float* __restrict__ lse, const T* __restrict__ dout, T* __restrict__ dq,
@@ -48,6 +50,7 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
     constexpr int VEC = E::VEC;
     constexpr int LPR = D / VEC;
     extern __shared__ float smem[];
+    const int win_t = KT ? KT : pr.kt, win_y = KT ? KH : pr.kh, win_x = KT ? KW : pr.kw, n_samples = KT ? KT * KH * KW : pr.P;
     const int lane = threadIdx.x & 31;
     const int gl = lane & (LPR - 1);
     constexpr unsigned gmask = kFullMask;
@@ -60,7 +63,7 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
     const bool want_doff = doffsets != nullptr;
     // with a table the box always has the +1 neighbours (that is how the table is laid out)
     const bool wide = want_doff || TABLE;
-    const int BT = pr.kt + (wide ? 1 : 0), BY = pr.kh + (wide ? 1 : 0), BX = pr.kw + (wide ? 1 : 0);
+    const int BT = win_t + (wide ? 1 : 0), BY = win_y + (wide ? 1 : 0), BX = win_x + (wide ? 1 : 0);
     const int NB = BT * BY * BX;
     const int NB8 = (NB + 7) & ~7;
     // per block: box_tab[NB8] = displacement of box position idx from the box origin and whether
@@ -68,23 +71,23 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
     // samp_tab[P] = box index of sample p's own position
     int4* box_tab = reinterpret_cast<int4*>(smem);
     int* samp_tab = reinterpret_cast<int*>(box_tab + NB8);
-    float* group0 = reinterpret_cast<float*>(samp_tab + ((pr.P + 3) & ~3));
+    float* group0 = reinterpret_cast<float*>(samp_tab + ((n_samples + 3) & ~3));
     for (int idx = threadIdx.x; idx < NB8; idx += blockDim.x) {
         const int bw = idx % BX, bv = (idx / BX) % BY, bu = idx / (BX * BY);
-        const int far = (bu == pr.kt) + (bv == pr.kh) + (bw == pr.kw);
+        const int far = (bu == win_t) + (bv == win_y) + (bw == win_x);
         box_tab[idx] = make_int4(bu, bv, bw, (idx < NB && far <= 1) ? 1 : 0);
     }
-    for (int p = threadIdx.x; p < pr.P; p += blockDim.x) {
-        const int w = p % pr.kw, vv = (p / pr.kw) % pr.kh, u = p / (pr.kw * pr.kh);
+    for (int p = threadIdx.x; p < n_samples; p += blockDim.x) {
+        const int w = p % win_x, vv = (p / win_x) % win_y, u = p / (win_x * win_y);
         samp_tab[p] = (u * BY + vv) * BX + w;
     }
     __syncthreads();
     if (whole_warp_idle) return;
     // per group: ta[NB8], tb[NB8] (dot products per box position), sa[P] (alpha), sk[P] (scale dS)
-    float* ta = group0 + static_cast<size_t>(threadIdx.x / LPR) * (2 * NB8 + 2 * pr.P);
+    float* ta = group0 + static_cast<size_t>(threadIdx.x / LPR) * (2 * NB8 + 2 * n_samples);
     float* tb = ta + NB8;
     float* sa = tb + NB8;
-    float* sk = sa + pr.P;
+    float* sk = sa + n_samples;
 
     const int m = static_cast<int>(item / pr.q_count);
     const long long n = pr.q_begin + (item - static_cast<long long>(m) * pr.q_count);
@@ -97,7 +100,7 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
     const long long tok_stride = static_cast<long long>(pr.heads) * D;
     const T* kh = k + static_cast<long long>(m) * D + ch;
     const long long v_minus_k = v - k;
-    const int ot = t - pr.kt / 2, oy = y - pr.kh / 2, ox = x - pr.kw / 2;      // box origin
+    const int ot = t - win_t / 2, oy = y - win_y / 2, ox = x - win_x / 2;      // box origin
 
     const float lse2 = __ldg(lse + row) * kLog2e;
 
@@ -159,7 +162,7 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
 
     // ---- softmax weights, delta
     float delta = 0.0f;
-    for (int p = gl; p < pr.P; p += LPR) {
+    for (int p = gl; p < n_samples; p += LPR) {
         const int idx = samp_tab[p];
         const float alpha = exp2f(fmaf(ta[idx], scale * kLog2e, -lse2));     // a position outside the grid: logit 0
         sa[p] = alpha;
@@ -168,16 +171,16 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
     delta = group_sum<LPR>(delta, gmask);
 
     // ---- dS, coefficients, dOffsets
-    for (int p = gl; p < pr.P; p += LPR) {
+    for (int p = gl; p < n_samples; p += LPR) {
         const int idx = samp_tab[p];
         const float alpha = sa[p];
         const float ck = scale * alpha * (tb[idx] - delta);
         sk[p] = ck;
         if (active) {
-            if (!coef_planes) coef[row * pr.P + p] = make_float2(ck, alpha);
+            if (!coef_planes) coef[row * n_samples + p] = make_float2(ck, alpha);
             if (want_doff) {
                 const float s0 = fmaf(ck, ta[idx], alpha * tb[idx]);
-                float* dst = doffsets + (row * pr.P + p) * 3;
+                float* dst = doffsets + (row * n_samples + p) * 3;
                 dst[0] = fmaf(ck, ta[idx + BY * BX], alpha * tb[idx + BY * BX]) - s0;
                 dst[1] = fmaf(ck, ta[idx + BX], alpha * tb[idx + BX]) - s0;
                 dst[2] = fmaf(ck, ta[idx + 1], alpha * tb[idx + 1]) - s0;
@@ -193,21 +196,21 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
         // the fp32 value in one word (relative error of the pair 2^-17).  The block's groups hold consecutive tokens: the block writes together, a run of
         // tokens per sample, from the groups' arrays in shared memory.
         const int groups = blockDim.x / LPR;
-        long long* group_at = reinterpret_cast<long long*>(group0 + static_cast<size_t>(groups) * (2 * NB8 + 2 * pr.P));
-        if (gl == 0) group_at[threadIdx.x / LPR] = static_cast<long long>(m) * pr.P * pr.N + n;
+        long long* group_at = reinterpret_cast<long long*>(group0 + static_cast<size_t>(groups) * (2 * NB8 + 2 * n_samples));
+        if (gl == 0) group_at[threadIdx.x / LPR] = static_cast<long long>(m) * n_samples * pr.N + n;
         __syncthreads();                                   // warps with no item at all have left: they count as arrived
         uint32_t* planes = reinterpret_cast<uint32_t*>(coef);
-        const long long plane_elems = pr.N * pr.heads * pr.P;
+        const long long plane_elems = pr.N * pr.heads * n_samples;
         const long long block_first = static_cast<long long>(blockIdx.x) * groups;     // item of group 0
         // the threads still here: the warps up to the last one that holds an item
         const long long lanes_with_items = (pr.items - block_first) * LPR;
         const int live = lanes_with_items >= blockDim.x ? static_cast<int>(blockDim.x) : static_cast<int>((lanes_with_items + 31) / 32 * 32);
-        for (int i = threadIdx.x; i < groups * pr.P; i += live) {
+        for (int i = threadIdx.x; i < groups * n_samples; i += live) {
             const int g = i % groups, p = i / groups;
             if (block_first + g >= pr.items) continue;     // a group without an item (its arrays and position are not set)
             const long long at = group_at[g];
-            const float* ga = group0 + static_cast<size_t>(g) * (2 * NB8 + 2 * pr.P) + 2 * NB8;     // sa, then sk
-            planes[at + p * pr.N] = split_bf16_pair(ga[pr.P + p]);
+            const float* ga = group0 + static_cast<size_t>(g) * (2 * NB8 + 2 * n_samples) + 2 * NB8;     // sa, then sk
+            planes[at + p * pr.N] = split_bf16_pair(ga[n_samples + p]);
             planes[plane_elems + at + p * pr.N] = split_bf16_pair(ga[p]);
         }
     }
@@ -217,14 +220,14 @@ fixed_window_backward_query_kernel(const T* __restrict__ q, const T* __restrict_
     float dqv[VEC];
 #pragma unroll
     for (int e = 0; e < VEC; ++e) dqv[e] = 0.0f;
-    for (int p0 = 0; p0 < pr.P; p0 += 8) {
+    for (int p0 = 0; p0 < n_samples; p0 += 8) {
         Row kk[8];
         float cks[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             kk[i] = E::zero();
             cks[i] = 0.0f;
-            if (p0 + i < pr.P) {
+            if (p0 + i < n_samples) {
                 const int4 bt = box_tab[samp_tab[p0 + i]];
                 const int pt = ot + bt.x, py = oy + bt.y, px = ox + bt.z;
                 if (pt >= 0 && pt < pr.T && py >= 0 && py < pr.H && px >= 0 && px < pr.W) {
@@ -303,7 +306,13 @@ cudaError_t launch_t(const void* q, const void* k, const void* v, const float* l
     int threads = 256;
     while (threads > 32 && tables + static_cast<size_t>(threads / LPR) * (per_group + sizeof(long long)) > 64 * 1024) threads /= 2;
     const size_t smem = tables + static_cast<size_t>(threads / LPR) * (per_group + sizeof(long long));   // + a position per group
-    auto qk = table ? fixed_window_backward_query_kernel<T, D, true> : fixed_window_backward_query_kernel<T, D, false>;
+    auto qk = fixed_window_backward_query_kernel<T, D, false>;
+    if (table) {
+        qk = fixed_window_backward_query_kernel<T, D, true>;
+        // measured: the compile-time window pays for (2,2,2) only (backward 5.36 -> 4.94 ms on the sweep grid); the
+        // instances for (3,3,3), (3,5,5) and (3,7,7) were 3 to 13 % slower than the generic kernel
+        if (pr.kt == 2 && pr.kh == 2 && pr.kw == 2) qk = fixed_window_backward_query_kernel<T, D, true, 2, 2, 2>;
+    }
     if (smem > 48 * 1024) {
         const cudaError_t e = cudaFuncSetAttribute(qk, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
