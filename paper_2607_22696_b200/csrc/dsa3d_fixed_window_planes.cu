@@ -31,6 +31,8 @@
 // through the rest of its tile without waiting, drains its loads and frees its TMEM.
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "dsa3d_common.cuh"
 #include "dsa3d_kernels.h"
 #include "dsa3d_tcgen05.cuh"
@@ -315,6 +317,51 @@ fixed_window_planes_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
             const uint32_t col = static_cast<uint32_t>((ly + vv) * RX + lx + ww);
             return (col >> 6) * (kPlQ * 128) + row_off + ((((col & 63) >> 3) ^ rx) << 4) + (col & 7) * 2;
         };
+        // The cells of one kernel row are KW neighbouring columns of the query's row of P: they are written as
+        // whole 16-byte chunks of 8 columns (one chunk, or two when the cells straddle a chunk boundary).  The
+        // other columns of those chunks belong to no cell of this query - the neighbouring kernel rows lie
+        // 8 + KW - 1 columns away - so writing them as zeros is right.  Per kernel row, the same for every
+        // plane and tile: bits 0-11 / 12-23 the byte offsets of the two chunks (in 16-byte units), bits 24-26
+        // the columns by which the cells are shifted inside them.
+        // Used for the box of learned offsets (forward 9.95 -> 7.42 ms on the sweep grid: its weights come from
+        // shared memory and were read once per matrix).  The fixed windows keep writing their cells one by one:
+        // (3,5,5) has its cell offsets in registers and measured 4 % slower this way, (3,7,7) has no registers
+        // left for it (84 window scores per thread; a block of this size gets 168 registers per thread).
+        constexpr bool kChunkStores = BOUNDED && VH <= 3;
+        static_assert(!kChunkStores || (S::P_BYTES <= 65536 && KW <= 7 && RX >= KW + 7),
+                      "chunk offsets in 12 bits; a kernel row's chunks touch no other row's cells");
+        uint32_t row_geo[VH];
+#pragma unroll
+        for (int vi = 0; vi < VH; ++vi) {
+            const int vv = vi + half * VH < KH ? vi + half * VH : 0;
+            const uint32_t col0 = static_cast<uint32_t>((ly + vv) * RX + lx);
+            auto chunk_off = [&](uint32_t col) { return (col >> 6) * (kPlQ * 128) + row_off + ((((col & 63) >> 3) ^ rx) << 4); };
+            row_geo[vi] = (chunk_off(col0) >> 4) | ((chunk_off(col0 + 8) >> 4) << 12) | ((col0 & 7u) << 24);
+        }
+        // KW cells (a word each: bf16 head | bf16 remainder << 16) moved to their places among the 16 columns of
+        // the row's two chunks by one network of selects, then parted into the words of the head matrix and of
+        // the remainder matrix (two columns per word)
+        auto align_row = [&](uint32_t geo, const uint32_t (&cell)[8], uint32_t (&head)[8], uint32_t (&rest)[8]) {
+            const bool s1 = (geo >> 24) & 1u, s2 = (geo >> 25) & 1u, s4 = (geo >> 26) & 1u;
+            uint32_t a[8], b[10], c[14];
+            a[0] = s1 ? 0u : cell[0];
+#pragma unroll
+            for (int i = 1; i < 8; ++i) a[i] = s1 ? cell[i - 1] : cell[i];              // cell[7] is always 0 (KW <= 7)
+#pragma unroll
+            for (int i = 0; i < 10; ++i) b[i] = s2 ? (i >= 2 ? a[i - 2] : 0u) : (i < 8 ? a[i] : 0u);
+#pragma unroll
+            for (int i = 0; i < 14; ++i) c[i] = s4 ? (i >= 4 ? b[i - 4] : 0u) : (i < 10 ? b[i] : 0u);
+#pragma unroll
+            for (int j = 0; j < 7; ++j) {
+                head[j] = __byte_perm(c[2 * j], c[2 * j + 1], 0x5410);
+                rest[j] = __byte_perm(c[2 * j], c[2 * j + 1], 0x7632);
+            }
+            head[7] = rest[7] = 0u;
+        };
+        auto store_chunks = [&](unsigned char* dst, uint32_t geo, const uint32_t (&w)[8]) {
+            *reinterpret_cast<uint4*>(dst + ((geo & 0xfffu) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+            if (((geo >> 24) & 7u) + KW > 8u) *reinterpret_cast<uint4*>(dst + (((geo >> 12) & 0xfffu) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+        };
         if constexpr (kCacheCells) {
 #pragma unroll
             for (int vi = 0; vi < VH; ++vi)
@@ -534,36 +581,108 @@ fixed_window_planes_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                         *reinterpret_cast<uint4*>(dst + (c >> 3) * (kPlQ * 128) + (((c & 7) ^ rx) << 4)) = make_uint4(0u, 0u, 0u, 0u);
                     named_barrier_sync(1 + lt, 64);                   // both matrices of the row are clear before cells land
                 }
+                if constexpr (kChunkStores) {
+                    // The words of kernel row vi of this plane for the head and the remainder matrix.  With few rows per
+                    // thread the remainder words wait in registers while the head matrix goes out; with four rows
+                    // (the (3,7,7) window: 84 window scores live in registers already) they are formed again.
+                    constexpr bool kKeepRest = VH <= 3;
+                    auto row_words = [&](auto vi_c, uint32_t (&head)[8], uint32_t (&rest)[8]) {
+                        constexpr int vi = decltype(vi_c)::value;         // a constant, so that sc[][vi][] stays in registers
+                        const int vv = vi + half * VH;
+                        uint32_t cell[8];
 #pragma unroll
-                for (int part = 0; part < 2; ++part) {
-                    if (pl > 0) wait(&s.bar_p_free[part], static_cast<uint32_t>((pvc - 1) & 1), 22);   // the chain of the plane before
-                    if (mine || u_rt == KT) {
-                        unsigned char* dst = part ? p_rest : p_head;
+                        for (int ww = 0; ww < 8; ++ww) cell[ww] = 0u;
 #pragma unroll
-                        for (int u = 0; u <= KT; ++u) {
+                        for (int u = 0; u < KT; ++u) {
                             if (u != u_rt) continue;
 #pragma unroll
-                            for (int vi = 0; vi < VH; ++vi) {
-                                const int vv = vi + half * VH;
-                                if (vv >= KH) continue;
+                            for (int ww = 0; ww < KW; ++ww) {
+                                float p;
+                                if constexpr (BOUNDED) p = s.box[((u * KH + vv) * KW + ww) * kPlQ + r];
+                                else p = sc[u][vi][ww] * inv;
+                                const __nv_bfloat16 hd = __float2bfloat16_rn(p);
+                                const __nv_bfloat16 rm = __float2bfloat16_rn(p - __bfloat162float(hd));
+                                cell[ww] = static_cast<uint32_t>(__bfloat16_as_ushort(hd)) | (static_cast<uint32_t>(__bfloat16_as_ushort(rm)) << 16);
+                            }
+                        }
+                        align_row(row_geo[vi], cell, head, rest);
+                    };
+                    uint32_t kept[kKeepRest ? VH : 1][8];
+                    const bool writes = mine || u_rt == KT;               // u_rt == KT: the cells go back to zero
+                    if (pl > 0) wait(&s.bar_p_free[0], static_cast<uint32_t>((pvc - 1) & 1), 22);   // the head chain of the plane before
+                    // f(constant) for every kernel row of this thread
+                    auto for_rows = [&](auto&& f) {
+                        f(std::integral_constant<int, 0>{});
+                        if constexpr (VH > 1) f(std::integral_constant<int, 1>{});
+                        if constexpr (VH > 2) f(std::integral_constant<int, 2>{});
+                        if constexpr (VH > 3) f(std::integral_constant<int, 3>{});
+                        static_assert(VH <= 4, "kernel rows per thread");
+                    };
+                    if (writes) {
+                        for_rows([&](auto vi_c) {
+                            constexpr int vi = decltype(vi_c)::value;
+                            if (vi + half * VH >= KH) return;
+                            uint32_t head[8], rest[8];
+                            row_words(vi_c, head, rest);
+                            store_chunks(p_head, row_geo[vi], head);
+                            if constexpr (kKeepRest) {
 #pragma unroll
-                                for (int ww = 0; ww < KW; ++ww) {
-                                    float p = 0.0f;
-                                    if constexpr (BOUNDED) {
-                                        if (u < KT) p = s.box[(((u < KT ? u : 0) * KH + vv) * KW + ww) * kPlQ + r];
-                                    } else {
-                                        if (u < KT) p = sc[u < KT ? u : 0][vi][ww] * inv;
+                                for (int j = 0; j < 8; ++j) kept[vi][j] = rest[j];
+                            }
+                        });
+                    }
+                    fence_async_smem();                                   // the MMAs read P through the async proxy
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&s.bar_p_full[0]));
+                    if (pl > 0) wait(&s.bar_p_free[1], static_cast<uint32_t>((pvc - 1) & 1), 22);   // the remainder chain of the plane before
+                    if (writes) {
+                        for_rows([&](auto vi_c) {
+                            constexpr int vi = decltype(vi_c)::value;
+                            if (vi + half * VH >= KH) return;
+                            if constexpr (kKeepRest) {
+                                store_chunks(p_rest, row_geo[vi], kept[vi]);
+                            } else {
+                                uint32_t head[8], rest[8];
+                                row_words(vi_c, head, rest);
+                                store_chunks(p_rest, row_geo[vi], rest);
+                            }
+                        });
+                    }
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&s.bar_p_full[1]));
+                } else {
+#pragma unroll
+                    for (int part = 0; part < 2; ++part) {
+                        if (pl > 0) wait(&s.bar_p_free[part], static_cast<uint32_t>((pvc - 1) & 1), 22);   // the chain of the plane before
+                        if (mine || u_rt == KT) {
+                            unsigned char* dst = part ? p_rest : p_head;
+#pragma unroll
+                            for (int u = 0; u <= KT; ++u) {
+                                if (u != u_rt) continue;
+#pragma unroll
+                                for (int vi = 0; vi < VH; ++vi) {
+                                    const int vv = vi + half * VH;
+                                    if (vv >= KH) continue;
+#pragma unroll
+                                    for (int ww = 0; ww < KW; ++ww) {
+                                        float p = 0.0f;
+                                        if constexpr (BOUNDED) {
+                                            if (u < KT) p = s.box[(((u < KT ? u : 0) * KH + vv) * KW + ww) * kPlQ + r];
+                                        } else {
+                                            if (u < KT) p = sc[u < KT ? u : 0][vi][ww] * inv;
+                                        }
+                                        __nv_bfloat16 val = __float2bfloat16_rn(p);
+                                        if (part) val = __float2bfloat16_rn(p - __bfloat162float(val));
+                                        *reinterpret_cast<__nv_bfloat16*>(dst + (kCacheCells ? cell_p[kCacheCells ? vi : 0][kCacheCells ? ww : 0] : p_offset(vv, ww))) = val;
                                     }
-                                    __nv_bfloat16 val = __float2bfloat16_rn(p);
-                                    if (part) val = __float2bfloat16_rn(p - __bfloat162float(val));
-                                    *reinterpret_cast<__nv_bfloat16*>(dst + (kCacheCells ? cell_p[kCacheCells ? vi : 0][kCacheCells ? ww : 0] : p_offset(vv, ww))) = val;
                                 }
                             }
                         }
+                        fence_async_smem();                               // the MMAs read P through the async proxy
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&s.bar_p_full[part]));
                     }
-                    fence_async_smem();                               // the MMAs read P through the async proxy
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&s.bar_p_full[part]));
                 }
             }
 
