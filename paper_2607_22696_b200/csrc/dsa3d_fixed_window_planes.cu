@@ -421,18 +421,29 @@ fixed_window_planes_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                         for (int i = 0; i < 32; ++i) stage[(piece * 32 + i) * kPlQ + r] = __uint_as_float(regs[i]);
                     }
                     named_barrier_sync(1 + lt, 64);                   // the two warps of this quadrant: plane staged
-#pragma unroll
-                    for (int u = 0; u < KT; ++u) {
-                        if (u != u_rt) continue;
+                    if constexpr (BOUNDED) {
+                        // the box lives in shared memory: the plane's index may stay a run-time value (one copy of
+                        // the code instead of one per kernel plane)
 #pragma unroll
                         for (int vi = 0; vi < VH; ++vi) {
                             const int vv = vi + half * VH;
                             if (vv >= KH) continue;
 #pragma unroll
-                            for (int ww = 0; ww < KW; ++ww) {
-                                const float sv = stage[kCacheCells ? cell_stage[kCacheCells ? vi : 0][kCacheCells ? ww : 0] : stage_index(vv, ww)] * lscale;
-                                if constexpr (BOUNDED) s.box[((u * KH + vv) * KW + ww) * kPlQ + r] = sv;
-                                else sc[u][vi][ww] = sv;
+                            for (int ww = 0; ww < KW; ++ww)
+                                s.box[((u_rt * KH + vv) * KW + ww) * kPlQ + r] =
+                                    stage[kCacheCells ? cell_stage[kCacheCells ? vi : 0][kCacheCells ? ww : 0] : stage_index(vv, ww)] * lscale;
+                        }
+                    } else {
+#pragma unroll
+                        for (int u = 0; u < KT; ++u) {
+                            if (u != u_rt) continue;                  // static register indices for sc
+#pragma unroll
+                            for (int vi = 0; vi < VH; ++vi) {
+                                const int vv = vi + half * VH;
+                                if (vv >= KH) continue;
+#pragma unroll
+                                for (int ww = 0; ww < KW; ++ww)
+                                    sc[u][vi][ww] = stage[kCacheCells ? cell_stage[kCacheCells ? vi : 0][kCacheCells ? ww : 0] : stage_index(vv, ww)] * lscale;
                             }
                         }
                     }
@@ -592,17 +603,22 @@ fixed_window_planes_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                         uint32_t cell[8];
 #pragma unroll
                         for (int ww = 0; ww < 8; ++ww) cell[ww] = 0u;
+                        auto split = [](float p) {
+                            const __nv_bfloat16 hd = __float2bfloat16_rn(p);
+                            const __nv_bfloat16 rm = __float2bfloat16_rn(p - __bfloat162float(hd));
+                            return static_cast<uint32_t>(__bfloat16_as_ushort(hd)) | (static_cast<uint32_t>(__bfloat16_as_ushort(rm)) << 16);
+                        };
+                        if constexpr (BOUNDED) {
+                            if (u_rt < KT) {
 #pragma unroll
-                        for (int u = 0; u < KT; ++u) {
-                            if (u != u_rt) continue;
+                                for (int ww = 0; ww < KW; ++ww) cell[ww] = split(s.box[((u_rt * KH + vv) * KW + ww) * kPlQ + r]);
+                            }
+                        } else {
 #pragma unroll
-                            for (int ww = 0; ww < KW; ++ww) {
-                                float p;
-                                if constexpr (BOUNDED) p = s.box[((u * KH + vv) * KW + ww) * kPlQ + r];
-                                else p = sc[u][vi][ww] * inv;
-                                const __nv_bfloat16 hd = __float2bfloat16_rn(p);
-                                const __nv_bfloat16 rm = __float2bfloat16_rn(p - __bfloat162float(hd));
-                                cell[ww] = static_cast<uint32_t>(__bfloat16_as_ushort(hd)) | (static_cast<uint32_t>(__bfloat16_as_ushort(rm)) << 16);
+                            for (int u = 0; u < KT; ++u) {
+                                if (u != u_rt) continue;
+#pragma unroll
+                                for (int ww = 0; ww < KW; ++ww) cell[ww] = split(sc[u][vi][ww] * inv);
                             }
                         }
                         align_row(row_geo[vi], cell, head, rest);
