@@ -268,11 +268,24 @@ int dsa3d_backward_bounded_offsets(const void* q, const void* k, const void* v, 
     e = dsa3d::launch_offsets_bound_check(offsets, pr.items * pr.P * 3, gate, st);
     if (e != cudaSuccess) return cuda_failed(e);
     // the three tile kernels run if the check left 0 in the gate, the general kernels behind them if it left 1
+    // profile events: the whole backward (either route) lies between the backward's start and stop events; the
+    // gated general kernels behind the tile kernels do not move them
+    e = record(2, st);
+    if (e != cudaSuccess) return cuda_failed(e);
     const bool tiled = dsa3d::try_bounded_offsets_backward(q, k, v, offsets, lse, dout, dq, dk, dv, doffsets, workspace, gate,
                                                           pr, st, &e);
     if (tiled && e != cudaSuccess) return cuda_failed(e);
-    return dsa3d::backward_impl(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets, workspace,
-                                workspace_bytes, dtype, stream, true, tiled ? gate : nullptr);
+    if (!tiled)
+        return dsa3d::backward_impl(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets, workspace,
+                                    workspace_bytes, dtype, stream, true);
+    cudaEvent_t held[6];
+    for (int i = 0; i < 6; ++i) { held[i] = g_events[i]; g_events[i] = nullptr; }
+    const int rc2 = dsa3d::backward_impl(q, k, v, offsets, lse, dout, T, H, W, heads, d, window, dq, dk, dv, doffsets, workspace,
+                                         workspace_bytes, dtype, stream, true, gate);
+    for (int i = 0; i < 6; ++i) g_events[i] = held[i];
+    if (rc2 != DSA3D_OK) return rc2;
+    e = record(3, st);
+    return e == cudaSuccess ? DSA3D_OK : cuda_failed(e);
 }
 
 size_t dsa3d_backward_fixed_window_workspace_bytes(int T, int H, int W, int heads, int d, const int window[3],
