@@ -199,3 +199,46 @@ def test_backward_other_shapes_take_the_general_kernels(shape, window, dtype):
     P = window[0] * window[1] * window[2]
     off = _bounded_offsets((T, H, W, heads, P, 3), 770, "uniform")
     _run_backward(shape, window, dtype, 177, off)
+
+
+def test_two_calls_in_flight_on_two_streams_do_not_share_a_gate():
+    """One call whose offsets pass the check and one whose offsets do not, queued on two streams before either
+    has run: each takes its own gate word, so each must equal the same call made alone."""
+    shape, window = (8, 12, 24, 2, 128), (3, 3, 3)
+    T, H, W, heads, d = shape
+    off_ok = _bounded_offsets((T, H, W, heads, 27, 3), 780, "uniform")
+    off_big = off_ok.clone()
+    off_big.view(-1)[7::101] = 2.5
+    q, k, v, dout = (inputs.normal(shape, 178, i, 1.0, BF16).cuda() for i in range(4))
+    nbytes = binding.dsa3d_backward_bounded_offsets_workspace_bytes(T, H, W, heads, d, window, BF16)
+
+    def run(off, stream):
+        out = torch.empty(shape, dtype=BF16, device="cuda")
+        lse = torch.empty((T, H, W, heads), dtype=F32, device="cuda")
+        g = [torch.empty(shape, dtype=BF16, device="cuda") for _ in range(3)]
+        doff = torch.empty((T, H, W, heads, 27, 3), dtype=F32, device="cuda")
+        ws = torch.empty((nbytes,), dtype=torch.uint8, device="cuda")
+        with torch.cuda.stream(stream):
+            binding.dsa3d_forward_bounded_offsets(q, k, v, off, T, H, W, heads, d, window, out, lse, stream=stream)
+            binding.dsa3d_backward_bounded_offsets(q, k, v, off, lse, dout, T, H, W, heads, d, window, g[0], g[1], g[2], doff, ws,
+                                                   stream=stream)
+        return out, lse, g, doff, ws
+
+    offs = [off_ok.cuda(), off_big.cuda()]
+    torch.cuda.synchronize()
+    alone = []
+    for off in offs:
+        alone.append(run(off, torch.cuda.current_stream()))
+        torch.cuda.synchronize()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    together = [run(offs[0], s1), run(offs[1], s2)]
+    torch.cuda.synchronize()
+    assert binding.dsa3d_device_timeout_flag() == 0
+    for a, b in zip(alone, together):
+        assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])               # out, lse
+        assert torch.equal(a[2][0], b[2][0]) and torch.equal(a[3], b[3])         # dq, doffsets
+    # the tile route writes dk and dv without atomics: bit for bit; the general route up to the order of its sums
+    for i in (1, 2):
+        assert torch.equal(alone[0][2][i], together[0][2][i])
+        fa, fb = alone[1][2][i].float(), together[1][2][i].float()
+        assert bool(((fa - fb).abs() <= (fb.abs() * 2.0 ** -7).clamp_min(2e-3)).all())
